@@ -1,0 +1,6 @@
+"""CPU fp64 oracle of the DART token-reduction step: test infrastructure only.
+
+Nothing in the product package may import this; see ``dart_oracle.c`` for the arithmetic.
+"""
+from .dart_oracle import (OracleResult, build, compact, pivots, reduce, retention, scores,  # noqa: F401
+                          similarity)

@@ -1,0 +1,323 @@
+/*
+ * DART token-reduction oracle: TEST INFRASTRUCTURE, not the product.
+ *
+ * A plain, slow, single-threaded fp64 restatement of the duplication-aware
+ * token-reduction step of DART (arxiv 2502.11494), written from the paper's
+ * definitions.  It exists so that the CUDA library can be checked against
+ * something that can be compared with the paper by eye.  It shares no code,
+ * header, table or helper with the CUDA path.  Only the tests, the smoke
+ * check and the CPU-baseline leg of the benchmark may call it.
+ *
+ * Inputs are bf16 bit patterns (uint16_t) that are widened exactly to fp64;
+ * every sum is a plain left-to-right fp64 accumulation; every ordering is a
+ * full sort with an explicit total order (value, then token index).
+ *
+ * Steps (one sample; the batch entry point loops over samples):
+ *   scores      Sec. 3.3, footnote on "K-norm": L1 norm of each token's row
+ *               of the key matrix; the Euclidean norm needed by Eq. 7.
+ *   pivots      Def. 1 + Table 1 caption: the k tokens of maximum K-norm.
+ *   similarity  Def. 2, Eq. 7: dup(p_i, x_j) = p_i.x_j / (|p_i| |x_j|).
+ *   retention   Eq. 9-10 with a per-pivot threshold set by the budget:
+ *               pivot i (rank order) retains its q_i not-yet-retained,
+ *               non-pivot tokens of LOWEST dup; eps_i = largest retained dup;
+ *               R = P u U_i R_i, |R| = n_keep exactly.
+ *   compaction  the retained tokens stay in original order; text tokens
+ *               are all kept; hidden rows and position ids are gathered.
+ *
+ * Readings of points the paper leaves open (ties -> lower index; the r
+ * highest-ranked pivots take one extra token when (n_keep - P) % P = r;
+ * a zero-norm row has dup 0) are the library's documented readings; the
+ * functions whose behaviour rests on such a reading say so below.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_OK 0
+#define ORACLE_ERR_SHAPE (-2)
+#define ORACLE_ERR_NOMEM (-6)
+
+/* owner[] codes */
+#define OWNER_DROPPED (-1)
+
+static double bf16_to_f64(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16; /* bf16 is the top half of an IEEE binary32 */
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+typedef struct {
+    double v;
+    int32_t idx;
+} keyed_t;
+
+/* descending value, ascending index */
+static int cmp_desc(const void *a, const void *b)
+{
+    const keyed_t *x = (const keyed_t *)a, *y = (const keyed_t *)b;
+    if (x->v > y->v) return -1;
+    if (x->v < y->v) return 1;
+    return (x->idx > y->idx) - (x->idx < y->idx);
+}
+
+/* ascending value, ascending index */
+static int cmp_asc(const void *a, const void *b)
+{
+    const keyed_t *x = (const keyed_t *)a, *y = (const keyed_t *)b;
+    if (x->v < y->v) return -1;
+    if (x->v > y->v) return 1;
+    return (x->idx > y->idx) - (x->idx < y->idx);
+}
+
+/*
+ * Scores of the vision tokens of one sample (Sec. 3.3 footnote: K-norm is the
+ * L1 norm of the K matrix, taken per token row; Eq. 7 needs the Euclidean norm).
+ *   keys   [S, d] bf16 bits, row-major; vision rows are [vis_offset, vis_offset+n_vis)
+ *   l1     [n_vis]  sum_c |K[j,c]|
+ *   l2     [n_vis]  sqrt(sum_c K[j,c]^2)
+ */
+int dart_oracle_scores(const uint16_t *keys, int S, int d, int vis_offset, int n_vis,
+                       double *l1, double *l2)
+{
+    if (S < 1 || d < 1 || vis_offset < 0 || n_vis < 0 || vis_offset + n_vis > S) return ORACLE_ERR_SHAPE;
+    for (int j = 0; j < n_vis; ++j) {
+        const uint16_t *row = keys + (size_t)(vis_offset + j) * (size_t)d;
+        double a = 0.0, q = 0.0;
+        for (int c = 0; c < d; ++c) {
+            double x = bf16_to_f64(row[c]);
+            a += fabs(x);
+            q += x * x;
+        }
+        l1[j] = a;
+        l2[j] = sqrt(q);
+    }
+    return ORACLE_OK;
+}
+
+/*
+ * Pivot tokens (Def. 1; Table 1 caption: chosen by maximum K-norm).
+ * The P tokens of largest score, in rank order (rank 0 = largest).
+ * largest != 0 : maximum-score pivots (the paper's main setting);
+ * largest == 0 : minimum-score pivots (the ablation's "smallest value" variant).
+ * Equal scores: the lower token index ranks first (reading; the paper is silent).
+ *   gap_out (may be NULL): min over ranks t = 0..P-1 of the relative gap
+ *   |s_(t) - s_(t+1)| / |s_(t)| between consecutive tokens in the ranking
+ *   (up to and including the gap to the first non-pivot); +inf when P = n_vis
+ *   has no successor for the last rank.
+ */
+int dart_oracle_pivots(const double *score, int n_vis, int P, int largest,
+                       int32_t *pivot_idx, double *gap_out)
+{
+    if (P < 1 || P > n_vis) return ORACLE_ERR_SHAPE;
+    keyed_t *k = (keyed_t *)malloc((size_t)n_vis * sizeof *k);
+    if (!k) return ORACLE_ERR_NOMEM;
+    for (int j = 0; j < n_vis; ++j) {
+        k[j].v = score[j];
+        k[j].idx = j;
+    }
+    qsort(k, (size_t)n_vis, sizeof *k, largest ? cmp_desc : cmp_asc);
+    for (int i = 0; i < P; ++i) pivot_idx[i] = k[i].idx;
+    if (gap_out) {
+        double g = INFINITY;
+        for (int t = 0; t < P && t + 1 < n_vis; ++t) {
+            double den = fabs(k[t].v);
+            double rel = den > 0.0 ? fabs(k[t].v - k[t + 1].v) / den : 0.0;
+            if (rel < g) g = rel;
+        }
+        *gap_out = g;
+    }
+    free(k);
+    return ORACLE_OK;
+}
+
+/*
+ * Duplication scores (Def. 2, Eq. 7): cosine of pivot i and vision token j,
+ * dup[i*n_vis + j] = (K_{p_i} . K_j) / (|K_{p_i}| |K_j|).
+ * A zero-norm operand gives dup = 0 (reading; Eq. 7 is undefined there).
+ */
+int dart_oracle_similarity(const uint16_t *keys, int S, int d, int vis_offset, int n_vis,
+                           const int32_t *pivot_idx, int P, const double *l2, double *dup)
+{
+    if (S < 1 || d < 1 || vis_offset < 0 || n_vis < 0 || vis_offset + n_vis > S || P < 1) return ORACLE_ERR_SHAPE;
+    for (int i = 0; i < P; ++i) {
+        int p = pivot_idx[i];
+        if (p < 0 || p >= n_vis) return ORACLE_ERR_SHAPE;
+        const uint16_t *prow = keys + (size_t)(vis_offset + p) * (size_t)d;
+        for (int j = 0; j < n_vis; ++j) {
+            const uint16_t *xrow = keys + (size_t)(vis_offset + j) * (size_t)d;
+            double dot = 0.0;
+            for (int c = 0; c < d; ++c) dot += bf16_to_f64(prow[c]) * bf16_to_f64(xrow[c]);
+            double den = l2[p] * l2[j];
+            dup[(size_t)i * (size_t)n_vis + j] = den > 0.0 ? dot / den : 0.0;
+        }
+    }
+    return ORACLE_OK;
+}
+
+/*
+ * Retention under the budget (Eq. 9-10; Sec. 1: "retain the vision tokens with the
+ * lowest cosine similarity to the pivots"; eps is set per pivot from the ratio).
+ *
+ *   kept := { p_0 .. p_{P-1} }                         (P subset of R, Eq. 10)
+ *   q = (n_keep - P) / P, r = (n_keep - P) % P; q_i = q + 1 for rank i < r, else q
+ *   for i = 0 .. P-1 (rank order):
+ *       candidates := vision tokens not in kept
+ *       order them by (dup[i][j] ascending, j ascending)
+ *       R_i := the first q_i;  kept := kept u R_i;  eps_i := max dup over R_i  (Eq. 9)
+ *
+ * Outputs (any may be NULL except keep):
+ *   keep   [n_vis] 1 = retained
+ *   owner  [n_vis] -1 dropped, i in [0,P) = retained by pivot i, P + i = is pivot of rank i
+ *   eps    [P]     eps_i, NaN when q_i = 0
+ *   gap    scalar  min over pivots with q_i > 0 of (dup of the best candidate NOT taken) - eps_i,
+ *                  +inf if no pivot leaves a candidate behind
+ * The equal split of the budget, the order of the pivots' turns and the exclusion of already
+ * retained tokens are readings of the sentence that eps follows from the reduction ratio.
+ */
+int dart_oracle_retention(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep,
+                          uint8_t *keep, int32_t *owner, double *eps, double *gap_out)
+{
+    if (P < 1 || P > n_keep || n_keep > n_vis) return ORACLE_ERR_SHAPE;
+    keyed_t *cand = (keyed_t *)malloc((size_t)n_vis * sizeof *cand);
+    if (!cand) return ORACLE_ERR_NOMEM;
+    memset(keep, 0, (size_t)n_vis);
+    if (owner)
+        for (int j = 0; j < n_vis; ++j) owner[j] = OWNER_DROPPED;
+    for (int i = 0; i < P; ++i) {
+        int p = pivot_idx[i];
+        if (p < 0 || p >= n_vis || keep[p]) {
+            free(cand);
+            return ORACLE_ERR_SHAPE; /* pivots must be distinct vision tokens */
+        }
+        keep[p] = 1;
+        if (owner) owner[p] = P + i;
+    }
+    const int q = (n_keep - P) / P, r = (n_keep - P) % P;
+    double gap = INFINITY;
+    for (int i = 0; i < P; ++i) {
+        const int qi = q + (i < r ? 1 : 0);
+        if (eps) eps[i] = NAN;
+        if (qi == 0) continue;
+        int m = 0;
+        for (int j = 0; j < n_vis; ++j)
+            if (!keep[j]) {
+                cand[m].v = dup[(size_t)i * (size_t)n_vis + j];
+                cand[m].idx = j;
+                ++m;
+            }
+        /* m >= qi always: n_vis - (tokens kept so far) >= n_vis - n_keep + qi */
+        qsort(cand, (size_t)m, sizeof *cand, cmp_asc);
+        for (int t = 0; t < qi; ++t) {
+            keep[cand[t].idx] = 1;
+            if (owner) owner[cand[t].idx] = i;
+        }
+        if (eps) eps[i] = cand[qi - 1].v;
+        if (m > qi) {
+            double g = cand[qi].v - cand[qi - 1].v;
+            if (g < gap) gap = g;
+        }
+    }
+    if (gap_out) *gap_out = gap;
+    free(cand);
+    return ORACLE_OK;
+}
+
+/*
+ * Sequence shortening (Table 1 caption: tokens are pruned after layer K; the remaining
+ * layers see a dense, shorter sequence).  Kept rows stay in original order:
+ *   out_idx    = [0, vis_offset) ++ sorted{vis_offset + j : keep[j]} ++ [vis_offset + n_vis, S)
+ *   out_pos[t] = pos_in[out_idx[t]]   (pos_in NULL means pos_in[s] = s)
+ *   out_hidden[t, :] = hidden[out_idx[t], :]   (bit copy of the bf16 row)
+ * Returns the packed length S_out through *S_out_p.
+ */
+int dart_oracle_compact(const uint8_t *keep, const uint16_t *hidden, const int64_t *pos_in,
+                        int S, int d, int vis_offset, int n_vis,
+                        uint16_t *out_hidden, int32_t *out_idx, int64_t *out_pos, int *S_out_p)
+{
+    if (S < 1 || d < 1 || vis_offset < 0 || n_vis < 0 || vis_offset + n_vis > S) return ORACLE_ERR_SHAPE;
+    int t = 0;
+    for (int s = 0; s < S; ++s) {
+        int is_vis = (s >= vis_offset && s < vis_offset + n_vis);
+        if (is_vis && !keep[s - vis_offset]) continue;
+        out_idx[t] = s;
+        out_pos[t] = pos_in ? pos_in[s] : (int64_t)s;
+        if (out_hidden && hidden)
+            memcpy(out_hidden + (size_t)t * (size_t)d, hidden + (size_t)s * (size_t)d, (size_t)d * sizeof(uint16_t));
+        ++t;
+    }
+    if (S_out_p) *S_out_p = t;
+    return ORACLE_OK;
+}
+
+/*
+ * The whole step over a batch of independent samples (the paper's step has no
+ * cross-sample term).  hidden/keys are [B, S, d] bf16 bits in host memory; keys == NULL
+ * means the hidden states are scored and compared.  pos_in is [B, S] or NULL.
+ * norm_kind: 1 = L1 score (the paper's K-norm), 2 = Euclidean score.
+ * Per-sample debug outputs (each may be NULL):
+ *   l1, l2 [B, n_vis]; pivot_idx [B, P]; dup [B, P, n_vis]; keep [B, n_vis];
+ *   owner [B, n_vis]; eps [B, P]; pivot_gap [B]; retain_gap [B].
+ * Packed outputs: out_hidden [B, S_out, d], out_idx [B, S_out], out_pos [B, S_out],
+ * S_out = S - n_vis + n_keep.
+ */
+int dart_oracle_reduce(const uint16_t *hidden, const uint16_t *keys, const int64_t *pos_in,
+                       int B, int S, int d, int vis_offset, int n_vis, int n_pivot, int n_keep,
+                       int norm_kind, int largest,
+                       uint16_t *out_hidden, int32_t *out_idx, int64_t *out_pos,
+                       double *l1_out, double *l2_out, int32_t *pivot_out, double *dup_out,
+                       uint8_t *keep_out, int32_t *owner_out, double *eps_out,
+                       double *pivot_gap_out, double *retain_gap_out)
+{
+    if (B < 0 || S < 1 || d < 1 || vis_offset < 0 || n_vis < 1 || vis_offset + n_vis > S) return ORACLE_ERR_SHAPE;
+    if (n_pivot < 1 || n_pivot > n_keep || n_keep > n_vis) return ORACLE_ERR_SHAPE;
+    if (norm_kind != 1 && norm_kind != 2) return ORACLE_ERR_SHAPE;
+    const int P = n_pivot, S_out = S - n_vis + n_keep;
+    double *l1 = (double *)malloc((size_t)n_vis * sizeof(double));
+    double *l2 = (double *)malloc((size_t)n_vis * sizeof(double));
+    double *dup = (double *)malloc((size_t)P * (size_t)n_vis * sizeof(double));
+    int32_t *piv = (int32_t *)malloc((size_t)P * sizeof(int32_t));
+    uint8_t *keep = (uint8_t *)malloc((size_t)n_vis);
+    int rc = ORACLE_OK;
+    if (!l1 || !l2 || !dup || !piv || !keep) rc = ORACLE_ERR_NOMEM;
+    for (int b = 0; b < B && rc == ORACLE_OK; ++b) {
+        const uint16_t *h = hidden + (size_t)b * (size_t)S * (size_t)d;
+        const uint16_t *k = keys ? keys + (size_t)b * (size_t)S * (size_t)d : h;
+        const int64_t *pos = pos_in ? pos_in + (size_t)b * (size_t)S : NULL;
+        double pgap = 0.0, rgap = 0.0;
+        int so = 0;
+        rc = dart_oracle_scores(k, S, d, vis_offset, n_vis, l1, l2);
+        if (rc) break;
+        rc = dart_oracle_pivots(norm_kind == 1 ? l1 : l2, n_vis, P, largest, piv, &pgap);
+        if (rc) break;
+        rc = dart_oracle_similarity(k, S, d, vis_offset, n_vis, piv, P, l2, dup);
+        if (rc) break;
+        rc = dart_oracle_retention(dup, piv, n_vis, P, n_keep, keep,
+                                   owner_out ? owner_out + (size_t)b * n_vis : NULL,
+                                   eps_out ? eps_out + (size_t)b * P : NULL, &rgap);
+        if (rc) break;
+        rc = dart_oracle_compact(keep, h, pos, S, d, vis_offset, n_vis,
+                                 out_hidden ? out_hidden + (size_t)b * (size_t)S_out * (size_t)d : NULL,
+                                 out_idx + (size_t)b * S_out, out_pos + (size_t)b * S_out, &so);
+        if (rc) break;
+        if (so != S_out) {
+            rc = ORACLE_ERR_SHAPE;
+            break;
+        }
+        if (l1_out) memcpy(l1_out + (size_t)b * n_vis, l1, (size_t)n_vis * sizeof(double));
+        if (l2_out) memcpy(l2_out + (size_t)b * n_vis, l2, (size_t)n_vis * sizeof(double));
+        if (pivot_out) memcpy(pivot_out + (size_t)b * P, piv, (size_t)P * sizeof(int32_t));
+        if (dup_out) memcpy(dup_out + (size_t)b * P * n_vis, dup, (size_t)P * (size_t)n_vis * sizeof(double));
+        if (keep_out) memcpy(keep_out + (size_t)b * n_vis, keep, (size_t)n_vis);
+        if (pivot_gap_out) pivot_gap_out[b] = pgap;
+        if (retain_gap_out) retain_gap_out[b] = rgap;
+    }
+    free(l1);
+    free(l2);
+    free(dup);
+    free(piv);
+    free(keep);
+    return rc;
+}
