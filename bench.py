@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""Throughput of the DART reduction step on synthetic LLaVA-NeXT-shaped batches.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload sweep_b256] [--pivots 8] [--keep 320] [--sweep]
+
+One "step" is one pass of the whole reduction (scores, pivots, similarities, retention, packed
+gather) over one batch.  Prints ONE JSON line on rank 0.  For N > 1 launch with torch.distributed.run:
+every rank reduces its own batch (samples are independent; there is no collective on the data
+path), the timed region is bracketed by a barrier and a device synchronise, and the time is the
+maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "vision_tokens_reduced_per_sec"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="sweep_b256")
+    ap.add_argument("--pivots", type=int, default=None)
+    ap.add_argument("--keep", type=int, default=None)
+    ap.add_argument("--batch", type=int, default=None, help="override the workload's batch size")
+    ap.add_argument("--sweep", action="store_true", help="also time every (pivots, keep) cell of the sweep")
+    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 staged, 2 fused")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def pick_workload(args):
+    from paper_2502_11494_b200 import workloads as W
+
+    w = {c.name: c for c in W.CONFIGS}[args.workload]
+    kw = {}
+    if args.pivots:
+        kw["n_pivot"] = args.pivots
+    if args.keep:
+        kw["n_keep"] = args.keep
+    if args.batch:
+        kw["B"] = args.batch
+    return w.with_(**kw) if kw else w
+
+
+def path_bytes_per_sample(w):
+    """Algorithmic bytes of the whole step for one sample: the vision rows of the keys once, the kept
+    hidden rows read and written, the packed indices and position ids."""
+    return 2 * w.d * w.n_vis + 2 * (2 * w.d * w.S_out) + 12 * w.S_out
+
+
+def kernel_bytes_per_launch(name, w, B):
+    """Algorithmic bytes of one launch of a kernel, for B samples."""
+    keys = 2 * w.d * w.n_vis * B
+    return {
+        "score": keys + 8 * w.n_vis * B,
+        "sim": keys + 4 * w.n_pivot * w.n_vis * B,
+        "sweep": keys,                       # fused scores + pivots + similarities: the keys count once
+        "gather": 2 * (2 * w.d * w.S_out) * B,
+        "pivot": 4 * w.n_vis * B,
+        "retain": 4 * w.n_pivot * w.n_vis * B + 12 * w.S_out * B,
+    }[name]
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock and throttle-reason samples taken while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower() == "active":
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def time_oracle(w, keys_bits, hidden_bits, budget_s):
+    """Time the oracle, single-threaded and as it stands, on as many leading samples as fit the budget."""
+    import oracle
+
+    t0 = time.perf_counter()
+    oracle.reduce(hidden_bits[:1], keys_bits[:1], w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, want_dup=False)
+    t1 = time.perf_counter() - t0
+    n = int(max(1, min(keys_bits.shape[0], budget_s / max(t1, 1e-6))))
+    t0 = time.perf_counter()
+    oracle.reduce(hidden_bits[:n], keys_bits[:n], w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, want_dup=False)
+    dt = time.perf_counter() - t0
+    return n, dt
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    from paper_2502_11494_b200 import workloads as W
+
+    oracle.build()
+    w = pick_workload(args)
+    total = args.steps + args.warmup
+    per_step_budget = max(0.5, 150.0 / max(total, 1))
+    k1, h1 = W.make_batch(w, device="cpu", samples=range(1))
+    t0 = time.perf_counter()
+    oracle.reduce(W.bits(h1), W.bits(k1), w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, want_dup=False)
+    t1 = time.perf_counter() - t0
+    n = int(max(1, min(w.B, per_step_budget / t1)))
+    keys, hidden = W.make_batch(w, device="cpu", samples=range(n))
+    kb, hb = W.bits(keys), W.bits(hidden)
+    for _ in range(args.warmup):
+        oracle.reduce(hb, kb, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, want_dup=False)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.reduce(hb, kb, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, want_dup=False)
+    dt = time.perf_counter() - t0
+    value = n * w.n_vis * args.steps / dt
+    sample = "first %d of %d samples of %s per step" % (n, w.B, w.name)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, n),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def workload_config(w, B):
+    return {"workload": w.name, "batch": B, "n_vis": w.n_vis, "seq_len": w.S, "d": w.d, "n_pivot": w.n_pivot,
+            "n_keep": w.n_keep, "vis_offset": w.vis_offset, "l2": "inputs larger than L2 (no flush needed)"}
+
+
+def time_steps(ctx, dart, torch, w, keys, hidden, outs, steps, warmup, opts, dist_on):
+    """Warm up, then time exactly `steps` reductions with CUDA events on the launching stream."""
+    import torch.distributed as dist
+
+    st = torch.cuda.current_stream()
+    sp = ctypes.c_void_p(st.cuda_stream)
+    P = lambda t: ctypes.c_void_p(t.data_ptr())  # noqa: E731
+
+    def step():
+        rc = dart.dart_reduce_ex(ctx.handle, P(hidden), P(keys), None, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep,
+                                 P(outs[0]), P(outs[1]), P(outs[2]), opts, None, sp)
+        if rc != 0:
+            raise dart.DartError(rc, "dart_reduce_ex")
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    dart.dart_profile_read(ctx.handle)
+    dart.dart_profile_enable(ctx.handle, True)
+    n0 = dart.dart_launch_count(ctx.handle)
+    if dist_on:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(st)
+    for _ in range(steps):
+        step()
+    e1.record(st)
+    torch.cuda.synchronize()
+    if dist_on:
+        dist.barrier()
+    ms = e0.elapsed_time(e1)
+    launches = dart.dart_launch_count(ctx.handle) - n0
+    dart.dart_profile_enable(ctx.handle, False)
+    _, prof = dart.dart_profile_read(ctx.handle)
+    if ctx.status() != 0:
+        raise RuntimeError("device status word reports an error")
+    return ms, launches, prof
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2502_11494_b200 import dart, workloads as W
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist_on = world > 1
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if dist_on:
+        dist.init_process_group("nccl", device_id=dev)
+    w = pick_workload(args)
+    B = w.B
+    # weak scaling: every rank reduces its own batch of B samples
+    keys, hidden = W.make_batch(w, device=dev, samples=range(rank * B, rank * B + B))
+    flags = 0 if args.no_e2e else dart.DART_FLAG_HOST_STAGING
+    ctx = dart.Dart(B, w.S, w.d, max(w.n_pivot, max(W.SWEEP_PIVOTS) if args.sweep else 0),
+                    max(w.n_keep, max(W.SWEEP_KEEP) if args.sweep else 0), device=local, flags=flags)
+    dart.dart_set_shape(ctx.handle, B, w.S)
+    opts = dart.dart_opts(0, 0, args.path, 0)
+
+    def alloc_outs(wl):
+        return (torch.empty((B, wl.S_out, wl.d), dtype=torch.bfloat16, device=dev),
+                torch.empty((B, wl.S_out), dtype=torch.int32, device=dev),
+                torch.empty((B, wl.S_out), dtype=torch.int64, device=dev))
+
+    outs = alloc_outs(w)
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms, launches, prof = time_steps(ctx, dart, torch, w, keys, hidden, outs, args.steps, args.warmup, opts, dist_on)
+    clocks = sampler.stop()
+    t = torch.tensor([ms], device=dev, dtype=torch.float64)
+    if dist_on:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * B * w.n_vis * args.steps / (ms * 1e-3)
+
+    peak, peak_src = measured_peak()
+    # dominant kernel = the slot with the largest share of the timed region
+    dom = max(prof, key=lambda k: prof[k][0]) if prof else None
+    roofline = None
+    if dom and prof[dom][1] > 0:
+        avg_ms = prof[dom][0] / prof[dom][1]
+        achieved = kernel_bytes_per_launch(dom, w, B) / (avg_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "traffic": None, "peak_source": peak_src + " copy bandwidth",
+                    "avg_launch_ms": avg_ms,
+                    "shares": {k: v[0] / max(sum(x[0] for x in prof.values()), 1e-9) for k, v in prof.items()}}
+    path_gbs = path_bytes_per_sample(w) * B / (ms_per_step * 1e-3) / 1e9
+    path_roof = {"algorithmic_bytes_per_step": path_bytes_per_sample(w) * B, "achieved": path_gbs, "unit": "GB/s",
+                 "frac_of_measured_copy": path_gbs / peak, "frac_of_nominal_8TBs": path_gbs / 8000.0}
+
+    sweep = None
+    if args.sweep and rank == 0:
+        sweep = []
+        for (p, k) in W.sweep_cells():
+            wc = w.with_(n_pivot=p, n_keep=k)
+            o2 = alloc_outs(wc)
+            ms2, _, _ = time_steps(ctx, dart, torch, wc, keys, hidden, o2, max(3, args.steps // 4), 2, opts, False)
+            n2 = max(3, args.steps // 4)
+            sweep.append({"n_pivot": p, "n_keep": k, "ms_per_step": ms2 / n2,
+                          "tokens_per_s": B * wc.n_vis * n2 / (ms2 * 1e-3),
+                          "path_frac_of_measured_copy": path_bytes_per_sample(wc) * B / (ms2 / n2 * 1e-3) / 1e9 / peak})
+            del o2
+
+    e2e = None
+    if not args.no_e2e:
+        # the same step through the host-buffer entry point: pinned inputs -> device -> pinned outputs
+        import psutil
+
+        need = 2 * keys.numel() * 2 + outs[0].numel() * 2
+        Be = B
+        while Be > 1 and need * Be // B * 2 > psutil.virtual_memory().available:
+            Be //= 2
+        hk = keys[:Be].cpu().pin_memory()
+        hh = hidden[:Be].cpu().pin_memory()
+        ho = (torch.empty((Be, w.S_out, w.d), dtype=torch.bfloat16).pin_memory(),
+              torch.empty((Be, w.S_out), dtype=torch.int32).pin_memory(),
+              torch.empty((Be, w.S_out), dtype=torch.int64).pin_memory())
+        dart.dart_set_shape(ctx.handle, Be, w.S)
+        P = lambda x: ctypes.c_void_p(x.data_ptr())  # noqa: E731
+        n_e2e = 2
+
+        def host_step():
+            rc = dart.dart_reduce_host(ctx.handle, P(hh), P(hk), w.vis_offset, w.n_vis, w.n_pivot, w.n_keep,
+                                       P(ho[0]), P(ho[1]), P(ho[2]))
+            if rc != 0:
+                raise dart.DartError(rc, "dart_reduce_host")
+
+        host_step()
+        if dist_on:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            host_step()
+        dt = time.perf_counter() - t0
+        td = torch.tensor([dt], device=dev, dtype=torch.float64)
+        if dist_on:
+            dist.all_reduce(td, op=dist.ReduceOp.MAX)
+        dt = float(td.item())
+        ok = bool(torch.equal(ho[1], outs[1][:Be].cpu())) if not args.sweep else None
+        e2e = {"value": world * Be * w.n_vis * n_e2e / dt, "unit": UNIT,
+               "h2d_bytes_per_step": int(hk.numel() * 2 + hh.numel() * 2),
+               "d2h_bytes_per_step": int(sum(x.numel() * x.element_size() for x in ho)),
+               "samples": Be, "steps": n_e2e, "ms_per_step": 1e3 * dt / n_e2e, "matches_device_run": ok}
+        dart.dart_set_shape(ctx.handle, B, w.S)
+
+    cpu = None
+    if rank == 0 and not args.no_cpu_baseline:
+        import oracle
+
+        oracle.build()
+        nb = min(B, 64)
+        kb, hb = W.bits(keys[:nb]), W.bits(hidden[:nb])
+        n, dt = time_oracle(w, kb, hb, budget_s=15.0)
+        cpu = {"value": n * w.n_vis / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": "first %d of %d samples of %s, one pass, %.1f s" % (n, B, w.name, dt)}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
+            "config": workload_config(w, B), "roofline": roofline, "path_roofline": path_roof,
+            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+        }
+        if sweep is not None:
+            line["sweep"] = sweep
+        print(json.dumps(line))
+    ctx.close()
+    if dist_on:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

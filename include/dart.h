@@ -1,0 +1,180 @@
+/*
+ * dart.h - C ABI of the B200 (sm_100a) implementation of DART's duplication-aware
+ * vision-token reduction step (arxiv 2502.11494, Sec. 3.3: Def. 1-2, Eq. 7-10).
+ *
+ * The step is inserted into MLLM prefill after a shallow layer: from the layer's key states it
+ * picks a few pivot tokens, scores every vision token by its cosine similarity to each pivot,
+ * keeps, per pivot, the least similar tokens under a budget, and packs the kept rows of the
+ * hidden states (with their indices and position ids) into a shorter dense sequence.
+ *
+ * Conventions
+ *   - Every function returns an int: DART_OK (0) or a negative DART_ERR_* code.  Nothing throws,
+ *     aborts or prints.  Errors found on the host are returned before anything is launched.
+ *   - "device" pointers are CUDA device memory of the context's device, "host" pointers are
+ *     ordinary (preferably pinned) host memory.  The caller owns every tensor; the library owns only
+ *     the context and its workspace.  bf16 tensors are passed as void*.
+ *   - Tensors are dense row-major: hidden/keys [B, S, d], out_hidden [B, S_out, d],
+ *     out_idx / out_pos [B, S_out], with S_out = S - n_vis + n_keep.  Vision tokens occupy rows
+ *     [vis_offset, vis_offset + n_vis) of every sample; all other rows are text and always kept.
+ *   - All device work is enqueued on the caller's stream; no call synchronises the host except
+ *     dart_create, dart_destroy, dart_status, dart_profile_read and dart_reduce_host.
+ *   - One context serves one stream at a time.  Results are bitwise reproducible for identical
+ *     inputs (no floating-point atomics anywhere).
+ */
+#ifndef DART_H
+#define DART_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DART_VERSION 100 /* major * 10000 + minor * 100 + patch */
+
+enum {
+    DART_OK = 0,
+    DART_ERR_NULL = -1,        /* a required pointer is NULL */
+    DART_ERR_BAD_SHAPE = -2,   /* sizes violate the rules listed at dart_reduce, or exceed the context's maxima */
+    DART_ERR_ALIGN = -3,       /* a tensor pointer is not 16-byte aligned */
+    DART_ERR_ALIAS = -4,       /* an output overlaps an input */
+    DART_ERR_CUDA = -5,        /* a CUDA call failed; see dart_last_cuda_error */
+    DART_ERR_NOMEM = -6,       /* host or device allocation failed */
+    DART_ERR_TIMEOUT = -7,     /* a bounded device-side wait gave up (reported by dart_status) */
+    DART_ERR_CHECK = -8,       /* a device-side self-check failed (reported by dart_status) */
+    DART_ERR_UNSUPPORTED = -9  /* option combination not available */
+};
+
+/* dart_desc.flags */
+#define DART_FLAG_HOST_STAGING 1u /* also allocate the device staging buffers dart_reduce_host needs */
+
+/* dart_opts.path */
+#define DART_PATH_AUTO 0
+#define DART_PATH_STAGED 1 /* one kernel per step of the method, every intermediate in the workspace */
+#define DART_PATH_FUSED 2  /* persistent sweep kernel (scores, pivots and similarities in one launch) */
+
+typedef struct dart_ctx dart_ctx; /* opaque: workspace, device status word, profiling events */
+
+/* Maxima a context is sized for.  d is fixed per context (a multiple of 8). */
+typedef struct {
+    int32_t B_max;  /* samples per call */
+    int32_t S_max;  /* sequence length (text + vision) */
+    int32_t d;      /* row width of hidden and keys, in elements */
+    int32_t P_max;  /* pivots */
+    int32_t Kp_max; /* retained vision tokens */
+    int32_t device; /* CUDA device ordinal */
+    uint32_t flags; /* DART_FLAG_* */
+} dart_desc;
+
+/* Options of dart_reduce_ex.  A zeroed struct means the defaults of dart_reduce. */
+typedef struct {
+    int32_t norm_kind;     /* 0 or 1: L1 row norm (the paper's "K-norm", Sec. 3.3 footnote); 2: Euclidean norm */
+    int32_t pivot_smallest; /* 0: pivots = largest scores (Table 1 caption); 1: smallest (ablation variant) */
+    int32_t path;          /* DART_PATH_* */
+    int32_t wait_limit;    /* 0: default; > 0: iteration limit of bounded device-side waits (testing) */
+} dart_opts;
+
+/* Optional per-step outputs of dart_reduce_ex; every member is a device pointer or NULL. */
+typedef struct {
+    float *l1;          /* [B, n_vis] sum_c |K[j,c]|                       (K-norm footnote)  */
+    float *ssq;         /* [B, n_vis] sum_c K[j,c]^2                       (Eq. 7 denominators) */
+    int32_t *pivot_idx; /* [B, n_pivot] vision-relative indices in rank order (Def. 1)        */
+    float *sim;         /* [B, n_pivot, n_vis] dup(p_i, x_j)               (Eq. 7)             */
+    float *eps;         /* [B, n_pivot] per-pivot threshold eps_i, NaN if the pivot's quota is 0 (Eq. 9) */
+    uint8_t *keep;      /* [B, n_vis] 1 = retained                         (Eq. 10)            */
+    int32_t *owner;     /* [B, n_vis] -1 dropped; i retained by pivot i; n_pivot + i pivot of rank i */
+} dart_debug;
+
+/*
+ * Create a context for shapes up to the maxima in *desc on desc->device and allocate its
+ * workspace with cudaMalloc (the only device allocations the library ever makes).
+ * Errors: NULL, BAD_SHAPE (non-positive sizes, d % 8 != 0, P_max > Kp_max, Kp_max > S_max), CUDA, NOMEM.
+ */
+int dart_create(dart_ctx **out, const dart_desc *desc);
+
+/* Free the workspace and the context.  Synchronises the device.  NULL is accepted. */
+int dart_destroy(dart_ctx *ctx);
+
+/* Batch size and sequence length of the following calls (1 <= B <= B_max, 1 <= S <= S_max). */
+int dart_set_shape(dart_ctx *ctx, int B, int S);
+
+/*
+ * The reduction step (Sec. 3.3), for every sample b independently:
+ *   1. score_j = L1 norm of keys[b, vis_offset + j, :]                       (K-norm footnote)
+ *   2. pivots p_0..p_{P-1} = the n_pivot vision tokens of largest score, in rank order; equal
+ *      scores rank the lower index first                                     (Def. 1, Table 1 caption)
+ *   3. dup[i][j] = cosine of key rows p_i and j, fp32 accumulation           (Def. 2, Eq. 7)
+ *   4. kept = pivots; with q = (n_keep - P) / P and r = (n_keep - P) % P, pivot i in rank order keeps
+ *      its q (+1 if i < r) not-yet-kept tokens of lowest dup[i][.], ties to the lower index; eps_i
+ *      is the largest dup it kept                                            (Eq. 9-10)
+ *   5. out_idx[b] = ascending sequence indices of all text rows and the kept vision rows;
+ *      out_hidden[b, t, :] = hidden[b, out_idx[b, t], :]; out_pos[b, t] = out_idx[b, t].
+ *
+ *   hidden     [B, S, d] bf16, device, 16-byte aligned, read-only
+ *   keys       [B, S, d] bf16, device, or NULL to score and compare the hidden states themselves
+ *   out_hidden [B, S_out, d] bf16, device, 16-byte aligned, must not overlap hidden or keys
+ *   out_idx    [B, S_out] int32, device
+ *   out_pos    [B, S_out] int64, device
+ *   stream     a cudaStream_t (NULL = the legacy default stream)
+ * Shape rules: 1 <= n_pivot <= n_keep <= n_vis, 0 <= vis_offset, vis_offset + n_vis <= S,
+ * n_pivot <= P_max, n_keep <= Kp_max.  n_keep == n_vis is the identity.  Inputs must be finite.
+ * Errors: NULL, BAD_SHAPE, ALIGN, ALIAS, CUDA (launch failure).  Asynchronous: dart_status.
+ */
+int dart_reduce(dart_ctx *ctx, const void *hidden, const void *keys, int vis_offset, int n_vis,
+                int n_pivot, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos,
+                void *stream);
+
+/*
+ * dart_reduce with caller position ids, options and per-step outputs.
+ *   pos_in [B, S] int64 device, or NULL for pos_in[b, s] = s; out_pos[b, t] = pos_in[b, out_idx[b, t]]
+ *   opts   NULL = defaults;  dbg NULL = no per-step outputs.
+ * Asking for dbg->sim makes every path materialise the whole similarity matrix.
+ */
+int dart_reduce_ex(dart_ctx *ctx, const void *hidden, const void *keys, const int64_t *pos_in,
+                   int vis_offset, int n_vis, int n_pivot, int n_keep, void *out_hidden,
+                   int32_t *out_idx, int64_t *out_pos, const dart_opts *opts, const dart_debug *dbg,
+                   void *stream);
+
+/*
+ * The same step for HOST buffers: copies hidden and keys to the device in chunks of samples,
+ * reduces each chunk while the next one is in flight, copies the packed outputs back and returns
+ * after everything has completed.  All pointers are host memory (pinned memory makes the copies
+ * asynchronous); keys may be NULL.  Needs a context created with DART_FLAG_HOST_STAGING
+ * (else UNSUPPORTED).  The shape of the call is the one set by dart_set_shape; B may exceed the
+ * chunk size but not B_max.
+ */
+int dart_reduce_host(dart_ctx *ctx, const void *hidden, const void *keys, int vis_offset, int n_vis,
+                     int n_pivot, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos);
+
+/*
+ * Read the device status word (synchronises the context's device): DART_OK, DART_ERR_TIMEOUT if a
+ * bounded wait inside a kernel gave up, DART_ERR_CHECK if a self-check failed.  Reading clears it.
+ */
+int dart_status(dart_ctx *ctx);
+
+/* The cudaError_t of the last failed CUDA call made on behalf of this context (0 if none). */
+int dart_last_cuda_error(const dart_ctx *ctx);
+
+/* Bytes of device memory the context holds. */
+size_t dart_workspace_bytes(const dart_ctx *ctx);
+
+/* Kernels launched on behalf of this context since it was created. */
+int64_t dart_launch_count(const dart_ctx *ctx);
+
+/*
+ * Per-kernel timing.  While enabled, every kernel launch of dart_reduce* is bracketed by CUDA events
+ * on the caller's stream.  dart_profile_read synchronises those events and returns, for each kernel
+ * slot k < *n_slots, the accumulated milliseconds and launch count since the last read; names[k]
+ * (if names != NULL) points to a static string.  On entry *n_slots is the capacity of the arrays.
+ */
+int dart_profile_enable(dart_ctx *ctx, int on);
+int dart_profile_read(dart_ctx *ctx, float *ms, int32_t *launches, const char **names, int *n_slots);
+
+const char *dart_strerror(int code);
+int dart_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DART_H */

@@ -1,0 +1,173 @@
+"""Parity rules between a candidate implementation's outputs and the oracle (TEST INFRASTRUCTURE).
+
+Takes plain numpy arrays from both sides; imports nothing from the CUDA path.
+
+Rules (bf16 inputs, fp32 accumulation on the candidate side, fp64 in the oracle):
+  * norms and similarities: relative error <= 1e-2 (similarities: |d| <= 1e-2 |dup| + 1e-4, since a
+    relative bound is void near 0);
+  * wherever the oracle's selection margin exceeds 1e-3 (relative score gap along the pivot ranking,
+    absolute dup gap at every retention boundary) pivots, kept indices, gathered rows and position ids
+    are bit-exact;
+  * below that margin several results are equally right: the candidate's choice must be *valid under
+    tolerance* - replaying its own per-pivot assignment against the oracle's fp64 similarities, no
+    token it left behind beats its threshold by more than the tolerance - and everything that does
+    not depend on the near-tie (counts, order, text rows, gathered bits, position ids) is exact.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+
+from . import dart_oracle as _o
+
+REL_TOL = 1e-2
+SIM_ABS_FLOOR = 1e-4
+MARGIN = 1e-3
+
+
+@dataclass
+class ParityReport:
+    samples: int = 0
+    exact: int = 0                 # samples whose out_idx equals the oracle's
+    above_margin: int = 0          # samples with margin > MARGIN (exactness enforced)
+    max_rel_l1: float = 0.0
+    max_rel_l2: float = 0.0
+    max_abs_sim: float = 0.0
+    min_margin: float = float("inf")
+    notes: list = field(default_factory=list)
+
+    def merge(self, o: "ParityReport"):
+        self.samples += o.samples
+        self.exact += o.exact
+        self.above_margin += o.above_margin
+        self.max_rel_l1 = max(self.max_rel_l1, o.max_rel_l1)
+        self.max_rel_l2 = max(self.max_rel_l2, o.max_rel_l2)
+        self.max_abs_sim = max(self.max_abs_sim, o.max_abs_sim)
+        self.min_margin = min(self.min_margin, o.min_margin)
+        self.notes += o.notes
+        return self
+
+
+def quotas(P: int, n_keep: int):
+    q, r = divmod(n_keep - P, P)
+    return [q + (1 if i < r else 0) for i in range(P)]
+
+
+def check_packed_outputs(out_hidden, out_idx, out_pos, hidden_bits, pos_in, vis_offset, n_vis, n_keep):
+    """Rules that hold whatever the near-ties decide (one sample)."""
+    S = hidden_bits.shape[0]
+    S_out = S - n_vis + n_keep
+    assert out_idx.shape == (S_out,), "packed length"
+    assert np.all(np.diff(out_idx.astype(np.int64)) > 0), "out_idx must be strictly ascending (original order)"
+    assert np.array_equal(out_idx[:vis_offset], np.arange(vis_offset)), "text rows before the vision block"
+    n_after = S - vis_offset - n_vis
+    assert np.array_equal(out_idx[S_out - n_after:], np.arange(vis_offset + n_vis, S)), "text rows after"
+    mid = out_idx[vis_offset:vis_offset + n_keep]
+    assert mid.min() >= vis_offset and mid.max() < vis_offset + n_vis, "kept rows lie in the vision block"
+    expect_pos = out_idx.astype(np.int64) if pos_in is None else pos_in[out_idx]
+    assert np.array_equal(out_pos, expect_pos), "position ids follow the kept rows"
+    if out_hidden is not None:
+        assert np.array_equal(out_hidden, hidden_bits[out_idx]), "gathered rows are bit copies of hidden rows"
+
+
+def check_scores(l1, ssq, ora_l1, ora_l2, rep: ParityReport, tol=REL_TOL):
+    rl1 = np.abs(l1.astype(np.float64) - ora_l1) / np.maximum(ora_l1, 1e-300)
+    l2 = np.sqrt(ssq.astype(np.float64))
+    rl2 = np.abs(l2 - ora_l2) / np.maximum(ora_l2, 1e-300)
+    rep.max_rel_l1 = max(rep.max_rel_l1, float(rl1.max()))
+    rep.max_rel_l2 = max(rep.max_rel_l2, float(rl2.max()))
+    assert rl1.max() <= tol, "L1 scores off by %g relative" % rl1.max()
+    assert rl2.max() <= tol, "Euclidean norms off by %g relative" % rl2.max()
+
+
+def check_sim(sim, ora_dup, rep: ParityReport, tol=REL_TOL, floor=SIM_ABS_FLOOR):
+    err = np.abs(sim.astype(np.float64) - ora_dup)
+    rep.max_abs_sim = max(rep.max_abs_sim, float(err.max()))
+    bad = err > tol * np.abs(ora_dup) + floor
+    assert not bad.any(), "similarities off by up to %g" % err.max()
+
+
+def check_valid_under_tolerance(keys_bits, vis_offset, n_vis, n_keep, pivot_idx, owner, ora_score, ora_l2,
+                                largest=True, tol=MARGIN):
+    """Replay the candidate's own pivots and per-pivot assignment against fp64 quantities (one sample).
+    ora_score is the oracle's ranking score (L1 norms, or the Euclidean norms for that variant)."""
+    P = len(pivot_idx)
+    assert len(set(pivot_idx.tolist())) == P, "pivots must be distinct"
+    s = ora_score
+    sgn = 1.0 if largest else -1.0
+    others = np.setdiff1d(np.arange(n_vis), pivot_idx)
+    if len(others):
+        worst_piv = (sgn * s[pivot_idx]).min()
+        best_other = (sgn * s[others]).max()
+        assert worst_piv >= best_other - tol * abs(best_other), "a non-pivot beats a pivot beyond tolerance"
+    ranked = sgn * s[pivot_idx]
+    assert np.all(ranked[:-1] >= ranked[1:] - tol * np.abs(ranked[:-1])), "pivot rank order beyond tolerance"
+    dup = _o.similarity(keys_bits, vis_offset, n_vis, pivot_idx, ora_l2)
+    kept = np.zeros(n_vis, bool)
+    kept[pivot_idx] = True
+    assert [int(owner[p]) for p in pivot_idx] == [P + i for i in range(P)], "pivots carry their rank in owner"
+    for i, qi in enumerate(quotas(P, n_keep)):
+        mine = np.nonzero(owner == i)[0]
+        assert len(mine) == qi, "pivot %d retained %d tokens, quota %d" % (i, len(mine), qi)
+        if qi == 0:
+            continue
+        assert not kept[mine].any(), "pivot %d retained a token that was already kept" % i
+        eps_i = dup[i, mine].max()
+        left = ~kept
+        left[mine] = False
+        if left.any():
+            assert dup[i, left].min() >= eps_i - tol, \
+                "pivot %d left behind a token %g below its threshold" % (i, eps_i - dup[i, left].min())
+        kept[mine] = True
+    assert int(kept.sum()) == n_keep
+    assert np.array_equal(np.nonzero(owner >= 0)[0], np.nonzero(kept)[0]), "owner and kept set disagree"
+    return kept
+
+
+def check_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, n_vis, n_pivot, n_keep,
+                out_hidden, out_idx, out_pos, dbg=None, pos_in=None, largest=True, norm_kind=1,
+                require_exact_above=MARGIN) -> ParityReport:
+    """All rules over a batch.  ``dbg`` (optional) holds the candidate's per-step outputs as numpy arrays:
+    l1, ssq, pivot_idx, sim, eps, keep, owner.  Without it only the packed outputs are checked."""
+    B = out_idx.shape[0]
+    rep = ParityReport()
+    margin = ora.margin
+    for b in range(B):
+        rep.samples += 1
+        rep.min_margin = min(rep.min_margin, float(margin[b]))
+        pin = None if pos_in is None else pos_in[b]
+        check_packed_outputs(None if out_hidden is None else out_hidden[b], out_idx[b], out_pos[b], hidden_bits[b],
+                             pin, vis_offset, n_vis, n_keep)
+        same = np.array_equal(out_idx[b], ora.out_idx[b])
+        rep.exact += int(same)
+        if margin[b] > require_exact_above:
+            rep.above_margin += 1
+            assert same, "sample %d: kept indices differ although the margin is %g" % (b, margin[b])
+            if out_hidden is not None and ora.out_hidden is not None:
+                assert np.array_equal(out_hidden[b], ora.out_hidden[b])
+            assert np.array_equal(out_pos[b], ora.out_pos[b])
+        if dbg is None:
+            continue
+        check_scores(dbg["l1"][b], dbg["ssq"][b], ora.l1[b], ora.l2[b], rep)
+        kept_gpu = np.zeros(n_vis, bool)
+        kept_gpu[out_idx[b][vis_offset:vis_offset + n_keep] - vis_offset] = True
+        assert np.array_equal(dbg["keep"][b].astype(bool), kept_gpu), "keep flags and out_idx disagree"
+        assert np.array_equal(dbg["owner"][b] >= 0, kept_gpu), "owner and out_idx disagree"
+        same_piv = np.array_equal(dbg["pivot_idx"][b], ora.pivot_idx[b])
+        if ora.pivot_gap[b] > require_exact_above:
+            assert same_piv, "sample %d: pivots differ although the score gap is %g" % (b, ora.pivot_gap[b])
+        if same_piv and ora.dup is not None:
+            check_sim(dbg["sim"][b], ora.dup[b], rep)
+        if margin[b] > require_exact_above:
+            assert np.array_equal(dbg["owner"][b], ora.owner[b])
+            qs = quotas(n_pivot, n_keep)
+            has = np.array([q > 0 for q in qs])
+            e = dbg["eps"][b].astype(np.float64)
+            assert np.all(np.isnan(e[~has])) and np.all(np.abs(e[has] - ora.eps[b][has]) <= REL_TOL * np.abs(ora.eps[b][has]) + SIM_ABS_FLOOR)
+        else:
+            check_valid_under_tolerance(keys_bits[b], vis_offset, n_vis, n_keep, dbg["pivot_idx"][b], dbg["owner"][b],
+                                        ora.l1[b] if norm_kind == 1 else ora.l2[b], ora.l2[b], largest=largest)
+            if not same:
+                rep.notes.append("sample %d differs below margin %.2e (valid under tolerance)" % (b, margin[b]))
+    return rep

@@ -1,0 +1,468 @@
+// Host side of the C ABI declared in include/dart.h: argument checks, workspace, launches.
+#include "../../include/dart.h"
+
+#include <cuda_runtime.h>
+
+#include <new>
+#include <vector>
+
+#include "dart_staged.cuh"
+
+namespace {
+
+enum Slot { SLOT_SCORE = 0, SLOT_PIVOT, SLOT_SIM, SLOT_RETAIN, SLOT_GATHER, SLOT_COUNT };
+const char *const kSlotNames[SLOT_COUNT] = {"score", "pivot", "sim", "retain", "gather"};
+
+struct EventPair {
+    cudaEvent_t start, stop;
+    int slot;
+};
+
+} // namespace
+
+struct dart_ctx {
+    dart_desc desc;
+    int B, S;
+    int last_cuda;
+    int64_t launches;
+    size_t bytes;
+    // workspace (device), indexed with the shapes of the current call
+    float *l1, *ssq, *sim, *eps;
+    int32_t *pivot_idx, *owner;
+    uint8_t *keep;
+    int *status; // device status word
+    // profiling
+    bool profiling;
+    std::vector<EventPair> pending, spare;
+    float slot_ms[SLOT_COUNT];
+    int32_t slot_launches[SLOT_COUNT];
+    int max_smem_optin;
+    // host staging (DART_FLAG_HOST_STAGING): two sets of device buffers for chunks of samples
+    int chunk;                      // samples per chunk
+    void *st_hidden[2], *st_keys[2], *st_out_hidden[2];
+    int32_t *st_out_idx[2];
+    int64_t *st_out_pos[2];
+    cudaStream_t s_h2d, s_run, s_d2h;
+    cudaEvent_t ev_in[2], ev_run[2], ev_out[2];
+};
+
+namespace {
+
+int cuda_fail(dart_ctx *ctx, cudaError_t e)
+{
+    if (ctx) ctx->last_cuda = (int)e;
+    return e == cudaErrorMemoryAllocation ? DART_ERR_NOMEM : DART_ERR_CUDA;
+}
+
+#define DART_CUDA(ctx, call)                                   \
+    do {                                                       \
+        cudaError_t e__ = (call);                              \
+        if (e__ != cudaSuccess) return cuda_fail((ctx), e__);  \
+    } while (0)
+
+template <typename T>
+int ws_alloc(dart_ctx *ctx, T **p, size_t count)
+{
+    size_t bytes = (count * sizeof(T) + 255) / 256 * 256;
+    cudaError_t e = cudaMalloc((void **)p, bytes);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->bytes += bytes;
+    return DART_OK;
+}
+
+// Scoped device switch: the library never leaves another device current.
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || (cudaSetDevice(dev) == cudaSuccess);
+        if (prev == dev) prev = -1;
+    }
+    ~DeviceGuard()
+    {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+struct Prof {
+    dart_ctx *ctx;
+    cudaStream_t st;
+    EventPair ev;
+    bool on;
+    Prof(dart_ctx *c, cudaStream_t s, int slot) : ctx(c), st(s), on(c->profiling)
+    {
+        ++ctx->launches;
+        if (!on) return;
+        if (!ctx->spare.empty()) {
+            ev = ctx->spare.back();
+            ctx->spare.pop_back();
+        } else if (cudaEventCreate(&ev.start) != cudaSuccess || cudaEventCreate(&ev.stop) != cudaSuccess) {
+            on = false;
+            return;
+        }
+        ev.slot = slot;
+        cudaEventRecord(ev.start, st);
+    }
+    ~Prof()
+    {
+        if (!on) return;
+        cudaEventRecord(ev.stop, st);
+        ctx->pending.push_back(ev);
+    }
+};
+
+bool overlaps(const void *a, size_t na, const void *b, size_t nb)
+{
+    if (!a || !b) return false;
+    uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
+    return x < y + nb && y < x + na;
+}
+
+int next_pow2(int v)
+{
+    int p = 1;
+    while (p < v) p <<= 1;
+    return p;
+}
+
+int check_call(const dart_ctx *ctx, const void *hidden, const void *keys, int vis_offset, int n_vis, int n_pivot,
+               int n_keep, const void *out_hidden, const void *out_idx, const void *out_pos, bool host = false)
+{
+    if (!ctx || !hidden || !out_hidden || !out_idx || !out_pos) return DART_ERR_NULL;
+    const int S = ctx->S;
+    if (ctx->B < 1 || S < 1) return DART_ERR_BAD_SHAPE;
+    if (n_pivot < 1 || n_pivot > n_keep || n_keep > n_vis || vis_offset < 0 || n_vis < 1) return DART_ERR_BAD_SHAPE;
+    if ((long long)vis_offset + n_vis > S) return DART_ERR_BAD_SHAPE;
+    if (n_pivot > ctx->desc.P_max || n_keep > ctx->desc.Kp_max) return DART_ERR_BAD_SHAPE;
+    if (!host && (((uintptr_t)hidden | (uintptr_t)keys | (uintptr_t)out_hidden) & 15u)) return DART_ERR_ALIGN;
+    if (((uintptr_t)out_idx & 3u) || ((uintptr_t)out_pos & 7u)) return DART_ERR_ALIGN;
+    const size_t in_bytes = (size_t)ctx->B * S * ctx->desc.d * 2;
+    const size_t S_out = (size_t)S - n_vis + n_keep;
+    const size_t out_bytes = (size_t)ctx->B * S_out * ctx->desc.d * 2;
+    if (overlaps(out_hidden, out_bytes, hidden, in_bytes) || overlaps(out_hidden, out_bytes, keys, in_bytes))
+        return DART_ERR_ALIAS;
+    return DART_OK;
+}
+
+int launch_staged(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, const int64_t *pos_in, int vis_offset,
+                  int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos,
+                  const dart_opts &o, const dart_debug *dbg, cudaStream_t st)
+{
+    using namespace dart;
+    const int S = ctx->S, d8 = ctx->desc.d / 8, S_out = S - n_vis + n_keep;
+    const uint4 *keys = (const uint4 *)(keys_in ? keys_in : hidden);
+    const long long rows = (long long)B * n_vis;
+    {
+        Prof p(ctx, st, SLOT_SCORE);
+        unsigned grid = (unsigned)((rows + kScoreWarps - 1) / kScoreWarps);
+        score_kernel<<<grid, kScoreWarps * 32, 0, st>>>(keys, S, d8, vis_offset, n_vis, rows, ctx->l1, ctx->ssq);
+    }
+    {
+        Prof p(ctx, st, SLOT_PIVOT);
+        int P_pad = next_pow2(P);
+        pivot_kernel<<<B, kSelectThreads, (size_t)P_pad * 8, st>>>(o.norm_kind == 2 ? ctx->ssq : ctx->l1, n_vis, P,
+                                                                  P_pad, o.pivot_smallest, ctx->pivot_idx);
+    }
+    {
+        Prof p(ctx, st, SLOT_SIM);
+        size_t smem = (size_t)kSimPivotChunk * d8 * 16;
+        dim3 grid((n_vis + kSimRowsPerCta - 1) / kSimRowsPerCta, B);
+        for (int p0 = 0; p0 < P; p0 += kSimPivotChunk)
+            sim_alu_kernel<<<grid, kSimWarps * 32, smem, st>>>(keys, S, d8, vis_offset, n_vis, P, p0, ctx->pivot_idx,
+                                                              ctx->ssq, ctx->sim);
+        ctx->launches += (P - 1) / kSimPivotChunk;
+    }
+    {
+        Prof p(ctx, st, SLOT_RETAIN);
+        retain_kernel<<<B, kSelectThreads, (size_t)n_vis, st>>>(ctx->sim, ctx->pivot_idx, pos_in, S, vis_offset, n_vis, P,
+                                                               n_keep, out_idx, out_pos, ctx->keep, ctx->owner,
+                                                               ctx->eps);
+    }
+    {
+        Prof p(ctx, st, SLOT_GATHER);
+        long long orows = (long long)B * S_out;
+        unsigned grid = (unsigned)((orows + kGatherWarps - 1) / kGatherWarps);
+        gather_kernel<<<grid, kGatherWarps * 32, 0, st>>>((const uint4 *)hidden, out_idx, S, S_out, d8, orows,
+                                                         (uint4 *)out_hidden);
+    }
+    DART_CUDA(ctx, cudaGetLastError());
+    if (dbg) {
+        const size_t nv = (size_t)B * n_vis, np = (size_t)B * P;
+        if (dbg->l1) DART_CUDA(ctx, cudaMemcpyAsync(dbg->l1, ctx->l1, nv * 4, cudaMemcpyDeviceToDevice, st));
+        if (dbg->ssq) DART_CUDA(ctx, cudaMemcpyAsync(dbg->ssq, ctx->ssq, nv * 4, cudaMemcpyDeviceToDevice, st));
+        if (dbg->pivot_idx)
+            DART_CUDA(ctx, cudaMemcpyAsync(dbg->pivot_idx, ctx->pivot_idx, np * 4, cudaMemcpyDeviceToDevice, st));
+        if (dbg->sim) DART_CUDA(ctx, cudaMemcpyAsync(dbg->sim, ctx->sim, np * n_vis * 4, cudaMemcpyDeviceToDevice, st));
+        if (dbg->eps) DART_CUDA(ctx, cudaMemcpyAsync(dbg->eps, ctx->eps, np * 4, cudaMemcpyDeviceToDevice, st));
+        if (dbg->keep) DART_CUDA(ctx, cudaMemcpyAsync(dbg->keep, ctx->keep, nv, cudaMemcpyDeviceToDevice, st));
+        if (dbg->owner) DART_CUDA(ctx, cudaMemcpyAsync(dbg->owner, ctx->owner, nv * 4, cudaMemcpyDeviceToDevice, st));
+    }
+    return DART_OK;
+}
+
+} // namespace
+
+extern "C" {
+
+int dart_create(dart_ctx **out, const dart_desc *desc)
+{
+    if (!out || !desc) return DART_ERR_NULL;
+    *out = nullptr;
+    if (desc->B_max < 1 || desc->S_max < 1 || desc->d < 8 || desc->d % 8 != 0 || desc->P_max < 1 ||
+        desc->P_max > desc->Kp_max || desc->Kp_max > desc->S_max || desc->P_max > 1024)
+        return DART_ERR_BAD_SHAPE;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || desc->device < 0 || desc->device >= ndev) return DART_ERR_CUDA;
+    dart_ctx *ctx = new (std::nothrow) dart_ctx();
+    if (!ctx) return DART_ERR_NOMEM;
+    ctx->desc = *desc;
+    ctx->B = desc->B_max;
+    ctx->S = desc->S_max;
+    DeviceGuard g(desc->device);
+    if (!g.ok) {
+        delete ctx;
+        return DART_ERR_CUDA;
+    }
+    const size_t nv = (size_t)desc->B_max * desc->S_max, np = (size_t)desc->B_max * desc->P_max;
+    int rc = DART_OK;
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->l1, nv);
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->ssq, nv);
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->sim, np * desc->S_max);
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->eps, np);
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->pivot_idx, np);
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->owner, nv);
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->keep, nv);
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->status, 64);
+    if (rc == DART_OK && cudaMemset(ctx->status, 0, 256) != cudaSuccess) rc = DART_ERR_CUDA;
+    if (rc == DART_OK) {
+        cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, desc->device);
+        size_t sim_smem = (size_t)dart::kSimPivotChunk * (desc->d / 8) * 16;
+        if (sim_smem > (size_t)ctx->max_smem_optin || (size_t)desc->S_max > (size_t)ctx->max_smem_optin)
+            rc = DART_ERR_BAD_SHAPE; // rows wider than 8 pivot rows of shared memory are not supported
+        else if (cudaFuncSetAttribute(dart::sim_alu_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)sim_smem) != cudaSuccess ||
+                 cudaFuncSetAttribute(dart::retain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      desc->S_max) != cudaSuccess)
+            rc = DART_ERR_CUDA;
+    }
+    if (rc == DART_OK && (desc->flags & DART_FLAG_HOST_STAGING)) {
+        // chunk = as many samples as fit ~512 MiB of input staging per buffer set (at least one)
+        const size_t per_sample = (size_t)desc->S_max * desc->d * 2;
+        size_t c = ((size_t)512 << 20) / (2 * per_sample);
+        ctx->chunk = (int)(c < 1 ? 1 : (c > (size_t)desc->B_max ? (size_t)desc->B_max : c));
+        for (int k = 0; k < 2 && rc == DART_OK; ++k) {
+            if (rc == DART_OK) rc = ws_alloc(ctx, (uint8_t **)&ctx->st_hidden[k], ctx->chunk * per_sample);
+            if (rc == DART_OK) rc = ws_alloc(ctx, (uint8_t **)&ctx->st_keys[k], ctx->chunk * per_sample);
+            if (rc == DART_OK) rc = ws_alloc(ctx, (uint8_t **)&ctx->st_out_hidden[k], ctx->chunk * per_sample);
+            if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->st_out_idx[k], (size_t)ctx->chunk * desc->S_max);
+            if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->st_out_pos[k], (size_t)ctx->chunk * desc->S_max);
+            if (rc == DART_OK && (cudaEventCreateWithFlags(&ctx->ev_in[k], cudaEventDisableTiming) != cudaSuccess ||
+                                  cudaEventCreateWithFlags(&ctx->ev_run[k], cudaEventDisableTiming) != cudaSuccess ||
+                                  cudaEventCreateWithFlags(&ctx->ev_out[k], cudaEventDisableTiming) != cudaSuccess))
+                rc = DART_ERR_CUDA;
+        }
+        if (rc == DART_OK && (cudaStreamCreateWithFlags(&ctx->s_h2d, cudaStreamNonBlocking) != cudaSuccess ||
+                              cudaStreamCreateWithFlags(&ctx->s_run, cudaStreamNonBlocking) != cudaSuccess ||
+                              cudaStreamCreateWithFlags(&ctx->s_d2h, cudaStreamNonBlocking) != cudaSuccess))
+            rc = DART_ERR_CUDA;
+    }
+    if (rc != DART_OK) {
+        dart_destroy(ctx);
+        return rc;
+    }
+    *out = ctx;
+    return DART_OK;
+}
+
+int dart_destroy(dart_ctx *ctx)
+{
+    if (!ctx) return DART_OK;
+    DeviceGuard g(ctx->desc.device);
+    cudaDeviceSynchronize();
+    for (auto &e : ctx->pending) ctx->spare.push_back(e);
+    for (auto &e : ctx->spare) {
+        cudaEventDestroy(e.start);
+        cudaEventDestroy(e.stop);
+    }
+    cudaFree(ctx->l1);
+    cudaFree(ctx->ssq);
+    cudaFree(ctx->sim);
+    cudaFree(ctx->eps);
+    cudaFree(ctx->pivot_idx);
+    cudaFree(ctx->owner);
+    cudaFree(ctx->keep);
+    cudaFree(ctx->status);
+    for (int k = 0; k < 2; ++k) {
+        cudaFree(ctx->st_hidden[k]);
+        cudaFree(ctx->st_keys[k]);
+        cudaFree(ctx->st_out_hidden[k]);
+        cudaFree(ctx->st_out_idx[k]);
+        cudaFree(ctx->st_out_pos[k]);
+        if (ctx->ev_in[k]) cudaEventDestroy(ctx->ev_in[k]);
+        if (ctx->ev_run[k]) cudaEventDestroy(ctx->ev_run[k]);
+        if (ctx->ev_out[k]) cudaEventDestroy(ctx->ev_out[k]);
+    }
+    if (ctx->s_h2d) cudaStreamDestroy(ctx->s_h2d);
+    if (ctx->s_run) cudaStreamDestroy(ctx->s_run);
+    if (ctx->s_d2h) cudaStreamDestroy(ctx->s_d2h);
+    delete ctx;
+    return DART_OK;
+}
+
+int dart_set_shape(dart_ctx *ctx, int B, int S)
+{
+    if (!ctx) return DART_ERR_NULL;
+    if (B < 1 || S < 1 || B > ctx->desc.B_max || S > ctx->desc.S_max) return DART_ERR_BAD_SHAPE;
+    ctx->B = B;
+    ctx->S = S;
+    return DART_OK;
+}
+
+int dart_reduce_ex(dart_ctx *ctx, const void *hidden, const void *keys, const int64_t *pos_in, int vis_offset,
+                   int n_vis, int n_pivot, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos,
+                   const dart_opts *opts, const dart_debug *dbg, void *stream)
+{
+    int rc = check_call(ctx, hidden, keys, vis_offset, n_vis, n_pivot, n_keep, out_hidden, out_idx, out_pos);
+    if (rc != DART_OK) return rc;
+    dart_opts o = {};
+    if (opts) o = *opts;
+    if (o.norm_kind == 0) o.norm_kind = 1;
+    if (o.norm_kind != 1 && o.norm_kind != 2) return DART_ERR_UNSUPPORTED;
+    if (o.path != DART_PATH_AUTO && o.path != DART_PATH_STAGED) return DART_ERR_UNSUPPORTED;
+    if ((uintptr_t)pos_in & 7u) return DART_ERR_ALIGN;
+    DeviceGuard g(ctx->desc.device);
+    if (!g.ok) return DART_ERR_CUDA;
+    return launch_staged(ctx, ctx->B, hidden, keys, pos_in, vis_offset, n_vis, n_pivot, n_keep, out_hidden, out_idx,
+                         out_pos, o, dbg, (cudaStream_t)stream);
+}
+
+int dart_reduce(dart_ctx *ctx, const void *hidden, const void *keys, int vis_offset, int n_vis, int n_pivot,
+                int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos, void *stream)
+{
+    return dart_reduce_ex(ctx, hidden, keys, nullptr, vis_offset, n_vis, n_pivot, n_keep, out_hidden, out_idx, out_pos,
+                          nullptr, nullptr, stream);
+}
+
+int dart_reduce_host(dart_ctx *ctx, const void *hidden, const void *keys, int vis_offset, int n_vis, int n_pivot,
+                     int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos)
+{
+    int rc = check_call(ctx, hidden, keys, vis_offset, n_vis, n_pivot, n_keep, out_hidden, out_idx, out_pos, true);
+    if (rc != DART_OK) return rc;
+    if (!(ctx->desc.flags & DART_FLAG_HOST_STAGING)) return DART_ERR_UNSUPPORTED;
+    DeviceGuard g(ctx->desc.device);
+    if (!g.ok) return DART_ERR_CUDA;
+    const int B = ctx->B, S = ctx->S, d = ctx->desc.d, S_out = S - n_vis + n_keep;
+    const size_t in_row = (size_t)S * d * 2, out_row = (size_t)S_out * d * 2;
+    dart_opts o = {};
+    o.norm_kind = 1;
+    int n_chunks = (B + ctx->chunk - 1) / ctx->chunk;
+    // three streams: copy-in of chunk c+1 and copy-out of chunk c-1 overlap the reduction of chunk c
+    for (int c = 0; c < n_chunks; ++c) {
+        const int k = c & 1, b0 = c * ctx->chunk, nb = (B - b0 < ctx->chunk) ? B - b0 : ctx->chunk;
+        if (c >= 2) { // buffer set k is free once chunk c-2 has been reduced and copied out
+            DART_CUDA(ctx, cudaStreamWaitEvent(ctx->s_h2d, ctx->ev_run[k], 0));
+            DART_CUDA(ctx, cudaStreamWaitEvent(ctx->s_run, ctx->ev_out[k], 0));
+        }
+        DART_CUDA(ctx, cudaMemcpyAsync(ctx->st_hidden[k], (const char *)hidden + b0 * in_row, nb * in_row,
+                                       cudaMemcpyHostToDevice, ctx->s_h2d));
+        if (keys)
+            DART_CUDA(ctx, cudaMemcpyAsync(ctx->st_keys[k], (const char *)keys + b0 * in_row, nb * in_row,
+                                           cudaMemcpyHostToDevice, ctx->s_h2d));
+        DART_CUDA(ctx, cudaEventRecord(ctx->ev_in[k], ctx->s_h2d));
+        DART_CUDA(ctx, cudaStreamWaitEvent(ctx->s_run, ctx->ev_in[k], 0));
+        rc = launch_staged(ctx, nb, ctx->st_hidden[k], keys ? ctx->st_keys[k] : nullptr, nullptr, vis_offset, n_vis,
+                           n_pivot, n_keep, ctx->st_out_hidden[k], ctx->st_out_idx[k], ctx->st_out_pos[k], o, nullptr,
+                           ctx->s_run);
+        if (rc != DART_OK) break;
+        DART_CUDA(ctx, cudaEventRecord(ctx->ev_run[k], ctx->s_run));
+        DART_CUDA(ctx, cudaStreamWaitEvent(ctx->s_d2h, ctx->ev_run[k], 0));
+        DART_CUDA(ctx, cudaMemcpyAsync((char *)out_hidden + b0 * out_row, ctx->st_out_hidden[k], nb * out_row,
+                                       cudaMemcpyDeviceToHost, ctx->s_d2h));
+        DART_CUDA(ctx, cudaMemcpyAsync(out_idx + (size_t)b0 * S_out, ctx->st_out_idx[k], (size_t)nb * S_out * 4,
+                                       cudaMemcpyDeviceToHost, ctx->s_d2h));
+        DART_CUDA(ctx, cudaMemcpyAsync(out_pos + (size_t)b0 * S_out, ctx->st_out_pos[k], (size_t)nb * S_out * 8,
+                                       cudaMemcpyDeviceToHost, ctx->s_d2h));
+        DART_CUDA(ctx, cudaEventRecord(ctx->ev_out[k], ctx->s_d2h));
+    }
+    cudaError_t e1 = cudaStreamSynchronize(ctx->s_h2d), e2 = cudaStreamSynchronize(ctx->s_run),
+                e3 = cudaStreamSynchronize(ctx->s_d2h);
+    if (rc != DART_OK) return rc;
+    DART_CUDA(ctx, e1);
+    DART_CUDA(ctx, e2);
+    DART_CUDA(ctx, e3);
+    return DART_OK;
+}
+
+int dart_status(dart_ctx *ctx)
+{
+    if (!ctx) return DART_ERR_NULL;
+    DeviceGuard g(ctx->desc.device);
+    if (!g.ok) return DART_ERR_CUDA;
+    int word = 0;
+    DART_CUDA(ctx, cudaDeviceSynchronize());
+    DART_CUDA(ctx, cudaMemcpy(&word, ctx->status, sizeof word, cudaMemcpyDeviceToHost));
+    if (word != 0) DART_CUDA(ctx, cudaMemset(ctx->status, 0, sizeof word));
+    return word;
+}
+
+int dart_last_cuda_error(const dart_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
+size_t dart_workspace_bytes(const dart_ctx *ctx) { return ctx ? ctx->bytes : 0; }
+int64_t dart_launch_count(const dart_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int dart_profile_enable(dart_ctx *ctx, int on)
+{
+    if (!ctx) return DART_ERR_NULL;
+    ctx->profiling = on != 0;
+    return DART_OK;
+}
+
+int dart_profile_read(dart_ctx *ctx, float *ms, int32_t *launches, const char **names, int *n_slots)
+{
+    if (!ctx || !ms || !launches || !n_slots) return DART_ERR_NULL;
+    DeviceGuard g(ctx->desc.device);
+    if (!g.ok) return DART_ERR_CUDA;
+    for (auto &e : ctx->pending) {
+        float t = 0.f;
+        DART_CUDA(ctx, cudaEventSynchronize(e.stop));
+        DART_CUDA(ctx, cudaEventElapsedTime(&t, e.start, e.stop));
+        ctx->slot_ms[e.slot] += t;
+        ctx->slot_launches[e.slot] += 1;
+        ctx->spare.push_back(e);
+    }
+    ctx->pending.clear();
+    int n = *n_slots < SLOT_COUNT ? *n_slots : SLOT_COUNT;
+    for (int k = 0; k < n; ++k) {
+        ms[k] = ctx->slot_ms[k];
+        launches[k] = ctx->slot_launches[k];
+        if (names) names[k] = kSlotNames[k];
+    }
+    for (int k = 0; k < SLOT_COUNT; ++k) {
+        ctx->slot_ms[k] = 0.f;
+        ctx->slot_launches[k] = 0;
+    }
+    *n_slots = n;
+    return DART_OK;
+}
+
+const char *dart_strerror(int code)
+{
+    switch (code) {
+    case DART_OK: return "ok";
+    case DART_ERR_NULL: return "a required pointer is NULL";
+    case DART_ERR_BAD_SHAPE: return "sizes violate the shape rules or exceed the context's maxima";
+    case DART_ERR_ALIGN: return "a tensor pointer is not sufficiently aligned";
+    case DART_ERR_ALIAS: return "an output overlaps an input";
+    case DART_ERR_CUDA: return "a CUDA call failed";
+    case DART_ERR_NOMEM: return "out of memory";
+    case DART_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    case DART_ERR_CHECK: return "a device-side self-check failed";
+    case DART_ERR_UNSUPPORTED: return "option not available";
+    default: return "unknown error code";
+    }
+}
+
+int dart_version(void) { return DART_VERSION; }
+
+} // extern "C"

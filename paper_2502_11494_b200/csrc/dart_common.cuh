@@ -1,0 +1,153 @@
+// Shared device helpers of the DART reduction kernels (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace dart {
+
+constexpr int kWarp = 32;
+
+// ---- memory access -------------------------------------------------------------------------
+// 128-bit read-only load that does not allocate in L1: every key/hidden byte is used once per sweep.
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// 128-bit streaming store (evict-first): packed rows are not read again by this library.
+__device__ __forceinline__ void st_stream(uint4 *p, uint4 v)
+{
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+// ---- bf16 pairs ----------------------------------------------------------------------------
+// A 32-bit word holds two bf16 values; each widens to fp32 by placing its 16 bits on top.
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// ---- order-preserving float keys --------------------------------------------------------------
+// Unsigned key whose order equals the float order (-0 and +0 are merged first so that they tie).
+__device__ __forceinline__ uint32_t order_key(float f)
+{
+    uint32_t u = __float_as_uint(f + 0.0f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float order_key_inv(uint32_t k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// ---- block-wide selection of the k smallest (key, index) pairs -----------------------------------
+// Radix select over 32-bit keys, 8 bits per pass, most significant first.  KeyFn(j, key&) returns
+// whether element j takes part and, if so, its key.  After the call every thread holds the same
+// threshold key T (the k-th smallest), the number `need_eq` of elements with key == T that belong to
+// the selection (those of lowest index) and the number `cnt_eq` of elements with key == T.
+struct SelectSmem {
+    uint32_t hist[256];
+    uint32_t warp_tot[32];
+    uint32_t bin, before, cnt;
+};
+
+template <typename KeyFn>
+__device__ void block_select_threshold(KeyFn keyfn, int n, uint32_t k, SelectSmem &sm, uint32_t &T,
+                                       uint32_t &need_eq, uint32_t &cnt_eq)
+{
+    uint32_t prefix = 0, mask = 0, remaining = k, cnt = 0;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) sm.hist[i] = 0;
+        __syncthreads();
+        for (int j = threadIdx.x; j < n; j += blockDim.x) {
+            uint32_t key;
+            if (keyfn(j, key) && (key & mask) == prefix) atomicAdd(&sm.hist[(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x < kWarp) {
+            // lane l owns bins [8l, 8l+8); find the bin where the running count reaches `remaining`
+            uint32_t c[8], s = 0;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                c[t] = sm.hist[threadIdx.x * 8 + t];
+                s += c[t];
+            }
+            uint32_t incl = s;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+                if ((int)threadIdx.x >= o) incl += v;
+            }
+            uint32_t excl = incl - s;
+            if (excl < remaining && remaining <= incl) {
+                uint32_t run = excl;
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    if (run < remaining && remaining <= run + c[t]) {
+                        sm.bin = threadIdx.x * 8 + t;
+                        sm.before = run;
+                        sm.cnt = c[t];
+                    }
+                    run += c[t];
+                }
+            }
+        }
+        __syncthreads();
+        prefix |= sm.bin << shift;
+        mask |= 255u << shift;
+        remaining -= sm.before;
+        cnt = sm.cnt;
+        __syncthreads();
+    }
+    T = prefix;
+    need_eq = remaining;
+    cnt_eq = cnt;
+}
+
+// Invoke pick(j, key) for every selected element: all with key < T, and the need_eq lowest-index
+// elements with key == T.  Block-uniform control flow; ends with a __syncthreads().
+template <typename KeyFn, typename PickFn>
+__device__ void block_select_apply(KeyFn keyfn, int n, uint32_t T, uint32_t need_eq, uint32_t cnt_eq,
+                                   SelectSmem &sm, PickFn pick)
+{
+    const bool all_eq = (need_eq == cnt_eq);
+    for (int j = threadIdx.x; j < n; j += blockDim.x) {
+        uint32_t key;
+        if (keyfn(j, key) && (key < T || (all_eq && key == T))) pick(j, key);
+    }
+    if (!all_eq) {
+        // ties at the threshold: walk the indices in order and take the first need_eq
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+        uint32_t base = 0;
+        for (int start = 0; start < n && base < need_eq; start += blockDim.x) {
+            int j = start + threadIdx.x;
+            uint32_t key = 0;
+            bool f = (j < n) && keyfn(j, key) && key == T;
+            uint32_t bal = __ballot_sync(0xffffffffu, f);
+            if (lane == 0) sm.warp_tot[warp] = __popc(bal);
+            __syncthreads();
+            uint32_t before = 0, total = 0;
+            for (int w = 0; w < nwarp; ++w) {
+                uint32_t t = sm.warp_tot[w];
+                if (w < warp) before += t;
+                total += t;
+            }
+            uint32_t rank = base + before + __popc(bal & ((1u << lane) - 1u));
+            if (f && rank < need_eq) pick(j, key);
+            base += total;
+            __syncthreads();
+        }
+    }
+    __syncthreads();
+}
+
+} // namespace dart

@@ -1,0 +1,305 @@
+// Staged path: one kernel per step of the reduction (Sec. 3.3 of the paper), every intermediate
+// in the context's workspace.  It is the plain realisation of the method and the path that
+// materialises the per-step outputs.
+#pragma once
+#include "dart_common.cuh"
+
+namespace dart {
+
+// ------------------------------------------------------------------------------------------------
+// Step 1: scores.  One warp per vision token: l1 = sum |k| (the "K-norm" of the Sec. 3.3 footnote),
+// ssq = sum k^2 (the squared Euclidean norm in Eq. 7's denominator).  fp32 accumulation, fixed
+// order: each lane sums its column groups in order, then a butterfly over the lanes.
+// ------------------------------------------------------------------------------------------------
+constexpr int kScoreWarps = 8;
+
+__global__ void __launch_bounds__(kScoreWarps * 32)
+score_kernel(const uint4 *__restrict__ keys, int S, int d8, int vis_offset, int n_vis, long long rows_total,
+             float *__restrict__ l1, float *__restrict__ ssq)
+{
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * kScoreWarps + (threadIdx.x >> 5);
+    if (row >= rows_total) return;
+    const int b = (int)(row / n_vis), j = (int)(row % n_vis);
+    const uint4 *src = keys + ((size_t)b * S + vis_offset + j) * (size_t)d8;
+    float a = 0.f, q = 0.f;
+    for (int c0 = 0; c0 < d8; c0 += 32 * 8) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            int c = c0 + u * 32 + lane;
+            v[u] = (c < d8) ? ld_stream(src + c) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                float lo = bf16_lo(w[t]), hi = bf16_hi(w[t]);
+                a += fabsf(lo);
+                a += fabsf(hi);
+                q = fmaf(lo, lo, q);
+                q = fmaf(hi, hi, q);
+            }
+        }
+    }
+    a = warp_sum(a);
+    q = warp_sum(q);
+    if (lane == 0) {
+        l1[row] = a;
+        ssq[row] = q;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Step 2: pivots (Def. 1; maximum K-norm per the caption of Table 1).  One CTA per sample: radix
+// select of the P best scores, then a bitonic sort of the P (key, index) pairs into rank order.
+// Dynamic shared memory: P_pad * 8 bytes, P_pad = next power of two >= P.
+// ------------------------------------------------------------------------------------------------
+constexpr int kSelectThreads = 512;
+
+__global__ void __launch_bounds__(kSelectThreads)
+pivot_kernel(const float *__restrict__ score, int n_vis, int P, int P_pad, int smallest,
+             int32_t *__restrict__ pivot_idx)
+{
+    extern __shared__ unsigned long long piv_list[]; // [P_pad]
+    __shared__ SelectSmem sel;
+    __shared__ uint32_t n_picked;
+    const int b = blockIdx.x;
+    const float *s = score + (size_t)b * n_vis;
+    // smaller key = better pivot
+    auto keyfn = [&](int j, uint32_t &key) {
+        uint32_t k = order_key(s[j]);
+        key = smallest ? k : ~k;
+        return true;
+    };
+    for (int i = threadIdx.x; i < P_pad; i += blockDim.x) piv_list[i] = ~0ull;
+    if (threadIdx.x == 0) n_picked = 0;
+    uint32_t T, need_eq, cnt_eq;
+    block_select_threshold(keyfn, n_vis, (uint32_t)P, sel, T, need_eq, cnt_eq);
+    block_select_apply(keyfn, n_vis, T, need_eq, cnt_eq, sel, [&](int j, uint32_t key) {
+        uint32_t slot = atomicAdd(&n_picked, 1u);
+        piv_list[slot] = ((unsigned long long)key << 32) | (uint32_t)j;
+    });
+    // ascending bitonic sort of (key, index): rank 0 = best score, ties to the lower index
+    for (int k = 2; k <= P_pad; k <<= 1) {
+        for (int jj = k >> 1; jj > 0; jj >>= 1) {
+            for (int i = threadIdx.x; i < P_pad; i += blockDim.x) {
+                int l = i ^ jj;
+                if (l > i) {
+                    unsigned long long x = piv_list[i], y = piv_list[l];
+                    bool up = ((i & k) == 0);
+                    if ((x > y) == up) {
+                        piv_list[i] = y;
+                        piv_list[l] = x;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    for (int i = threadIdx.x; i < P; i += blockDim.x)
+        pivot_idx[(size_t)b * P + i] = (int32_t)(piv_list[i] & 0xffffffffu);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Step 3 on the CUDA cores: dup[i][j] = (K_{p_i} . K_j) / (|K_{p_i}| |K_j|)  (Def. 2, Eq. 7).
+// A CTA stages up to 8 pivot rows in shared memory and streams a tile of token rows against them,
+// 4 rows per warp at a time so that each pivot value read from shared memory feeds 4 FMAs.
+// Dynamic shared memory: 8 * d8 * 16 bytes.
+// ------------------------------------------------------------------------------------------------
+constexpr int kSimWarps = 8;
+constexpr int kSimRowsPerWarp = 4;
+constexpr int kSimPivotChunk = 8;
+constexpr int kSimRowsPerCta = 64;
+
+__global__ void __launch_bounds__(kSimWarps * 32)
+sim_alu_kernel(const uint4 *__restrict__ keys, int S, int d8, int vis_offset, int n_vis, int P, int p0,
+               const int32_t *__restrict__ pivot_idx, const float *__restrict__ ssq, float *__restrict__ sim)
+{
+    extern __shared__ uint4 piv_rows[]; // [kSimPivotChunk][d8]
+    const int b = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint4 *base = keys + ((size_t)b * S + vis_offset) * (size_t)d8;
+    const int np = min(kSimPivotChunk, P - p0);
+    for (int i = threadIdx.x; i < kSimPivotChunk * d8; i += blockDim.x) {
+        int p = i / d8, c = i - p * d8;
+        piv_rows[i] = (p < np) ? __ldg(base + (size_t)pivot_idx[(size_t)b * P + p0 + p] * d8 + c)
+                               : make_uint4(0, 0, 0, 0);
+    }
+    __syncthreads();
+    const int tile0 = blockIdx.x * kSimRowsPerCta;
+    for (int r0 = tile0 + warp * kSimRowsPerWarp; r0 < min(tile0 + kSimRowsPerCta, n_vis);
+         r0 += kSimWarps * kSimRowsPerWarp) {
+        float acc[kSimRowsPerWarp][kSimPivotChunk];
+#pragma unroll
+        for (int r = 0; r < kSimRowsPerWarp; ++r)
+#pragma unroll
+            for (int p = 0; p < kSimPivotChunk; ++p) acc[r][p] = 0.f;
+        for (int c = lane; c < d8; c += 32) {
+            float x[kSimRowsPerWarp][8];
+#pragma unroll
+            for (int r = 0; r < kSimRowsPerWarp; ++r) {
+                int row = min(r0 + r, n_vis - 1);
+                uint4 v = ld_stream(base + (size_t)row * d8 + c);
+                x[r][0] = bf16_lo(v.x), x[r][1] = bf16_hi(v.x), x[r][2] = bf16_lo(v.y), x[r][3] = bf16_hi(v.y);
+                x[r][4] = bf16_lo(v.z), x[r][5] = bf16_hi(v.z), x[r][6] = bf16_lo(v.w), x[r][7] = bf16_hi(v.w);
+            }
+#pragma unroll
+            for (int p = 0; p < kSimPivotChunk; ++p) {
+                uint4 w = piv_rows[p * d8 + c];
+                float y[8] = {bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y),
+                              bf16_lo(w.z), bf16_hi(w.z), bf16_lo(w.w), bf16_hi(w.w)};
+#pragma unroll
+                for (int r = 0; r < kSimRowsPerWarp; ++r)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[r][p] = fmaf(x[r][e], y[e], acc[r][p]);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < kSimRowsPerWarp; ++r)
+#pragma unroll
+            for (int p = 0; p < kSimPivotChunk; ++p) acc[r][p] = warp_sum(acc[r][p]);
+        if (lane == 0) {
+#pragma unroll
+            for (int r = 0; r < kSimRowsPerWarp; ++r) {
+                int row = r0 + r;
+                if (row >= n_vis) break;
+                float nj = sqrtf(ssq[(size_t)b * n_vis + row]);
+#pragma unroll
+                for (int p = 0; p < kSimPivotChunk; ++p) {
+                    if (p >= np) break;
+                    float np_ = sqrtf(ssq[(size_t)b * n_vis + pivot_idx[(size_t)b * P + p0 + p]]);
+                    float den = np_ * nj;
+                    sim[((size_t)b * P + p0 + p) * n_vis + row] = den > 0.f ? acc[r][p] / den : 0.f;
+                }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Steps 4 and 5a: retention (Eq. 9-10) and the packed index list.  One CTA per sample.
+// kept := pivots; pivot i in rank order selects its q_i not-yet-kept tokens of lowest dup (radix
+// select on order-preserving keys, ties to the lower index); eps_i is the selection threshold.
+// Then an ordered scan over the keep flags writes the ascending kept indices and position ids.
+// Dynamic shared memory: n_vis bytes (keep flags).
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kSelectThreads)
+retain_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx, const int64_t *__restrict__ pos_in,
+              int S, int vis_offset, int n_vis, int P, int n_keep,
+              int32_t *__restrict__ out_idx, int64_t *__restrict__ out_pos,
+              uint8_t *__restrict__ keep_out, int32_t *__restrict__ owner_out, float *__restrict__ eps_out)
+{
+    extern __shared__ uint8_t keep[]; // [n_vis]
+    __shared__ SelectSmem sel;
+    const int b = blockIdx.x;
+    const int S_out = S - n_vis + n_keep;
+    int32_t *owner = owner_out ? owner_out + (size_t)b * n_vis : nullptr;
+    for (int j = threadIdx.x; j < n_vis; j += blockDim.x) {
+        keep[j] = 0;
+        if (owner) owner[j] = -1;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < P; i += blockDim.x) {
+        int p = pivot_idx[(size_t)b * P + i];
+        keep[p] = 1;
+        if (owner) owner[p] = P + i;
+    }
+    __syncthreads();
+    const int q = (n_keep - P) / P, r = (n_keep - P) % P;
+    for (int i = 0; i < P; ++i) {
+        const int qi = q + (i < r ? 1 : 0);
+        if (qi == 0) {
+            if (eps_out && threadIdx.x == 0) eps_out[(size_t)b * P + i] = __int_as_float(0x7fc00000);
+            continue;
+        }
+        const float *row = sim + ((size_t)b * P + i) * n_vis;
+        auto keyfn = [&](int j, uint32_t &key) {
+            if (keep[j]) return false;
+            key = order_key(row[j]);
+            return true;
+        };
+        uint32_t T, need_eq, cnt_eq;
+        block_select_threshold(keyfn, n_vis, (uint32_t)qi, sel, T, need_eq, cnt_eq);
+        // picks only flip flags of elements that stay selected, so keyfn may run while others pick:
+        // an element picked by another thread is never examined again by this round's owner thread
+        block_select_apply(keyfn, n_vis, T, need_eq, cnt_eq, sel, [&](int j, uint32_t) {
+            keep[j] = 1;
+            if (owner) owner[j] = i;
+        });
+        if (eps_out && threadIdx.x == 0) eps_out[(size_t)b * P + i] = order_key_inv(T);
+    }
+    // packed index list: text before, kept vision tokens in ascending order, text after
+    int32_t *oi = out_idx + (size_t)b * S_out;
+    int64_t *op = out_pos + (size_t)b * S_out;
+    const int64_t *pin = pos_in ? pos_in + (size_t)b * S : nullptr;
+    for (int t = threadIdx.x; t < vis_offset; t += blockDim.x) {
+        oi[t] = t;
+        op[t] = pin ? pin[t] : (int64_t)t;
+    }
+    const int n_after = S - vis_offset - n_vis;
+    for (int t = threadIdx.x; t < n_after; t += blockDim.x) {
+        int s = vis_offset + n_vis + t;
+        oi[vis_offset + n_keep + t] = s;
+        op[vis_offset + n_keep + t] = pin ? pin[s] : (int64_t)s;
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    uint32_t base = 0;
+    for (int start = 0; start < n_vis; start += blockDim.x) {
+        int j = start + threadIdx.x;
+        bool f = (j < n_vis) && keep[j];
+        uint32_t bal = __ballot_sync(0xffffffffu, f);
+        if (lane == 0) sel.warp_tot[warp] = __popc(bal);
+        __syncthreads();
+        uint32_t before = 0, total = 0;
+        for (int w = 0; w < nwarp; ++w) {
+            uint32_t t = sel.warp_tot[w];
+            if (w < warp) before += t;
+            total += t;
+        }
+        if (f) {
+            uint32_t t = vis_offset + base + before + __popc(bal & ((1u << lane) - 1u));
+            int s = vis_offset + j;
+            oi[t] = s;
+            op[t] = pin ? pin[s] : (int64_t)s;
+        }
+        base += total;
+        __syncthreads();
+    }
+    if (keep_out)
+        for (int j = threadIdx.x; j < n_vis; j += blockDim.x) keep_out[(size_t)b * n_vis + j] = keep[j];
+}
+
+// ------------------------------------------------------------------------------------------------
+// Step 5b: gather the kept hidden rows into the packed sequence.  One warp per output row,
+// 128-bit loads and streaming stores, 8 loads in flight per lane.
+// ------------------------------------------------------------------------------------------------
+constexpr int kGatherWarps = 8;
+
+__global__ void __launch_bounds__(kGatherWarps * 32)
+gather_kernel(const uint4 *__restrict__ hidden, const int32_t *__restrict__ out_idx, int S, int S_out, int d8,
+              long long rows_total, uint4 *__restrict__ out_hidden)
+{
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * kGatherWarps + (threadIdx.x >> 5);
+    if (row >= rows_total) return;
+    const int b = (int)(row / S_out);
+    const int s = out_idx[row];
+    const uint4 *src = hidden + ((size_t)b * S + s) * (size_t)d8;
+    uint4 *dst = out_hidden + (size_t)row * (size_t)d8;
+    for (int c0 = 0; c0 < d8; c0 += 32 * 8) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            int c = c0 + u * 32 + lane;
+            if (c < d8) v[u] = ld_stream(src + c);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            int c = c0 + u * 32 + lane;
+            if (c < d8) st_stream(dst + c, v[u]);
+        }
+    }
+}
+
+} // namespace dart
