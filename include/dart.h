@@ -171,6 +171,34 @@ int64_t dart_launch_count(const dart_ctx *ctx);
 int dart_profile_enable(dart_ctx *ctx, int on);
 int dart_profile_read(dart_ctx *ctx, float *ms, int32_t *launches, const char **names, int *n_slots);
 
+/*
+ * Pivot selection without any allocation (the paper has no counterpart of this entry point; it
+ * exists for deployment, not for the method).
+ *
+ * Some hosts of this library cannot call cudaMalloc when the step runs: serving engines that hand
+ * the whole HBM to their own pool at start-up (a later cudaMalloc simply fails), and latency-bound
+ * loops that cannot afford cudaMalloc's device-wide synchronisation.  dart_create allocates, so a
+ * context is out of reach for them.  This call needs no context: it computes steps 1-2 of
+ * dart_reduce (row scores, then the n_pivot best vision tokens per sample in rank order, L1 score,
+ * largest first, ties to the lower index) and keeps the per-row scores, its only scratch, in a
+ * fixed array that is part of the library image: DART_STATIC_MAX_ROWS rows, 2 MiB, resident on
+ * every GPU that loads the library until the process exits.
+ *
+ *   keys       [B, S, d] bf16, device, 16-byte aligned, read-only
+ *   pivot_idx  [B, n_pivot] int32, device: vision-relative indices, rank 0 first (the output)
+ *   device     CUDA device ordinal the pointers belong to;  stream: a cudaStream_t on that device
+ * Limits: B * n_vis <= DART_STATIC_MAX_ROWS and n_pivot <= 1024, else DART_ERR_BAD_SHAPE; d % 8 == 0;
+ * 1 <= n_pivot <= n_vis; vis_offset + n_vis <= S.
+ * The first call on a device looks up the array's device address (no allocation); make that call
+ * before any stream capture begins.  Every call on a device uses the same array and leaves its
+ * scores there: nothing in it has to start at zero (each call overwrites the rows it reads), but
+ * two calls whose kernels overlap on the GPU, from different streams or threads, race on it.
+ * Calls cudaMalloc, cudaFree or an allocating routine never.  Errors: NULL, BAD_SHAPE, ALIGN, CUDA.
+ */
+#define DART_STATIC_MAX_ROWS 262144
+int dart_pivots_static(const void *keys, int B, int S, int d, int vis_offset, int n_vis, int n_pivot,
+                       int32_t *pivot_idx, int device, void *stream);
+
 const char *dart_strerror(int code);
 int dart_version(void);
 

@@ -3,6 +3,7 @@
 
 #include <cuda_runtime.h>
 
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -444,6 +445,50 @@ int dart_profile_read(dart_ctx *ctx, float *ms, int32_t *launches, const char **
     }
     *n_slots = n;
     return DART_OK;
+}
+
+// ---- allocation-free pivot selection ---------------------------------------------------------------
+// Scratch of dart_pivots_static: L1 scores in the first half, sums of squares in the second.  The
+// name below is only a host-side handle; kernels get the address cudaGetSymbolAddress returns.
+static __device__ __align__(256) float g_static_scores[2 * DART_STATIC_MAX_ROWS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float *g_static_ptr[kMaxDevices]; // device address of g_static_scores, per device; looked up once
+std::mutex g_static_mutex;
+} // namespace
+
+int dart_pivots_static(const void *keys, int B, int S, int d, int vis_offset, int n_vis, int n_pivot,
+                       int32_t *pivot_idx, int device, void *stream)
+{
+    if (!keys || !pivot_idx) return DART_ERR_NULL;
+    if (B < 1 || S < 1 || d < 8 || d % 8 != 0 || vis_offset < 0 || n_vis < 1 || (long long)vis_offset + n_vis > S)
+        return DART_ERR_BAD_SHAPE;
+    if (n_pivot < 1 || n_pivot > n_vis || n_pivot > 1024) return DART_ERR_BAD_SHAPE;
+    if ((long long)B * n_vis > DART_STATIC_MAX_ROWS) return DART_ERR_BAD_SHAPE; // beyond the fixed scratch
+    if (((uintptr_t)keys & 15u) || ((uintptr_t)pivot_idx & 3u)) return DART_ERR_ALIGN;
+    if (device < 0 || device >= kMaxDevices) return DART_ERR_CUDA;
+    DeviceGuard g(device);
+    if (!g.ok) return DART_ERR_CUDA;
+    float *scratch;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[device]) { // set-up, once per device, with that device current
+            float *ptr = nullptr;
+            if (cudaGetSymbolAddress((void **)&ptr, g_static_scores) != cudaSuccess || !ptr) return DART_ERR_CUDA;
+            g_static_ptr[device] = ptr;
+        }
+        scratch = g_static_ptr[device];
+    }
+    using namespace dart;
+    cudaStream_t st = (cudaStream_t)stream;
+    const long long rows = (long long)B * n_vis;
+    float *l1 = scratch, *ssq = scratch + DART_STATIC_MAX_ROWS;
+    score_kernel<<<(unsigned)((rows + kScoreWarps - 1) / kScoreWarps), kScoreWarps * 32, 0, st>>>(
+        (const uint4 *)keys, S, d / 8, vis_offset, n_vis, rows, l1, ssq);
+    const int P_pad = next_pow2(n_pivot);
+    pivot_kernel<<<B, kSelectThreads, (size_t)P_pad * 8, st>>>(l1, n_vis, n_pivot, P_pad, 0, pivot_idx);
+    return cudaGetLastError() == cudaSuccess ? DART_OK : DART_ERR_CUDA;
 }
 
 const char *dart_strerror(int code)

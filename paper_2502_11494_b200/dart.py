@@ -23,8 +23,9 @@ DART_PATH_AUTO, DART_PATH_STAGED, DART_PATH_FUSED = 0, 1, 2
 EXPORTS = (
     "dart_create", "dart_destroy", "dart_set_shape", "dart_reduce", "dart_reduce_ex", "dart_reduce_host",
     "dart_status", "dart_last_cuda_error", "dart_workspace_bytes", "dart_launch_count",
-    "dart_profile_enable", "dart_profile_read", "dart_strerror", "dart_version",
+    "dart_profile_enable", "dart_profile_read", "dart_strerror", "dart_version", "dart_pivots_static",
 )
+DART_STATIC_MAX_ROWS = 262144
 
 
 class dart_desc(ctypes.Structure):
@@ -78,6 +79,7 @@ def lib() -> ctypes.CDLL:
         L.dart_profile_enable.argtypes = [vp, i32]
         L.dart_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32),
                                         ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_int)]
+        L.dart_pivots_static.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32p, i32, vp]
         L.dart_strerror.argtypes = [i32]
         L.dart_strerror.restype = ctypes.c_char_p
         L.dart_version.argtypes = []
@@ -124,6 +126,11 @@ def dart_reduce_ex(ctx, hidden, keys, pos_in, vis_offset, n_vis, n_pivot, n_keep
 
 def dart_reduce_host(ctx, hidden, keys, vis_offset, n_vis, n_pivot, n_keep, out_hidden, out_idx, out_pos) -> int:
     return lib().dart_reduce_host(ctx, hidden, keys, vis_offset, n_vis, n_pivot, n_keep, out_hidden, out_idx, out_pos)
+
+
+def dart_pivots_static(keys, B, S, d, vis_offset, n_vis, n_pivot, pivot_idx, device, stream) -> int:
+    """Context-free, allocation-free pivot selection (raw device pointers); see include/dart.h."""
+    return lib().dart_pivots_static(keys, B, S, d, vis_offset, n_vis, n_pivot, pivot_idx, device, stream)
 
 
 def dart_status(ctx) -> int:
