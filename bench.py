@@ -41,6 +41,7 @@ def parse():
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch size")
     ap.add_argument("--sweep", action="store_true", help="also time every (pivots, keep) cell of the sweep")
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 staged, 2 fused")
+    ap.add_argument("--lag", type=int, default=0, help="fused path: extra tasks between a row's two sweeps")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -73,6 +74,7 @@ def kernel_bytes_per_launch(name, w, B):
         "score": keys + 8 * w.n_vis * B,
         "sim": keys + 4 * w.n_pivot * w.n_vis * B,
         "sweep": keys,                       # fused scores + pivots + similarities: the keys count once
+        "finalize": 4 * w.n_pivot * w.n_vis * B,
         "gather": 2 * (2 * w.d * w.S_out) * B,
         "pivot": 4 * w.n_vis * B,
         "retain": 4 * w.n_pivot * w.n_vis * B + 12 * w.S_out * B,
@@ -257,7 +259,7 @@ def main():
     ctx = dart.Dart(B, w.S, w.d, max(w.n_pivot, max(W.SWEEP_PIVOTS) if args.sweep else 0),
                     max(w.n_keep, max(W.SWEEP_KEEP) if args.sweep else 0), device=local, flags=flags)
     dart.dart_set_shape(ctx.handle, B, w.S)
-    opts = dart.dart_opts(0, 0, args.path, 0)
+    opts = dart.dart_opts(0, 0, args.path, 0, args.lag)
 
     def alloc_outs(wl):
         return (torch.empty((B, wl.S_out, wl.d), dtype=torch.bfloat16, device=dev),

@@ -52,7 +52,8 @@ enum {
 /* dart_opts.path */
 #define DART_PATH_AUTO 0
 #define DART_PATH_STAGED 1 /* one kernel per step of the method, every intermediate in the workspace */
-#define DART_PATH_FUSED 2  /* persistent sweep kernel (scores, pivots and similarities in one launch) */
+#define DART_PATH_FUSED 2  /* persistent sweep kernel (scores, pivots and similarities in one launch); needs
+                              d % 64 == 0 and n_pivot <= 256, else UNSUPPORTED.  AUTO picks it when it applies. */
 
 typedef struct dart_ctx dart_ctx; /* opaque: workspace, device status word, profiling events */
 
@@ -72,7 +73,8 @@ typedef struct {
     int32_t norm_kind;     /* 0 or 1: L1 row norm (the paper's "K-norm", Sec. 3.3 footnote); 2: Euclidean norm */
     int32_t pivot_smallest; /* 0: pivots = largest scores (Table 1 caption); 1: smallest (ablation variant) */
     int32_t path;          /* DART_PATH_* */
-    int32_t wait_limit;    /* 0: default; > 0: iteration limit of bounded device-side waits (testing) */
+    int32_t wait_limit;    /* 0: default (2 s); > 0: time limit in microseconds of every bounded device-side wait */
+    int32_t sweep_lag;     /* 0: default; > 0: fused path, extra tasks between a row's two sweeps (tuning) */
 } dart_opts;
 
 /* Optional per-step outputs of dart_reduce_ex; every member is a device pointer or NULL. */

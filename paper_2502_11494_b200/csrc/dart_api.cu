@@ -8,11 +8,16 @@
 #include <vector>
 
 #include "dart_staged.cuh"
+#include "dart_sweep.cuh"
 
 namespace {
 
-enum Slot { SLOT_SCORE = 0, SLOT_PIVOT, SLOT_SIM, SLOT_RETAIN, SLOT_GATHER, SLOT_COUNT };
-const char *const kSlotNames[SLOT_COUNT] = {"score", "pivot", "sim", "retain", "gather"};
+enum Slot { SLOT_SCORE = 0, SLOT_PIVOT, SLOT_SIM, SLOT_RETAIN, SLOT_GATHER, SLOT_SWEEP, SLOT_FINALIZE, SLOT_COUNT };
+const char *const kSlotNames[SLOT_COUNT] = {"score", "pivot", "sim", "retain", "gather", "sweep", "finalize"};
+
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                      const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 struct EventPair {
     cudaEvent_t start, stop;
@@ -45,6 +50,14 @@ struct dart_ctx {
     int64_t *st_out_pos[2];
     cudaStream_t s_h2d, s_run, s_d2h;
     cudaEvent_t ev_in[2], ev_run[2], ev_out[2];
+    // fused path (csrc/dart_sweep.cuh); available when d is a multiple of 64 and the device is sm_100
+    bool fused_ok;
+    int sm_count, KS, n_atoms, N_max;
+    float *pl1, *pssq, *psim;
+    uint4 *pivK;
+    int *counters;
+    size_t counters_bytes;
+    TensorMapEncodeFn encode;
 };
 
 namespace {
@@ -147,6 +160,22 @@ int check_call(const dart_ctx *ctx, const void *hidden, const void *keys, int vi
     return DART_OK;
 }
 
+int copy_debug(dart_ctx *ctx, int B, int n_vis, int P, const dart_debug *dbg, cudaStream_t st)
+{
+    if (dbg) {
+        const size_t nv = (size_t)B * n_vis, np = (size_t)B * P;
+        if (dbg->l1) DART_CUDA(ctx, cudaMemcpyAsync(dbg->l1, ctx->l1, nv * 4, cudaMemcpyDeviceToDevice, st));
+        if (dbg->ssq) DART_CUDA(ctx, cudaMemcpyAsync(dbg->ssq, ctx->ssq, nv * 4, cudaMemcpyDeviceToDevice, st));
+        if (dbg->pivot_idx)
+            DART_CUDA(ctx, cudaMemcpyAsync(dbg->pivot_idx, ctx->pivot_idx, np * 4, cudaMemcpyDeviceToDevice, st));
+        if (dbg->sim) DART_CUDA(ctx, cudaMemcpyAsync(dbg->sim, ctx->sim, np * n_vis * 4, cudaMemcpyDeviceToDevice, st));
+        if (dbg->eps) DART_CUDA(ctx, cudaMemcpyAsync(dbg->eps, ctx->eps, np * 4, cudaMemcpyDeviceToDevice, st));
+        if (dbg->keep) DART_CUDA(ctx, cudaMemcpyAsync(dbg->keep, ctx->keep, nv, cudaMemcpyDeviceToDevice, st));
+        if (dbg->owner) DART_CUDA(ctx, cudaMemcpyAsync(dbg->owner, ctx->owner, nv * 4, cudaMemcpyDeviceToDevice, st));
+    }
+    return DART_OK;
+}
+
 int launch_staged(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, const int64_t *pos_in, int vis_offset,
                   int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos,
                   const dart_opts &o, const dart_debug *dbg, cudaStream_t st)
@@ -189,18 +218,139 @@ int launch_staged(dart_ctx *ctx, int B, const void *hidden, const void *keys_in,
                                                          (uint4 *)out_hidden);
     }
     DART_CUDA(ctx, cudaGetLastError());
-    if (dbg) {
-        const size_t nv = (size_t)B * n_vis, np = (size_t)B * P;
-        if (dbg->l1) DART_CUDA(ctx, cudaMemcpyAsync(dbg->l1, ctx->l1, nv * 4, cudaMemcpyDeviceToDevice, st));
-        if (dbg->ssq) DART_CUDA(ctx, cudaMemcpyAsync(dbg->ssq, ctx->ssq, nv * 4, cudaMemcpyDeviceToDevice, st));
-        if (dbg->pivot_idx)
-            DART_CUDA(ctx, cudaMemcpyAsync(dbg->pivot_idx, ctx->pivot_idx, np * 4, cudaMemcpyDeviceToDevice, st));
-        if (dbg->sim) DART_CUDA(ctx, cudaMemcpyAsync(dbg->sim, ctx->sim, np * n_vis * 4, cudaMemcpyDeviceToDevice, st));
-        if (dbg->eps) DART_CUDA(ctx, cudaMemcpyAsync(dbg->eps, ctx->eps, np * 4, cudaMemcpyDeviceToDevice, st));
-        if (dbg->keep) DART_CUDA(ctx, cudaMemcpyAsync(dbg->keep, ctx->keep, nv, cudaMemcpyDeviceToDevice, st));
-        if (dbg->owner) DART_CUDA(ctx, cudaMemcpyAsync(dbg->owner, ctx->owner, nv * 4, cudaMemcpyDeviceToDevice, st));
+    return copy_debug(ctx, B, n_vis, P, dbg, st);
+}
+
+// ---- fused path ------------------------------------------------------------------------------------
+int fused_setup(dart_ctx *ctx)
+{
+    using namespace dart::sweep;
+    const dart_desc &D = ctx->desc;
+    ctx->fused_ok = false;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, D.device) != cudaSuccess) return DART_ERR_CUDA;
+    ctx->sm_count = prop.multiProcessorCount;
+    if (prop.major != 10 || D.d % kAtomCols != 0 || !prop.cooperativeLaunch) return DART_OK; // staged path only
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
+        q != cudaDriverEntryPointSuccess)
+        return DART_OK;
+    ctx->encode = (TensorMapEncodeFn)fn;
+    ctx->n_atoms = D.d / kAtomCols;
+    ctx->KS = (ctx->n_atoms + kSlabAtoms - 1) / kSlabAtoms;
+    const int P_cap = D.P_max < kMaxN ? D.P_max : kMaxN;
+    ctx->N_max = (P_cap + 15) / 16 * 16;
+    const size_t nv = (size_t)D.B_max * D.S_max;
+    const int n_rt_max = (D.S_max + kTileRows - 1) / kTileRows;
+    int rc = ws_alloc(ctx, &ctx->pl1, nv * ctx->KS);
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->pssq, nv * ctx->KS);
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->psim, nv * ctx->KS * P_cap);
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->pivK, (size_t)D.B_max * ctx->N_max * (D.d / 8));
+    ctx->counters_bytes = (size_t)D.B_max * (n_rt_max + 2) * sizeof(int);
+    if (rc == DART_OK) rc = ws_alloc(ctx, (uint8_t **)&ctx->counters, ctx->counters_bytes);
+    if (rc != DART_OK) return rc;
+    // rows of the gathered-pivot blocks beyond the pivot count are read by the MMA and must stay finite
+    if (cudaMemset(ctx->pivK, 0, (size_t)D.B_max * ctx->N_max * (D.d / 8) * 16) != cudaSuccess) return DART_ERR_CUDA;
+    if (cudaFuncSetAttribute(sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - 8192) !=
+        cudaSuccess)
+        return DART_ERR_CUDA;
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sweep_kernel, kThreads,
+                                                      smem_bytes(16, ring_depth(16, ctx->max_smem_optin))) != cudaSuccess ||
+        per_sm < 1)
+        return DART_ERR_CUDA;
+    ctx->fused_ok = true;
+    return DART_OK;
+}
+
+int encode_2d(dart_ctx *ctx, CUtensorMap *tm, const void *base, uint64_t cols, uint64_t rows, uint32_t box_rows)
+{
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)dart::sweep::kAtomCols, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = ctx->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        ctx->last_cuda = (int)r;
+        return DART_ERR_CUDA;
     }
     return DART_OK;
+}
+
+bool fused_applies(const dart_ctx *ctx, int P) { return ctx->fused_ok && P <= dart::sweep::kMaxN; }
+
+int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, const int64_t *pos_in, int vis_offset,
+                 int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos, const dart_opts &o,
+                 const dart_debug *dbg, cudaStream_t st)
+{
+    using namespace dart;
+    using namespace dart::sweep;
+    const int S = ctx->S, d8 = ctx->desc.d / 8, S_out = S - n_vis + n_keep;
+    const void *keys = keys_in ? keys_in : hidden;
+    Params p = {};
+    p.B = B, p.S = S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.N = (P + 15) / 16 * 16, p.d8 = d8;
+    p.n_atoms = ctx->n_atoms, p.KS = ctx->KS, p.n_rt = (n_vis + kTileRows - 1) / kTileRows, p.T = p.n_rt * p.KS;
+    p.n_stages = ring_depth(p.N, ctx->max_smem_optin);
+    if (p.n_stages < 2) return DART_ERR_UNSUPPORTED;
+    const long long n_all = (long long)B * p.T;
+    // a row's second sweep follows its first by one sample plus the time the pivots take to appear
+    long long lag = (long long)p.T + (o.sweep_lag > 0 ? o.sweep_lag : 3 * ctx->sm_count);
+    p.lag = lag < n_all ? lag : n_all;
+    p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest;
+    p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
+    p.keys = (const uint4 *)keys;
+    p.pl1 = ctx->pl1, p.pssq = ctx->pssq, p.psim = ctx->psim, p.l1 = ctx->l1, p.ssq = ctx->ssq;
+    p.pivot_idx = ctx->pivot_idx, p.pivK = ctx->pivK;
+    p.rt_done = ctx->counters, p.s1_done = ctx->counters + (size_t)B * p.n_rt, p.piv_ready = p.s1_done + B;
+    p.status = ctx->status;
+    CUtensorMap tm_keys, tm_piv;
+    int rc = encode_2d(ctx, &tm_keys, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, kSubRows);
+    if (rc == DART_OK) rc = encode_2d(ctx, &tm_piv, ctx->pivK, (uint64_t)ctx->desc.d, (uint64_t)B * p.N, (uint32_t)p.N);
+    if (rc != DART_OK) return rc;
+    DART_CUDA(ctx, cudaMemsetAsync(ctx->counters, 0, (size_t)B * (p.n_rt + 2) * sizeof(int), st));
+    {
+        Prof pr(ctx, st, SLOT_SWEEP);
+        long long grid = 2 * n_all < ctx->sm_count ? 2 * n_all : ctx->sm_count;
+        void *args[3] = {&tm_keys, &tm_piv, &p};
+        DART_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)sweep_kernel, dim3((unsigned)grid), dim3(kThreads), args,
+                                                   smem_bytes(p.N, p.n_stages), st));
+    }
+    {
+        Prof pr(ctx, st, SLOT_FINALIZE);
+        dim3 grid((n_vis + kFinalizeThreads - 1) / kFinalizeThreads, B);
+        finalize_sim_kernel<<<grid, kFinalizeThreads, 0, st>>>(ctx->psim, ctx->ssq, ctx->pivot_idx, n_vis, P, p.KS,
+                                                               ctx->sim);
+    }
+    {
+        Prof pr(ctx, st, SLOT_RETAIN);
+        retain_kernel<<<B, kSelectThreads, (size_t)n_vis, st>>>(ctx->sim, ctx->pivot_idx, pos_in, S, vis_offset, n_vis, P,
+                                                               n_keep, out_idx, out_pos, ctx->keep, ctx->owner,
+                                                               ctx->eps);
+    }
+    {
+        Prof pr(ctx, st, SLOT_GATHER);
+        long long orows = (long long)B * S_out;
+        unsigned grid = (unsigned)((orows + kGatherWarps - 1) / kGatherWarps);
+        gather_kernel<<<grid, kGatherWarps * 32, 0, st>>>((const uint4 *)hidden, out_idx, S, S_out, d8, orows,
+                                                         (uint4 *)out_hidden);
+    }
+    DART_CUDA(ctx, cudaGetLastError());
+    return copy_debug(ctx, B, n_vis, P, dbg, st);
+}
+
+int launch_reduce(dart_ctx *ctx, int B, const void *hidden, const void *keys, const int64_t *pos_in, int vis_offset,
+                  int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos, const dart_opts &o,
+                  const dart_debug *dbg, cudaStream_t st)
+{
+    const bool fused = o.path == DART_PATH_FUSED || (o.path == DART_PATH_AUTO && fused_applies(ctx, P));
+    if (fused && !fused_applies(ctx, P)) return DART_ERR_UNSUPPORTED;
+    return fused ? launch_fused(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos,
+                                o, dbg, st)
+                 : launch_staged(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos,
+                                 o, dbg, st);
 }
 
 } // namespace
@@ -248,6 +398,7 @@ int dart_create(dart_ctx **out, const dart_desc *desc)
                                       desc->S_max) != cudaSuccess)
             rc = DART_ERR_CUDA;
     }
+    if (rc == DART_OK) rc = fused_setup(ctx);
     if (rc == DART_OK && (desc->flags & DART_FLAG_HOST_STAGING)) {
         // chunk = as many samples as fit ~512 MiB of input staging per buffer set (at least one)
         const size_t per_sample = (size_t)desc->S_max * desc->d * 2;
@@ -295,6 +446,11 @@ int dart_destroy(dart_ctx *ctx)
     cudaFree(ctx->owner);
     cudaFree(ctx->keep);
     cudaFree(ctx->status);
+    cudaFree(ctx->pl1);
+    cudaFree(ctx->pssq);
+    cudaFree(ctx->psim);
+    cudaFree(ctx->pivK);
+    cudaFree(ctx->counters);
     for (int k = 0; k < 2; ++k) {
         cudaFree(ctx->st_hidden[k]);
         cudaFree(ctx->st_keys[k]);
@@ -331,11 +487,11 @@ int dart_reduce_ex(dart_ctx *ctx, const void *hidden, const void *keys, const in
     if (opts) o = *opts;
     if (o.norm_kind == 0) o.norm_kind = 1;
     if (o.norm_kind != 1 && o.norm_kind != 2) return DART_ERR_UNSUPPORTED;
-    if (o.path != DART_PATH_AUTO && o.path != DART_PATH_STAGED) return DART_ERR_UNSUPPORTED;
+    if (o.path != DART_PATH_AUTO && o.path != DART_PATH_STAGED && o.path != DART_PATH_FUSED) return DART_ERR_UNSUPPORTED;
     if ((uintptr_t)pos_in & 7u) return DART_ERR_ALIGN;
     DeviceGuard g(ctx->desc.device);
     if (!g.ok) return DART_ERR_CUDA;
-    return launch_staged(ctx, ctx->B, hidden, keys, pos_in, vis_offset, n_vis, n_pivot, n_keep, out_hidden, out_idx,
+    return launch_reduce(ctx, ctx->B, hidden, keys, pos_in, vis_offset, n_vis, n_pivot, n_keep, out_hidden, out_idx,
                          out_pos, o, dbg, (cudaStream_t)stream);
 }
 
@@ -373,7 +529,7 @@ int dart_reduce_host(dart_ctx *ctx, const void *hidden, const void *keys, int vi
                                            cudaMemcpyHostToDevice, ctx->s_h2d));
         DART_CUDA(ctx, cudaEventRecord(ctx->ev_in[k], ctx->s_h2d));
         DART_CUDA(ctx, cudaStreamWaitEvent(ctx->s_run, ctx->ev_in[k], 0));
-        rc = launch_staged(ctx, nb, ctx->st_hidden[k], keys ? ctx->st_keys[k] : nullptr, nullptr, vis_offset, n_vis,
+        rc = launch_reduce(ctx, nb, ctx->st_hidden[k], keys ? ctx->st_keys[k] : nullptr, nullptr, vis_offset, n_vis,
                            n_pivot, n_keep, ctx->st_out_hidden[k], ctx->st_out_idx[k], ctx->st_out_pos[k], o, nullptr,
                            ctx->s_run);
         if (rc != DART_OK) break;

@@ -49,7 +49,25 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
-// ---- block-wide selection of the k smallest (key, index) pairs -----------------------------------
+// ---- thread groups ---------------------------------------------------------------------------------
+// The selection helpers below run either on a whole CTA or on a group of warps inside one
+// (a named barrier), so that a few warps of a persistent kernel can select while others stream.
+struct CtaGroup {
+    __device__ __forceinline__ int tid() const { return threadIdx.x; }
+    __device__ __forceinline__ int size() const { return blockDim.x; }
+    __device__ __forceinline__ void sync() const { __syncthreads(); }
+};
+template <int kFirstWarp, int kWarps, int kBarrierId>
+struct WarpGroup {
+    __device__ __forceinline__ int tid() const { return (int)threadIdx.x - kFirstWarp * 32; }
+    __device__ __forceinline__ int size() const { return kWarps * 32; }
+    __device__ __forceinline__ void sync() const
+    {
+        asm volatile("bar.sync %0, %1;" ::"n"(kBarrierId), "n"(kWarps * 32) : "memory");
+    }
+};
+
+// ---- group-wide selection of the k smallest (key, index) pairs -----------------------------------
 // Radix select over 32-bit keys, 8 bits per pass, most significant first.  KeyFn(j, key&) returns
 // whether element j takes part and, if so, its key.  After the call every thread holds the same
 // threshold key T (the k-th smallest), the number `need_eq` of elements with key == T that belong to
@@ -60,32 +78,33 @@ struct SelectSmem {
     uint32_t bin, before, cnt;
 };
 
-template <typename KeyFn>
-__device__ void block_select_threshold(KeyFn keyfn, int n, uint32_t k, SelectSmem &sm, uint32_t &T,
+template <typename Group, typename KeyFn>
+__device__ void block_select_threshold(Group g, KeyFn keyfn, int n, uint32_t k, SelectSmem &sm, uint32_t &T,
                                        uint32_t &need_eq, uint32_t &cnt_eq)
 {
     uint32_t prefix = 0, mask = 0, remaining = k, cnt = 0;
+    const int tid = g.tid(), gsz = g.size();
     for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int i = threadIdx.x; i < 256; i += blockDim.x) sm.hist[i] = 0;
-        __syncthreads();
-        for (int j = threadIdx.x; j < n; j += blockDim.x) {
+        for (int i = tid; i < 256; i += gsz) sm.hist[i] = 0;
+        g.sync();
+        for (int j = tid; j < n; j += gsz) {
             uint32_t key;
             if (keyfn(j, key) && (key & mask) == prefix) atomicAdd(&sm.hist[(key >> shift) & 255u], 1u);
         }
-        __syncthreads();
-        if (threadIdx.x < kWarp) {
+        g.sync();
+        if (tid < kWarp) {
             // lane l owns bins [8l, 8l+8); find the bin where the running count reaches `remaining`
             uint32_t c[8], s = 0;
 #pragma unroll
             for (int t = 0; t < 8; ++t) {
-                c[t] = sm.hist[threadIdx.x * 8 + t];
+                c[t] = sm.hist[tid * 8 + t];
                 s += c[t];
             }
             uint32_t incl = s;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-                if ((int)threadIdx.x >= o) incl += v;
+                if (tid >= o) incl += v;
             }
             uint32_t excl = incl - s;
             if (excl < remaining && remaining <= incl) {
@@ -93,7 +112,7 @@ __device__ void block_select_threshold(KeyFn keyfn, int n, uint32_t k, SelectSme
 #pragma unroll
                 for (int t = 0; t < 8; ++t) {
                     if (run < remaining && remaining <= run + c[t]) {
-                        sm.bin = threadIdx.x * 8 + t;
+                        sm.bin = tid * 8 + t;
                         sm.before = run;
                         sm.cnt = c[t];
                     }
@@ -101,12 +120,12 @@ __device__ void block_select_threshold(KeyFn keyfn, int n, uint32_t k, SelectSme
                 }
             }
         }
-        __syncthreads();
+        g.sync();
         prefix |= sm.bin << shift;
         mask |= 255u << shift;
         remaining -= sm.before;
         cnt = sm.cnt;
-        __syncthreads();
+        g.sync();
     }
     T = prefix;
     need_eq = remaining;
@@ -114,27 +133,28 @@ __device__ void block_select_threshold(KeyFn keyfn, int n, uint32_t k, SelectSme
 }
 
 // Invoke pick(j, key) for every selected element: all with key < T, and the need_eq lowest-index
-// elements with key == T.  Block-uniform control flow; ends with a __syncthreads().
-template <typename KeyFn, typename PickFn>
-__device__ void block_select_apply(KeyFn keyfn, int n, uint32_t T, uint32_t need_eq, uint32_t cnt_eq,
+// elements with key == T.  Group-uniform control flow; ends with a group sync.
+template <typename Group, typename KeyFn, typename PickFn>
+__device__ void block_select_apply(Group g, KeyFn keyfn, int n, uint32_t T, uint32_t need_eq, uint32_t cnt_eq,
                                    SelectSmem &sm, PickFn pick)
 {
     const bool all_eq = (need_eq == cnt_eq);
-    for (int j = threadIdx.x; j < n; j += blockDim.x) {
+    const int tid = g.tid(), gsz = g.size();
+    for (int j = tid; j < n; j += gsz) {
         uint32_t key;
         if (keyfn(j, key) && (key < T || (all_eq && key == T))) pick(j, key);
     }
     if (!all_eq) {
         // ties at the threshold: walk the indices in order and take the first need_eq
-        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+        const int lane = tid & 31, warp = tid >> 5, nwarp = gsz >> 5;
         uint32_t base = 0;
-        for (int start = 0; start < n && base < need_eq; start += blockDim.x) {
-            int j = start + threadIdx.x;
+        for (int start = 0; start < n && base < need_eq; start += gsz) {
+            int j = start + tid;
             uint32_t key = 0;
             bool f = (j < n) && keyfn(j, key) && key == T;
             uint32_t bal = __ballot_sync(0xffffffffu, f);
             if (lane == 0) sm.warp_tot[warp] = __popc(bal);
-            __syncthreads();
+            g.sync();
             uint32_t before = 0, total = 0;
             for (int w = 0; w < nwarp; ++w) {
                 uint32_t t = sm.warp_tot[w];
@@ -144,10 +164,10 @@ __device__ void block_select_apply(KeyFn keyfn, int n, uint32_t T, uint32_t need
             uint32_t rank = base + before + __popc(bal & ((1u << lane) - 1u));
             if (f && rank < need_eq) pick(j, key);
             base += total;
-            __syncthreads();
+            g.sync();
         }
     }
-    __syncthreads();
+    g.sync();
 }
 
 } // namespace dart

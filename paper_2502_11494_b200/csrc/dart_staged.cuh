@@ -76,8 +76,8 @@ pivot_kernel(const float *__restrict__ score, int n_vis, int P, int P_pad, int s
     for (int i = threadIdx.x; i < P_pad; i += blockDim.x) piv_list[i] = ~0ull;
     if (threadIdx.x == 0) n_picked = 0;
     uint32_t T, need_eq, cnt_eq;
-    block_select_threshold(keyfn, n_vis, (uint32_t)P, sel, T, need_eq, cnt_eq);
-    block_select_apply(keyfn, n_vis, T, need_eq, cnt_eq, sel, [&](int j, uint32_t key) {
+    block_select_threshold(CtaGroup(), keyfn, n_vis, (uint32_t)P, sel, T, need_eq, cnt_eq);
+    block_select_apply(CtaGroup(), keyfn, n_vis, T, need_eq, cnt_eq, sel, [&](int j, uint32_t key) {
         uint32_t slot = atomicAdd(&n_picked, 1u);
         piv_list[slot] = ((unsigned long long)key << 32) | (uint32_t)j;
     });
@@ -220,10 +220,10 @@ retain_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_i
             return true;
         };
         uint32_t T, need_eq, cnt_eq;
-        block_select_threshold(keyfn, n_vis, (uint32_t)qi, sel, T, need_eq, cnt_eq);
+        block_select_threshold(CtaGroup(), keyfn, n_vis, (uint32_t)qi, sel, T, need_eq, cnt_eq);
         // picks only flip flags of elements that stay selected, so keyfn may run while others pick:
         // an element picked by another thread is never examined again by this round's owner thread
-        block_select_apply(keyfn, n_vis, T, need_eq, cnt_eq, sel, [&](int j, uint32_t) {
+        block_select_apply(CtaGroup(), keyfn, n_vis, T, need_eq, cnt_eq, sel, [&](int j, uint32_t) {
             keep[j] = 1;
             if (owner) owner[j] = i;
         });

@@ -1,0 +1,614 @@
+// Fused path, sweeps: ONE persistent kernel computes the scores (sweep 1), the pivots and the
+// pivot x token dot products (sweep 2) of a whole batch, so that the second read of every key row
+// is served by the L2 cache instead of HBM.
+//
+// Work is cut into tasks of 128 token rows x 512 columns (128 KB of keys).  Every task appears
+// twice in one global, static order: as a sweep-1 task (row L1 norms and sums of squares: the
+// K-norm of the Sec. 3.3 footnote and Eq. 7's denominator) and, `lag` tasks later, as a sweep-2
+// task (dot products with the sample's pivot rows: Eq. 7's numerator).  CTA c executes tasks
+// c, c + grid, c + 2 grid, ...  Because a task is only 128 KB, all SMs together hold < 20 MB in
+// flight, and the distance between the two reads of a row is the sample size plus the lag.
+//
+// Per CTA (192 threads):
+//   warp 0     producer: TMA loads of key tiles (and of the gathered pivot rows for sweep 2) into
+//              an 8-stage shared-memory ring; L2 evict_last on the first read, evict_first on the second
+//   warp 1     sweep 2: one thread issues tcgen05.mma (tokens = M 128, pivots = N, bf16 -> fp32 in TMEM)
+//   warps 2-5  sweep 1: each thread owns one tile row and sums it from shared memory;
+//              sweep 2: read the accumulators out of TMEM and store the partial dot products;
+//              the CTA that completes a row tile adds up its column-slab partials, the CTA that
+//              completes a sample selects the pivots (Def. 1) and publishes them.
+// A task covers 512 of the d columns; the per-slab partial sums are added in slab order by a single
+// thread per row, so every result is bitwise reproducible.
+//
+// Every wait (mbarrier or global flag) is bounded in time; on expiry the kernel records
+// DART_ERR_TIMEOUT in the status word, drains and exits normally.
+#pragma once
+#include <cuda.h>
+
+#include "dart_common.cuh"
+
+namespace dart {
+namespace sweep {
+
+constexpr int kTileRows = 128;
+constexpr int kAtomCols = 64;  // 64 bf16 = 128 bytes = one swizzle row
+constexpr int kSubRows = 32;   // rows per TMA box of the key tensor
+constexpr int kSlabAtoms = 8;  // a task spans 8 atoms = 512 columns
+constexpr int kMaxStages = 8; // ring depth; fewer when many pivots make the stages large
+constexpr int kAtomBytes = kTileRows * 128; // 16 KB: 128 rows x 128 bytes, 128B-swizzled, K-major
+constexpr int kSubBytes = kSubRows * 128;
+constexpr int kThreads = 192;
+constexpr int kWorkerWarp0 = 2, kWorkerWarps = 4, kWorkers = kWorkerWarps * 32;
+constexpr int kMaxN = 256; // pivots per MMA (N dimension)
+constexpr int kStatusTimeout = -7;
+
+using Workers = WarpGroup<kWorkerWarp0, kWorkerWarps, 1>;
+
+struct Params {
+    int B, S, vis_offset, n_vis, P, N; // N = P rounded up to a multiple of 16 (MMA N)
+    int d8;                            // row width in 16-byte units
+    int n_atoms, KS, n_rt, T;          // atoms per row; column slabs; row tiles per sample; tasks per sample and sweep
+    int n_stages;                      // ring depth (<= kMaxStages)
+    long long lag;                     // tasks between a task's first and second sweep (T <= lag <= B * T)
+    int norm_kind, smallest;
+    unsigned long long wait_ns;        // time limit of every wait
+    const uint4 *keys;
+    float *pl1, *pssq;                 // [B][KS][n_vis] per-slab partial sums
+    float *psim;                       // [B][KS][n_vis][P] per-slab partial dot products
+    float *l1, *ssq;                   // [B][n_vis]
+    int32_t *pivot_idx;                // [B][P]
+    uint4 *pivK;                       // [B][N][d8] pivot rows gathered for the MMA's B operand
+    int *rt_done;                      // [B][n_rt] column slabs finished per row tile
+    int *s1_done;                      // [B] row tiles finished per sample
+    int *piv_ready;                    // [B] 1 once the pivots of the sample are published
+    int *status;
+};
+
+struct Task {
+    int kind; // 0 = sweep 1, 1 = sweep 2
+    int b, rt, ks;
+};
+
+__device__ __forceinline__ long long total_tasks(const Params &p) { return 2ll * p.B * p.T; }
+
+__device__ __forceinline__ Task decode(const Params &p, long long g)
+{
+    // order: sweep-1 tasks [0, lag) alone; then pairs (sweep-1 task lag + k, sweep-2 task k); then the
+    // last `lag` sweep-2 tasks alone
+    const long long n_all = (long long)p.B * p.T, head = p.lag, mid = 2 * (n_all - p.lag);
+    Task t;
+    long long n;
+    if (g < head) {
+        t.kind = 0;
+        n = g;
+    } else if (g < head + mid) {
+        const long long h = g - head;
+        t.kind = (int)(h & 1);
+        n = t.kind ? (h >> 1) : (h >> 1) + p.lag;
+    } else {
+        t.kind = 1;
+        n = n_all - p.lag + (g - head - mid);
+    }
+    t.b = (int)(n / p.T);
+    const int u = (int)(n % p.T);
+    t.rt = u / p.KS;
+    t.ks = u % p.KS;
+    return t;
+}
+
+__device__ __forceinline__ int slab_atoms(const Params &p, int ks) { return min(kSlabAtoms, p.n_atoms - ks * kSlabAtoms); }
+
+// ---- PTX wrappers -------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *ptr) { return (uint32_t)__cvta_generic_to_shared(ptr); }
+__device__ __forceinline__ unsigned long long now_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok)
+                 : "r"(bar), "r"(parity)
+                 : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int x, int y, uint32_t bar,
+                                            unsigned long long policy)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+                 " [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
+                 "l"(tm), "r"(x), "r"(y), "r"(bar), "l"(policy)
+                 : "memory");
+}
+__device__ __forceinline__ int ld_acquire(const int *ptr)
+{
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release(int *ptr, int v)
+{
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(ptr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+// OR of a predicate over the worker warps; doubles as their barrier
+__device__ __forceinline__ bool workers_any(bool pred)
+{
+    uint32_t r;
+    asm volatile("{\n.reg .pred p, q;\nsetp.ne.u32 q, %1, 0;\nbar.red.or.pred p, 1, %2, q;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(r)
+                 : "r"((uint32_t)pred), "n"(kWorkers)
+                 : "memory");
+    return r != 0;
+}
+
+// Shared-memory matrix descriptor of a K-major, 128B-swizzled bf16 tile (rows at a 128-byte pitch,
+// groups of 8 rows 1024 bytes apart).
+__device__ __forceinline__ unsigned long long umma_desc(uint32_t saddr)
+{
+    unsigned long long d = 0;
+    d |= (unsigned long long)((saddr & 0x3ffffu) >> 4);  // start address
+    d |= (unsigned long long)1 << 16;                    // leading byte offset (unused for this layout)
+    d |= (unsigned long long)(1024 >> 4) << 32;          // stride byte offset: 8 rows x 128 bytes
+    d |= (unsigned long long)1 << 46;                    // descriptor version of sm_100
+    d |= (unsigned long long)2 << 61;                    // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n
+__device__ __forceinline__ uint32_t umma_idesc(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, unsigned long long da, unsigned long long db, uint32_t idesc,
+                                          uint32_t accumulate)
+{
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
+                 "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+                 : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float *v)
+{
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// ---- bounded waits --------------------------------------------------------------------------------
+struct Ctl {
+    volatile int *abort_flag; // shared memory
+    int *status;              // global status word
+    unsigned long long limit_ns;
+    __device__ __forceinline__ bool aborted() const { return *abort_flag != 0; }
+    __device__ void give_up() const
+    {
+        *abort_flag = 1;
+        atomicCAS(status, 0, kStatusTimeout);
+    }
+    __device__ bool wait_bar(uint32_t bar, uint32_t parity) const
+    {
+        if (mbar_try_wait(bar, parity)) return true;
+        const unsigned long long t0 = now_ns();
+        for (uint32_t it = 0;; ++it) {
+            if (mbar_try_wait(bar, parity)) return true;
+            if ((it & 15u) == 15u) {
+                if (aborted()) return false;
+                if (now_ns() - t0 > limit_ns) {
+                    give_up();
+                    return false;
+                }
+            }
+        }
+    }
+    __device__ bool wait_flag(const int *flag) const
+    {
+        if (ld_acquire(flag) != 0) return true;
+        const unsigned long long t0 = now_ns();
+        for (uint32_t it = 0;; ++it) {
+            if (ld_acquire(flag) != 0) return true;
+            __nanosleep(64);
+            if ((it & 15u) == 15u) {
+                if (aborted()) return false;
+                if (now_ns() - t0 > limit_ns) {
+                    give_up();
+                    return false;
+                }
+            }
+        }
+    }
+};
+
+struct Ring {
+    int depth;
+    int stage = 0;
+    uint32_t phase = 0;
+    __device__ explicit Ring(int n_stages) : depth(n_stages) {}
+    __device__ __forceinline__ void advance(int n = 1)
+    {
+        stage += n;
+        while (stage >= depth) {
+            stage -= depth;
+            phase ^= 1u;
+        }
+    }
+};
+
+struct Shared {
+    unsigned long long full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[2], tmem_empty[2];
+    unsigned long long piv_list[kMaxN];
+    SelectSmem sel;
+    uint32_t tmem_base, n_picked;
+    int abort_flag, bcast;
+};
+
+__host__ __device__ inline uint32_t b_stage_bytes(int N) { return (uint32_t)((N * 128 + 1023) / 1024 * 1024); }
+__host__ inline int ring_depth(int N, size_t smem_limit)
+{
+    size_t n = (smem_limit - 1024 - 8192) / (kAtomBytes + b_stage_bytes(N)); // 8 KB left for static shared memory
+    return (int)(n > (size_t)kMaxStages ? (size_t)kMaxStages : n);
+}
+__host__ inline size_t smem_bytes(int N, int n_stages) { return 1024 + (size_t)n_stages * (kAtomBytes + b_stage_bytes(N)); }
+
+// The sample finisher (worker warps): pivots of sample b (Def. 1) and their rows gathered for sweep 2.
+__device__ void select_pivots(const Params &p, Shared &sh, int b)
+{
+    const Workers g;
+    const int tid = g.tid();
+    const float *score = (p.norm_kind == 2 ? p.ssq : p.l1) + (size_t)b * p.n_vis;
+    const int smallest = p.smallest;
+    auto keyfn = [&](int j, uint32_t &key) {
+        uint32_t k = order_key(__ldcg(score + j));
+        key = smallest ? k : ~k; // smaller key = better pivot
+        return true;
+    };
+    int P_pad = 1;
+    while (P_pad < p.P) P_pad <<= 1;
+    for (int i = tid; i < P_pad; i += kWorkers) sh.piv_list[i] = ~0ull;
+    if (tid == 0) sh.n_picked = 0;
+    uint32_t T, need_eq, cnt_eq;
+    block_select_threshold(g, keyfn, p.n_vis, (uint32_t)p.P, sh.sel, T, need_eq, cnt_eq);
+    block_select_apply(g, keyfn, p.n_vis, T, need_eq, cnt_eq, sh.sel, [&](int j, uint32_t key) {
+        uint32_t slot = atomicAdd(&sh.n_picked, 1u);
+        sh.piv_list[slot] = ((unsigned long long)key << 32) | (uint32_t)j;
+    });
+    for (int k = 2; k <= P_pad; k <<= 1) {
+        for (int jj = k >> 1; jj > 0; jj >>= 1) {
+            for (int i = tid; i < P_pad; i += kWorkers) {
+                int l = i ^ jj;
+                if (l > i) {
+                    unsigned long long x = sh.piv_list[i], y = sh.piv_list[l];
+                    bool up = ((i & k) == 0);
+                    if ((x > y) == up) {
+                        sh.piv_list[i] = y;
+                        sh.piv_list[l] = x;
+                    }
+                }
+            }
+            g.sync();
+        }
+    }
+    for (int i = tid; i < p.P; i += kWorkers) p.pivot_idx[(size_t)b * p.P + i] = (int32_t)(sh.piv_list[i] & 0xffffffffu);
+    // gather the pivot rows (rows >= P of the N-row block keep whatever finite data they hold: their
+    // accumulator columns are never read)
+    const uint4 *base = p.keys + ((size_t)b * p.S + p.vis_offset) * (size_t)p.d8;
+    uint4 *dst = p.pivK + (size_t)b * p.N * p.d8;
+    const int total = p.P * p.d8;
+    for (int i0 = tid; i0 < total; i0 += kWorkers * 8) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            int i = i0 + u * kWorkers;
+            if (i < total) {
+                int r = i / p.d8, c = i - r * p.d8;
+                v[u] = __ldcg(base + (size_t)(uint32_t)(sh.piv_list[r] & 0xffffffffu) * p.d8 + c);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            int i = i0 + u * kWorkers;
+            if (i < total) dst[i] = v[u];
+        }
+    }
+    // make the rows visible to other SMs' TMA reads, then publish
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+    __threadfence();
+    g.sync();
+    if (tid == 0) st_release(p.piv_ready + b, 1);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant__ CUtensorMap tm_piv, const Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ Shared sh;
+    const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bstage = b_stage_bytes(p.N);
+    auto a_addr = [&](int s) { return smem0 + (uint32_t)s * kAtomBytes; };
+    auto b_addr = [&](int s) { return smem0 + (uint32_t)p.n_stages * kAtomBytes + (uint32_t)s * bstage; };
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const Ctl ctl{&sh.abort_flag, p.status, p.wait_ns};
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.n_stages; ++s) {
+            mbar_init(smem_u32(&sh.full_bar[s]), 1);
+            mbar_init(smem_u32(&sh.empty_bar[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&sh.tmem_full[a]), 1);
+            mbar_init(smem_u32(&sh.tmem_empty[a]), kWorkerWarps);
+        }
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    uint32_t tmem_cols = 32;
+    while (tmem_cols < 2u * p.N) tmem_cols <<= 1;
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = sh.tmem_base;
+    const long long total = total_tasks(p);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            unsigned long long pol_keep, pol_drop;
+            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_drop));
+            Ring ring(p.n_stages);
+            long long issued = 0;
+            bool ok = true;
+            for (long long g = blockIdx.x; ok && g < total; g += gridDim.x) {
+                const Task t = decode(p, g);
+                if (t.kind == 1) {
+                    ok = ctl.wait_flag(p.piv_ready + t.b);
+                    if (!ok) break;
+                    asm volatile("fence.proxy.async.global;" ::: "memory");
+                }
+                const int na = slab_atoms(p, t.ks);
+                const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
+                const int n_sub = (rows + kSubRows - 1) / kSubRows;
+                const int y0 = t.b * p.S + p.vis_offset + t.rt * kTileRows;
+                for (int a = 0; a < na; ++a) {
+                    ok = ctl.wait_bar(smem_u32(&sh.empty_bar[ring.stage]), ring.phase ^ 1u);
+                    if (!ok) break;
+                    const uint32_t full = smem_u32(&sh.full_bar[ring.stage]);
+                    mbar_arrive_expect_tx(full, (uint32_t)n_sub * kSubBytes + (t.kind ? (uint32_t)p.N * 128u : 0u));
+                    const int x = (t.ks * kSlabAtoms + a) * kAtomCols;
+                    for (int s = 0; s < n_sub; ++s)
+                        tma_load_2d(a_addr(ring.stage) + (uint32_t)s * kSubBytes, &tm_keys, x, y0 + s * kSubRows, full,
+                                    t.kind ? pol_drop : pol_keep);
+                    if (t.kind) tma_load_2d(b_addr(ring.stage), &tm_piv, x, t.b * p.N, full, pol_keep);
+                    ring.advance();
+                    ++issued;
+                }
+            }
+            if (!ok) {
+                // drain: let the copies already issued land before the CTA may exit
+                const long long first = issued > p.n_stages ? issued - p.n_stages : 0;
+                for (long long i = first; i < issued; ++i)
+                    ctl.wait_bar(smem_u32(&sh.full_bar[i % p.n_stages]), (uint32_t)((i / p.n_stages) & 1));
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ sweep-2 MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc(p.N);
+            Ring ring(p.n_stages);
+            uint32_t s2n = 0;
+            bool ok = true;
+            for (long long g = blockIdx.x; ok && g < total; g += gridDim.x) {
+                const Task t = decode(p, g);
+                const int na = slab_atoms(p, t.ks);
+                if (t.kind == 0) {
+                    ring.advance(na);
+                    continue;
+                }
+                const uint32_t acc = s2n & 1u;
+                ok = ctl.wait_bar(smem_u32(&sh.tmem_empty[acc]), ((s2n >> 1) & 1u) ^ 1u);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)p.N;
+                for (int a = 0; a < na; ++a) {
+                    ok = ctl.wait_bar(smem_u32(&sh.full_bar[ring.stage]), ring.phase);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const unsigned long long da = umma_desc(a_addr(ring.stage)), db = umma_desc(b_addr(ring.stage));
+#pragma unroll
+                    for (int k = 0; k < kAtomCols / 16; ++k) // 16 columns = 32 bytes per MMA: advance the start address
+                        umma_bf16(d_tmem, da + (unsigned long long)(2 * k), db + (unsigned long long)(2 * k), idesc,
+                                  (a | k) != 0);
+                    umma_commit(smem_u32(&sh.empty_bar[ring.stage])); // frees the stage once the MMAs have read it
+                    ring.advance();
+                }
+                if (!ok) break;
+                umma_commit(smem_u32(&sh.tmem_full[acc]));
+                ++s2n;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ workers
+        const int wt = threadIdx.x - kWorkerWarp0 * 32;      // 0..127
+        const int quarter = warp & 3;                        // TMEM lane quarter this warp may read
+        const int row = quarter * 32 + lane;                 // tile row owned by this thread
+        Ring ring(p.n_stages);
+        uint32_t s2n = 0;
+        bool dead = false; // group-uniform after every workers_any()
+        for (long long g = blockIdx.x; g < total; g += gridDim.x) {
+            const Task t = decode(p, g);
+            const int na = slab_atoms(p, t.ks);
+            const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
+            const int j = t.rt * kTileRows + row;
+            if (t.kind == 0) {
+                float a0 = 0.f, a1 = 0.f, q0 = 0.f, q1 = 0.f;
+                for (int a = 0; a < na; ++a) {
+                    bool fail = dead;
+                    if (!fail) fail = !ctl.wait_bar(smem_u32(&sh.full_bar[ring.stage]), ring.phase);
+                    if (!fail && row < rows) {
+                        const uint32_t base = a_addr(ring.stage) + (uint32_t)row * 128u;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            // logical 16-byte chunk c of this row sits at chunk c ^ (row & 7)
+                            const uint4 v = lds128(base + (uint32_t)((c ^ (row & 7)) << 4));
+                            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float lo = bf16_lo(w[e]), hi = bf16_hi(w[e]);
+                                a0 += fabsf(lo);
+                                a1 += fabsf(hi);
+                                q0 = fmaf(lo, lo, q0);
+                                q1 = fmaf(hi, hi, q1);
+                            }
+                        }
+                    }
+                    dead = workers_any(fail); // also: every worker has finished reading the stage
+                    if (!dead && wt == 0) mbar_arrive(smem_u32(&sh.empty_bar[ring.stage]));
+                    ring.advance();
+                }
+                if (!dead && row < rows) {
+                    const size_t o = ((size_t)t.b * p.KS + t.ks) * p.n_vis + j;
+                    p.pl1[o] = a0 + a1;
+                    p.pssq[o] = q0 + q1;
+                }
+                // count the slab; the CTA that delivers a row tile's last slab adds up the partials
+                __threadfence();
+                dead = workers_any(dead);
+                if (wt == 0) {
+                    int old = dead ? -1 : atomicAdd(p.rt_done + (size_t)t.b * p.n_rt + t.rt, 1);
+                    __threadfence();
+                    sh.bcast = old;
+                }
+                dead = workers_any(dead);
+                if (!dead && sh.bcast == p.KS - 1) {
+                    if (row < rows) {
+                        float s1 = 0.f, s2 = 0.f;
+                        for (int ks = 0; ks < p.KS; ++ks) {
+                            const size_t o = ((size_t)t.b * p.KS + ks) * p.n_vis + j;
+                            s1 += __ldcg(p.pl1 + o);
+                            s2 += __ldcg(p.pssq + o);
+                        }
+                        p.l1[(size_t)t.b * p.n_vis + j] = s1;
+                        p.ssq[(size_t)t.b * p.n_vis + j] = s2;
+                    }
+                    __threadfence();
+                    workers_any(false);
+                    if (wt == 0) {
+                        int old = atomicAdd(p.s1_done + t.b, 1);
+                        __threadfence();
+                        sh.bcast = old;
+                    }
+                    workers_any(false);
+                    if (sh.bcast == p.n_rt - 1) select_pivots(p, sh, t.b);
+                }
+                workers_any(false); // sh.bcast may be rewritten by the next task only after everyone has read it
+            } else {
+                ring.advance(na);
+                if (dead) continue;
+                const uint32_t acc = s2n & 1u;
+                bool ok = ctl.wait_bar(smem_u32(&sh.tmem_full[acc]), (s2n >> 1) & 1u);
+                ok = __all_sync(0xffffffffu, ok);
+                if (ok) {
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t taddr = tmem_base + acc * (uint32_t)p.N + ((uint32_t)(quarter * 32) << 16);
+                    float *dst = p.psim + (((size_t)t.b * p.KS + t.ks) * p.n_vis + j) * p.P;
+                    for (int c0 = 0; c0 < p.P; c0 += 8) {
+                        float v[8];
+                        tmem_ld8(taddr + (uint32_t)c0, v); // warp-collective: rows outside the tile still take part
+                        if (row < rows) {
+                            if (c0 + 8 <= p.P && (p.P & 3) == 0) {
+                                *reinterpret_cast<float4 *>(dst + c0) = make_float4(v[0], v[1], v[2], v[3]);
+                                *reinterpret_cast<float4 *>(dst + c0 + 4) = make_float4(v[4], v[5], v[6], v[7]);
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 8; ++e)
+                                    if (c0 + e < p.P) dst[c0 + e] = v[e];
+                            }
+                        }
+                    }
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sh.tmem_empty[acc]));
+                } else {
+                    dead = true; // reaches the other worker warps at their next group barrier
+                }
+                ++s2n;
+            }
+        }
+    }
+    // ---------------------------------------------------------------------- teardown
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+}
+
+// Adds up the per-slab partial dot products in slab order and normalises them (Eq. 7):
+// sim[b][i][j] = (sum_ks psim[b][ks][j][i]) / (|K_{p_i}| |K_j|); a zero norm gives 0.
+constexpr int kFinalizeThreads = 128;
+
+__global__ void __launch_bounds__(kFinalizeThreads)
+finalize_sim_kernel(const float *__restrict__ psim, const float *__restrict__ ssq, const int32_t *__restrict__ pivot_idx,
+                    int n_vis, int P, int KS, float *__restrict__ sim)
+{
+    const int b = blockIdx.y, j = blockIdx.x * kFinalizeThreads + threadIdx.x;
+    if (j >= n_vis) return;
+    const float nj = sqrtf(ssq[(size_t)b * n_vis + j]);
+    const int32_t *piv = pivot_idx + (size_t)b * P;
+    for (int p0 = 0; p0 < P; p0 += 4) {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int ks = 0; ks < KS; ++ks) {
+            const float *src = psim + (((size_t)b * KS + ks) * n_vis + j) * P + p0;
+            if ((P & 3) == 0) {
+                const float4 v = __ldcs(reinterpret_cast<const float4 *>(src));
+                acc[0] += v.x, acc[1] += v.y, acc[2] += v.z, acc[3] += v.w;
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (p0 + e < P) acc[e] += __ldcs(src + e);
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (p0 + e >= P) break;
+            const float den = sqrtf(ssq[(size_t)b * n_vis + piv[p0 + e]]) * nj;
+            sim[((size_t)b * P + p0 + e) * n_vis + j] = den > 0.f ? acc[e] / den : 0.f;
+        }
+    }
+}
+
+} // namespace sweep
+} // namespace dart

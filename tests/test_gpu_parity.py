@@ -11,7 +11,8 @@ from paper_2502_11494_b200 import dart, workloads as W  # noqa: E402
 
 pytestmark = pytest.mark.gpu
 
-PATHS = [dart.DART_PATH_STAGED]
+PATHS = [dart.DART_PATH_STAGED, dart.DART_PATH_FUSED]
+PATH_IDS = {dart.DART_PATH_STAGED: "staged", dart.DART_PATH_FUSED: "fused"}
 
 
 def _np(t):
@@ -19,11 +20,14 @@ def _np(t):
     return W.bits(t) if t.dtype == torch.bfloat16 else t.numpy()
 
 
-def run_gpu(keys, hidden, vo, nv, P, Kp, pos_in=None, path=dart.DART_PATH_AUTO, norm_kind=0, smallest=0, debug=True):
+def run_gpu(keys, hidden, vo, nv, P, Kp, pos_in=None, path=dart.DART_PATH_AUTO, norm_kind=0, smallest=0, debug=True,
+            sweep_lag=0):
     B, S, d = hidden.shape
+    if path == dart.DART_PATH_FUSED and (d % 64 or P > 256):
+        pytest.skip("the fused path needs d % 64 == 0 and at most 256 pivots")
     ctx = dart.Dart(B, S, d, P, Kp)
     try:
-        opts = dart.dart_opts(norm_kind, smallest, path, 0)
+        opts = dart.dart_opts(norm_kind, smallest, path, 0, sweep_lag)
         res = ctx.reduce(hidden, keys, vo, nv, P, Kp, pos_in=pos_in, opts=opts, debug=debug)
         torch.cuda.synchronize()
         assert ctx.status() == dart.DART_OK
@@ -70,7 +74,7 @@ SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
 @pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(map(str, s)))
 def test_shapes_against_oracle(oracle, shape, path):
     B, S, d, vo, nv, P, Kp = shape
@@ -80,28 +84,28 @@ def test_shapes_against_oracle(oracle, shape, path):
     assert rep.max_rel_l1 < 5e-5 and rep.max_rel_l2 < 5e-5 and rep.max_abs_sim < 2e-5   # fp32-accumulation level
 
 
-@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
 def test_keys_null_scores_the_hidden_states(oracle, path):
     _, h = gaussian(2, 120, 256, seed=7)
     rep = compare(oracle, None, h, 10, 100, 4, 30, path=path)
     assert rep.samples == 2
 
 
-@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
 def test_position_ids_are_gathered(oracle, path):
     k, h = gaussian(2, 90, 64, seed=8)
     pos = torch.randint(0, 1 << 40, (2, 90), device="cuda", dtype=torch.int64)
     compare(oracle, k, h, 5, 70, 3, 20, pos_in=pos, path=path)
 
 
-@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
 @pytest.mark.parametrize("norm_kind,smallest", [(2, 0), (1, 1), (2, 1)])
 def test_score_variants(oracle, path, norm_kind, smallest):
     k, h = gaussian(2, 300, 128, seed=9)
     compare(oracle, k, h, 20, 260, 6, 50, path=path, norm_kind=norm_kind, smallest=smallest)
 
 
-@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
 def test_ties_and_exact_duplicates(oracle, path):
     """Exact copies of rows tie on score and on similarity; the lower index must win on both sides.
     All values are small integers so that fp32 and fp64 sums agree exactly and every tie is a true tie."""
@@ -118,7 +122,7 @@ def test_ties_and_exact_duplicates(oracle, path):
     assert np.array_equal(oh, ora.out_hidden) and np.array_equal(op, ora.out_pos)
 
 
-@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
 def test_zero_rows_and_all_equal_scores(oracle, path):
     S, d = 64, 32
     x = torch.zeros((1, S, d), dtype=torch.bfloat16, device="cuda")
@@ -130,7 +134,7 @@ def test_zero_rows_and_all_equal_scores(oracle, path):
     assert oi[0].tolist() == list(range(12))         # zero rows have the lowest dup (0 < 1) and are kept
 
 
-@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
 def test_scaled_copies_of_the_pivot_are_dropped(oracle, path):
     k, h = gaussian(1, 80, 128, seed=12)
     k[0, 5] *= 4.0
@@ -141,7 +145,7 @@ def test_scaled_copies_of_the_pivot_are_dropped(oracle, path):
     assert sorted(set(range(80)) - set(oi[0].tolist())) == [9, 23, 41]
 
 
-@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
 @pytest.mark.parametrize("w", [W.LLAVA15_B1, W.LLAVA15_B64, W.LLAVA_NEXT_B8, W.VIDEO_B4], ids=lambda w: w.name)
 def test_benchmark_configs(oracle, w, path):
     k, h = W.make_batch(w, device="cuda")
@@ -153,14 +157,39 @@ def test_benchmark_configs(oracle, w, path):
     assert rep.max_rel_l1 < 5e-5 and rep.max_abs_sim < 2e-5
 
 
-def test_runs_are_bitwise_reproducible():
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
+def test_runs_are_bitwise_reproducible(path):
     w = W.LLAVA15_B64.with_(B=4)
     k, h = W.make_batch(w, device="cuda")
-    a = run_gpu(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep)
+    a = run_gpu(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, path=path)
     for _ in range(3):
-        b = run_gpu(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep)
+        b = run_gpu(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, path=path)
         assert all(np.array_equal(x, y) for x, y in zip(a[:3], b[:3]))
         assert all(np.array_equal(a[3][n], b[3][n], equal_nan=(n == "eps")) for n in a[3])
+
+
+def test_fused_path_rejects_what_it_cannot_do():
+    k, h = gaussian(1, 64, 72, seed=15)                      # d = 72 is not a multiple of 64
+    ctx = dart.Dart(1, 64, 72, 2, 8)
+    with pytest.raises(dart.DartError) as e:
+        ctx.reduce(h, k, 0, 64, 2, 8, opts=dart.dart_opts(0, 0, dart.DART_PATH_FUSED, 0, 0))
+    assert e.value.code == dart.DART_ERR_UNSUPPORTED
+    ctx.reduce(h, k, 0, 64, 2, 8)                            # AUTO falls back to the staged kernels
+    torch.cuda.synchronize()
+    assert ctx.status() == dart.DART_OK
+    ctx.close()
+
+
+@pytest.mark.parametrize("lag", [1, 40, 100000])
+def test_fused_path_with_short_and_long_lags(oracle, lag):
+    """The distance between a row's two sweeps only changes the schedule (how long sweep 2 waits for the
+    pivots), never the result."""
+    w = W.LLAVA15_B64.with_(B=6)
+    k, h = W.make_batch(w, device="cuda")
+    a = run_gpu(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, path=dart.DART_PATH_FUSED, sweep_lag=lag)
+    b = run_gpu(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, path=dart.DART_PATH_FUSED)
+    assert all(np.array_equal(x, y) for x, y in zip(a[:3], b[:3]))
+    assert all(np.array_equal(a[3][n], b[3][n], equal_nan=(n == "eps")) for n in a[3])
 
 
 def test_argument_validation_launches_nothing():
