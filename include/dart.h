@@ -155,6 +155,16 @@ int dart_reduce_host(dart_ctx *ctx, const void *hidden, const void *keys, int vi
  */
 int dart_status(dart_ctx *ctx);
 
+/*
+ * Where the last non-zero status came from (as read by the last dart_status call that returned an error):
+ * detail[0] = which bounded wait expired (1 pivots not published, 2 ring stage not freed, 3 drain,
+ * 4 accumulator not freed, 5/6 tile not loaded (MMA / row sums), 7 accumulator not filled),
+ * detail[1] = index of the task in the kernel's schedule, detail[2] = CTA; for wait 1 also detail[3] = sample,
+ * detail[4] = row tiles it had completed, detail[5..10] = column slabs completed in its first row tiles.
+ * For bug reports.
+ */
+int dart_status_detail(const dart_ctx *ctx, int32_t detail[11]);
+
 /* The cudaError_t of the last failed CUDA call made on behalf of this context (0 if none). */
 int dart_last_cuda_error(const dart_ctx *ctx);
 

@@ -36,7 +36,8 @@ struct dart_ctx {
     float *l1, *ssq, *sim, *eps;
     int32_t *pivot_idx, *owner;
     uint8_t *keep;
-    int *status; // device status word
+    int *status; // device status word, followed by three words of detail
+    int32_t status_detail[11];
     // profiling
     bool profiling;
     std::vector<EventPair> pending, spare;
@@ -208,14 +209,14 @@ int launch_staged(dart_ctx *ctx, int B, const void *hidden, const void *keys_in,
         Prof p(ctx, st, SLOT_RETAIN);
         retain_kernel<<<B, kSelectThreads, (size_t)n_vis, st>>>(ctx->sim, ctx->pivot_idx, pos_in, S, vis_offset, n_vis, P,
                                                                n_keep, out_idx, out_pos, ctx->keep, ctx->owner,
-                                                               ctx->eps);
+                                                               ctx->eps, ctx->status);
     }
     {
         Prof p(ctx, st, SLOT_GATHER);
         long long orows = (long long)B * S_out;
         unsigned grid = (unsigned)((orows + kGatherWarps - 1) / kGatherWarps);
         gather_kernel<<<grid, kGatherWarps * 32, 0, st>>>((const uint4 *)hidden, out_idx, S, S_out, d8, orows,
-                                                         (uint4 *)out_hidden);
+                                                         ctx->status, (uint4 *)out_hidden);
     }
     DART_CUDA(ctx, cudaGetLastError());
     return copy_debug(ctx, B, n_vis, P, dbg, st);
@@ -256,8 +257,10 @@ int fused_setup(dart_ctx *ctx)
         cudaSuccess)
         return DART_ERR_CUDA;
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sweep_kernel, kThreads,
-                                                      smem_bytes(16, ring_depth(16, ctx->max_smem_optin))) != cudaSuccess ||
+    int n1 = 0, n2 = 0;
+    ring_depths(16, ctx->max_smem_optin, n1, n2);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sweep_kernel, kThreads, smem_bytes(16, n1, n2)) !=
+            cudaSuccess ||
         per_sm < 1)
         return DART_ERR_CUDA;
     ctx->fused_ok = true;
@@ -293,8 +296,8 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     Params p = {};
     p.B = B, p.S = S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.N = (P + 15) / 16 * 16, p.d8 = d8;
     p.n_atoms = ctx->n_atoms, p.KS = ctx->KS, p.n_rt = (n_vis + kTileRows - 1) / kTileRows, p.T = p.n_rt * p.KS;
-    p.n_stages = ring_depth(p.N, ctx->max_smem_optin);
-    if (p.n_stages < 2) return DART_ERR_UNSUPPORTED;
+    ring_depths(p.N, ctx->max_smem_optin, p.n1, p.n2);
+    if (p.n1 < 2) return DART_ERR_UNSUPPORTED;
     const long long n_all = (long long)B * p.T;
     // a row's second sweep follows its first by one sample plus the time the pivots take to appear
     long long lag = (long long)p.T + (o.sweep_lag > 0 ? o.sweep_lag : 3 * ctx->sm_count);
@@ -316,26 +319,26 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
         long long grid = 2 * n_all < ctx->sm_count ? 2 * n_all : ctx->sm_count;
         void *args[3] = {&tm_keys, &tm_piv, &p};
         DART_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)sweep_kernel, dim3((unsigned)grid), dim3(kThreads), args,
-                                                   smem_bytes(p.N, p.n_stages), st));
+                                                   smem_bytes(p.N, p.n1, p.n2), st));
     }
     {
         Prof pr(ctx, st, SLOT_FINALIZE);
         dim3 grid((n_vis + kFinalizeThreads - 1) / kFinalizeThreads, B);
         finalize_sim_kernel<<<grid, kFinalizeThreads, 0, st>>>(ctx->psim, ctx->ssq, ctx->pivot_idx, n_vis, P, p.KS,
-                                                               ctx->sim);
+                                                               ctx->status, ctx->sim);
     }
     {
         Prof pr(ctx, st, SLOT_RETAIN);
         retain_kernel<<<B, kSelectThreads, (size_t)n_vis, st>>>(ctx->sim, ctx->pivot_idx, pos_in, S, vis_offset, n_vis, P,
                                                                n_keep, out_idx, out_pos, ctx->keep, ctx->owner,
-                                                               ctx->eps);
+                                                               ctx->eps, ctx->status);
     }
     {
         Prof pr(ctx, st, SLOT_GATHER);
         long long orows = (long long)B * S_out;
         unsigned grid = (unsigned)((orows + kGatherWarps - 1) / kGatherWarps);
         gather_kernel<<<grid, kGatherWarps * 32, 0, st>>>((const uint4 *)hidden, out_idx, S, S_out, d8, orows,
-                                                         (uint4 *)out_hidden);
+                                                         ctx->status, (uint4 *)out_hidden);
     }
     DART_CUDA(ctx, cudaGetLastError());
     return copy_debug(ctx, B, n_vis, P, dbg, st);
@@ -557,11 +560,21 @@ int dart_status(dart_ctx *ctx)
     if (!ctx) return DART_ERR_NULL;
     DeviceGuard g(ctx->desc.device);
     if (!g.ok) return DART_ERR_CUDA;
-    int word = 0;
+    int word[12] = {0};
     DART_CUDA(ctx, cudaDeviceSynchronize());
-    DART_CUDA(ctx, cudaMemcpy(&word, ctx->status, sizeof word, cudaMemcpyDeviceToHost));
-    if (word != 0) DART_CUDA(ctx, cudaMemset(ctx->status, 0, sizeof word));
-    return word;
+    DART_CUDA(ctx, cudaMemcpy(word, ctx->status, sizeof word, cudaMemcpyDeviceToHost));
+    if (word[0] != 0) {
+        for (int k = 0; k < 11; ++k) ctx->status_detail[k] = word[k + 1];
+        DART_CUDA(ctx, cudaMemset(ctx->status, 0, sizeof word));
+    }
+    return word[0];
+}
+
+int dart_status_detail(const dart_ctx *ctx, int32_t detail[11])
+{
+    if (!ctx || !detail) return DART_ERR_NULL;
+    for (int k = 0; k < 11; ++k) detail[k] = ctx->status_detail[k];
+    return DART_OK;
 }
 
 int dart_last_cuda_error(const dart_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }

@@ -188,10 +188,12 @@ __global__ void __launch_bounds__(kSelectThreads)
 retain_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx, const int64_t *__restrict__ pos_in,
               int S, int vis_offset, int n_vis, int P, int n_keep,
               int32_t *__restrict__ out_idx, int64_t *__restrict__ out_pos,
-              uint8_t *__restrict__ keep_out, int32_t *__restrict__ owner_out, float *__restrict__ eps_out)
+              uint8_t *__restrict__ keep_out, int32_t *__restrict__ owner_out, float *__restrict__ eps_out,
+              const int *__restrict__ status)
 {
     extern __shared__ uint8_t keep[]; // [n_vis]
     __shared__ SelectSmem sel;
+    if (*status != 0) return; // an earlier kernel of this call failed: its outputs are undefined
     const int b = blockIdx.x;
     const int S_out = S - n_vis + n_keep;
     int32_t *owner = owner_out ? owner_out + (size_t)b * n_vis : nullptr;
@@ -278,11 +280,11 @@ constexpr int kGatherWarps = 8;
 
 __global__ void __launch_bounds__(kGatherWarps * 32)
 gather_kernel(const uint4 *__restrict__ hidden, const int32_t *__restrict__ out_idx, int S, int S_out, int d8,
-              long long rows_total, uint4 *__restrict__ out_hidden)
+              long long rows_total, const int *__restrict__ status, uint4 *__restrict__ out_hidden)
 {
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * kGatherWarps + (threadIdx.x >> 5);
-    if (row >= rows_total) return;
+    if (row >= rows_total || *status != 0) return; // after a failed kernel out_idx is undefined
     const int b = (int)(row / S_out);
     const int s = out_idx[row];
     const uint4 *src = hidden + ((size_t)b * S + s) * (size_t)d8;

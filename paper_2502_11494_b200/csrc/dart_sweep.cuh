@@ -10,8 +10,9 @@
 // flight, and the distance between the two reads of a row is the sample size plus the lag.
 //
 // Per CTA (192 threads):
-//   warp 0     producer: TMA loads of key tiles (and of the gathered pivot rows for sweep 2) into
-//              an 8-stage shared-memory ring; L2 evict_last on the first read, evict_first on the second
+//   warp 0     producer: TMA loads of key tiles (and of the gathered pivot rows for sweep 2) into two
+//              shared-memory rings, one per sweep, so that each ring has exactly one consumer role and
+//              no role ever skips a barrier phase; L2 evict_last on the first read, evict_first on the second
 //   warp 1     sweep 2: one thread issues tcgen05.mma (tokens = M 128, pivots = N, bf16 -> fp32 in TMEM)
 //   warps 2-5  sweep 1: each thread owns one tile row and sums it from shared memory;
 //              sweep 2: read the accumulators out of TMEM and store the partial dot products;
@@ -34,13 +35,15 @@ constexpr int kTileRows = 128;
 constexpr int kAtomCols = 64;  // 64 bf16 = 128 bytes = one swizzle row
 constexpr int kSubRows = 32;   // rows per TMA box of the key tensor
 constexpr int kSlabAtoms = 8;  // a task spans 8 atoms = 512 columns
-constexpr int kMaxStages = 8; // ring depth; fewer when many pivots make the stages large
+constexpr int kMaxStages = 8; // per ring; fewer when many pivots make the sweep-2 stages large
 constexpr int kAtomBytes = kTileRows * 128; // 16 KB: 128 rows x 128 bytes, 128B-swizzled, K-major
 constexpr int kSubBytes = kSubRows * 128;
 constexpr int kThreads = 192;
 constexpr int kWorkerWarp0 = 2, kWorkerWarps = 4, kWorkers = kWorkerWarps * 32;
 constexpr int kMaxN = 256; // pivots per MMA (N dimension)
 constexpr int kStatusTimeout = -7;
+// which wait expired (second status word)
+enum { kWaitPivots = 1, kWaitEmptyStage, kWaitDrain, kWaitAccumFree, kWaitStageMma, kWaitStageRows, kWaitAccumFull };
 
 using Workers = WarpGroup<kWorkerWarp0, kWorkerWarps, 1>;
 
@@ -48,7 +51,7 @@ struct Params {
     int B, S, vis_offset, n_vis, P, N; // N = P rounded up to a multiple of 16 (MMA N)
     int d8;                            // row width in 16-byte units
     int n_atoms, KS, n_rt, T;          // atoms per row; column slabs; row tiles per sample; tasks per sample and sweep
-    int n_stages;                      // ring depth (<= kMaxStages)
+    int n1, n2;                        // depth of the sweep-1 and of the sweep-2 ring (<= kMaxStages each)
     long long lag;                     // tasks between a task's first and second sweep (T <= lag <= B * T)
     int norm_kind, smallest;
     unsigned long long wait_ns;        // time limit of every wait
@@ -208,12 +211,17 @@ struct Ctl {
     int *status;              // global status word
     unsigned long long limit_ns;
     __device__ __forceinline__ bool aborted() const { return *abort_flag != 0; }
-    __device__ void give_up() const
+    // records the first wait that expired: status[1] = where (kWait*), status[2] = task index, status[3] = CTA
+    __device__ void give_up(int where, long long task) const
     {
         *abort_flag = 1;
-        atomicCAS(status, 0, kStatusTimeout);
+        if (atomicCAS(status, 0, kStatusTimeout) == 0) {
+            status[1] = where;
+            status[2] = (int)task;
+            status[3] = (int)blockIdx.x;
+        }
     }
-    __device__ bool wait_bar(uint32_t bar, uint32_t parity) const
+    __device__ bool wait_bar(uint32_t bar, uint32_t parity, int where, long long task) const
     {
         if (mbar_try_wait(bar, parity)) return true;
         const unsigned long long t0 = now_ns();
@@ -222,13 +230,13 @@ struct Ctl {
             if ((it & 15u) == 15u) {
                 if (aborted()) return false;
                 if (now_ns() - t0 > limit_ns) {
-                    give_up();
+                    give_up(where, task);
                     return false;
                 }
             }
         }
     }
-    __device__ bool wait_flag(const int *flag) const
+    __device__ bool wait_flag(const int *flag, int where, long long task) const
     {
         if (ld_acquire(flag) != 0) return true;
         const unsigned long long t0 = now_ns();
@@ -238,7 +246,7 @@ struct Ctl {
             if ((it & 15u) == 15u) {
                 if (aborted()) return false;
                 if (now_ns() - t0 > limit_ns) {
-                    give_up();
+                    give_up(where, task);
                     return false;
                 }
             }
@@ -250,7 +258,7 @@ struct Ring {
     int depth;
     int stage = 0;
     uint32_t phase = 0;
-    __device__ explicit Ring(int n_stages) : depth(n_stages) {}
+    __device__ explicit Ring(int d) : depth(d) {}
     __device__ __forceinline__ void advance(int n = 1)
     {
         stage += n;
@@ -262,7 +270,8 @@ struct Ring {
 };
 
 struct Shared {
-    unsigned long long full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[2], tmem_empty[2];
+    unsigned long long full1[kMaxStages], empty1[kMaxStages], full2[kMaxStages], empty2[kMaxStages];
+    unsigned long long tmem_full[2], tmem_empty[2];
     unsigned long long piv_list[kMaxN];
     SelectSmem sel;
     uint32_t tmem_base, n_picked;
@@ -270,12 +279,22 @@ struct Shared {
 };
 
 __host__ __device__ inline uint32_t b_stage_bytes(int N) { return (uint32_t)((N * 128 + 1023) / 1024 * 1024); }
-__host__ inline int ring_depth(int N, size_t smem_limit)
+// Ring depths for a shared-memory budget: half of it to the sweep-2 ring (at least 2 stages), the rest to sweep 1.
+__host__ inline void ring_depths(int N, size_t smem_limit, int &n1, int &n2)
 {
-    size_t n = (smem_limit - 1024 - 8192) / (kAtomBytes + b_stage_bytes(N)); // 8 KB left for static shared memory
-    return (int)(n > (size_t)kMaxStages ? (size_t)kMaxStages : n);
+    const size_t budget = smem_limit - 1024 - 8192; // alignment slack; 8 KB left for static shared memory
+    const size_t s2 = kAtomBytes + b_stage_bytes(N);
+    size_t b = budget / 2 / s2;
+    b = b < 2 ? 2 : (b > (size_t)kMaxStages ? (size_t)kMaxStages : b);
+    size_t a = budget > b * s2 ? (budget - b * s2) / kAtomBytes : 0;
+    a = a > (size_t)kMaxStages ? (size_t)kMaxStages : a;
+    n1 = (int)a;
+    n2 = (int)b;
 }
-__host__ inline size_t smem_bytes(int N, int n_stages) { return 1024 + (size_t)n_stages * (kAtomBytes + b_stage_bytes(N)); }
+__host__ inline size_t smem_bytes(int N, int n1, int n2)
+{
+    return 1024 + (size_t)n1 * kAtomBytes + (size_t)n2 * (kAtomBytes + b_stage_bytes(N));
+}
 
 // The sample finisher (worker warps): pivots of sample b (Def. 1) and their rows gathered for sweep 2.
 __device__ void select_pivots(const Params &p, Shared &sh, int b)
@@ -328,7 +347,8 @@ __device__ void select_pivots(const Params &p, Shared &sh, int b)
             int i = i0 + u * kWorkers;
             if (i < total) {
                 int r = i / p.d8, c = i - r * p.d8;
-                v[u] = __ldcg(base + (size_t)(uint32_t)(sh.piv_list[r] & 0xffffffffu) * p.d8 + c);
+                const uint32_t pr = min((uint32_t)(sh.piv_list[r] & 0xffffffffu), (uint32_t)(p.n_vis - 1));
+                v[u] = __ldcg(base + (size_t)pr * p.d8 + c);
             }
         }
 #pragma unroll
@@ -351,15 +371,20 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
     __shared__ Shared sh;
     const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bstage = b_stage_bytes(p.N);
-    auto a_addr = [&](int s) { return smem0 + (uint32_t)s * kAtomBytes; };
-    auto b_addr = [&](int s) { return smem0 + (uint32_t)p.n_stages * kAtomBytes + (uint32_t)s * bstage; };
+    // ring 1: n1 key tiles; ring 2: n2 key tiles followed by n2 pivot tiles
+    auto a1_addr = [&](int s) { return smem0 + (uint32_t)s * kAtomBytes; };
+    auto a2_addr = [&](int s) { return smem0 + (uint32_t)(p.n1 + s) * kAtomBytes; };
+    auto b2_addr = [&](int s) { return smem0 + (uint32_t)(p.n1 + p.n2) * kAtomBytes + (uint32_t)s * bstage; };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const Ctl ctl{&sh.abort_flag, p.status, p.wait_ns};
+    // consumers get a longer limit than the producer, so that the wait nearest the cause reports first
+    const Ctl ctl{&sh.abort_flag, p.status, warp == 0 ? p.wait_ns : p.wait_ns + p.wait_ns / 4};
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.n_stages; ++s) {
-            mbar_init(smem_u32(&sh.full_bar[s]), 1);
-            mbar_init(smem_u32(&sh.empty_bar[s]), 1);
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(smem_u32(&sh.full1[s]), 1);
+            mbar_init(smem_u32(&sh.empty1[s]), 1);
+            mbar_init(smem_u32(&sh.full2[s]), 1);
+            mbar_init(smem_u32(&sh.empty2[s]), 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&sh.tmem_full[a]), 1);
@@ -388,70 +413,79 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
             unsigned long long pol_keep, pol_drop;
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_drop));
-            Ring ring(p.n_stages);
-            long long issued = 0;
+            Ring r1(p.n1), r2(p.n2);
+            long long issued1 = 0, issued2 = 0;
             bool ok = true;
             for (long long g = blockIdx.x; ok && g < total; g += gridDim.x) {
                 const Task t = decode(p, g);
                 if (t.kind == 1) {
-                    ok = ctl.wait_flag(p.piv_ready + t.b);
-                    if (!ok) break;
+                    ok = ctl.wait_flag(p.piv_ready + t.b, kWaitPivots, g);
+                    if (!ok) {
+                        if (p.status[1] == kWaitPivots && p.status[3] == (int)blockIdx.x) {
+                            p.status[4] = t.b;
+                            p.status[5] = ld_acquire(p.s1_done + t.b);
+                            for (int r = 0; r < 6 && r < p.n_rt; ++r)
+                                p.status[6 + r] = ld_acquire(p.rt_done + (size_t)t.b * p.n_rt + r);
+                        }
+                        break;
+                    }
                     asm volatile("fence.proxy.async.global;" ::: "memory");
                 }
                 const int na = slab_atoms(p, t.ks);
                 const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
                 const int n_sub = (rows + kSubRows - 1) / kSubRows;
                 const int y0 = t.b * p.S + p.vis_offset + t.rt * kTileRows;
+                Ring &ring = t.kind ? r2 : r1;
                 for (int a = 0; a < na; ++a) {
-                    ok = ctl.wait_bar(smem_u32(&sh.empty_bar[ring.stage]), ring.phase ^ 1u);
+                    const uint32_t empty = smem_u32(t.kind ? &sh.empty2[ring.stage] : &sh.empty1[ring.stage]);
+                    const uint32_t full = smem_u32(t.kind ? &sh.full2[ring.stage] : &sh.full1[ring.stage]);
+                    ok = ctl.wait_bar(empty, ring.phase ^ 1u, kWaitEmptyStage, g);
                     if (!ok) break;
-                    const uint32_t full = smem_u32(&sh.full_bar[ring.stage]);
                     mbar_arrive_expect_tx(full, (uint32_t)n_sub * kSubBytes + (t.kind ? (uint32_t)p.N * 128u : 0u));
                     const int x = (t.ks * kSlabAtoms + a) * kAtomCols;
+                    const uint32_t dst = t.kind ? a2_addr(ring.stage) : a1_addr(ring.stage);
                     for (int s = 0; s < n_sub; ++s)
-                        tma_load_2d(a_addr(ring.stage) + (uint32_t)s * kSubBytes, &tm_keys, x, y0 + s * kSubRows, full,
+                        tma_load_2d(dst + (uint32_t)s * kSubBytes, &tm_keys, x, y0 + s * kSubRows, full,
                                     t.kind ? pol_drop : pol_keep);
-                    if (t.kind) tma_load_2d(b_addr(ring.stage), &tm_piv, x, t.b * p.N, full, pol_keep);
+                    if (t.kind) tma_load_2d(b2_addr(ring.stage), &tm_piv, x, t.b * p.N, full, pol_keep);
                     ring.advance();
-                    ++issued;
+                    ++(t.kind ? issued2 : issued1);
                 }
             }
             if (!ok) {
                 // drain: let the copies already issued land before the CTA may exit
-                const long long first = issued > p.n_stages ? issued - p.n_stages : 0;
-                for (long long i = first; i < issued; ++i)
-                    ctl.wait_bar(smem_u32(&sh.full_bar[i % p.n_stages]), (uint32_t)((i / p.n_stages) & 1));
+                for (long long i = issued1 > p.n1 ? issued1 - p.n1 : 0; i < issued1; ++i)
+                    ctl.wait_bar(smem_u32(&sh.full1[i % p.n1]), (uint32_t)((i / p.n1) & 1), kWaitDrain, i);
+                for (long long i = issued2 > p.n2 ? issued2 - p.n2 : 0; i < issued2; ++i)
+                    ctl.wait_bar(smem_u32(&sh.full2[i % p.n2]), (uint32_t)((i / p.n2) & 1), kWaitDrain, i);
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ sweep-2 MMA issuer
         if (lane == 0) {
             const uint32_t idesc = umma_idesc(p.N);
-            Ring ring(p.n_stages);
+            Ring ring(p.n2);
             uint32_t s2n = 0;
             bool ok = true;
             for (long long g = blockIdx.x; ok && g < total; g += gridDim.x) {
                 const Task t = decode(p, g);
                 const int na = slab_atoms(p, t.ks);
-                if (t.kind == 0) {
-                    ring.advance(na);
-                    continue;
-                }
+                if (t.kind == 0) continue;
                 const uint32_t acc = s2n & 1u;
-                ok = ctl.wait_bar(smem_u32(&sh.tmem_empty[acc]), ((s2n >> 1) & 1u) ^ 1u);
+                ok = ctl.wait_bar(smem_u32(&sh.tmem_empty[acc]), ((s2n >> 1) & 1u) ^ 1u, kWaitAccumFree, g);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem_base + acc * (uint32_t)p.N;
                 for (int a = 0; a < na; ++a) {
-                    ok = ctl.wait_bar(smem_u32(&sh.full_bar[ring.stage]), ring.phase);
+                    ok = ctl.wait_bar(smem_u32(&sh.full2[ring.stage]), ring.phase, kWaitStageMma, g);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const unsigned long long da = umma_desc(a_addr(ring.stage)), db = umma_desc(b_addr(ring.stage));
+                    const unsigned long long da = umma_desc(a2_addr(ring.stage)), db = umma_desc(b2_addr(ring.stage));
 #pragma unroll
                     for (int k = 0; k < kAtomCols / 16; ++k) // 16 columns = 32 bytes per MMA: advance the start address
                         umma_bf16(d_tmem, da + (unsigned long long)(2 * k), db + (unsigned long long)(2 * k), idesc,
                                   (a | k) != 0);
-                    umma_commit(smem_u32(&sh.empty_bar[ring.stage])); // frees the stage once the MMAs have read it
+                    umma_commit(smem_u32(&sh.empty2[ring.stage])); // frees the stage once the MMAs have read it
                     ring.advance();
                 }
                 if (!ok) break;
@@ -464,7 +498,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
         const int wt = threadIdx.x - kWorkerWarp0 * 32;      // 0..127
         const int quarter = warp & 3;                        // TMEM lane quarter this warp may read
         const int row = quarter * 32 + lane;                 // tile row owned by this thread
-        Ring ring(p.n_stages);
+        Ring ring(p.n1);
         uint32_t s2n = 0;
         bool dead = false; // group-uniform after every workers_any()
         for (long long g = blockIdx.x; g < total; g += gridDim.x) {
@@ -476,9 +510,9 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
                 float a0 = 0.f, a1 = 0.f, q0 = 0.f, q1 = 0.f;
                 for (int a = 0; a < na; ++a) {
                     bool fail = dead;
-                    if (!fail) fail = !ctl.wait_bar(smem_u32(&sh.full_bar[ring.stage]), ring.phase);
+                    if (!fail) fail = !ctl.wait_bar(smem_u32(&sh.full1[ring.stage]), ring.phase, kWaitStageRows, g);
                     if (!fail && row < rows) {
-                        const uint32_t base = a_addr(ring.stage) + (uint32_t)row * 128u;
+                        const uint32_t base = a1_addr(ring.stage) + (uint32_t)row * 128u;
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
                             // logical 16-byte chunk c of this row sits at chunk c ^ (row & 7)
@@ -495,7 +529,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
                         }
                     }
                     dead = workers_any(fail); // also: every worker has finished reading the stage
-                    if (!dead && wt == 0) mbar_arrive(smem_u32(&sh.empty_bar[ring.stage]));
+                    if (!dead && wt == 0) mbar_arrive(smem_u32(&sh.empty1[ring.stage]));
                     ring.advance();
                 }
                 if (!dead && row < rows) {
@@ -535,10 +569,9 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
                 }
                 workers_any(false); // sh.bcast may be rewritten by the next task only after everyone has read it
             } else {
-                ring.advance(na);
                 if (dead) continue;
                 const uint32_t acc = s2n & 1u;
-                bool ok = ctl.wait_bar(smem_u32(&sh.tmem_full[acc]), (s2n >> 1) & 1u);
+                bool ok = ctl.wait_bar(smem_u32(&sh.tmem_full[acc]), (s2n >> 1) & 1u, kWaitAccumFull, g);
                 ok = __all_sync(0xffffffffu, ok);
                 if (ok) {
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -582,10 +615,10 @@ constexpr int kFinalizeThreads = 128;
 
 __global__ void __launch_bounds__(kFinalizeThreads)
 finalize_sim_kernel(const float *__restrict__ psim, const float *__restrict__ ssq, const int32_t *__restrict__ pivot_idx,
-                    int n_vis, int P, int KS, float *__restrict__ sim)
+                    int n_vis, int P, int KS, const int *__restrict__ status, float *__restrict__ sim)
 {
     const int b = blockIdx.y, j = blockIdx.x * kFinalizeThreads + threadIdx.x;
-    if (j >= n_vis) return;
+    if (j >= n_vis || *status != 0) return; // after a failed sweep the pivots are undefined
     const float nj = sqrtf(ssq[(size_t)b * n_vis + j]);
     const int32_t *piv = pivot_idx + (size_t)b * P;
     for (int p0 = 0; p0 < P; p0 += 4) {

@@ -22,7 +22,7 @@ DART_PATH_AUTO, DART_PATH_STAGED, DART_PATH_FUSED = 0, 1, 2
 
 EXPORTS = (
     "dart_create", "dart_destroy", "dart_set_shape", "dart_reduce", "dart_reduce_ex", "dart_reduce_host",
-    "dart_status", "dart_last_cuda_error", "dart_workspace_bytes", "dart_launch_count",
+    "dart_status", "dart_status_detail", "dart_last_cuda_error", "dart_workspace_bytes", "dart_launch_count",
     "dart_profile_enable", "dart_profile_read", "dart_strerror", "dart_version", "dart_pivots_static",
 )
 DART_STATIC_MAX_ROWS = 262144
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
                                      ctypes.POINTER(dart_opts), ctypes.POINTER(dart_debug), vp]
         L.dart_reduce_host.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, i32p, i64p]
         L.dart_status.argtypes = [vp]
+        L.dart_status_detail.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
         L.dart_last_cuda_error.argtypes = [vp]
         L.dart_workspace_bytes.argtypes = [vp]
         L.dart_workspace_bytes.restype = ctypes.c_size_t
@@ -135,6 +136,13 @@ def dart_pivots_static(keys, B, S, d, vis_offset, n_vis, n_pivot, pivot_idx, dev
 
 def dart_status(ctx) -> int:
     return lib().dart_status(ctx)
+
+
+def dart_status_detail(ctx):
+    """-> (return code, [which wait, task index, CTA]) of the last error that dart_status reported."""
+    d = (ctypes.c_int32 * 11)()
+    rc = lib().dart_status_detail(ctx, d)
+    return rc, list(d)
 
 
 def dart_last_cuda_error(ctx) -> int:

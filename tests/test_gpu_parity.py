@@ -30,7 +30,8 @@ def run_gpu(keys, hidden, vo, nv, P, Kp, pos_in=None, path=dart.DART_PATH_AUTO, 
         opts = dart.dart_opts(norm_kind, smallest, path, 0, sweep_lag)
         res = ctx.reduce(hidden, keys, vo, nv, P, Kp, pos_in=pos_in, opts=opts, debug=debug)
         torch.cuda.synchronize()
-        assert ctx.status() == dart.DART_OK
+        st = ctx.status()
+        assert st == dart.DART_OK, (st, dart.dart_status_detail(ctx.handle))
     finally:
         ctx.close()
     oh, oi, op = _np(res[0]), _np(res[1]), _np(res[2])
