@@ -55,7 +55,7 @@ struct dart_ctx {
     bool fused_ok;
     int sm_count, KS, n_atoms, N_max;
     float *pl1, *pssq, *psim;
-    uint4 *pivK;
+    unsigned long long *cand;
     int *counters;
     size_t counters_bytes;
     TensorMapEncodeFn encode;
@@ -247,13 +247,12 @@ int fused_setup(dart_ctx *ctx)
     int rc = ws_alloc(ctx, &ctx->pl1, nv * ctx->KS);
     if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->pssq, nv * ctx->KS);
     if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->psim, nv * ctx->KS * P_cap);
-    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->pivK, (size_t)D.B_max * ctx->N_max * (D.d / 8));
+    const int Pc_max = P_cap < kTileRows ? P_cap : kTileRows;
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->cand, (size_t)D.B_max * n_rt_max * Pc_max);
     ctx->counters_bytes = (size_t)D.B_max * (n_rt_max + 2) * sizeof(int);
     if (rc == DART_OK) rc = ws_alloc(ctx, (uint8_t **)&ctx->counters, ctx->counters_bytes);
     if (rc != DART_OK) return rc;
-    // rows of the gathered-pivot blocks beyond the pivot count are read by the MMA and must stay finite
-    if (cudaMemset(ctx->pivK, 0, (size_t)D.B_max * ctx->N_max * (D.d / 8) * 16) != cudaSuccess) return DART_ERR_CUDA;
-    if (cudaFuncSetAttribute(sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - 8192) !=
+    if (cudaFuncSetAttribute(sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - kStaticSmemReserve) !=
         cudaSuccess)
         return DART_ERR_CUDA;
     int per_sm = 0;
@@ -295,6 +294,7 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     const void *keys = keys_in ? keys_in : hidden;
     Params p = {};
     p.B = B, p.S = S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.N = (P + 15) / 16 * 16, p.d8 = d8;
+    p.Pc = P < kTileRows ? P : kTileRows;
     p.n_atoms = ctx->n_atoms, p.KS = ctx->KS, p.n_rt = (n_vis + kTileRows - 1) / kTileRows, p.T = p.n_rt * p.KS;
     ring_depths(p.N, ctx->max_smem_optin, p.n1, p.n2);
     if (p.n1 < 2) return DART_ERR_UNSUPPORTED;
@@ -304,20 +304,19 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     p.lag = lag < n_all ? lag : n_all;
     p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
-    p.keys = (const uint4 *)keys;
     p.pl1 = ctx->pl1, p.pssq = ctx->pssq, p.psim = ctx->psim, p.l1 = ctx->l1, p.ssq = ctx->ssq;
-    p.pivot_idx = ctx->pivot_idx, p.pivK = ctx->pivK;
+    p.pivot_idx = ctx->pivot_idx, p.cand = ctx->cand;
     p.rt_done = ctx->counters, p.s1_done = ctx->counters + (size_t)B * p.n_rt, p.piv_ready = p.s1_done + B;
     p.status = ctx->status;
-    CUtensorMap tm_keys, tm_piv;
+    CUtensorMap tm_keys, tm_row; // the same tensor with a 32-row box (tiles) and a one-row box (pivot rows)
     int rc = encode_2d(ctx, &tm_keys, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, kSubRows);
-    if (rc == DART_OK) rc = encode_2d(ctx, &tm_piv, ctx->pivK, (uint64_t)ctx->desc.d, (uint64_t)B * p.N, (uint32_t)p.N);
+    if (rc == DART_OK) rc = encode_2d(ctx, &tm_row, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, 1);
     if (rc != DART_OK) return rc;
     DART_CUDA(ctx, cudaMemsetAsync(ctx->counters, 0, (size_t)B * (p.n_rt + 2) * sizeof(int), st));
     {
         Prof pr(ctx, st, SLOT_SWEEP);
         long long grid = 2 * n_all < ctx->sm_count ? 2 * n_all : ctx->sm_count;
-        void *args[3] = {&tm_keys, &tm_piv, &p};
+        void *args[3] = {&tm_keys, &tm_row, &p};
         DART_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)sweep_kernel, dim3((unsigned)grid), dim3(kThreads), args,
                                                    smem_bytes(p.N, p.n1, p.n2), st));
     }
@@ -452,7 +451,7 @@ int dart_destroy(dart_ctx *ctx)
     cudaFree(ctx->pl1);
     cudaFree(ctx->pssq);
     cudaFree(ctx->psim);
-    cudaFree(ctx->pivK);
+    cudaFree(ctx->cand);
     cudaFree(ctx->counters);
     for (int k = 0; k < 2; ++k) {
         cudaFree(ctx->st_hidden[k]);

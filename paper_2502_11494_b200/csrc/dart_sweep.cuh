@@ -9,17 +9,20 @@
 // c, c + grid, c + 2 grid, ...  Because a task is only 128 KB, all SMs together hold < 20 MB in
 // flight, and the distance between the two reads of a row is the sample size plus the lag.
 //
-// Per CTA (192 threads):
-//   warp 0     producer: TMA loads of key tiles (and of the gathered pivot rows for sweep 2) into two
-//              shared-memory rings, one per sweep, so that each ring has exactly one consumer role and
-//              no role ever skips a barrier phase; L2 evict_last on the first read, evict_first on the second
+// Per CTA (320 threads):
+//   warp 0     producer: TMA loads of key tiles into two shared-memory rings, one per sweep, so that
+//              each ring has exactly one consumer role and no role ever skips a barrier phase; for
+//              sweep 2 it also loads the sample's pivot rows (one-row TMA boxes straight from the key
+//              tensor).  L2 evict_last on the first read of a tile, evict_first on the second.
 //   warp 1     sweep 2: one thread issues tcgen05.mma (tokens = M 128, pivots = N, bf16 -> fp32 in TMEM)
-//   warps 2-5  sweep 1: each thread owns one tile row and sums it from shared memory;
-//              sweep 2: read the accumulators out of TMEM and store the partial dot products;
-//              the CTA that completes a row tile adds up its column-slab partials, the CTA that
-//              completes a sample selects the pivots (Def. 1) and publishes them.
-// A task covers 512 of the d columns; the per-slab partial sums are added in slab order by a single
-// thread per row, so every result is bitwise reproducible.
+//   warps 2-5  workers.  Sweep 1: each thread owns one tile row and sums it from shared memory.
+//              Sweep 2: read the accumulators out of TMEM and store the partial dot products.
+//   warps 6-9  control: everything that needs a global-memory round trip, fed by a mailbox so that the
+//              workers never wait for it: counts finished column slabs; the CTA that delivers a row
+//              tile's last slab adds the slab partials up (fixed order) and leaves the tile's P best
+//              (score, index) candidates; the CTA that delivers a sample's last row tile merges the
+//              candidates into the pivots (Def. 1) and publishes them.
+// Every result is bitwise reproducible: partial sums are added in slab order by one thread per row.
 //
 // Every wait (mbarrier or global flag) is bounded in time; on expiry the kernel records
 // DART_ERR_TIMEOUT in the status word, drains and exits normally.
@@ -35,32 +38,38 @@ constexpr int kTileRows = 128;
 constexpr int kAtomCols = 64;  // 64 bf16 = 128 bytes = one swizzle row
 constexpr int kSubRows = 32;   // rows per TMA box of the key tensor
 constexpr int kSlabAtoms = 8;  // a task spans 8 atoms = 512 columns
-constexpr int kMaxStages = 8; // per ring; fewer when many pivots make the sweep-2 stages large
+constexpr int kMaxStages = 8;  // per ring; fewer when many pivots make the sweep-2 stages large
 constexpr int kAtomBytes = kTileRows * 128; // 16 KB: 128 rows x 128 bytes, 128B-swizzled, K-major
 constexpr int kSubBytes = kSubRows * 128;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
 constexpr int kWorkerWarp0 = 2, kWorkerWarps = 4, kWorkers = kWorkerWarps * 32;
-constexpr int kMaxN = 256; // pivots per MMA (N dimension)
+constexpr int kCtrlWarp0 = 6, kCtrlWarps = 4, kCtrl = kCtrlWarps * 32;
+constexpr int kMaxN = 256;      // pivots per MMA (N dimension)
+constexpr int kMail = 8;        // mailbox slots between workers and control warps
+constexpr int kMergeMax = 1024; // candidates merged in shared memory; beyond that a radix select over all scores
+constexpr int kStaticSmemReserve = 12288;
 constexpr int kStatusTimeout = -7;
 // which wait expired (second status word)
-enum { kWaitPivots = 1, kWaitEmptyStage, kWaitDrain, kWaitAccumFree, kWaitStageMma, kWaitStageRows, kWaitAccumFull };
+enum { kWaitPivots = 1, kWaitEmptyStage, kWaitDrain, kWaitAccumFree, kWaitStageMma, kWaitStageRows, kWaitAccumFull,
+       kWaitMailSlot, kWaitMail };
 
 using Workers = WarpGroup<kWorkerWarp0, kWorkerWarps, 1>;
+using Control = WarpGroup<kCtrlWarp0, kCtrlWarps, 2>;
 
 struct Params {
     int B, S, vis_offset, n_vis, P, N; // N = P rounded up to a multiple of 16 (MMA N)
+    int Pc;                            // candidates a row tile leaves: min(P, 128)
     int d8;                            // row width in 16-byte units
     int n_atoms, KS, n_rt, T;          // atoms per row; column slabs; row tiles per sample; tasks per sample and sweep
     int n1, n2;                        // depth of the sweep-1 and of the sweep-2 ring (<= kMaxStages each)
     long long lag;                     // tasks between a task's first and second sweep (T <= lag <= B * T)
     int norm_kind, smallest;
     unsigned long long wait_ns;        // time limit of every wait
-    const uint4 *keys;
     float *pl1, *pssq;                 // [B][KS][n_vis] per-slab partial sums
     float *psim;                       // [B][KS][n_vis][P] per-slab partial dot products
     float *l1, *ssq;                   // [B][n_vis]
+    unsigned long long *cand;          // [B][n_rt][Pc] best (key, index) pairs of every row tile, best first
     int32_t *pivot_idx;                // [B][P]
-    uint4 *pivK;                       // [B][N][d8] pivot rows gathered for the MMA's B operand
     int *rt_done;                      // [B][n_rt] column slabs finished per row tile
     int *s1_done;                      // [B] row tiles finished per sample
     int *piv_ready;                    // [B] 1 once the pivots of the sample are published
@@ -103,12 +112,6 @@ __device__ __forceinline__ int slab_atoms(const Params &p, int ks) { return min(
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *ptr) { return (uint32_t)__cvta_generic_to_shared(ptr); }
-__device__ __forceinline__ unsigned long long now_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
@@ -154,16 +157,19 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
-// OR of a predicate over the worker warps; doubles as their barrier
-__device__ __forceinline__ bool workers_any(bool pred)
+// OR of a predicate over a 128-thread warp group; doubles as the group's barrier
+template <int kBarrierId>
+__device__ __forceinline__ bool group_any(bool pred)
 {
     uint32_t r;
-    asm volatile("{\n.reg .pred p, q;\nsetp.ne.u32 q, %1, 0;\nbar.red.or.pred p, 1, %2, q;\nselp.u32 %0, 1, 0, p;\n}"
+    asm volatile("{\n.reg .pred p, q;\nsetp.ne.u32 q, %1, 0;\nbar.red.or.pred p, %2, 128, q;\nselp.u32 %0, 1, 0, p;\n}"
                  : "=r"(r)
-                 : "r"((uint32_t)pred), "n"(kWorkers)
+                 : "r"((uint32_t)pred), "n"(kBarrierId)
                  : "memory");
     return r != 0;
 }
+__device__ __forceinline__ bool workers_any(bool pred) { return group_any<1>(pred); }
+__device__ __forceinline__ bool control_any(bool pred) { return group_any<2>(pred); }
 
 // Shared-memory matrix descriptor of a K-major, 128B-swizzled bf16 tile (rows at a 128-byte pitch,
 // groups of 8 rows 1024 bytes apart).
@@ -209,7 +215,7 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float *v)
 struct Ctl {
     volatile int *abort_flag; // shared memory
     int *status;              // global status word
-    unsigned long long limit_ns;
+    unsigned long long limit_cycles; // SM clock cycles (the clock runs at <= 2.1 GHz)
     __device__ __forceinline__ bool aborted() const { return *abort_flag != 0; }
     // records the first wait that expired: status[1] = where (kWait*), status[2] = task index, status[3] = CTA
     __device__ void give_up(int where, long long task) const
@@ -221,15 +227,18 @@ struct Ctl {
             status[3] = (int)blockIdx.x;
         }
     }
+    // Waits poll without any bookkeeping first; only a wait that lasts starts reading the SM's cycle
+    // counter (cheap, unlike the global nanosecond timer) and compares it with the limit.
     __device__ bool wait_bar(uint32_t bar, uint32_t parity, int where, long long task) const
     {
-        if (mbar_try_wait(bar, parity)) return true;
-        const unsigned long long t0 = now_ns();
+        for (int it = 0; it < 64; ++it)
+            if (mbar_try_wait(bar, parity)) return true;
+        const long long t0 = clock64();
         for (uint32_t it = 0;; ++it) {
             if (mbar_try_wait(bar, parity)) return true;
-            if ((it & 15u) == 15u) {
+            if ((it & 31u) == 31u) {
                 if (aborted()) return false;
-                if (now_ns() - t0 > limit_ns) {
+                if ((unsigned long long)(clock64() - t0) > limit_cycles) {
                     give_up(where, task);
                     return false;
                 }
@@ -238,14 +247,17 @@ struct Ctl {
     }
     __device__ bool wait_flag(const int *flag, int where, long long task) const
     {
-        if (ld_acquire(flag) != 0) return true;
-        const unsigned long long t0 = now_ns();
+        for (int it = 0; it < 16; ++it) {
+            if (ld_acquire(flag) != 0) return true;
+            __nanosleep(32);
+        }
+        const long long t0 = clock64();
         for (uint32_t it = 0;; ++it) {
             if (ld_acquire(flag) != 0) return true;
             __nanosleep(64);
             if ((it & 15u) == 15u) {
                 if (aborted()) return false;
-                if (now_ns() - t0 > limit_ns) {
+                if ((unsigned long long)(clock64() - t0) > limit_cycles) {
                     give_up(where, task);
                     return false;
                 }
@@ -259,11 +271,10 @@ struct Ring {
     int stage = 0;
     uint32_t phase = 0;
     __device__ explicit Ring(int d) : depth(d) {}
-    __device__ __forceinline__ void advance(int n = 1)
+    __device__ __forceinline__ void advance()
     {
-        stage += n;
-        while (stage >= depth) {
-            stage -= depth;
+        if (++stage == depth) {
+            stage = 0;
             phase ^= 1u;
         }
     }
@@ -271,18 +282,26 @@ struct Ring {
 
 struct Shared {
     unsigned long long full1[kMaxStages], empty1[kMaxStages], full2[kMaxStages], empty2[kMaxStages];
-    unsigned long long tmem_full[2], tmem_empty[2];
-    unsigned long long piv_list[kMaxN];
-    SelectSmem sel;
+    unsigned long long tmem_full[2], tmem_empty[2], mail_full[kMail], mail_empty[kMail];
+    int4 mail[kMail]; // (sample, row tile, column slab, valid rows); sample < 0 ends the stream
+    union {
+        unsigned long long cand[kMergeMax]; // candidate merge
+        struct {
+            SelectSmem sel; // radix-select path for very many pivots
+            unsigned long long list[kMaxN];
+        } rs;
+    } u;
+    unsigned long long ckey[kTileRows]; // (key, index) of the rows of the tile being finalised
     uint32_t tmem_base, n_picked;
-    int abort_flag, bcast;
+    int abort_flag, bcast, bcast2;
 };
+static_assert(sizeof(Shared) + 64 <= kStaticSmemReserve, "static shared memory exceeds its reserve");
 
 __host__ __device__ inline uint32_t b_stage_bytes(int N) { return (uint32_t)((N * 128 + 1023) / 1024 * 1024); }
 // Ring depths for a shared-memory budget: half of it to the sweep-2 ring (at least 2 stages), the rest to sweep 1.
 __host__ inline void ring_depths(int N, size_t smem_limit, int &n1, int &n2)
 {
-    const size_t budget = smem_limit - 1024 - 8192; // alignment slack; 8 KB left for static shared memory
+    const size_t budget = smem_limit - 1024 - kStaticSmemReserve; // alignment slack and static shared memory
     const size_t s2 = kAtomBytes + b_stage_bytes(N);
     size_t b = budget / 2 / s2;
     b = b < 2 ? 2 : (b > (size_t)kMaxStages ? (size_t)kMaxStages : b);
@@ -296,76 +315,117 @@ __host__ inline size_t smem_bytes(int N, int n1, int n2)
     return 1024 + (size_t)n1 * kAtomBytes + (size_t)n2 * (kAtomBytes + b_stage_bytes(N));
 }
 
-// The sample finisher (worker warps): pivots of sample b (Def. 1) and their rows gathered for sweep 2.
-__device__ void select_pivots(const Params &p, Shared &sh, int b)
+// (key, index) composite of a score: smaller composite = better pivot, equal scores -> lower index first
+__device__ __forceinline__ unsigned long long pivot_key(const Params &p, float score, int j)
 {
-    const Workers g;
+    const uint32_t k = order_key(score);
+    return ((unsigned long long)(p.smallest ? k : ~k) << 32) | (uint32_t)j;
+}
+
+// Control warps, row tile (b, rt) complete: add up the slab partials of every row in slab order, store the
+// final sums, and leave the tile's Pc best candidates, best first.
+__device__ void finalize_row_tile(const Params &p, Shared &sh, int b, int rt, int rows)
+{
+    const Control g;
+    const int r = g.tid(), j = rt * kTileRows + r;
+    unsigned long long mine = ~0ull;
+    if (r < rows) {
+        float s1 = 0.f, s2 = 0.f;
+        for (int k0 = 0; k0 < p.KS; k0 += 8) {
+            float a[8], q[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const size_t o = ((size_t)b * p.KS + min(k0 + k, p.KS - 1)) * p.n_vis + j;
+                a[k] = __ldcg(p.pl1 + o);
+                q[k] = __ldcg(p.pssq + o);
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (k0 + k < p.KS) {
+                    s1 += a[k];
+                    s2 += q[k];
+                }
+        }
+        p.l1[(size_t)b * p.n_vis + j] = s1;
+        p.ssq[(size_t)b * p.n_vis + j] = s2;
+        mine = pivot_key(p, p.norm_kind == 2 ? s2 : s1, j);
+    }
+    sh.ckey[r] = mine;
+    g.sync();
+    int rank = 0;
+#pragma unroll 8
+    for (int i = 0; i < kTileRows; ++i) rank += (sh.ckey[i] < mine) ? 1 : 0;
+    unsigned long long *dst = p.cand + ((size_t)b * p.n_rt + rt) * p.Pc;
+    if (r < rows) {
+        if (rank < p.Pc) dst[rank] = mine;
+    } else if (r < p.Pc) {
+        dst[r] = ~0ull; // a short tile has fewer rows than candidate slots: slots rows..Pc-1 stay empty
+    }
+}
+
+// Control warps, sample b complete: pivots (Def. 1) = the P best of the row tiles' candidates, in rank order.
+__device__ void merge_pivots(const Params &p, Shared &sh, int b)
+{
+    const Control g;
     const int tid = g.tid();
-    const float *score = (p.norm_kind == 2 ? p.ssq : p.l1) + (size_t)b * p.n_vis;
-    const int smallest = p.smallest;
-    auto keyfn = [&](int j, uint32_t &key) {
-        uint32_t k = order_key(__ldcg(score + j));
-        key = smallest ? k : ~k; // smaller key = better pivot
-        return true;
-    };
-    int P_pad = 1;
-    while (P_pad < p.P) P_pad <<= 1;
-    for (int i = tid; i < P_pad; i += kWorkers) sh.piv_list[i] = ~0ull;
-    if (tid == 0) sh.n_picked = 0;
-    uint32_t T, need_eq, cnt_eq;
-    block_select_threshold(g, keyfn, p.n_vis, (uint32_t)p.P, sh.sel, T, need_eq, cnt_eq);
-    block_select_apply(g, keyfn, p.n_vis, T, need_eq, cnt_eq, sh.sel, [&](int j, uint32_t key) {
-        uint32_t slot = atomicAdd(&sh.n_picked, 1u);
-        sh.piv_list[slot] = ((unsigned long long)key << 32) | (uint32_t)j;
-    });
-    for (int k = 2; k <= P_pad; k <<= 1) {
-        for (int jj = k >> 1; jj > 0; jj >>= 1) {
-            for (int i = tid; i < P_pad; i += kWorkers) {
-                int l = i ^ jj;
-                if (l > i) {
-                    unsigned long long x = sh.piv_list[i], y = sh.piv_list[l];
-                    bool up = ((i & k) == 0);
-                    if ((x > y) == up) {
-                        sh.piv_list[i] = y;
-                        sh.piv_list[l] = x;
+    const int C = p.n_rt * p.Pc;
+    if (C <= kMergeMax) {
+        const unsigned long long *src = p.cand + (size_t)b * C;
+        for (int i = tid; i < C; i += kCtrl) sh.u.cand[i] = __ldcg(src + i);
+        g.sync();
+        for (int i = tid; i < C; i += kCtrl) {
+            const unsigned long long mine = sh.u.cand[i];
+            if (mine == ~0ull) continue;
+            int rank = 0;
+#pragma unroll 8
+            for (int k = 0; k < C; ++k) rank += (sh.u.cand[k] < mine) ? 1 : 0;
+            if (rank < p.P) p.pivot_idx[(size_t)b * p.P + rank] = (int32_t)(mine & 0xffffffffu);
+        }
+    } else {
+        // very many pivots: radix select over all scores of the sample, then sort the winners
+        const float *score = (p.norm_kind == 2 ? p.ssq : p.l1) + (size_t)b * p.n_vis;
+        const int smallest = p.smallest;
+        auto keyfn = [&](int j, uint32_t &key) {
+            uint32_t k = order_key(__ldcg(score + j));
+            key = smallest ? k : ~k;
+            return true;
+        };
+        int P_pad = 1;
+        while (P_pad < p.P) P_pad <<= 1;
+        for (int i = tid; i < P_pad; i += kCtrl) sh.u.rs.list[i] = ~0ull;
+        if (tid == 0) sh.n_picked = 0;
+        uint32_t T, need_eq, cnt_eq;
+        block_select_threshold(g, keyfn, p.n_vis, (uint32_t)p.P, sh.u.rs.sel, T, need_eq, cnt_eq);
+        block_select_apply(g, keyfn, p.n_vis, T, need_eq, cnt_eq, sh.u.rs.sel, [&](int j, uint32_t key) {
+            uint32_t slot = atomicAdd(&sh.n_picked, 1u);
+            if (slot < (uint32_t)kMaxN) sh.u.rs.list[slot] = ((unsigned long long)key << 32) | (uint32_t)j;
+        });
+        for (int k = 2; k <= P_pad; k <<= 1) {
+            for (int jj = k >> 1; jj > 0; jj >>= 1) {
+                for (int i = tid; i < P_pad; i += kCtrl) {
+                    int l = i ^ jj;
+                    if (l > i) {
+                        unsigned long long x = sh.u.rs.list[i], y = sh.u.rs.list[l];
+                        bool up = ((i & k) == 0);
+                        if ((x > y) == up) {
+                            sh.u.rs.list[i] = y;
+                            sh.u.rs.list[l] = x;
+                        }
                     }
                 }
-            }
-            g.sync();
-        }
-    }
-    for (int i = tid; i < p.P; i += kWorkers) p.pivot_idx[(size_t)b * p.P + i] = (int32_t)(sh.piv_list[i] & 0xffffffffu);
-    // gather the pivot rows (rows >= P of the N-row block keep whatever finite data they hold: their
-    // accumulator columns are never read)
-    const uint4 *base = p.keys + ((size_t)b * p.S + p.vis_offset) * (size_t)p.d8;
-    uint4 *dst = p.pivK + (size_t)b * p.N * p.d8;
-    const int total = p.P * p.d8;
-    for (int i0 = tid; i0 < total; i0 += kWorkers * 8) {
-        uint4 v[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            int i = i0 + u * kWorkers;
-            if (i < total) {
-                int r = i / p.d8, c = i - r * p.d8;
-                const uint32_t pr = min((uint32_t)(sh.piv_list[r] & 0xffffffffu), (uint32_t)(p.n_vis - 1));
-                v[u] = __ldcg(base + (size_t)pr * p.d8 + c);
+                g.sync();
             }
         }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            int i = i0 + u * kWorkers;
-            if (i < total) dst[i] = v[u];
-        }
+        for (int i = tid; i < p.P; i += kCtrl)
+            p.pivot_idx[(size_t)b * p.P + i] = (int32_t)min((uint32_t)(sh.u.rs.list[i] & 0xffffffffu), (uint32_t)(p.n_vis - 1));
     }
-    // make the rows visible to other SMs' TMA reads, then publish
-    asm volatile("fence.proxy.async.global;" ::: "memory");
     __threadfence();
     g.sync();
     if (tid == 0) st_release(p.piv_ready + b, 1);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant__ CUtensorMap tm_piv, const Params p)
+sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant__ CUtensorMap tm_row, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ Shared sh;
@@ -376,8 +436,9 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
     auto a2_addr = [&](int s) { return smem0 + (uint32_t)(p.n1 + s) * kAtomBytes; };
     auto b2_addr = [&](int s) { return smem0 + (uint32_t)(p.n1 + p.n2) * kAtomBytes + (uint32_t)s * bstage; };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned long long limit = 2ull * p.wait_ns; // ns -> cycles at the highest SM clock: never shorter than asked
     // consumers get a longer limit than the producer, so that the wait nearest the cause reports first
-    const Ctl ctl{&sh.abort_flag, p.status, warp == 0 ? p.wait_ns : p.wait_ns + p.wait_ns / 4};
+    const Ctl ctl{&sh.abort_flag, p.status, warp == 0 ? limit : limit + limit / 4};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
@@ -389,6 +450,10 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&sh.tmem_full[a]), 1);
             mbar_init(smem_u32(&sh.tmem_empty[a]), kWorkerWarps);
+        }
+        for (int m = 0; m < kMail; ++m) {
+            mbar_init(smem_u32(&sh.mail_full[m]), 1);
+            mbar_init(smem_u32(&sh.mail_empty[m]), 1);
         }
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -408,57 +473,73 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
     const long long total = total_tasks(p);
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ producer
-        if (lane == 0) {
-            unsigned long long pol_keep, pol_drop;
-            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
-            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_drop));
-            Ring r1(p.n1), r2(p.n2);
-            long long issued1 = 0, issued2 = 0;
-            bool ok = true;
-            for (long long g = blockIdx.x; ok && g < total; g += gridDim.x) {
-                const Task t = decode(p, g);
-                if (t.kind == 1) {
+        // ------------------------------------------------------------------ producer (whole warp; lane 0 waits)
+        unsigned long long pol_keep, pol_drop;
+        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_drop));
+        Ring r1(p.n1), r2(p.n2);
+        long long issued1 = 0, issued2 = 0;
+        bool ok = true;
+        int cur_b = -1;
+        int my_piv[kMaxN / 32]; // pivot rows this lane loads: ranks lane, lane + 32, ...
+        for (long long g = blockIdx.x; ok && g < total; g += gridDim.x) {
+            const Task t = decode(p, g);
+            if (t.kind == 1 && t.b != cur_b) {
+                if (lane == 0) {
                     ok = ctl.wait_flag(p.piv_ready + t.b, kWaitPivots, g);
-                    if (!ok) {
-                        if (p.status[1] == kWaitPivots && p.status[3] == (int)blockIdx.x) {
-                            p.status[4] = t.b;
-                            p.status[5] = ld_acquire(p.s1_done + t.b);
-                            for (int r = 0; r < 6 && r < p.n_rt; ++r)
-                                p.status[6 + r] = ld_acquire(p.rt_done + (size_t)t.b * p.n_rt + r);
-                        }
-                        break;
+                    if (!ok && p.status[1] == kWaitPivots && p.status[3] == (int)blockIdx.x) {
+                        p.status[4] = t.b;
+                        p.status[5] = ld_acquire(p.s1_done + t.b);
+                        for (int r = 0; r < 6 && r < p.n_rt; ++r)
+                            p.status[6 + r] = ld_acquire(p.rt_done + (size_t)t.b * p.n_rt + r);
                     }
-                    asm volatile("fence.proxy.async.global;" ::: "memory");
                 }
-                const int na = slab_atoms(p, t.ks);
-                const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
-                const int n_sub = (rows + kSubRows - 1) / kSubRows;
-                const int y0 = t.b * p.S + p.vis_offset + t.rt * kTileRows;
-                Ring &ring = t.kind ? r2 : r1;
-                for (int a = 0; a < na; ++a) {
-                    const uint32_t empty = smem_u32(t.kind ? &sh.empty2[ring.stage] : &sh.empty1[ring.stage]);
-                    const uint32_t full = smem_u32(t.kind ? &sh.full2[ring.stage] : &sh.full1[ring.stage]);
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                if (!ok) break;
+#pragma unroll
+                for (int k = 0; k < kMaxN / 32; ++k) {
+                    const int i = lane + 32 * k;
+                    my_piv[k] = i < p.P ? min(max(__ldcg(p.pivot_idx + (size_t)t.b * p.P + i), 0), p.n_vis - 1) : 0;
+                }
+                cur_b = t.b;
+            }
+            const int na = slab_atoms(p, t.ks);
+            const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
+            const int n_sub = (rows + kSubRows - 1) / kSubRows;
+            const int yb = t.b * p.S + p.vis_offset, y0 = yb + t.rt * kTileRows;
+            Ring &ring = t.kind ? r2 : r1;
+            for (int a = 0; a < na; ++a) {
+                const uint32_t empty = smem_u32(t.kind ? &sh.empty2[ring.stage] : &sh.empty1[ring.stage]);
+                const uint32_t full = smem_u32(t.kind ? &sh.full2[ring.stage] : &sh.full1[ring.stage]);
+                if (lane == 0) {
                     ok = ctl.wait_bar(empty, ring.phase ^ 1u, kWaitEmptyStage, g);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(full, (uint32_t)n_sub * kSubBytes + (t.kind ? (uint32_t)p.N * 128u : 0u));
-                    const int x = (t.ks * kSlabAtoms + a) * kAtomCols;
-                    const uint32_t dst = t.kind ? a2_addr(ring.stage) : a1_addr(ring.stage);
-                    for (int s = 0; s < n_sub; ++s)
-                        tma_load_2d(dst + (uint32_t)s * kSubBytes, &tm_keys, x, y0 + s * kSubRows, full,
-                                    t.kind ? pol_drop : pol_keep);
-                    if (t.kind) tma_load_2d(b2_addr(ring.stage), &tm_piv, x, t.b * p.N, full, pol_keep);
-                    ring.advance();
-                    ++(t.kind ? issued2 : issued1);
+                    if (ok) mbar_arrive_expect_tx(full, (uint32_t)n_sub * kSubBytes + (t.kind ? (uint32_t)p.P * 128u : 0u));
                 }
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                if (!ok) break;
+                const int x = (t.ks * kSlabAtoms + a) * kAtomCols;
+                const uint32_t dst = t.kind ? a2_addr(ring.stage) : a1_addr(ring.stage);
+                if (lane < n_sub)
+                    tma_load_2d(dst + (uint32_t)lane * kSubBytes, &tm_keys, x, y0 + lane * kSubRows, full,
+                                t.kind ? pol_drop : pol_keep);
+                if (t.kind) {
+#pragma unroll
+                    for (int k = 0; k < kMaxN / 32; ++k) {
+                        const int i = lane + 32 * k;
+                        if (i < p.P) // pivot row of rank i -> row i of the B tile (one-row box; the swizzle follows the address)
+                            tma_load_2d(b2_addr(ring.stage) + (uint32_t)i * 128u, &tm_row, x, yb + my_piv[k], full, pol_keep);
+                    }
+                }
+                ring.advance();
+                ++(t.kind ? issued2 : issued1);
             }
-            if (!ok) {
-                // drain: let the copies already issued land before the CTA may exit
-                for (long long i = issued1 > p.n1 ? issued1 - p.n1 : 0; i < issued1; ++i)
-                    ctl.wait_bar(smem_u32(&sh.full1[i % p.n1]), (uint32_t)((i / p.n1) & 1), kWaitDrain, i);
-                for (long long i = issued2 > p.n2 ? issued2 - p.n2 : 0; i < issued2; ++i)
-                    ctl.wait_bar(smem_u32(&sh.full2[i % p.n2]), (uint32_t)((i / p.n2) & 1), kWaitDrain, i);
-            }
+        }
+        if (!ok && lane == 0) {
+            // drain: let the copies already issued land before the CTA may exit
+            for (long long i = issued1 > p.n1 ? issued1 - p.n1 : 0; i < issued1; ++i)
+                ctl.wait_bar(smem_u32(&sh.full1[i % p.n1]), (uint32_t)((i / p.n1) & 1), kWaitDrain, i);
+            for (long long i = issued2 > p.n2 ? issued2 - p.n2 : 0; i < issued2; ++i)
+                ctl.wait_bar(smem_u32(&sh.full2[i % p.n2]), (uint32_t)((i / p.n2) & 1), kWaitDrain, i);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ sweep-2 MMA issuer
@@ -469,8 +550,8 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
             bool ok = true;
             for (long long g = blockIdx.x; ok && g < total; g += gridDim.x) {
                 const Task t = decode(p, g);
-                const int na = slab_atoms(p, t.ks);
                 if (t.kind == 0) continue;
+                const int na = slab_atoms(p, t.ks);
                 const uint32_t acc = s2n & 1u;
                 ok = ctl.wait_bar(smem_u32(&sh.tmem_empty[acc]), ((s2n >> 1) & 1u) ^ 1u, kWaitAccumFree, g);
                 if (!ok) break;
@@ -493,20 +574,29 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
                 ++s2n;
             }
         }
-    } else {
+    } else if (warp < kCtrlWarp0) {
         // ------------------------------------------------------------------ workers
         const int wt = threadIdx.x - kWorkerWarp0 * 32;      // 0..127
         const int quarter = warp & 3;                        // TMEM lane quarter this warp may read
         const int row = quarter * 32 + lane;                 // tile row owned by this thread
         Ring ring(p.n1);
-        uint32_t s2n = 0;
+        int ms = 0;
+        uint32_t mph = 0, s2n = 0;
         bool dead = false; // group-uniform after every workers_any()
+        auto post = [&](int4 m) { // thread wt == 0: hand a finished slab (or the end mark) to the control warps
+            bool ok = ctl.wait_bar(smem_u32(&sh.mail_empty[ms]), mph ^ 1u, kWaitMailSlot, 0);
+            if (ok) {
+                sh.mail[ms] = m;
+                mbar_arrive(smem_u32(&sh.mail_full[ms])); // release: the group's partial sums are ordered before it
+            }
+            return ok;
+        };
         for (long long g = blockIdx.x; g < total; g += gridDim.x) {
             const Task t = decode(p, g);
-            const int na = slab_atoms(p, t.ks);
             const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
             const int j = t.rt * kTileRows + row;
             if (t.kind == 0) {
+                const int na = slab_atoms(p, t.ks);
                 float a0 = 0.f, a1 = 0.f, q0 = 0.f, q1 = 0.f;
                 for (int a = 0; a < na; ++a) {
                     bool fail = dead;
@@ -537,37 +627,12 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
                     p.pl1[o] = a0 + a1;
                     p.pssq[o] = q0 + q1;
                 }
-                // count the slab; the CTA that delivers a row tile's last slab adds up the partials
-                __threadfence();
-                dead = workers_any(dead);
-                if (wt == 0) {
-                    int old = dead ? -1 : atomicAdd(p.rt_done + (size_t)t.b * p.n_rt + t.rt, 1);
-                    __threadfence();
-                    sh.bcast = old;
+                dead = workers_any(dead); // every worker's partial sums are issued
+                if (!dead && wt == 0 && !post(make_int4(t.b, t.rt, t.ks, rows))) dead = true;
+                if (++ms == kMail) {
+                    ms = 0;
+                    mph ^= 1u;
                 }
-                dead = workers_any(dead);
-                if (!dead && sh.bcast == p.KS - 1) {
-                    if (row < rows) {
-                        float s1 = 0.f, s2 = 0.f;
-                        for (int ks = 0; ks < p.KS; ++ks) {
-                            const size_t o = ((size_t)t.b * p.KS + ks) * p.n_vis + j;
-                            s1 += __ldcg(p.pl1 + o);
-                            s2 += __ldcg(p.pssq + o);
-                        }
-                        p.l1[(size_t)t.b * p.n_vis + j] = s1;
-                        p.ssq[(size_t)t.b * p.n_vis + j] = s2;
-                    }
-                    __threadfence();
-                    workers_any(false);
-                    if (wt == 0) {
-                        int old = atomicAdd(p.s1_done + t.b, 1);
-                        __threadfence();
-                        sh.bcast = old;
-                    }
-                    workers_any(false);
-                    if (sh.bcast == p.n_rt - 1) select_pivots(p, sh, t.b);
-                }
-                workers_any(false); // sh.bcast may be rewritten by the next task only after everyone has read it
             } else {
                 if (dead) continue;
                 const uint32_t acc = s2n & 1u;
@@ -599,6 +664,46 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
                 }
                 ++s2n;
             }
+        }
+        workers_any(dead);
+        if (wt == 0) post(make_int4(-1, 0, 0, 0)); // end of the stream (also after a failure, so that control exits)
+    } else {
+        // ------------------------------------------------------------------ control
+        const Control cg;
+        const int ct = cg.tid();
+        int mi = 0;
+        uint32_t mph = 0;
+        for (;;) {
+            bool fail = !ctl.wait_bar(smem_u32(&sh.mail_full[mi]), mph, kWaitMail, 0);
+            if (control_any(fail)) break;
+            const int4 m = sh.mail[mi];
+            cg.sync(); // everyone has read the slot
+            if (ct == 0) mbar_arrive(smem_u32(&sh.mail_empty[mi]));
+            if (++mi == kMail) {
+                mi = 0;
+                mph ^= 1u;
+            }
+            if (m.x < 0) break;
+            if (ct == 0) {
+                __threadfence(); // the workers' partial sums (ordered before the mail) become visible GPU-wide
+                const int old = atomicAdd(p.rt_done + (size_t)m.x * p.n_rt + m.y, 1);
+                __threadfence();
+                sh.bcast = old;
+            }
+            cg.sync();
+            if (sh.bcast == p.KS - 1) {
+                finalize_row_tile(p, sh, m.x, m.y, m.w);
+                __threadfence();
+                cg.sync();
+                if (ct == 0) {
+                    const int old = atomicAdd(p.s1_done + m.x, 1);
+                    __threadfence();
+                    sh.bcast2 = old;
+                }
+                cg.sync();
+                if (sh.bcast2 == p.n_rt - 1) merge_pivots(p, sh, m.x);
+            }
+            cg.sync(); // sh.bcast is rewritten only after everyone has read it
         }
     }
     // ---------------------------------------------------------------------- teardown
