@@ -301,22 +301,25 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     const long long n_all = (long long)B * p.T;
     // a row's second sweep follows its first by one sample plus the time the pivots take to appear
     long long lag = (long long)p.T + (o.sweep_lag > 0 ? o.sweep_lag : 3 * ctx->sm_count);
-    p.lag = lag < n_all ? lag : n_all;
+    if (2 * n_all >= (1ll << 31)) return DART_ERR_UNSUPPORTED;
+    p.lag = (uint32_t)(lag < n_all ? lag : n_all);
     p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
     p.pl1 = ctx->pl1, p.pssq = ctx->pssq, p.psim = ctx->psim, p.l1 = ctx->l1, p.ssq = ctx->ssq;
     p.pivot_idx = ctx->pivot_idx, p.cand = ctx->cand;
     p.rt_done = ctx->counters, p.s1_done = ctx->counters + (size_t)B * p.n_rt, p.piv_ready = p.s1_done + B;
     p.status = ctx->status;
-    CUtensorMap tm_keys, tm_row; // the same tensor with a 32-row box (tiles) and a one-row box (pivot rows)
-    int rc = encode_2d(ctx, &tm_keys, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, kSubRows);
+    // the same tensor with a 128-row box (full tiles), a 32-row box (short last tiles) and a one-row box (pivot rows)
+    CUtensorMap tm_tile, tm_keys, tm_row;
+    int rc = encode_2d(ctx, &tm_tile, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, kTileRows);
+    if (rc == DART_OK) rc = encode_2d(ctx, &tm_keys, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, kSubRows);
     if (rc == DART_OK) rc = encode_2d(ctx, &tm_row, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, 1);
     if (rc != DART_OK) return rc;
     DART_CUDA(ctx, cudaMemsetAsync(ctx->counters, 0, (size_t)B * (p.n_rt + 2) * sizeof(int), st));
     {
         Prof pr(ctx, st, SLOT_SWEEP);
         long long grid = 2 * n_all < ctx->sm_count ? 2 * n_all : ctx->sm_count;
-        void *args[3] = {&tm_keys, &tm_row, &p};
+        void *args[4] = {&tm_tile, &tm_keys, &tm_row, &p};
         DART_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)sweep_kernel, dim3((unsigned)grid), dim3(kThreads), args,
                                                    smem_bytes(p.N, p.n1, p.n2), st));
     }

@@ -62,7 +62,7 @@ struct Params {
     int d8;                            // row width in 16-byte units
     int n_atoms, KS, n_rt, T;          // atoms per row; column slabs; row tiles per sample; tasks per sample and sweep
     int n1, n2;                        // depth of the sweep-1 and of the sweep-2 ring (<= kMaxStages each)
-    long long lag;                     // tasks between a task's first and second sweep (T <= lag <= B * T)
+    uint32_t lag;                      // tasks between a task's first and second sweep (T <= lag <= B * T)
     int norm_kind, smallest;
     unsigned long long wait_ns;        // time limit of every wait
     float *pl1, *pssq;                 // [B][KS][n_vis] per-slab partial sums
@@ -81,30 +81,32 @@ struct Task {
     int b, rt, ks;
 };
 
-__device__ __forceinline__ long long total_tasks(const Params &p) { return 2ll * p.B * p.T; }
+// the host guarantees 2 * B * T < 2^31, so task indices fit 32 bits
+__device__ __forceinline__ uint32_t total_tasks(const Params &p) { return 2u * (uint32_t)p.B * (uint32_t)p.T; }
 
-__device__ __forceinline__ Task decode(const Params &p, long long g)
+__device__ __forceinline__ Task decode(const Params &p, uint32_t g)
 {
     // order: sweep-1 tasks [0, lag) alone; then pairs (sweep-1 task lag + k, sweep-2 task k); then the
     // last `lag` sweep-2 tasks alone
-    const long long n_all = (long long)p.B * p.T, head = p.lag, mid = 2 * (n_all - p.lag);
+    const uint32_t n_all = (uint32_t)p.B * (uint32_t)p.T, head = p.lag, mid = 2u * (n_all - p.lag);
     Task t;
-    long long n;
+    uint32_t n;
     if (g < head) {
         t.kind = 0;
         n = g;
     } else if (g < head + mid) {
-        const long long h = g - head;
-        t.kind = (int)(h & 1);
+        const uint32_t h = g - head;
+        t.kind = (int)(h & 1u);
         n = t.kind ? (h >> 1) : (h >> 1) + p.lag;
     } else {
         t.kind = 1;
         n = n_all - p.lag + (g - head - mid);
     }
-    t.b = (int)(n / p.T);
-    const int u = (int)(n % p.T);
-    t.rt = u / p.KS;
-    t.ks = u % p.KS;
+    const uint32_t T = (uint32_t)p.T, KS = (uint32_t)p.KS;
+    t.b = (int)(n / T);
+    const uint32_t u = n - (uint32_t)t.b * T;
+    t.rt = (int)(u / KS);
+    t.ks = (int)(u - (uint32_t)t.rt * KS);
     return t;
 }
 
@@ -139,6 +141,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm,
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
                  " [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
                  "l"(tm), "r"(x), "r"(y), "r"(bar), "l"(policy)
+                 : "memory");
+}
+// Four rows (given by index) x one box width of columns -> four consecutive 128-byte rows at dst.
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap *tm, int x, int r0, int r1, int r2, int r3,
+                                            uint32_t bar, unsigned long long policy)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes.L2::cache_hint"
+                 " [%0], [%1, {%2, %3, %4, %5, %6}], [%7], %8;" ::"r"(dst),
+                 "l"(tm), "r"(x), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar), "l"(policy)
                  : "memory");
 }
 __device__ __forceinline__ int ld_acquire(const int *ptr)
@@ -425,7 +436,8 @@ __device__ void merge_pivots(const Params &p, Shared &sh, int b)
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant__ CUtensorMap tm_row, const Params p)
+sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant__ CUtensorMap tm_keys,
+             const __grid_constant__ CUtensorMap tm_row, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ Shared sh;
@@ -470,7 +482,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = sh.tmem_base;
-    const long long total = total_tasks(p);
+    const uint32_t total = total_tasks(p);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer (whole warp; lane 0 waits)
@@ -481,8 +493,8 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
         long long issued1 = 0, issued2 = 0;
         bool ok = true;
         int cur_b = -1;
-        int my_piv[kMaxN / 32]; // pivot rows this lane loads: ranks lane, lane + 32, ...
-        for (long long g = blockIdx.x; ok && g < total; g += gridDim.x) {
+        int my_piv[kMaxN / 128][4]; // lane l loads pivot ranks 4l..4l+3, 4(l+32).., as rows of the key tensor
+        for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
             const Task t = decode(p, g);
             if (t.kind == 1 && t.b != cur_b) {
                 if (lane == 0) {
@@ -497,37 +509,46 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
                 ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
                 if (!ok) break;
 #pragma unroll
-                for (int k = 0; k < kMaxN / 32; ++k) {
-                    const int i = lane + 32 * k;
-                    my_piv[k] = i < p.P ? min(max(__ldcg(p.pivot_idx + (size_t)t.b * p.P + i), 0), p.n_vis - 1) : 0;
-                }
+                for (int k = 0; k < kMaxN / 128; ++k)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int i = min(4 * (lane + 32 * k) + e, p.P - 1); // ranks beyond P repeat the last pivot
+                        const int piv = min(max(__ldcg(p.pivot_idx + (size_t)t.b * p.P + i), 0), p.n_vis - 1);
+                        my_piv[k][e] = t.b * p.S + p.vis_offset + piv;
+                    }
                 cur_b = t.b;
             }
             const int na = slab_atoms(p, t.ks);
             const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
             const int n_sub = (rows + kSubRows - 1) / kSubRows;
-            const int yb = t.b * p.S + p.vis_offset, y0 = yb + t.rt * kTileRows;
+            const int y0 = t.b * p.S + p.vis_offset + t.rt * kTileRows;
             Ring &ring = t.kind ? r2 : r1;
             for (int a = 0; a < na; ++a) {
                 const uint32_t empty = smem_u32(t.kind ? &sh.empty2[ring.stage] : &sh.empty1[ring.stage]);
                 const uint32_t full = smem_u32(t.kind ? &sh.full2[ring.stage] : &sh.full1[ring.stage]);
                 if (lane == 0) {
                     ok = ctl.wait_bar(empty, ring.phase ^ 1u, kWaitEmptyStage, g);
-                    if (ok) mbar_arrive_expect_tx(full, (uint32_t)n_sub * kSubBytes + (t.kind ? (uint32_t)p.P * 128u : 0u));
+                    if (ok)
+                        mbar_arrive_expect_tx(full, (rows == kTileRows ? (uint32_t)kAtomBytes : (uint32_t)n_sub * kSubBytes) +
+                                                        (t.kind ? (uint32_t)((p.P + 3) / 4) * 512u : 0u));
                 }
                 ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
                 if (!ok) break;
                 const int x = (t.ks * kSlabAtoms + a) * kAtomCols;
                 const uint32_t dst = t.kind ? a2_addr(ring.stage) : a1_addr(ring.stage);
-                if (lane < n_sub)
+                if (rows == kTileRows) { // a full tile is one 128-row box; a short last tile is 32-row boxes
+                    if (lane == 0) tma_load_2d(dst, &tm_tile, x, y0, full, t.kind ? pol_drop : pol_keep);
+                } else if (lane < n_sub) {
                     tma_load_2d(dst + (uint32_t)lane * kSubBytes, &tm_keys, x, y0 + lane * kSubRows, full,
                                 t.kind ? pol_drop : pol_keep);
+                }
                 if (t.kind) {
 #pragma unroll
-                    for (int k = 0; k < kMaxN / 32; ++k) {
-                        const int i = lane + 32 * k;
-                        if (i < p.P) // pivot row of rank i -> row i of the B tile (one-row box; the swizzle follows the address)
-                            tma_load_2d(b2_addr(ring.stage) + (uint32_t)i * 128u, &tm_row, x, yb + my_piv[k], full, pol_keep);
+                    for (int k = 0; k < kMaxN / 128; ++k) {
+                        const int q = lane + 32 * k; // pivot ranks 4q..4q+3 -> rows 4q..4q+3 of the B tile
+                        if (4 * q < p.P)
+                            tma_gather4(b2_addr(ring.stage) + (uint32_t)q * 512u, &tm_row, x, my_piv[k][0], my_piv[k][1],
+                                        my_piv[k][2], my_piv[k][3], full, pol_keep);
                     }
                 }
                 ring.advance();
@@ -548,7 +569,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
             Ring ring(p.n2);
             uint32_t s2n = 0;
             bool ok = true;
-            for (long long g = blockIdx.x; ok && g < total; g += gridDim.x) {
+            for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
                 const Task t = decode(p, g);
                 if (t.kind == 0) continue;
                 const int na = slab_atoms(p, t.ks);
@@ -591,7 +612,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_keys, const __grid_constant_
             }
             return ok;
         };
-        for (long long g = blockIdx.x; g < total; g += gridDim.x) {
+        for (uint32_t g = blockIdx.x; g < total; g += gridDim.x) {
             const Task t = decode(p, g);
             const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
             const int j = t.rt * kTileRows + row;
