@@ -301,8 +301,8 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     const long long n_all = (long long)B * p.T;
     // a row's second sweep follows its first by one sample plus the time the pivots take to appear
     long long lag = (long long)p.T + (o.sweep_lag > 0 ? o.sweep_lag : 3 * ctx->sm_count);
-    if (2 * n_all >= (1ll << 31)) return DART_ERR_UNSUPPORTED;
     p.lag = (uint32_t)(lag < n_all ? lag : n_all);
+    if (n_all + p.lag >= (1ll << 30)) return DART_ERR_UNSUPPORTED;
     p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
     p.pl1 = ctx->pl1, p.pssq = ctx->pssq, p.psim = ctx->psim, p.l1 = ctx->l1, p.ssq = ctx->ssq;
@@ -318,7 +318,7 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     DART_CUDA(ctx, cudaMemsetAsync(ctx->counters, 0, (size_t)B * (p.n_rt + 2) * sizeof(int), st));
     {
         Prof pr(ctx, st, SLOT_SWEEP);
-        long long grid = 2 * n_all < ctx->sm_count ? 2 * n_all : ctx->sm_count;
+        long long grid = n_all < ctx->sm_count ? n_all : ctx->sm_count;
         void *args[4] = {&tm_tile, &tm_keys, &tm_row, &p};
         DART_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)sweep_kernel, dim3((unsigned)grid), dim3(kThreads), args,
                                                    smem_bytes(p.N, p.n1, p.n2), st));

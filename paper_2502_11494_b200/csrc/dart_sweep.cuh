@@ -51,7 +51,7 @@ constexpr int kStaticSmemReserve = 12288;
 constexpr int kStatusTimeout = -7;
 // which wait expired (second status word)
 enum { kWaitPivots = 1, kWaitEmptyStage, kWaitDrain, kWaitAccumFree, kWaitStageMma, kWaitStageRows, kWaitAccumFull,
-       kWaitMailSlot, kWaitMail };
+       kWaitMailSlot, kWaitMail, kWaitSlabs, kWaitRowTiles };
 
 using Workers = WarpGroup<kWorkerWarp0, kWorkerWarps, 1>;
 using Control = WarpGroup<kCtrlWarp0, kCtrlWarps, 2>;
@@ -81,33 +81,24 @@ struct Task {
     int b, rt, ks;
 };
 
-// the host guarantees 2 * B * T < 2^31, so task indices fit 32 bits
-__device__ __forceinline__ uint32_t total_tasks(const Params &p) { return 2u * (uint32_t)p.B * (uint32_t)p.T; }
+// Schedule.  Step q of the global order is the pair (sweep-1 task q, sweep-2 task q - lag); CTA c runs steps
+// c, c + grid, ... and, within a step, the sweep-1 task first.  So every CTA alternates between the two kinds
+// of task, and a sweep-2 task comes `lag` steps after the sweep-1 task of the same tile (lag >= T, hence after
+// the whole sample has been scored).  The host guarantees B * T + lag < 2^31.
+__device__ __forceinline__ uint32_t total_steps(const Params &p) { return (uint32_t)p.B * (uint32_t)p.T + p.lag; }
 
-__device__ __forceinline__ Task decode(const Params &p, uint32_t g)
+// kind 0: sweep-1 task of step q; kind 1: its sweep-2 task.  Returns false if the step has no such task.
+__device__ __forceinline__ bool decode(const Params &p, uint32_t q, int kind, Task &t)
 {
-    // order: sweep-1 tasks [0, lag) alone; then pairs (sweep-1 task lag + k, sweep-2 task k); then the
-    // last `lag` sweep-2 tasks alone
-    const uint32_t n_all = (uint32_t)p.B * (uint32_t)p.T, head = p.lag, mid = 2u * (n_all - p.lag);
-    Task t;
-    uint32_t n;
-    if (g < head) {
-        t.kind = 0;
-        n = g;
-    } else if (g < head + mid) {
-        const uint32_t h = g - head;
-        t.kind = (int)(h & 1u);
-        n = t.kind ? (h >> 1) : (h >> 1) + p.lag;
-    } else {
-        t.kind = 1;
-        n = n_all - p.lag + (g - head - mid);
-    }
-    const uint32_t T = (uint32_t)p.T, KS = (uint32_t)p.KS;
+    const uint32_t n_all = (uint32_t)p.B * (uint32_t)p.T;
+    if (kind == 0 ? q >= n_all : q < p.lag) return false;
+    const uint32_t n = kind ? q - p.lag : q, T = (uint32_t)p.T, KS = (uint32_t)p.KS;
+    t.kind = kind;
     t.b = (int)(n / T);
     const uint32_t u = n - (uint32_t)t.b * T;
     t.rt = (int)(u / KS);
     t.ks = (int)(u - (uint32_t)t.rt * KS);
-    return t;
+    return true;
 }
 
 __device__ __forceinline__ int slab_atoms(const Params &p, int ks) { return min(kSlabAtoms, p.n_atoms - ks * kSlabAtoms); }
@@ -256,15 +247,16 @@ struct Ctl {
             }
         }
     }
-    __device__ bool wait_flag(const int *flag, int where, long long task) const
+    // waits until *flag >= target
+    __device__ bool wait_flag(const int *flag, int where, long long task, int target = 1) const
     {
         for (int it = 0; it < 16; ++it) {
-            if (ld_acquire(flag) != 0) return true;
+            if (ld_acquire(flag) >= target) return true;
             __nanosleep(32);
         }
         const long long t0 = clock64();
         for (uint32_t it = 0;; ++it) {
-            if (ld_acquire(flag) != 0) return true;
+            if (ld_acquire(flag) >= target) return true;
             __nanosleep(64);
             if ((it & 15u) == 15u) {
                 if (aborted()) return false;
@@ -304,7 +296,7 @@ struct Shared {
     } u;
     unsigned long long ckey[kTileRows]; // (key, index) of the rows of the tile being finalised
     uint32_t tmem_base, n_picked;
-    int abort_flag, bcast, bcast2;
+    int abort_flag;
 };
 static_assert(sizeof(Shared) + 64 <= kStaticSmemReserve, "static shared memory exceeds its reserve");
 
@@ -482,7 +474,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = sh.tmem_base;
-    const uint32_t total = total_tasks(p);
+    const uint32_t total = total_steps(p);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer (whole warp; lane 0 waits)
@@ -494,8 +486,9 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
         bool ok = true;
         int cur_b = -1;
         int my_piv[kMaxN / 128][4]; // lane l loads pivot ranks 4l..4l+3, 4(l+32).., as rows of the key tensor
-        for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
-            const Task t = decode(p, g);
+        for (uint32_t g = blockIdx.x * 2; ok && g < 2 * total; g = (g & 1u) ? g + 2 * gridDim.x - 1 : g + 1) {
+            Task t; // g = 2 * step + kind
+            if (!decode(p, g >> 1, (int)(g & 1u), t)) continue;
             if (t.kind == 1 && t.b != cur_b) {
                 if (lane == 0) {
                     ok = ctl.wait_flag(p.piv_ready + t.b, kWaitPivots, g);
@@ -570,8 +563,8 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             uint32_t s2n = 0;
             bool ok = true;
             for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
-                const Task t = decode(p, g);
-                if (t.kind == 0) continue;
+                Task t;
+                if (!decode(p, g, 1, t)) continue;
                 const int na = slab_atoms(p, t.ks);
                 const uint32_t acc = s2n & 1u;
                 ok = ctl.wait_bar(smem_u32(&sh.tmem_empty[acc]), ((s2n >> 1) & 1u) ^ 1u, kWaitAccumFree, g);
@@ -612,8 +605,9 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             }
             return ok;
         };
-        for (uint32_t g = blockIdx.x; g < total; g += gridDim.x) {
-            const Task t = decode(p, g);
+        for (uint32_t g = blockIdx.x * 2; g < 2 * total; g = (g & 1u) ? g + 2 * gridDim.x - 1 : g + 1) {
+            Task t; // g = 2 * step + kind
+            if (!decode(p, g >> 1, (int)(g & 1u), t)) continue;
             const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
             const int j = t.rt * kTileRows + row;
             if (t.kind == 0) {
@@ -655,7 +649,11 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                     mph ^= 1u;
                 }
             } else {
-                if (dead) continue;
+                // warp-uniform: after a failed post only one lane knows, and the code below is warp-collective
+                if (__any_sync(0xffffffffu, dead || ctl.aborted())) {
+                    dead = true;
+                    continue;
+                }
                 const uint32_t acc = s2n & 1u;
                 bool ok = ctl.wait_bar(smem_u32(&sh.tmem_full[acc]), (s2n >> 1) & 1u, kWaitAccumFull, g);
                 ok = __all_sync(0xffffffffu, ok);
@@ -705,26 +703,31 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                 mph ^= 1u;
             }
             if (m.x < 0) break;
+            // Who finalises is fixed by the schedule, not by arrival order: the CTA that holds slab
+            // (b + rt) % KS of a row tile finalises it, and the one that finalises a sample's LAST row tile
+            // merges the sample, so that it only ever waits for work that precedes its own in the schedule
+            // (its own later mails can then never be what it waits for).  Letting the last arriver do it
+            // instead makes a busy control group ever later, hence ever last.
+            int *slabs = p.rt_done + (size_t)m.x * p.n_rt + m.y;
+            const bool fin_tile = m.z == (m.x + m.y) % p.KS, fin_sample = fin_tile && m.y == p.n_rt - 1;
+            bool late = false;
             if (ct == 0) {
                 __threadfence(); // the workers' partial sums (ordered before the mail) become visible GPU-wide
-                const int old = atomicAdd(p.rt_done + (size_t)m.x * p.n_rt + m.y, 1);
-                __threadfence();
-                sh.bcast = old;
+                atomicAdd(slabs, 1);
+                if (fin_tile) late = !ctl.wait_flag(slabs, kWaitSlabs, m.x, p.KS);
             }
-            cg.sync();
-            if (sh.bcast == p.KS - 1) {
+            if (control_any(late)) break;
+            if (fin_tile) {
                 finalize_row_tile(p, sh, m.x, m.y, m.w);
                 __threadfence();
                 cg.sync();
                 if (ct == 0) {
-                    const int old = atomicAdd(p.s1_done + m.x, 1);
-                    __threadfence();
-                    sh.bcast2 = old;
+                    atomicAdd(p.s1_done + m.x, 1);
+                    if (fin_sample) late = !ctl.wait_flag(p.s1_done + m.x, kWaitRowTiles, m.x, p.n_rt);
                 }
-                cg.sync();
-                if (sh.bcast2 == p.n_rt - 1) merge_pivots(p, sh, m.x);
+                if (control_any(late)) break;
+                if (fin_sample) merge_pivots(p, sh, m.x);
             }
-            cg.sync(); // sh.bcast is rewritten only after everyone has read it
         }
     }
     // ---------------------------------------------------------------------- teardown
