@@ -9,11 +9,12 @@
 // c, c + grid, c + 2 grid, ...  Because a task is only 128 KB, all SMs together hold < 20 MB in
 // flight, and the distance between the two reads of a row is the sample size plus the lag.
 //
-// Per CTA (320 threads):
-//   warp 0     producer: TMA loads of key tiles into two shared-memory rings, one per sweep, so that
-//              each ring has exactly one consumer role and no role ever skips a barrier phase; for
-//              sweep 2 it also loads the sample's pivot rows (one-row TMA boxes straight from the key
-//              tensor).  L2 evict_last on the first read of a tile, evict_first on the second.
+// Per CTA (352 threads):
+//   warp 0     sweep-1 producer and warp 10 sweep-2 producer: TMA loads of key tiles into two
+//              shared-memory rings, one per sweep, each with its own producer and exactly one consumer
+//              role, so that neither sweep blocks the other and no role ever skips a barrier phase; the
+//              sweep-2 producer also gathers the sample's pivot rows (tile::gather4 boxes straight from
+//              the key tensor).  L2 evict_last on the first read of a tile, evict_first on the second.
 //   warp 1     sweep 2: one thread issues tcgen05.mma (tokens = M 128, pivots = N, bf16 -> fp32 in TMEM)
 //   warps 2-5  workers.  Sweep 1: each thread owns one tile row and sums it from shared memory.
 //              Sweep 2: read the accumulators out of TMEM and store the partial dot products.
@@ -41,9 +42,10 @@ constexpr int kSlabAtoms = 8;  // a task spans 8 atoms = 512 columns
 constexpr int kMaxStages = 8;  // per ring; fewer when many pivots make the sweep-2 stages large
 constexpr int kAtomBytes = kTileRows * 128; // 16 KB: 128 rows x 128 bytes, 128B-swizzled, K-major
 constexpr int kSubBytes = kSubRows * 128;
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;
 constexpr int kWorkerWarp0 = 2, kWorkerWarps = 4, kWorkers = kWorkerWarps * 32;
 constexpr int kCtrlWarp0 = 6, kCtrlWarps = 4, kCtrl = kCtrlWarps * 32;
+constexpr int kProducer2Warp = 10;
 constexpr int kMaxN = 256;      // pivots per MMA (N dimension)
 constexpr int kMail = 8;        // mailbox slots between workers and control warps
 constexpr int kMergeMax = 1024; // candidates merged in shared memory; beyond that a radix select over all scores
@@ -442,12 +444,12 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned long long limit = 2ull * p.wait_ns; // ns -> cycles at the highest SM clock: never shorter than asked
     // consumers get a longer limit than the producer, so that the wait nearest the cause reports first
-    const Ctl ctl{&sh.abort_flag, p.status, warp == 0 ? limit : limit + limit / 4};
+    const Ctl ctl{&sh.abort_flag, p.status, (warp == 0 || warp == kProducer2Warp) ? limit : limit + limit / 4};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(smem_u32(&sh.full1[s]), 1);
-            mbar_init(smem_u32(&sh.empty1[s]), 1);
+            mbar_init(smem_u32(&sh.empty1[s]), kWorkerWarps); // every worker warp releases a stage by itself
             mbar_init(smem_u32(&sh.full2[s]), 1);
             mbar_init(smem_u32(&sh.empty2[s]), 1);
         }
@@ -477,19 +479,55 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
     const uint32_t total = total_steps(p);
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ producer (whole warp; lane 0 waits)
+        // ------------------------------------------------------------------ sweep-1 producer (lane 0 waits, lanes issue)
+        unsigned long long pol_keep;
+        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+        Ring ring(p.n1);
+        long long issued = 0;
+        bool ok = true;
+        for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
+            Task t;
+            if (!decode(p, g, 0, t)) continue;
+            const int na = slab_atoms(p, t.ks);
+            const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
+            const int n_sub = (rows + kSubRows - 1) / kSubRows;
+            const int y0 = t.b * p.S + p.vis_offset + t.rt * kTileRows;
+            for (int a = 0; a < na; ++a) {
+                const uint32_t full = smem_u32(&sh.full1[ring.stage]);
+                if (lane == 0) {
+                    ok = ctl.wait_bar(smem_u32(&sh.empty1[ring.stage]), ring.phase ^ 1u, kWaitEmptyStage, g);
+                    if (ok) mbar_arrive_expect_tx(full, rows == kTileRows ? (uint32_t)kAtomBytes : (uint32_t)n_sub * kSubBytes);
+                }
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                if (!ok) break;
+                const int x = (t.ks * kSlabAtoms + a) * kAtomCols;
+                const uint32_t dst = a1_addr(ring.stage);
+                if (rows == kTileRows) { // a full tile is one 128-row box; a short last tile is 32-row boxes
+                    if (lane == 0) tma_load_2d(dst, &tm_tile, x, y0, full, pol_keep);
+                } else if (lane < n_sub) {
+                    tma_load_2d(dst + (uint32_t)lane * kSubBytes, &tm_keys, x, y0 + lane * kSubRows, full, pol_keep);
+                }
+                ring.advance();
+                ++issued;
+            }
+        }
+        if (!ok && lane == 0) // drain: let the copies already issued land before the CTA may exit
+            for (long long i = issued > p.n1 ? issued - p.n1 : 0; i < issued; ++i)
+                ctl.wait_bar(smem_u32(&sh.full1[i % p.n1]), (uint32_t)((i / p.n1) & 1), kWaitDrain, i);
+    } else if (warp == kProducer2Warp) {
+        // ------------------------------------------------------------------ sweep-2 producer
         unsigned long long pol_keep, pol_drop;
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_drop));
-        Ring r1(p.n1), r2(p.n2);
-        long long issued1 = 0, issued2 = 0;
+        Ring ring(p.n2);
+        long long issued = 0;
         bool ok = true;
         int cur_b = -1;
         int my_piv[kMaxN / 128][4]; // lane l loads pivot ranks 4l..4l+3, 4(l+32).., as rows of the key tensor
-        for (uint32_t g = blockIdx.x * 2; ok && g < 2 * total; g = (g & 1u) ? g + 2 * gridDim.x - 1 : g + 1) {
-            Task t; // g = 2 * step + kind
-            if (!decode(p, g >> 1, (int)(g & 1u), t)) continue;
-            if (t.kind == 1 && t.b != cur_b) {
+        for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
+            Task t;
+            if (!decode(p, g, 1, t)) continue;
+            if (t.b != cur_b) {
                 if (lane == 0) {
                     ok = ctl.wait_flag(p.piv_ready + t.b, kWaitPivots, g);
                     if (!ok && p.status[1] == kWaitPivots && p.status[3] == (int)blockIdx.x) {
@@ -515,46 +553,37 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
             const int n_sub = (rows + kSubRows - 1) / kSubRows;
             const int y0 = t.b * p.S + p.vis_offset + t.rt * kTileRows;
-            Ring &ring = t.kind ? r2 : r1;
             for (int a = 0; a < na; ++a) {
-                const uint32_t empty = smem_u32(t.kind ? &sh.empty2[ring.stage] : &sh.empty1[ring.stage]);
-                const uint32_t full = smem_u32(t.kind ? &sh.full2[ring.stage] : &sh.full1[ring.stage]);
+                const uint32_t full = smem_u32(&sh.full2[ring.stage]);
                 if (lane == 0) {
-                    ok = ctl.wait_bar(empty, ring.phase ^ 1u, kWaitEmptyStage, g);
+                    ok = ctl.wait_bar(smem_u32(&sh.empty2[ring.stage]), ring.phase ^ 1u, kWaitEmptyStage, g);
                     if (ok)
                         mbar_arrive_expect_tx(full, (rows == kTileRows ? (uint32_t)kAtomBytes : (uint32_t)n_sub * kSubBytes) +
-                                                        (t.kind ? (uint32_t)((p.P + 3) / 4) * 512u : 0u));
+                                                        (uint32_t)((p.P + 3) / 4) * 512u);
                 }
                 ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
                 if (!ok) break;
                 const int x = (t.ks * kSlabAtoms + a) * kAtomCols;
-                const uint32_t dst = t.kind ? a2_addr(ring.stage) : a1_addr(ring.stage);
-                if (rows == kTileRows) { // a full tile is one 128-row box; a short last tile is 32-row boxes
-                    if (lane == 0) tma_load_2d(dst, &tm_tile, x, y0, full, t.kind ? pol_drop : pol_keep);
+                const uint32_t dst = a2_addr(ring.stage);
+                if (rows == kTileRows) {
+                    if (lane == 0) tma_load_2d(dst, &tm_tile, x, y0, full, pol_drop);
                 } else if (lane < n_sub) {
-                    tma_load_2d(dst + (uint32_t)lane * kSubBytes, &tm_keys, x, y0 + lane * kSubRows, full,
-                                t.kind ? pol_drop : pol_keep);
+                    tma_load_2d(dst + (uint32_t)lane * kSubBytes, &tm_keys, x, y0 + lane * kSubRows, full, pol_drop);
                 }
-                if (t.kind) {
 #pragma unroll
-                    for (int k = 0; k < kMaxN / 128; ++k) {
-                        const int q = lane + 32 * k; // pivot ranks 4q..4q+3 -> rows 4q..4q+3 of the B tile
-                        if (4 * q < p.P)
-                            tma_gather4(b2_addr(ring.stage) + (uint32_t)q * 512u, &tm_row, x, my_piv[k][0], my_piv[k][1],
-                                        my_piv[k][2], my_piv[k][3], full, pol_keep);
-                    }
+                for (int k = 0; k < kMaxN / 128; ++k) {
+                    const int q = lane + 32 * k; // pivot ranks 4q..4q+3 -> rows 4q..4q+3 of the B tile
+                    if (4 * q < p.P)
+                        tma_gather4(b2_addr(ring.stage) + (uint32_t)q * 512u, &tm_row, x, my_piv[k][0], my_piv[k][1],
+                                    my_piv[k][2], my_piv[k][3], full, pol_keep);
                 }
                 ring.advance();
-                ++(t.kind ? issued2 : issued1);
+                ++issued;
             }
         }
-        if (!ok && lane == 0) {
-            // drain: let the copies already issued land before the CTA may exit
-            for (long long i = issued1 > p.n1 ? issued1 - p.n1 : 0; i < issued1; ++i)
-                ctl.wait_bar(smem_u32(&sh.full1[i % p.n1]), (uint32_t)((i / p.n1) & 1), kWaitDrain, i);
-            for (long long i = issued2 > p.n2 ? issued2 - p.n2 : 0; i < issued2; ++i)
+        if (!ok && lane == 0)
+            for (long long i = issued > p.n2 ? issued - p.n2 : 0; i < issued; ++i)
                 ctl.wait_bar(smem_u32(&sh.full2[i % p.n2]), (uint32_t)((i / p.n2) & 1), kWaitDrain, i);
-        }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ sweep-2 MMA issuer
         if (lane == 0) {
@@ -588,7 +617,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                 ++s2n;
             }
         }
-    } else if (warp < kCtrlWarp0) {
+    } else if (warp >= kWorkerWarp0 && warp < kCtrlWarp0) {
         // ------------------------------------------------------------------ workers
         const int wt = threadIdx.x - kWorkerWarp0 * 32;      // 0..127
         const int quarter = warp & 3;                        // TMEM lane quarter this warp may read
@@ -614,9 +643,10 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                 const int na = slab_atoms(p, t.ks);
                 float a0 = 0.f, a1 = 0.f, q0 = 0.f, q1 = 0.f;
                 for (int a = 0; a < na; ++a) {
-                    bool fail = dead;
-                    if (!fail) fail = !ctl.wait_bar(smem_u32(&sh.full1[ring.stage]), ring.phase, kWaitStageRows, g);
-                    if (!fail && row < rows) {
+                    // warp-uniform: either the whole warp reads the stage and releases it, or none of it does
+                    if (!dead) dead = !ctl.wait_bar(smem_u32(&sh.full1[ring.stage]), ring.phase, kWaitStageRows, g);
+                    dead = __any_sync(0xffffffffu, dead);
+                    if (!dead && row < rows) {
                         const uint32_t base = a1_addr(ring.stage) + (uint32_t)row * 128u;
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
@@ -633,8 +663,8 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                             }
                         }
                     }
-                    dead = workers_any(fail); // also: every worker has finished reading the stage
-                    if (!dead && wt == 0) mbar_arrive(smem_u32(&sh.empty1[ring.stage]));
+                    __syncwarp(); // the warp's reads of the stage are done
+                    if (!dead && lane == 0) mbar_arrive(smem_u32(&sh.empty1[ring.stage]));
                     ring.advance();
                 }
                 if (!dead && row < rows) {
@@ -686,7 +716,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
         }
         workers_any(dead);
         if (wt == 0) post(make_int4(-1, 0, 0, 0)); // end of the stream (also after a failure, so that control exits)
-    } else {
+    } else if (warp >= kCtrlWarp0 && warp < kCtrlWarp0 + kCtrlWarps) {
         // ------------------------------------------------------------------ control
         const Control cg;
         const int ct = cg.tid();
