@@ -9,16 +9,19 @@
 // c, c + grid, c + 2 grid, ...  Because a task is only 128 KB, all SMs together hold < 20 MB in
 // flight, and the distance between the two reads of a row is the sample size plus the lag.
 //
-// Per CTA (352 threads):
-//   warp 0     sweep-1 producer and warp 10 sweep-2 producer: TMA loads of key tiles into two
+// Per CTA (512 threads; warp 3 idles):
+//   warps 0, 2 sweep-1 producer and sweep-2 producer: TMA loads of key tiles into two
 //              shared-memory rings, one per sweep, each with its own producer and exactly one consumer
 //              role, so that neither sweep blocks the other and no role ever skips a barrier phase; the
 //              sweep-2 producer also gathers the sample's pivot rows (tile::gather4 boxes straight from
 //              the key tensor).  L2 evict_last on the first read of a tile, evict_first on the second.
 //   warp 1     sweep 2: one thread issues tcgen05.mma (tokens = M 128, pivots = N, bf16 -> fp32 in TMEM)
-//   warps 2-5  workers.  Sweep 1: each thread owns one tile row and sums it from shared memory.
-//              Sweep 2: read the accumulators out of TMEM and store the partial dot products.
-//   warps 6-9  control: everything that needs a global-memory round trip, fed by a mailbox so that the
+//   warps 4-7  sweep-1 workers: each thread owns one tile row and sums it from shared memory.
+//   warps 8-11 sweep-2 epilogue: read the accumulators out of TMEM and store the partial dot products
+//              (separate from the workers so that neither sweep ever waits for the other; the sweep-1
+//              producer only stays within one round of the CTA's sweep-2 progress, which bounds the
+//              distance between the two reads of a tile).
+//   warps 12-15 control: everything that needs a global-memory round trip, fed by a mailbox so that the
 //              workers never wait for it: counts finished column slabs; the CTA that delivers a row
 //              tile's last slab adds the slab partials up (fixed order) and leaves the tile's P best
 //              (score, index) candidates; the CTA that delivers a sample's last row tile merges the
@@ -42,10 +45,11 @@ constexpr int kSlabAtoms = 8;  // a task spans 8 atoms = 512 columns
 constexpr int kMaxStages = 8;  // per ring; fewer when many pivots make the sweep-2 stages large
 constexpr int kAtomBytes = kTileRows * 128; // 16 KB: 128 rows x 128 bytes, 128B-swizzled, K-major
 constexpr int kSubBytes = kSubRows * 128;
-constexpr int kThreads = 352;
-constexpr int kWorkerWarp0 = 2, kWorkerWarps = 4, kWorkers = kWorkerWarps * 32;
-constexpr int kCtrlWarp0 = 6, kCtrlWarps = 4, kCtrl = kCtrlWarps * 32;
-constexpr int kProducer2Warp = 10;
+constexpr int kThreads = 512;
+constexpr int kWorkerWarp0 = 4, kWorkerWarps = 4, kWorkers = kWorkerWarps * 32;
+constexpr int kEpiWarp0 = 8, kEpiWarps = 4; // kEpiWarp0 % 4 == 0: warp w reads TMEM lanes 32 (w % 4) ...
+constexpr int kCtrlWarp0 = 12, kCtrlWarps = 4, kCtrl = kCtrlWarps * 32;
+constexpr int kProducer2Warp = 2;
 constexpr int kMaxN = 256;      // pivots per MMA (N dimension)
 constexpr int kMail = 8;        // mailbox slots between workers and control warps
 constexpr int kMergeMax = 1024; // candidates merged in shared memory; beyond that a radix select over all scores
@@ -53,7 +57,7 @@ constexpr int kStaticSmemReserve = 12288;
 constexpr int kStatusTimeout = -7;
 // which wait expired (second status word)
 enum { kWaitPivots = 1, kWaitEmptyStage, kWaitDrain, kWaitAccumFree, kWaitStageMma, kWaitStageRows, kWaitAccumFull,
-       kWaitMailSlot, kWaitMail, kWaitSlabs, kWaitRowTiles };
+       kWaitMailSlot, kWaitMail, kWaitSlabs, kWaitRowTiles, kWaitSweep2 };
 
 using Workers = WarpGroup<kWorkerWarp0, kWorkerWarps, 1>;
 using Control = WarpGroup<kCtrlWarp0, kCtrlWarps, 2>;
@@ -249,6 +253,23 @@ struct Ctl {
             }
         }
     }
+    // waits until a shared-memory counter reaches target
+    __device__ bool wait_count(const volatile int *cnt, int target, int where, long long task) const
+    {
+        if (*cnt >= target) return true;
+        const long long t0 = clock64();
+        for (uint32_t it = 0;; ++it) {
+            if (*cnt >= target) return true;
+            __nanosleep(64);
+            if ((it & 15u) == 15u) {
+                if (aborted()) return false;
+                if ((unsigned long long)(clock64() - t0) > limit_cycles) {
+                    give_up(where, task);
+                    return false;
+                }
+            }
+        }
+    }
     // waits until *flag >= target
     __device__ bool wait_flag(const int *flag, int where, long long task, int target = 1) const
     {
@@ -299,6 +320,7 @@ struct Shared {
     unsigned long long ckey[kTileRows]; // (key, index) of the rows of the tile being finalised
     uint32_t tmem_base, n_picked;
     int abort_flag;
+    volatile int s2_step; // last schedule step whose sweep-2 task this CTA has finished (-1: none yet)
 };
 static_assert(sizeof(Shared) + 64 <= kStaticSmemReserve, "static shared memory exceeds its reserve");
 
@@ -455,13 +477,14 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&sh.tmem_full[a]), 1);
-            mbar_init(smem_u32(&sh.tmem_empty[a]), kWorkerWarps);
+            mbar_init(smem_u32(&sh.tmem_empty[a]), kEpiWarps);
         }
         for (int m = 0; m < kMail; ++m) {
             mbar_init(smem_u32(&sh.mail_full[m]), 1);
             mbar_init(smem_u32(&sh.mail_empty[m]), 1);
         }
         sh.abort_flag = 0;
+        sh.s2_step = -1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     uint32_t tmem_cols = 32;
@@ -488,6 +511,13 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
         for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
             Task t;
             if (!decode(p, g, 0, t)) continue;
+            // stay within one round of this CTA's sweep-2 progress: the step one round back has a sweep-2
+            // task if it is >= lag, and that task must be finished before more tiles are pulled in
+            if (g >= gridDim.x && g - gridDim.x >= p.lag) {
+                if (lane == 0) ok = ctl.wait_count(&sh.s2_step, (int)(g - gridDim.x), kWaitSweep2, g);
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                if (!ok) break;
+            }
             const int na = slab_atoms(p, t.ks);
             const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
             const int n_sub = (rows + kSubRows - 1) / kSubRows;
@@ -617,15 +647,14 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                 ++s2n;
             }
         }
-    } else if (warp >= kWorkerWarp0 && warp < kCtrlWarp0) {
-        // ------------------------------------------------------------------ workers
-        const int wt = threadIdx.x - kWorkerWarp0 * 32;      // 0..127
-        const int quarter = warp & 3;                        // TMEM lane quarter this warp may read
-        const int row = quarter * 32 + lane;                 // tile row owned by this thread
+    } else if (warp >= kWorkerWarp0 && warp < kWorkerWarp0 + kWorkerWarps) {
+        // ------------------------------------------------------------------ sweep-1 workers
+        const int wt = threadIdx.x - kWorkerWarp0 * 32; // 0..127 = tile row owned by this thread
+        const int row = wt;
         Ring ring(p.n1);
         int ms = 0;
-        uint32_t mph = 0, s2n = 0;
-        bool dead = false; // group-uniform after every workers_any()
+        uint32_t mph = 0;
+        bool dead = false; // warp-uniform inside a task, group-uniform after every workers_any()
         auto post = [&](int4 m) { // thread wt == 0: hand a finished slab (or the end mark) to the control warps
             bool ok = ctl.wait_bar(smem_u32(&sh.mail_empty[ms]), mph ^ 1u, kWaitMailSlot, 0);
             if (ok) {
@@ -634,88 +663,90 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             }
             return ok;
         };
-        for (uint32_t g = blockIdx.x * 2; g < 2 * total; g = (g & 1u) ? g + 2 * gridDim.x - 1 : g + 1) {
-            Task t; // g = 2 * step + kind
-            if (!decode(p, g >> 1, (int)(g & 1u), t)) continue;
+        for (uint32_t g = blockIdx.x; g < total; g += gridDim.x) {
+            Task t;
+            if (!decode(p, g, 0, t)) continue;
             const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
             const int j = t.rt * kTileRows + row;
-            if (t.kind == 0) {
-                const int na = slab_atoms(p, t.ks);
-                float a0 = 0.f, a1 = 0.f, q0 = 0.f, q1 = 0.f;
-                for (int a = 0; a < na; ++a) {
-                    // warp-uniform: either the whole warp reads the stage and releases it, or none of it does
-                    if (!dead) dead = !ctl.wait_bar(smem_u32(&sh.full1[ring.stage]), ring.phase, kWaitStageRows, g);
-                    dead = __any_sync(0xffffffffu, dead);
-                    if (!dead && row < rows) {
-                        const uint32_t base = a1_addr(ring.stage) + (uint32_t)row * 128u;
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            // logical 16-byte chunk c of this row sits at chunk c ^ (row & 7)
-                            const uint4 v = lds128(base + (uint32_t)((c ^ (row & 7)) << 4));
-                            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const float lo = bf16_lo(w[e]), hi = bf16_hi(w[e]);
-                                a0 += fabsf(lo);
-                                a1 += fabsf(hi);
-                                q0 = fmaf(lo, lo, q0);
-                                q1 = fmaf(hi, hi, q1);
-                            }
-                        }
-                    }
-                    __syncwarp(); // the warp's reads of the stage are done
-                    if (!dead && lane == 0) mbar_arrive(smem_u32(&sh.empty1[ring.stage]));
-                    ring.advance();
-                }
+            const int na = slab_atoms(p, t.ks);
+            float a0 = 0.f, a1 = 0.f, q0 = 0.f, q1 = 0.f;
+            for (int a = 0; a < na; ++a) {
+                // warp-uniform: either the whole warp reads the stage and releases it, or none of it does
+                if (!dead) dead = !ctl.wait_bar(smem_u32(&sh.full1[ring.stage]), ring.phase, kWaitStageRows, g);
+                dead = __any_sync(0xffffffffu, dead);
                 if (!dead && row < rows) {
-                    const size_t o = ((size_t)t.b * p.KS + t.ks) * p.n_vis + j;
-                    p.pl1[o] = a0 + a1;
-                    p.pssq[o] = q0 + q1;
-                }
-                dead = workers_any(dead); // every worker's partial sums are issued
-                if (!dead && wt == 0 && !post(make_int4(t.b, t.rt, t.ks, rows))) dead = true;
-                if (++ms == kMail) {
-                    ms = 0;
-                    mph ^= 1u;
-                }
-            } else {
-                // warp-uniform: after a failed post only one lane knows, and the code below is warp-collective
-                if (__any_sync(0xffffffffu, dead || ctl.aborted())) {
-                    dead = true;
-                    continue;
-                }
-                const uint32_t acc = s2n & 1u;
-                bool ok = ctl.wait_bar(smem_u32(&sh.tmem_full[acc]), (s2n >> 1) & 1u, kWaitAccumFull, g);
-                ok = __all_sync(0xffffffffu, ok);
-                if (ok) {
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t taddr = tmem_base + acc * (uint32_t)p.N + ((uint32_t)(quarter * 32) << 16);
-                    float *dst = p.psim + (((size_t)t.b * p.KS + t.ks) * p.n_vis + j) * p.P;
-                    for (int c0 = 0; c0 < p.P; c0 += 8) {
-                        float v[8];
-                        tmem_ld8(taddr + (uint32_t)c0, v); // warp-collective: rows outside the tile still take part
-                        if (row < rows) {
-                            if (c0 + 8 <= p.P && (p.P & 3) == 0) {
-                                *reinterpret_cast<float4 *>(dst + c0) = make_float4(v[0], v[1], v[2], v[3]);
-                                *reinterpret_cast<float4 *>(dst + c0 + 4) = make_float4(v[4], v[5], v[6], v[7]);
-                            } else {
+                    const uint32_t base = a1_addr(ring.stage) + (uint32_t)row * 128u;
 #pragma unroll
-                                for (int e = 0; e < 8; ++e)
-                                    if (c0 + e < p.P) dst[c0 + e] = v[e];
-                            }
+                    for (int c = 0; c < 8; ++c) {
+                        // logical 16-byte chunk c of this row sits at chunk c ^ (row & 7)
+                        const uint4 v = lds128(base + (uint32_t)((c ^ (row & 7)) << 4));
+                        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float lo = bf16_lo(w[e]), hi = bf16_hi(w[e]);
+                            a0 += fabsf(lo);
+                            a1 += fabsf(hi);
+                            q0 = fmaf(lo, lo, q0);
+                            q1 = fmaf(hi, hi, q1);
                         }
                     }
-                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&sh.tmem_empty[acc]));
-                } else {
-                    dead = true; // reaches the other worker warps at their next group barrier
                 }
-                ++s2n;
+                __syncwarp(); // the warp's reads of the stage are done
+                if (!dead && lane == 0) mbar_arrive(smem_u32(&sh.empty1[ring.stage]));
+                ring.advance();
+            }
+            if (!dead && row < rows) {
+                const size_t o = ((size_t)t.b * p.KS + t.ks) * p.n_vis + j;
+                p.pl1[o] = a0 + a1;
+                p.pssq[o] = q0 + q1;
+            }
+            dead = workers_any(dead); // every worker's partial sums are issued
+            if (!dead && wt == 0 && !post(make_int4(t.b, t.rt, t.ks, rows))) dead = true;
+            if (++ms == kMail) {
+                ms = 0;
+                mph ^= 1u;
             }
         }
         workers_any(dead);
         if (wt == 0) post(make_int4(-1, 0, 0, 0)); // end of the stream (also after a failure, so that control exits)
+    } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
+        // ------------------------------------------------------------------ sweep-2 epilogue (warps independent)
+        const int quarter = warp & 3;        // TMEM lane quarter this warp may read
+        const int row = quarter * 32 + lane; // tile row owned by this thread
+        uint32_t s2n = 0;
+        for (uint32_t g = blockIdx.x; g < total; g += gridDim.x) {
+            Task t;
+            if (!decode(p, g, 1, t)) continue;
+            const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
+            const int j = t.rt * kTileRows + row;
+            const uint32_t acc = s2n & 1u;
+            bool ok = ctl.wait_bar(smem_u32(&sh.tmem_full[acc]), (s2n >> 1) & 1u, kWaitAccumFull, g);
+            if (!__all_sync(0xffffffffu, ok)) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t taddr = tmem_base + acc * (uint32_t)p.N + ((uint32_t)(quarter * 32) << 16);
+            float *dst = p.psim + (((size_t)t.b * p.KS + t.ks) * p.n_vis + j) * p.P;
+            for (int c0 = 0; c0 < p.P; c0 += 8) {
+                float v[8];
+                tmem_ld8(taddr + (uint32_t)c0, v); // warp-collective: rows outside the tile still take part
+                if (row < rows) {
+                    if (c0 + 8 <= p.P && (p.P & 3) == 0) {
+                        *reinterpret_cast<float4 *>(dst + c0) = make_float4(v[0], v[1], v[2], v[3]);
+                        *reinterpret_cast<float4 *>(dst + c0 + 4) = make_float4(v[4], v[5], v[6], v[7]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            if (c0 + e < p.P) dst[c0 + e] = v[e];
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&sh.tmem_empty[acc]));
+                if (quarter == 0) sh.s2_step = (int)g; // progress mark for the sweep-1 producer's throttle
+            }
+            ++s2n;
+        }
     } else if (warp >= kCtrlWarp0 && warp < kCtrlWarp0 + kCtrlWarps) {
         // ------------------------------------------------------------------ control
         const Control cg;
