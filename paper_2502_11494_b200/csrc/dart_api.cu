@@ -54,8 +54,7 @@ struct dart_ctx {
     // fused path (csrc/dart_sweep.cuh); available when d is a multiple of 64 and the device is sm_100
     bool fused_ok;
     int sm_count, KS, n_atoms, N_max;
-    float *pl1, *pssq, *psim;
-    unsigned long long *cand;
+    float *psim;
     int *counters;
     size_t counters_bytes;
     TensorMapEncodeFn encode;
@@ -231,7 +230,8 @@ int fused_setup(dart_ctx *ctx)
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, D.device) != cudaSuccess) return DART_ERR_CUDA;
     ctx->sm_count = prop.multiProcessorCount;
-    if (prop.major != 10 || D.d % kAtomCols != 0 || !prop.cooperativeLaunch) return DART_OK; // staged path only
+    if (prop.major != 10 || D.d % kAtomCols != 0 || D.d * 2 > kMaxRowBytes || !prop.cooperativeLaunch)
+        return DART_OK; // staged path only
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
@@ -243,13 +243,8 @@ int fused_setup(dart_ctx *ctx)
     const int P_cap = D.P_max < kMaxN ? D.P_max : kMaxN;
     ctx->N_max = (P_cap + 15) / 16 * 16;
     const size_t nv = (size_t)D.B_max * D.S_max;
-    const int n_rt_max = (D.S_max + kTileRows - 1) / kTileRows;
-    int rc = ws_alloc(ctx, &ctx->pl1, nv * ctx->KS);
-    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->pssq, nv * ctx->KS);
-    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->psim, nv * ctx->KS * P_cap);
-    const int Pc_max = P_cap < kTileRows ? P_cap : kTileRows;
-    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->cand, (size_t)D.B_max * n_rt_max * Pc_max);
-    ctx->counters_bytes = (size_t)D.B_max * (n_rt_max + 2) * sizeof(int);
+    int rc = ws_alloc(ctx, &ctx->psim, nv * ctx->KS * P_cap);
+    ctx->counters_bytes = (size_t)D.B_max * 2 * sizeof(int);
     if (rc == DART_OK) rc = ws_alloc(ctx, (uint8_t **)&ctx->counters, ctx->counters_bytes);
     if (rc != DART_OK) return rc;
     if (cudaFuncSetAttribute(sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - kStaticSmemReserve) !=
@@ -257,8 +252,10 @@ int fused_setup(dart_ctx *ctx)
         return DART_ERR_CUDA;
     int per_sm = 0;
     int n1 = 0, n2 = 0;
-    ring_depths(16, ctx->max_smem_optin, n1, n2);
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sweep_kernel, kThreads, smem_bytes(16, n1, n2)) !=
+    ring_depths(16, (uint32_t)D.d * 2, ctx->max_smem_optin, n1, n2);
+    if (n1 < 2) return DART_OK;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sweep_kernel, kThreads,
+                                                      smem_bytes(16, (uint32_t)D.d * 2, n1, n2)) !=
             cudaSuccess ||
         per_sm < 1)
         return DART_ERR_CUDA;
@@ -294,20 +291,21 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     const void *keys = keys_in ? keys_in : hidden;
     Params p = {};
     p.B = B, p.S = S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.N = (P + 15) / 16 * 16, p.d8 = d8;
-    p.Pc = P < kTileRows ? P : kTileRows;
-    p.n_atoms = ctx->n_atoms, p.KS = ctx->KS, p.n_rt = (n_vis + kTileRows - 1) / kTileRows, p.T = p.n_rt * p.KS;
-    ring_depths(p.N, ctx->max_smem_optin, p.n1, p.n2);
+    p.n_atoms = ctx->n_atoms, p.KS = ctx->KS, p.n_rt = (n_vis + kTileRows - 1) / kTileRows;
+    p.T1 = (n_vis + kS1Rows - 1) / kS1Rows, p.T2 = p.n_rt * p.KS, p.Tm = p.T1 > p.T2 ? p.T1 : p.T2;
+    p.row_bytes = (uint32_t)ctx->desc.d * 2, p.stage1_bytes = stage1_bytes(p.row_bytes);
+    ring_depths(p.N, p.row_bytes, ctx->max_smem_optin, p.n1, p.n2);
     if (p.n1 < 2) return DART_ERR_UNSUPPORTED;
-    const long long n_all = (long long)B * p.T;
+    const long long n_all = (long long)B * p.Tm;
     // a row's second sweep follows its first by one sample plus the time the pivots take to appear
-    long long lag = (long long)p.T + (o.sweep_lag > 0 ? o.sweep_lag : 3 * ctx->sm_count);
+    long long lag = (long long)p.Tm + (o.sweep_lag > 0 ? o.sweep_lag : 2 * ctx->sm_count);
     p.lag = (uint32_t)(lag < n_all ? lag : n_all);
     if (n_all + p.lag >= (1ll << 30)) return DART_ERR_UNSUPPORTED;
     p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
-    p.pl1 = ctx->pl1, p.pssq = ctx->pssq, p.psim = ctx->psim, p.l1 = ctx->l1, p.ssq = ctx->ssq;
-    p.pivot_idx = ctx->pivot_idx, p.cand = ctx->cand;
-    p.rt_done = ctx->counters, p.s1_done = ctx->counters + (size_t)B * p.n_rt, p.piv_ready = p.s1_done + B;
+    p.keys = (const char *)keys;
+    p.psim = ctx->psim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
+    p.s1_done = ctx->counters, p.piv_ready = ctx->counters + B;
     p.status = ctx->status;
     // the same tensor with a 128-row box (full tiles), a 32-row box (short last tiles) and a one-row box (pivot rows)
     CUtensorMap tm_tile, tm_keys, tm_row;
@@ -315,13 +313,13 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     if (rc == DART_OK) rc = encode_2d(ctx, &tm_keys, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, kSubRows);
     if (rc == DART_OK) rc = encode_2d(ctx, &tm_row, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, 1);
     if (rc != DART_OK) return rc;
-    DART_CUDA(ctx, cudaMemsetAsync(ctx->counters, 0, (size_t)B * (p.n_rt + 2) * sizeof(int), st));
+    DART_CUDA(ctx, cudaMemsetAsync(ctx->counters, 0, (size_t)B * 2 * sizeof(int), st));
     {
         Prof pr(ctx, st, SLOT_SWEEP);
         long long grid = n_all < ctx->sm_count ? n_all : ctx->sm_count;
         void *args[4] = {&tm_tile, &tm_keys, &tm_row, &p};
         DART_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)sweep_kernel, dim3((unsigned)grid), dim3(kThreads), args,
-                                                   smem_bytes(p.N, p.n1, p.n2), st));
+                                                   smem_bytes(p.N, p.row_bytes, p.n1, p.n2), st));
     }
     {
         Prof pr(ctx, st, SLOT_FINALIZE);
@@ -451,10 +449,7 @@ int dart_destroy(dart_ctx *ctx)
     cudaFree(ctx->owner);
     cudaFree(ctx->keep);
     cudaFree(ctx->status);
-    cudaFree(ctx->pl1);
-    cudaFree(ctx->pssq);
     cudaFree(ctx->psim);
-    cudaFree(ctx->cand);
     cudaFree(ctx->counters);
     for (int k = 0; k < 2; ++k) {
         cudaFree(ctx->st_hidden[k]);

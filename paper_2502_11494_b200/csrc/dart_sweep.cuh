@@ -1,34 +1,32 @@
 // Fused path, sweeps: ONE persistent kernel computes the scores (sweep 1), the pivots and the
-// pivot x token dot products (sweep 2) of a whole batch, so that the second read of every key row
-// is served by the L2 cache instead of HBM.
+// pivot x token dot products (sweep 2) of a whole batch, so that the second read of a key row can be
+// served by the L2 cache instead of HBM.
 //
-// Work is cut into tasks of 128 token rows x 512 columns (128 KB of keys).  Every task appears
-// twice in one global, static order: as a sweep-1 task (row L1 norms and sums of squares: the
-// K-norm of the Sec. 3.3 footnote and Eq. 7's denominator) and, `lag` tasks later, as a sweep-2
-// task (dot products with the sample's pivot rows: Eq. 7's numerator).  CTA c executes tasks
-// c, c + grid, c + 2 grid, ...  Because a task is only 128 KB, all SMs together hold < 20 MB in
-// flight, and the distance between the two reads of a row is the sample size plus the lag.
+// Sweep-1 task: 16 whole key rows (one contiguous block of 16 * d * 2 bytes), streamed through shared
+// memory four rows at a time; each of four worker warps sums one row (L1 norm: the K-norm of the
+// Sec. 3.3 footnote; sum of squares: Eq. 7's denominator) and writes the final values - no partial sums.
+// Sweep-2 task: 128 rows x 512 columns as 128-byte-swizzled TMA tiles, multiplied on the tensor cores
+// with the sample's pivot rows (Eq. 7's numerator); the per-column-slab partial products are added up
+// by a small kernel afterwards.
+// Both kinds of task sit in one global, static order: step q = (sweep-1 task q, sweep-2 task q - lag),
+// CTA c runs steps c, c + grid, ...  A sweep-2 task therefore follows the sweep-1 pass over its sample
+// by `lag` steps, which is what bounds the distance between the two reads of a row.
 //
 // Per CTA (512 threads; warp 3 idles):
-//   warps 0, 2 sweep-1 producer and sweep-2 producer: TMA loads of key tiles into two
-//              shared-memory rings, one per sweep, each with its own producer and exactly one consumer
-//              role, so that neither sweep blocks the other and no role ever skips a barrier phase; the
-//              sweep-2 producer also gathers the sample's pivot rows (tile::gather4 boxes straight from
-//              the key tensor).  L2 evict_last on the first read of a tile, evict_first on the second.
+//   warp 0     sweep-1 producer: bulk copies into ring 1 (L2 evict_last), at most one round ahead of
+//              the CTA's own sweep-2 progress
+//   warp 2     sweep-2 producer: waits for the sample's pivots, then TMA tiles (L2 evict_first) and the
+//              pivot rows (tile::gather4 straight from the key tensor) into ring 2
 //   warp 1     sweep 2: one thread issues tcgen05.mma (tokens = M 128, pivots = N, bf16 -> fp32 in TMEM)
-//   warps 4-7  sweep-1 workers: each thread owns one tile row and sums it from shared memory.
-//   warps 8-11 sweep-2 epilogue: read the accumulators out of TMEM and store the partial dot products
-//              (separate from the workers so that neither sweep ever waits for the other; the sweep-1
-//              producer only stays within one round of the CTA's sweep-2 progress, which bounds the
-//              distance between the two reads of a tile).
-//   warps 12-15 control: everything that needs a global-memory round trip, fed by a mailbox so that the
-//              workers never wait for it: counts finished column slabs; the CTA that delivers a row
-//              tile's last slab adds the slab partials up (fixed order) and leaves the tile's P best
-//              (score, index) candidates; the CTA that delivers a sample's last row tile merges the
-//              candidates into the pivots (Def. 1) and publishes them.
-// Every result is bitwise reproducible: partial sums are added in slab order by one thread per row.
+//   warps 4-7  sweep-1 workers (one row per warp and stage)
+//   warps 8-11 sweep-2 epilogue: TMEM -> partial dot products in global memory
+//   warps 12-15 control, each on its own: count finished sweep-1 tasks (the fence and the atomic are
+//              kept off the workers by a mailbox); the warp that counts a sample's LAST task waits for the
+//              others, selects the pivots (Def. 1) by a radix select in shared memory and publishes them.
+// Each ring has one producer and one consumer role, so no role ever skips a barrier phase.
+// Every result is bitwise reproducible: all sums run in a fixed order.
 //
-// Every wait (mbarrier or global flag) is bounded in time; on expiry the kernel records
+// Every wait (mbarrier, flag or lock) is bounded in time; on expiry the kernel records
 // DART_ERR_TIMEOUT in the status word, drains and exits normally.
 #pragma once
 #include <cuda.h>
@@ -38,72 +36,79 @@
 namespace dart {
 namespace sweep {
 
-constexpr int kTileRows = 128;
-constexpr int kAtomCols = 64;  // 64 bf16 = 128 bytes = one swizzle row
-constexpr int kSubRows = 32;   // rows per TMA box of the key tensor
-constexpr int kSlabAtoms = 8;  // a task spans 8 atoms = 512 columns
-constexpr int kMaxStages = 8;  // per ring; fewer when many pivots make the sweep-2 stages large
+constexpr int kTileRows = 128;   // sweep-2 tile rows (MMA M)
+constexpr int kAtomCols = 64;    // 64 bf16 = 128 bytes = one swizzle row
+constexpr int kSubRows = 32;     // rows per TMA box of a short last tile
+constexpr int kSlabAtoms = 8;    // a sweep-2 task spans 8 atoms = 512 columns
+constexpr int kS1Rows = 16;      // rows per sweep-1 task
+constexpr int kS1StageRows = 4;  // rows per sweep-1 stage: one per worker warp
+constexpr int kMaxRowBytes = 16384; // widest row the fused path takes (d <= 8192)
+constexpr int kMaxStages = 8;    // per ring
 constexpr int kAtomBytes = kTileRows * 128; // 16 KB: 128 rows x 128 bytes, 128B-swizzled, K-major
 constexpr int kSubBytes = kSubRows * 128;
 constexpr int kThreads = 512;
+constexpr int kProducer2Warp = 2;
 constexpr int kWorkerWarp0 = 4, kWorkerWarps = 4, kWorkers = kWorkerWarps * 32;
 constexpr int kEpiWarp0 = 8, kEpiWarps = 4; // kEpiWarp0 % 4 == 0: warp w reads TMEM lanes 32 (w % 4) ...
-constexpr int kCtrlWarp0 = 12, kCtrlWarps = 4, kCtrl = kCtrlWarps * 32;
-constexpr int kProducer2Warp = 2;
-constexpr int kMaxN = 256;      // pivots per MMA (N dimension)
-constexpr int kMail = 8;        // mailbox slots between workers and control warps
-constexpr int kMergeMax = 1024; // candidates merged in shared memory; beyond that a radix select over all scores
-constexpr int kStaticSmemReserve = 12288;
+constexpr int kCtrlWarp0 = 12, kCtrlWarps = 4;
+constexpr int kMaxN = 256;       // pivots per MMA (N dimension)
+constexpr int kMail = 8;         // mailbox slots between workers and control warps (slot s -> control warp s % 4)
+constexpr int kSelMax = 4096;    // scores of a sample that fit the shared-memory select buffer
+constexpr int kStaticSmemReserve = 24576;
 constexpr int kStatusTimeout = -7;
 // which wait expired (second status word)
 enum { kWaitPivots = 1, kWaitEmptyStage, kWaitDrain, kWaitAccumFree, kWaitStageMma, kWaitStageRows, kWaitAccumFull,
-       kWaitMailSlot, kWaitMail, kWaitSlabs, kWaitRowTiles, kWaitSweep2 };
+       kWaitMailSlot, kWaitMail, kWaitTasks, kWaitLock, kWaitSweep2 };
 
 using Workers = WarpGroup<kWorkerWarp0, kWorkerWarps, 1>;
-using Control = WarpGroup<kCtrlWarp0, kCtrlWarps, 2>;
+struct OneWarp { // the selection helpers of dart_common.cuh, run by a single warp
+    __device__ __forceinline__ int tid() const { return threadIdx.x & 31; }
+    __device__ __forceinline__ int size() const { return 32; }
+    __device__ __forceinline__ void sync() const { __syncwarp(); }
+};
 
 struct Params {
     int B, S, vis_offset, n_vis, P, N; // N = P rounded up to a multiple of 16 (MMA N)
-    int Pc;                            // candidates a row tile leaves: min(P, 128)
     int d8;                            // row width in 16-byte units
-    int n_atoms, KS, n_rt, T;          // atoms per row; column slabs; row tiles per sample; tasks per sample and sweep
-    int n1, n2;                        // depth of the sweep-1 and of the sweep-2 ring (<= kMaxStages each)
-    uint32_t lag;                      // tasks between a task's first and second sweep (T <= lag <= B * T)
+    int n_atoms, KS, n_rt;             // sweep 2: atoms per row; column slabs; row tiles per sample
+    int T1, T2, Tm;                    // tasks per sample: sweep 1, sweep 2; slots per sample = max of both
+    int n1, n2;                        // depth of ring 1 and ring 2 (<= kMaxStages each)
+    uint32_t row_bytes, stage1_bytes;  // d * 2; shared-memory bytes of a ring-1 stage (4 rows, 1 KB granules)
+    uint32_t lag;                      // steps between the two sweeps (Tm <= lag <= B * Tm)
     int norm_kind, smallest;
     unsigned long long wait_ns;        // time limit of every wait
-    float *pl1, *pssq;                 // [B][KS][n_vis] per-slab partial sums
+    const char *keys;                  // [B][S][d] bf16
     float *psim;                       // [B][KS][n_vis][P] per-slab partial dot products
     float *l1, *ssq;                   // [B][n_vis]
-    unsigned long long *cand;          // [B][n_rt][Pc] best (key, index) pairs of every row tile, best first
     int32_t *pivot_idx;                // [B][P]
-    int *rt_done;                      // [B][n_rt] column slabs finished per row tile
-    int *s1_done;                      // [B] row tiles finished per sample
+    int *s1_done;                      // [B] sweep-1 tasks counted per sample
     int *piv_ready;                    // [B] 1 once the pivots of the sample are published
     int *status;
 };
 
 struct Task {
-    int kind; // 0 = sweep 1, 1 = sweep 2
-    int b, rt, ks;
+    int b;
+    int u;      // sweep 1: task index within the sample (rows 16 u ...)
+    int rt, ks; // sweep 2: row tile and column slab
 };
 
-// Schedule.  Step q of the global order is the pair (sweep-1 task q, sweep-2 task q - lag); CTA c runs steps
-// c, c + grid, ... and, within a step, the sweep-1 task first.  So every CTA alternates between the two kinds
-// of task, and a sweep-2 task comes `lag` steps after the sweep-1 task of the same tile (lag >= T, hence after
-// the whole sample has been scored).  The host guarantees B * T + lag < 2^31.
-__device__ __forceinline__ uint32_t total_steps(const Params &p) { return (uint32_t)p.B * (uint32_t)p.T + p.lag; }
+// Schedule.  Every sample owns Tm consecutive slots in each sweep (a slot beyond the sweep's own task count is
+// empty).  Step q = (sweep-1 slot q, sweep-2 slot q - lag).  The host guarantees B * Tm + lag < 2^30.
+__device__ __forceinline__ uint32_t total_steps(const Params &p) { return (uint32_t)p.B * (uint32_t)p.Tm + p.lag; }
 
 // kind 0: sweep-1 task of step q; kind 1: its sweep-2 task.  Returns false if the step has no such task.
 __device__ __forceinline__ bool decode(const Params &p, uint32_t q, int kind, Task &t)
 {
-    const uint32_t n_all = (uint32_t)p.B * (uint32_t)p.T;
+    const uint32_t n_all = (uint32_t)p.B * (uint32_t)p.Tm;
     if (kind == 0 ? q >= n_all : q < p.lag) return false;
-    const uint32_t n = kind ? q - p.lag : q, T = (uint32_t)p.T, KS = (uint32_t)p.KS;
-    t.kind = kind;
-    t.b = (int)(n / T);
-    const uint32_t u = n - (uint32_t)t.b * T;
-    t.rt = (int)(u / KS);
-    t.ks = (int)(u - (uint32_t)t.rt * KS);
+    const uint32_t n = kind ? q - p.lag : q, Tm = (uint32_t)p.Tm;
+    t.b = (int)(n / Tm);
+    const uint32_t u = n - (uint32_t)t.b * Tm;
+    t.u = (int)u;
+    if (kind == 0) return u < (uint32_t)p.T1;
+    if (u >= (uint32_t)p.T2) return false;
+    t.rt = (int)(u / (uint32_t)p.KS);
+    t.ks = (int)(u - (uint32_t)t.rt * (uint32_t)p.KS);
     return true;
 }
 
@@ -138,6 +143,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm,
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
                  " [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
                  "l"(tm), "r"(x), "r"(y), "r"(bar), "l"(policy)
+                 : "memory");
+}
+// Plain bulk copy of `bytes` contiguous bytes (16-byte aligned, a multiple of 16) into shared memory.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar, unsigned long long policy)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar), "l"(policy)
                  : "memory");
 }
 // Four rows (given by index) x one box width of columns -> four consecutive 128-byte rows at dst.
@@ -309,146 +321,124 @@ struct Ring {
 struct Shared {
     unsigned long long full1[kMaxStages], empty1[kMaxStages], full2[kMaxStages], empty2[kMaxStages];
     unsigned long long tmem_full[2], tmem_empty[2], mail_full[kMail], mail_empty[kMail];
-    int4 mail[kMail]; // (sample, row tile, column slab, valid rows); sample < 0 ends the stream
-    union {
-        unsigned long long cand[kMergeMax]; // candidate merge
-        struct {
-            SelectSmem sel; // radix-select path for very many pivots
-            unsigned long long list[kMaxN];
-        } rs;
-    } u;
-    unsigned long long ckey[kTileRows]; // (key, index) of the rows of the tile being finalised
+    int4 mail[kMail]; // (sample, task index, 1 if it is the sample's last task, -); sample < 0 ends the stream
+    // pivot selection (one control warp at a time, guarded by sel_lock)
+    uint32_t sel_keys[kSelMax];
+    unsigned long long sel_list[kMaxN];
+    SelectSmem sel;
     uint32_t tmem_base, n_picked;
+    int sel_lock;
     int abort_flag;
     volatile int s2_step; // last schedule step whose sweep-2 task this CTA has finished (-1: none yet)
 };
 static_assert(sizeof(Shared) + 64 <= kStaticSmemReserve, "static shared memory exceeds its reserve");
 
 __host__ __device__ inline uint32_t b_stage_bytes(int N) { return (uint32_t)((N * 128 + 1023) / 1024 * 1024); }
-// Ring depths for a shared-memory budget: half of it to the sweep-2 ring (at least 2 stages), the rest to sweep 1.
-__host__ inline void ring_depths(int N, size_t smem_limit, int &n1, int &n2)
+__host__ __device__ inline uint32_t stage1_bytes(uint32_t row_bytes)
+{
+    return (kS1StageRows * row_bytes + 1023u) / 1024u * 1024u;
+}
+// Ring depths for a shared-memory budget: about a third to ring 2 (second reads mostly come from L2 and need
+// less in flight), the rest to ring 1.
+__host__ inline void ring_depths(int N, uint32_t row_bytes, size_t smem_limit, int &n1, int &n2)
 {
     const size_t budget = smem_limit - 1024 - kStaticSmemReserve; // alignment slack and static shared memory
-    const size_t s2 = kAtomBytes + b_stage_bytes(N);
-    size_t b = budget / 2 / s2;
+    const size_t s1 = stage1_bytes(row_bytes), s2 = kAtomBytes + b_stage_bytes(N);
+    size_t b = budget / 3 / s2;
     b = b < 2 ? 2 : (b > (size_t)kMaxStages ? (size_t)kMaxStages : b);
-    size_t a = budget > b * s2 ? (budget - b * s2) / kAtomBytes : 0;
+    size_t a = budget > b * s2 ? (budget - b * s2) / s1 : 0;
     a = a > (size_t)kMaxStages ? (size_t)kMaxStages : a;
     n1 = (int)a;
     n2 = (int)b;
 }
-__host__ inline size_t smem_bytes(int N, int n1, int n2)
+__host__ inline size_t smem_bytes(int N, uint32_t row_bytes, int n1, int n2)
 {
-    return 1024 + (size_t)n1 * kAtomBytes + (size_t)n2 * (kAtomBytes + b_stage_bytes(N));
+    return 1024 + (size_t)n1 * stage1_bytes(row_bytes) + (size_t)n2 * (kAtomBytes + b_stage_bytes(N));
 }
 
-// (key, index) composite of a score: smaller composite = better pivot, equal scores -> lower index first
-__device__ __forceinline__ unsigned long long pivot_key(const Params &p, float score, int j)
+// One control warp: the pivots of sample b (Def. 1) = its P best scores in rank order, equal scores to the
+// lower index.  Radix select over order-preserving keys held in shared memory, then a bitonic sort of the
+// P winners.  Returns false if the lock could not be had in time.
+__device__ bool select_pivots_warp(const Params &p, Shared &sh, const Ctl &ctl, int b)
 {
-    const uint32_t k = order_key(score);
-    return ((unsigned long long)(p.smallest ? k : ~k) << 32) | (uint32_t)j;
-}
-
-// Control warps, row tile (b, rt) complete: add up the slab partials of every row in slab order, store the
-// final sums, and leave the tile's Pc best candidates, best first.
-__device__ void finalize_row_tile(const Params &p, Shared &sh, int b, int rt, int rows)
-{
-    const Control g;
-    const int r = g.tid(), j = rt * kTileRows + r;
-    unsigned long long mine = ~0ull;
-    if (r < rows) {
-        float s1 = 0.f, s2 = 0.f;
-        for (int k0 = 0; k0 < p.KS; k0 += 8) {
-            float a[8], q[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const size_t o = ((size_t)b * p.KS + min(k0 + k, p.KS - 1)) * p.n_vis + j;
-                a[k] = __ldcg(p.pl1 + o);
-                q[k] = __ldcg(p.pssq + o);
+    const OneWarp g;
+    const int lane = g.tid();
+    // one selection at a time per CTA: the buffers below are shared by the four control warps
+    bool ok = true;
+    if (lane == 0) {
+        const long long t0 = clock64();
+        while (atomicCAS(&sh.sel_lock, 0, 1) != 0) {
+            __nanosleep(100);
+            if (ctl.aborted() || (unsigned long long)(clock64() - t0) > ctl.limit_cycles) {
+                if (!ctl.aborted()) ctl.give_up(kWaitLock, b);
+                ok = false;
+                break;
             }
+        }
+    }
+    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+    if (!ok) return false;
+    const float *score = (p.norm_kind == 2 ? p.ssq : p.l1) + (size_t)b * p.n_vis;
+    const int smallest = p.smallest;
+    const bool cached = p.n_vis <= kSelMax;
+    if (cached) { // the scores were written by other SMs: read them from L2, eight loads in flight per lane
+        for (int j0 = lane; j0 < p.n_vis; j0 += 32 * 8) {
+            float v[8];
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
-                if (k0 + k < p.KS) {
-                    s1 += a[k];
-                    s2 += q[k];
+            for (int u = 0; u < 8; ++u) v[u] = (j0 + 32 * u < p.n_vis) ? __ldcg(score + j0 + 32 * u) : 0.f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (j0 + 32 * u < p.n_vis) {
+                    const uint32_t k = order_key(v[u]);
+                    sh.sel_keys[j0 + 32 * u] = smallest ? k : ~k; // smaller key = better pivot
                 }
         }
-        p.l1[(size_t)b * p.n_vis + j] = s1;
-        p.ssq[(size_t)b * p.n_vis + j] = s2;
-        mine = pivot_key(p, p.norm_kind == 2 ? s2 : s1, j);
     }
-    sh.ckey[r] = mine;
+    int P_pad = 1;
+    while (P_pad < p.P) P_pad <<= 1;
+    for (int i = lane; i < P_pad; i += 32) sh.sel_list[i] = ~0ull;
+    if (lane == 0) sh.n_picked = 0;
     g.sync();
-    int rank = 0;
-#pragma unroll 8
-    for (int i = 0; i < kTileRows; ++i) rank += (sh.ckey[i] < mine) ? 1 : 0;
-    unsigned long long *dst = p.cand + ((size_t)b * p.n_rt + rt) * p.Pc;
-    if (r < rows) {
-        if (rank < p.Pc) dst[rank] = mine;
-    } else if (r < p.Pc) {
-        dst[r] = ~0ull; // a short tile has fewer rows than candidate slots: slots rows..Pc-1 stay empty
-    }
-}
-
-// Control warps, sample b complete: pivots (Def. 1) = the P best of the row tiles' candidates, in rank order.
-__device__ void merge_pivots(const Params &p, Shared &sh, int b)
-{
-    const Control g;
-    const int tid = g.tid();
-    const int C = p.n_rt * p.Pc;
-    if (C <= kMergeMax) {
-        const unsigned long long *src = p.cand + (size_t)b * C;
-        for (int i = tid; i < C; i += kCtrl) sh.u.cand[i] = __ldcg(src + i);
-        g.sync();
-        for (int i = tid; i < C; i += kCtrl) {
-            const unsigned long long mine = sh.u.cand[i];
-            if (mine == ~0ull) continue;
-            int rank = 0;
-#pragma unroll 8
-            for (int k = 0; k < C; ++k) rank += (sh.u.cand[k] < mine) ? 1 : 0;
-            if (rank < p.P) p.pivot_idx[(size_t)b * p.P + rank] = (int32_t)(mine & 0xffffffffu);
-        }
-    } else {
-        // very many pivots: radix select over all scores of the sample, then sort the winners
-        const float *score = (p.norm_kind == 2 ? p.ssq : p.l1) + (size_t)b * p.n_vis;
-        const int smallest = p.smallest;
-        auto keyfn = [&](int j, uint32_t &key) {
-            uint32_t k = order_key(__ldcg(score + j));
+    auto keyfn = [&](int j, uint32_t &key) {
+        if (cached) {
+            key = sh.sel_keys[j];
+        } else {
+            const uint32_t k = order_key(__ldcg(score + j));
             key = smallest ? k : ~k;
-            return true;
-        };
-        int P_pad = 1;
-        while (P_pad < p.P) P_pad <<= 1;
-        for (int i = tid; i < P_pad; i += kCtrl) sh.u.rs.list[i] = ~0ull;
-        if (tid == 0) sh.n_picked = 0;
-        uint32_t T, need_eq, cnt_eq;
-        block_select_threshold(g, keyfn, p.n_vis, (uint32_t)p.P, sh.u.rs.sel, T, need_eq, cnt_eq);
-        block_select_apply(g, keyfn, p.n_vis, T, need_eq, cnt_eq, sh.u.rs.sel, [&](int j, uint32_t key) {
-            uint32_t slot = atomicAdd(&sh.n_picked, 1u);
-            if (slot < (uint32_t)kMaxN) sh.u.rs.list[slot] = ((unsigned long long)key << 32) | (uint32_t)j;
-        });
-        for (int k = 2; k <= P_pad; k <<= 1) {
-            for (int jj = k >> 1; jj > 0; jj >>= 1) {
-                for (int i = tid; i < P_pad; i += kCtrl) {
-                    int l = i ^ jj;
-                    if (l > i) {
-                        unsigned long long x = sh.u.rs.list[i], y = sh.u.rs.list[l];
-                        bool up = ((i & k) == 0);
-                        if ((x > y) == up) {
-                            sh.u.rs.list[i] = y;
-                            sh.u.rs.list[l] = x;
-                        }
+        }
+        return true;
+    };
+    uint32_t T, need_eq, cnt_eq;
+    block_select_threshold(g, keyfn, p.n_vis, (uint32_t)p.P, sh.sel, T, need_eq, cnt_eq);
+    block_select_apply(g, keyfn, p.n_vis, T, need_eq, cnt_eq, sh.sel, [&](int j, uint32_t key) {
+        const uint32_t slot = atomicAdd(&sh.n_picked, 1u);
+        if (slot < (uint32_t)kMaxN) sh.sel_list[slot] = ((unsigned long long)key << 32) | (uint32_t)j;
+    });
+    for (int k = 2; k <= P_pad; k <<= 1) { // ascending bitonic sort of (key, index): rank 0 = best
+        for (int jj = k >> 1; jj > 0; jj >>= 1) {
+            for (int i = lane; i < P_pad; i += 32) {
+                const int l = i ^ jj;
+                if (l > i) {
+                    const unsigned long long x = sh.sel_list[i], y = sh.sel_list[l];
+                    const bool up = ((i & k) == 0);
+                    if ((x > y) == up) {
+                        sh.sel_list[i] = y;
+                        sh.sel_list[l] = x;
                     }
                 }
-                g.sync();
             }
+            g.sync();
         }
-        for (int i = tid; i < p.P; i += kCtrl)
-            p.pivot_idx[(size_t)b * p.P + i] = (int32_t)min((uint32_t)(sh.u.rs.list[i] & 0xffffffffu), (uint32_t)(p.n_vis - 1));
     }
+    for (int i = lane; i < p.P; i += 32)
+        p.pivot_idx[(size_t)b * p.P + i] = (int32_t)min((uint32_t)(sh.sel_list[i] & 0xffffffffu), (uint32_t)(p.n_vis - 1));
     __threadfence();
     g.sync();
-    if (tid == 0) st_release(p.piv_ready + b, 1);
+    if (lane == 0) {
+        st_release(p.piv_ready + b, 1);
+        atomicExch(&sh.sel_lock, 0);
+    }
+    return true;
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -459,13 +449,14 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
     __shared__ Shared sh;
     const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bstage = b_stage_bytes(p.N);
-    // ring 1: n1 key tiles; ring 2: n2 key tiles followed by n2 pivot tiles
-    auto a1_addr = [&](int s) { return smem0 + (uint32_t)s * kAtomBytes; };
-    auto a2_addr = [&](int s) { return smem0 + (uint32_t)(p.n1 + s) * kAtomBytes; };
-    auto b2_addr = [&](int s) { return smem0 + (uint32_t)(p.n1 + p.n2) * kAtomBytes + (uint32_t)s * bstage; };
+    // ring 1: n1 stages of four plain rows; ring 2: n2 swizzled key tiles followed by n2 pivot tiles
+    const uint32_t ring2_0 = smem0 + (uint32_t)p.n1 * p.stage1_bytes;
+    auto a1_addr = [&](int s) { return smem0 + (uint32_t)s * p.stage1_bytes; };
+    auto a2_addr = [&](int s) { return ring2_0 + (uint32_t)s * kAtomBytes; };
+    auto b2_addr = [&](int s) { return ring2_0 + (uint32_t)p.n2 * kAtomBytes + (uint32_t)s * bstage; };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned long long limit = 2ull * p.wait_ns; // ns -> cycles at the highest SM clock: never shorter than asked
-    // consumers get a longer limit than the producer, so that the wait nearest the cause reports first
+    // consumers get a longer limit than the producers, so that the wait nearest the cause reports first
     const Ctl ctl{&sh.abort_flag, p.status, (warp == 0 || warp == kProducer2Warp) ? limit : limit + limit / 4};
 
     if (threadIdx.x == 0) {
@@ -484,6 +475,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             mbar_init(smem_u32(&sh.mail_empty[m]), 1);
         }
         sh.abort_flag = 0;
+        sh.sel_lock = 0;
         sh.s2_step = -1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -502,48 +494,40 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
     const uint32_t total = total_steps(p);
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ sweep-1 producer (lane 0 waits, lanes issue)
-        unsigned long long pol_keep;
-        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
-        Ring ring(p.n1);
-        long long issued = 0;
-        bool ok = true;
-        for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
-            Task t;
-            if (!decode(p, g, 0, t)) continue;
-            // stay within one round of this CTA's sweep-2 progress: the step one round back has a sweep-2
-            // task if it is >= lag, and that task must be finished before more tiles are pulled in
-            if (g >= gridDim.x && g - gridDim.x >= p.lag) {
-                if (lane == 0) ok = ctl.wait_count(&sh.s2_step, (int)(g - gridDim.x), kWaitSweep2, g);
-                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                if (!ok) break;
-            }
-            const int na = slab_atoms(p, t.ks);
-            const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
-            const int n_sub = (rows + kSubRows - 1) / kSubRows;
-            const int y0 = t.b * p.S + p.vis_offset + t.rt * kTileRows;
-            for (int a = 0; a < na; ++a) {
-                const uint32_t full = smem_u32(&sh.full1[ring.stage]);
-                if (lane == 0) {
+        // ------------------------------------------------------------------ sweep-1 producer
+        if (lane == 0) {
+            unsigned long long pol_keep;
+            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+            Ring ring(p.n1);
+            long long issued = 0;
+            bool ok = true;
+            for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
+                Task t;
+                if (!decode(p, g, 0, t)) continue;
+                // stay within one round of this CTA's sweep-2 progress: the step one round back has a sweep-2
+                // task if it is >= lag, and that task must be finished before more rows are pulled in
+                if (g >= gridDim.x && g - gridDim.x >= p.lag) {
+                    Task t2;
+                    if (decode(p, g - gridDim.x, 1, t2)) ok = ctl.wait_count(&sh.s2_step, (int)(g - gridDim.x), kWaitSweep2, g);
+                    if (!ok) break;
+                }
+                const int row0 = t.u * kS1Rows, rows = min(kS1Rows, p.n_vis - row0);
+                const char *src = p.keys + ((size_t)t.b * p.S + p.vis_offset + row0) * (size_t)p.row_bytes;
+                for (int r = 0; r < rows; r += kS1StageRows) {
+                    const uint32_t bytes = (uint32_t)min(kS1StageRows, rows - r) * p.row_bytes;
                     ok = ctl.wait_bar(smem_u32(&sh.empty1[ring.stage]), ring.phase ^ 1u, kWaitEmptyStage, g);
-                    if (ok) mbar_arrive_expect_tx(full, rows == kTileRows ? (uint32_t)kAtomBytes : (uint32_t)n_sub * kSubBytes);
+                    if (!ok) break;
+                    const uint32_t full = smem_u32(&sh.full1[ring.stage]);
+                    mbar_arrive_expect_tx(full, bytes);
+                    bulk_load(a1_addr(ring.stage), src + (size_t)r * p.row_bytes, bytes, full, pol_keep);
+                    ring.advance();
+                    ++issued;
                 }
-                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                if (!ok) break;
-                const int x = (t.ks * kSlabAtoms + a) * kAtomCols;
-                const uint32_t dst = a1_addr(ring.stage);
-                if (rows == kTileRows) { // a full tile is one 128-row box; a short last tile is 32-row boxes
-                    if (lane == 0) tma_load_2d(dst, &tm_tile, x, y0, full, pol_keep);
-                } else if (lane < n_sub) {
-                    tma_load_2d(dst + (uint32_t)lane * kSubBytes, &tm_keys, x, y0 + lane * kSubRows, full, pol_keep);
-                }
-                ring.advance();
-                ++issued;
             }
+            if (!ok) // drain: let the copies already issued land before the CTA may exit
+                for (long long i = issued > p.n1 ? issued - p.n1 : 0; i < issued; ++i)
+                    ctl.wait_bar(smem_u32(&sh.full1[i % p.n1]), (uint32_t)((i / p.n1) & 1), kWaitDrain, i);
         }
-        if (!ok && lane == 0) // drain: let the copies already issued land before the CTA may exit
-            for (long long i = issued > p.n1 ? issued - p.n1 : 0; i < issued; ++i)
-                ctl.wait_bar(smem_u32(&sh.full1[i % p.n1]), (uint32_t)((i / p.n1) & 1), kWaitDrain, i);
     } else if (warp == kProducer2Warp) {
         // ------------------------------------------------------------------ sweep-2 producer
         unsigned long long pol_keep, pol_drop;
@@ -563,8 +547,6 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                     if (!ok && p.status[1] == kWaitPivots && p.status[3] == (int)blockIdx.x) {
                         p.status[4] = t.b;
                         p.status[5] = ld_acquire(p.s1_done + t.b);
-                        for (int r = 0; r < 6 && r < p.n_rt; ++r)
-                            p.status[6 + r] = ld_acquire(p.rt_done + (size_t)t.b * p.n_rt + r);
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -647,68 +629,6 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                 ++s2n;
             }
         }
-    } else if (warp >= kWorkerWarp0 && warp < kWorkerWarp0 + kWorkerWarps) {
-        // ------------------------------------------------------------------ sweep-1 workers
-        const int wt = threadIdx.x - kWorkerWarp0 * 32; // 0..127 = tile row owned by this thread
-        const int row = wt;
-        Ring ring(p.n1);
-        int ms = 0;
-        uint32_t mph = 0;
-        bool dead = false; // warp-uniform inside a task, group-uniform after every workers_any()
-        auto post = [&](int4 m) { // thread wt == 0: hand a finished slab (or the end mark) to the control warps
-            bool ok = ctl.wait_bar(smem_u32(&sh.mail_empty[ms]), mph ^ 1u, kWaitMailSlot, 0);
-            if (ok) {
-                sh.mail[ms] = m;
-                mbar_arrive(smem_u32(&sh.mail_full[ms])); // release: the group's partial sums are ordered before it
-            }
-            return ok;
-        };
-        for (uint32_t g = blockIdx.x; g < total; g += gridDim.x) {
-            Task t;
-            if (!decode(p, g, 0, t)) continue;
-            const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
-            const int j = t.rt * kTileRows + row;
-            const int na = slab_atoms(p, t.ks);
-            float a0 = 0.f, a1 = 0.f, q0 = 0.f, q1 = 0.f;
-            for (int a = 0; a < na; ++a) {
-                // warp-uniform: either the whole warp reads the stage and releases it, or none of it does
-                if (!dead) dead = !ctl.wait_bar(smem_u32(&sh.full1[ring.stage]), ring.phase, kWaitStageRows, g);
-                dead = __any_sync(0xffffffffu, dead);
-                if (!dead && row < rows) {
-                    const uint32_t base = a1_addr(ring.stage) + (uint32_t)row * 128u;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        // logical 16-byte chunk c of this row sits at chunk c ^ (row & 7)
-                        const uint4 v = lds128(base + (uint32_t)((c ^ (row & 7)) << 4));
-                        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float lo = bf16_lo(w[e]), hi = bf16_hi(w[e]);
-                            a0 += fabsf(lo);
-                            a1 += fabsf(hi);
-                            q0 = fmaf(lo, lo, q0);
-                            q1 = fmaf(hi, hi, q1);
-                        }
-                    }
-                }
-                __syncwarp(); // the warp's reads of the stage are done
-                if (!dead && lane == 0) mbar_arrive(smem_u32(&sh.empty1[ring.stage]));
-                ring.advance();
-            }
-            if (!dead && row < rows) {
-                const size_t o = ((size_t)t.b * p.KS + t.ks) * p.n_vis + j;
-                p.pl1[o] = a0 + a1;
-                p.pssq[o] = q0 + q1;
-            }
-            dead = workers_any(dead); // every worker's partial sums are issued
-            if (!dead && wt == 0 && !post(make_int4(t.b, t.rt, t.ks, rows))) dead = true;
-            if (++ms == kMail) {
-                ms = 0;
-                mph ^= 1u;
-            }
-        }
-        workers_any(dead);
-        if (wt == 0) post(make_int4(-1, 0, 0, 0)); // end of the stream (also after a failure, so that control exits)
     } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
         // ------------------------------------------------------------------ sweep-2 epilogue (warps independent)
         const int quarter = warp & 3;        // TMEM lane quarter this warp may read
@@ -747,48 +667,91 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             }
             ++s2n;
         }
-    } else if (warp >= kCtrlWarp0 && warp < kCtrlWarp0 + kCtrlWarps) {
-        // ------------------------------------------------------------------ control
-        const Control cg;
-        const int ct = cg.tid();
-        int mi = 0;
+    } else if (warp >= kWorkerWarp0 && warp < kWorkerWarp0 + kWorkerWarps) {
+        // ------------------------------------------------------------------ sweep-1 workers: one row per warp and stage
+        const int wq = warp - kWorkerWarp0, wt = threadIdx.x - kWorkerWarp0 * 32;
+        Ring ring(p.n1);
+        int ms = 0;
         uint32_t mph = 0;
-        for (;;) {
-            bool fail = !ctl.wait_bar(smem_u32(&sh.mail_full[mi]), mph, kWaitMail, 0);
-            if (control_any(fail)) break;
-            const int4 m = sh.mail[mi];
-            cg.sync(); // everyone has read the slot
-            if (ct == 0) mbar_arrive(smem_u32(&sh.mail_empty[mi]));
-            if (++mi == kMail) {
-                mi = 0;
+        bool dead = false; // warp-uniform inside a task, group-uniform after every workers_any()
+        auto post = [&](int4 m) { // thread wt == 0: hand a finished task (or an end mark) to a control warp
+            bool ok = ctl.wait_bar(smem_u32(&sh.mail_empty[ms]), mph ^ 1u, kWaitMailSlot, 0);
+            if (ok) {
+                sh.mail[ms] = m;
+                mbar_arrive(smem_u32(&sh.mail_full[ms])); // release: the group's scores are ordered before it
+            }
+            if (++ms == kMail) {
+                ms = 0;
                 mph ^= 1u;
             }
-            if (m.x < 0) break;
-            // Who finalises is fixed by the schedule, not by arrival order: the CTA that holds slab
-            // (b + rt) % KS of a row tile finalises it, and the one that finalises a sample's LAST row tile
-            // merges the sample, so that it only ever waits for work that precedes its own in the schedule
-            // (its own later mails can then never be what it waits for).  Letting the last arriver do it
-            // instead makes a busy control group ever later, hence ever last.
-            int *slabs = p.rt_done + (size_t)m.x * p.n_rt + m.y;
-            const bool fin_tile = m.z == (m.x + m.y) % p.KS, fin_sample = fin_tile && m.y == p.n_rt - 1;
-            bool late = false;
-            if (ct == 0) {
-                __threadfence(); // the workers' partial sums (ordered before the mail) become visible GPU-wide
-                atomicAdd(slabs, 1);
-                if (fin_tile) late = !ctl.wait_flag(slabs, kWaitSlabs, m.x, p.KS);
-            }
-            if (control_any(late)) break;
-            if (fin_tile) {
-                finalize_row_tile(p, sh, m.x, m.y, m.w);
-                __threadfence();
-                cg.sync();
-                if (ct == 0) {
-                    atomicAdd(p.s1_done + m.x, 1);
-                    if (fin_sample) late = !ctl.wait_flag(p.s1_done + m.x, kWaitRowTiles, m.x, p.n_rt);
+            return ok;
+        };
+        for (uint32_t g = blockIdx.x; g < total; g += gridDim.x) {
+            Task t;
+            if (!decode(p, g, 0, t)) continue;
+            const int row0 = t.u * kS1Rows, rows = min(kS1Rows, p.n_vis - row0);
+            for (int r = 0; r < rows; r += kS1StageRows) {
+                // warp-uniform: either the whole warp reads the stage and releases it, or none of it does
+                if (!dead) dead = !ctl.wait_bar(smem_u32(&sh.full1[ring.stage]), ring.phase, kWaitStageRows, g);
+                dead = __any_sync(0xffffffffu, dead);
+                if (!dead && r + wq < rows) {
+                    const uint32_t base = a1_addr(ring.stage) + (uint32_t)wq * p.row_bytes + (uint32_t)lane * 16u;
+                    float a0 = 0.f, a1 = 0.f, q0 = 0.f, q1 = 0.f;
+#pragma unroll 4
+                    for (int c = lane; c < p.d8; c += 32) { // lanes read consecutive 16-byte chunks: no bank conflicts
+                        const uint4 v = lds128(base + (uint32_t)(c - lane) * 16u);
+                        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float lo = bf16_lo(w[e]), hi = bf16_hi(w[e]);
+                            a0 += fabsf(lo);
+                            a1 += fabsf(hi);
+                            q0 = fmaf(lo, lo, q0);
+                            q1 = fmaf(hi, hi, q1);
+                        }
+                    }
+                    const float a = warp_sum(a0 + a1), q = warp_sum(q0 + q1); // fixed order; every lane gets the sum
+                    if (lane == 0) {
+                        const size_t o = (size_t)t.b * p.n_vis + row0 + r + wq;
+                        p.l1[o] = a;
+                        p.ssq[o] = q;
+                    }
                 }
-                if (control_any(late)) break;
-                if (fin_sample) merge_pivots(p, sh, m.x);
+                __syncwarp(); // the warp's reads of the stage are done
+                if (!dead && lane == 0) mbar_arrive(smem_u32(&sh.empty1[ring.stage]));
+                ring.advance();
             }
+            dead = workers_any(dead); // every warp's scores of this task are issued
+            if (wt == 0 && !dead && !post(make_int4(t.b, t.u, t.u == p.T1 - 1, 0))) dead = true;
+        }
+        workers_any(dead);
+        if (wt == 0) // one end mark per control warp (also after a failure, so that they exit)
+            for (int k = 0; k < kCtrlWarps; ++k) post(make_int4(-1, 0, 0, 0)); // four consecutive slots: one per warp
+    } else if (warp >= kCtrlWarp0 && warp < kCtrlWarp0 + kCtrlWarps) {
+        // ------------------------------------------------------------------ control: warp cw serves mail slots cw, cw + 4
+        const int cw = warp - kCtrlWarp0;
+        for (uint32_t m = 0;; ++m) {
+            const int slot = cw + kCtrlWarps * (int)(m & 1u);
+            int4 mail = make_int4(-1, 0, 0, 0);
+            bool ok = true;
+            if (lane == 0) {
+                ok = ctl.wait_bar(smem_u32(&sh.mail_full[slot]), (m >> 1) & 1u, kWaitMail, 0);
+                if (ok) {
+                    mail = sh.mail[slot];
+                    mbar_arrive(smem_u32(&sh.mail_empty[slot]));
+                    if (mail.x >= 0) {
+                        __threadfence(); // the workers' scores (ordered before the mail) become visible GPU-wide
+                        atomicAdd(p.s1_done + mail.x, 1);
+                        // the warp that counts a sample's last task selects its pivots: everything it waits for
+                        // precedes its own task in the schedule, so it can never wait for its own later mail
+                        if (mail.z) ok = ctl.wait_flag(p.s1_done + mail.x, kWaitTasks, mail.x, p.T1);
+                    }
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+            const int b = __shfl_sync(0xffffffffu, mail.x, 0), last = __shfl_sync(0xffffffffu, mail.z, 0);
+            if (!ok || b == -1) break;
+            if (b >= 0 && last && !select_pivots_warp(p, sh, ctl, b)) break;
         }
     }
     // ---------------------------------------------------------------------- teardown
