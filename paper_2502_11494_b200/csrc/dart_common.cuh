@@ -87,9 +87,15 @@ __device__ void block_select_threshold(Group g, KeyFn keyfn, int n, uint32_t k, 
     for (int shift = 24; shift >= 0; shift -= 8) {
         for (int i = tid; i < 256; i += gsz) sm.hist[i] = 0;
         g.sync();
-        for (int j = tid; j < n; j += gsz) {
-            uint32_t key;
-            if (keyfn(j, key) && (key & mask) == prefix) atomicAdd(&sm.hist[(key >> shift) & 255u], 1u);
+        // warp-aggregated histogram: lanes of a warp that hit the same bin add once (scores of real
+        // tokens share their leading key bytes, which would serialise one atomic per lane)
+        for (int j0 = 0; j0 < n; j0 += gsz) {
+            const int j = j0 + tid;
+            uint32_t key = 0;
+            const bool v = j < n && keyfn(j, key) && (key & mask) == prefix;
+            const uint32_t bin = v ? ((key >> shift) & 255u) : 256u;
+            const uint32_t peers = __match_any_sync(0xffffffffu, bin);
+            if (v && (tid & 31) == __ffs(peers) - 1) atomicAdd(&sm.hist[bin], (uint32_t)__popc(peers));
         }
         g.sync();
         if (tid < kWarp) {

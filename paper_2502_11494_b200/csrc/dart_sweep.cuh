@@ -20,9 +20,10 @@
 //   warp 1     sweep 2: one thread issues tcgen05.mma (tokens = M 128, pivots = N, bf16 -> fp32 in TMEM)
 //   warps 4-7  sweep-1 workers (one row per warp and stage)
 //   warps 8-11 sweep-2 epilogue: TMEM -> partial dot products in global memory
-//   warps 12-15 control, each on its own: count finished sweep-1 tasks (the fence and the atomic are
-//              kept off the workers by a mailbox); the warp that counts a sample's LAST task waits for the
-//              others, selects the pivots (Def. 1) by a radix select in shared memory and publishes them.
+//   warp 12    counter: counts finished sweep-1 tasks (the fence and the atomic are kept off the
+//              workers by a mailbox); when it counts a sample's LAST task it hands the sample over to
+//   warps 13-15 selection: wait until all of the sample's tasks are counted, select the pivots (Def. 1)
+//              by a radix select in shared memory and publish them.  Counting never waits for a selection.
 // Each ring has one producer and one consumer role, so no role ever skips a barrier phase.
 // Every result is bitwise reproducible: all sums run in a fixed order.
 //
@@ -50,22 +51,19 @@ constexpr int kThreads = 512;
 constexpr int kProducer2Warp = 2;
 constexpr int kWorkerWarp0 = 4, kWorkerWarps = 4, kWorkers = kWorkerWarps * 32;
 constexpr int kEpiWarp0 = 8, kEpiWarps = 4; // kEpiWarp0 % 4 == 0: warp w reads TMEM lanes 32 (w % 4) ...
-constexpr int kCtrlWarp0 = 12, kCtrlWarps = 4;
+constexpr int kCountWarp = 12, kSelWarp0 = 13, kSelWarps = 3, kSel = kSelWarps * 32;
+constexpr int kDuty = 4;         // samples waiting for their selection
 constexpr int kMaxN = 256;       // pivots per MMA (N dimension)
-constexpr int kMail = 8;         // mailbox slots between workers and control warps (slot s -> control warp s % 4)
+constexpr int kMail = 8;         // mailbox slots between the workers and the counter warp
 constexpr int kSelMax = 4096;    // scores of a sample that fit the shared-memory select buffer
 constexpr int kStaticSmemReserve = 24576;
 constexpr int kStatusTimeout = -7;
 // which wait expired (second status word)
 enum { kWaitPivots = 1, kWaitEmptyStage, kWaitDrain, kWaitAccumFree, kWaitStageMma, kWaitStageRows, kWaitAccumFull,
-       kWaitMailSlot, kWaitMail, kWaitTasks, kWaitLock, kWaitSweep2 };
+       kWaitMailSlot, kWaitMail, kWaitTasks, kWaitDutySlot, kWaitDuty, kWaitSweep2 };
 
 using Workers = WarpGroup<kWorkerWarp0, kWorkerWarps, 1>;
-struct OneWarp { // the selection helpers of dart_common.cuh, run by a single warp
-    __device__ __forceinline__ int tid() const { return threadIdx.x & 31; }
-    __device__ __forceinline__ int size() const { return 32; }
-    __device__ __forceinline__ void sync() const { __syncwarp(); }
-};
+using Selectors = WarpGroup<kSelWarp0, kSelWarps, 2>;
 
 struct Params {
     int B, S, vis_offset, n_vis, P, N; // N = P rounded up to a multiple of 16 (MMA N)
@@ -178,18 +176,18 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
     return v;
 }
 // OR of a predicate over a 128-thread warp group; doubles as the group's barrier
-template <int kBarrierId>
+template <int kBarrierId, int kCount>
 __device__ __forceinline__ bool group_any(bool pred)
 {
     uint32_t r;
-    asm volatile("{\n.reg .pred p, q;\nsetp.ne.u32 q, %1, 0;\nbar.red.or.pred p, %2, 128, q;\nselp.u32 %0, 1, 0, p;\n}"
+    asm volatile("{\n.reg .pred p, q;\nsetp.ne.u32 q, %1, 0;\nbar.red.or.pred p, %2, %3, q;\nselp.u32 %0, 1, 0, p;\n}"
                  : "=r"(r)
-                 : "r"((uint32_t)pred), "n"(kBarrierId)
+                 : "r"((uint32_t)pred), "n"(kBarrierId), "n"(kCount)
                  : "memory");
     return r != 0;
 }
-__device__ __forceinline__ bool workers_any(bool pred) { return group_any<1>(pred); }
-__device__ __forceinline__ bool control_any(bool pred) { return group_any<2>(pred); }
+__device__ __forceinline__ bool workers_any(bool pred) { return group_any<1, kWorkers>(pred); }
+__device__ __forceinline__ bool selectors_any(bool pred) { return group_any<2, kSel>(pred); }
 
 // Shared-memory matrix descriptor of a K-major, 128B-swizzled bf16 tile (rows at a 128-byte pitch,
 // groups of 8 rows 1024 bytes apart).
@@ -321,13 +319,14 @@ struct Ring {
 struct Shared {
     unsigned long long full1[kMaxStages], empty1[kMaxStages], full2[kMaxStages], empty2[kMaxStages];
     unsigned long long tmem_full[2], tmem_empty[2], mail_full[kMail], mail_empty[kMail];
+    unsigned long long duty_full[kDuty], duty_empty[kDuty];
+    int duty[kDuty]; // samples whose last task has been counted; < 0 ends the stream
     int4 mail[kMail]; // (sample, task index, 1 if it is the sample's last task, -); sample < 0 ends the stream
-    // pivot selection (one control warp at a time, guarded by sel_lock)
+    // pivot selection (the selection warps, one sample at a time)
     uint32_t sel_keys[kSelMax];
     unsigned long long sel_list[kMaxN];
     SelectSmem sel;
     uint32_t tmem_base, n_picked;
-    int sel_lock;
     int abort_flag;
     volatile int s2_step; // last schedule step whose sweep-2 task this CTA has finished (-1: none yet)
 };
@@ -356,47 +355,32 @@ __host__ inline size_t smem_bytes(int N, uint32_t row_bytes, int n1, int n2)
     return 1024 + (size_t)n1 * stage1_bytes(row_bytes) + (size_t)n2 * (kAtomBytes + b_stage_bytes(N));
 }
 
-// One control warp: the pivots of sample b (Def. 1) = its P best scores in rank order, equal scores to the
+// The selection warps: the pivots of sample b (Def. 1) = its P best scores in rank order, equal scores to the
 // lower index.  Radix select over order-preserving keys held in shared memory, then a bitonic sort of the
-// P winners.  Returns false if the lock could not be had in time.
-__device__ bool select_pivots_warp(const Params &p, Shared &sh, const Ctl &ctl, int b)
+// P winners.
+__device__ void select_pivots(const Params &p, Shared &sh, int b)
 {
-    const OneWarp g;
-    const int lane = g.tid();
-    // one selection at a time per CTA: the buffers below are shared by the four control warps
-    bool ok = true;
-    if (lane == 0) {
-        const long long t0 = clock64();
-        while (atomicCAS(&sh.sel_lock, 0, 1) != 0) {
-            __nanosleep(100);
-            if (ctl.aborted() || (unsigned long long)(clock64() - t0) > ctl.limit_cycles) {
-                if (!ctl.aborted()) ctl.give_up(kWaitLock, b);
-                ok = false;
-                break;
-            }
-        }
-    }
-    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-    if (!ok) return false;
+    const Selectors g;
+    const int lane = g.tid(); // 0 .. kSel-1
     const float *score = (p.norm_kind == 2 ? p.ssq : p.l1) + (size_t)b * p.n_vis;
     const int smallest = p.smallest;
     const bool cached = p.n_vis <= kSelMax;
     if (cached) { // the scores were written by other SMs: read them from L2, eight loads in flight per lane
-        for (int j0 = lane; j0 < p.n_vis; j0 += 32 * 8) {
+        for (int j0 = lane; j0 < p.n_vis; j0 += kSel * 8) {
             float v[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) v[u] = (j0 + 32 * u < p.n_vis) ? __ldcg(score + j0 + 32 * u) : 0.f;
+            for (int u = 0; u < 8; ++u) v[u] = (j0 + kSel * u < p.n_vis) ? __ldcg(score + j0 + kSel * u) : 0.f;
 #pragma unroll
             for (int u = 0; u < 8; ++u)
-                if (j0 + 32 * u < p.n_vis) {
+                if (j0 + kSel * u < p.n_vis) {
                     const uint32_t k = order_key(v[u]);
-                    sh.sel_keys[j0 + 32 * u] = smallest ? k : ~k; // smaller key = better pivot
+                    sh.sel_keys[j0 + kSel * u] = smallest ? k : ~k; // smaller key = better pivot
                 }
         }
     }
     int P_pad = 1;
     while (P_pad < p.P) P_pad <<= 1;
-    for (int i = lane; i < P_pad; i += 32) sh.sel_list[i] = ~0ull;
+    for (int i = lane; i < P_pad; i += kSel) sh.sel_list[i] = ~0ull;
     if (lane == 0) sh.n_picked = 0;
     g.sync();
     auto keyfn = [&](int j, uint32_t &key) {
@@ -416,7 +400,7 @@ __device__ bool select_pivots_warp(const Params &p, Shared &sh, const Ctl &ctl, 
     });
     for (int k = 2; k <= P_pad; k <<= 1) { // ascending bitonic sort of (key, index): rank 0 = best
         for (int jj = k >> 1; jj > 0; jj >>= 1) {
-            for (int i = lane; i < P_pad; i += 32) {
+            for (int i = lane; i < P_pad; i += kSel) {
                 const int l = i ^ jj;
                 if (l > i) {
                     const unsigned long long x = sh.sel_list[i], y = sh.sel_list[l];
@@ -430,15 +414,11 @@ __device__ bool select_pivots_warp(const Params &p, Shared &sh, const Ctl &ctl, 
             g.sync();
         }
     }
-    for (int i = lane; i < p.P; i += 32)
+    for (int i = lane; i < p.P; i += kSel)
         p.pivot_idx[(size_t)b * p.P + i] = (int32_t)min((uint32_t)(sh.sel_list[i] & 0xffffffffu), (uint32_t)(p.n_vis - 1));
     __threadfence();
     g.sync();
-    if (lane == 0) {
-        st_release(p.piv_ready + b, 1);
-        atomicExch(&sh.sel_lock, 0);
-    }
-    return true;
+    if (lane == 0) st_release(p.piv_ready + b, 1);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -474,8 +454,11 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             mbar_init(smem_u32(&sh.mail_full[m]), 1);
             mbar_init(smem_u32(&sh.mail_empty[m]), 1);
         }
+        for (int m = 0; m < kDuty; ++m) {
+            mbar_init(smem_u32(&sh.duty_full[m]), 1);
+            mbar_init(smem_u32(&sh.duty_empty[m]), 1);
+        }
         sh.abort_flag = 0;
-        sh.sel_lock = 0;
         sh.s2_step = -1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -725,33 +708,53 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             if (wt == 0 && !dead && !post(make_int4(t.b, t.u, t.u == p.T1 - 1, 0))) dead = true;
         }
         workers_any(dead);
-        if (wt == 0) // one end mark per control warp (also after a failure, so that they exit)
-            for (int k = 0; k < kCtrlWarps; ++k) post(make_int4(-1, 0, 0, 0)); // four consecutive slots: one per warp
-    } else if (warp >= kCtrlWarp0 && warp < kCtrlWarp0 + kCtrlWarps) {
-        // ------------------------------------------------------------------ control: warp cw serves mail slots cw, cw + 4
-        const int cw = warp - kCtrlWarp0;
-        for (uint32_t m = 0;; ++m) {
-            const int slot = cw + kCtrlWarps * (int)(m & 1u);
-            int4 mail = make_int4(-1, 0, 0, 0);
-            bool ok = true;
-            if (lane == 0) {
-                ok = ctl.wait_bar(smem_u32(&sh.mail_full[slot]), (m >> 1) & 1u, kWaitMail, 0);
+        if (wt == 0) post(make_int4(-1, 0, 0, 0)); // end mark (also after a failure, so that the control warps exit)
+    } else if (warp == kCountWarp) {
+        // ------------------------------------------------------------------ counter (one thread)
+        if (lane == 0) {
+            int ds = 0;
+            uint32_t dph = 0;
+            auto hand_over = [&](int b) { // sample b is complete once s1_done[b] reaches T1: the selectors' job
+                bool ok = ctl.wait_bar(smem_u32(&sh.duty_empty[ds]), dph ^ 1u, kWaitDutySlot, b);
                 if (ok) {
-                    mail = sh.mail[slot];
-                    mbar_arrive(smem_u32(&sh.mail_empty[slot]));
-                    if (mail.x >= 0) {
-                        __threadfence(); // the workers' scores (ordered before the mail) become visible GPU-wide
-                        atomicAdd(p.s1_done + mail.x, 1);
-                        // the warp that counts a sample's last task selects its pivots: everything it waits for
-                        // precedes its own task in the schedule, so it can never wait for its own later mail
-                        if (mail.z) ok = ctl.wait_flag(p.s1_done + mail.x, kWaitTasks, mail.x, p.T1);
-                    }
+                    sh.duty[ds] = b;
+                    mbar_arrive(smem_u32(&sh.duty_full[ds]));
                 }
+                if (++ds == kDuty) {
+                    ds = 0;
+                    dph ^= 1u;
+                }
+                return ok;
+            };
+            for (uint32_t m = 0;; ++m) {
+                const int slot = (int)(m % kMail);
+                if (!ctl.wait_bar(smem_u32(&sh.mail_full[slot]), (m / kMail) & 1u, kWaitMail, 0)) break;
+                const int4 mail = sh.mail[slot];
+                mbar_arrive(smem_u32(&sh.mail_empty[slot]));
+                if (mail.x < 0) break;
+                __threadfence(); // the workers' scores (ordered before the mail) become visible GPU-wide
+                atomicAdd(p.s1_done + mail.x, 1);
+                if (mail.z && !hand_over(mail.x)) break;
             }
-            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-            const int b = __shfl_sync(0xffffffffu, mail.x, 0), last = __shfl_sync(0xffffffffu, mail.z, 0);
-            if (!ok || b == -1) break;
-            if (b >= 0 && last && !select_pivots_warp(p, sh, ctl, b)) break;
+            hand_over(-1); // end mark for the selectors (also after a failure)
+        }
+    } else if (warp >= kSelWarp0 && warp < kSelWarp0 + kSelWarps) {
+        // ------------------------------------------------------------------ selection
+        const Selectors sg;
+        const int st = sg.tid();
+        for (uint32_t m = 0;; ++m) {
+            const int slot = (int)(m % kDuty);
+            bool fail = !ctl.wait_bar(smem_u32(&sh.duty_full[slot]), (m / kDuty) & 1u, kWaitDuty, 0);
+            if (selectors_any(fail)) break;
+            const int b = sh.duty[slot];
+            sg.sync(); // everyone has read the slot
+            if (st == 0) mbar_arrive(smem_u32(&sh.duty_empty[slot]));
+            if (b < 0) break;
+            // the sample's last task has been counted; the other tasks precede it in the schedule, so their
+            // counts do not depend on anything this CTA still has to do
+            fail = st == 0 && !ctl.wait_flag(p.s1_done + b, kWaitTasks, b, p.T1);
+            if (selectors_any(fail)) break;
+            select_pivots(p, sh, b);
         }
     }
     // ---------------------------------------------------------------------- teardown
