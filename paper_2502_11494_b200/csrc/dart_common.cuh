@@ -87,15 +87,24 @@ __device__ void block_select_threshold(Group g, KeyFn keyfn, int n, uint32_t k, 
     for (int shift = 24; shift >= 0; shift -= 8) {
         for (int i = tid; i < 256; i += gsz) sm.hist[i] = 0;
         g.sync();
-        // warp-aggregated histogram: lanes of a warp that hit the same bin add once (scores of real
-        // tokens share their leading key bytes, which would serialise one atomic per lane)
+        // histogram with one cheap aggregation: the lanes of a warp that share the first valid lane's bin add
+        // once (scores of real tokens share their leading key bytes, which would otherwise serialise one
+        // atomic per lane); lanes in other bins add individually
         for (int j0 = 0; j0 < n; j0 += gsz) {
             const int j = j0 + tid;
             uint32_t key = 0;
             const bool v = j < n && keyfn(j, key) && (key & mask) == prefix;
-            const uint32_t bin = v ? ((key >> shift) & 255u) : 256u;
-            const uint32_t peers = __match_any_sync(0xffffffffu, bin);
-            if (v && (tid & 31) == __ffs(peers) - 1) atomicAdd(&sm.hist[bin], (uint32_t)__popc(peers));
+            const uint32_t bin = (key >> shift) & 255u;
+            const uint32_t valid = __ballot_sync(0xffffffffu, v);
+            if (valid == 0) continue;
+            const uint32_t bin0 = __shfl_sync(0xffffffffu, bin, __ffs(valid) - 1);
+            const uint32_t same = __ballot_sync(0xffffffffu, v && bin == bin0);
+            if (v) {
+                if (bin != bin0)
+                    atomicAdd(&sm.hist[bin], 1u);
+                else if ((tid & 31) == __ffs(same) - 1)
+                    atomicAdd(&sm.hist[bin], (uint32_t)__popc(same));
+            }
         }
         g.sync();
         if (tid < kWarp) {

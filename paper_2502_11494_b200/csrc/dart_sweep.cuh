@@ -56,6 +56,7 @@ constexpr int kDuty = 4;         // samples waiting for their selection
 constexpr int kMaxN = 256;       // pivots per MMA (N dimension)
 constexpr int kMail = 8;         // mailbox slots between the workers and the counter warp
 constexpr int kSelMax = 4096;    // scores of a sample that fit the shared-memory select buffer
+constexpr int kArgminMaxP = 32;  // up to this many pivots: P rounds of group-wide argmin; above: radix select
 constexpr int kStaticSmemReserve = 24576;
 constexpr int kStatusTimeout = -7;
 // which wait expired (second status word)
@@ -366,17 +367,58 @@ __device__ void select_pivots(const Params &p, Shared &sh, int b)
     const int smallest = p.smallest;
     const bool cached = p.n_vis <= kSelMax;
     if (cached) { // the scores were written by other SMs: read them from L2, eight loads in flight per lane
-        for (int j0 = lane; j0 < p.n_vis; j0 += kSel * 8) {
-            float v[8];
+        for (int j0 = lane; j0 < p.n_vis; j0 += kSel * 16) {
+            float v[16];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) v[u] = (j0 + kSel * u < p.n_vis) ? __ldcg(score + j0 + kSel * u) : 0.f;
+            for (int u = 0; u < 16; ++u) v[u] = (j0 + kSel * u < p.n_vis) ? __ldcg(score + j0 + kSel * u) : 0.f;
 #pragma unroll
-            for (int u = 0; u < 8; ++u)
+            for (int u = 0; u < 16; ++u)
                 if (j0 + kSel * u < p.n_vis) {
                     const uint32_t k = order_key(v[u]);
                     sh.sel_keys[j0 + kSel * u] = smallest ? k : ~k; // smaller key = better pivot
                 }
         }
+    }
+    if (cached && p.P <= kArgminMaxP) {
+        // few pivots: every thread keeps the best (key, index) among its own scores; each round the group's
+        // minimum is the next pivot, and only its owner looks for a new best.  (key, index) pairs are unique,
+        // so this is the same order as a full sort: best score first, equal scores by index.
+        g.sync();
+        auto scan = [&]() {
+            unsigned long long best = ~0ull;
+            for (int j = lane; j < p.n_vis; j += kSel) {
+                const unsigned long long k = ((unsigned long long)sh.sel_keys[j] << 32) | (uint32_t)j;
+                best = k < best ? k : best;
+            }
+            return best;
+        };
+        unsigned long long mine = scan();
+        for (int r = 0; r < p.P; ++r) {
+            unsigned long long w = mine;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const unsigned long long x = __shfl_xor_sync(0xffffffffu, w, o);
+                w = x < w ? x : w;
+            }
+            if ((lane & 31) == 0) sh.sel_list[(r & 1) * kSelWarps + (lane >> 5)] = w; // double-buffered by round
+            g.sync();
+            unsigned long long win = sh.sel_list[(r & 1) * kSelWarps];
+#pragma unroll
+            for (int k = 1; k < kSelWarps; ++k) {
+                const unsigned long long x = sh.sel_list[(r & 1) * kSelWarps + k];
+                win = x < win ? x : win;
+            }
+            const uint32_t idx = (uint32_t)(win & 0xffffffffu);
+            if (lane == 0) p.pivot_idx[(size_t)b * p.P + r] = (int32_t)min(idx, (uint32_t)(p.n_vis - 1));
+            if (mine == win) { // the owner: retire the winner and find this thread's next best
+                sh.sel_keys[idx] = 0xffffffffu;
+                mine = scan();
+            }
+        }
+        __threadfence();
+        g.sync();
+        if (lane == 0) st_release(p.piv_ready + b, 1);
+        return;
     }
     int P_pad = 1;
     while (P_pad < p.P) P_pad <<= 1;
