@@ -32,7 +32,7 @@ FALLBACK_HBM_GBS = 6650.0
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="sweep_b256")
@@ -103,7 +103,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -353,7 +353,7 @@ def main():
         import oracle
 
         oracle.build()
-        nb = min(B, 64)
+        nb = min(B, 128)
         kb, hb = W.bits(keys[:nb]), W.bits(hidden[:nb])
         n, dt = time_oracle(w, kb, hb, budget_s=15.0)
         cpu = {"value": n * w.n_vis / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
