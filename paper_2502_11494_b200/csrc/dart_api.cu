@@ -298,7 +298,7 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     if (p.n1 < 2) return DART_ERR_UNSUPPORTED;
     const long long n_all = (long long)B * p.Tm;
     // a row's second sweep follows its first by one sample plus the time the pivots take to appear
-    long long lag = (long long)p.Tm + (o.sweep_lag > 0 ? o.sweep_lag : 4 * ctx->sm_count);
+    long long lag = (long long)p.Tm + (o.sweep_lag > 0 ? o.sweep_lag : 7 * ctx->sm_count);
     p.lag = (uint32_t)(lag < n_all ? lag : n_all);
     if (n_all + p.lag >= (1ll << 30)) return DART_ERR_UNSUPPORTED;
     p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest;
