@@ -75,6 +75,8 @@ typedef struct {
     int32_t path;          /* DART_PATH_* */
     int32_t wait_limit;    /* 0: default (2 s); > 0: time limit in microseconds of every bounded device-side wait */
     int32_t sweep_lag;     /* 0: default; > 0: fused path, extra tasks between a row's two sweeps (tuning) */
+    int32_t test_withhold_pivots; /* testing only: nonzero makes the fused kernel never publish a sample's pivots, so that
+                                     its bounded waits expire and the call ends with DART_ERR_TIMEOUT in dart_status */
 } dart_opts;
 
 /* Optional per-step outputs of dart_reduce_ex; every member is a device pointer or NULL. */
@@ -157,11 +159,11 @@ int dart_status(dart_ctx *ctx);
 
 /*
  * Where the last non-zero status came from (as read by the last dart_status call that returned an error):
- * detail[0] = which bounded wait expired (1 pivots not published, 2 ring stage not freed, 3 drain,
- * 4 accumulator not freed, 5/6 tile not loaded (MMA / row sums), 7 accumulator not filled),
- * detail[1] = index of the task in the kernel's schedule, detail[2] = CTA; for wait 1 also detail[3] = sample,
- * detail[4] = row tiles it had completed, detail[5..10] = column slabs completed in its first row tiles.
- * For bug reports.
+ * detail[0] = which bounded wait of the fused kernel expired (1 pivots not published, 2 ring stage not freed,
+ * 3 drain, 4 accumulator not freed, 5/6 tile not loaded (MMA / row sums), 7 accumulator not filled, 8/9 mailbox,
+ * 10 sweep-1 tasks not all counted, 11/12 selection queue, 13 the CTA's sweep 2 not progressing),
+ * detail[1] = index of the step in the kernel's schedule (or the sample), detail[2] = CTA; for wait 1 also
+ * detail[3] = sample.  For bug reports.
  */
 int dart_status_detail(const dart_ctx *ctx, int32_t detail[11]);
 

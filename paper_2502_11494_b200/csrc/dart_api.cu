@@ -302,6 +302,7 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     p.lag = (uint32_t)(lag < n_all ? lag : n_all);
     if (n_all + p.lag >= (1ll << 30)) return DART_ERR_UNSUPPORTED;
     p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest;
+    p.withhold_pivots = o.test_withhold_pivots;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
     p.keys = (const char *)keys;
     p.psim = ctx->psim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;

@@ -75,6 +75,7 @@ struct Params {
     uint32_t row_bytes, stage1_bytes;  // d * 2; shared-memory bytes of a ring-1 stage (4 rows, 1 KB granules)
     uint32_t lag;                      // steps between the two sweeps (Tm <= lag <= B * Tm)
     int norm_kind, smallest;
+    int withhold_pivots;               // test hook: never publish pivots, so that the bounded waits expire
     unsigned long long wait_ns;        // time limit of every wait
     const char *keys;                  // [B][S][d] bf16
     float *psim;                       // [B][KS][n_vis][P] per-slab partial dot products
@@ -320,6 +321,7 @@ struct Ring {
 struct Shared {
     unsigned long long full1[kMaxStages], empty1[kMaxStages], full2[kMaxStages], empty2[kMaxStages];
     unsigned long long tmem_full[2], tmem_empty[2], mail_full[kMail], mail_empty[kMail];
+    unsigned long long mma_drain; // abort path: completes when the MMAs issued so far have finished
     unsigned long long duty_full[kDuty], duty_empty[kDuty];
     int duty[kDuty]; // samples whose last task has been counted; < 0 ends the stream
     int4 mail[kMail]; // (sample, task index, 1 if it is the sample's last task, -); sample < 0 ends the stream
@@ -418,7 +420,7 @@ __device__ void select_pivots(const Params &p, Shared &sh, int b)
         }
         __threadfence();
         g.sync();
-        if (lane == 0) st_release(p.piv_ready + b, 1);
+        if (lane == 0 && !p.withhold_pivots) st_release(p.piv_ready + b, 1);
         return;
     }
     int P_pad = 1;
@@ -461,7 +463,7 @@ __device__ void select_pivots(const Params &p, Shared &sh, int b)
         p.pivot_idx[(size_t)b * p.P + i] = (int32_t)min((uint32_t)(sh.sel_list[i] & 0xffffffffu), (uint32_t)(p.n_vis - 1));
     __threadfence();
     g.sync();
-    if (lane == 0) st_release(p.piv_ready + b, 1);
+    if (lane == 0 && !p.withhold_pivots) st_release(p.piv_ready + b, 1);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -493,6 +495,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             mbar_init(smem_u32(&sh.tmem_full[a]), 1);
             mbar_init(smem_u32(&sh.tmem_empty[a]), kEpiWarps);
         }
+        mbar_init(smem_u32(&sh.mma_drain), 1);
         for (int m = 0; m < kMail; ++m) {
             mbar_init(smem_u32(&sh.mail_full[m]), 1);
             mbar_init(smem_u32(&sh.mail_empty[m]), 1);
@@ -550,7 +553,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                     ++issued;
                 }
             }
-            if (!ok) // drain: let the copies already issued land before the CTA may exit
+            if (!ok || ctl.aborted()) // drain: let the copies already issued land before the CTA may exit
                 for (long long i = issued > p.n1 ? issued - p.n1 : 0; i < issued; ++i)
                     ctl.wait_bar(smem_u32(&sh.full1[i % p.n1]), (uint32_t)((i / p.n1) & 1), kWaitDrain, i);
         }
@@ -619,7 +622,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                 ++issued;
             }
         }
-        if (!ok && lane == 0)
+        if ((!ok || ctl.aborted()) && lane == 0) // drain, as above
             for (long long i = issued > p.n2 ? issued - p.n2 : 0; i < issued; ++i)
                 ctl.wait_bar(smem_u32(&sh.full2[i % p.n2]), (uint32_t)((i / p.n2) & 1), kWaitDrain, i);
     } else if (warp == 1) {
@@ -653,6 +656,10 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                 if (!ok) break;
                 umma_commit(smem_u32(&sh.tmem_full[acc]));
                 ++s2n;
+            }
+            if (!ok || ctl.aborted()) { // TMEM is freed at the end: first let the MMAs issued so far finish
+                umma_commit(smem_u32(&sh.mma_drain));
+                ctl.wait_bar(smem_u32(&sh.mma_drain), 0, kWaitDrain, -1);
             }
         }
     } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {

@@ -36,7 +36,8 @@ class dart_desc(ctypes.Structure):
 
 class dart_opts(ctypes.Structure):
     _fields_ = [("norm_kind", ctypes.c_int32), ("pivot_smallest", ctypes.c_int32), ("path", ctypes.c_int32),
-                ("wait_limit", ctypes.c_int32), ("sweep_lag", ctypes.c_int32)]
+                ("wait_limit", ctypes.c_int32), ("sweep_lag", ctypes.c_int32),
+                ("test_withhold_pivots", ctypes.c_int32)]
 
 
 class dart_debug(ctypes.Structure):

@@ -193,6 +193,27 @@ def test_fused_path_with_short_and_long_lags(oracle, lag):
     assert all(np.array_equal(a[3][n], b[3][n], equal_nan=(n == "eps")) for n in a[3])
 
 
+def test_expired_wait_is_reported_not_hung():
+    """Bounded waits: with the pivots withheld (a flag that nothing sets) the fused kernel must give up within
+    its time limit, say where, exit normally, and leave the context usable for the next call."""
+    w = W.LLAVA15_B64.with_(B=8)
+    k, h = W.make_batch(w, device="cuda")
+    ctx = dart.Dart(w.B, w.S, w.d, w.n_pivot, w.n_keep)
+    opts = dart.dart_opts(0, 0, dart.DART_PATH_FUSED, 20000, 0, 1)        # 20 ms limit, pivots withheld
+    ctx.reduce(h, k, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, opts=opts)
+    torch.cuda.synchronize()
+    assert ctx.status() == dart.DART_ERR_TIMEOUT
+    rc, detail = dart.dart_status_detail(ctx.handle)
+    assert rc == dart.DART_OK and detail[0] in (1, 13)                    # waiting for pivots / for sweep-2 progress
+    assert ctx.status() == dart.DART_OK                                   # reading cleared it
+    good = ctx.reduce(h, k, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep)   # same context, normal call
+    torch.cuda.synchronize()
+    assert ctx.status() == dart.DART_OK
+    ref = run_gpu(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, path=dart.DART_PATH_STAGED, debug=False)
+    assert np.array_equal(_np(good[1]), ref[1]) and np.array_equal(_np(good[0]), ref[0])
+    ctx.close()
+
+
 def test_argument_validation_launches_nothing():
     k, h = gaussian(2, 64, 32, seed=13)
     ctx = dart.Dart(2, 64, 32, 4, 16)
