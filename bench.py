@@ -188,6 +188,28 @@ def run_reference(args):
     }))
 
 
+def rank_samples(rank, B):
+    """Weak scaling over independent samples: rank r reduces samples [r * B, (r + 1) * B) of the workload's
+    seeded stream, so no two ranks hold the same sample and no data-path exchange is needed."""
+    return range(rank * B, rank * B + B)
+
+
+def max_over_ranks(value, device, dist_on):
+    """The slowest rank's value (a job is as fast as its slowest rank)."""
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    if dist_on:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tokens_per_s(world, B, n_vis, steps, ms):
+    """Whole-job throughput: the tokens all ranks reduced divided by the slowest rank's time."""
+    return world * B * n_vis * steps / (ms * 1e-3)
+
+
 def workload_config(w, B):
     return {"workload": w.name, "batch": B, "n_vis": w.n_vis, "seq_len": w.S, "d": w.d, "n_pivot": w.n_pivot,
             "n_keep": w.n_keep, "vis_offset": w.vis_offset, "l2": "inputs larger than L2 (no flush needed)"}
@@ -254,7 +276,7 @@ def main():
     w = pick_workload(args)
     B = w.B
     # weak scaling: every rank reduces its own batch of B samples
-    keys, hidden = W.make_batch(w, device=dev, samples=range(rank * B, rank * B + B))
+    keys, hidden = W.make_batch(w, device=dev, samples=rank_samples(rank, B))
     flags = 0 if args.no_e2e else dart.DART_FLAG_HOST_STAGING
     ctx = dart.Dart(B, w.S, w.d, max(w.n_pivot, max(W.SWEEP_PIVOTS) if args.sweep else 0),
                     max(w.n_keep, max(W.SWEEP_KEEP) if args.sweep else 0), device=local, flags=flags)
@@ -271,12 +293,9 @@ def main():
     sampler.start()
     ms, launches, prof = time_steps(ctx, dart, torch, w, keys, hidden, outs, args.steps, args.warmup, opts, dist_on)
     clocks = sampler.stop()
-    t = torch.tensor([ms], device=dev, dtype=torch.float64)
-    if dist_on:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms = float(t.item())
+    ms = max_over_ranks(ms, dev, dist_on)
     ms_per_step = ms / args.steps
-    value = world * B * w.n_vis * args.steps / (ms * 1e-3)
+    value = job_tokens_per_s(world, B, w.n_vis, args.steps, ms)
 
     peak, peak_src = measured_peak()
     # dominant kernel = the slot with the largest share of the timed region
@@ -337,10 +356,7 @@ def main():
         for _ in range(n_e2e):
             host_step()
         dt = time.perf_counter() - t0
-        td = torch.tensor([dt], device=dev, dtype=torch.float64)
-        if dist_on:
-            dist.all_reduce(td, op=dist.ReduceOp.MAX)
-        dt = float(td.item())
+        dt = max_over_ranks(dt, dev, dist_on)
         ok = bool(torch.equal(ho[1], outs[1][:Be].cpu())) if not args.sweep else None
         e2e = {"value": world * Be * w.n_vis * n_e2e / dt, "unit": UNIT,
                "h2d_bytes_per_step": int(hk.numel() * 2 + hh.numel() * 2),
