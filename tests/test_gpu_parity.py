@@ -158,6 +158,53 @@ def test_benchmark_configs(oracle, w, path):
     assert rep.max_rel_l1 < 5e-5 and rep.max_abs_sim < 2e-5
 
 
+@pytest.fixture(scope="module")
+def sweep_batch():
+    """The benchmark's batch: 256 x 2980 x 4096 bf16 keys and hidden states (12.5 GB), generated once."""
+    w = W.SWEEP_B256
+    k, h = W.make_batch(w, device="cuda")
+    yield w, k, h
+    del k, h
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("cell", [(8, 320), (8, 64), (32, 320), (128, 640), (128, 320)], ids=lambda c: "P%d_K%d" % c)
+def test_full_size_sweep_cells(oracle, sweep_batch, cell):
+    """Config 5 at its full size, called exactly as bench.py calls it (default path, no per-step outputs):
+    the oracle checks sampled samples one by one; properties that hold at any size are checked on all 256."""
+    w, k, h = sweep_batch
+    P, Kp = cell
+    ctx = dart.Dart(w.B, w.S, w.d, P, Kp)
+    try:
+        oh, oi, op = ctx.reduce(h, k, w.vis_offset, w.n_vis, P, Kp)
+        torch.cuda.synchronize()
+        st = ctx.status()
+        assert st == dart.DART_OK, (st, dart.dart_status_detail(ctx.handle))
+    finally:
+        ctx.close()
+    S_out = w.S - w.n_vis + Kp
+    # all samples: strictly ascending indices, text rows intact, position ids = indices, gathered rows = hidden rows
+    d_oi = oi[:, 1:] - oi[:, :-1]
+    assert bool((d_oi > 0).all()) and oi.shape == (w.B, S_out)
+    assert bool((oi[:, :w.vis_offset] == torch.arange(w.vis_offset, device="cuda", dtype=torch.int32)).all())
+    n_after = w.S - w.vis_offset - w.n_vis
+    assert bool((oi[:, S_out - n_after:] == torch.arange(w.vis_offset + w.n_vis, w.S, device="cuda", dtype=torch.int32)).all())
+    assert bool((op == oi.to(torch.int64)).all())
+    rows = torch.gather(h.view(torch.int16), 1, oi.to(torch.int64).unsqueeze(-1).expand(-1, -1, w.d))
+    assert bool((rows == oh.view(torch.int16)).all())
+    del rows
+    # sampled samples against the oracle (first, last and a few in between)
+    sel = [0, 97, 255] if P >= 128 else [0, 1, 63, 128, 200, 255]
+    kb, hb = W.bits(k[sel]), W.bits(h[sel])
+    ora = oracle.reduce(hb, kb, w.vis_offset, w.n_vis, P, Kp, want_dup=False)
+    rep = parity.check_batch(ora, kb, hb, w.vis_offset, w.n_vis, P, Kp, W.bits(oh[sel]), oi[sel].cpu().numpy(),
+                             op[sel].cpu().numpy())
+    assert rep.exact >= rep.above_margin
+    # without per-step outputs the replay under tolerance is not available: fp32 accumulation keeps the CUDA
+    # path ~1e-6 from the oracle, so near-ties that flip are rare
+    assert rep.exact >= len(sel) - 1, rep.notes
+
+
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
 def test_runs_are_bitwise_reproducible(path):
     w = W.LLAVA15_B64.with_(B=4)
