@@ -74,7 +74,6 @@ def kernel_bytes_per_launch(name, w, B):
         "score": keys + 8 * w.n_vis * B,
         "sim": keys + 4 * w.n_pivot * w.n_vis * B,
         "sweep": keys,                       # fused scores + pivots + similarities: the keys count once
-        "finalize": 4 * w.n_pivot * w.n_vis * B,
         "gather": 2 * (2 * w.d * w.S_out) * B,
         "pivot": 4 * w.n_vis * B,
         "retain": 4 * w.n_pivot * w.n_vis * B + 12 * w.S_out * B,

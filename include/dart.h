@@ -161,7 +161,7 @@ int dart_status(dart_ctx *ctx);
  * Where the last non-zero status came from (as read by the last dart_status call that returned an error):
  * detail[0] = which bounded wait of the fused kernel expired (1 pivots not published, 2 ring stage not freed,
  * 3 drain, 4 accumulator not freed, 5/6 tile not loaded (MMA / row sums), 7 accumulator not filled, 8/9 mailbox,
- * 10 sweep-1 tasks not all counted, 11/12 selection queue, 13 the CTA's sweep 2 not progressing),
+ * 10 sweep-1 tasks not all counted, 11/12 selection queue),
  * detail[1] = index of the step in the kernel's schedule (or the sample), detail[2] = CTA; for wait 1 also
  * detail[3] = sample.  For bug reports.
  */

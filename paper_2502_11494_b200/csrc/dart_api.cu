@@ -12,8 +12,8 @@
 
 namespace {
 
-enum Slot { SLOT_SCORE = 0, SLOT_PIVOT, SLOT_SIM, SLOT_RETAIN, SLOT_GATHER, SLOT_SWEEP, SLOT_FINALIZE, SLOT_COUNT };
-const char *const kSlotNames[SLOT_COUNT] = {"score", "pivot", "sim", "retain", "gather", "sweep", "finalize"};
+enum Slot { SLOT_SCORE = 0, SLOT_PIVOT, SLOT_SIM, SLOT_RETAIN, SLOT_GATHER, SLOT_SWEEP, SLOT_COUNT };
+const char *const kSlotNames[SLOT_COUNT] = {"score", "pivot", "sim", "retain", "gather", "sweep"};
 
 typedef CUresult (*TensorMapEncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                       const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -53,8 +53,7 @@ struct dart_ctx {
     cudaEvent_t ev_in[2], ev_run[2], ev_out[2];
     // fused path (csrc/dart_sweep.cuh); available when d is a multiple of 64 and the device is sm_100
     bool fused_ok;
-    int sm_count, KS, n_atoms, N_max;
-    float *psim;
+    int sm_count, n_atoms;
     int *counters;
     size_t counters_bytes;
     TensorMapEncodeFn encode;
@@ -239,11 +238,7 @@ int fused_setup(dart_ctx *ctx)
         return DART_OK;
     ctx->encode = (TensorMapEncodeFn)fn;
     ctx->n_atoms = D.d / kAtomCols;
-    ctx->KS = (ctx->n_atoms + kSlabAtoms - 1) / kSlabAtoms;
-    const int P_cap = D.P_max < kMaxN ? D.P_max : kMaxN;
-    ctx->N_max = (P_cap + 15) / 16 * 16;
-    const size_t nv = (size_t)D.B_max * D.S_max;
-    int rc = ws_alloc(ctx, &ctx->psim, nv * ctx->KS * P_cap);
+    int rc = DART_OK;
     ctx->counters_bytes = (size_t)D.B_max * 2 * sizeof(int);
     if (rc == DART_OK) rc = ws_alloc(ctx, (uint8_t **)&ctx->counters, ctx->counters_bytes);
     if (rc != DART_OK) return rc;
@@ -291,8 +286,8 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     const void *keys = keys_in ? keys_in : hidden;
     Params p = {};
     p.B = B, p.S = S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.N = (P + 15) / 16 * 16, p.d8 = d8;
-    p.n_atoms = ctx->n_atoms, p.KS = ctx->KS, p.n_rt = (n_vis + kTileRows - 1) / kTileRows;
-    p.T1 = (n_vis + kS1Rows - 1) / kS1Rows, p.T2 = p.n_rt * p.KS, p.Tm = p.T1 > p.T2 ? p.T1 : p.T2;
+    p.n_atoms = ctx->n_atoms, p.n_rt = (n_vis + kTileRows - 1) / kTileRows;
+    p.T1 = (n_vis + kS1Rows - 1) / kS1Rows, p.T2 = p.n_rt, p.Tm = p.T1 > p.T2 ? p.T1 : p.T2;
     p.row_bytes = (uint32_t)ctx->desc.d * 2, p.stage1_bytes = stage1_bytes(p.row_bytes);
     ring_depths(p.N, p.row_bytes, ctx->max_smem_optin, p.n1, p.n2);
     if (p.n1 < 2) return DART_ERR_UNSUPPORTED;
@@ -305,7 +300,7 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     p.withhold_pivots = o.test_withhold_pivots;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
     p.keys = (const char *)keys;
-    p.psim = ctx->psim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
+    p.sim = ctx->sim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
     p.s1_done = ctx->counters, p.piv_ready = ctx->counters + B;
     p.status = ctx->status;
     // the same tensor with a 128-row box (full tiles), a 32-row box (short last tiles) and a one-row box (pivot rows)
@@ -321,12 +316,6 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
         void *args[4] = {&tm_tile, &tm_keys, &tm_row, &p};
         DART_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)sweep_kernel, dim3((unsigned)grid), dim3(kThreads), args,
                                                    smem_bytes(p.N, p.row_bytes, p.n1, p.n2), st));
-    }
-    {
-        Prof pr(ctx, st, SLOT_FINALIZE);
-        dim3 grid((n_vis + kFinalizeThreads - 1) / kFinalizeThreads, B);
-        finalize_sim_kernel<<<grid, kFinalizeThreads, 0, st>>>(ctx->psim, ctx->ssq, ctx->pivot_idx, n_vis, P, p.KS,
-                                                               ctx->status, ctx->sim);
     }
     {
         Prof pr(ctx, st, SLOT_RETAIN);
@@ -450,7 +439,6 @@ int dart_destroy(dart_ctx *ctx)
     cudaFree(ctx->owner);
     cudaFree(ctx->keep);
     cudaFree(ctx->status);
-    cudaFree(ctx->psim);
     cudaFree(ctx->counters);
     for (int k = 0; k < 2; ++k) {
         cudaFree(ctx->st_hidden[k]);

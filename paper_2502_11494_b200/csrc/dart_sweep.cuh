@@ -5,21 +5,20 @@
 // Sweep-1 task: 16 whole key rows (one contiguous block of 16 * d * 2 bytes), streamed through shared
 // memory four rows at a time; each of four worker warps sums one row (L1 norm: the K-norm of the
 // Sec. 3.3 footnote; sum of squares: Eq. 7's denominator) and writes the final values - no partial sums.
-// Sweep-2 task: 128 rows x 512 columns as 128-byte-swizzled TMA tiles, multiplied on the tensor cores
-// with the sample's pivot rows (Eq. 7's numerator); the per-column-slab partial products are added up
-// by a small kernel afterwards.
+// Sweep-2 task: 128 rows x all d columns, streamed as 128-byte-swizzled TMA tiles of 64 columns and
+// multiplied on the tensor cores with the sample's pivot rows, accumulating over all of d in TMEM
+// (Eq. 7's numerator); the epilogue divides by the two norms and writes dup(p_i, x_j) (Eq. 7).
 // Both kinds of task sit in one global, static order: step q = (sweep-1 task q, sweep-2 task q - lag),
 // CTA c runs steps c, c + grid, ...  A sweep-2 task therefore follows the sweep-1 pass over its sample
 // by `lag` steps, which is what bounds the distance between the two reads of a row.
 //
 // Per CTA (512 threads; warp 3 idles):
-//   warp 0     sweep-1 producer: bulk copies into ring 1 (L2 evict_last), at most one round ahead of
-//              the CTA's own sweep-2 progress
+//   warp 0     sweep-1 producer: bulk copies into ring 1
 //   warp 2     sweep-2 producer: waits for the sample's pivots, then TMA tiles (L2 evict_first) and the
 //              pivot rows (tile::gather4 straight from the key tensor) into ring 2
 //   warp 1     sweep 2: one thread issues tcgen05.mma (tokens = M 128, pivots = N, bf16 -> fp32 in TMEM)
 //   warps 4-7  sweep-1 workers (one row per warp and stage)
-//   warps 8-11 sweep-2 epilogue: TMEM -> partial dot products in global memory
+//   warps 8-11 sweep-2 epilogue: TMEM -> normalised similarities [B][P][n_vis] in global memory
 //   warp 12    counter: counts finished sweep-1 tasks (the fence and the atomic are kept off the
 //              workers by a mailbox); when it counts a sample's LAST task it hands the sample over to
 //   warps 13-15 selection: wait until all of the sample's tasks are counted, select the pivots (Def. 1)
@@ -40,7 +39,6 @@ namespace sweep {
 constexpr int kTileRows = 128;   // sweep-2 tile rows (MMA M)
 constexpr int kAtomCols = 64;    // 64 bf16 = 128 bytes = one swizzle row
 constexpr int kSubRows = 32;     // rows per TMA box of a short last tile
-constexpr int kSlabAtoms = 8;    // a sweep-2 task spans 8 atoms = 512 columns
 constexpr int kS1Rows = 16;      // rows per sweep-1 task
 constexpr int kS1StageRows = 4;  // rows per sweep-1 stage: one per worker warp
 constexpr int kMaxRowBytes = 16384; // widest row the fused path takes (d <= 8192)
@@ -57,11 +55,11 @@ constexpr int kMaxN = 256;       // pivots per MMA (N dimension)
 constexpr int kMail = 8;         // mailbox slots between the workers and the counter warp
 constexpr int kSelMax = 4096;    // scores of a sample that fit the shared-memory select buffer
 constexpr int kArgminMaxP = 32;  // up to this many pivots: P rounds of group-wide argmin; above: radix select
-constexpr int kStaticSmemReserve = 24576;
+constexpr int kStaticSmemReserve = 28672;
 constexpr int kStatusTimeout = -7;
 // which wait expired (second status word)
 enum { kWaitPivots = 1, kWaitEmptyStage, kWaitDrain, kWaitAccumFree, kWaitStageMma, kWaitStageRows, kWaitAccumFull,
-       kWaitMailSlot, kWaitMail, kWaitTasks, kWaitDutySlot, kWaitDuty, kWaitSweep2 };
+       kWaitMailSlot, kWaitMail, kWaitTasks, kWaitDutySlot, kWaitDuty };
 
 using Workers = WarpGroup<kWorkerWarp0, kWorkerWarps, 1>;
 using Selectors = WarpGroup<kSelWarp0, kSelWarps, 2>;
@@ -69,7 +67,7 @@ using Selectors = WarpGroup<kSelWarp0, kSelWarps, 2>;
 struct Params {
     int B, S, vis_offset, n_vis, P, N; // N = P rounded up to a multiple of 16 (MMA N)
     int d8;                            // row width in 16-byte units
-    int n_atoms, KS, n_rt;             // sweep 2: atoms per row; column slabs; row tiles per sample
+    int n_atoms, n_rt;                 // sweep 2: 64-column atoms per row; row tiles (tasks) per sample
     int T1, T2, Tm;                    // tasks per sample: sweep 1, sweep 2; slots per sample = max of both
     int n1, n2;                        // depth of ring 1 and ring 2 (<= kMaxStages each)
     uint32_t row_bytes, stage1_bytes;  // d * 2; shared-memory bytes of a ring-1 stage (4 rows, 1 KB granules)
@@ -78,7 +76,7 @@ struct Params {
     int withhold_pivots;               // test hook: never publish pivots, so that the bounded waits expire
     unsigned long long wait_ns;        // time limit of every wait
     const char *keys;                  // [B][S][d] bf16
-    float *psim;                       // [B][KS][n_vis][P] per-slab partial dot products
+    float *sim;                        // [B][P][n_vis] dup(p_i, x_j)
     float *l1, *ssq;                   // [B][n_vis]
     int32_t *pivot_idx;                // [B][P]
     int *s1_done;                      // [B] sweep-1 tasks counted per sample
@@ -89,7 +87,7 @@ struct Params {
 struct Task {
     int b;
     int u;      // sweep 1: task index within the sample (rows 16 u ...)
-    int rt, ks; // sweep 2: row tile and column slab
+    int rt;     // sweep 2: row tile
 };
 
 // Schedule.  Every sample owns Tm consecutive slots in each sweep (a slot beyond the sweep's own task count is
@@ -106,13 +104,12 @@ __device__ __forceinline__ bool decode(const Params &p, uint32_t q, int kind, Ta
     const uint32_t u = n - (uint32_t)t.b * Tm;
     t.u = (int)u;
     if (kind == 0) return u < (uint32_t)p.T1;
-    if (u >= (uint32_t)p.T2) return false;
-    t.rt = (int)(u / (uint32_t)p.KS);
-    t.ks = (int)(u - (uint32_t)t.rt * (uint32_t)p.KS);
-    return true;
+    // a sample's T2 sweep-2 tasks are spread evenly over its Tm slots (every stride-th slot carries one)
+    const uint32_t stride = Tm / (uint32_t)p.T2;
+    t.rt = (int)(u / stride);
+    return u % stride == 0 && t.rt < p.T2;
 }
 
-__device__ __forceinline__ int slab_atoms(const Params &p, int ks) { return min(kSlabAtoms, p.n_atoms - ks * kSlabAtoms); }
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *ptr) { return (uint32_t)__cvta_generic_to_shared(ptr); }
@@ -265,23 +262,6 @@ struct Ctl {
             }
         }
     }
-    // waits until a shared-memory counter reaches target
-    __device__ bool wait_count(const volatile int *cnt, int target, int where, long long task) const
-    {
-        if (*cnt >= target) return true;
-        const long long t0 = clock64();
-        for (uint32_t it = 0;; ++it) {
-            if (*cnt >= target) return true;
-            __nanosleep(64);
-            if ((it & 15u) == 15u) {
-                if (aborted()) return false;
-                if ((unsigned long long)(clock64() - t0) > limit_cycles) {
-                    give_up(where, task);
-                    return false;
-                }
-            }
-        }
-    }
     // waits until *flag >= target
     __device__ bool wait_flag(const int *flag, int where, long long task, int target = 1) const
     {
@@ -330,8 +310,8 @@ struct Shared {
     unsigned long long sel_list[kMaxN];
     SelectSmem sel;
     uint32_t tmem_base, n_picked;
+    float pivot_norm[kEpiWarps][kMaxN]; // per epilogue warp: Euclidean norms of the current sample's pivots
     int abort_flag;
-    volatile int s2_step; // last schedule step whose sweep-2 task this CTA has finished (-1: none yet)
 };
 static_assert(sizeof(Shared) + 64 <= kStaticSmemReserve, "static shared memory exceeds its reserve");
 
@@ -505,7 +485,6 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             mbar_init(smem_u32(&sh.duty_empty[m]), 1);
         }
         sh.abort_flag = 0;
-        sh.s2_step = -1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     uint32_t tmem_cols = 32;
@@ -533,13 +512,6 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
                 Task t;
                 if (!decode(p, g, 0, t)) continue;
-                // stay within one round of this CTA's sweep-2 progress: the step one round back has a sweep-2
-                // task if it is >= lag, and that task must be finished before more rows are pulled in
-                if (g >= gridDim.x && g - gridDim.x >= p.lag) {
-                    Task t2;
-                    if (decode(p, g - gridDim.x, 1, t2)) ok = ctl.wait_count(&sh.s2_step, (int)(g - gridDim.x), kWaitSweep2, g);
-                    if (!ok) break;
-                }
                 const int row0 = t.u * kS1Rows, rows = min(kS1Rows, p.n_vis - row0);
                 const char *src = p.keys + ((size_t)t.b * p.S + p.vis_offset + row0) * (size_t)p.row_bytes;
                 for (int r = 0; r < rows; r += kS1StageRows) {
@@ -590,7 +562,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                     }
                 cur_b = t.b;
             }
-            const int na = slab_atoms(p, t.ks);
+            const int na = p.n_atoms;
             const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
             const int n_sub = (rows + kSubRows - 1) / kSubRows;
             const int y0 = t.b * p.S + p.vis_offset + t.rt * kTileRows;
@@ -604,7 +576,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                 }
                 ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
                 if (!ok) break;
-                const int x = (t.ks * kSlabAtoms + a) * kAtomCols;
+                const int x = a * kAtomCols;
                 const uint32_t dst = a2_addr(ring.stage);
                 if (rows == kTileRows) {
                     if (lane == 0) tma_load_2d(dst, &tm_tile, x, y0, full, pol_drop);
@@ -635,7 +607,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
                 Task t;
                 if (!decode(p, g, 1, t)) continue;
-                const int na = slab_atoms(p, t.ks);
+                const int na = p.n_atoms;
                 const uint32_t acc = s2n & 1u;
                 ok = ctl.wait_bar(smem_u32(&sh.tmem_empty[acc]), ((s2n >> 1) & 1u) ^ 1u, kWaitAccumFree, g);
                 if (!ok) break;
@@ -666,6 +638,8 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
         // ------------------------------------------------------------------ sweep-2 epilogue (warps independent)
         const int quarter = warp & 3;        // TMEM lane quarter this warp may read
         const int row = quarter * 32 + lane; // tile row owned by this thread
+        float *pn = sh.pivot_norm[quarter];
+        int cur_b = -1;
         uint32_t s2n = 0;
         for (uint32_t g = blockIdx.x; g < total; g += gridDim.x) {
             Task t;
@@ -676,27 +650,35 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             bool ok = ctl.wait_bar(smem_u32(&sh.tmem_full[acc]), (s2n >> 1) & 1u, kWaitAccumFull, g);
             if (!__all_sync(0xffffffffu, ok)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            // the accumulator exists, so the sample's pivots and all of its norms were published long ago
+            if (t.b != cur_b) {
+                __syncwarp();
+                for (int i = lane; i < p.P; i += 32) {
+                    const int piv = min(max(__ldcg(p.pivot_idx + (size_t)t.b * p.P + i), 0), p.n_vis - 1);
+                    pn[i] = sqrtf(__ldcg(p.ssq + (size_t)t.b * p.n_vis + piv));
+                }
+                __syncwarp();
+                cur_b = t.b;
+            }
+            const float nj = row < rows ? sqrtf(__ldcg(p.ssq + (size_t)t.b * p.n_vis + j)) : 0.f;
             const uint32_t taddr = tmem_base + acc * (uint32_t)p.N + ((uint32_t)(quarter * 32) << 16);
-            float *dst = p.psim + (((size_t)t.b * p.KS + t.ks) * p.n_vis + j) * p.P;
+            float *dst = p.sim + (size_t)t.b * p.P * p.n_vis + j;
             for (int c0 = 0; c0 < p.P; c0 += 8) {
                 float v[8];
                 tmem_ld8(taddr + (uint32_t)c0, v); // warp-collective: rows outside the tile still take part
                 if (row < rows) {
-                    if (c0 + 8 <= p.P && (p.P & 3) == 0) {
-                        *reinterpret_cast<float4 *>(dst + c0) = make_float4(v[0], v[1], v[2], v[3]);
-                        *reinterpret_cast<float4 *>(dst + c0 + 4) = make_float4(v[4], v[5], v[6], v[7]);
-                    } else {
 #pragma unroll
-                        for (int e = 0; e < 8; ++e)
-                            if (c0 + e < p.P) dst[c0 + e] = v[e];
-                    }
+                    for (int e = 0; e < 8; ++e)
+                        if (c0 + e < p.P) { // dup = dot / (|pivot| |row|); a zero norm gives 0; a warp writes 128 contiguous bytes
+                            const float den = pn[c0 + e] * nj;
+                            dst[(size_t)(c0 + e) * p.n_vis] = den > 0.f ? v[e] / den : 0.f;
+                        }
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(smem_u32(&sh.tmem_empty[acc]));
-                if (quarter == 0) sh.s2_step = (int)g; // progress mark for the sweep-1 producer's throttle
             }
             ++s2n;
         }
@@ -813,40 +795,6 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (warp == 1)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
-}
-
-// Adds up the per-slab partial dot products in slab order and normalises them (Eq. 7):
-// sim[b][i][j] = (sum_ks psim[b][ks][j][i]) / (|K_{p_i}| |K_j|); a zero norm gives 0.
-constexpr int kFinalizeThreads = 128;
-
-__global__ void __launch_bounds__(kFinalizeThreads)
-finalize_sim_kernel(const float *__restrict__ psim, const float *__restrict__ ssq, const int32_t *__restrict__ pivot_idx,
-                    int n_vis, int P, int KS, const int *__restrict__ status, float *__restrict__ sim)
-{
-    const int b = blockIdx.y, j = blockIdx.x * kFinalizeThreads + threadIdx.x;
-    if (j >= n_vis || *status != 0) return; // after a failed sweep the pivots are undefined
-    const float nj = sqrtf(ssq[(size_t)b * n_vis + j]);
-    const int32_t *piv = pivot_idx + (size_t)b * P;
-    for (int p0 = 0; p0 < P; p0 += 4) {
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int ks = 0; ks < KS; ++ks) {
-            const float *src = psim + (((size_t)b * KS + ks) * n_vis + j) * P + p0;
-            if ((P & 3) == 0) {
-                const float4 v = __ldcs(reinterpret_cast<const float4 *>(src));
-                acc[0] += v.x, acc[1] += v.y, acc[2] += v.z, acc[3] += v.w;
-            } else {
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (p0 + e < P) acc[e] += __ldcs(src + e);
-            }
-        }
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            if (p0 + e >= P) break;
-            const float den = sqrtf(ssq[(size_t)b * n_vis + piv[p0 + e]]) * nj;
-            sim[((size_t)b * P + p0 + e) * n_vis + j] = den > 0.f ? acc[e] / den : 0.f;
-        }
-    }
 }
 
 } // namespace sweep

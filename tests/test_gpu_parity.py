@@ -251,7 +251,7 @@ def test_expired_wait_is_reported_not_hung():
     torch.cuda.synchronize()
     assert ctx.status() == dart.DART_ERR_TIMEOUT
     rc, detail = dart.dart_status_detail(ctx.handle)
-    assert rc == dart.DART_OK and detail[0] in (1, 13)                    # waiting for pivots / for sweep-2 progress
+    assert rc == dart.DART_OK and detail[0] == 1                          # the wait for the pivots gave up first
     assert ctx.status() == dart.DART_OK                                   # reading cleared it
     good = ctx.reduce(h, k, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep)   # same context, normal call
     torch.cuda.synchronize()
