@@ -205,9 +205,9 @@ int launch_staged(dart_ctx *ctx, int B, const void *hidden, const void *keys_in,
     }
     {
         Prof p(ctx, st, SLOT_RETAIN);
-        retain_kernel<<<B, kSelectThreads, (size_t)n_vis, st>>>(ctx->sim, ctx->pivot_idx, pos_in, S, vis_offset, n_vis, P,
+        retain_kernel<<<B, kSelectThreads, retain_smem_bytes(n_vis, P), st>>>(ctx->sim, ctx->pivot_idx, pos_in, S, vis_offset, n_vis, P,
                                                                n_keep, out_idx, out_pos, ctx->keep, ctx->owner,
-                                                               ctx->eps, ctx->status);
+                                                               ctx->eps, ctx->status, retain_cache_rows(n_vis, P));
     }
     {
         Prof p(ctx, st, SLOT_GATHER);
@@ -319,9 +319,9 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     }
     {
         Prof pr(ctx, st, SLOT_RETAIN);
-        retain_kernel<<<B, kSelectThreads, (size_t)n_vis, st>>>(ctx->sim, ctx->pivot_idx, pos_in, S, vis_offset, n_vis, P,
+        retain_kernel<<<B, kSelectThreads, retain_smem_bytes(n_vis, P), st>>>(ctx->sim, ctx->pivot_idx, pos_in, S, vis_offset, n_vis, P,
                                                                n_keep, out_idx, out_pos, ctx->keep, ctx->owner,
-                                                               ctx->eps, ctx->status);
+                                                               ctx->eps, ctx->status, retain_cache_rows(n_vis, P));
     }
     {
         Prof pr(ctx, st, SLOT_GATHER);
@@ -383,12 +383,13 @@ int dart_create(dart_ctx **out, const dart_desc *desc)
     if (rc == DART_OK) {
         cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, desc->device);
         size_t sim_smem = (size_t)dart::kSimPivotChunk * (desc->d / 8) * 16;
-        if (sim_smem > (size_t)ctx->max_smem_optin || (size_t)desc->S_max > (size_t)ctx->max_smem_optin)
+        if (sim_smem > (size_t)ctx->max_smem_optin ||
+            (size_t)desc->S_max + 16 + dart::kRetainCacheBytes > (size_t)ctx->max_smem_optin)
             rc = DART_ERR_BAD_SHAPE; // rows wider than 8 pivot rows of shared memory are not supported
         else if (cudaFuncSetAttribute(dart::sim_alu_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)sim_smem) != cudaSuccess ||
                  cudaFuncSetAttribute(dart::retain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      desc->S_max) != cudaSuccess)
+                                      desc->S_max + 16 + dart::kRetainCacheBytes) != cudaSuccess)
             rc = DART_ERR_CUDA;
     }
     if (rc == DART_OK) rc = fused_setup(ctx);

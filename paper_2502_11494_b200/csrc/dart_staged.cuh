@@ -182,16 +182,29 @@ sim_alu_kernel(const uint4 *__restrict__ keys, int S, int d8, int vis_offset, in
 // kept := pivots; pivot i in rank order selects its q_i not-yet-kept tokens of lowest dup (radix
 // select on order-preserving keys, ties to the lower index); eps_i is the selection threshold.
 // Then an ordered scan over the keep flags writes the ascending kept indices and position ids.
-// Dynamic shared memory: n_vis bytes (keep flags).
+// Dynamic shared memory: n_vis bytes (keep flags, rounded up to 16) + cache_rows * n_vis * 4 bytes: the
+// similarity rows of cache_rows pivots at a time are held as order-preserving keys, so that the select's
+// passes read shared memory (cache_rows = 0: every pass reads the row from global memory).
+constexpr int kRetainCacheBytes = 96 * 1024; // shared-memory budget of the row cache (two CTAs per SM)
+inline int retain_cache_rows(int n_vis, int P)
+{
+    int r = (int)((size_t)kRetainCacheBytes / ((size_t)n_vis * 4));
+    return r > P ? P : r;
+}
+inline size_t retain_smem_bytes(int n_vis, int P)
+{
+    return ((size_t)n_vis + 15) / 16 * 16 + (size_t)retain_cache_rows(n_vis, P) * n_vis * 4;
+}
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kSelectThreads)
 retain_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx, const int64_t *__restrict__ pos_in,
               int S, int vis_offset, int n_vis, int P, int n_keep,
               int32_t *__restrict__ out_idx, int64_t *__restrict__ out_pos,
               uint8_t *__restrict__ keep_out, int32_t *__restrict__ owner_out, float *__restrict__ eps_out,
-              const int *__restrict__ status)
+              const int *__restrict__ status, int cache_rows)
 {
-    extern __shared__ uint8_t keep[]; // [n_vis]
+    extern __shared__ __align__(16) uint8_t keep[]; // [n_vis] flags, then the key cache
+    uint32_t *cache = reinterpret_cast<uint32_t *>(keep + ((size_t)n_vis + 15) / 16 * 16); // [cache_rows][n_vis]
     __shared__ SelectSmem sel;
     if (*status != 0) return; // an earlier kernel of this call failed: its outputs are undefined
     const int b = blockIdx.x;
@@ -216,9 +229,16 @@ retain_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_i
             continue;
         }
         const float *row = sim + ((size_t)b * P + i) * n_vis;
+        if (cache_rows > 0 && i % cache_rows == 0) { // load the next cache_rows rows (all loads independent)
+            const int nr = min(cache_rows, P - i);
+            __syncthreads();
+            for (int idx = threadIdx.x; idx < nr * n_vis; idx += blockDim.x) cache[idx] = order_key(row[idx]);
+            __syncthreads();
+        }
+        const uint32_t *krow = cache + (size_t)(cache_rows > 0 ? i % cache_rows : 0) * n_vis;
         auto keyfn = [&](int j, uint32_t &key) {
             if (keep[j]) return false;
-            key = order_key(row[j]);
+            key = cache_rows > 0 ? krow[j] : order_key(row[j]);
             return true;
         };
         uint32_t T, need_eq, cnt_eq;

@@ -8,9 +8,9 @@
 // Sweep-2 task: 128 rows x all d columns, streamed as 128-byte-swizzled TMA tiles of 64 columns and
 // multiplied on the tensor cores with the sample's pivot rows, accumulating over all of d in TMEM
 // (Eq. 7's numerator); the epilogue divides by the two norms and writes dup(p_i, x_j) (Eq. 7).
-// Both kinds of task sit in one global, static order: step q = (sweep-1 task q, sweep-2 task q - lag),
+// Both kinds of task sit in one global, static order: step q = (sweep-1 slot q, sweep-2 slot q - lag),
 // CTA c runs steps c, c + grid, ...  A sweep-2 task therefore follows the sweep-1 pass over its sample
-// by `lag` steps, which is what bounds the distance between the two reads of a row.
+// by `lag` steps: enough for the sample's pivots to have been selected and published meanwhile.
 //
 // Per CTA (512 threads; warp 3 idles):
 //   warp 0     sweep-1 producer: bulk copies into ring 1
@@ -505,7 +505,8 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
         // ------------------------------------------------------------------ sweep-1 producer
         if (lane == 0) {
             unsigned long long pol_keep;
-            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+            // the second read of a row comes too late to find it in L2 (see the design notes), so nothing is kept
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_keep));
             Ring ring(p.n1);
             long long issued = 0;
             bool ok = true;
