@@ -80,6 +80,12 @@ def kernel_bytes_per_launch(name, w, B):
     }[name]
 
 
+# DRAM traffic of one launch per sample (dram__bytes_read.sum + dram__bytes_write.sum), from the ncu capture of the
+# sweep workload at batch 32 summarised in profiles/sweep_kernel_sweep_b32.md; traffic is proportional to the batch
+# (every sample is read and written independently), so a launch over B samples moves B times this.
+NCU_TRAFFIC_PER_SAMPLE = {("sweep", 2880, 4096, 8): (1.508212e9 + 5.538816e6) / 32}
+
+
 def measured_peak():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -304,7 +310,10 @@ def main():
         avg_ms = prof[dom][0] / prof[dom][1]
         achieved = kernel_bytes_per_launch(dom, w, B) / (avg_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                    "frac": achieved / peak, "traffic": None, "peak_source": peak_src + " copy bandwidth",
+                    "frac": achieved / peak,
+                    "traffic": (NCU_TRAFFIC_PER_SAMPLE[(dom, w.n_vis, w.d, w.n_pivot)] * B
+                                if (dom, w.n_vis, w.d, w.n_pivot) in NCU_TRAFFIC_PER_SAMPLE and args.path == 0 else None),
+                    "peak_source": peak_src + " copy bandwidth",
                     "avg_launch_ms": avg_ms,
                     "shares": {k: v[0] / max(sum(x[0] for x in prof.values()), 1e-9) for k, v in prof.items()}}
     path_gbs = path_bytes_per_sample(w) * B / (ms_per_step * 1e-3) / 1e9

@@ -262,6 +262,14 @@ struct Ctl {
             }
         }
     }
+    // After a failure: waits for work that is already in flight (a copy into shared memory, an MMA), whatever the
+    // abort flag says: a CTA must not exit, nor free TMEM, while such work is pending.  Bounded by the time limit only.
+    __device__ void wait_landed(uint32_t bar, uint32_t parity) const
+    {
+        const long long t0 = clock64();
+        while (!mbar_try_wait(bar, parity))
+            if ((unsigned long long)(clock64() - t0) > limit_cycles) return;
+    }
     // waits until *flag >= target
     __device__ bool wait_flag(const int *flag, int where, long long task, int target = 1) const
     {
@@ -528,7 +536,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             }
             if (!ok || ctl.aborted()) // drain: let the copies already issued land before the CTA may exit
                 for (long long i = issued > p.n1 ? issued - p.n1 : 0; i < issued; ++i)
-                    ctl.wait_bar(smem_u32(&sh.full1[i % p.n1]), (uint32_t)((i / p.n1) & 1), kWaitDrain, i);
+                    ctl.wait_landed(smem_u32(&sh.full1[i % p.n1]), (uint32_t)((i / p.n1) & 1));
         }
     } else if (warp == kProducer2Warp) {
         // ------------------------------------------------------------------ sweep-2 producer
@@ -597,7 +605,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
         }
         if ((!ok || ctl.aborted()) && lane == 0) // drain, as above
             for (long long i = issued > p.n2 ? issued - p.n2 : 0; i < issued; ++i)
-                ctl.wait_bar(smem_u32(&sh.full2[i % p.n2]), (uint32_t)((i / p.n2) & 1), kWaitDrain, i);
+                ctl.wait_landed(smem_u32(&sh.full2[i % p.n2]), (uint32_t)((i / p.n2) & 1));
     } else if (warp == 1) {
         // ------------------------------------------------------------------ sweep-2 MMA issuer
         if (lane == 0) {
@@ -632,7 +640,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             }
             if (!ok || ctl.aborted()) { // TMEM is freed at the end: first let the MMAs issued so far finish
                 umma_commit(smem_u32(&sh.mma_drain));
-                ctl.wait_bar(smem_u32(&sh.mma_drain), 0, kWaitDrain, -1);
+                ctl.wait_landed(smem_u32(&sh.mma_drain), 0);
             }
         }
     } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
