@@ -42,6 +42,7 @@ def parse():
     ap.add_argument("--sweep", action="store_true", help="also time every (pivots, keep) cell of the sweep")
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 staged, 2 fused")
     ap.add_argument("--lag", type=int, default=0, help="fused path: extra tasks between a row's two sweeps")
+    ap.add_argument("--retention", type=int, default=0, help="0 auto, 1 one kernel, 2 candidate lists + walks")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -215,9 +216,20 @@ def job_tokens_per_s(world, B, n_vis, steps, ms):
     return world * B * n_vis * steps / (ms * 1e-3)
 
 
+L2_FLUSH_BYTES = 256 << 20      # written between timed steps when the inputs could stay in the 126 MB L2
+L2_SAFE_INPUT_BYTES = 512 << 20  # inputs at least this large cannot be served from L2
+
+
+def needs_flush(w, B):
+    """True when the keys of one step could (partly) survive in L2 from one step to the next."""
+    return 2 * B * w.S * w.d < L2_SAFE_INPUT_BYTES
+
+
 def workload_config(w, B):
     return {"workload": w.name, "batch": B, "n_vis": w.n_vis, "seq_len": w.S, "d": w.d, "n_pivot": w.n_pivot,
-            "n_keep": w.n_keep, "vis_offset": w.vis_offset, "l2": "inputs larger than L2 (no flush needed)"}
+            "n_keep": w.n_keep, "vis_offset": w.vis_offset,
+            "l2": ("flushed between steps (%d MiB write), steps timed one by one" % (L2_FLUSH_BYTES >> 20)
+                   if needs_flush(w, B) else "inputs larger than L2 (no flush needed)")}
 
 
 def time_steps(ctx, dart, torch, w, keys, hidden, outs, steps, warmup, opts, dist_on):
@@ -243,15 +255,28 @@ def time_steps(ctx, dart, torch, w, keys, hidden, outs, steps, warmup, opts, dis
     if dist_on:
         dist.barrier()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(st)
-    for _ in range(steps):
-        step()
-    e1.record(st)
-    torch.cuda.synchronize()
+    if needs_flush(w, keys.shape[0]):
+        # small inputs: write a buffer larger than L2 before every step and time the steps one by one
+        junk = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=keys.device)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for e0, e1 in evs:
+            junk.fill_(1)
+            e0.record(st)
+            step()
+            e1.record(st)
+        torch.cuda.synchronize()
+        ms = sum(e0.elapsed_time(e1) for e0, e1 in evs)
+        del junk
+    else:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        for _ in range(steps):
+            step()
+        e1.record(st)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
     if dist_on:
         dist.barrier()
-    ms = e0.elapsed_time(e1)
     launches = dart.dart_launch_count(ctx.handle) - n0
     dart.dart_profile_enable(ctx.handle, False)
     _, prof = dart.dart_profile_read(ctx.handle)
@@ -286,7 +311,7 @@ def main():
     ctx = dart.Dart(B, w.S, w.d, max(w.n_pivot, max(W.SWEEP_PIVOTS) if args.sweep else 0),
                     max(w.n_keep, max(W.SWEEP_KEEP) if args.sweep else 0), device=local, flags=flags)
     dart.dart_set_shape(ctx.handle, B, w.S)
-    opts = dart.dart_opts(0, 0, args.path, 0, args.lag)
+    opts = dart.dart_opts(0, 0, args.path, 0, args.lag, 0, args.retention)
 
     def alloc_outs(wl):
         return (torch.empty((B, wl.S_out, wl.d), dtype=torch.bfloat16, device=dev),

@@ -55,6 +55,12 @@ enum {
 #define DART_PATH_FUSED 2  /* persistent sweep kernel (scores, pivots and similarities in one launch); needs
                               d % 64 == 0 and n_pivot <= 256, else UNSUPPORTED.  AUTO picks it when it applies. */
 
+/* dart_opts.retention */
+#define DART_RETAIN_AUTO 0   /* two phases when the batch alone cannot fill the GPU, else one kernel */
+#define DART_RETAIN_SERIAL 1 /* one kernel, one CTA per sample: the pivots' selections one after the other */
+#define DART_RETAIN_LISTS 2  /* two phases: sorted candidate lists for all (sample, pivot) pairs at once, then the pivots'
+                                turns as walks over the lists; needs n_keep - n_pivot <= 4096, else the one-kernel form runs */
+
 typedef struct dart_ctx dart_ctx; /* opaque: workspace, device status word, profiling events */
 
 /* Maxima a context is sized for.  d is fixed per context (a multiple of 8). */
@@ -77,6 +83,7 @@ typedef struct {
     int32_t sweep_lag;     /* 0: default; > 0: fused path, extra tasks between a row's two sweeps (tuning) */
     int32_t test_withhold_pivots; /* testing only: nonzero makes the fused kernel never publish a sample's pivots, so that
                                      its bounded waits expire and the call ends with DART_ERR_TIMEOUT in dart_status */
+    int32_t retention;     /* DART_RETAIN_*: how step 4 is scheduled (same result either way) */
 } dart_opts;
 
 /* Optional per-step outputs of dart_reduce_ex; every member is a device pointer or NULL. */

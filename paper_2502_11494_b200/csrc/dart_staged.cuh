@@ -178,7 +178,8 @@ sim_alu_kernel(const uint4 *__restrict__ keys, int S, int d8, int vis_offset, in
 }
 
 // ------------------------------------------------------------------------------------------------
-// Steps 4 and 5a: retention (Eq. 9-10) and the packed index list.  One CTA per sample.
+// Steps 4 and 5a in one kernel: retention (Eq. 9-10) and the packed index list.  One CTA per sample.
+// (Used when the two-phase form below does not apply: more than 4096 tokens to keep beside the pivots.)
 // kept := pivots; pivot i in rank order selects its q_i not-yet-kept tokens of lowest dup (radix
 // select on order-preserving keys, ties to the lower index); eps_i is the selection threshold.
 // Then an ordered scan over the keep flags writes the ascending kept indices and position ids.
@@ -282,6 +283,204 @@ retain_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_i
         if (f) {
             uint32_t t = vis_offset + base + before + __popc(bal & ((1u << lane) - 1u));
             int s = vis_offset + j;
+            oi[t] = s;
+            op[t] = pin ? pin[s] : (int64_t)s;
+        }
+        base += total;
+        __syncthreads();
+    }
+    if (keep_out)
+        for (int j = threadIdx.x; j < n_vis; j += blockDim.x) keep_out[(size_t)b * n_vis + j] = keep[j];
+}
+
+// ------------------------------------------------------------------------------------------------
+// Steps 4 and 5a in two phases (the default; retain_kernel above is the plain one-kernel form).
+//
+// Pivot i keeps its q_i not-yet-kept tokens of lowest dup (Eq. 9-10, rank order).  Before its turn at
+// most Q_{i-1} = q_0 + ... + q_{i-1} non-pivot tokens have been kept, so its picks are among the
+// M_i = Q_{i-1} + q_i = Q_i smallest (dup, index) pairs of its row.  Phase 1 therefore works on all
+// (sample, pivot) pairs at once: one CTA selects those M_i candidates (radix select over keys cached in
+// shared memory, pivots excluded), sorts them by (dup, index) and stores their indices.  Phase 2, one CTA
+// per sample, takes the pivots' turns in rank order: a warp walks pivot i's sorted list 32 entries at a
+// time and keeps the first q_i that are still free; eps_i is the dup of the last one kept.  Then the
+// ordered scan writes the packed index list as above.  The result equals retain_kernel's exactly.
+//
+// Dynamic shared memory, phase 1: n_vis * 4 (keys) and n_vis (pivot flags), each rounded to 16, + M_pad * 8 (sort
+// buffer, M_pad = next power of two >= n_keep - P).  Phase 2: n_vis rounded to 16 (keep flags) +
+// kWalkStageEntries * 4 (staged candidate lists).
+// ------------------------------------------------------------------------------------------------
+constexpr int kCandThreads = 256;
+constexpr int kCandMax = 4096;           // candidates per pivot the sort buffer takes (n_keep - P <= 4096)
+constexpr int kWalkThreads = 256;
+constexpr int kWalkStageEntries = 12288; // 48 KB of staged candidate indices per round of phase 2
+
+__host__ __device__ inline int quota_prefix(int i, int q, int r) { return (i + 1) * q + (i + 1 < r ? i + 1 : r); } // Q_i
+
+inline size_t candidates_smem_bytes(int n_vis, int m_pad)
+{
+    return ((size_t)n_vis * 4 + 15) / 16 * 16 + ((size_t)n_vis + 15) / 16 * 16 + (size_t)m_pad * 8;
+}
+inline size_t walk_smem_bytes(int n_vis) { return ((size_t)n_vis + 15) / 16 * 16 + (size_t)kWalkStageEntries * 4; }
+
+__global__ void __launch_bounds__(kCandThreads)
+candidates_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx, int n_vis, int P, int n_keep,
+                  int m_pad, int cand_stride, int32_t *__restrict__ cand, const int *__restrict__ status)
+{
+    extern __shared__ __align__(16) uint8_t cand_smem[];
+    uint32_t *keys = reinterpret_cast<uint32_t *>(cand_smem);                      // [n_vis] order-preserving keys of the row
+    uint8_t *is_pivot = cand_smem + ((size_t)n_vis * 4 + 15) / 16 * 16;            // [n_vis]
+    unsigned long long *list = reinterpret_cast<unsigned long long *>(is_pivot + ((size_t)n_vis + 15) / 16 * 16); // [m_pad]
+    __shared__ SelectSmem sel;
+    __shared__ uint32_t n_picked;
+    if (*status != 0) return; // an earlier kernel of this call failed: its outputs are undefined
+    const int i = blockIdx.x, b = blockIdx.y;
+    const int q = (n_keep - P) / P, r = (n_keep - P) % P;
+    const int qi = q + (i < r ? 1 : 0);
+    if (qi == 0) return; // this pivot keeps nothing (and so do all later ones)
+    const int M = quota_prefix(i, q, r);
+    const float *row = sim + ((size_t)b * P + i) * n_vis;
+    for (int j = threadIdx.x; j < n_vis; j += blockDim.x) {
+        keys[j] = order_key(row[j]);
+        is_pivot[j] = 0;
+    }
+    int mp = 1; // this pivot's own sort size
+    while (mp < M) mp <<= 1;
+    for (int t = threadIdx.x; t < mp; t += blockDim.x) list[t] = ~0ull;
+    if (threadIdx.x == 0) n_picked = 0;
+    __syncthreads();
+    for (int t = threadIdx.x; t < P; t += blockDim.x) is_pivot[pivot_idx[(size_t)b * P + t]] = 1;
+    __syncthreads();
+    auto keyfn = [&](int j, uint32_t &key) {
+        if (is_pivot[j]) return false;
+        key = keys[j];
+        return true;
+    };
+    uint32_t T, need_eq, cnt_eq;
+    block_select_threshold(CtaGroup(), keyfn, n_vis, (uint32_t)M, sel, T, need_eq, cnt_eq);
+    block_select_apply(CtaGroup(), keyfn, n_vis, T, need_eq, cnt_eq, sel, [&](int j, uint32_t key) {
+        const uint32_t slot = atomicAdd(&n_picked, 1u);
+        if (slot < (uint32_t)mp) list[slot] = ((unsigned long long)key << 32) | (uint32_t)j;
+    });
+    // ascending bitonic sort of (key, index): lowest dup first, equal dups by index
+    for (int k = 2; k <= mp; k <<= 1) {
+        for (int jj = k >> 1; jj > 0; jj >>= 1) {
+            for (int t = threadIdx.x; t < mp; t += blockDim.x) {
+                const int l = t ^ jj;
+                if (l > t) {
+                    const unsigned long long x = list[t], y = list[l];
+                    const bool up = ((t & k) == 0);
+                    if ((x > y) == up) {
+                        list[t] = y;
+                        list[l] = x;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    int32_t *out = cand + ((size_t)b * P + i) * cand_stride;
+    for (int t = threadIdx.x; t < M; t += blockDim.x) out[t] = (int32_t)(list[t] & 0xffffffffu);
+}
+
+__global__ void __launch_bounds__(kWalkThreads)
+retain_walk_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx, const int32_t *__restrict__ cand,
+                   int cand_stride, const int64_t *__restrict__ pos_in, int S, int vis_offset, int n_vis, int P, int n_keep,
+                   int32_t *__restrict__ out_idx, int64_t *__restrict__ out_pos, uint8_t *__restrict__ keep_out,
+                   int32_t *__restrict__ owner_out, float *__restrict__ eps_out, const int *__restrict__ status)
+{
+    extern __shared__ __align__(16) uint8_t keep[]; // [n_vis] flags, then the staged candidate lists
+    int32_t *stage = reinterpret_cast<int32_t *>(keep + ((size_t)n_vis + 15) / 16 * 16); // [kWalkStageEntries]
+    __shared__ uint32_t warp_tot[kWalkThreads / 32];
+    if (*status != 0) return;
+    const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int S_out = S - n_vis + n_keep;
+    const int q = (n_keep - P) / P, r = (n_keep - P) % P;
+    int32_t *owner = owner_out ? owner_out + (size_t)b * n_vis : nullptr;
+    for (int j = threadIdx.x; j < n_vis; j += blockDim.x) {
+        keep[j] = 0;
+        if (owner) owner[j] = -1;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < P; i += blockDim.x) {
+        const int pv = pivot_idx[(size_t)b * P + i];
+        keep[pv] = 1;
+        if (owner) owner[pv] = P + i;
+        if (eps_out && q + (i < r ? 1 : 0) == 0) eps_out[(size_t)b * P + i] = __int_as_float(0x7fc00000);
+    }
+    __syncthreads();
+    // rounds: stage the lists of as many pivots as fit, then warp 0 takes their turns in rank order
+    const int n_active = q > 0 ? P : r; // pivots with a quota (all later ones keep nothing)
+    for (int i0 = 0; i0 < n_active;) {
+        int i1 = i0, total = 0;
+        while (i1 < n_active && (i1 == i0 || total + quota_prefix(i1, q, r) <= kWalkStageEntries)) {
+            total += quota_prefix(i1, q, r);
+            ++i1;
+        }
+        // list of pivot i starts at the sum of the lengths before it (recomputed by every thread: a few adds)
+        for (int i = i0, off = 0; i < i1; ++i) {
+            const int M = quota_prefix(i, q, r);
+            const int32_t *src = cand + ((size_t)b * P + i) * cand_stride;
+            for (int t = threadIdx.x; t < M; t += blockDim.x) stage[off + t] = src[t];
+            off += M;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            for (int i = i0, off = 0; i < i1; ++i) {
+                const int M = quota_prefix(i, q, r);
+                int remaining = q + (i < r ? 1 : 0), last = -1;
+                for (int t = 0; t < M && remaining > 0; t += 32) {
+                    const bool valid = t + lane < M;
+                    const int j = valid ? stage[off + t + lane] : 0;
+                    const bool free = valid && !keep[j];
+                    const uint32_t bal = __ballot_sync(0xffffffffu, free);
+                    const bool take = free && (int)__popc(bal & ((1u << lane) - 1u)) < remaining;
+                    const uint32_t took = __ballot_sync(0xffffffffu, take);
+                    if (take) {
+                        keep[j] = 1;
+                        if (owner) owner[j] = i;
+                    }
+                    if (took) last = __shfl_sync(0xffffffffu, j, 31 - __clz(took)); // the list is sorted: the highest lane is the largest dup
+                    remaining -= __popc(took);
+                    __syncwarp(); // the flags are visible to the next chunk and the next pivot
+                }
+                if (eps_out && lane == 0 && last >= 0) eps_out[(size_t)b * P + i] = sim[((size_t)b * P + i) * n_vis + last];
+                off += M;
+            }
+        }
+        __syncthreads();
+        i0 = i1;
+    }
+    // packed index list: text before, kept vision tokens in ascending order, text after
+    int32_t *oi = out_idx + (size_t)b * S_out;
+    int64_t *op = out_pos + (size_t)b * S_out;
+    const int64_t *pin = pos_in ? pos_in + (size_t)b * S : nullptr;
+    for (int t = threadIdx.x; t < vis_offset; t += blockDim.x) {
+        oi[t] = t;
+        op[t] = pin ? pin[t] : (int64_t)t;
+    }
+    const int n_after = S - vis_offset - n_vis;
+    for (int t = threadIdx.x; t < n_after; t += blockDim.x) {
+        const int s = vis_offset + n_vis + t;
+        oi[vis_offset + n_keep + t] = s;
+        op[vis_offset + n_keep + t] = pin ? pin[s] : (int64_t)s;
+    }
+    const int nwarp = blockDim.x >> 5;
+    uint32_t base = 0;
+    for (int start = 0; start < n_vis; start += blockDim.x) {
+        const int j = start + threadIdx.x;
+        const bool f = (j < n_vis) && keep[j];
+        const uint32_t bal = __ballot_sync(0xffffffffu, f);
+        if (lane == 0) warp_tot[warp] = __popc(bal);
+        __syncthreads();
+        uint32_t before = 0, total = 0;
+        for (int w = 0; w < nwarp; ++w) {
+            const uint32_t t = warp_tot[w];
+            if (w < warp) before += t;
+            total += t;
+        }
+        if (f) {
+            const uint32_t t = vis_offset + base + before + __popc(bal & ((1u << lane) - 1u));
+            const int s = vis_offset + j;
             oi[t] = s;
             op[t] = pin ? pin[s] : (int64_t)s;
         }

@@ -19,6 +19,7 @@ DART_ERR_NULL, DART_ERR_BAD_SHAPE, DART_ERR_ALIGN, DART_ERR_ALIAS = -1, -2, -3, 
 DART_ERR_CUDA, DART_ERR_NOMEM, DART_ERR_TIMEOUT, DART_ERR_CHECK, DART_ERR_UNSUPPORTED = -5, -6, -7, -8, -9
 DART_FLAG_HOST_STAGING = 1
 DART_PATH_AUTO, DART_PATH_STAGED, DART_PATH_FUSED = 0, 1, 2
+DART_RETAIN_AUTO, DART_RETAIN_SERIAL, DART_RETAIN_LISTS = 0, 1, 2
 
 EXPORTS = (
     "dart_create", "dart_destroy", "dart_set_shape", "dart_reduce", "dart_reduce_ex", "dart_reduce_host",
@@ -37,7 +38,7 @@ class dart_desc(ctypes.Structure):
 class dart_opts(ctypes.Structure):
     _fields_ = [("norm_kind", ctypes.c_int32), ("pivot_smallest", ctypes.c_int32), ("path", ctypes.c_int32),
                 ("wait_limit", ctypes.c_int32), ("sweep_lag", ctypes.c_int32),
-                ("test_withhold_pivots", ctypes.c_int32)]
+                ("test_withhold_pivots", ctypes.c_int32), ("retention", ctypes.c_int32)]
 
 
 class dart_debug(ctypes.Structure):

@@ -21,13 +21,13 @@ def _np(t):
 
 
 def run_gpu(keys, hidden, vo, nv, P, Kp, pos_in=None, path=dart.DART_PATH_AUTO, norm_kind=0, smallest=0, debug=True,
-            sweep_lag=0):
+            sweep_lag=0, retention=dart.DART_RETAIN_AUTO):
     B, S, d = hidden.shape
     if path == dart.DART_PATH_FUSED and (d % 64 or P > 256):
         pytest.skip("the fused path needs d % 64 == 0 and at most 256 pivots")
     ctx = dart.Dart(B, S, d, P, Kp)
     try:
-        opts = dart.dart_opts(norm_kind, smallest, path, 0, sweep_lag)
+        opts = dart.dart_opts(norm_kind, smallest, path, 0, sweep_lag, 0, retention)
         res = ctx.reduce(hidden, keys, vo, nv, P, Kp, pos_in=pos_in, opts=opts, debug=debug)
         torch.cuda.synchronize()
         st = ctx.status()
@@ -83,6 +83,32 @@ def test_shapes_against_oracle(oracle, shape, path):
     rep = compare(oracle, k, h, vo, nv, P, Kp, path=path)
     assert rep.exact >= rep.above_margin
     assert rep.max_rel_l1 < 5e-5 and rep.max_rel_l2 < 5e-5 and rep.max_abs_sim < 2e-5   # fp32-accumulation level
+
+
+RETENTION_SHAPES = SHAPES + [
+    (3, 700, 64, 10, 640, 128, 640),    # every pivot keeps four: 128 short lists per sample
+    (2, 5000, 64, 0, 5000, 2, 4098),    # 4096 kept beside the pivots: the longest candidate lists
+    (2, 5000, 64, 0, 5000, 2, 4500),    # more than that: the two-phase form does not apply and the one-kernel form runs
+    (150, 80, 64, 5, 70, 4, 30),        # more samples than SMs
+]
+
+
+@pytest.mark.parametrize("shape", RETENTION_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_both_forms_of_the_retention_agree(oracle, shape):
+    """One kernel per sample (the pivots' selections one after the other) and candidate lists + walks make the
+    same selections: every output is bitwise equal, and one of them is checked against the oracle."""
+    B, S, d, vo, nv, P, Kp = shape
+    k, h = gaussian(B, S, d, seed=3 + sum(shape))
+    a = run_gpu(k, h, vo, nv, P, Kp, path=dart.DART_PATH_STAGED, retention=dart.DART_RETAIN_SERIAL)
+    b = run_gpu(k, h, vo, nv, P, Kp, path=dart.DART_PATH_STAGED, retention=dart.DART_RETAIN_LISTS)
+    assert all(np.array_equal(x, y) for x, y in zip(a[:3], b[:3]))
+    assert all(np.array_equal(a[3][n], b[3][n], equal_nan=(n == "eps")) for n in a[3])
+    sel = list(range(min(B, 3)))
+    kb, hb = W.bits(k[sel]), W.bits(h[sel])
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp)
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, b[0][sel], b[1][sel], b[2][sel],
+                             dbg={n: v[sel] for n, v in b[3].items()})
+    assert rep.exact >= rep.above_margin
 
 
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
