@@ -2,5 +2,5 @@
 
 Nothing in the product package may import this; see ``dart_oracle.c`` for the arithmetic.
 """
-from .dart_oracle import (OracleResult, build, compact, pivots, reduce, retention, scores,  # noqa: F401
-                          similarity)
+from .dart_oracle import (OracleResult, build, compact, gather_rows, pivots, reduce, retention,  # noqa: F401
+                          retention_global, scores, similarity)

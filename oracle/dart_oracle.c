@@ -226,6 +226,87 @@ int dart_oracle_retention(const double *dup, const int32_t *pivot_idx, int n_vis
 }
 
 /*
+ * Retention with ONE threshold for all pivots (a second reading of Def. 2 / Eq. 8-9): a token is an
+ * eps-duplicate of the pivot set if its dup to SOME pivot exceeds eps, so a token's duplication is its
+ * highest dup over the pivots, u_j = max_i dup(p_i, x_j); the n_keep - P non-pivot tokens of lowest u_j are
+ * retained (equal values: lower index first), eps = the largest retained u_j, R = P u {x_j : u_j <= eps}.
+ *   owner  [n_vis] -1 dropped, i = retained and most similar to pivot i (lowest i on equal dup), P + i = pivot
+ *   eps    [P]     the one threshold, repeated; NaN when n_keep = P
+ *   gap    scalar  (u of the best token NOT taken) - eps, +inf if none is left behind
+ */
+int dart_oracle_retention_global(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep,
+                                 uint8_t *keep, int32_t *owner, double *eps, double *gap_out)
+{
+    if (P < 1 || P > n_keep || n_keep > n_vis) return ORACLE_ERR_SHAPE;
+    keyed_t *cand = (keyed_t *)malloc((size_t)n_vis * sizeof *cand);
+    int32_t *nearest = (int32_t *)malloc((size_t)n_vis * sizeof *nearest);
+    if (!cand || !nearest) {
+        free(cand);
+        free(nearest);
+        return ORACLE_ERR_NOMEM;
+    }
+    memset(keep, 0, (size_t)n_vis);
+    if (owner)
+        for (int j = 0; j < n_vis; ++j) owner[j] = OWNER_DROPPED;
+    for (int i = 0; i < P; ++i) {
+        int p = pivot_idx[i];
+        if (p < 0 || p >= n_vis || keep[p]) {
+            free(cand);
+            free(nearest);
+            return ORACLE_ERR_SHAPE; /* pivots must be distinct vision tokens */
+        }
+        keep[p] = 1;
+        if (owner) owner[p] = P + i;
+    }
+    int m = 0;
+    for (int j = 0; j < n_vis; ++j) {
+        if (keep[j]) continue;
+        double u = dup[j];
+        int arg = 0;
+        for (int i = 1; i < P; ++i)
+            if (dup[(size_t)i * (size_t)n_vis + j] > u) {
+                u = dup[(size_t)i * (size_t)n_vis + j];
+                arg = i;
+            }
+        cand[m].v = u;
+        cand[m].idx = j;
+        nearest[j] = arg;
+        ++m;
+    }
+    const int take = n_keep - P;
+    qsort(cand, (size_t)m, sizeof *cand, cmp_asc);
+    for (int t = 0; t < take; ++t) {
+        keep[cand[t].idx] = 1;
+        if (owner) owner[cand[t].idx] = nearest[cand[t].idx];
+    }
+    if (eps)
+        for (int i = 0; i < P; ++i) eps[i] = take > 0 ? cand[take - 1].v : NAN;
+    if (gap_out) *gap_out = (take > 0 && m > take) ? cand[take].v - cand[take - 1].v : INFINITY;
+    free(cand);
+    free(nearest);
+    return ORACLE_OK;
+}
+
+/*
+ * Row gather by a packed index list: out[b, t, :] = src[b, idx[b, t], :] (bit copies of rows of `row_elems`
+ * 16-bit words).  This is how a cache kept per token (the key and value rows of the layers already run) follows
+ * the shortened sequence: the paper counts the KV cache of the retained tokens only (Table 2).
+ */
+int dart_oracle_gather_rows(const uint16_t *src, const int32_t *idx, int B, int S, int S_out, int row_elems,
+                            uint16_t *out)
+{
+    if (B < 0 || S < 1 || S_out < 0 || row_elems < 1) return ORACLE_ERR_SHAPE;
+    for (int b = 0; b < B; ++b)
+        for (int t = 0; t < S_out; ++t) {
+            const int32_t s = idx[(size_t)b * S_out + t];
+            if (s < 0 || s >= S) return ORACLE_ERR_SHAPE;
+            memcpy(out + ((size_t)b * S_out + t) * (size_t)row_elems, src + ((size_t)b * S + s) * (size_t)row_elems,
+                   (size_t)row_elems * sizeof(uint16_t));
+        }
+    return ORACLE_OK;
+}
+
+/*
  * Sequence shortening (Table 1 caption: tokens are pruned after layer K; the remaining
  * layers see a dense, shorter sequence).  Kept rows stay in original order:
  *   out_idx    = [0, vis_offset) ++ sorted{vis_offset + j : keep[j]} ++ [vis_offset + n_vis, S)
@@ -262,18 +343,24 @@ int dart_oracle_compact(const uint8_t *keep, const uint16_t *hidden, const int64
  *   owner [B, n_vis]; eps [B, P]; pivot_gap [B]; retain_gap [B].
  * Packed outputs: out_hidden [B, S_out, d], out_idx [B, S_out], out_pos [B, S_out],
  * S_out = S - n_vis + n_keep.
+ * pivots_in: NULL, or [B, P] distinct vision-relative indices that replace the pivot step (their
+ * order is the order of the pivots' turns); the retention step rejects repeated or out-of-range ones.
+ * rule: 0 = one threshold per pivot from equal quotas (dart_oracle_retention), 1 = one threshold for all
+ * (dart_oracle_retention_global).
  */
-int dart_oracle_reduce(const uint16_t *hidden, const uint16_t *keys, const int64_t *pos_in,
-                       int B, int S, int d, int vis_offset, int n_vis, int n_pivot, int n_keep,
-                       int norm_kind, int largest,
-                       uint16_t *out_hidden, int32_t *out_idx, int64_t *out_pos,
-                       double *l1_out, double *l2_out, int32_t *pivot_out, double *dup_out,
-                       uint8_t *keep_out, int32_t *owner_out, double *eps_out,
-                       double *pivot_gap_out, double *retain_gap_out)
+int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const int64_t *pos_in,
+                          const int32_t *pivots_in,
+                          int B, int S, int d, int vis_offset, int n_vis, int n_pivot, int n_keep,
+                          int norm_kind, int largest, int rule,
+                          uint16_t *out_hidden, int32_t *out_idx, int64_t *out_pos,
+                          double *l1_out, double *l2_out, int32_t *pivot_out, double *dup_out,
+                          uint8_t *keep_out, int32_t *owner_out, double *eps_out,
+                          double *pivot_gap_out, double *retain_gap_out)
 {
     if (B < 0 || S < 1 || d < 1 || vis_offset < 0 || n_vis < 1 || vis_offset + n_vis > S) return ORACLE_ERR_SHAPE;
     if (n_pivot < 1 || n_pivot > n_keep || n_keep > n_vis) return ORACLE_ERR_SHAPE;
     if (norm_kind != 1 && norm_kind != 2) return ORACLE_ERR_SHAPE;
+    if (rule != 0 && rule != 1) return ORACLE_ERR_SHAPE;
     const int P = n_pivot, S_out = S - n_vis + n_keep;
     double *l1 = (double *)malloc((size_t)n_vis * sizeof(double));
     double *l2 = (double *)malloc((size_t)n_vis * sizeof(double));
@@ -290,13 +377,18 @@ int dart_oracle_reduce(const uint16_t *hidden, const uint16_t *keys, const int64
         int so = 0;
         rc = dart_oracle_scores(k, S, d, vis_offset, n_vis, l1, l2);
         if (rc) break;
-        rc = dart_oracle_pivots(norm_kind == 1 ? l1 : l2, n_vis, P, largest, piv, &pgap);
-        if (rc) break;
+        if (pivots_in) { /* the caller names the pivots and their order (Sec. 5.2 compares several ways to choose them) */
+            memcpy(piv, pivots_in + (size_t)b * P, (size_t)P * sizeof(int32_t));
+            pgap = INFINITY; /* nothing is ranked, so no ranking can be close */
+        } else {
+            rc = dart_oracle_pivots(norm_kind == 1 ? l1 : l2, n_vis, P, largest, piv, &pgap);
+            if (rc) break;
+        }
         rc = dart_oracle_similarity(k, S, d, vis_offset, n_vis, piv, P, l2, dup);
         if (rc) break;
-        rc = dart_oracle_retention(dup, piv, n_vis, P, n_keep, keep,
-                                   owner_out ? owner_out + (size_t)b * n_vis : NULL,
-                                   eps_out ? eps_out + (size_t)b * P : NULL, &rgap);
+        rc = (rule == 1 ? dart_oracle_retention_global : dart_oracle_retention)(
+            dup, piv, n_vis, P, n_keep, keep, owner_out ? owner_out + (size_t)b * n_vis : NULL,
+            eps_out ? eps_out + (size_t)b * P : NULL, &rgap);
         if (rc) break;
         rc = dart_oracle_compact(keep, h, pos, S, d, vis_offset, n_vis,
                                  out_hidden ? out_hidden + (size_t)b * (size_t)S_out * (size_t)d : NULL,
@@ -320,4 +412,18 @@ int dart_oracle_reduce(const uint16_t *hidden, const uint16_t *keys, const int64
     free(piv);
     free(keep);
     return rc;
+}
+
+/* The step with pivots chosen by score (the paper's main setting). */
+int dart_oracle_reduce(const uint16_t *hidden, const uint16_t *keys, const int64_t *pos_in,
+                       int B, int S, int d, int vis_offset, int n_vis, int n_pivot, int n_keep,
+                       int norm_kind, int largest,
+                       uint16_t *out_hidden, int32_t *out_idx, int64_t *out_pos,
+                       double *l1_out, double *l2_out, int32_t *pivot_out, double *dup_out,
+                       uint8_t *keep_out, int32_t *owner_out, double *eps_out,
+                       double *pivot_gap_out, double *retain_gap_out)
+{
+    return dart_oracle_reduce_ex(hidden, keys, pos_in, NULL, B, S, d, vis_offset, n_vis, n_pivot, n_keep, norm_kind,
+                                 largest, 0, out_hidden, out_idx, out_pos, l1_out, l2_out, pivot_out, dup_out, keep_out,
+                                 owner_out, eps_out, pivot_gap_out, retain_gap_out);
 }

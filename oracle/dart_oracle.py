@@ -39,7 +39,8 @@ def _load():
     if _lib is None:
         _lib = ctypes.CDLL(build())
         for name in ("dart_oracle_scores", "dart_oracle_pivots", "dart_oracle_similarity",
-                     "dart_oracle_retention", "dart_oracle_compact", "dart_oracle_reduce"):
+                     "dart_oracle_retention", "dart_oracle_retention_global", "dart_oracle_compact",
+                     "dart_oracle_gather_rows", "dart_oracle_reduce", "dart_oracle_reduce_ex"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
@@ -121,6 +122,33 @@ def retention(dup, pivot_idx, n_keep: int):
     return keep, owner, eps, gap.value
 
 
+def retention_global(dup, pivot_idx, n_keep: int):
+    """dup [P, n_vis] -> (keep, owner, eps [P], gap) with one threshold on max_i dup for all pivots."""
+    dd = np.ascontiguousarray(dup, np.float64)
+    P, n_vis = dd.shape
+    piv = np.ascontiguousarray(pivot_idx, np.int32)
+    keep = np.empty(n_vis, np.uint8)
+    owner = np.empty(n_vis, np.int32)
+    eps = np.empty(P, np.float64)
+    gap = ctypes.c_double(0.0)
+    _check(_load().dart_oracle_retention_global(_p(dd, ctypes.c_double), _p(piv, ctypes.c_int32), n_vis, P, n_keep,
+                                                _p(keep, ctypes.c_uint8), _p(owner, ctypes.c_int32),
+                                                _p(eps, ctypes.c_double), ctypes.byref(gap)), "retention_global")
+    return keep, owner, eps, gap.value
+
+
+def gather_rows(src, idx):
+    """src [B, S, w] 16-bit words (bf16 bits), idx [B, S_out] int32 -> out [B, S_out, w] (bit copies)."""
+    a = _u16(src)
+    B, S, w = a.shape
+    ii = np.ascontiguousarray(idx, np.int32)
+    S_out = ii.shape[1]
+    out = np.empty((B, S_out, w), np.uint16)
+    _check(_load().dart_oracle_gather_rows(_p(a, ctypes.c_uint16), _p(ii, ctypes.c_int32), B, S, S_out, w,
+                                           _p(out, ctypes.c_uint16)), "gather_rows")
+    return out
+
+
 def compact(keep, hidden, vis_offset: int, n_vis: int, pos_in=None):
     """keep [n_vis], hidden [S, d] bf16 bits -> (out_hidden [S_out, d] uint16, out_idx int32, out_pos int64)."""
     h = _u16(hidden)
@@ -162,8 +190,10 @@ class OracleResult:
 
 def reduce(hidden, keys, vis_offset: int, n_vis: int, n_pivot: int, n_keep: int,
            pos_in=None, norm_kind: int = 1, largest: bool = True, want_dup: bool = True,
-           want_hidden: bool = True) -> OracleResult:
-    """The whole step over a batch.  hidden/keys: [B, S, d] bf16 bits (keys None -> hidden is scored)."""
+           want_hidden: bool = True, pivots_in=None, rule: int = 0) -> OracleResult:
+    """The whole step over a batch.  hidden/keys: [B, S, d] bf16 bits (keys None -> hidden is scored).
+    pivots_in: None, or [B, n_pivot] distinct vision-relative indices that replace the pivot step.
+    rule: 0 = per-pivot thresholds from equal quotas, 1 = one threshold for all pivots."""
     h = _u16(hidden)
     B, S, d = h.shape
     k = None if keys is None else _u16(keys)
@@ -183,9 +213,12 @@ def reduce(hidden, keys, vis_offset: int, n_vis: int, n_pivot: int, n_keep: int,
     eps = np.empty((B, n_pivot), np.float64)
     pg = np.empty(B, np.float64)
     rg = np.empty(B, np.float64)
-    _check(_load().dart_oracle_reduce(
-        _p(h, ctypes.c_uint16), _p(k, ctypes.c_uint16), _p(pos, ctypes.c_int64),
-        B, S, d, vis_offset, n_vis, n_pivot, n_keep, norm_kind, int(bool(largest)),
+    piv_in = None if pivots_in is None else np.ascontiguousarray(pivots_in, np.int32)
+    if piv_in is not None and piv_in.shape != (B, n_pivot):
+        raise ValueError("pivots_in must be [B, n_pivot]")
+    _check(_load().dart_oracle_reduce_ex(
+        _p(h, ctypes.c_uint16), _p(k, ctypes.c_uint16), _p(pos, ctypes.c_int64), _p(piv_in, ctypes.c_int32),
+        B, S, d, vis_offset, n_vis, n_pivot, n_keep, norm_kind, int(bool(largest)), int(rule),
         _p(oh, ctypes.c_uint16), _p(oi, ctypes.c_int32), _p(op, ctypes.c_int64),
         _p(l1, ctypes.c_double), _p(l2, ctypes.c_double), _p(piv, ctypes.c_int32), _p(dup, ctypes.c_double),
         _p(keep, ctypes.c_uint8), _p(owner, ctypes.c_int32), _p(eps, ctypes.c_double),

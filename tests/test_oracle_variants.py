@@ -1,0 +1,147 @@
+"""Pins of the oracle's variants (caller-chosen pivots, one threshold for all pivots, row gather by the packed
+index list) against things other than themselves: brute force on tiny inputs, numpy routines, invariants and
+the special cases in which a variant must coincide with the main method.  CPU only."""
+import itertools
+import math
+
+import numpy as np
+import pytest
+
+from test_oracle_pins import bf16_bits, rand_tokens
+
+
+# ----------------------------------------------------------------------------- one threshold for all pivots
+
+def test_global_threshold_is_minimal_by_exhaustion(oracle):
+    """Among ALL subsets of the non-pivot tokens of the right size the retained one has the smallest sum of
+    u_j = max_i dup[i][j] (unique without ties): 'the tokens least duplicated by any pivot'."""
+    rng = np.random.default_rng(21)
+    for trial in range(40):
+        n = int(rng.integers(4, 12))
+        P = int(rng.integers(1, min(4, n) + 1))
+        n_keep = int(rng.integers(P, n + 1))
+        dup = rng.uniform(-1, 1, (P, n))
+        piv = rng.permutation(n)[:P].astype(np.int32)
+        keep, owner, eps, gap = oracle.retention_global(dup, piv, n_keep)
+        u = dup.max(axis=0)
+        cands = [j for j in range(n) if j not in set(piv.tolist())]
+        mine = [j for j in cands if keep[j]]
+        assert int(keep.sum()) == n_keep and np.all(keep[piv] == 1) and len(mine) == n_keep - P
+        if mine:
+            best = min(itertools.combinations(cands, len(mine)), key=lambda c: sum(u[j] for j in c))
+            assert sorted(best) == sorted(mine)
+            assert np.all(eps == max(u[j] for j in mine))
+            assert all(owner[j] == int(np.argmax(dup[:, j])) for j in mine)
+        else:
+            assert np.all(np.isnan(eps)) and gap == math.inf
+
+
+def test_global_threshold_against_numpy_and_invariants(oracle):
+    rng = np.random.default_rng(22)
+    n, P, n_keep = 400, 7, 90
+    dup = rng.uniform(-1, 1, (P, n))
+    piv = rng.permutation(n)[:P].astype(np.int32)
+    keep, owner, eps, gap = oracle.retention_global(dup, piv, n_keep)
+    u = dup.max(axis=0)
+    u[piv] = np.inf                                          # pivots are no candidates
+    order = np.argsort(u, kind="stable")                     # an independent routine: stable sort = ties to lower index
+    expect = set(order[: n_keep - P].tolist()) | set(piv.tolist())
+    assert set(np.nonzero(keep)[0].tolist()) == expect
+    dropped = np.nonzero(keep == 0)[0]
+    kept_np = np.array(sorted(expect - set(piv.tolist())))
+    assert np.all(u[kept_np] <= eps[0]) and np.all(u[dropped] >= eps[0])   # R = P u {x_j : max_i dup <= eps}
+    assert gap == pytest.approx(u[dropped].min() - eps[0]) and gap >= 0
+    assert [int(owner[p]) for p in piv] == [P + i for i in range(P)]
+    assert np.all(owner[dropped] == -1)
+
+
+def test_global_threshold_special_cases(oracle):
+    rng = np.random.default_rng(23)
+    dup = rng.uniform(-1, 1, (1, 60))
+    piv = np.array([11], np.int32)
+    a = oracle.retention_global(dup, piv, 20)                # one pivot: both rules are the same partial sort
+    b = oracle.retention(dup, piv, 20)
+    assert np.array_equal(a[0], b[0]) and a[2][0] == b[2][0] and a[3] == b[3]
+    # ties: equal u_j go to the lower index; the nearest pivot is the first of equal dups
+    dup = np.array([[9, 9, .3, .3, .1, .3],
+                    [9, 9, .3, .2, .1, .3]], float)
+    keep, owner, eps, gap = oracle.retention_global(dup, np.array([0, 1], np.int32), 4)
+    assert keep.tolist() == [1, 1, 1, 0, 1, 0] and owner.tolist() == [2, 3, 0, -1, 0, -1]
+    assert eps.tolist() == [.3, .3] and gap == 0.0
+    with pytest.raises(RuntimeError):
+        oracle.retention_global(dup, np.array([1, 1], np.int32), 4)   # repeated pivot
+    with pytest.raises(RuntimeError):
+        oracle.retention_global(dup, np.array([0, 1], np.int32), 7)   # more kept than tokens
+
+
+def test_global_rule_differs_from_quotas_where_it_should(oracle):
+    """Two pivots; token 2 is far from pivot 0 but a near copy of pivot 1.  Under per-pivot quotas pivot 0 keeps
+    it (its own lowest dup); under one threshold its duplication is 0.99 and it is dropped."""
+    dup = np.array([[9, 9, -.9, .1, .2, .3],
+                    [9, 9, .99, .5, .4, .3]], float)
+    piv = np.array([0, 1], np.int32)
+    assert oracle.retention(dup, piv, 4)[0].tolist() == [1, 1, 1, 0, 0, 1]
+    assert oracle.retention_global(dup, piv, 4)[0].tolist() == [1, 1, 0, 0, 1, 1]
+
+
+# ----------------------------------------------------------------------------- pivots chosen by the caller
+
+def test_given_pivots_replace_only_the_pivot_step(oracle):
+    rng = np.random.default_rng(24)
+    B, S, d, vo, nv, P, Kp = 3, 64, 32, 4, 50, 4, 19
+    hb, _ = rand_tokens(rng, B * S, d)
+    kb, _ = rand_tokens(rng, B * S, d)
+    hb, kb = hb.reshape(B, S, d), kb.reshape(B, S, d)
+    base = oracle.reduce(hb, kb, vo, nv, P, Kp)
+    same = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=base.pivot_idx)      # its own pivots: nothing changes
+    assert np.array_equal(same.out_idx, base.out_idx) and np.array_equal(same.owner, base.owner)
+    assert np.all(np.isinf(same.pivot_gap))                                    # nothing was ranked
+    given = np.stack([rng.permutation(nv)[:P] for _ in range(B)]).astype(np.int32)
+    r = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=given)
+    for b in range(B):                                                         # = the steps, composed by hand
+        l1, l2 = oracle.scores(kb[b], vo, nv)
+        dup = oracle.similarity(kb[b], vo, nv, given[b], l2)
+        keep, owner, eps, _ = oracle.retention(dup, given[b], Kp)
+        oh, oi, op = oracle.compact(keep, hb[b], vo, nv)
+        assert np.array_equal(r.pivot_idx[b], given[b]) and np.array_equal(r.owner[b], owner)
+        assert np.array_equal(r.out_idx[b], oi) and np.array_equal(r.out_hidden[b], oh)
+        assert np.all(r.keep[b][given[b]] == 1)                                # P subset of R whatever the pivots
+    swapped = given[:, ::-1].copy()                                            # the order given is the order of the turns
+    r2 = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=swapped)
+    assert np.array_equal(r2.pivot_idx, swapped)
+    assert not np.array_equal(r2.owner, r.owner)
+    bad = given.copy()
+    bad[1, 2] = bad[1, 0]
+    with pytest.raises(RuntimeError):
+        oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=bad)                    # repeated pivot
+    g = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=given, rule=1)          # both variants together
+    for b in range(B):
+        l1, l2 = oracle.scores(kb[b], vo, nv)
+        dup = oracle.similarity(kb[b], vo, nv, given[b], l2)
+        assert np.array_equal(g.keep[b], oracle.retention_global(dup, given[b], Kp)[0])
+
+
+# ----------------------------------------------------------------------------- rows gathered by the packed list
+
+def test_gather_rows_against_numpy(oracle):
+    rng = np.random.default_rng(25)
+    B, S, w, S_out = 3, 40, 24, 17
+    src = rng.integers(0, 1 << 16, (B, S, w)).astype(np.uint16)
+    idx = np.stack([np.sort(rng.permutation(S)[:S_out]) for _ in range(B)]).astype(np.int32)
+    out = oracle.gather_rows(src, idx)
+    assert np.array_equal(out, np.take_along_axis(src, idx[:, :, None].astype(np.int64), axis=1))
+    ident = np.tile(np.arange(S, dtype=np.int32), (B, 1))
+    assert np.array_equal(oracle.gather_rows(src, ident), src)                 # the identity list copies
+    idx[2, 5] = S
+    with pytest.raises(RuntimeError):
+        oracle.gather_rows(src, idx)                                           # index past the end
+
+
+def test_gather_rows_follows_the_reduction(oracle):
+    """The packed list of a reduction applied to the hidden states themselves gives the packed hidden states."""
+    rng = np.random.default_rng(26)
+    B, S, d, vo, nv, P, Kp = 2, 50, 16, 3, 40, 2, 9
+    hb, _ = rand_tokens(rng, B * S, d)
+    hb = hb.reshape(B, S, d)
+    r = oracle.reduce(hb, None, vo, nv, P, Kp)
+    assert np.array_equal(oracle.gather_rows(hb, r.out_idx), r.out_hidden)
