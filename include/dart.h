@@ -61,6 +61,13 @@ enum {
 #define DART_RETAIN_LISTS 2  /* two phases: sorted candidate lists for all (sample, pivot) pairs at once, then the pivots'
                                 turns as walks over the lists; needs n_keep - n_pivot <= 4096, else the one-kernel form runs */
 
+/* dart_opts.rule */
+#define DART_RULE_QUOTAS 0 /* one threshold per pivot: pivot i keeps its q_i not-yet-kept tokens of lowest dup (dart_reduce) */
+#define DART_RULE_GLOBAL 1 /* one threshold for all pivots (Def. 2 / Eq. 8-9 with a common eps): a token's duplication is
+                              its highest dup to any pivot; the n_keep - n_pivot non-pivot tokens of lowest duplication
+                              are kept, ties to the lower index.  dbg->eps holds the threshold n_pivot times, dbg->owner the
+                              pivot a kept token is most similar to (the first of equals). */
+
 typedef struct dart_ctx dart_ctx; /* opaque: workspace, device status word, profiling events */
 
 /* Maxima a context is sized for.  d is fixed per context (a multiple of 8). */
@@ -84,6 +91,12 @@ typedef struct {
     int32_t test_withhold_pivots; /* testing only: nonzero makes the fused kernel never publish a sample's pivots, so that
                                      its bounded waits expire and the call ends with DART_ERR_TIMEOUT in dart_status */
     int32_t retention;     /* DART_RETAIN_*: how step 4 is scheduled (same result either way) */
+    int32_t rule;          /* DART_RULE_*: which tokens step 4 retains */
+    const int32_t *pivots_in; /* NULL: pivots by score (steps 1-2).  Else [B, n_pivot] int32, device: the caller's pivots
+                              as vision-relative indices, distinct and in [0, n_vis); their order is the order of the
+                              pivots' turns in step 4.  This covers the paper's other ways to choose pivots (Sec. 5.2:
+                              random, attention score, value norm): the caller ranks, the library does steps 3-5.
+                              Repeated or out-of-range indices end the call with DART_ERR_CHECK in dart_status. */
 } dart_opts;
 
 /* Optional per-step outputs of dart_reduce_ex; every member is a device pointer or NULL. */
@@ -159,6 +172,20 @@ int dart_reduce_host(dart_ctx *ctx, const void *hidden, const void *keys, int vi
                      int n_pivot, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos);
 
 /*
+ * Row gather by a packed index list, without a context: out[b, t, :] = src[b, idx[b, t], :].  With idx = the
+ * out_idx of a reduction this packs any other per-token tensor the same way as out_hidden: the key and value
+ * rows of the layers already run (the paper counts the KV cache of the retained tokens only, Table 2), or the
+ * hidden states of a second stream.
+ *   src  [B, S, row_bytes] device, 16-byte aligned;  idx [B, S_out] int32 device, every entry in [0, S)
+ *   out  [B, S_out, row_bytes] device, 16-byte aligned, must not overlap src
+ *   row_bytes a multiple of 16;  device: CUDA device ordinal of the pointers;  stream: a cudaStream_t
+ * Allocates nothing and does not synchronise.  Errors: NULL, BAD_SHAPE, ALIGN, ALIAS, CUDA.  Entries of idx are
+ * not checked on the device.
+ */
+int dart_gather_rows(const void *src, const int32_t *idx, int B, int S, int S_out, int row_bytes, void *out,
+                     int device, void *stream);
+
+/*
  * Read the device status word (synchronises the context's device): DART_OK, DART_ERR_TIMEOUT if a
  * bounded wait inside a kernel gave up, DART_ERR_CHECK if a self-check failed.  Reading clears it.
  */
@@ -168,7 +195,7 @@ int dart_status(dart_ctx *ctx);
  * Where the last non-zero status came from (as read by the last dart_status call that returned an error):
  * detail[0] = which bounded wait of the fused kernel expired (1 pivots not published, 2 ring stage not freed,
  * 3 drain, 4 accumulator not freed, 5/6 tile not loaded (MMA / row sums), 7 accumulator not filled, 8/9 mailbox,
- * 10 sweep-1 tasks not all counted, 11/12 selection queue),
+ * 10 sweep-1 tasks not all counted, 11/12 selection queue; 100 = a failed check of opts->pivots_in),
  * detail[1] = index of the step in the kernel's schedule (or the sample), detail[2] = CTA; for wait 1 also
  * detail[3] = sample.  For bug reports.
  */

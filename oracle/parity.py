@@ -89,24 +89,42 @@ def check_sim(sim, ora_dup, rep: ParityReport, tol=REL_TOL, floor=SIM_ABS_FLOOR)
 
 
 def check_valid_under_tolerance(keys_bits, vis_offset, n_vis, n_keep, pivot_idx, owner, ora_score, ora_l2,
-                                largest=True, tol=MARGIN):
-    """Replay the candidate's own pivots and per-pivot assignment against fp64 quantities (one sample).
-    ora_score is the oracle's ranking score (L1 norms, or the Euclidean norms for that variant)."""
+                                largest=True, tol=MARGIN, pivots_given=False, rule=0):
+    """Replay the candidate's own pivots and assignment against fp64 quantities (one sample).
+    ora_score is the oracle's ranking score (L1 norms, or the Euclidean norms for that variant); with
+    pivots_given the caller chose the pivots and nothing about their ranking is checked; rule 1 is the
+    variant with one threshold for all pivots."""
     P = len(pivot_idx)
     assert len(set(pivot_idx.tolist())) == P, "pivots must be distinct"
     s = ora_score
     sgn = 1.0 if largest else -1.0
     others = np.setdiff1d(np.arange(n_vis), pivot_idx)
-    if len(others):
+    if len(others) and not pivots_given:
         worst_piv = (sgn * s[pivot_idx]).min()
         best_other = (sgn * s[others]).max()
         assert worst_piv >= best_other - tol * abs(best_other), "a non-pivot beats a pivot beyond tolerance"
     ranked = sgn * s[pivot_idx]
-    assert np.all(ranked[:-1] >= ranked[1:] - tol * np.abs(ranked[:-1])), "pivot rank order beyond tolerance"
+    if not pivots_given:
+        assert np.all(ranked[:-1] >= ranked[1:] - tol * np.abs(ranked[:-1])), "pivot rank order beyond tolerance"
     dup = _o.similarity(keys_bits, vis_offset, n_vis, pivot_idx, ora_l2)
     kept = np.zeros(n_vis, bool)
     kept[pivot_idx] = True
     assert [int(owner[p]) for p in pivot_idx] == [P + i for i in range(P)], "pivots carry their rank in owner"
+    if rule == 1:
+        u = dup.max(axis=0)
+        mine = np.nonzero((owner >= 0) & (owner < P))[0]
+        assert len(mine) == n_keep - P, "retained %d tokens beside the pivots, budget %d" % (len(mine), n_keep - P)
+        if len(mine):
+            assert np.all(dup[owner[mine], mine] >= u[mine] - tol), "owner is not (nearly) the most similar pivot"
+            left = np.ones(n_vis, bool)
+            left[pivot_idx] = False
+            left[mine] = False
+            if left.any():
+                assert u[left].min() >= u[mine].max() - tol, \
+                    "a token %g below the threshold was left behind" % (u[mine].max() - u[left].min())
+        kept[mine] = True
+        assert int(kept.sum()) == n_keep
+        return kept
     for i, qi in enumerate(quotas(P, n_keep)):
         mine = np.nonzero(owner == i)[0]
         assert len(mine) == qi, "pivot %d retained %d tokens, quota %d" % (i, len(mine), qi)
@@ -127,7 +145,7 @@ def check_valid_under_tolerance(keys_bits, vis_offset, n_vis, n_keep, pivot_idx,
 
 def check_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, n_vis, n_pivot, n_keep,
                 out_hidden, out_idx, out_pos, dbg=None, pos_in=None, largest=True, norm_kind=1,
-                require_exact_above=MARGIN) -> ParityReport:
+                require_exact_above=MARGIN, pivots_given=False, rule=0) -> ParityReport:
     """All rules over a batch.  ``dbg`` (optional) holds the candidate's per-step outputs as numpy arrays:
     l1, ssq, pivot_idx, sim, eps, keep, owner.  Without it only the packed outputs are checked."""
     B = out_idx.shape[0]
@@ -161,13 +179,14 @@ def check_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, n_vis,
             check_sim(dbg["sim"][b], ora.dup[b], rep)
         if margin[b] > require_exact_above:
             assert np.array_equal(dbg["owner"][b], ora.owner[b])
-            qs = quotas(n_pivot, n_keep)
+            qs = quotas(n_pivot, n_keep) if rule == 0 else [n_keep - n_pivot] * n_pivot
             has = np.array([q > 0 for q in qs])
             e = dbg["eps"][b].astype(np.float64)
             assert np.all(np.isnan(e[~has])) and np.all(np.abs(e[has] - ora.eps[b][has]) <= REL_TOL * np.abs(ora.eps[b][has]) + SIM_ABS_FLOOR)
         else:
             check_valid_under_tolerance(keys_bits[b], vis_offset, n_vis, n_keep, dbg["pivot_idx"][b], dbg["owner"][b],
-                                        ora.l1[b] if norm_kind == 1 else ora.l2[b], ora.l2[b], largest=largest)
+                                        ora.l1[b] if norm_kind == 1 else ora.l2[b], ora.l2[b], largest=largest,
+                                        pivots_given=pivots_given, rule=rule)
             if not same:
                 rep.notes.append("sample %d differs below margin %.2e (valid under tolerance)" % (b, margin[b]))
     return rep

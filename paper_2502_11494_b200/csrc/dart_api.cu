@@ -180,10 +180,17 @@ int copy_debug(dart_ctx *ctx, int B, int n_vis, int P, const dart_debug *dbg, cu
 // Steps 4 and 5a.  Two phases (candidate lists for all pivots at once, then the pivots' turns) when the lists fit
 // the workspace and shared memory, else the one-kernel form.
 void launch_retention(dart_ctx *ctx, int B, const int64_t *pos_in, int vis_offset, int n_vis, int P, int n_keep,
-                      int32_t *out_idx, int64_t *out_pos, int mode, cudaStream_t st)
+                      int32_t *out_idx, int64_t *out_pos, const dart_opts &o, cudaStream_t st)
 {
     using namespace dart;
-    const int S = ctx->S, m = n_keep - P;
+    const int S = ctx->S, m = n_keep - P, mode = o.retention;
+    if (o.rule == DART_RULE_GLOBAL) { // one threshold for all pivots: a single selection per sample
+        Prof p(ctx, st, SLOT_RETAIN);
+        retain_global_kernel<<<B, kSelectThreads, retain_global_smem_bytes(n_vis), st>>>(
+            ctx->sim, ctx->pivot_idx, pos_in, S, vis_offset, n_vis, P, n_keep, out_idx, out_pos, ctx->keep, ctx->owner, ctx->eps,
+            ctx->status);
+        return;
+    }
     const int m_pad = next_pow2(m > 1 ? m : 1);
     const bool can_lists = ctx->cand && m <= ctx->cand_stride && m <= kCandMax &&
                            candidates_smem_bytes(n_vis, m_pad) <= (size_t)ctx->max_smem_optin - 2048 &&
@@ -211,6 +218,13 @@ void launch_retention(dart_ctx *ctx, int B, const int64_t *pos_in, int vis_offse
     }
 }
 
+// Step 2 with the caller's pivots: checked and copied into the workspace.
+void launch_pivots_given(dart_ctx *ctx, int B, int n_vis, int P, const int32_t *pivots_in, cudaStream_t st)
+{
+    Prof p(ctx, st, SLOT_PIVOT);
+    dart::pivots_given_kernel<<<B, 256, (size_t)((n_vis + 31) / 32) * 4, st>>>(pivots_in, n_vis, P, ctx->pivot_idx, ctx->status);
+}
+
 int launch_staged(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, const int64_t *pos_in, int vis_offset,
                   int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos,
                   const dart_opts &o, const dart_debug *dbg, cudaStream_t st)
@@ -224,7 +238,9 @@ int launch_staged(dart_ctx *ctx, int B, const void *hidden, const void *keys_in,
         unsigned grid = (unsigned)((rows + kScoreWarps - 1) / kScoreWarps);
         score_kernel<<<grid, kScoreWarps * 32, 0, st>>>(keys, S, d8, vis_offset, n_vis, rows, ctx->l1, ctx->ssq);
     }
-    {
+    if (o.pivots_in) {
+        launch_pivots_given(ctx, B, n_vis, P, o.pivots_in, st);
+    } else {
         Prof p(ctx, st, SLOT_PIVOT);
         int P_pad = next_pow2(P);
         pivot_kernel<<<B, kSelectThreads, (size_t)P_pad * 8, st>>>(o.norm_kind == 2 ? ctx->ssq : ctx->l1, n_vis, P,
@@ -239,7 +255,7 @@ int launch_staged(dart_ctx *ctx, int B, const void *hidden, const void *keys_in,
                                                               ctx->ssq, ctx->sim);
         ctx->launches += (P - 1) / kSimPivotChunk;
     }
-    launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o.retention, st);
+    launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
     {
         Prof p(ctx, st, SLOT_GATHER);
         long long orows = (long long)B * S_out;
@@ -329,6 +345,7 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     if (n_all + p.lag >= (1ll << 30)) return DART_ERR_UNSUPPORTED;
     p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest;
     p.withhold_pivots = o.test_withhold_pivots;
+    p.pivots_given = o.pivots_in != nullptr;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
     p.keys = (const char *)keys;
     p.sim = ctx->sim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
@@ -341,6 +358,7 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     if (rc == DART_OK) rc = encode_2d(ctx, &tm_row, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, 1);
     if (rc != DART_OK) return rc;
     DART_CUDA(ctx, cudaMemsetAsync(ctx->counters, 0, (size_t)B * 2 * sizeof(int), st));
+    if (o.pivots_in) launch_pivots_given(ctx, B, n_vis, P, o.pivots_in, st); // the sweep then only waits for the norms
     {
         Prof pr(ctx, st, SLOT_SWEEP);
         long long grid = n_all < ctx->sm_count ? n_all : ctx->sm_count;
@@ -348,7 +366,7 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
         DART_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)sweep_kernel, dim3((unsigned)grid), dim3(kThreads), args,
                                                    smem_bytes(p.N, p.row_bytes, p.n1, p.n2), st));
     }
-    launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o.retention, st);
+    launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
     {
         Prof pr(ctx, st, SLOT_GATHER);
         long long orows = (long long)B * S_out;
@@ -425,6 +443,9 @@ int dart_create(dart_ctx **out, const dart_desc *desc)
                                       desc->S_max + 16 + dart::kRetainCacheBytes) != cudaSuccess)
             rc = DART_ERR_CUDA;
     }
+    if (rc == DART_OK && cudaFuncSetAttribute(dart::retain_global_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              ctx->max_smem_optin - 2048) != cudaSuccess)
+        rc = DART_ERR_CUDA;
     if (rc == DART_OK && ctx->cand) {
         // the two-phase kernels may use up to the device's shared memory; shapes that need more fall back at launch
         if (cudaFuncSetAttribute(dart::candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -520,6 +541,11 @@ int dart_reduce_ex(dart_ctx *ctx, const void *hidden, const void *keys, const in
     if (o.norm_kind == 0) o.norm_kind = 1;
     if (o.norm_kind != 1 && o.norm_kind != 2) return DART_ERR_UNSUPPORTED;
     if (o.path != DART_PATH_AUTO && o.path != DART_PATH_STAGED && o.path != DART_PATH_FUSED) return DART_ERR_UNSUPPORTED;
+    if (o.rule != DART_RULE_QUOTAS && o.rule != DART_RULE_GLOBAL) return DART_ERR_UNSUPPORTED;
+    if ((uintptr_t)o.pivots_in & 3u) return DART_ERR_ALIGN;
+    if (o.rule == DART_RULE_GLOBAL &&
+        dart::retain_global_smem_bytes(n_vis) > (size_t)ctx->max_smem_optin - 2048)
+        return DART_ERR_UNSUPPORTED; // the sample's duplication values must fit shared memory
     if (o.retention != DART_RETAIN_AUTO && o.retention != DART_RETAIN_SERIAL && o.retention != DART_RETAIN_LISTS)
         return DART_ERR_UNSUPPORTED;
     if ((uintptr_t)pos_in & 7u) return DART_ERR_ALIGN;
@@ -688,6 +714,23 @@ int dart_pivots_static(const void *keys, int B, int S, int d, int vis_offset, in
         (const uint4 *)keys, S, d / 8, vis_offset, n_vis, rows, l1, ssq);
     const int P_pad = next_pow2(n_pivot);
     pivot_kernel<<<B, kSelectThreads, (size_t)P_pad * 8, st>>>(l1, n_vis, n_pivot, P_pad, 0, pivot_idx);
+    return cudaGetLastError() == cudaSuccess ? DART_OK : DART_ERR_CUDA;
+}
+
+int dart_gather_rows(const void *src, const int32_t *idx, int B, int S, int S_out, int row_bytes, void *out, int device,
+                     void *stream)
+{
+    if (!src || !idx || !out) return DART_ERR_NULL;
+    if (B < 1 || S < 1 || S_out < 1 || row_bytes < 16 || row_bytes % 16 != 0) return DART_ERR_BAD_SHAPE;
+    if ((((uintptr_t)src | (uintptr_t)out) & 15u) || ((uintptr_t)idx & 3u)) return DART_ERR_ALIGN;
+    if (overlaps(out, (size_t)B * S_out * row_bytes, src, (size_t)B * S * row_bytes)) return DART_ERR_ALIAS;
+    DeviceGuard g(device);
+    if (!g.ok) return DART_ERR_CUDA;
+    using namespace dart;
+    const long long orows = (long long)B * S_out;
+    const unsigned grid = (unsigned)((orows + kGatherWarps - 1) / kGatherWarps);
+    gather_kernel<<<grid, kGatherWarps * 32, 0, (cudaStream_t)stream>>>((const uint4 *)src, idx, S, S_out, row_bytes / 16, orows,
+                                                                       nullptr, (uint4 *)out);
     return cudaGetLastError() == cudaSuccess ? DART_OK : DART_ERR_CUDA;
 }
 

@@ -178,6 +178,81 @@ sim_alu_kernel(const uint4 *__restrict__ keys, int S, int d8, int vis_offset, in
 }
 
 // ------------------------------------------------------------------------------------------------
+// Step 2 when the caller names the pivots (Sec. 5.2 compares several ways to choose them): the indices
+// are checked - in range, no repeats - and copied into the workspace, clamped so that no later kernel
+// can read outside the sample.  A failed check sets DART_ERR_CHECK in the status word (the retention and
+// gather kernels then leave the outputs alone).  One CTA per sample; dynamic shared memory: one bit per
+// vision token.
+// ------------------------------------------------------------------------------------------------
+constexpr int kStatusCheck = -8;       // DART_ERR_CHECK
+constexpr int kCheckPivotsGiven = 100; // second status word: which check failed
+
+__global__ void __launch_bounds__(256)
+pivots_given_kernel(const int32_t *__restrict__ pivots_in, int n_vis, int P, int32_t *__restrict__ pivot_idx, int *status)
+{
+    extern __shared__ uint32_t seen[]; // [(n_vis + 31) / 32]
+    const int b = blockIdx.x;
+    for (int w = threadIdx.x; w < (n_vis + 31) / 32; w += blockDim.x) seen[w] = 0;
+    __syncthreads();
+    for (int t = threadIdx.x; t < P; t += blockDim.x) {
+        const int pv = pivots_in[(size_t)b * P + t];
+        bool bad = pv < 0 || pv >= n_vis;
+        const int c = min(max(pv, 0), n_vis - 1);
+        if (!bad) bad = (atomicOr(&seen[c >> 5], 1u << (c & 31)) >> (c & 31)) & 1u;
+        pivot_idx[(size_t)b * P + t] = c;
+        if (bad && atomicCAS(status, 0, kStatusCheck) == 0) {
+            status[1] = kCheckPivotsGiven;
+            status[2] = b;
+            status[3] = t;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Step 5a for one sample (all threads of the CTA): the packed index list - text rows before, kept vision
+// tokens in ascending order (ordered ballot scan over the keep flags), text rows after - and the position
+// ids of those rows.  warp_tot: shared scratch, one word per warp.
+// ------------------------------------------------------------------------------------------------
+__device__ inline void pack_indices(const uint8_t *keep, int S, int vis_offset, int n_vis, int n_keep,
+                                    const int64_t *__restrict__ pin, int32_t *__restrict__ oi, int64_t *__restrict__ op,
+                                    uint32_t *warp_tot)
+{
+    for (int t = threadIdx.x; t < vis_offset; t += blockDim.x) {
+        oi[t] = t;
+        op[t] = pin ? pin[t] : (int64_t)t;
+    }
+    const int n_after = S - vis_offset - n_vis;
+    for (int t = threadIdx.x; t < n_after; t += blockDim.x) {
+        const int s = vis_offset + n_vis + t;
+        oi[vis_offset + n_keep + t] = s;
+        op[vis_offset + n_keep + t] = pin ? pin[s] : (int64_t)s;
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    uint32_t base = 0;
+    for (int start = 0; start < n_vis; start += blockDim.x) {
+        const int j = start + threadIdx.x;
+        const bool f = (j < n_vis) && keep[j];
+        const uint32_t bal = __ballot_sync(0xffffffffu, f);
+        if (lane == 0) warp_tot[warp] = __popc(bal);
+        __syncthreads();
+        uint32_t before = 0, total = 0;
+        for (int w = 0; w < nwarp; ++w) {
+            const uint32_t t = warp_tot[w];
+            if (w < warp) before += t;
+            total += t;
+        }
+        if (f) {
+            const uint32_t t = vis_offset + base + before + __popc(bal & ((1u << lane) - 1u));
+            const int s = vis_offset + j;
+            oi[t] = s;
+            op[t] = pin ? pin[s] : (int64_t)s;
+        }
+        base += total;
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Steps 4 and 5a in one kernel: retention (Eq. 9-10) and the packed index list.  One CTA per sample.
 // (Used when the two-phase form below does not apply: more than 4096 tokens to keep beside the pivots.)
 // kept := pivots; pivot i in rank order selects its q_i not-yet-kept tokens of lowest dup (radix
@@ -252,43 +327,8 @@ retain_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_i
         });
         if (eps_out && threadIdx.x == 0) eps_out[(size_t)b * P + i] = order_key_inv(T);
     }
-    // packed index list: text before, kept vision tokens in ascending order, text after
-    int32_t *oi = out_idx + (size_t)b * S_out;
-    int64_t *op = out_pos + (size_t)b * S_out;
-    const int64_t *pin = pos_in ? pos_in + (size_t)b * S : nullptr;
-    for (int t = threadIdx.x; t < vis_offset; t += blockDim.x) {
-        oi[t] = t;
-        op[t] = pin ? pin[t] : (int64_t)t;
-    }
-    const int n_after = S - vis_offset - n_vis;
-    for (int t = threadIdx.x; t < n_after; t += blockDim.x) {
-        int s = vis_offset + n_vis + t;
-        oi[vis_offset + n_keep + t] = s;
-        op[vis_offset + n_keep + t] = pin ? pin[s] : (int64_t)s;
-    }
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-    uint32_t base = 0;
-    for (int start = 0; start < n_vis; start += blockDim.x) {
-        int j = start + threadIdx.x;
-        bool f = (j < n_vis) && keep[j];
-        uint32_t bal = __ballot_sync(0xffffffffu, f);
-        if (lane == 0) sel.warp_tot[warp] = __popc(bal);
-        __syncthreads();
-        uint32_t before = 0, total = 0;
-        for (int w = 0; w < nwarp; ++w) {
-            uint32_t t = sel.warp_tot[w];
-            if (w < warp) before += t;
-            total += t;
-        }
-        if (f) {
-            uint32_t t = vis_offset + base + before + __popc(bal & ((1u << lane) - 1u));
-            int s = vis_offset + j;
-            oi[t] = s;
-            op[t] = pin ? pin[s] : (int64_t)s;
-        }
-        base += total;
-        __syncthreads();
-    }
+    pack_indices(keep, S, vis_offset, n_vis, n_keep, pos_in ? pos_in + (size_t)b * S : nullptr, out_idx + (size_t)b * S_out,
+                 out_pos + (size_t)b * S_out, sel.warp_tot);
     if (keep_out)
         for (int j = threadIdx.x; j < n_vis; j += blockDim.x) keep_out[(size_t)b * n_vis + j] = keep[j];
 }
@@ -450,43 +490,82 @@ retain_walk_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pi
         __syncthreads();
         i0 = i1;
     }
-    // packed index list: text before, kept vision tokens in ascending order, text after
-    int32_t *oi = out_idx + (size_t)b * S_out;
-    int64_t *op = out_pos + (size_t)b * S_out;
-    const int64_t *pin = pos_in ? pos_in + (size_t)b * S : nullptr;
-    for (int t = threadIdx.x; t < vis_offset; t += blockDim.x) {
-        oi[t] = t;
-        op[t] = pin ? pin[t] : (int64_t)t;
+    pack_indices(keep, S, vis_offset, n_vis, n_keep, pos_in ? pos_in + (size_t)b * S : nullptr, out_idx + (size_t)b * S_out,
+                 out_pos + (size_t)b * S_out, warp_tot);
+    if (keep_out)
+        for (int j = threadIdx.x; j < n_vis; j += blockDim.x) keep_out[(size_t)b * n_vis + j] = keep[j];
+}
+
+// ------------------------------------------------------------------------------------------------
+// Steps 4 and 5a with ONE threshold for all pivots (Def. 2 / Eq. 8-9 read with a common eps): a token's
+// duplication is its highest dup to any pivot, u_j = max_i dup[i][j]; the n_keep - P non-pivot tokens of
+// lowest u_j are kept (radix select on order-preserving keys, ties to the lower index), eps = the largest
+// kept u_j.  owner[j] = the pivot token j is most similar to (the first of equals).  One CTA per sample;
+// dynamic shared memory: n_vis rounded to 16 (keep flags) + n_vis * 4 (keys of u_j).
+// ------------------------------------------------------------------------------------------------
+inline size_t retain_global_smem_bytes(int n_vis) { return ((size_t)n_vis + 15) / 16 * 16 + (size_t)n_vis * 4; }
+
+__global__ void __launch_bounds__(kSelectThreads)
+retain_global_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx, const int64_t *__restrict__ pos_in,
+                     int S, int vis_offset, int n_vis, int P, int n_keep,
+                     int32_t *__restrict__ out_idx, int64_t *__restrict__ out_pos,
+                     uint8_t *__restrict__ keep_out, int32_t *__restrict__ owner_out, float *__restrict__ eps_out,
+                     const int *__restrict__ status)
+{
+    extern __shared__ __align__(16) uint8_t keep[]; // [n_vis] flags, then the keys
+    uint32_t *ukey = reinterpret_cast<uint32_t *>(keep + ((size_t)n_vis + 15) / 16 * 16); // [n_vis]
+    __shared__ SelectSmem sel;
+    if (*status != 0) return; // an earlier kernel of this call failed: its outputs are undefined
+    const int b = blockIdx.x;
+    const int S_out = S - n_vis + n_keep;
+    const float *rows = sim + (size_t)b * P * n_vis;
+    int32_t *owner = owner_out ? owner_out + (size_t)b * n_vis : nullptr;
+    for (int j = threadIdx.x; j < n_vis; j += blockDim.x) {
+        float u = rows[j];
+        for (int i = 1; i < P; ++i) u = fmaxf(u, rows[(size_t)i * n_vis + j]); // finite inputs: fmaxf is the plain maximum
+        ukey[j] = order_key(u);
+        keep[j] = 0;
+        if (owner) owner[j] = -1;
     }
-    const int n_after = S - vis_offset - n_vis;
-    for (int t = threadIdx.x; t < n_after; t += blockDim.x) {
-        const int s = vis_offset + n_vis + t;
-        oi[vis_offset + n_keep + t] = s;
-        op[vis_offset + n_keep + t] = pin ? pin[s] : (int64_t)s;
+    __syncthreads();
+    for (int i = threadIdx.x; i < P; i += blockDim.x) {
+        const int pv = pivot_idx[(size_t)b * P + i];
+        keep[pv] = 1;
+        if (owner) owner[pv] = P + i;
     }
-    const int nwarp = blockDim.x >> 5;
-    uint32_t base = 0;
-    for (int start = 0; start < n_vis; start += blockDim.x) {
-        const int j = start + threadIdx.x;
-        const bool f = (j < n_vis) && keep[j];
-        const uint32_t bal = __ballot_sync(0xffffffffu, f);
-        if (lane == 0) warp_tot[warp] = __popc(bal);
-        __syncthreads();
-        uint32_t before = 0, total = 0;
-        for (int w = 0; w < nwarp; ++w) {
-            const uint32_t t = warp_tot[w];
-            if (w < warp) before += t;
-            total += t;
-        }
-        if (f) {
-            const uint32_t t = vis_offset + base + before + __popc(bal & ((1u << lane) - 1u));
-            const int s = vis_offset + j;
-            oi[t] = s;
-            op[t] = pin ? pin[s] : (int64_t)s;
-        }
-        base += total;
-        __syncthreads();
+    __syncthreads();
+    const int take = n_keep - P;
+    float eps = __int_as_float(0x7fc00000);
+    if (take > 0) {
+        auto keyfn = [&](int j, uint32_t &key) {
+            if (keep[j]) return false;
+            key = ukey[j];
+            return true;
+        };
+        uint32_t T, need_eq, cnt_eq;
+        block_select_threshold(CtaGroup(), keyfn, n_vis, (uint32_t)take, sel, T, need_eq, cnt_eq);
+        // picks only flip flags of elements that stay selected, so keyfn may run while others pick
+        block_select_apply(CtaGroup(), keyfn, n_vis, T, need_eq, cnt_eq, sel, [&](int j, uint32_t) {
+            keep[j] = 1;
+            if (owner) {
+                int arg = 0;
+                float u = rows[j];
+                for (int i = 1; i < P; ++i) {
+                    const float v = rows[(size_t)i * n_vis + j];
+                    if (v > u) {
+                        u = v;
+                        arg = i;
+                    }
+                }
+                owner[j] = arg;
+            }
+        });
+        eps = order_key_inv(T);
     }
+    if (eps_out)
+        for (int i = threadIdx.x; i < P; i += blockDim.x) eps_out[(size_t)b * P + i] = eps;
+    pack_indices(keep, S, vis_offset, n_vis, n_keep, pos_in ? pos_in + (size_t)b * S : nullptr, out_idx + (size_t)b * S_out,
+                 out_pos + (size_t)b * S_out, sel.warp_tot);
     if (keep_out)
         for (int j = threadIdx.x; j < n_vis; j += blockDim.x) keep_out[(size_t)b * n_vis + j] = keep[j];
 }
@@ -503,7 +582,7 @@ gather_kernel(const uint4 *__restrict__ hidden, const int32_t *__restrict__ out_
 {
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * kGatherWarps + (threadIdx.x >> 5);
-    if (row >= rows_total || *status != 0) return; // after a failed kernel out_idx is undefined
+    if (row >= rows_total || (status && *status != 0)) return; // after a failed kernel out_idx is undefined
     const int b = (int)(row / S_out);
     const int s = out_idx[row];
     const uint4 *src = hidden + ((size_t)b * S + s) * (size_t)d8;

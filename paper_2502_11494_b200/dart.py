@@ -20,11 +20,13 @@ DART_ERR_CUDA, DART_ERR_NOMEM, DART_ERR_TIMEOUT, DART_ERR_CHECK, DART_ERR_UNSUPP
 DART_FLAG_HOST_STAGING = 1
 DART_PATH_AUTO, DART_PATH_STAGED, DART_PATH_FUSED = 0, 1, 2
 DART_RETAIN_AUTO, DART_RETAIN_SERIAL, DART_RETAIN_LISTS = 0, 1, 2
+DART_RULE_QUOTAS, DART_RULE_GLOBAL = 0, 1
 
 EXPORTS = (
     "dart_create", "dart_destroy", "dart_set_shape", "dart_reduce", "dart_reduce_ex", "dart_reduce_host",
     "dart_status", "dart_status_detail", "dart_last_cuda_error", "dart_workspace_bytes", "dart_launch_count",
     "dart_profile_enable", "dart_profile_read", "dart_strerror", "dart_version", "dart_pivots_static",
+    "dart_gather_rows",
 )
 DART_STATIC_MAX_ROWS = 262144
 
@@ -38,7 +40,8 @@ class dart_desc(ctypes.Structure):
 class dart_opts(ctypes.Structure):
     _fields_ = [("norm_kind", ctypes.c_int32), ("pivot_smallest", ctypes.c_int32), ("path", ctypes.c_int32),
                 ("wait_limit", ctypes.c_int32), ("sweep_lag", ctypes.c_int32),
-                ("test_withhold_pivots", ctypes.c_int32), ("retention", ctypes.c_int32)]
+                ("test_withhold_pivots", ctypes.c_int32), ("retention", ctypes.c_int32), ("rule", ctypes.c_int32),
+                ("pivots_in", ctypes.c_void_p)]
 
 
 class dart_debug(ctypes.Structure):
@@ -83,6 +86,7 @@ def lib() -> ctypes.CDLL:
         L.dart_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32),
                                         ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_int)]
         L.dart_pivots_static.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32p, i32, vp]
+        L.dart_gather_rows.argtypes = [vp, i32p, i32, i32, i32, i32, vp, i32, vp]
         L.dart_strerror.argtypes = [i32]
         L.dart_strerror.restype = ctypes.c_char_p
         L.dart_version.argtypes = []
@@ -134,6 +138,11 @@ def dart_reduce_host(ctx, hidden, keys, vis_offset, n_vis, n_pivot, n_keep, out_
 def dart_pivots_static(keys, B, S, d, vis_offset, n_vis, n_pivot, pivot_idx, device, stream) -> int:
     """Context-free, allocation-free pivot selection (raw device pointers); see include/dart.h."""
     return lib().dart_pivots_static(keys, B, S, d, vis_offset, n_vis, n_pivot, pivot_idx, device, stream)
+
+
+def dart_gather_rows(src, idx, B, S, S_out, row_bytes, out, device, stream) -> int:
+    """Context-free row gather by a packed index list (raw device pointers); see include/dart.h."""
+    return lib().dart_gather_rows(src, idx, B, S, S_out, row_bytes, out, device, stream)
 
 
 def dart_status(ctx) -> int:

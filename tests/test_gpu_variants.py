@@ -1,0 +1,180 @@
+"""The variants next to the main method, CUDA path vs oracle through the C ABI (needs a B200): pivots chosen
+by the caller, retention with one threshold for all pivots, row gather by the packed index list."""
+import ctypes
+
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from oracle import parity  # noqa: E402
+from paper_2502_11494_b200 import dart, workloads as W  # noqa: E402
+from test_gpu_parity import PATH_IDS, PATHS, _np, gaussian  # noqa: E402
+
+pytestmark = pytest.mark.gpu
+
+
+def run(keys, hidden, vo, nv, P, Kp, path, pivots=None, rule=dart.DART_RULE_QUOTAS, expect_status=dart.DART_OK):
+    B, S, d = hidden.shape
+    if path == dart.DART_PATH_FUSED and (d % 64 or P > 256):
+        pytest.skip("the fused path needs d % 64 == 0 and at most 256 pivots")
+    ctx = dart.Dart(B, S, d, P, Kp)
+    try:
+        opts = dart.dart_opts(0, 0, path, 0, 0, 0, 0, rule, None if pivots is None else pivots.data_ptr())
+        res = ctx.reduce(hidden, keys, vo, nv, P, Kp, opts=opts, debug=True)
+        torch.cuda.synchronize()
+        st = ctx.status()
+        detail = dart.dart_status_detail(ctx.handle)
+        assert st == expect_status, (st, detail)
+    finally:
+        ctx.close()
+    return _np(res[0]), _np(res[1]), _np(res[2]), {k: _np(v) for k, v in res[3].items()}, detail
+
+
+def random_pivots(B, nv, P, seed):
+    rng = np.random.default_rng(seed)
+    return np.stack([rng.permutation(nv)[:P] for _ in range(B)]).astype(np.int32)
+
+
+SHAPES = [
+    (2, 120, 64, 5, 100, 4, 30),
+    (3, 333, 264, 17, 301, 7, 60),       # d not a multiple of 64: staged kernels only
+    (2, 700, 4096, 40, 576, 8, 64),      # the LLaVA-1.5 shape
+    (1, 3000, 512, 12, 2880, 16, 320),   # the LLaVA-NeXT token count
+]
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_pivots_given_by_the_caller(oracle, shape, path):
+    B, S, d, vo, nv, P, Kp = shape
+    k, h = gaussian(B, S, d, seed=100 + sum(shape))
+    piv = random_pivots(B, nv, P, seed=sum(shape))
+    oh, oi, op, dbg, _ = run(k, h, vo, nv, P, Kp, path, pivots=torch.from_numpy(piv).cuda())
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=piv)
+    assert np.array_equal(dbg["pivot_idx"], piv)
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, dbg=dbg, pivots_given=True)
+    assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
+def test_own_pivots_given_back_change_nothing(path):
+    w = W.LLAVA15_B64.with_(B=5)
+    k, h = W.make_batch(w, device="cuda")
+    a = run(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, path)
+    piv = torch.from_numpy(a[3]["pivot_idx"]).cuda()
+    b = run(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, path, pivots=piv)
+    assert all(np.array_equal(x, y) for x, y in zip(a[:3], b[:3]))
+    assert all(np.array_equal(a[3][n], b[3][n], equal_nan=(n == "eps")) for n in a[3])
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
+@pytest.mark.parametrize("fault", ["repeated", "negative", "too large"])
+def test_bad_pivots_are_reported_not_used(path, fault):
+    k, h = gaussian(3, 200, 64, seed=31)
+    piv = random_pivots(3, 180, 4, seed=32)
+    piv[1, 3] = {"repeated": piv[1, 0], "negative": -1, "too large": 180}[fault]
+    *_, detail = run(k, h, 10, 180, 4, 40, path, pivots=torch.from_numpy(piv).cuda(), expect_status=dart.DART_ERR_CHECK)
+    assert detail[1][0] == 100 and detail[1][1] == 1 and detail[1][2] == 3   # which check, sample, rank
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
+@pytest.mark.parametrize("shape", SHAPES + [(2, 64, 64, 0, 64, 5, 5), (2, 64, 64, 0, 64, 3, 64)],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_one_threshold_for_all_pivots(oracle, shape, path):
+    B, S, d, vo, nv, P, Kp = shape
+    k, h = gaussian(B, S, d, seed=200 + sum(shape))
+    oh, oi, op, dbg, _ = run(k, h, vo, nv, P, Kp, path, rule=dart.DART_RULE_GLOBAL)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, rule=1)
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, dbg=dbg, rule=1)
+    assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5
+
+
+def test_one_threshold_on_clustered_tokens(oracle):
+    """The LLaVA-1.5-shaped workload (duplicates exist, boundary gaps are small): exact above the margin, valid
+    under tolerance below it, and not the same selection as per-pivot quotas."""
+    w = W.LLAVA15_B64.with_(B=6)
+    k, h = W.make_batch(w, device="cuda")
+    oh, oi, op, dbg, _ = run(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, dart.DART_PATH_AUTO, rule=dart.DART_RULE_GLOBAL)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, rule=1)
+    rep = parity.check_batch(ora, kb, hb, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, oh, oi, op, dbg=dbg, rule=1)
+    assert rep.exact >= rep.above_margin and rep.exact >= 5, rep.notes
+    quota = run(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, dart.DART_PATH_AUTO)
+    assert not np.array_equal(quota[1], oi)
+
+
+def test_both_variants_together(oracle):
+    B, S, d, vo, nv, P, Kp = 2, 300, 128, 20, 260, 6, 50
+    k, h = gaussian(B, S, d, seed=41)
+    piv = random_pivots(B, nv, P, seed=42)
+    oh, oi, op, dbg, _ = run(k, h, vo, nv, P, Kp, dart.DART_PATH_AUTO, pivots=torch.from_numpy(piv).cuda(),
+                             rule=dart.DART_RULE_GLOBAL)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=piv, rule=1)
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, dbg=dbg, pivots_given=True, rule=1)
+    assert rep.exact >= rep.above_margin
+
+
+def test_unknown_rule_is_rejected():
+    k, h = gaussian(1, 64, 64, seed=43)
+    ctx = dart.Dart(1, 64, 64, 2, 8)
+    with pytest.raises(dart.DartError) as e:
+        ctx.reduce(h, k, 0, 64, 2, 8, opts=dart.dart_opts(0, 0, 0, 0, 0, 0, 0, 7, None))
+    assert e.value.code == dart.DART_ERR_UNSUPPORTED
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------- rows gathered by the packed list
+
+def _gather(src, idx, out=None, S_out=None):
+    B, S, w = src.shape
+    S_out = idx.shape[1] if S_out is None else S_out
+    out = torch.empty((B, S_out, w), dtype=src.dtype, device="cuda") if out is None else out
+    P = lambda t: ctypes.c_void_p(t.data_ptr())  # noqa: E731
+    rc = dart.dart_gather_rows(P(src), P(idx), B, S, S_out, w * src.element_size(), P(out), 0,
+                               ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+    return rc, out
+
+
+@pytest.mark.parametrize("B,S,w,S_out", [(1, 16, 8, 16), (3, 700, 4096, 164), (2, 3000, 3584, 420), (5, 90, 24, 1)])
+def test_gather_rows_against_the_oracle(oracle, B, S, w, S_out):
+    g = torch.Generator(device="cuda").manual_seed(B + S + w)
+    src = torch.randint(-32768, 32767, (B, S, w), generator=g, device="cuda", dtype=torch.int16)
+    rng = np.random.default_rng(S_out)
+    idx = np.stack([np.sort(rng.permutation(S)[:S_out]) for _ in range(B)]).astype(np.int32)
+    rc, out = _gather(src, torch.from_numpy(idx).cuda())
+    torch.cuda.synchronize()
+    assert rc == dart.DART_OK
+    assert np.array_equal(out.cpu().numpy().view(np.uint16), oracle.gather_rows(src.cpu().numpy().view(np.uint16), idx))
+
+
+def test_gather_rows_packs_a_kv_cache_like_the_hidden_states(oracle):
+    """The packed list of a reduction, applied to the key states, gives the key rows of the retained tokens."""
+    w = W.LLAVA15_B64.with_(B=3)
+    k, h = W.make_batch(w, device="cuda")
+    ctx = dart.Dart(w.B, w.S, w.d, w.n_pivot, w.n_keep)
+    oh, oi, op = ctx.reduce(h, k, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep)
+    rc_h, again = _gather(h, oi)
+    rc_k, packed_k = _gather(k, oi)
+    torch.cuda.synchronize()
+    assert ctx.status() == dart.DART_OK and rc_h == dart.DART_OK and rc_k == dart.DART_OK
+    ctx.close()
+    assert torch.equal(again.view(torch.int16), oh.view(torch.int16))
+    assert np.array_equal(W.bits(packed_k), oracle.gather_rows(W.bits(k), oi.cpu().numpy()))
+
+
+def test_gather_rows_argument_checks():
+    src = torch.zeros((2, 10, 8), dtype=torch.int16, device="cuda")
+    idx = torch.zeros((2, 4), dtype=torch.int32, device="cuda")
+    P = lambda t: ctypes.c_void_p(t.data_ptr())  # noqa: E731
+    out = torch.empty((2, 4, 8), dtype=torch.int16, device="cuda")
+    assert dart.dart_gather_rows(None, P(idx), 2, 10, 4, 16, P(out), 0, None) == dart.DART_ERR_NULL
+    assert dart.dart_gather_rows(P(src), P(idx), 2, 10, 4, 24, P(out), 0, None) == dart.DART_ERR_BAD_SHAPE   # not a multiple of 16
+    assert dart.dart_gather_rows(P(src), P(idx), 0, 10, 4, 16, P(out), 0, None) == dart.DART_ERR_BAD_SHAPE
+    assert dart.dart_gather_rows(ctypes.c_void_p(src.data_ptr() + 2), P(idx), 2, 10, 4, 16, P(out), 0, None) == dart.DART_ERR_ALIGN
+    assert dart.dart_gather_rows(P(src), P(idx), 2, 10, 4, 16, P(src), 0, None) == dart.DART_ERR_ALIAS
+    assert dart.dart_gather_rows(P(src), P(idx), 2, 10, 4, 16, P(out), 0, None) == dart.DART_OK
+    torch.cuda.synchronize()
