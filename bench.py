@@ -43,6 +43,8 @@ def parse():
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 staged, 2 fused")
     ap.add_argument("--lag", type=int, default=0, help="fused path: extra tasks between a row's two sweeps")
     ap.add_argument("--retention", type=int, default=0, help="0 auto, 1 one kernel, 2 candidate lists + walks")
+    ap.add_argument("--variants", action="store_true",
+                    help="also time the variants: one threshold for all pivots, pivots given by the caller, KV-row gather")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -358,6 +360,39 @@ def main():
                           "path_frac_of_measured_copy": path_bytes_per_sample(wc) * B / (ms2 / n2 * 1e-3) / 1e9 / peak})
             del o2
 
+    variants = None
+    if args.variants and rank == 0:
+        variants = {}
+        n_v = max(3, args.steps // 4)
+        # (a) retention with one threshold for all pivots
+        o_g = dart.dart_opts(0, 0, args.path, 0, args.lag, 0, args.retention, dart.DART_RULE_GLOBAL, None)
+        ms_g, _, prof_g = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_g, False)
+        variants["one_threshold"] = {"ms_per_step": ms_g / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_g * 1e-3),
+                                     "retain_ms": prof_g["retain"][0] / max(prof_g["retain"][1], 1)}
+        # (b) pivots named by the caller (here: random distinct tokens): steps 3-5 only wait for the norms
+        piv = torch.stack([torch.randperm(w.n_vis, device=dev)[:w.n_pivot] for _ in range(B)]).to(torch.int32).contiguous()
+        o_p = dart.dart_opts(0, 0, args.path, 0, args.lag, 0, args.retention, 0, piv.data_ptr())
+        ms_p, _, _ = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_p, False)
+        variants["pivots_given"] = {"ms_per_step": ms_p / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_p * 1e-3)}
+        # (c) the key rows of the retained tokens, packed by the list of the last reduction (one KV tensor of one layer)
+        packed = torch.empty_like(outs[0])
+        st = torch.cuda.current_stream()
+        P_ = lambda t: ctypes.c_void_p(t.data_ptr())  # noqa: E731
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for k_ in range(2 + n_v):
+            if k_ == 2:
+                e0.record(st)
+            rc = dart.dart_gather_rows(P_(keys), P_(outs[1]), B, w.S, w.S_out, 2 * w.d, P_(packed), local,
+                                       ctypes.c_void_p(st.cuda_stream))
+            if rc != 0:
+                raise dart.DartError(rc, "dart_gather_rows")
+        e1.record(st)
+        torch.cuda.synchronize()
+        ms_k = e0.elapsed_time(e1) / n_v
+        gbs = 2 * (2 * w.d * w.S_out) * B / (ms_k * 1e-3) / 1e9
+        variants["kv_row_gather"] = {"ms_per_launch": ms_k, "achieved_GBps": gbs, "frac_of_measured_copy": gbs / peak}
+        del packed, piv
+
     e2e = None
     if not args.no_e2e:
         # the same step through the host-buffer entry point: pinned inputs -> device -> pinned outputs
@@ -418,6 +453,8 @@ def main():
         }
         if sweep is not None:
             line["sweep"] = sweep
+        if variants is not None:
+            line["variants"] = variants
         print(json.dumps(line))
     ctx.close()
     if dist_on:
