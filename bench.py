@@ -77,6 +77,7 @@ def kernel_bytes_per_launch(name, w, B):
         "score": keys + 8 * w.n_vis * B,
         "sim": keys + 4 * w.n_pivot * w.n_vis * B,
         "sweep": keys,                       # fused scores + pivots + similarities: the keys count once
+        "onepass": keys,                     # the caller's pivots: scores + similarities from one pass
         "gather": 2 * (2 * w.d * w.S_out) * B,
         "pivot": 4 * w.n_vis * B,
         "retain": 4 * w.n_pivot * w.n_vis * B + 12 * w.S_out * B,
@@ -372,8 +373,14 @@ def main():
         # (b) pivots named by the caller (here: random distinct tokens): steps 3-5 only wait for the norms
         piv = torch.stack([torch.randperm(w.n_vis, device=dev)[:w.n_pivot] for _ in range(B)]).to(torch.int32).contiguous()
         o_p = dart.dart_opts(0, 0, args.path, 0, args.lag, 0, args.retention, 0, piv.data_ptr())
-        ms_p, _, _ = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_p, False)
-        variants["pivots_given"] = {"ms_per_step": ms_p / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_p * 1e-3)}
+        ms_p, _, prof_p = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_p, False)
+        variants["pivots_given"] = {"ms_per_step": ms_p / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_p * 1e-3),
+                                    "path_frac_of_measured_copy": path_bytes_per_sample(w) * B / (ms_p / n_v * 1e-3) / 1e9 / peak}
+        if prof_p.get("onepass", (0, 0))[1]:
+            ms_o = prof_p["onepass"][0] / prof_p["onepass"][1]
+            gbs_o = kernel_bytes_per_launch("onepass", w, B) / (ms_o * 1e-3) / 1e9
+            variants["pivots_given"]["onepass_kernel"] = {"ms_per_launch": ms_o, "achieved_GBps": gbs_o,
+                                                          "frac_of_measured_copy": gbs_o / peak}
         # (c) the key rows of the retained tokens, packed by the list of the last reduction (one KV tensor of one layer)
         packed = torch.empty_like(outs[0])
         st = torch.cuda.current_stream()

@@ -52,8 +52,9 @@ enum {
 /* dart_opts.path */
 #define DART_PATH_AUTO 0
 #define DART_PATH_STAGED 1 /* one kernel per step of the method, every intermediate in the workspace */
-#define DART_PATH_FUSED 2  /* persistent sweep kernel (scores, pivots and similarities in one launch); needs
-                              d % 64 == 0 and n_pivot <= 256, else UNSUPPORTED.  AUTO picks it when it applies. */
+#define DART_PATH_FUSED 2  /* persistent sweep kernel (scores, pivots and similarities in one launch; with the caller's
+                              pivots: scores and similarities from one pass over the keys); needs d % 64 == 0 and
+                              n_pivot <= 256, else UNSUPPORTED.  AUTO picks it when it applies. */
 
 /* dart_opts.retention */
 #define DART_RETAIN_AUTO 0   /* two phases when the batch alone cannot fill the GPU, else one kernel */
@@ -195,7 +196,9 @@ int dart_status(dart_ctx *ctx);
  * Where the last non-zero status came from (as read by the last dart_status call that returned an error):
  * detail[0] = which bounded wait of the fused kernel expired (1 pivots not published, 2 ring stage not freed,
  * 3 drain, 4 accumulator not freed, 5/6 tile not loaded (MMA / row sums), 7 accumulator not filled, 8/9 mailbox,
- * 10 sweep-1 tasks not all counted, 11/12 selection queue; 100 = a failed check of opts->pivots_in),
+ * 10 sweep-1 tasks not all counted, 11/12 selection queue; 64-70 the one-pass kernel's waits (stage not freed, tile not
+ * loaded (MMA / norms), accumulator not freed / not filled, norms not taken / not ready); 100 = a failed check of
+ * opts->pivots_in),
  * detail[1] = index of the step in the kernel's schedule (or the sample), detail[2] = CTA; for wait 1 also
  * detail[3] = sample.  For bug reports.
  */

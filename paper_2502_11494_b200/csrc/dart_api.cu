@@ -9,11 +9,12 @@
 
 #include "dart_staged.cuh"
 #include "dart_sweep.cuh"
+#include "dart_onepass.cuh"
 
 namespace {
 
-enum Slot { SLOT_SCORE = 0, SLOT_PIVOT, SLOT_SIM, SLOT_RETAIN, SLOT_GATHER, SLOT_SWEEP, SLOT_COUNT };
-const char *const kSlotNames[SLOT_COUNT] = {"score", "pivot", "sim", "retain", "gather", "sweep"};
+enum Slot { SLOT_SCORE = 0, SLOT_PIVOT, SLOT_SIM, SLOT_RETAIN, SLOT_GATHER, SLOT_SWEEP, SLOT_ONEPASS, SLOT_COUNT };
+const char *const kSlotNames[SLOT_COUNT] = {"score", "pivot", "sim", "retain", "gather", "sweep", "onepass"};
 
 typedef CUresult (*TensorMapEncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                       const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -302,6 +303,10 @@ int fused_setup(dart_ctx *ctx)
         per_sm < 1)
         return DART_ERR_CUDA;
     ctx->fused_ok = true;
+    // the one-pass kernel for the caller's pivots uses the same tensor maps
+    if (cudaFuncSetAttribute(dart::onepass::onepass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             ctx->max_smem_optin - dart::onepass::kStaticSmemReserve) != cudaSuccess)
+        return DART_ERR_CUDA;
     return DART_OK;
 }
 
@@ -345,7 +350,6 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     if (n_all + p.lag >= (1ll << 30)) return DART_ERR_UNSUPPORTED;
     p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest;
     p.withhold_pivots = o.test_withhold_pivots;
-    p.pivots_given = o.pivots_in != nullptr;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
     p.keys = (const char *)keys;
     p.sim = ctx->sim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
@@ -358,7 +362,6 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     if (rc == DART_OK) rc = encode_2d(ctx, &tm_row, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, 1);
     if (rc != DART_OK) return rc;
     DART_CUDA(ctx, cudaMemsetAsync(ctx->counters, 0, (size_t)B * 2 * sizeof(int), st));
-    if (o.pivots_in) launch_pivots_given(ctx, B, n_vis, P, o.pivots_in, st); // the sweep then only waits for the norms
     {
         Prof pr(ctx, st, SLOT_SWEEP);
         long long grid = n_all < ctx->sm_count ? n_all : ctx->sm_count;
@@ -378,12 +381,56 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     return copy_debug(ctx, B, n_vis, P, dbg, st);
 }
 
+// The caller's pivots: scores and similarities from one read of the keys (csrc/dart_onepass.cuh), then steps 4-5.
+int launch_onepass(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, const int64_t *pos_in, int vis_offset,
+                   int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos, const dart_opts &o,
+                   const dart_debug *dbg, cudaStream_t st)
+{
+    using namespace dart;
+    using sweep::kSubRows;
+    using sweep::kTileRows;
+    const int S = ctx->S, d8 = ctx->desc.d / 8, S_out = S - n_vis + n_keep;
+    const void *keys = keys_in ? keys_in : hidden;
+    onepass::Params p = {};
+    p.B = B, p.S = S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.N = (P + 15) / 16 * 16;
+    p.n_atoms = ctx->n_atoms, p.n_rt = (n_vis + kTileRows - 1) / kTileRows;
+    p.n_st = onepass::ring_depth(p.N, ctx->max_smem_optin);
+    if (p.n_st < 2) return DART_ERR_UNSUPPORTED;
+    p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
+    p.sim = ctx->sim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
+    p.status = ctx->status;
+    CUtensorMap tm_tile, tm_keys, tm_row;
+    int rc = encode_2d(ctx, &tm_tile, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, kTileRows);
+    if (rc == DART_OK) rc = encode_2d(ctx, &tm_keys, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, kSubRows);
+    if (rc == DART_OK) rc = encode_2d(ctx, &tm_row, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, 1);
+    if (rc != DART_OK) return rc;
+    launch_pivots_given(ctx, B, n_vis, P, o.pivots_in, st);
+    {
+        Prof pr(ctx, st, SLOT_ONEPASS);
+        const long long tasks = (long long)B * p.n_rt;
+        const unsigned grid = (unsigned)(tasks < ctx->sm_count ? tasks : ctx->sm_count); // no CTA waits for another
+        onepass::onepass_kernel<<<grid, onepass::kThreads, onepass::smem_bytes(p.N, p.n_st), st>>>(tm_tile, tm_keys, tm_row, p);
+    }
+    launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
+    {
+        Prof pr(ctx, st, SLOT_GATHER);
+        long long orows = (long long)B * S_out;
+        unsigned grid = (unsigned)((orows + kGatherWarps - 1) / kGatherWarps);
+        gather_kernel<<<grid, kGatherWarps * 32, 0, st>>>((const uint4 *)hidden, out_idx, S, S_out, d8, orows,
+                                                         ctx->status, (uint4 *)out_hidden);
+    }
+    DART_CUDA(ctx, cudaGetLastError());
+    return copy_debug(ctx, B, n_vis, P, dbg, st);
+}
+
 int launch_reduce(dart_ctx *ctx, int B, const void *hidden, const void *keys, const int64_t *pos_in, int vis_offset,
                   int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos, const dart_opts &o,
                   const dart_debug *dbg, cudaStream_t st)
 {
     const bool fused = o.path == DART_PATH_FUSED || (o.path == DART_PATH_AUTO && fused_applies(ctx, P));
     if (fused && !fused_applies(ctx, P)) return DART_ERR_UNSUPPORTED;
+    if (fused && o.pivots_in) // nothing waits for a selection: one pass over the keys
+        return launch_onepass(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o, dbg, st);
     return fused ? launch_fused(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos,
                                 o, dbg, st)
                  : launch_staged(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos,

@@ -1,0 +1,327 @@
+// One-pass path for pivots that are known before the step starts (the caller's pivots): scores and
+// similarities from ONE read of the key rows.
+//
+// With the pivots given, nothing in a row's dot products (Eq. 7's numerator) waits for another row, so a
+// row tile is streamed once and used twice while it sits in shared memory: the tensor cores multiply it
+// with the sample's pivot rows (tokens = M 128, pivots = N, bf16 -> fp32 in TMEM, accumulating over all
+// of d), and four warps add up |x| (the K-norm of the Sec. 3.3 footnote) and x^2 (Eq. 7's denominator)
+// of the same 128 rows, and of the pivot rows that came with the tile.  The epilogue divides by the two
+// norms and writes dup(p_i, x_j) (Eq. 7).  No CTA depends on another one: tasks (sample, row tile) are
+// dealt out round-robin to a persistent grid of one CTA per SM.
+//
+// Per CTA (384 threads; warps 2-3 idle):
+//   warp 0     producer: per 64-column atom one 128-row TMA tile (128-byte swizzle) and the pivot rows by
+//              tile::gather4, two atoms per stage of a ring
+//   warp 1     one thread issues tcgen05.mma; tcgen05.commit releases the stage on the tensor cores' behalf
+//   warps 4-7  norms: thread t owns tile row t (and pivot rows t, t + 128 of the stage's pivot tile) and sums
+//              its 128 bytes of every atom, in column order whatever the swizzle did to the chunks, so a
+//              row's norm does not depend on where in a tile it was read
+//   warps 8-11 epilogue: TMEM -> normalised similarities [B][P][n_vis]
+// Every wait is bounded in time; on expiry the kernel records DART_ERR_TIMEOUT in the status word, lets the
+// copies and MMAs in flight finish, frees TMEM and exits normally.  Results are bitwise reproducible.
+#pragma once
+#include "dart_sweep.cuh"
+
+namespace dart {
+namespace onepass {
+
+using namespace sweep; // PTX wrappers, Ctl, Ring, tile constants
+
+constexpr int kThreads = 384;
+constexpr int kNormWarp0 = 4, kNormWarps = 4;
+constexpr int kEpi0 = 8;          // kEpi0 % 4 == 0: warp w reads TMEM lanes 32 (w % 4) ...
+constexpr int kStages = 10;       // at most
+constexpr int kAtomsPerStage = 2; // one barrier round per two 64-column atoms: the producer's issue latency is per stage
+constexpr int kStaticSmemReserve = 8192;
+enum { kWaitStageFree = 64, kWaitStageMma, kWaitStageNorm, kWaitAccumFree1, kWaitAccumFull1, kWaitNormFree, kWaitNormFull };
+
+struct Params {
+    int B, S, vis_offset, n_vis, P, N; // N = P rounded up to a multiple of 16 (MMA N)
+    int n_atoms, n_rt;                 // 64-column atoms per row; row tiles per sample
+    int n_st;                          // ring depth
+    unsigned long long wait_ns;
+    float *sim;                        // [B][P][n_vis] dup(p_i, x_j)
+    float *l1, *ssq;                   // [B][n_vis]
+    const int32_t *pivot_idx;          // [B][P], checked and clamped
+    int *status;
+};
+
+struct Shared {
+    unsigned long long full[kStages], empty[kStages];
+    unsigned long long tmem_full[2], tmem_empty[2], norm_full[2], norm_empty[2];
+    unsigned long long mma_drain;
+    uint32_t tmem_base;
+    int abort_flag;
+    float row_ssq[2][kTileRows]; // per accumulator buffer: sum of squares of the tile's rows
+    float piv_ssq[2][kMaxN];     // ... and of the sample's pivot rows
+};
+static_assert(sizeof(Shared) + 64 <= kStaticSmemReserve, "static shared memory exceeds its reserve");
+
+__host__ __device__ inline uint32_t stage_bytes(int N) { return (uint32_t)kAtomsPerStage * (kAtomBytes + b_stage_bytes(N)); }
+__host__ inline int ring_depth(int N, size_t smem_limit)
+{
+    const size_t n = (smem_limit - 1024 - kStaticSmemReserve) / stage_bytes(N);
+    return (int)(n > (size_t)kStages ? (size_t)kStages : n);
+}
+__host__ inline size_t smem_bytes(int N, int n_st) { return 1024 + (size_t)n_st * stage_bytes(N); }
+
+// |x| and x^2 of one 128-byte row of a 128B-swizzled tile, added to the four running sums in column order:
+// logical 16-byte chunk c of row r sits at chunk position c ^ (r & 7)
+__device__ __forceinline__ void add_row(uint32_t tile, int r, float &a0, float &a1, float &q0, float &q1)
+{
+    const uint32_t row = tile + (uint32_t)r * 128u;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const uint4 v = lds128(row + (uint32_t)((c ^ (r & 7)) * 16));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float lo = bf16_lo(w[e]), hi = bf16_hi(w[e]);
+            a0 += fabsf(lo);
+            a1 += fabsf(hi);
+            q0 = fmaf(lo, lo, q0);
+            q1 = fmaf(hi, hi, q1);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant__ CUtensorMap tm_keys,
+               const __grid_constant__ CUtensorMap tm_row, const Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ Shared sh;
+    const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bstage = b_stage_bytes(p.N);
+    // stage s: kAtomsPerStage token tiles, then as many pivot tiles
+    auto a_addr = [&](int s, int h) { return smem0 + (uint32_t)s * stage_bytes(p.N) + (uint32_t)h * kAtomBytes; };
+    auto b_addr = [&](int s, int h) {
+        return smem0 + (uint32_t)s * stage_bytes(p.N) + (uint32_t)kAtomsPerStage * kAtomBytes + (uint32_t)h * bstage;
+    };
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned long long limit = 2ull * p.wait_ns; // ns -> cycles at the highest SM clock: never shorter than asked
+    const Ctl ctl{&sh.abort_flag, p.status, warp == 0 ? limit : limit + limit / 4};
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&sh.full[s]), 1);
+            mbar_init(smem_u32(&sh.empty[s]), 1 + kNormWarps); // the MMAs' commit and every norm warp
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&sh.tmem_full[a]), 1);
+            mbar_init(smem_u32(&sh.tmem_empty[a]), kEpiWarps);
+            mbar_init(smem_u32(&sh.norm_full[a]), kNormWarps);
+            mbar_init(smem_u32(&sh.norm_empty[a]), kEpiWarps);
+        }
+        mbar_init(smem_u32(&sh.mma_drain), 1);
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    uint32_t tmem_cols = 32;
+    while (tmem_cols < 2u * p.N) tmem_cols <<= 1;
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = sh.tmem_base;
+    const uint32_t total = (uint32_t)p.B * (uint32_t)p.n_rt; // tasks: (sample, row tile), sample-major
+    const int na = p.n_atoms;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        unsigned long long pol_keep, pol_drop;
+        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));  // pivot rows: every tile of the sample
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_drop)); // token rows: read once
+        Ring ring(p.n_st);
+        long long issued = 0;
+        bool ok = true;
+        int cur_b = -1;
+        int my_piv[kMaxN / 128][4]; // lane l loads pivot ranks 4l..4l+3, 4(l+32).., as rows of the key tensor
+        for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
+            const int b = (int)(g / (uint32_t)p.n_rt), rt = (int)(g - (uint32_t)b * (uint32_t)p.n_rt);
+            if (b != cur_b) {
+#pragma unroll
+                for (int k = 0; k < kMaxN / 128; ++k)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int i = min(4 * (lane + 32 * k) + e, p.P - 1); // ranks beyond P repeat the last pivot
+                        my_piv[k][e] = b * p.S + p.vis_offset + min(max(__ldg(p.pivot_idx + (size_t)b * p.P + i), 0), p.n_vis - 1);
+                    }
+                cur_b = b;
+            }
+            const int rows = min(kTileRows, p.n_vis - rt * kTileRows);
+            const int n_sub = (rows + kSubRows - 1) / kSubRows;
+            const int y0 = b * p.S + p.vis_offset + rt * kTileRows;
+            for (int a = 0; a < na; a += kAtomsPerStage) {
+                const int nh = min(kAtomsPerStage, na - a); // atoms in this stage
+                const uint32_t full = smem_u32(&sh.full[ring.stage]);
+                if (lane == 0) {
+                    ok = ctl.wait_bar(smem_u32(&sh.empty[ring.stage]), ring.phase ^ 1u, kWaitStageFree, g);
+                    if (ok)
+                        mbar_arrive_expect_tx(full, (uint32_t)nh * ((rows == kTileRows ? (uint32_t)kAtomBytes : (uint32_t)n_sub * kSubBytes) +
+                                                                    (uint32_t)((p.P + 3) / 4) * 512u));
+                }
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                if (!ok) break;
+                for (int h = 0; h < nh; ++h) {
+                    const int x = (a + h) * kAtomCols;
+                    const uint32_t dst = a_addr(ring.stage, h);
+                    if (rows == kTileRows) {
+                        if (lane == h) tma_load_2d(dst, &tm_tile, x, y0, full, pol_drop); // one lane per atom: issued side by side
+                    } else if (lane < n_sub) {
+                        tma_load_2d(dst + (uint32_t)lane * kSubBytes, &tm_keys, x, y0 + lane * kSubRows, full, pol_drop);
+                    }
+#pragma unroll
+                    for (int k = 0; k < kMaxN / 128; ++k) {
+                        const int q = lane + 32 * k; // pivot ranks 4q..4q+3 -> rows 4q..4q+3 of the pivot tile
+                        if (4 * q < p.P)
+                            tma_gather4(b_addr(ring.stage, h) + (uint32_t)q * 512u, &tm_row, x, my_piv[k][0], my_piv[k][1],
+                                        my_piv[k][2], my_piv[k][3], full, pol_keep);
+                    }
+                }
+                ring.advance();
+                ++issued;
+            }
+        }
+        if ((!ok || ctl.aborted()) && lane == 0) // let the copies already issued land before the CTA may exit
+            for (long long i = issued > p.n_st ? issued - p.n_st : 0; i < issued; ++i)
+                ctl.wait_landed(smem_u32(&sh.full[i % p.n_st]), (uint32_t)((i / p.n_st) & 1));
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc(p.N);
+            Ring ring(p.n_st);
+            uint32_t n = 0;
+            bool ok = true;
+            for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
+                const uint32_t acc = n & 1u;
+                ok = ctl.wait_bar(smem_u32(&sh.tmem_empty[acc]), ((n >> 1) & 1u) ^ 1u, kWaitAccumFree1, g);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)p.N;
+                for (int a = 0; a < na; a += kAtomsPerStage) {
+                    ok = ctl.wait_bar(smem_u32(&sh.full[ring.stage]), ring.phase, kWaitStageMma, g);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    for (int h = 0; h < min(kAtomsPerStage, na - a); ++h) {
+                        const unsigned long long da = umma_desc(a_addr(ring.stage, h)), db = umma_desc(b_addr(ring.stage, h));
+#pragma unroll
+                        for (int k = 0; k < kAtomCols / 16; ++k) // 16 columns = 32 bytes per MMA: advance the start address
+                            umma_bf16(d_tmem, da + (unsigned long long)(2 * k), db + (unsigned long long)(2 * k), idesc,
+                                      (a | h | k) != 0);
+                    }
+                    umma_commit(smem_u32(&sh.empty[ring.stage])); // the tensor cores' share of releasing the stage
+                    ring.advance();
+                }
+                if (!ok) break;
+                umma_commit(smem_u32(&sh.tmem_full[acc]));
+                ++n;
+            }
+            if (!ok || ctl.aborted()) { // TMEM is freed at the end: first let the MMAs issued so far finish
+                umma_commit(smem_u32(&sh.mma_drain));
+                ctl.wait_landed(smem_u32(&sh.mma_drain), 0);
+            }
+        }
+    } else if (warp >= kNormWarp0 && warp < kNormWarp0 + kNormWarps) {
+        // ------------------------------------------------------------------ norms of the tile's rows and of the pivot rows
+        const int t = (int)threadIdx.x - kNormWarp0 * 32; // tile row owned by this thread; pivot rows t and t + 128
+        Ring ring(p.n_st);
+        uint32_t n = 0;
+        bool dead = false; // warp-uniform
+        for (uint32_t g = blockIdx.x; !dead && g < total; g += gridDim.x) {
+            const int b = (int)(g / (uint32_t)p.n_rt), rt = (int)(g - (uint32_t)b * (uint32_t)p.n_rt);
+            const int rows = min(kTileRows, p.n_vis - rt * kTileRows);
+            float a0 = 0.f, a1 = 0.f, q0 = 0.f, q1 = 0.f; // own tile row
+            float pq[kMaxN / 128][2];                      // own pivot rows: sums of squares only
+#pragma unroll
+            for (int k = 0; k < kMaxN / 128; ++k) pq[k][0] = pq[k][1] = 0.f;
+            for (int a = 0; a < na; a += kAtomsPerStage) {
+                dead = !ctl.wait_bar(smem_u32(&sh.full[ring.stage]), ring.phase, kWaitStageNorm, g);
+                dead = __any_sync(0xffffffffu, dead);
+                if (dead) break;
+                for (int h = 0; h < min(kAtomsPerStage, na - a); ++h) { // atoms in column order: the sums do not depend on the staging
+                    if (t < rows) add_row(a_addr(ring.stage, h), t, a0, a1, q0, q1);
+#pragma unroll
+                    for (int k = 0; k < kMaxN / 128; ++k)
+                        if (t + 128 * k < p.P) {
+                            float x0 = 0.f, x1 = 0.f;
+                            add_row(b_addr(ring.stage, h), t + 128 * k, x0, x1, pq[k][0], pq[k][1]);
+                        }
+                }
+                __syncwarp(); // the warp's reads of the stage are done
+                if (lane == 0) mbar_arrive(smem_u32(&sh.empty[ring.stage]));
+                ring.advance();
+            }
+            if (dead) break;
+            const uint32_t acc = n & 1u;
+            // the slot is free once the epilogue has used the norms of the task two before
+            dead = !ctl.wait_bar(smem_u32(&sh.norm_empty[acc]), ((n >> 1) & 1u) ^ 1u, kWaitNormFree, g);
+            dead = __any_sync(0xffffffffu, dead);
+            if (dead) break;
+            const float q = q0 + q1;
+            sh.row_ssq[acc][t] = t < rows ? q : 0.f;
+#pragma unroll
+            for (int k = 0; k < kMaxN / 128; ++k)
+                if (t + 128 * k < p.P) sh.piv_ssq[acc][t + 128 * k] = pq[k][0] + pq[k][1];
+            if (t < rows) {
+                const size_t o = (size_t)b * p.n_vis + rt * kTileRows + t;
+                p.l1[o] = a0 + a1;
+                p.ssq[o] = q;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh.norm_full[acc])); // release: the warp's norms are ordered before it
+            ++n;
+        }
+    } else if (warp >= kEpi0 && warp < kEpi0 + kEpiWarps) {
+        // ------------------------------------------------------------------ epilogue (warps independent)
+        const int quarter = warp & 3;        // TMEM lane quarter this warp may read
+        const int row = quarter * 32 + lane; // tile row owned by this thread
+        uint32_t n = 0;
+        for (uint32_t g = blockIdx.x; g < total; g += gridDim.x) {
+            const int b = (int)(g / (uint32_t)p.n_rt), rt = (int)(g - (uint32_t)b * (uint32_t)p.n_rt);
+            const int rows = min(kTileRows, p.n_vis - rt * kTileRows);
+            const int j = rt * kTileRows + row;
+            const uint32_t acc = n & 1u;
+            bool ok = ctl.wait_bar(smem_u32(&sh.norm_full[acc]), (n >> 1) & 1u, kWaitNormFull, g);
+            if (ok) ok = ctl.wait_bar(smem_u32(&sh.tmem_full[acc]), (n >> 1) & 1u, kWaitAccumFull1, g);
+            if (!__all_sync(0xffffffffu, ok)) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const float nj = sqrtf(sh.row_ssq[acc][row]);
+            const uint32_t taddr = tmem_base + acc * (uint32_t)p.N + ((uint32_t)(quarter * 32) << 16);
+            float *dst = p.sim + (size_t)b * p.P * p.n_vis + j;
+            for (int c0 = 0; c0 < p.P; c0 += 8) {
+                float v[8];
+                tmem_ld8(taddr + (uint32_t)c0, v); // warp-collective: rows outside the tile still take part
+                if (row < rows) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        if (c0 + e < p.P) { // dup = dot / (|pivot| |row|); a zero norm gives 0; a warp writes 128 contiguous bytes
+                            const float den = sqrtf(sh.piv_ssq[acc][c0 + e]) * nj;
+                            dst[(size_t)(c0 + e) * p.n_vis] = den > 0.f ? v[e] / den : 0.f;
+                        }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&sh.tmem_empty[acc]));
+                mbar_arrive(smem_u32(&sh.norm_empty[acc]));
+            }
+            ++n;
+        }
+    }
+    // ---------------------------------------------------------------------- teardown
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+}
+
+} // namespace onepass
+} // namespace dart

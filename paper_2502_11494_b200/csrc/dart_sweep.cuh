@@ -74,7 +74,6 @@ struct Params {
     uint32_t lag;                      // steps between the two sweeps (Tm <= lag <= B * Tm)
     int norm_kind, smallest;
     int withhold_pivots;               // test hook: never publish pivots, so that the bounded waits expire
-    int pivots_given;                  // the caller's pivots are already in pivot_idx: selection only publishes
     unsigned long long wait_ns;        // time limit of every wait
     const char *keys;                  // [B][S][d] bf16
     float *sim;                        // [B][P][n_vis] dup(p_i, x_j)
@@ -355,10 +354,6 @@ __device__ void select_pivots(const Params &p, Shared &sh, int b)
 {
     const Selectors g;
     const int lane = g.tid(); // 0 .. kSel-1
-    if (p.pivots_given) { // nothing to select: the sample's norms are complete, which is all sweep 2 waited for
-        if (lane == 0 && !p.withhold_pivots) st_release(p.piv_ready + b, 1);
-        return;
-    }
     const float *score = (p.norm_kind == 2 ? p.ssq : p.l1) + (size_t)b * p.n_vis;
     const int smallest = p.smallest;
     const bool cached = p.n_vis <= kSelMax;

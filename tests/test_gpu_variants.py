@@ -66,7 +66,11 @@ def test_own_pivots_given_back_change_nothing(path):
     piv = torch.from_numpy(a[3]["pivot_idx"]).cuda()
     b = run(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, path, pivots=piv)
     assert all(np.array_equal(x, y) for x, y in zip(a[:3], b[:3]))
-    assert all(np.array_equal(a[3][n], b[3][n], equal_nan=(n == "eps")) for n in a[3])
+    for n in ("pivot_idx", "keep", "owner"):
+        assert np.array_equal(a[3][n], b[3][n])
+    # with the pivots given the fused path sums a row's norms in another order (one pass over swizzled tiles)
+    for n in ("l1", "ssq", "sim", "eps"):
+        assert np.allclose(a[3][n], b[3][n], rtol=1e-5, atol=1e-6, equal_nan=True)
 
 
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
