@@ -394,7 +394,8 @@ int launch_onepass(dart_ctx *ctx, int B, const void *hidden, const void *keys_in
     onepass::Params p = {};
     p.B = B, p.S = S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.N = (P + 15) / 16 * 16;
     p.n_atoms = ctx->n_atoms, p.n_rt = (n_vis + kTileRows - 1) / kTileRows;
-    p.n_st = onepass::ring_depth(p.N, ctx->max_smem_optin);
+    p.aps = onepass::atoms_per_stage(p.N, ctx->max_smem_optin);
+    p.n_st = onepass::ring_depth(p.N, p.aps, ctx->max_smem_optin);
     if (p.n_st < 2) return DART_ERR_UNSUPPORTED;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
     p.sim = ctx->sim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
@@ -409,7 +410,7 @@ int launch_onepass(dart_ctx *ctx, int B, const void *hidden, const void *keys_in
         Prof pr(ctx, st, SLOT_ONEPASS);
         const long long tasks = (long long)B * p.n_rt;
         const unsigned grid = (unsigned)(tasks < ctx->sm_count ? tasks : ctx->sm_count); // no CTA waits for another
-        onepass::onepass_kernel<<<grid, onepass::kThreads, onepass::smem_bytes(p.N, p.n_st), st>>>(tm_tile, tm_keys, tm_row, p);
+        onepass::onepass_kernel<<<grid, onepass::kThreads, onepass::smem_bytes(p.N, p.aps, p.n_st), st>>>(tm_tile, tm_keys, tm_row, p);
     }
     launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
     {

@@ -9,13 +9,13 @@
 // norms and writes dup(p_i, x_j) (Eq. 7).  No CTA depends on another one: tasks (sample, row tile) are
 // dealt out round-robin to a persistent grid of one CTA per SM.
 //
-// Per CTA (384 threads; warps 2-3 idle):
+// Per CTA (384 threads):
 //   warp 0     producer: per 64-column atom one 128-row TMA tile (128-byte swizzle) and the pivot rows by
-//              tile::gather4, two atoms per stage of a ring
+//              tile::gather4, up to four atoms per stage of a ring
 //   warp 1     one thread issues tcgen05.mma; tcgen05.commit releases the stage on the tensor cores' behalf
-//   warps 4-7  norms: thread t owns tile row t (and pivot rows t, t + 128 of the stage's pivot tile) and sums
-//              its 128 bytes of every atom, in column order whatever the swizzle did to the chunks, so a
-//              row's norm does not depend on where in a tile it was read
+//   warps 4-7  norms: thread t owns tile row t and sums its 128 bytes of every atom, in column order whatever
+//              the swizzle did to the chunks, so a row's norm does not depend on where in a tile it was read
+//   warps 2-3  the same for the pivot rows of the stage's pivot tile (thread u: rows u, u + 64, ...)
 //   warps 8-11 epilogue: TMEM -> normalised similarities [B][P][n_vis]
 // Every wait is bounded in time; on expiry the kernel records DART_ERR_TIMEOUT in the status word, lets the
 // copies and MMAs in flight finish, frees TMEM and exits normally.  Results are bitwise reproducible.
@@ -29,16 +29,18 @@ using namespace sweep; // PTX wrappers, Ctl, Ring, tile constants
 
 constexpr int kThreads = 384;
 constexpr int kNormWarp0 = 4, kNormWarps = 4;
+constexpr int kPivWarp0 = 2, kPivWarps = 2, kPivThreads = kPivWarps * 32;
 constexpr int kEpi0 = 8;          // kEpi0 % 4 == 0: warp w reads TMEM lanes 32 (w % 4) ...
 constexpr int kStages = 10;       // at most
-constexpr int kAtomsPerStage = 2; // one barrier round per two 64-column atoms: the producer's issue latency is per stage
+constexpr int kMaxAtomsPerStage = 4; // a stage holds up to four 64-column atoms: the producer's issue latency (wait, expect,
+                                     // issue: ~0.3 us) is paid per stage; measured at 8 pivots: 1 atom 1.40 ms, 2 1.14, 4 1.02
 constexpr int kStaticSmemReserve = 8192;
 enum { kWaitStageFree = 64, kWaitStageMma, kWaitStageNorm, kWaitAccumFree1, kWaitAccumFull1, kWaitNormFree, kWaitNormFull };
 
 struct Params {
     int B, S, vis_offset, n_vis, P, N; // N = P rounded up to a multiple of 16 (MMA N)
     int n_atoms, n_rt;                 // 64-column atoms per row; row tiles per sample
-    int n_st;                          // ring depth
+    int n_st, aps;                     // ring depth; atoms per stage (<= kMaxAtomsPerStage)
     unsigned long long wait_ns;
     float *sim;                        // [B][P][n_vis] dup(p_i, x_j)
     float *l1, *ssq;                   // [B][n_vis]
@@ -57,13 +59,20 @@ struct Shared {
 };
 static_assert(sizeof(Shared) + 64 <= kStaticSmemReserve, "static shared memory exceeds its reserve");
 
-__host__ __device__ inline uint32_t stage_bytes(int N) { return (uint32_t)kAtomsPerStage * (kAtomBytes + b_stage_bytes(N)); }
-__host__ inline int ring_depth(int N, size_t smem_limit)
+__host__ __device__ inline uint32_t stage_bytes(int N, int aps) { return (uint32_t)aps * (kAtomBytes + b_stage_bytes(N)); }
+__host__ inline int ring_depth(int N, int aps, size_t smem_limit)
 {
-    const size_t n = (smem_limit - 1024 - kStaticSmemReserve) / stage_bytes(N);
+    const size_t n = (smem_limit - 1024 - kStaticSmemReserve) / stage_bytes(N, aps);
     return (int)(n > (size_t)kStages ? (size_t)kStages : n);
 }
-__host__ inline size_t smem_bytes(int N, int n_st) { return 1024 + (size_t)n_st * stage_bytes(N); }
+// As many atoms per stage as still leave three stages (with many pivots the pivot tiles crowd them out)
+__host__ inline int atoms_per_stage(int N, size_t smem_limit)
+{
+    int aps = kMaxAtomsPerStage;
+    while (aps > 1 && ring_depth(N, aps, smem_limit) < 3) aps >>= 1;
+    return aps;
+}
+__host__ inline size_t smem_bytes(int N, int aps, int n_st) { return 1024 + (size_t)n_st * stage_bytes(N, aps); }
 
 // |x| and x^2 of one 128-byte row of a 128B-swizzled tile, added to the four running sums in column order:
 // logical 16-byte chunk c of row r sits at chunk position c ^ (r & 7)
@@ -93,10 +102,10 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
     __shared__ Shared sh;
     const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bstage = b_stage_bytes(p.N);
-    // stage s: kAtomsPerStage token tiles, then as many pivot tiles
-    auto a_addr = [&](int s, int h) { return smem0 + (uint32_t)s * stage_bytes(p.N) + (uint32_t)h * kAtomBytes; };
+    // stage s: p.aps token tiles, then as many pivot tiles
+    auto a_addr = [&](int s, int h) { return smem0 + (uint32_t)s * stage_bytes(p.N, p.aps) + (uint32_t)h * kAtomBytes; };
     auto b_addr = [&](int s, int h) {
-        return smem0 + (uint32_t)s * stage_bytes(p.N) + (uint32_t)kAtomsPerStage * kAtomBytes + (uint32_t)h * bstage;
+        return smem0 + (uint32_t)s * stage_bytes(p.N, p.aps) + (uint32_t)p.aps * kAtomBytes + (uint32_t)h * bstage;
     };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned long long limit = 2ull * p.wait_ns; // ns -> cycles at the highest SM clock: never shorter than asked
@@ -105,12 +114,12 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem_u32(&sh.full[s]), 1);
-            mbar_init(smem_u32(&sh.empty[s]), 1 + kNormWarps); // the MMAs' commit and every norm warp
+            mbar_init(smem_u32(&sh.empty[s]), 1 + kNormWarps + kPivWarps); // the MMAs' commit and every norm warp
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&sh.tmem_full[a]), 1);
             mbar_init(smem_u32(&sh.tmem_empty[a]), kEpiWarps);
-            mbar_init(smem_u32(&sh.norm_full[a]), kNormWarps);
+            mbar_init(smem_u32(&sh.norm_full[a]), kNormWarps + kPivWarps);
             mbar_init(smem_u32(&sh.norm_empty[a]), kEpiWarps);
         }
         mbar_init(smem_u32(&sh.mma_drain), 1);
@@ -157,8 +166,8 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
             const int rows = min(kTileRows, p.n_vis - rt * kTileRows);
             const int n_sub = (rows + kSubRows - 1) / kSubRows;
             const int y0 = b * p.S + p.vis_offset + rt * kTileRows;
-            for (int a = 0; a < na; a += kAtomsPerStage) {
-                const int nh = min(kAtomsPerStage, na - a); // atoms in this stage
+            for (int a = 0; a < na; a += p.aps) {
+                const int nh = min(p.aps, na - a); // atoms in this stage
                 const uint32_t full = smem_u32(&sh.full[ring.stage]);
                 if (lane == 0) {
                     ok = ctl.wait_bar(smem_u32(&sh.empty[ring.stage]), ring.phase ^ 1u, kWaitStageFree, g);
@@ -204,11 +213,11 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem_base + acc * (uint32_t)p.N;
-                for (int a = 0; a < na; a += kAtomsPerStage) {
+                for (int a = 0; a < na; a += p.aps) {
                     ok = ctl.wait_bar(smem_u32(&sh.full[ring.stage]), ring.phase, kWaitStageMma, g);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    for (int h = 0; h < min(kAtomsPerStage, na - a); ++h) {
+                    for (int h = 0; h < min(p.aps, na - a); ++h) {
                         const unsigned long long da = umma_desc(a_addr(ring.stage, h)), db = umma_desc(b_addr(ring.stage, h));
 #pragma unroll
                         for (int k = 0; k < kAtomCols / 16; ++k) // 16 columns = 32 bytes per MMA: advance the start address
@@ -229,7 +238,7 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
         }
     } else if (warp >= kNormWarp0 && warp < kNormWarp0 + kNormWarps) {
         // ------------------------------------------------------------------ norms of the tile's rows and of the pivot rows
-        const int t = (int)threadIdx.x - kNormWarp0 * 32; // tile row owned by this thread; pivot rows t and t + 128
+        const int t = (int)threadIdx.x - kNormWarp0 * 32; // tile row owned by this thread
         Ring ring(p.n_st);
         uint32_t n = 0;
         bool dead = false; // warp-uniform
@@ -237,22 +246,12 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
             const int b = (int)(g / (uint32_t)p.n_rt), rt = (int)(g - (uint32_t)b * (uint32_t)p.n_rt);
             const int rows = min(kTileRows, p.n_vis - rt * kTileRows);
             float a0 = 0.f, a1 = 0.f, q0 = 0.f, q1 = 0.f; // own tile row
-            float pq[kMaxN / 128][2];                      // own pivot rows: sums of squares only
-#pragma unroll
-            for (int k = 0; k < kMaxN / 128; ++k) pq[k][0] = pq[k][1] = 0.f;
-            for (int a = 0; a < na; a += kAtomsPerStage) {
+            for (int a = 0; a < na; a += p.aps) {
                 dead = !ctl.wait_bar(smem_u32(&sh.full[ring.stage]), ring.phase, kWaitStageNorm, g);
                 dead = __any_sync(0xffffffffu, dead);
                 if (dead) break;
-                for (int h = 0; h < min(kAtomsPerStage, na - a); ++h) { // atoms in column order: the sums do not depend on the staging
+                for (int h = 0; h < min(p.aps, na - a); ++h) // atoms in column order: the sums do not depend on the staging
                     if (t < rows) add_row(a_addr(ring.stage, h), t, a0, a1, q0, q1);
-#pragma unroll
-                    for (int k = 0; k < kMaxN / 128; ++k)
-                        if (t + 128 * k < p.P) {
-                            float x0 = 0.f, x1 = 0.f;
-                            add_row(b_addr(ring.stage, h), t + 128 * k, x0, x1, pq[k][0], pq[k][1]);
-                        }
-                }
                 __syncwarp(); // the warp's reads of the stage are done
                 if (lane == 0) mbar_arrive(smem_u32(&sh.empty[ring.stage]));
                 ring.advance();
@@ -265,9 +264,6 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
             if (dead) break;
             const float q = q0 + q1;
             sh.row_ssq[acc][t] = t < rows ? q : 0.f;
-#pragma unroll
-            for (int k = 0; k < kMaxN / 128; ++k)
-                if (t + 128 * k < p.P) sh.piv_ssq[acc][t + 128 * k] = pq[k][0] + pq[k][1];
             if (t < rows) {
                 const size_t o = (size_t)b * p.n_vis + rt * kTileRows + t;
                 p.l1[o] = a0 + a1;
@@ -275,6 +271,43 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh.norm_full[acc])); // release: the warp's norms are ordered before it
+            ++n;
+        }
+    } else if (warp >= kPivWarp0 && warp < kPivWarp0 + kPivWarps) {
+        // ------------------------------------------------------------------ norms of the pivot rows that come with every tile
+        const int u = (int)threadIdx.x - kPivWarp0 * 32; // pivot rows u, u + 64, u + 128, u + 192
+        Ring ring(p.n_st);
+        uint32_t n = 0;
+        bool dead = false; // warp-uniform
+        for (uint32_t g = blockIdx.x; !dead && g < total; g += gridDim.x) {
+            float pq[kMaxN / kPivThreads][2]; // sums of squares only
+#pragma unroll
+            for (int k = 0; k < kMaxN / kPivThreads; ++k) pq[k][0] = pq[k][1] = 0.f;
+            for (int a = 0; a < na; a += p.aps) {
+                dead = !ctl.wait_bar(smem_u32(&sh.full[ring.stage]), ring.phase, kWaitStageNorm, g);
+                dead = __any_sync(0xffffffffu, dead);
+                if (dead) break;
+                for (int h = 0; h < min(p.aps, na - a); ++h)
+#pragma unroll
+                    for (int k = 0; k < kMaxN / kPivThreads; ++k)
+                        if (u + kPivThreads * k < p.P) {
+                            float x0 = 0.f, x1 = 0.f;
+                            add_row(b_addr(ring.stage, h), u + kPivThreads * k, x0, x1, pq[k][0], pq[k][1]);
+                        }
+                __syncwarp(); // the warp's reads of the stage are done
+                if (lane == 0) mbar_arrive(smem_u32(&sh.empty[ring.stage]));
+                ring.advance();
+            }
+            if (dead) break;
+            const uint32_t acc = n & 1u;
+            dead = !ctl.wait_bar(smem_u32(&sh.norm_empty[acc]), ((n >> 1) & 1u) ^ 1u, kWaitNormFree, g);
+            dead = __any_sync(0xffffffffu, dead);
+            if (dead) break;
+#pragma unroll
+            for (int k = 0; k < kMaxN / kPivThreads; ++k)
+                if (u + kPivThreads * k < p.P) sh.piv_ssq[acc][u + kPivThreads * k] = pq[k][0] + pq[k][1];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh.norm_full[acc]));
             ++n;
         }
     } else if (warp >= kEpi0 && warp < kEpi0 + kEpiWarps) {

@@ -41,6 +41,8 @@ SHAPES = [
     (3, 333, 264, 17, 301, 7, 60),       # d not a multiple of 64: staged kernels only
     (2, 700, 4096, 40, 576, 8, 64),      # the LLaVA-1.5 shape
     (1, 3000, 512, 12, 2880, 16, 320),   # the LLaVA-NeXT token count
+    (2, 700, 512, 10, 640, 128, 320),    # many pivots: large pivot tiles, fewer atoms per stage of the one-pass kernel
+    (1, 400, 3584, 0, 333, 40, 100),     # 56 atoms per row, a short last row tile, pivot count not a multiple of 4 x 8
 ]
 
 
