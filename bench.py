@@ -87,7 +87,9 @@ def kernel_bytes_per_launch(name, w, B):
 # DRAM traffic of one launch per sample (dram__bytes_read.sum + dram__bytes_write.sum), from the ncu capture of the
 # sweep workload at batch 32 summarised in profiles/sweep_kernel_sweep_b32.md; traffic is proportional to the batch
 # (every sample is read and written independently), so a launch over B samples moves B times this.
-NCU_TRAFFIC_PER_SAMPLE = {("sweep", 2880, 4096, 8): (1.508212e9 + 5.538816e6) / 32}
+NCU_TRAFFIC_PER_SAMPLE = {("sweep", 2880, 4096, 8): (1.508212e9 + 5.538816e6) / 32,
+                          # profiles/onepass_kernel_sweep_b32.md
+                          ("onepass", 2880, 4096, 8): (755.18336e6 + 5.144064e6) / 32}
 
 
 def measured_peak():
@@ -379,8 +381,10 @@ def main():
         if prof_p.get("onepass", (0, 0))[1]:
             ms_o = prof_p["onepass"][0] / prof_p["onepass"][1]
             gbs_o = kernel_bytes_per_launch("onepass", w, B) / (ms_o * 1e-3) / 1e9
+            tr = NCU_TRAFFIC_PER_SAMPLE.get(("onepass", w.n_vis, w.d, w.n_pivot))
             variants["pivots_given"]["onepass_kernel"] = {"ms_per_launch": ms_o, "achieved_GBps": gbs_o,
-                                                          "frac_of_measured_copy": gbs_o / peak}
+                                                          "frac_of_measured_copy": gbs_o / peak,
+                                                          "traffic": tr * B if tr else None}
         # (c) the key rows of the retained tokens, packed by the list of the last reduction (one KV tensor of one layer)
         packed = torch.empty_like(outs[0])
         st = torch.cuda.current_stream()
