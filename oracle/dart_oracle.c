@@ -347,11 +347,15 @@ int dart_oracle_compact(const uint8_t *keep, const uint16_t *hidden, const int64
  * order is the order of the pivots' turns); the retention step rejects repeated or out-of-range ones.
  * rule: 0 = one threshold per pivot from equal quotas (dart_oracle_retention), 1 = one threshold for all
  * (dart_oracle_retention_global).
+ * cosine_on_hidden: the paper ranks pivots by the K-norm but defines dup on "tokens" (Def. 2) without saying
+ * which tensor represents them.  0: the key rows (one tensor for both); 1: the pivots are still chosen by the
+ * key rows' scores, Eq. 7 is evaluated on the hidden rows.  Then l1_out holds the key rows' L1 scores and
+ * l2_out the HIDDEN rows' Euclidean norms (Eq. 7's denominators).  Ignored when keys is NULL.
  */
 int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const int64_t *pos_in,
                           const int32_t *pivots_in,
                           int B, int S, int d, int vis_offset, int n_vis, int n_pivot, int n_keep,
-                          int norm_kind, int largest, int rule,
+                          int norm_kind, int largest, int rule, int cosine_on_hidden,
                           uint16_t *out_hidden, int32_t *out_idx, int64_t *out_pos,
                           double *l1_out, double *l2_out, int32_t *pivot_out, double *dup_out,
                           uint8_t *keep_out, int32_t *owner_out, double *eps_out,
@@ -364,11 +368,12 @@ int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const in
     const int P = n_pivot, S_out = S - n_vis + n_keep;
     double *l1 = (double *)malloc((size_t)n_vis * sizeof(double));
     double *l2 = (double *)malloc((size_t)n_vis * sizeof(double));
+    double *hl1 = (double *)malloc((size_t)n_vis * sizeof(double));
     double *dup = (double *)malloc((size_t)P * (size_t)n_vis * sizeof(double));
     int32_t *piv = (int32_t *)malloc((size_t)P * sizeof(int32_t));
     uint8_t *keep = (uint8_t *)malloc((size_t)n_vis);
     int rc = ORACLE_OK;
-    if (!l1 || !l2 || !dup || !piv || !keep) rc = ORACLE_ERR_NOMEM;
+    if (!l1 || !l2 || !hl1 || !dup || !piv || !keep) rc = ORACLE_ERR_NOMEM;
     for (int b = 0; b < B && rc == ORACLE_OK; ++b) {
         const uint16_t *h = hidden + (size_t)b * (size_t)S * (size_t)d;
         const uint16_t *k = keys ? keys + (size_t)b * (size_t)S * (size_t)d : h;
@@ -384,7 +389,12 @@ int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const in
             rc = dart_oracle_pivots(norm_kind == 1 ? l1 : l2, n_vis, P, largest, piv, &pgap);
             if (rc) break;
         }
-        rc = dart_oracle_similarity(k, S, d, vis_offset, n_vis, piv, P, l2, dup);
+        if (cosine_on_hidden && keys) {
+            /* the pivots are ranked by the key states, but the tokens that are compared are the hidden states */
+            rc = dart_oracle_scores(h, S, d, vis_offset, n_vis, hl1, l2);
+            if (rc) break;
+        }
+        rc = dart_oracle_similarity((cosine_on_hidden && keys) ? h : k, S, d, vis_offset, n_vis, piv, P, l2, dup);
         if (rc) break;
         rc = (rule == 1 ? dart_oracle_retention_global : dart_oracle_retention)(
             dup, piv, n_vis, P, n_keep, keep, owner_out ? owner_out + (size_t)b * n_vis : NULL,
@@ -408,6 +418,7 @@ int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const in
     }
     free(l1);
     free(l2);
+    free(hl1);
     free(dup);
     free(piv);
     free(keep);
@@ -424,6 +435,6 @@ int dart_oracle_reduce(const uint16_t *hidden, const uint16_t *keys, const int64
                        double *pivot_gap_out, double *retain_gap_out)
 {
     return dart_oracle_reduce_ex(hidden, keys, pos_in, NULL, B, S, d, vis_offset, n_vis, n_pivot, n_keep, norm_kind,
-                                 largest, 0, out_hidden, out_idx, out_pos, l1_out, l2_out, pivot_out, dup_out, keep_out,
+                                 largest, 0, 0, out_hidden, out_idx, out_pos, l1_out, l2_out, pivot_out, dup_out, keep_out,
                                  owner_out, eps_out, pivot_gap_out, retain_gap_out);
 }

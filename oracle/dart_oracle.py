@@ -190,10 +190,11 @@ class OracleResult:
 
 def reduce(hidden, keys, vis_offset: int, n_vis: int, n_pivot: int, n_keep: int,
            pos_in=None, norm_kind: int = 1, largest: bool = True, want_dup: bool = True,
-           want_hidden: bool = True, pivots_in=None, rule: int = 0) -> OracleResult:
+           want_hidden: bool = True, pivots_in=None, rule: int = 0, cosine_on_hidden: bool = False) -> OracleResult:
     """The whole step over a batch.  hidden/keys: [B, S, d] bf16 bits (keys None -> hidden is scored).
     pivots_in: None, or [B, n_pivot] distinct vision-relative indices that replace the pivot step.
-    rule: 0 = per-pivot thresholds from equal quotas, 1 = one threshold for all pivots."""
+    rule: 0 = per-pivot thresholds from equal quotas, 1 = one threshold for all pivots.
+    cosine_on_hidden: pivots by the key rows' scores, Eq. 7 on the hidden rows (then .l2 holds the hidden rows' norms)."""
     h = _u16(hidden)
     B, S, d = h.shape
     k = None if keys is None else _u16(keys)
@@ -218,7 +219,7 @@ def reduce(hidden, keys, vis_offset: int, n_vis: int, n_pivot: int, n_keep: int,
         raise ValueError("pivots_in must be [B, n_pivot]")
     _check(_load().dart_oracle_reduce_ex(
         _p(h, ctypes.c_uint16), _p(k, ctypes.c_uint16), _p(pos, ctypes.c_int64), _p(piv_in, ctypes.c_int32),
-        B, S, d, vis_offset, n_vis, n_pivot, n_keep, norm_kind, int(bool(largest)), int(rule),
+        B, S, d, vis_offset, n_vis, n_pivot, n_keep, norm_kind, int(bool(largest)), int(rule), int(bool(cosine_on_hidden)),
         _p(oh, ctypes.c_uint16), _p(oi, ctypes.c_int32), _p(op, ctypes.c_int64),
         _p(l1, ctypes.c_double), _p(l2, ctypes.c_double), _p(piv, ctypes.c_int32), _p(dup, ctypes.c_double),
         _p(keep, ctypes.c_uint8), _p(owner, ctypes.c_int32), _p(eps, ctypes.c_double),

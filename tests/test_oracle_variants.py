@@ -145,3 +145,35 @@ def test_gather_rows_follows_the_reduction(oracle):
     hb = hb.reshape(B, S, d)
     r = oracle.reduce(hb, None, vo, nv, P, Kp)
     assert np.array_equal(oracle.gather_rows(hb, r.out_idx), r.out_hidden)
+
+
+# ----------------------------------------------------------------------------- Eq. 7 on the hidden rows
+
+def test_cosine_on_hidden_rows_is_the_composition_of_the_steps(oracle):
+    """Pivots ranked by the key rows, dup evaluated on the hidden rows: equal to the step functions composed by
+    hand, to numpy's cosine of the hidden rows, and to the main method when both tensors are the same."""
+    rng = np.random.default_rng(27)
+    B, S, d, vo, nv, P, Kp = 3, 60, 32, 5, 48, 3, 14
+    hb, hv = rand_tokens(rng, B * S, d)
+    kb, _ = rand_tokens(rng, B * S, d)
+    hb, kb, hv = hb.reshape(B, S, d), kb.reshape(B, S, d), hv.reshape(B, S, d)
+    r = oracle.reduce(hb, kb, vo, nv, P, Kp, cosine_on_hidden=True)
+    base = oracle.reduce(hb, kb, vo, nv, P, Kp)
+    assert np.array_equal(r.pivot_idx, base.pivot_idx) and np.array_equal(r.l1, base.l1)   # the ranking is the keys'
+    assert not np.array_equal(r.keep, base.keep)
+    for b in range(B):
+        kl1, _ = oracle.scores(kb[b], vo, nv)
+        piv, _ = oracle.pivots(kl1, P)
+        _, hl2 = oracle.scores(hb[b], vo, nv)
+        dup = oracle.similarity(hb[b], vo, nv, piv, hl2)
+        keep, owner, eps, _ = oracle.retention(dup, piv, Kp)
+        assert np.array_equal(r.pivot_idx[b], piv) and np.array_equal(r.l2[b], hl2)
+        assert np.array_equal(r.dup[b], dup) and np.array_equal(r.keep[b], keep)
+        X = hv[b, vo:vo + nv]
+        Xn = X / np.linalg.norm(X, axis=1, keepdims=True)
+        assert np.allclose(r.dup[b], Xn[piv] @ Xn.T, rtol=0, atol=1e-12)                    # an independent routine
+    same = oracle.reduce(hb, hb, vo, nv, P, Kp, cosine_on_hidden=True)                      # one tensor: nothing changes
+    plain = oracle.reduce(hb, hb, vo, nv, P, Kp)
+    assert np.array_equal(same.out_idx, plain.out_idx) and np.array_equal(same.dup, plain.dup)
+    none = oracle.reduce(hb, None, vo, nv, P, Kp, cosine_on_hidden=True)                    # keys = None: likewise
+    assert np.array_equal(none.out_idx, plain.out_idx)
