@@ -93,6 +93,12 @@ typedef struct {
                                      its bounded waits expire and the call ends with DART_ERR_TIMEOUT in dart_status */
     int32_t retention;     /* DART_RETAIN_*: how step 4 is scheduled (same result either way) */
     int32_t rule;          /* DART_RULE_*: which tokens step 4 retains */
+    int32_t cosine_on_hidden; /* 0: Eq. 7 on the key rows that are scored (one tensor for steps 1-3).  1: the pivots are still
+                              ranked by the key rows' L1 scores, but dup(p_i, x_j) is the cosine of the HIDDEN rows (Def. 2
+                              speaks of "tokens" without naming the tensor): the keys are read once for the scores, the
+                              hidden states once for the similarities.  Needs norm_kind 0/1 (else UNSUPPORTED); no effect
+                              when keys is NULL.  dbg->l1 then holds the key rows' scores, dbg->ssq the hidden rows' sums
+                              of squares. */
     const int32_t *pivots_in; /* NULL: pivots by score (steps 1-2).  Else [B, n_pivot] int32, device: the caller's pivots
                               as vision-relative indices, distinct and in [0, n_vis); their order is the order of the
                               pivots' turns in step 4.  This covers the paper's other ways to choose pivots (Sec. 5.2:

@@ -145,9 +145,10 @@ def check_valid_under_tolerance(keys_bits, vis_offset, n_vis, n_keep, pivot_idx,
 
 def check_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, n_vis, n_pivot, n_keep,
                 out_hidden, out_idx, out_pos, dbg=None, pos_in=None, largest=True, norm_kind=1,
-                require_exact_above=MARGIN, pivots_given=False, rule=0) -> ParityReport:
+                require_exact_above=MARGIN, pivots_given=False, rule=0, sim_bits=None) -> ParityReport:
     """All rules over a batch.  ``dbg`` (optional) holds the candidate's per-step outputs as numpy arrays:
-    l1, ssq, pivot_idx, sim, eps, keep, owner.  Without it only the packed outputs are checked."""
+    l1, ssq, pivot_idx, sim, eps, keep, owner.  Without it only the packed outputs are checked.
+    ``sim_bits``: the tensor Eq. 7 is evaluated on when it is not the scored one (cosine on the hidden rows)."""
     B = out_idx.shape[0]
     rep = ParityReport()
     margin = ora.margin
@@ -184,7 +185,8 @@ def check_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, n_vis,
             e = dbg["eps"][b].astype(np.float64)
             assert np.all(np.isnan(e[~has])) and np.all(np.abs(e[has] - ora.eps[b][has]) <= REL_TOL * np.abs(ora.eps[b][has]) + SIM_ABS_FLOOR)
         else:
-            check_valid_under_tolerance(keys_bits[b], vis_offset, n_vis, n_keep, dbg["pivot_idx"][b], dbg["owner"][b],
+            check_valid_under_tolerance(keys_bits[b] if sim_bits is None else sim_bits[b], vis_offset, n_vis, n_keep,
+                                        dbg["pivot_idx"][b], dbg["owner"][b],
                                         ora.l1[b] if norm_kind == 1 else ora.l2[b], ora.l2[b], largest=largest,
                                         pivots_given=pivots_given, rule=rule)
             if not same:

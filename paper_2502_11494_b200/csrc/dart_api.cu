@@ -381,16 +381,15 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     return copy_debug(ctx, B, n_vis, P, dbg, st);
 }
 
-// The caller's pivots: scores and similarities from one read of the keys (csrc/dart_onepass.cuh), then steps 4-5.
-int launch_onepass(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, const int64_t *pos_in, int vis_offset,
-                   int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos, const dart_opts &o,
-                   const dart_debug *dbg, cudaStream_t st)
+// One pass over `src` (csrc/dart_onepass.cuh) with the pivots already in the workspace: sums of squares of src's rows
+// (and their L1 scores unless `scores_elsewhere`: then the scores came from another tensor) and the similarities.
+int launch_onepass_kernel(dart_ctx *ctx, int B, const void *src, bool scores_elsewhere, int vis_offset, int n_vis, int P,
+                          const dart_opts &o, cudaStream_t st)
 {
     using namespace dart;
     using sweep::kSubRows;
     using sweep::kTileRows;
-    const int S = ctx->S, d8 = ctx->desc.d / 8, S_out = S - n_vis + n_keep;
-    const void *keys = keys_in ? keys_in : hidden;
+    const int S = ctx->S;
     onepass::Params p = {};
     p.B = B, p.S = S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.N = (P + 15) / 16 * 16;
     p.n_atoms = ctx->n_atoms, p.n_rt = (n_vis + kTileRows - 1) / kTileRows;
@@ -398,28 +397,87 @@ int launch_onepass(dart_ctx *ctx, int B, const void *hidden, const void *keys_in
     p.n_st = onepass::ring_depth(p.N, p.aps, ctx->max_smem_optin);
     if (p.n_st < 2) return DART_ERR_UNSUPPORTED;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
-    p.sim = ctx->sim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
+    p.sim = ctx->sim, p.l1 = scores_elsewhere ? nullptr : ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
     p.status = ctx->status;
     CUtensorMap tm_tile, tm_keys, tm_row;
-    int rc = encode_2d(ctx, &tm_tile, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, kTileRows);
-    if (rc == DART_OK) rc = encode_2d(ctx, &tm_keys, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, kSubRows);
-    if (rc == DART_OK) rc = encode_2d(ctx, &tm_row, keys, (uint64_t)ctx->desc.d, (uint64_t)B * S, 1);
+    int rc = encode_2d(ctx, &tm_tile, src, (uint64_t)ctx->desc.d, (uint64_t)B * S, kTileRows);
+    if (rc == DART_OK) rc = encode_2d(ctx, &tm_keys, src, (uint64_t)ctx->desc.d, (uint64_t)B * S, kSubRows);
+    if (rc == DART_OK) rc = encode_2d(ctx, &tm_row, src, (uint64_t)ctx->desc.d, (uint64_t)B * S, 1);
     if (rc != DART_OK) return rc;
+    Prof pr(ctx, st, SLOT_ONEPASS);
+    const long long tasks = (long long)B * p.n_rt;
+    const unsigned grid = (unsigned)(tasks < ctx->sm_count ? tasks : ctx->sm_count); // no CTA waits for another
+    onepass::onepass_kernel<<<grid, onepass::kThreads, onepass::smem_bytes(p.N, p.aps, p.n_st), st>>>(tm_tile, tm_keys, tm_row, p);
+    return DART_OK;
+}
+
+void launch_gather(dart_ctx *ctx, int B, const void *hidden, int n_vis, int n_keep, const int32_t *out_idx, void *out_hidden,
+                   cudaStream_t st)
+{
+    using namespace dart;
+    const int S = ctx->S, d8 = ctx->desc.d / 8, S_out = S - n_vis + n_keep;
+    Prof pr(ctx, st, SLOT_GATHER);
+    const long long orows = (long long)B * S_out;
+    const unsigned grid = (unsigned)((orows + kGatherWarps - 1) / kGatherWarps);
+    gather_kernel<<<grid, kGatherWarps * 32, 0, st>>>((const uint4 *)hidden, out_idx, S, S_out, d8, orows, ctx->status,
+                                                     (uint4 *)out_hidden);
+}
+
+// The caller's pivots: scores and similarities from one read of the keys, then steps 4-5.
+int launch_onepass(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, const int64_t *pos_in, int vis_offset,
+                   int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos, const dart_opts &o,
+                   const dart_debug *dbg, cudaStream_t st)
+{
     launch_pivots_given(ctx, B, n_vis, P, o.pivots_in, st);
+    int rc = launch_onepass_kernel(ctx, B, keys_in ? keys_in : hidden, false, vis_offset, n_vis, P, o, st);
+    if (rc != DART_OK) return rc;
+    launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
+    launch_gather(ctx, B, hidden, n_vis, n_keep, out_idx, out_hidden, st);
+    DART_CUDA(ctx, cudaGetLastError());
+    return copy_debug(ctx, B, n_vis, P, dbg, st);
+}
+
+// dart_opts.cosine_on_hidden with distinct tensors: the key rows are read once for the L1 scores that rank the pivots,
+// the hidden rows once for their norms and the similarities (one pass when the tensor-core kernels apply, else the
+// plain kernels: norms, then similarities).
+int launch_hidden_cosine(dart_ctx *ctx, int B, const void *hidden, const void *keys, const int64_t *pos_in, int vis_offset,
+                         int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos,
+                         const dart_opts &o, const dart_debug *dbg, bool tensor_cores, cudaStream_t st)
+{
+    using namespace dart;
+    const int S = ctx->S, d8 = ctx->desc.d / 8;
+    const long long rows = (long long)B * n_vis;
+    const unsigned score_grid = (unsigned)((rows + kScoreWarps - 1) / kScoreWarps);
     {
-        Prof pr(ctx, st, SLOT_ONEPASS);
-        const long long tasks = (long long)B * p.n_rt;
-        const unsigned grid = (unsigned)(tasks < ctx->sm_count ? tasks : ctx->sm_count); // no CTA waits for another
-        onepass::onepass_kernel<<<grid, onepass::kThreads, onepass::smem_bytes(p.N, p.aps, p.n_st), st>>>(tm_tile, tm_keys, tm_row, p);
+        Prof p(ctx, st, SLOT_SCORE); // scores of the key rows only
+        score_kernel<<<score_grid, kScoreWarps * 32, 0, st>>>((const uint4 *)keys, S, d8, vis_offset, n_vis, rows, ctx->l1, nullptr);
+    }
+    if (o.pivots_in) {
+        launch_pivots_given(ctx, B, n_vis, P, o.pivots_in, st);
+    } else {
+        Prof p(ctx, st, SLOT_PIVOT);
+        const int P_pad = next_pow2(P);
+        pivot_kernel<<<B, kSelectThreads, (size_t)P_pad * 8, st>>>(ctx->l1, n_vis, P, P_pad, o.pivot_smallest, ctx->pivot_idx);
+    }
+    if (tensor_cores) {
+        int rc = launch_onepass_kernel(ctx, B, hidden, true, vis_offset, n_vis, P, o, st);
+        if (rc != DART_OK) return rc;
+    } else {
+        {
+            Prof p(ctx, st, SLOT_SCORE); // sums of squares of the hidden rows only
+            score_kernel<<<score_grid, kScoreWarps * 32, 0, st>>>((const uint4 *)hidden, S, d8, vis_offset, n_vis, rows, nullptr,
+                                                                 ctx->ssq);
+        }
+        Prof p(ctx, st, SLOT_SIM);
+        const size_t smem = (size_t)kSimPivotChunk * d8 * 16;
+        const dim3 grid((n_vis + kSimRowsPerCta - 1) / kSimRowsPerCta, B);
+        for (int p0 = 0; p0 < P; p0 += kSimPivotChunk)
+            sim_alu_kernel<<<grid, kSimWarps * 32, smem, st>>>((const uint4 *)hidden, S, d8, vis_offset, n_vis, P, p0, ctx->pivot_idx,
+                                                              ctx->ssq, ctx->sim);
+        ctx->launches += (P - 1) / kSimPivotChunk;
     }
     launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
-    {
-        Prof pr(ctx, st, SLOT_GATHER);
-        long long orows = (long long)B * S_out;
-        unsigned grid = (unsigned)((orows + kGatherWarps - 1) / kGatherWarps);
-        gather_kernel<<<grid, kGatherWarps * 32, 0, st>>>((const uint4 *)hidden, out_idx, S, S_out, d8, orows,
-                                                         ctx->status, (uint4 *)out_hidden);
-    }
+    launch_gather(ctx, B, hidden, n_vis, n_keep, out_idx, out_hidden, st);
     DART_CUDA(ctx, cudaGetLastError());
     return copy_debug(ctx, B, n_vis, P, dbg, st);
 }
@@ -430,6 +488,9 @@ int launch_reduce(dart_ctx *ctx, int B, const void *hidden, const void *keys, co
 {
     const bool fused = o.path == DART_PATH_FUSED || (o.path == DART_PATH_AUTO && fused_applies(ctx, P));
     if (fused && !fused_applies(ctx, P)) return DART_ERR_UNSUPPORTED;
+    if (o.cosine_on_hidden && keys && keys != hidden)
+        return launch_hidden_cosine(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o,
+                                    dbg, fused, st);
     if (fused && o.pivots_in) // nothing waits for a selection: one pass over the keys
         return launch_onepass(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o, dbg, st);
     return fused ? launch_fused(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos,
@@ -590,6 +651,7 @@ int dart_reduce_ex(dart_ctx *ctx, const void *hidden, const void *keys, const in
     if (o.norm_kind != 1 && o.norm_kind != 2) return DART_ERR_UNSUPPORTED;
     if (o.path != DART_PATH_AUTO && o.path != DART_PATH_STAGED && o.path != DART_PATH_FUSED) return DART_ERR_UNSUPPORTED;
     if (o.rule != DART_RULE_QUOTAS && o.rule != DART_RULE_GLOBAL) return DART_ERR_UNSUPPORTED;
+    if (o.cosine_on_hidden && o.norm_kind != 1) return DART_ERR_UNSUPPORTED; // the hidden rows' sums of squares take the slot
     if ((uintptr_t)o.pivots_in & 3u) return DART_ERR_ALIGN;
     if (o.rule == DART_RULE_GLOBAL &&
         dart::retain_global_smem_bytes(n_vis) > (size_t)ctx->max_smem_optin - 2048)

@@ -43,7 +43,7 @@ struct Params {
     int n_st, aps;                     // ring depth; atoms per stage (<= kMaxAtomsPerStage)
     unsigned long long wait_ns;
     float *sim;                        // [B][P][n_vis] dup(p_i, x_j)
-    float *l1, *ssq;                   // [B][n_vis]
+    float *l1, *ssq;                   // [B][n_vis]; l1 may be NULL (the scores come from another tensor)
     const int32_t *pivot_idx;          // [B][P], checked and clamped
     int *status;
 };
@@ -266,7 +266,7 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
             sh.row_ssq[acc][t] = t < rows ? q : 0.f;
             if (t < rows) {
                 const size_t o = (size_t)b * p.n_vis + rt * kTileRows + t;
-                p.l1[o] = a0 + a1;
+                if (p.l1) p.l1[o] = a0 + a1;
                 p.ssq[o] = q;
             }
             __syncwarp();

@@ -45,9 +45,9 @@ score_kernel(const uint4 *__restrict__ keys, int S, int d8, int vis_offset, int 
     }
     a = warp_sum(a);
     q = warp_sum(q);
-    if (lane == 0) {
-        l1[row] = a;
-        ssq[row] = q;
+    if (lane == 0) { // either output may be NULL (not wanted)
+        if (l1) l1[row] = a;
+        if (ssq) ssq[row] = q;
     }
 }
 

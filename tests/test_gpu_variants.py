@@ -14,13 +14,14 @@ from test_gpu_parity import PATH_IDS, PATHS, _np, gaussian  # noqa: E402
 pytestmark = pytest.mark.gpu
 
 
-def run(keys, hidden, vo, nv, P, Kp, path, pivots=None, rule=dart.DART_RULE_QUOTAS, expect_status=dart.DART_OK):
+def run(keys, hidden, vo, nv, P, Kp, path, pivots=None, rule=dart.DART_RULE_QUOTAS, expect_status=dart.DART_OK,
+        on_hidden=False):
     B, S, d = hidden.shape
     if path == dart.DART_PATH_FUSED and (d % 64 or P > 256):
         pytest.skip("the fused path needs d % 64 == 0 and at most 256 pivots")
     ctx = dart.Dart(B, S, d, P, Kp)
     try:
-        opts = dart.dart_opts(0, 0, path, 0, 0, 0, 0, rule, None if pivots is None else pivots.data_ptr())
+        opts = dart.dart_opts(0, 0, path, 0, 0, 0, 0, rule, int(on_hidden), None if pivots is None else pivots.data_ptr())
         res = ctx.reduce(hidden, keys, vo, nv, P, Kp, opts=opts, debug=True)
         torch.cuda.synchronize()
         st = ctx.status()
@@ -124,11 +125,45 @@ def test_both_variants_together(oracle):
     assert rep.exact >= rep.above_margin
 
 
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_cosine_on_the_hidden_rows(oracle, shape, path):
+    """Pivots ranked by the key rows, Eq. 7 evaluated on the hidden rows."""
+    B, S, d, vo, nv, P, Kp = shape
+    k, h = gaussian(B, S, d, seed=300 + sum(shape))
+    oh, oi, op, dbg, _ = run(k, h, vo, nv, P, Kp, path, on_hidden=True)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, cosine_on_hidden=True)
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, dbg=dbg, sim_bits=hb)
+    assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5 and rep.max_rel_l1 < 5e-5 and rep.max_rel_l2 < 5e-5
+
+
+def test_cosine_on_hidden_with_given_pivots_and_one_threshold(oracle):
+    B, S, d, vo, nv, P, Kp = 2, 400, 256, 10, 380, 8, 70
+    k, h = gaussian(B, S, d, seed=51)
+    piv = random_pivots(B, nv, P, seed=52)
+    oh, oi, op, dbg, _ = run(k, h, vo, nv, P, Kp, dart.DART_PATH_AUTO, pivots=torch.from_numpy(piv).cuda(),
+                             rule=dart.DART_RULE_GLOBAL, on_hidden=True)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=piv, rule=1, cosine_on_hidden=True)
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, dbg=dbg, pivots_given=True, rule=1, sim_bits=hb)
+    assert rep.exact >= rep.above_margin
+
+
+def test_cosine_on_hidden_needs_the_l1_score():
+    k, h = gaussian(1, 64, 64, seed=53)
+    ctx = dart.Dart(1, 64, 64, 2, 8)
+    with pytest.raises(dart.DartError) as e:
+        ctx.reduce(h, k, 0, 64, 2, 8, opts=dart.dart_opts(2, 0, 0, 0, 0, 0, 0, 0, 1, None))
+    assert e.value.code == dart.DART_ERR_UNSUPPORTED
+    ctx.close()
+
+
 def test_unknown_rule_is_rejected():
     k, h = gaussian(1, 64, 64, seed=43)
     ctx = dart.Dart(1, 64, 64, 2, 8)
     with pytest.raises(dart.DartError) as e:
-        ctx.reduce(h, k, 0, 64, 2, 8, opts=dart.dart_opts(0, 0, 0, 0, 0, 0, 0, 7, None))
+        ctx.reduce(h, k, 0, 64, 2, 8, opts=dart.dart_opts(0, 0, 0, 0, 0, 0, 0, 7, 0, None))
     assert e.value.code == dart.DART_ERR_UNSUPPORTED
     ctx.close()
 
