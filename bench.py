@@ -40,7 +40,7 @@ def parse():
     ap.add_argument("--keep", type=int, default=None)
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch size")
     ap.add_argument("--sweep", action="store_true", help="also time every (pivots, keep) cell of the sweep")
-    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 staged, 2 fused")
+    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 staged, 2 fused (persistent sweep), 3 two passes (score pass + one tensor-core pass)")
     ap.add_argument("--lag", type=int, default=0, help="fused path: extra tasks between a row's two sweeps")
     ap.add_argument("--retention", type=int, default=0, help="0 auto, 1 one kernel, 2 candidate lists + walks")
     ap.add_argument("--variants", action="store_true",

@@ -55,6 +55,9 @@ enum {
 #define DART_PATH_FUSED 2  /* persistent sweep kernel (scores, pivots and similarities in one launch; with the caller's
                               pivots: scores and similarities from one pass over the keys); needs d % 64 == 0 and
                               n_pivot <= 256, else UNSUPPORTED.  AUTO picks it when it applies. */
+#define DART_PATH_TWO_PASS 3 /* two launches instead of the persistent sweep: a plain score pass, pivot selection, then
+                              scores' sums of squares and similarities from one tensor-core pass; same limits as FUSED.
+                              Reads the keys twice like FUSED but has no waits between CTAs: faster for small batches. */
 
 /* dart_opts.retention */
 #define DART_RETAIN_AUTO 0   /* two phases when the batch alone cannot fill the GPU, else one kernel */

@@ -437,43 +437,47 @@ int launch_onepass(dart_ctx *ctx, int B, const void *hidden, const void *keys_in
     return copy_debug(ctx, B, n_vis, P, dbg, st);
 }
 
-// dart_opts.cosine_on_hidden with distinct tensors: the key rows are read once for the L1 scores that rank the pivots,
-// the hidden rows once for their norms and the similarities (one pass when the tensor-core kernels apply, else the
-// plain kernels: norms, then similarities).
-int launch_hidden_cosine(dart_ctx *ctx, int B, const void *hidden, const void *keys, const int64_t *pos_in, int vis_offset,
-                         int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos,
-                         const dart_opts &o, const dart_debug *dbg, bool tensor_cores, cudaStream_t st)
+// Two plain passes: the rows of `keys` are read once for the scores that rank the pivots, the rows of `sim_src` once for
+// their norms and the similarities (one pass when the tensor-core kernels apply, else the plain kernels: norms, then
+// similarities).  sim_src = hidden is dart_opts.cosine_on_hidden; sim_src = keys is the main method without the
+// persistent sweep: no launch waits inside for another CTA, which is what small batches want.
+int launch_two_pass(dart_ctx *ctx, int B, const void *hidden, const void *keys, const void *sim_src, const int64_t *pos_in,
+                    int vis_offset, int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos,
+                    const dart_opts &o, const dart_debug *dbg, bool tensor_cores, cudaStream_t st)
 {
     using namespace dart;
     const int S = ctx->S, d8 = ctx->desc.d / 8;
     const long long rows = (long long)B * n_vis;
     const unsigned score_grid = (unsigned)((rows + kScoreWarps - 1) / kScoreWarps);
+    const bool same = sim_src == keys;
     {
-        Prof p(ctx, st, SLOT_SCORE); // scores of the key rows only
-        score_kernel<<<score_grid, kScoreWarps * 32, 0, st>>>((const uint4 *)keys, S, d8, vis_offset, n_vis, rows, ctx->l1, nullptr);
+        Prof p(ctx, st, SLOT_SCORE); // the key rows' scores (their sums of squares too when they rank the pivots)
+        score_kernel<<<score_grid, kScoreWarps * 32, 0, st>>>((const uint4 *)keys, S, d8, vis_offset, n_vis, rows, ctx->l1,
+                                                             (same && (o.norm_kind == 2 || !tensor_cores)) ? ctx->ssq : nullptr);
     }
     if (o.pivots_in) {
         launch_pivots_given(ctx, B, n_vis, P, o.pivots_in, st);
     } else {
         Prof p(ctx, st, SLOT_PIVOT);
         const int P_pad = next_pow2(P);
-        pivot_kernel<<<B, kSelectThreads, (size_t)P_pad * 8, st>>>(ctx->l1, n_vis, P, P_pad, o.pivot_smallest, ctx->pivot_idx);
+        pivot_kernel<<<B, kSelectThreads, (size_t)P_pad * 8, st>>>(o.norm_kind == 2 ? ctx->ssq : ctx->l1, n_vis, P, P_pad,
+                                                                  o.pivot_smallest, ctx->pivot_idx);
     }
     if (tensor_cores) {
-        int rc = launch_onepass_kernel(ctx, B, hidden, true, vis_offset, n_vis, P, o, st);
+        int rc = launch_onepass_kernel(ctx, B, sim_src, true, vis_offset, n_vis, P, o, st);
         if (rc != DART_OK) return rc;
     } else {
-        {
+        if (!same) {
             Prof p(ctx, st, SLOT_SCORE); // sums of squares of the hidden rows only
-            score_kernel<<<score_grid, kScoreWarps * 32, 0, st>>>((const uint4 *)hidden, S, d8, vis_offset, n_vis, rows, nullptr,
+            score_kernel<<<score_grid, kScoreWarps * 32, 0, st>>>((const uint4 *)sim_src, S, d8, vis_offset, n_vis, rows, nullptr,
                                                                  ctx->ssq);
         }
         Prof p(ctx, st, SLOT_SIM);
         const size_t smem = (size_t)kSimPivotChunk * d8 * 16;
         const dim3 grid((n_vis + kSimRowsPerCta - 1) / kSimRowsPerCta, B);
         for (int p0 = 0; p0 < P; p0 += kSimPivotChunk)
-            sim_alu_kernel<<<grid, kSimWarps * 32, smem, st>>>((const uint4 *)hidden, S, d8, vis_offset, n_vis, P, p0, ctx->pivot_idx,
-                                                              ctx->ssq, ctx->sim);
+            sim_alu_kernel<<<grid, kSimWarps * 32, smem, st>>>((const uint4 *)sim_src, S, d8, vis_offset, n_vis, P, p0,
+                                                              ctx->pivot_idx, ctx->ssq, ctx->sim);
         ctx->launches += (P - 1) / kSimPivotChunk;
     }
     launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
@@ -489,8 +493,19 @@ int launch_reduce(dart_ctx *ctx, int B, const void *hidden, const void *keys, co
     const bool fused = o.path == DART_PATH_FUSED || (o.path == DART_PATH_AUTO && fused_applies(ctx, P));
     if (fused && !fused_applies(ctx, P)) return DART_ERR_UNSUPPORTED;
     if (o.cosine_on_hidden && keys && keys != hidden)
-        return launch_hidden_cosine(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o,
-                                    dbg, fused, st);
+        return launch_two_pass(ctx, B, hidden, keys, hidden, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o,
+                               dbg, fused, st);
+    // AUTO: the persistent sweep selects pivots from a shared-memory copy of a sample's scores; samples with more vision
+    // tokens than that holds select from global memory and stall the sweep (measured at 4608 tokens, batch 4: 253 us
+    // against 111 us for the three launches below)
+    const bool two_pass = o.path == DART_PATH_TWO_PASS ||
+                          (o.path == DART_PATH_AUTO && fused_applies(ctx, P) && n_vis > dart::sweep::kSelMax && !o.pivots_in);
+    if (two_pass) {
+        if (!fused_applies(ctx, P)) return DART_ERR_UNSUPPORTED;
+        const void *k = keys ? keys : hidden;
+        return launch_two_pass(ctx, B, hidden, k, k, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o, dbg,
+                               true, st);
+    }
     if (fused && o.pivots_in) // nothing waits for a selection: one pass over the keys
         return launch_onepass(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o, dbg, st);
     return fused ? launch_fused(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos,
@@ -649,7 +664,8 @@ int dart_reduce_ex(dart_ctx *ctx, const void *hidden, const void *keys, const in
     if (opts) o = *opts;
     if (o.norm_kind == 0) o.norm_kind = 1;
     if (o.norm_kind != 1 && o.norm_kind != 2) return DART_ERR_UNSUPPORTED;
-    if (o.path != DART_PATH_AUTO && o.path != DART_PATH_STAGED && o.path != DART_PATH_FUSED) return DART_ERR_UNSUPPORTED;
+    if (o.path != DART_PATH_AUTO && o.path != DART_PATH_STAGED && o.path != DART_PATH_FUSED && o.path != DART_PATH_TWO_PASS)
+        return DART_ERR_UNSUPPORTED;
     if (o.rule != DART_RULE_QUOTAS && o.rule != DART_RULE_GLOBAL) return DART_ERR_UNSUPPORTED;
     if (o.cosine_on_hidden && o.norm_kind != 1) return DART_ERR_UNSUPPORTED; // the hidden rows' sums of squares take the slot
     if ((uintptr_t)o.pivots_in & 3u) return DART_ERR_ALIGN;

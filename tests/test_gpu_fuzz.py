@@ -22,7 +22,7 @@ def random_case(seed):
     Kp = int(rng.integers(P, n_vis + 1))
     B = int(rng.integers(1, 5))
     return dict(B=B, S=before + n_vis + after, d=d, vo=before, nv=n_vis, P=P, Kp=Kp,
-                path=int(rng.choice([dart.DART_PATH_STAGED, dart.DART_PATH_FUSED])),
+                path=int(rng.choice([dart.DART_PATH_STAGED, dart.DART_PATH_FUSED, dart.DART_PATH_TWO_PASS])),
                 norm_kind=int(rng.choice([1, 2])), smallest=int(rng.integers(0, 2)),
                 retention=int(rng.integers(0, 3)), rule=int(rng.integers(0, 2)),
                 given=bool(rng.integers(0, 2)), on_hidden=bool(rng.integers(0, 2)), keys_null=bool(rng.integers(0, 4) == 0))
@@ -31,7 +31,7 @@ def random_case(seed):
 @pytest.mark.parametrize("seed", range(40))
 def test_random_shapes_and_options(oracle, seed):
     c = random_case(seed)
-    if c["path"] == dart.DART_PATH_FUSED and c["d"] % 64:
+    if c["path"] != dart.DART_PATH_STAGED and c["d"] % 64:
         c["path"] = dart.DART_PATH_STAGED
     if c["on_hidden"]:
         c["norm_kind"] = 1

@@ -11,8 +11,8 @@ from paper_2502_11494_b200 import dart, workloads as W  # noqa: E402
 
 pytestmark = pytest.mark.gpu
 
-PATHS = [dart.DART_PATH_STAGED, dart.DART_PATH_FUSED]
-PATH_IDS = {dart.DART_PATH_STAGED: "staged", dart.DART_PATH_FUSED: "fused"}
+PATHS = [dart.DART_PATH_STAGED, dart.DART_PATH_FUSED, dart.DART_PATH_TWO_PASS]
+PATH_IDS = {dart.DART_PATH_STAGED: "staged", dart.DART_PATH_FUSED: "fused", dart.DART_PATH_TWO_PASS: "two-pass"}
 
 
 def _np(t):
@@ -23,8 +23,8 @@ def _np(t):
 def run_gpu(keys, hidden, vo, nv, P, Kp, pos_in=None, path=dart.DART_PATH_AUTO, norm_kind=0, smallest=0, debug=True,
             sweep_lag=0, retention=dart.DART_RETAIN_AUTO):
     B, S, d = hidden.shape
-    if path == dart.DART_PATH_FUSED and (d % 64 or P > 256):
-        pytest.skip("the fused path needs d % 64 == 0 and at most 256 pivots")
+    if path in (dart.DART_PATH_FUSED, dart.DART_PATH_TWO_PASS) and (d % 64 or P > 256):
+        pytest.skip("the tensor-core paths need d % 64 == 0 and at most 256 pivots")
     ctx = dart.Dart(B, S, d, P, Kp)
     try:
         opts = dart.dart_opts(norm_kind, smallest, path, 0, sweep_lag, 0, retention)

@@ -17,8 +17,8 @@ pytestmark = pytest.mark.gpu
 def run(keys, hidden, vo, nv, P, Kp, path, pivots=None, rule=dart.DART_RULE_QUOTAS, expect_status=dart.DART_OK,
         on_hidden=False):
     B, S, d = hidden.shape
-    if path == dart.DART_PATH_FUSED and (d % 64 or P > 256):
-        pytest.skip("the fused path needs d % 64 == 0 and at most 256 pivots")
+    if path in (dart.DART_PATH_FUSED, dart.DART_PATH_TWO_PASS) and (d % 64 or P > 256):
+        pytest.skip("the tensor-core paths need d % 64 == 0 and at most 256 pivots")
     ctx = dart.Dart(B, S, d, P, Kp)
     try:
         opts = dart.dart_opts(0, 0, path, 0, 0, 0, 0, rule, int(on_hidden), None if pivots is None else pivots.data_ptr())
