@@ -36,6 +36,7 @@ struct dart_ctx {
     // workspace (device), indexed with the shapes of the current call
     float *l1, *ssq, *sim, *eps;
     int32_t *pivot_idx, *owner;
+    void *piv_rows;  // [B_max][P_max rounded to 16][d] bf16: compact copy of the pivot rows (NULL: not available)
     int32_t *cand;   // [B_max][P_max][cand_stride] sorted candidate lists of the two-phase retention (NULL: not available)
     int cand_stride;
     uint8_t *keep;
@@ -399,15 +400,25 @@ int launch_onepass_kernel(dart_ctx *ctx, int B, const void *src, bool scores_els
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
     p.sim = ctx->sim, p.l1 = scores_elsewhere ? nullptr : ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
     p.status = ctx->status;
-    CUtensorMap tm_tile, tm_keys, tm_row;
+    p.compact = ctx->piv_rows != nullptr && P > onepass::kGatherMaxP;
+    CUtensorMap tm_tile, tm_keys, tm_row, tm_piv;
     int rc = encode_2d(ctx, &tm_tile, src, (uint64_t)ctx->desc.d, (uint64_t)B * S, kTileRows);
     if (rc == DART_OK) rc = encode_2d(ctx, &tm_keys, src, (uint64_t)ctx->desc.d, (uint64_t)B * S, kSubRows);
     if (rc == DART_OK) rc = encode_2d(ctx, &tm_row, src, (uint64_t)ctx->desc.d, (uint64_t)B * S, 1);
+    if (rc == DART_OK)
+        rc = p.compact ? encode_2d(ctx, &tm_piv, ctx->piv_rows, (uint64_t)ctx->desc.d, (uint64_t)B * p.N, (uint32_t)p.N)
+                       : encode_2d(ctx, &tm_piv, src, (uint64_t)ctx->desc.d, (uint64_t)B * S, 1); // unused
     if (rc != DART_OK) return rc;
+    if (p.compact) { // the sample's pivot rows side by side, so that a pivot tile is one box
+        Prof pc(ctx, st, SLOT_PIVOT);
+        const long long prow = (long long)B * p.N;
+        pivot_rows_kernel<<<(unsigned)((prow + kPivotRowWarps - 1) / kPivotRowWarps), kPivotRowWarps * 32, 0, st>>>(
+            (const uint4 *)src, ctx->pivot_idx, S, ctx->desc.d / 8, vis_offset, n_vis, P, p.N, prow, (uint4 *)ctx->piv_rows);
+    }
     Prof pr(ctx, st, SLOT_ONEPASS);
     const long long tasks = (long long)B * p.n_rt;
     const unsigned grid = (unsigned)(tasks < ctx->sm_count ? tasks : ctx->sm_count); // no CTA waits for another
-    onepass::onepass_kernel<<<grid, onepass::kThreads, onepass::smem_bytes(p.N, p.aps, p.n_st), st>>>(tm_tile, tm_keys, tm_row, p);
+    onepass::onepass_kernel<<<grid, onepass::kThreads, onepass::smem_bytes(p.N, p.aps, p.n_st), st>>>(tm_tile, tm_keys, tm_row, tm_piv, p);
     return DART_OK;
 }
 
@@ -495,11 +506,14 @@ int launch_reduce(dart_ctx *ctx, int B, const void *hidden, const void *keys, co
     if (o.cosine_on_hidden && keys && keys != hidden)
         return launch_two_pass(ctx, B, hidden, keys, hidden, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o,
                                dbg, fused, st);
-    // AUTO: the persistent sweep selects pivots from a shared-memory copy of a sample's scores; samples with more vision
-    // tokens than that holds select from global memory and stall the sweep (measured at 4608 tokens, batch 4: 253 us
-    // against 111 us for the three launches below)
+    // AUTO prefers the three launches below to the persistent sweep in two cases.  (1) Samples with more vision tokens
+    // than the sweep's shared-memory score buffer holds: it then selects from global memory and stalls (measured at
+    // 4608 tokens, batch 4: 253 us against 111 us).  (2) 32 pivots or more: the sweep fetches pivot tiles four rows per
+    // TMA op, the one-pass kernel as one box from a compact copy (batch 256: 32 pivots 2.83 -> 2.71 ms, 128 pivots
+    // 6.15 -> 4.65 ms; at 16 pivots the sweep is still ahead, 2.33 against 2.40 ms).
     const bool two_pass = o.path == DART_PATH_TWO_PASS ||
-                          (o.path == DART_PATH_AUTO && fused_applies(ctx, P) && n_vis > dart::sweep::kSelMax && !o.pivots_in);
+                          (o.path == DART_PATH_AUTO && fused_applies(ctx, P) && !o.pivots_in &&
+                           (n_vis > dart::sweep::kSelMax || (P >= 32 && ctx->piv_rows)));
     if (two_pass) {
         if (!fused_applies(ctx, P)) return DART_ERR_UNSUPPORTED;
         const void *k = keys ? keys : hidden;
@@ -552,6 +566,11 @@ int dart_create(dart_ctx **out, const dart_desc *desc)
         ctx->cand_stride = desc->Kp_max < dart::kCandMax ? desc->Kp_max : dart::kCandMax;
         const size_t entries = np * (size_t)ctx->cand_stride;
         if (entries * sizeof(int32_t) <= ((size_t)1 << 30)) rc = ws_alloc(ctx, &ctx->cand, entries);
+    }
+    if (rc == DART_OK && desc->P_max > dart::onepass::kGatherMaxP) {
+        // compact pivot rows for the one-pass kernel at many pivots; contexts that would need more than 2 GiB go without
+        const size_t bytes = (size_t)desc->B_max * ((desc->P_max + 15) / 16 * 16) * desc->d * 2;
+        if (bytes <= ((size_t)2 << 30)) rc = ws_alloc(ctx, (uint8_t **)&ctx->piv_rows, bytes);
     }
     if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->status, 64);
     if (rc == DART_OK && cudaMemset(ctx->status, 0, 256) != cudaSuccess) rc = DART_ERR_CUDA;
@@ -626,6 +645,7 @@ int dart_destroy(dart_ctx *ctx)
     cudaFree(ctx->owner);
     cudaFree(ctx->keep);
     cudaFree(ctx->cand);
+    cudaFree(ctx->piv_rows);
     cudaFree(ctx->status);
     cudaFree(ctx->counters);
     for (int k = 0; k < 2; ++k) {

@@ -10,8 +10,10 @@
 // dealt out round-robin to a persistent grid of one CTA per SM.
 //
 // Per CTA (384 threads):
-//   warp 0     producer: per 64-column atom one 128-row TMA tile (128-byte swizzle) and the pivot rows by
-//              tile::gather4, up to four atoms per stage of a ring
+//   warp 0     producer: per 64-column atom one 128-row TMA tile (128-byte swizzle) and the pivot rows - by
+//              tile::gather4 straight from the key tensor (4 rows per op: fine for a few pivots), or as ONE box from
+//              a compact copy of the sample's pivot rows (many pivots: gather4 ops would bound the kernel) -
+//              up to four atoms per stage of a ring
 //   warp 1     one thread issues tcgen05.mma; tcgen05.commit releases the stage on the tensor cores' behalf
 //   warps 4-7  norms: thread t owns tile row t and sums its 128 bytes of every atom, in column order whatever
 //              the swizzle did to the chunks, so a row's norm does not depend on where in a tile it was read
@@ -34,6 +36,7 @@ constexpr int kEpi0 = 8;          // kEpi0 % 4 == 0: warp w reads TMEM lanes 32 
 constexpr int kStages = 10;       // at most
 constexpr int kMaxAtomsPerStage = 4; // a stage holds up to four 64-column atoms: the producer's issue latency (wait, expect,
                                      // issue: ~0.3 us) is paid per stage; measured at 8 pivots: 1 atom 1.40 ms, 2 1.14, 4 1.02
+constexpr int kGatherMaxP = 8;    // up to this many pivots the pivot rows come by gather4 (two ops per atom)
 constexpr int kStaticSmemReserve = 8192;
 enum { kWaitStageFree = 64, kWaitStageMma, kWaitStageNorm, kWaitAccumFree1, kWaitAccumFull1, kWaitNormFree, kWaitNormFull };
 
@@ -41,6 +44,7 @@ struct Params {
     int B, S, vis_offset, n_vis, P, N; // N = P rounded up to a multiple of 16 (MMA N)
     int n_atoms, n_rt;                 // 64-column atoms per row; row tiles per sample
     int n_st, aps;                     // ring depth; atoms per stage (<= kMaxAtomsPerStage)
+    int compact;                       // pivot tiles come from the compact copy [B][N][d] (tm_piv), not by gather4
     unsigned long long wait_ns;
     float *sim;                        // [B][P][n_vis] dup(p_i, x_j)
     float *l1, *ssq;                   // [B][n_vis]; l1 may be NULL (the scores come from another tensor)
@@ -96,7 +100,7 @@ __device__ __forceinline__ void add_row(uint32_t tile, int r, float &a0, float &
 
 __global__ void __launch_bounds__(kThreads, 1)
 onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant__ CUtensorMap tm_keys,
-               const __grid_constant__ CUtensorMap tm_row, const Params p)
+               const __grid_constant__ CUtensorMap tm_row, const __grid_constant__ CUtensorMap tm_piv, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ Shared sh;
@@ -173,7 +177,7 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
                     ok = ctl.wait_bar(smem_u32(&sh.empty[ring.stage]), ring.phase ^ 1u, kWaitStageFree, g);
                     if (ok)
                         mbar_arrive_expect_tx(full, (uint32_t)nh * ((rows == kTileRows ? (uint32_t)kAtomBytes : (uint32_t)n_sub * kSubBytes) +
-                                                                    (uint32_t)((p.P + 3) / 4) * 512u));
+                                                                    (p.compact ? (uint32_t)p.N * 128u : (uint32_t)((p.P + 3) / 4) * 512u)));
                 }
                 ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
                 if (!ok) break;
@@ -185,12 +189,16 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
                     } else if (lane < n_sub) {
                         tma_load_2d(dst + (uint32_t)lane * kSubBytes, &tm_keys, x, y0 + lane * kSubRows, full, pol_drop);
                     }
+                    if (p.compact) { // rows b N .. b N + N - 1 of the compact copy: the sample's pivots in rank order, zero padded
+                        if (lane == kMaxAtomsPerStage + h) tma_load_2d(b_addr(ring.stage, h), &tm_piv, x, b * p.N, full, pol_keep);
+                    } else {
 #pragma unroll
-                    for (int k = 0; k < kMaxN / 128; ++k) {
-                        const int q = lane + 32 * k; // pivot ranks 4q..4q+3 -> rows 4q..4q+3 of the pivot tile
-                        if (4 * q < p.P)
-                            tma_gather4(b_addr(ring.stage, h) + (uint32_t)q * 512u, &tm_row, x, my_piv[k][0], my_piv[k][1],
-                                        my_piv[k][2], my_piv[k][3], full, pol_keep);
+                        for (int k = 0; k < kMaxN / 128; ++k) {
+                            const int q = lane + 32 * k; // pivot ranks 4q..4q+3 -> rows 4q..4q+3 of the pivot tile
+                            if (4 * q < p.P)
+                                tma_gather4(b_addr(ring.stage, h) + (uint32_t)q * 512u, &tm_row, x, my_piv[k][0], my_piv[k][1],
+                                            my_piv[k][2], my_piv[k][3], full, pol_keep);
+                        }
                     }
                 }
                 ring.advance();

@@ -209,6 +209,30 @@ pivots_given_kernel(const int32_t *__restrict__ pivots_in, int n_vis, int P, int
 }
 
 // ------------------------------------------------------------------------------------------------
+// Compact copy of every sample's pivot rows, [B][N][d8] with N >= P rows per sample (rows P.. are zero), so that a
+// tensor-core kernel can fetch a sample's pivot tile as one box.  One warp per row.
+// ------------------------------------------------------------------------------------------------
+constexpr int kPivotRowWarps = 8;
+
+__global__ void __launch_bounds__(kPivotRowWarps * 32)
+pivot_rows_kernel(const uint4 *__restrict__ keys, const int32_t *__restrict__ pivot_idx, int S, int d8, int vis_offset, int n_vis,
+                  int P, int N, long long rows_total, uint4 *__restrict__ out)
+{
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * kPivotRowWarps + (threadIdx.x >> 5);
+    if (row >= rows_total) return;
+    const int b = (int)(row / N), i = (int)(row % N);
+    uint4 *dst = out + (size_t)row * d8;
+    if (i >= P) {
+        for (int c = lane; c < d8; c += 32) dst[c] = make_uint4(0, 0, 0, 0);
+        return;
+    }
+    const int pv = min(max(pivot_idx[(size_t)b * P + i], 0), n_vis - 1);
+    const uint4 *src = keys + ((size_t)b * S + vis_offset + pv) * (size_t)d8;
+    for (int c = lane; c < d8; c += 32) dst[c] = __ldg(src + c);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Step 5a for one sample (all threads of the CTA): the packed index list - text rows before, kept vision
 // tokens in ascending order (ordered ballot scan over the keep flags), text rows after - and the position
 // ids of those rows.  warp_tot: shared scratch, one word per warp.
