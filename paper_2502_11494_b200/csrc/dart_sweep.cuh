@@ -513,7 +513,8 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
         // ------------------------------------------------------------------ sweep-1 producer
         if (lane == 0) {
             unsigned long long pol_keep;
-            // the second read of a row comes too late to find it in L2 (see the design notes), so nothing is kept
+            // the second read of a row follows once the sample's pivots exist, 13-20 us later: by then ~100 MB of newer rows
+            // have passed and the L2 (which keeps a row for about 57 MB of traffic) no longer has it, so nothing is kept
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_keep));
             Ring ring(p.n1);
             long long issued = 0;
