@@ -209,7 +209,10 @@ void launch_retention(dart_ctx *ctx, int B, const int64_t *pos_in, int vis_offse
     }
     if (m > 0) {
         Prof p(ctx, st, SLOT_RETAIN);
-        candidates_kernel<<<dim3((unsigned)P, (unsigned)B), kCandThreads, candidates_smem_bytes(n_vis, m_pad), st>>>(
+        // one CTA per SM at most: big CTAs shorten each selection; more CTAs than SMs: small ones overlap better
+        // (measured: 8 x 16 lists 67 -> 54 us with 1024 threads, 64 x 8 lists 36 -> 45 us)
+        const int threads = (long long)B * P <= ctx->sm_count ? kCandThreads : 256;
+        candidates_kernel<<<dim3((unsigned)P, (unsigned)B), threads, candidates_smem_bytes(n_vis, m_pad), st>>>(
             ctx->sim, ctx->pivot_idx, n_vis, P, n_keep, m_pad, ctx->cand_stride, ctx->cand, ctx->status);
     }
     {

@@ -373,7 +373,7 @@ retain_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_i
 // buffer, M_pad = next power of two >= n_keep - P).  Phase 2: n_vis rounded to 16 (keep flags) +
 // kWalkStageEntries * 4 (staged candidate lists).
 // ------------------------------------------------------------------------------------------------
-constexpr int kCandThreads = 256;
+constexpr int kCandThreads = 1024;      // at most; the host launches fewer threads per CTA when there are many CTAs
 constexpr int kCandMax = 4096;           // candidates per pivot the sort buffer takes (n_keep - P <= 4096)
 constexpr int kWalkThreads = 256;
 constexpr int kWalkStageEntries = 12288; // 48 KB of staged candidate indices per round of phase 2
