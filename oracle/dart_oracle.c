@@ -158,6 +158,35 @@ int dart_oracle_similarity(const uint16_t *keys, int S, int d, int vis_offset, i
 }
 
 /*
+ * Eq. 7 when pivots may be ANY token of the sequence (the paper also tries pivots taken from the text tokens,
+ * Sec. 5.4): pivot_idx is still relative to the vision block, so a text token before it has a negative index and
+ * one after it an index >= n_vis.  Every norm is computed here from its row; a zero norm gives dup = 0.
+ */
+int dart_oracle_similarity_any(const uint16_t *keys, int S, int d, int vis_offset, int n_vis,
+                               const int32_t *pivot_idx, int P, double *dup)
+{
+    if (S < 1 || d < 1 || vis_offset < 0 || n_vis < 0 || vis_offset + n_vis > S || P < 1) return ORACLE_ERR_SHAPE;
+    for (int i = 0; i < P; ++i) {
+        const int s = vis_offset + pivot_idx[i];
+        if (s < 0 || s >= S) return ORACLE_ERR_SHAPE;
+        const uint16_t *prow = keys + (size_t)s * (size_t)d;
+        double pp = 0.0;
+        for (int c = 0; c < d; ++c) pp += bf16_to_f64(prow[c]) * bf16_to_f64(prow[c]);
+        for (int j = 0; j < n_vis; ++j) {
+            const uint16_t *xrow = keys + (size_t)(vis_offset + j) * (size_t)d;
+            double dot = 0.0, xx = 0.0;
+            for (int c = 0; c < d; ++c) {
+                dot += bf16_to_f64(prow[c]) * bf16_to_f64(xrow[c]);
+                xx += bf16_to_f64(xrow[c]) * bf16_to_f64(xrow[c]);
+            }
+            const double den = sqrt(pp) * sqrt(xx);
+            dup[(size_t)i * (size_t)n_vis + j] = den > 0.0 ? dot / den : 0.0;
+        }
+    }
+    return ORACLE_OK;
+}
+
+/*
  * Retention under the budget (Eq. 9-10; Sec. 1: "retain the vision tokens with the
  * lowest cosine similarity to the pivots"; eps is set per pivot from the ratio).
  *
@@ -177,8 +206,28 @@ int dart_oracle_similarity(const uint16_t *keys, int S, int d, int vis_offset, i
  * The equal split of the budget, the order of the pivots' turns and the exclusion of already
  * retained tokens are readings of the sentence that eps follows from the reduction ratio.
  */
+/*
+ * With text_pivots != 0 a pivot index outside [0, n_vis) names a text token: it takes its turn like any pivot but is
+ * not a vision token, so it is neither marked nor counted: the budget is split as q = (n_keep - Pv) / P,
+ * r = (n_keep - Pv) % P with Pv the pivots inside the vision block, and |kept| = n_keep vision tokens as always.
+ */
+static int retention_quotas(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep, int text_pivots,
+                            uint8_t *keep, int32_t *owner, double *eps, double *gap_out);
+
 int dart_oracle_retention(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep,
                           uint8_t *keep, int32_t *owner, double *eps, double *gap_out)
+{
+    return retention_quotas(dup, pivot_idx, n_vis, P, n_keep, 0, keep, owner, eps, gap_out);
+}
+
+int dart_oracle_retention_any(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep,
+                              uint8_t *keep, int32_t *owner, double *eps, double *gap_out)
+{
+    return retention_quotas(dup, pivot_idx, n_vis, P, n_keep, 1, keep, owner, eps, gap_out);
+}
+
+static int retention_quotas(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep, int text_pivots,
+                            uint8_t *keep, int32_t *owner, double *eps, double *gap_out)
 {
     if (P < 1 || P > n_keep || n_keep > n_vis) return ORACLE_ERR_SHAPE;
     keyed_t *cand = (keyed_t *)malloc((size_t)n_vis * sizeof *cand);
@@ -186,16 +235,26 @@ int dart_oracle_retention(const double *dup, const int32_t *pivot_idx, int n_vis
     memset(keep, 0, (size_t)n_vis);
     if (owner)
         for (int j = 0; j < n_vis; ++j) owner[j] = OWNER_DROPPED;
+    int Pv = 0;
     for (int i = 0; i < P; ++i) {
         int p = pivot_idx[i];
+        if (text_pivots && (p < 0 || p >= n_vis)) { /* a text token: distinctness among those is the caller's business */
+            for (int k = 0; k < i; ++k)
+                if (pivot_idx[k] == p) {
+                    free(cand);
+                    return ORACLE_ERR_SHAPE;
+                }
+            continue;
+        }
         if (p < 0 || p >= n_vis || keep[p]) {
             free(cand);
             return ORACLE_ERR_SHAPE; /* pivots must be distinct vision tokens */
         }
         keep[p] = 1;
         if (owner) owner[p] = P + i;
+        ++Pv;
     }
-    const int q = (n_keep - P) / P, r = (n_keep - P) % P;
+    const int q = (n_keep - Pv) / P, r = (n_keep - Pv) % P;
     double gap = INFINITY;
     for (int i = 0; i < P; ++i) {
         const int qi = q + (i < r ? 1 : 0);
@@ -351,11 +410,13 @@ int dart_oracle_compact(const uint8_t *keep, const uint16_t *hidden, const int64
  * which tensor represents them.  0: the key rows (one tensor for both); 1: the pivots are still chosen by the
  * key rows' scores, Eq. 7 is evaluated on the hidden rows.  Then l1_out holds the key rows' L1 scores and
  * l2_out the HIDDEN rows' Euclidean norms (Eq. 7's denominators).  Ignored when keys is NULL.
+ * text_pivots: entries of pivots_in outside [0, n_vis) name text tokens (index relative to the vision block);
+ * see dart_oracle_similarity_any and dart_oracle_retention_any.  Needs pivots_in and rule 0.
  */
 int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const int64_t *pos_in,
                           const int32_t *pivots_in,
                           int B, int S, int d, int vis_offset, int n_vis, int n_pivot, int n_keep,
-                          int norm_kind, int largest, int rule, int cosine_on_hidden,
+                          int norm_kind, int largest, int rule, int cosine_on_hidden, int text_pivots,
                           uint16_t *out_hidden, int32_t *out_idx, int64_t *out_pos,
                           double *l1_out, double *l2_out, int32_t *pivot_out, double *dup_out,
                           uint8_t *keep_out, int32_t *owner_out, double *eps_out,
@@ -365,6 +426,7 @@ int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const in
     if (n_pivot < 1 || n_pivot > n_keep || n_keep > n_vis) return ORACLE_ERR_SHAPE;
     if (norm_kind != 1 && norm_kind != 2) return ORACLE_ERR_SHAPE;
     if (rule != 0 && rule != 1) return ORACLE_ERR_SHAPE;
+    if (text_pivots && (!pivots_in || rule != 0)) return ORACLE_ERR_SHAPE; /* text pivots are the caller's, quota rule only */
     const int P = n_pivot, S_out = S - n_vis + n_keep;
     double *l1 = (double *)malloc((size_t)n_vis * sizeof(double));
     double *l2 = (double *)malloc((size_t)n_vis * sizeof(double));
@@ -394,9 +456,12 @@ int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const in
             rc = dart_oracle_scores(h, S, d, vis_offset, n_vis, hl1, l2);
             if (rc) break;
         }
-        rc = dart_oracle_similarity((cosine_on_hidden && keys) ? h : k, S, d, vis_offset, n_vis, piv, P, l2, dup);
+        if (text_pivots)
+            rc = dart_oracle_similarity_any((cosine_on_hidden && keys) ? h : k, S, d, vis_offset, n_vis, piv, P, dup);
+        else
+            rc = dart_oracle_similarity((cosine_on_hidden && keys) ? h : k, S, d, vis_offset, n_vis, piv, P, l2, dup);
         if (rc) break;
-        rc = (rule == 1 ? dart_oracle_retention_global : dart_oracle_retention)(
+        rc = (text_pivots ? dart_oracle_retention_any : rule == 1 ? dart_oracle_retention_global : dart_oracle_retention)(
             dup, piv, n_vis, P, n_keep, keep, owner_out ? owner_out + (size_t)b * n_vis : NULL,
             eps_out ? eps_out + (size_t)b * P : NULL, &rgap);
         if (rc) break;
@@ -435,6 +500,6 @@ int dart_oracle_reduce(const uint16_t *hidden, const uint16_t *keys, const int64
                        double *pivot_gap_out, double *retain_gap_out)
 {
     return dart_oracle_reduce_ex(hidden, keys, pos_in, NULL, B, S, d, vis_offset, n_vis, n_pivot, n_keep, norm_kind,
-                                 largest, 0, 0, out_hidden, out_idx, out_pos, l1_out, l2_out, pivot_out, dup_out, keep_out,
+                                 largest, 0, 0, 0, out_hidden, out_idx, out_pos, l1_out, l2_out, pivot_out, dup_out, keep_out,
                                  owner_out, eps_out, pivot_gap_out, retain_gap_out);
 }

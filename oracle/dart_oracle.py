@@ -39,7 +39,8 @@ def _load():
     if _lib is None:
         _lib = ctypes.CDLL(build())
         for name in ("dart_oracle_scores", "dart_oracle_pivots", "dart_oracle_similarity",
-                     "dart_oracle_retention", "dart_oracle_retention_global", "dart_oracle_compact",
+                     "dart_oracle_retention", "dart_oracle_retention_global", "dart_oracle_retention_any",
+                     "dart_oracle_similarity_any", "dart_oracle_compact",
                      "dart_oracle_gather_rows", "dart_oracle_reduce", "dart_oracle_reduce_ex"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
@@ -122,6 +123,32 @@ def retention(dup, pivot_idx, n_keep: int):
     return keep, owner, eps, gap.value
 
 
+def similarity_any(keys, vis_offset: int, n_vis: int, pivot_idx):
+    """Eq. 7 for pivots that may be text tokens (indices relative to the vision block) -> dup [P, n_vis]."""
+    k = _u16(keys)
+    S, d = k.shape
+    piv = np.ascontiguousarray(pivot_idx, np.int32)
+    dup = np.empty((len(piv), n_vis), np.float64)
+    _check(_load().dart_oracle_similarity_any(_p(k, ctypes.c_uint16), S, d, vis_offset, n_vis, _p(piv, ctypes.c_int32),
+                                              len(piv), _p(dup, ctypes.c_double)), "similarity_any")
+    return dup
+
+
+def retention_any(dup, pivot_idx, n_keep: int):
+    """Quota retention where pivots outside [0, n_vis) are text tokens: (keep, owner, eps, gap)."""
+    dd = np.ascontiguousarray(dup, np.float64)
+    P, n_vis = dd.shape
+    piv = np.ascontiguousarray(pivot_idx, np.int32)
+    keep = np.empty(n_vis, np.uint8)
+    owner = np.empty(n_vis, np.int32)
+    eps = np.empty(P, np.float64)
+    gap = ctypes.c_double(0.0)
+    _check(_load().dart_oracle_retention_any(_p(dd, ctypes.c_double), _p(piv, ctypes.c_int32), n_vis, P, n_keep,
+                                             _p(keep, ctypes.c_uint8), _p(owner, ctypes.c_int32),
+                                             _p(eps, ctypes.c_double), ctypes.byref(gap)), "retention_any")
+    return keep, owner, eps, gap.value
+
+
 def retention_global(dup, pivot_idx, n_keep: int):
     """dup [P, n_vis] -> (keep, owner, eps [P], gap) with one threshold on max_i dup for all pivots."""
     dd = np.ascontiguousarray(dup, np.float64)
@@ -190,11 +217,13 @@ class OracleResult:
 
 def reduce(hidden, keys, vis_offset: int, n_vis: int, n_pivot: int, n_keep: int,
            pos_in=None, norm_kind: int = 1, largest: bool = True, want_dup: bool = True,
-           want_hidden: bool = True, pivots_in=None, rule: int = 0, cosine_on_hidden: bool = False) -> OracleResult:
+           want_hidden: bool = True, pivots_in=None, rule: int = 0, cosine_on_hidden: bool = False,
+           text_pivots: bool = False) -> OracleResult:
     """The whole step over a batch.  hidden/keys: [B, S, d] bf16 bits (keys None -> hidden is scored).
     pivots_in: None, or [B, n_pivot] distinct vision-relative indices that replace the pivot step.
     rule: 0 = per-pivot thresholds from equal quotas, 1 = one threshold for all pivots.
-    cosine_on_hidden: pivots by the key rows' scores, Eq. 7 on the hidden rows (then .l2 holds the hidden rows' norms)."""
+    cosine_on_hidden: pivots by the key rows' scores, Eq. 7 on the hidden rows (then .l2 holds the hidden rows' norms).
+    text_pivots: entries of pivots_in outside [0, n_vis) name text tokens (indices relative to the vision block)."""
     h = _u16(hidden)
     B, S, d = h.shape
     k = None if keys is None else _u16(keys)
@@ -219,7 +248,7 @@ def reduce(hidden, keys, vis_offset: int, n_vis: int, n_pivot: int, n_keep: int,
         raise ValueError("pivots_in must be [B, n_pivot]")
     _check(_load().dart_oracle_reduce_ex(
         _p(h, ctypes.c_uint16), _p(k, ctypes.c_uint16), _p(pos, ctypes.c_int64), _p(piv_in, ctypes.c_int32),
-        B, S, d, vis_offset, n_vis, n_pivot, n_keep, norm_kind, int(bool(largest)), int(rule), int(bool(cosine_on_hidden)),
+        B, S, d, vis_offset, n_vis, n_pivot, n_keep, norm_kind, int(bool(largest)), int(rule), int(bool(cosine_on_hidden)), int(bool(text_pivots)),
         _p(oh, ctypes.c_uint16), _p(oi, ctypes.c_int32), _p(op, ctypes.c_int64),
         _p(l1, ctypes.c_double), _p(l2, ctypes.c_double), _p(piv, ctypes.c_int32), _p(dup, ctypes.c_double),
         _p(keep, ctypes.c_uint8), _p(owner, ctypes.c_int32), _p(eps, ctypes.c_double),

@@ -177,3 +177,63 @@ def test_cosine_on_hidden_rows_is_the_composition_of_the_steps(oracle):
     assert np.array_equal(same.out_idx, plain.out_idx) and np.array_equal(same.dup, plain.dup)
     none = oracle.reduce(hb, None, vo, nv, P, Kp, cosine_on_hidden=True)                    # keys = None: likewise
     assert np.array_equal(none.out_idx, plain.out_idx)
+
+
+# ----------------------------------------------------------------------------- pivots taken from the text tokens
+
+def test_text_pivots_similarity_and_budget(oracle):
+    """Pivots outside the vision block: their cosines against numpy, the budget split over all pivots but counted
+    in vision tokens only, and the coincidence with the plain functions when every pivot is a vision token."""
+    rng = np.random.default_rng(28)
+    S, d, vo, nv = 70, 32, 8, 50
+    kb, kv = rand_tokens(rng, S, d)
+    piv = np.array([3, -5, 17, nv + 6, -8], np.int32)            # vision, text before, vision, text after, first token
+    dup = oracle.similarity_any(kb, vo, nv, piv)
+    X = kv[vo:vo + nv]
+    Xn = X / np.linalg.norm(X, axis=1, keepdims=True)
+    Pr = kv[vo + piv]
+    Pn = Pr / np.linalg.norm(Pr, axis=1, keepdims=True)
+    assert np.allclose(dup, Pn @ Xn.T, rtol=0, atol=1e-12)       # an independent routine
+    n_keep = 20                                                  # 2 vision pivots + 18 over 5 pivots: quotas 4,4,4,3,3
+    keep, owner, eps, gap = oracle.retention_any(dup, piv, n_keep)
+    assert int(keep.sum()) == n_keep and keep[3] == 1 and keep[17] == 1
+    assert [int((owner == i).sum()) for i in range(5)] == [4, 4, 4, 3, 3]
+    assert owner[3] == 5 + 0 and owner[17] == 5 + 2
+    kept = {3, 17}
+    for i, qi in enumerate([4, 4, 4, 3, 3]):                     # every turn takes the lowest dup among what is left
+        cands = [j for j in range(nv) if j not in kept]
+        best = sorted(cands, key=lambda j: (dup[i, j], j))[:qi]
+        assert sorted(best) == sorted(np.nonzero(owner == i)[0].tolist())
+        assert eps[i] == max(dup[i, j] for j in best)
+        kept |= set(best)
+    vis_only = np.array([3, 17, 30], np.int32)                   # no text pivot: the plain functions
+    _, l2 = oracle.scores(kb, vo, nv)
+    assert np.allclose(oracle.similarity_any(kb, vo, nv, vis_only), oracle.similarity(kb, vo, nv, vis_only, l2), rtol=0, atol=1e-15)
+    d2 = oracle.similarity(kb, vo, nv, vis_only, l2)
+    a, b = oracle.retention_any(d2, vis_only, 12), oracle.retention(d2, vis_only, 12)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    with pytest.raises(RuntimeError):
+        oracle.similarity_any(kb, vo, nv, np.array([-9], np.int32))          # before the sequence
+    with pytest.raises(RuntimeError):
+        oracle.retention_any(dup, np.array([3, -5, 17, -5, -8], np.int32), n_keep)   # repeated text pivot
+    with pytest.raises(RuntimeError):
+        oracle.retention(dup, piv, n_keep)                                   # the plain rule takes vision pivots only
+
+
+def test_text_pivots_through_the_whole_step(oracle):
+    rng = np.random.default_rng(29)
+    B, S, d, vo, nv, P, Kp = 2, 64, 32, 6, 50, 4, 15
+    hb, _ = rand_tokens(rng, B * S, d)
+    kb, _ = rand_tokens(rng, B * S, d)
+    hb, kb = hb.reshape(B, S, d), kb.reshape(B, S, d)
+    piv = np.array([[4, -2, nv + 3, 20], [-6, -1, nv, nv + 7]], np.int32)   # sample 1: text pivots only
+    r = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=piv, text_pivots=True)
+    for b in range(B):
+        dup = oracle.similarity_any(kb[b], vo, nv, piv[b])
+        keep, owner, eps, _ = oracle.retention_any(dup, piv[b], Kp)
+        oh, oi, op = oracle.compact(keep, hb[b], vo, nv)
+        assert np.array_equal(r.keep[b], keep) and np.array_equal(r.out_idx[b], oi) and np.array_equal(r.out_hidden[b], oh)
+        assert int(keep.sum()) == Kp                                        # the budget counts vision tokens
+        assert r.out_idx.shape[1] == S - nv + Kp
+    with pytest.raises(RuntimeError):
+        oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=piv)                 # text pivots must be asked for
