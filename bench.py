@@ -368,13 +368,13 @@ def main():
         variants = {}
         n_v = max(3, args.steps // 4)
         # (a) retention with one threshold for all pivots
-        o_g = dart.dart_opts(0, 0, args.path, 0, args.lag, 0, args.retention, dart.DART_RULE_GLOBAL, 0, None)
+        o_g = dart.dart_opts(path=args.path, sweep_lag=args.lag, retention=args.retention, rule=dart.DART_RULE_GLOBAL)
         ms_g, _, prof_g = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_g, False)
         variants["one_threshold"] = {"ms_per_step": ms_g / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_g * 1e-3),
                                      "retain_ms": prof_g["retain"][0] / max(prof_g["retain"][1], 1)}
         # (b) pivots named by the caller (here: random distinct tokens): steps 3-5 only wait for the norms
         piv = torch.stack([torch.randperm(w.n_vis, device=dev)[:w.n_pivot] for _ in range(B)]).to(torch.int32).contiguous()
-        o_p = dart.dart_opts(0, 0, args.path, 0, args.lag, 0, args.retention, 0, 0, piv.data_ptr())
+        o_p = dart.dart_opts(path=args.path, sweep_lag=args.lag, retention=args.retention, pivots_in=piv.data_ptr())
         ms_p, _, prof_p = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_p, False)
         variants["pivots_given"] = {"ms_per_step": ms_p / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_p * 1e-3),
                                     "path_frac_of_measured_copy": path_bytes_per_sample(w) * B / (ms_p / n_v * 1e-3) / 1e9 / peak}
@@ -385,8 +385,15 @@ def main():
             variants["pivots_given"]["onepass_kernel"] = {"ms_per_launch": ms_o, "achieved_GBps": gbs_o,
                                                           "frac_of_measured_copy": gbs_o / peak,
                                                           "traffic": tr * B if tr else None}
+        # (b1) the caller's pivots drawn from the whole sample, text tokens included (indices relative to the vision block)
+        piv_t = (torch.stack([torch.randperm(w.S, device=dev)[:w.n_pivot] for _ in range(B)]) - w.vis_offset).to(torch.int32).contiguous()
+        o_t = dart.dart_opts(path=args.path, sweep_lag=args.lag, retention=args.retention, text_pivots=1, pivots_in=piv_t.data_ptr())
+        ms_t, _, _ = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_t, False)
+        variants["text_pivots"] = {"ms_per_step": ms_t / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_t * 1e-3),
+                                   "path_frac_of_measured_copy": path_bytes_per_sample(w) * B / (ms_t / n_v * 1e-3) / 1e9 / peak}
+        del piv_t
         # (b2) pivots ranked by the key rows, Eq. 7 on the hidden rows: keys once (scores), hidden once (one pass)
-        o_h = dart.dart_opts(0, 0, args.path, 0, args.lag, 0, args.retention, 0, 1, None)
+        o_h = dart.dart_opts(path=args.path, sweep_lag=args.lag, retention=args.retention, cosine_on_hidden=1)
         ms_h, _, prof_h = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_h, False)
         bytes_h = (path_bytes_per_sample(w) + 2 * w.d * w.n_vis) * B   # one more read of n_vis x d than the main method
         variants["cosine_on_hidden"] = {"ms_per_step": ms_h / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_h * 1e-3),

@@ -102,6 +102,14 @@ typedef struct {
                               hidden states once for the similarities.  Needs norm_kind 0/1 (else UNSUPPORTED); no effect
                               when keys is NULL.  dbg->l1 then holds the key rows' scores, dbg->ssq the hidden rows' sums
                               of squares. */
+    int32_t text_pivots;   /* with pivots_in: 1 lets an entry name ANY token of the sample (the paper also draws pivots from
+                              the text tokens, Sec. 5.4).  Entries stay relative to the vision block, so a text token
+                              before it has a negative index and one after it an index >= n_vis; the range is
+                              [-vis_offset, S - vis_offset), entries distinct.  A text pivot takes its turn in step 4 like
+                              any other but is no vision token: with Pv the pivots inside the vision block, step 4 uses
+                              q = (n_keep - Pv) / P and r = (n_keep - Pv) % P, and n_keep vision tokens are kept as
+                              always.  dbg->owner marks only the vision pivots.  Needs pivots_in, DART_RULE_QUOTAS and a
+                              shape the FUSED path takes (else UNSUPPORTED). */
     const int32_t *pivots_in; /* NULL: pivots by score (steps 1-2).  Else [B, n_pivot] int32, device: the caller's pivots
                               as vision-relative indices, distinct and in [0, n_vis); their order is the order of the
                               pivots' turns in step 4.  This covers the paper's other ways to choose pivots (Sec. 5.2:

@@ -49,6 +49,14 @@ class ParityReport:
         return self
 
 
+def quotas_any(pivot_idx, n_vis: int, n_keep: int):
+    """Quotas when pivots outside [0, n_vis) are text tokens: only the vision pivots count against the budget."""
+    P = len(pivot_idx)
+    Pv = int(sum(0 <= int(p) < n_vis for p in pivot_idx))
+    q, r = divmod(n_keep - Pv, P)
+    return [q + (1 if i < r else 0) for i in range(P)]
+
+
 def quotas(P: int, n_keep: int):
     q, r = divmod(n_keep - P, P)
     return [q + (1 if i < r else 0) for i in range(P)]
@@ -89,11 +97,15 @@ def check_sim(sim, ora_dup, rep: ParityReport, tol=REL_TOL, floor=SIM_ABS_FLOOR)
 
 
 def check_valid_under_tolerance(keys_bits, vis_offset, n_vis, n_keep, pivot_idx, owner, ora_score, ora_l2,
-                                largest=True, tol=MARGIN, pivots_given=False, rule=0):
+                                largest=True, tol=MARGIN, pivots_given=False, rule=0, text_pivots=False):
     """Replay the candidate's own pivots and assignment against fp64 quantities (one sample).
     ora_score is the oracle's ranking score (L1 norms, or the Euclidean norms for that variant); with
     pivots_given the caller chose the pivots and nothing about their ranking is checked; rule 1 is the
-    variant with one threshold for all pivots."""
+    variant with one threshold for all pivots; text_pivots (with pivots_given, rule 0): pivots outside [0, n_vis) are
+    text tokens."""
+    if text_pivots:
+        assert pivots_given and rule == 0
+        return _replay_text_pivots(keys_bits, vis_offset, n_vis, n_keep, pivot_idx, owner, tol)
     P = len(pivot_idx)
     assert len(set(pivot_idx.tolist())) == P, "pivots must be distinct"
     s = ora_score
@@ -143,9 +155,37 @@ def check_valid_under_tolerance(keys_bits, vis_offset, n_vis, n_keep, pivot_idx,
     return kept
 
 
+def _replay_text_pivots(keys_bits, vis_offset, n_vis, n_keep, pivot_idx, owner, tol):
+    P = len(pivot_idx)
+    assert len(set(pivot_idx.tolist())) == P, "pivots must be distinct"
+    dup = _o.similarity_any(keys_bits, vis_offset, n_vis, pivot_idx)
+    kept = np.zeros(n_vis, bool)
+    for i, p in enumerate(pivot_idx.tolist()):
+        if 0 <= p < n_vis:
+            kept[p] = True
+            assert int(owner[p]) == P + i, "vision pivots carry their rank in owner"
+    assert int((owner >= P).sum()) == int(kept.sum()), "only vision pivots are marked as pivots"
+    for i, qi in enumerate(quotas_any(pivot_idx, n_vis, n_keep)):
+        mine = np.nonzero(owner == i)[0]
+        assert len(mine) == qi, "pivot %d retained %d tokens, quota %d" % (i, len(mine), qi)
+        if qi == 0:
+            continue
+        assert not kept[mine].any(), "pivot %d retained a token that was already kept" % i
+        eps_i = dup[i, mine].max()
+        left = ~kept
+        left[mine] = False
+        if left.any():
+            assert dup[i, left].min() >= eps_i - tol, \
+                "pivot %d left behind a token %g below its threshold" % (i, eps_i - dup[i, left].min())
+        kept[mine] = True
+    assert int(kept.sum()) == n_keep
+    assert np.array_equal(np.nonzero(owner >= 0)[0], np.nonzero(kept)[0]), "owner and kept set disagree"
+    return kept
+
+
 def check_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, n_vis, n_pivot, n_keep,
                 out_hidden, out_idx, out_pos, dbg=None, pos_in=None, largest=True, norm_kind=1,
-                require_exact_above=MARGIN, pivots_given=False, rule=0, sim_bits=None) -> ParityReport:
+                require_exact_above=MARGIN, pivots_given=False, rule=0, sim_bits=None, text_pivots=False) -> ParityReport:
     """All rules over a batch.  ``dbg`` (optional) holds the candidate's per-step outputs as numpy arrays:
     l1, ssq, pivot_idx, sim, eps, keep, owner.  Without it only the packed outputs are checked.
     ``sim_bits``: the tensor Eq. 7 is evaluated on when it is not the scored one (cosine on the hidden rows)."""
@@ -180,7 +220,8 @@ def check_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, n_vis,
             check_sim(dbg["sim"][b], ora.dup[b], rep)
         if margin[b] > require_exact_above:
             assert np.array_equal(dbg["owner"][b], ora.owner[b])
-            qs = quotas(n_pivot, n_keep) if rule == 0 else [n_keep - n_pivot] * n_pivot
+            qs = (quotas_any(dbg["pivot_idx"][b], n_vis, n_keep) if text_pivots else
+                  quotas(n_pivot, n_keep) if rule == 0 else [n_keep - n_pivot] * n_pivot)
             has = np.array([q > 0 for q in qs])
             e = dbg["eps"][b].astype(np.float64)
             assert np.all(np.isnan(e[~has])) and np.all(np.abs(e[has] - ora.eps[b][has]) <= REL_TOL * np.abs(ora.eps[b][has]) + SIM_ABS_FLOOR)
@@ -188,7 +229,7 @@ def check_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, n_vis,
             check_valid_under_tolerance(keys_bits[b] if sim_bits is None else sim_bits[b], vis_offset, n_vis, n_keep,
                                         dbg["pivot_idx"][b], dbg["owner"][b],
                                         ora.l1[b] if norm_kind == 1 else ora.l2[b], ora.l2[b], largest=largest,
-                                        pivots_given=pivots_given, rule=rule)
+                                        pivots_given=pivots_given, rule=rule, text_pivots=text_pivots)
             if not same:
                 rep.notes.append("sample %d differs below margin %.2e (valid under tolerance)" % (b, margin[b]))
     return rep

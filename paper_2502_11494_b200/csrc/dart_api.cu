@@ -185,7 +185,8 @@ void launch_retention(dart_ctx *ctx, int B, const int64_t *pos_in, int vis_offse
                       int32_t *out_idx, int64_t *out_pos, const dart_opts &o, cudaStream_t st)
 {
     using namespace dart;
-    const int S = ctx->S, m = n_keep - P, mode = o.retention;
+    // the tokens shared out beside the pivots: n_keep - P, or up to n_keep when pivots may be text tokens
+    const int S = ctx->S, m = o.text_pivots ? n_keep : n_keep - P, mode = o.retention;
     if (o.rule == DART_RULE_GLOBAL) { // one threshold for all pivots: a single selection per sample
         Prof p(ctx, st, SLOT_RETAIN);
         retain_global_kernel<<<B, kSelectThreads, retain_global_smem_bytes(n_vis), st>>>(
@@ -224,10 +225,11 @@ void launch_retention(dart_ctx *ctx, int B, const int64_t *pos_in, int vis_offse
 }
 
 // Step 2 with the caller's pivots: checked and copied into the workspace.
-void launch_pivots_given(dart_ctx *ctx, int B, int n_vis, int P, const int32_t *pivots_in, cudaStream_t st)
+void launch_pivots_given(dart_ctx *ctx, int B, int vis_offset, int n_vis, int P, const dart_opts &o, cudaStream_t st)
 {
     Prof p(ctx, st, SLOT_PIVOT);
-    dart::pivots_given_kernel<<<B, 256, (size_t)((n_vis + 31) / 32) * 4, st>>>(pivots_in, n_vis, P, ctx->pivot_idx, ctx->status);
+    const int lo = o.text_pivots ? -vis_offset : 0, hi = o.text_pivots ? ctx->S - vis_offset : n_vis;
+    dart::pivots_given_kernel<<<B, 256, (size_t)((hi - lo + 31) / 32) * 4, st>>>(o.pivots_in, lo, hi, P, ctx->pivot_idx, ctx->status);
 }
 
 int launch_staged(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, const int64_t *pos_in, int vis_offset,
@@ -244,7 +246,7 @@ int launch_staged(dart_ctx *ctx, int B, const void *hidden, const void *keys_in,
         score_kernel<<<grid, kScoreWarps * 32, 0, st>>>(keys, S, d8, vis_offset, n_vis, rows, ctx->l1, ctx->ssq);
     }
     if (o.pivots_in) {
-        launch_pivots_given(ctx, B, n_vis, P, o.pivots_in, st);
+        launch_pivots_given(ctx, B, vis_offset, n_vis, P, o, st);
     } else {
         Prof p(ctx, st, SLOT_PIVOT);
         int P_pad = next_pow2(P);
@@ -442,7 +444,7 @@ int launch_onepass(dart_ctx *ctx, int B, const void *hidden, const void *keys_in
                    int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos, const dart_opts &o,
                    const dart_debug *dbg, cudaStream_t st)
 {
-    launch_pivots_given(ctx, B, n_vis, P, o.pivots_in, st);
+    launch_pivots_given(ctx, B, vis_offset, n_vis, P, o, st);
     int rc = launch_onepass_kernel(ctx, B, keys_in ? keys_in : hidden, false, vis_offset, n_vis, P, o, st);
     if (rc != DART_OK) return rc;
     launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
@@ -470,7 +472,7 @@ int launch_two_pass(dart_ctx *ctx, int B, const void *hidden, const void *keys, 
                                                              (same && (o.norm_kind == 2 || !tensor_cores)) ? ctx->ssq : nullptr);
     }
     if (o.pivots_in) {
-        launch_pivots_given(ctx, B, n_vis, P, o.pivots_in, st);
+        launch_pivots_given(ctx, B, vis_offset, n_vis, P, o, st);
     } else {
         Prof p(ctx, st, SLOT_PIVOT);
         const int P_pad = next_pow2(P);
@@ -506,6 +508,7 @@ int launch_reduce(dart_ctx *ctx, int B, const void *hidden, const void *keys, co
 {
     const bool fused = o.path == DART_PATH_FUSED || (o.path == DART_PATH_AUTO && fused_applies(ctx, P));
     if (fused && !fused_applies(ctx, P)) return DART_ERR_UNSUPPORTED;
+    if (o.text_pivots && !fused) return DART_ERR_UNSUPPORTED; // only the tensor-core kernel takes a text row's norm from the row
     if (o.cosine_on_hidden && keys && keys != hidden)
         return launch_two_pass(ctx, B, hidden, keys, hidden, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o,
                                dbg, fused, st);
@@ -692,6 +695,7 @@ int dart_reduce_ex(dart_ctx *ctx, const void *hidden, const void *keys, const in
     if (o.rule != DART_RULE_QUOTAS && o.rule != DART_RULE_GLOBAL) return DART_ERR_UNSUPPORTED;
     if (o.cosine_on_hidden && o.norm_kind != 1) return DART_ERR_UNSUPPORTED; // the hidden rows' sums of squares take the slot
     if ((uintptr_t)o.pivots_in & 3u) return DART_ERR_ALIGN;
+    if (o.text_pivots && (!o.pivots_in || o.rule != DART_RULE_QUOTAS)) return DART_ERR_UNSUPPORTED;
     if (o.rule == DART_RULE_GLOBAL &&
         dart::retain_global_smem_bytes(n_vis) > (size_t)ctx->max_smem_optin - 2048)
         return DART_ERR_UNSUPPORTED; // the sample's duplication values must fit shared memory

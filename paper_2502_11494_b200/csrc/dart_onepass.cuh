@@ -48,7 +48,7 @@ struct Params {
     unsigned long long wait_ns;
     float *sim;                        // [B][P][n_vis] dup(p_i, x_j)
     float *l1, *ssq;                   // [B][n_vis]; l1 may be NULL (the scores come from another tensor)
-    const int32_t *pivot_idx;          // [B][P], checked and clamped
+    const int32_t *pivot_idx;          // [B][P], checked and clamped; outside [0, n_vis): a text row of the sample
     int *status;
 };
 
@@ -163,7 +163,7 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const int i = min(4 * (lane + 32 * k) + e, p.P - 1); // ranks beyond P repeat the last pivot
-                        my_piv[k][e] = b * p.S + p.vis_offset + min(max(__ldg(p.pivot_idx + (size_t)b * p.P + i), 0), p.n_vis - 1);
+                        my_piv[k][e] = b * p.S + min(max(p.vis_offset + __ldg(p.pivot_idx + (size_t)b * p.P + i), 0), p.S - 1); // any row of the sample
                     }
                 cur_b = b;
             }

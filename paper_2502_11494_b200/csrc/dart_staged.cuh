@@ -187,18 +187,20 @@ sim_alu_kernel(const uint4 *__restrict__ keys, int S, int d8, int vis_offset, in
 constexpr int kStatusCheck = -8;       // DART_ERR_CHECK
 constexpr int kCheckPivotsGiven = 100; // second status word: which check failed
 
+// [lo, hi) is the range a pivot may lie in, relative to the vision block: [0, n_vis), or the whole sequence
+// [-vis_offset, S - vis_offset) when text tokens may serve as pivots (Sec. 5.4).
 __global__ void __launch_bounds__(256)
-pivots_given_kernel(const int32_t *__restrict__ pivots_in, int n_vis, int P, int32_t *__restrict__ pivot_idx, int *status)
+pivots_given_kernel(const int32_t *__restrict__ pivots_in, int lo, int hi, int P, int32_t *__restrict__ pivot_idx, int *status)
 {
-    extern __shared__ uint32_t seen[]; // [(n_vis + 31) / 32]
+    extern __shared__ uint32_t seen[]; // [(hi - lo + 31) / 32]
     const int b = blockIdx.x;
-    for (int w = threadIdx.x; w < (n_vis + 31) / 32; w += blockDim.x) seen[w] = 0;
+    for (int w = threadIdx.x; w < (hi - lo + 31) / 32; w += blockDim.x) seen[w] = 0;
     __syncthreads();
     for (int t = threadIdx.x; t < P; t += blockDim.x) {
         const int pv = pivots_in[(size_t)b * P + t];
-        bool bad = pv < 0 || pv >= n_vis;
-        const int c = min(max(pv, 0), n_vis - 1);
-        if (!bad) bad = (atomicOr(&seen[c >> 5], 1u << (c & 31)) >> (c & 31)) & 1u;
+        bool bad = pv < lo || pv >= hi;
+        const int c = min(max(pv, lo), hi - 1);
+        if (!bad) bad = (atomicOr(&seen[(c - lo) >> 5], 1u << ((c - lo) & 31)) >> ((c - lo) & 31)) & 1u;
         pivot_idx[(size_t)b * P + t] = c;
         if (bad && atomicCAS(status, 0, kStatusCheck) == 0) {
             status[1] = kCheckPivotsGiven;
@@ -227,9 +229,36 @@ pivot_rows_kernel(const uint4 *__restrict__ keys, const int32_t *__restrict__ pi
         for (int c = lane; c < d8; c += 32) dst[c] = make_uint4(0, 0, 0, 0);
         return;
     }
-    const int pv = min(max(pivot_idx[(size_t)b * P + i], 0), n_vis - 1);
+    const int pv = min(max(pivot_idx[(size_t)b * P + i], -vis_offset), S - vis_offset - 1); // any row of the sample
     const uint4 *src = keys + ((size_t)b * S + vis_offset + pv) * (size_t)d8;
     for (int c = lane; c < d8; c += 32) dst[c] = __ldg(src + c);
+}
+
+// ------------------------------------------------------------------------------------------------
+// kept := pivots, for one sample (all threads of the CTA; flags[] zeroed and the CTA synchronised before the call).
+// A pivot outside [0, n_vis) is a text token (Sec. 5.4): it takes its turn in step 4 but is no vision token, so it
+// is neither flagged nor counted.  Returns Pv, the pivots inside the vision block: the budget left to share out is
+// n_keep - Pv.  `word` is a shared scratch word; the CTA is synchronised on return.
+// ------------------------------------------------------------------------------------------------
+__device__ inline int mark_pivots(const int32_t *__restrict__ piv, int P, int n_vis, uint8_t *flags, int32_t *owner,
+                                  uint32_t *word)
+{
+    if (threadIdx.x == 0) *word = 0;
+    __syncthreads();
+    uint32_t mine = 0;
+    for (int i = threadIdx.x; i < P; i += blockDim.x) {
+        const int pv = piv[i];
+        if (pv >= 0 && pv < n_vis) {
+            flags[pv] = 1;
+            if (owner) owner[pv] = P + i;
+            ++mine;
+        }
+    }
+    if (mine) atomicAdd(word, mine);
+    __syncthreads();
+    const int Pv = (int)*word;
+    __syncthreads(); // the word may be reused
+    return Pv;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -315,13 +344,8 @@ retain_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_i
         if (owner) owner[j] = -1;
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < P; i += blockDim.x) {
-        int p = pivot_idx[(size_t)b * P + i];
-        keep[p] = 1;
-        if (owner) owner[p] = P + i;
-    }
-    __syncthreads();
-    const int q = (n_keep - P) / P, r = (n_keep - P) % P;
+    const int Pv = mark_pivots(pivot_idx + (size_t)b * P, P, n_vis, keep, owner, &sel.cnt);
+    const int q = (n_keep - Pv) / P, r = (n_keep - Pv) % P;
     for (int i = 0; i < P; ++i) {
         const int qi = q + (i < r ? 1 : 0);
         if (qi == 0) {
@@ -370,7 +394,7 @@ retain_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_i
 // ordered scan writes the packed index list as above.  The result equals retain_kernel's exactly.
 //
 // Dynamic shared memory, phase 1: n_vis * 4 (keys) and n_vis (pivot flags), each rounded to 16, + M_pad * 8 (sort
-// buffer, M_pad = next power of two >= n_keep - P).  Phase 2: n_vis rounded to 16 (keep flags) +
+// buffer, M_pad = next power of two >= n_keep - Pv, Pv = the pivots that are vision tokens).  Phase 2: n_vis rounded to 16 (keep flags) +
 // kWalkStageEntries * 4 (staged candidate lists).
 // ------------------------------------------------------------------------------------------------
 constexpr int kCandThreads = 1024;      // at most; the host launches fewer threads per CTA when there are many CTAs
@@ -398,21 +422,19 @@ candidates_kernel(const float *__restrict__ sim, const int32_t *__restrict__ piv
     __shared__ uint32_t n_picked;
     if (*status != 0) return; // an earlier kernel of this call failed: its outputs are undefined
     const int i = blockIdx.x, b = blockIdx.y;
-    const int q = (n_keep - P) / P, r = (n_keep - P) % P;
+    for (int j = threadIdx.x; j < n_vis; j += blockDim.x) is_pivot[j] = 0;
+    __syncthreads();
+    const int Pv = mark_pivots(pivot_idx + (size_t)b * P, P, n_vis, is_pivot, nullptr, &n_picked);
+    const int q = (n_keep - Pv) / P, r = (n_keep - Pv) % P;
     const int qi = q + (i < r ? 1 : 0);
     if (qi == 0) return; // this pivot keeps nothing (and so do all later ones)
     const int M = quota_prefix(i, q, r);
     const float *row = sim + ((size_t)b * P + i) * n_vis;
-    for (int j = threadIdx.x; j < n_vis; j += blockDim.x) {
-        keys[j] = order_key(row[j]);
-        is_pivot[j] = 0;
-    }
+    for (int j = threadIdx.x; j < n_vis; j += blockDim.x) keys[j] = order_key(row[j]);
     int mp = 1; // this pivot's own sort size
     while (mp < M) mp <<= 1;
     for (int t = threadIdx.x; t < mp; t += blockDim.x) list[t] = ~0ull;
     if (threadIdx.x == 0) n_picked = 0;
-    __syncthreads();
-    for (int t = threadIdx.x; t < P; t += blockDim.x) is_pivot[pivot_idx[(size_t)b * P + t]] = 1;
     __syncthreads();
     auto keyfn = [&](int j, uint32_t &key) {
         if (is_pivot[j]) return false;
@@ -458,20 +480,17 @@ retain_walk_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pi
     if (*status != 0) return;
     const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int S_out = S - n_vis + n_keep;
-    const int q = (n_keep - P) / P, r = (n_keep - P) % P;
     int32_t *owner = owner_out ? owner_out + (size_t)b * n_vis : nullptr;
     for (int j = threadIdx.x; j < n_vis; j += blockDim.x) {
         keep[j] = 0;
         if (owner) owner[j] = -1;
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < P; i += blockDim.x) {
-        const int pv = pivot_idx[(size_t)b * P + i];
-        keep[pv] = 1;
-        if (owner) owner[pv] = P + i;
-        if (eps_out && q + (i < r ? 1 : 0) == 0) eps_out[(size_t)b * P + i] = __int_as_float(0x7fc00000);
-    }
-    __syncthreads();
+    const int Pv = mark_pivots(pivot_idx + (size_t)b * P, P, n_vis, keep, owner, &warp_tot[0]);
+    const int q = (n_keep - Pv) / P, r = (n_keep - Pv) % P;
+    if (eps_out)
+        for (int i = threadIdx.x; i < P; i += blockDim.x)
+            if (q + (i < r ? 1 : 0) == 0) eps_out[(size_t)b * P + i] = __int_as_float(0x7fc00000);
     // rounds: stage the lists of as many pivots as fit, then warp 0 takes their turns in rank order
     const int n_active = q > 0 ? P : r; // pivots with a quota (all later ones keep nothing)
     for (int i0 = 0; i0 < n_active;) {

@@ -41,7 +41,7 @@ class dart_opts(ctypes.Structure):
     _fields_ = [("norm_kind", ctypes.c_int32), ("pivot_smallest", ctypes.c_int32), ("path", ctypes.c_int32),
                 ("wait_limit", ctypes.c_int32), ("sweep_lag", ctypes.c_int32),
                 ("test_withhold_pivots", ctypes.c_int32), ("retention", ctypes.c_int32), ("rule", ctypes.c_int32),
-                ("cosine_on_hidden", ctypes.c_int32), ("pivots_in", ctypes.c_void_p)]
+                ("cosine_on_hidden", ctypes.c_int32), ("text_pivots", ctypes.c_int32), ("pivots_in", ctypes.c_void_p)]
 
 
 class dart_debug(ctypes.Structure):

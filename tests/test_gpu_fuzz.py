@@ -45,8 +45,9 @@ def test_random_shapes_and_options(oracle, seed):
     piv_t = None if piv is None else torch.from_numpy(piv).cuda()
     ctx = dart.Dart(c["B"], c["S"], c["d"], c["P"], c["Kp"])
     try:
-        opts = dart.dart_opts(c["norm_kind"], c["smallest"], c["path"], 0, 0, 0, c["retention"], c["rule"], int(c["on_hidden"]),
-                              None if piv_t is None else piv_t.data_ptr())
+        opts = dart.dart_opts(norm_kind=c["norm_kind"], pivot_smallest=c["smallest"], path=c["path"], retention=c["retention"],
+                              rule=c["rule"], cosine_on_hidden=int(c["on_hidden"]),
+                              pivots_in=None if piv_t is None else piv_t.data_ptr())
         res = ctx.reduce(h, k, c["vo"], c["nv"], c["P"], c["Kp"], opts=opts, debug=True)
         torch.cuda.synchronize()
         assert ctx.status() == dart.DART_OK, (c, dart.dart_status_detail(ctx.handle))

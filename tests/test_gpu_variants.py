@@ -15,13 +15,14 @@ pytestmark = pytest.mark.gpu
 
 
 def run(keys, hidden, vo, nv, P, Kp, path, pivots=None, rule=dart.DART_RULE_QUOTAS, expect_status=dart.DART_OK,
-        on_hidden=False):
+        on_hidden=False, text=False):
     B, S, d = hidden.shape
     if path in (dart.DART_PATH_FUSED, dart.DART_PATH_TWO_PASS) and (d % 64 or P > 256):
         pytest.skip("the tensor-core paths need d % 64 == 0 and at most 256 pivots")
     ctx = dart.Dart(B, S, d, P, Kp)
     try:
-        opts = dart.dart_opts(0, 0, path, 0, 0, 0, 0, rule, int(on_hidden), None if pivots is None else pivots.data_ptr())
+        opts = dart.dart_opts(path=path, rule=rule, cosine_on_hidden=int(on_hidden), text_pivots=int(text),
+                              pivots_in=None if pivots is None else pivots.data_ptr())
         res = ctx.reduce(hidden, keys, vo, nv, P, Kp, opts=opts, debug=True)
         torch.cuda.synchronize()
         st = ctx.status()
@@ -154,7 +155,7 @@ def test_cosine_on_hidden_needs_the_l1_score():
     k, h = gaussian(1, 64, 64, seed=53)
     ctx = dart.Dart(1, 64, 64, 2, 8)
     with pytest.raises(dart.DartError) as e:
-        ctx.reduce(h, k, 0, 64, 2, 8, opts=dart.dart_opts(2, 0, 0, 0, 0, 0, 0, 0, 1, None))
+        ctx.reduce(h, k, 0, 64, 2, 8, opts=dart.dart_opts(norm_kind=2, cosine_on_hidden=1))
     assert e.value.code == dart.DART_ERR_UNSUPPORTED
     ctx.close()
 
@@ -163,7 +164,7 @@ def test_unknown_rule_is_rejected():
     k, h = gaussian(1, 64, 64, seed=43)
     ctx = dart.Dart(1, 64, 64, 2, 8)
     with pytest.raises(dart.DartError) as e:
-        ctx.reduce(h, k, 0, 64, 2, 8, opts=dart.dart_opts(0, 0, 0, 0, 0, 0, 0, 7, 0, None))
+        ctx.reduce(h, k, 0, 64, 2, 8, opts=dart.dart_opts(rule=7))
     assert e.value.code == dart.DART_ERR_UNSUPPORTED
     ctx.close()
 
@@ -219,3 +220,130 @@ def test_gather_rows_argument_checks():
     assert dart.dart_gather_rows(P(src), P(idx), 2, 10, 4, 16, P(src), 0, None) == dart.DART_ERR_ALIAS
     assert dart.dart_gather_rows(P(src), P(idx), 2, 10, 4, 16, P(out), 0, None) == dart.DART_OK
     torch.cuda.synchronize()
+
+
+# ----------------------------------------------------------------------------- pivots taken from the text tokens (Sec. 5.4)
+
+def text_pivots(B, vo, nv, S, P, seed, n_text=None):
+    """Distinct pivots anywhere in the sample, relative to the vision block; at least one text token when there is one."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(B):
+        p = rng.permutation(S)[:P] - vo
+        text = np.concatenate([np.arange(-vo, 0), np.arange(nv, S - vo)])
+        if len(text) and not ((p < 0) | (p >= nv)).any():
+            p[rng.integers(P)] = rng.choice(text)
+        if n_text == "all":
+            p = rng.permutation(text)[:P]
+        out.append(p)
+    return np.stack(out).astype(np.int32)
+
+
+TEXT_SHAPES = [
+    (2, 120, 64, 9, 100, 4, 30),
+    (2, 700, 4096, 40, 576, 8, 64),      # the LLaVA-1.5 shape
+    (1, 3000, 512, 60, 2880, 16, 320),   # the LLaVA-NeXT token count
+    (2, 700, 512, 30, 640, 128, 320),    # the compact pivot tile
+    (1, 400, 3584, 0, 333, 40, 100),     # text after the vision block only
+    (3, 96, 64, 20, 60, 6, 6),           # n_keep = P: text pivots free budget for their own picks
+]
+
+
+@pytest.mark.parametrize("path", [dart.DART_PATH_AUTO, dart.DART_PATH_FUSED], ids=PATH_IDS.get)
+@pytest.mark.parametrize("retention", [dart.DART_RETAIN_SERIAL, dart.DART_RETAIN_LISTS], ids=["serial", "lists"])
+@pytest.mark.parametrize("shape", TEXT_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_pivots_from_the_text_tokens(oracle, shape, retention, path):
+    B, S, d, vo, nv, P, Kp = shape
+    k, h = gaussian(B, S, d, seed=400 + sum(shape))
+    piv = text_pivots(B, vo, nv, S, P, seed=sum(shape))
+    ctx = dart.Dart(B, S, d, P, Kp)
+    try:
+        piv_t = torch.from_numpy(piv).cuda()
+        res = ctx.reduce(h, k, vo, nv, P, Kp, debug=True,
+                         opts=dart.dart_opts(path=path, retention=retention, text_pivots=1, pivots_in=piv_t.data_ptr()))
+        torch.cuda.synchronize()
+        assert ctx.status() == dart.DART_OK, dart.dart_status_detail(ctx.handle)
+    finally:
+        ctx.close()
+    oh, oi, op = _np(res[0]), _np(res[1]), _np(res[2])
+    dbg = {n: _np(v) for n, v in res[3].items()}
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=piv, text_pivots=True)
+    assert np.array_equal(dbg["pivot_idx"], piv)
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, dbg=dbg, pivots_given=True, text_pivots=True)
+    assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5
+
+
+def test_text_pivots_only(oracle):
+    """Every pivot a text token: nothing is kept but the pivots' picks, n_keep of them."""
+    B, S, d, vo, nv, P, Kp = 2, 300, 128, 40, 200, 8, 50
+    k, h = gaussian(B, S, d, seed=61)
+    piv = text_pivots(B, vo, nv, S, P, seed=62, n_text="all")
+    oh, oi, op, dbg, _ = run(k, h, vo, nv, P, Kp, dart.DART_PATH_AUTO, pivots=torch.from_numpy(piv).cuda(), text=True)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=piv, text_pivots=True)
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, dbg=dbg, pivots_given=True, text_pivots=True)
+    assert rep.exact >= rep.above_margin and (dbg["owner"] < P).all()
+
+
+def test_vision_pivots_with_the_text_option_change_nothing():
+    k, h = gaussian(2, 200, 64, seed=63)
+    piv = torch.from_numpy(random_pivots(2, 150, 5, seed=64)).cuda()
+    a = run(k, h, 20, 150, 5, 40, dart.DART_PATH_AUTO, pivots=piv)
+    b = run(k, h, 20, 150, 5, 40, dart.DART_PATH_AUTO, pivots=piv, text=True)
+    assert all(np.array_equal(x, y) for x, y in zip(a[:3], b[:3]))
+    assert all(np.array_equal(a[3][n], b[3][n], equal_nan=True) for n in a[3])
+
+
+@pytest.mark.parametrize("fault", ["repeated text", "before the sample", "after the sample"])
+def test_bad_text_pivots_are_reported_not_used(fault):
+    k, h = gaussian(3, 200, 64, seed=65)
+    piv = random_pivots(3, 150, 4, seed=66)
+    piv[0, 1] = -7
+    piv[1, 0] = 160
+    piv[1, 3] = {"repeated text": 160, "before the sample": -21, "after the sample": 180}[fault]
+    *_, detail = run(k, h, 20, 150, 4, 40, dart.DART_PATH_AUTO, pivots=torch.from_numpy(piv).cuda(), text=True,
+                     expect_status=dart.DART_ERR_CHECK)
+    assert detail[1][0] == 100 and detail[1][1] == 1 and detail[1][2] in (0, 3)
+
+
+def test_text_pivots_need_given_pivots_quotas_and_the_tensor_core_path():
+    k, h = gaussian(1, 64, 64, seed=67)
+    piv = torch.zeros(1, 2, dtype=torch.int32, device="cuda")
+    ctx = dart.Dart(1, 64, 64, 2, 8)
+    for o in (dart.dart_opts(text_pivots=1),
+              dart.dart_opts(text_pivots=1, pivots_in=piv.data_ptr(), rule=dart.DART_RULE_GLOBAL),
+              dart.dart_opts(text_pivots=1, pivots_in=piv.data_ptr(), path=dart.DART_PATH_STAGED)):
+        with pytest.raises(dart.DartError) as e:
+            ctx.reduce(h, k, 4, 50, 2, 8, opts=o)
+        assert e.value.code == dart.DART_ERR_UNSUPPORTED
+    ctx.close()
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_text_pivots_random_shapes(oracle, seed):
+    rng = np.random.default_rng(2000 + seed)
+    d = int(rng.choice([64, 128, 192, 320, 512, 1024]))
+    nv = int(rng.integers(1, 500))
+    vo, after = int(rng.integers(0, 40)), int(rng.integers(0, 40))
+    S = vo + nv + after
+    P = int(rng.integers(1, min(S, nv, 40) + 1))
+    Kp = int(rng.integers(P, nv + 1))
+    B = int(rng.integers(1, 4))
+    k, h = gaussian(B, S, d, seed=500 + seed)
+    piv = text_pivots(B, vo, nv, S, P, seed=seed)
+    ctx = dart.Dart(B, S, d, P, Kp)
+    try:
+        piv_t = torch.from_numpy(piv).cuda()
+        res = ctx.reduce(h, k, vo, nv, P, Kp, debug=True,
+                         opts=dart.dart_opts(retention=int(rng.integers(0, 3)), text_pivots=1, pivots_in=piv_t.data_ptr()))
+        torch.cuda.synchronize()
+        assert ctx.status() == dart.DART_OK, dart.dart_status_detail(ctx.handle)
+    finally:
+        ctx.close()
+    oh, oi, op = _np(res[0]), _np(res[1]), _np(res[2])
+    dbg = {n: _np(v) for n, v in res[3].items()}
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=piv, text_pivots=True)
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, dbg=dbg, pivots_given=True, text_pivots=True)
+    assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5, (B, S, d, vo, nv, P, Kp)
