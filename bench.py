@@ -78,6 +78,7 @@ def kernel_bytes_per_launch(name, w, B):
         "sim": keys + 4 * w.n_pivot * w.n_vis * B,
         "sweep": keys,                       # fused scores + pivots + similarities: the keys count once
         "onepass": keys,                     # the caller's pivots: scores + similarities from one pass
+        "resident": keys,                    # scores + pivots + similarities, rows held on the chip: one read
         "gather": 2 * (2 * w.d * w.S_out) * B,
         "pivot": 4 * w.n_vis * B,
         "retain": 4 * w.n_pivot * w.n_vis * B + 12 * w.S_out * B,

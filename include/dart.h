@@ -59,6 +59,11 @@ enum {
                               scores' sums of squares and similarities from one tensor-core pass; same limits as FUSED.
                               Reads the keys twice like FUSED but has no waits between CTAs: faster for small batches. */
 
+#define DART_PATH_RESIDENT 4 /* steps 1-3 from ONE read of the keys: every sample is spread over all SMs and stays in their
+                              shared and tensor memory until its pivots are known.  Needs n_pivot <= 8, d % 64 == 0,
+                              d <= 4096, n_vis <= 32 rows per SM (and the pivots chosen by score, one tensor for
+                              steps 1-3), else UNSUPPORTED. */
+
 /* dart_opts.retention */
 #define DART_RETAIN_AUTO 0   /* two phases when the batch alone cannot fill the GPU, else one kernel */
 #define DART_RETAIN_SERIAL 1 /* one kernel, one CTA per sample: the pivots' selections one after the other */

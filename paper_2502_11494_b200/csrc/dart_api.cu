@@ -10,11 +10,12 @@
 #include "dart_staged.cuh"
 #include "dart_sweep.cuh"
 #include "dart_onepass.cuh"
+#include "dart_resident.cuh"
 
 namespace {
 
-enum Slot { SLOT_SCORE = 0, SLOT_PIVOT, SLOT_SIM, SLOT_RETAIN, SLOT_GATHER, SLOT_SWEEP, SLOT_ONEPASS, SLOT_COUNT };
-const char *const kSlotNames[SLOT_COUNT] = {"score", "pivot", "sim", "retain", "gather", "sweep", "onepass"};
+enum Slot { SLOT_SCORE = 0, SLOT_PIVOT, SLOT_SIM, SLOT_RETAIN, SLOT_GATHER, SLOT_SWEEP, SLOT_ONEPASS, SLOT_RESIDENT, SLOT_COUNT };
+const char *const kSlotNames[SLOT_COUNT] = {"score", "pivot", "sim", "retain", "gather", "sweep", "onepass", "resident"};
 
 typedef CUresult (*TensorMapEncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                       const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -61,6 +62,10 @@ struct dart_ctx {
     int *counters;
     size_t counters_bytes;
     TensorMapEncodeFn encode;
+    // resident sweep (csrc/dart_resident.cuh)
+    bool resident_ok;
+    int res_landing;  // landing slots in shared memory
+    uint4 *res_cand;  // [B_max][sm_count][8] candidate records
 };
 
 namespace {
@@ -309,6 +314,24 @@ int fused_setup(dart_ctx *ctx)
         per_sm < 1)
         return DART_ERR_CUDA;
     ctx->fused_ok = true;
+    // the resident sweep: rows of at most 8 KB, two landing slots or more, one CTA per SM
+    ctx->resident_ok = false;
+    if (D.d * 2 <= dart::resident::kMaxRowBytes && ctx->sm_count <= dart::resident::kMaxGrid) {
+        namespace R = dart::resident;
+        const int L = R::landing_slots(D.d, ctx->sm_count, ctx->max_smem_optin);
+        int res_per_sm = 0;
+        if (L >= 2 &&
+            cudaFuncSetAttribute(R::resident_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)R::smem_bytes(D.d, ctx->sm_count, L)) == cudaSuccess &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&res_per_sm, R::resident_kernel, R::kThreads,
+                                                          R::smem_bytes(D.d, ctx->sm_count, L)) == cudaSuccess &&
+            res_per_sm >= 1) {
+            rc = ws_alloc(ctx, &ctx->res_cand, (size_t)D.B_max * ctx->sm_count * R::kMaxP);
+            if (rc != DART_OK) return rc;
+            ctx->res_landing = L;
+            ctx->resident_ok = true;
+        }
+    }
     // the one-pass kernel for the caller's pivots uses the same tensor maps
     if (cudaFuncSetAttribute(dart::onepass::onepass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              ctx->max_smem_optin - dart::onepass::kStaticSmemReserve) != cudaSuccess)
@@ -439,6 +462,46 @@ void launch_gather(dart_ctx *ctx, int B, const void *hidden, int n_vis, int n_ke
                                                      (uint4 *)out_hidden);
 }
 
+// The resident sweep applies when a sample's rows fit the chip: at most 8 pivots and, per CTA, no more octets of one
+// sample than the exchange warp has lane groups and tensor memory has slots.
+bool resident_applies(const dart_ctx *ctx, int n_vis, int P)
+{
+    namespace R = dart::resident;
+    if (!ctx->resident_ok || P > R::kMaxP) return false;
+    const int n_oct = (n_vis + R::kOctRows - 1) / R::kOctRows;
+    const int per_cta = (n_oct + ctx->sm_count - 1) / ctx->sm_count;
+    return per_cta <= R::kMaxOctPerSample && per_cta <= R::tmem_slots(ctx->desc.d);
+}
+
+// Steps 1-3 from one read of the keys (csrc/dart_resident.cuh), then steps 4-5.
+int launch_resident(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, const int64_t *pos_in, int vis_offset,
+                    int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos, const dart_opts &o,
+                    const dart_debug *dbg, cudaStream_t st)
+{
+    namespace R = dart::resident;
+    R::Params p = {};
+    p.B = B, p.S = ctx->S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.d = ctx->desc.d;
+    p.n_oct = (n_vis + R::kOctRows - 1) / R::kOctRows;
+    p.n_slots = R::tmem_slots(ctx->desc.d), p.n_landing = ctx->res_landing;
+    p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest;
+    p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
+    p.keys = (const char *)(keys_in ? keys_in : hidden);
+    p.sim = ctx->sim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
+    p.cand = ctx->res_cand, p.arrived = ctx->counters, p.status = ctx->status;
+    DART_CUDA(ctx, cudaMemsetAsync(ctx->counters, 0, (size_t)B * sizeof(int), st));
+    {
+        Prof pr(ctx, st, SLOT_RESIDENT);
+        void *args[1] = {&p};
+        // every CTA waits for all others (the candidates of a sample come from all of them): co-residency is required
+        DART_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)R::resident_kernel, dim3((unsigned)ctx->sm_count), dim3(R::kThreads),
+                                                   args, R::smem_bytes(ctx->desc.d, ctx->sm_count, p.n_landing), st));
+    }
+    launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
+    launch_gather(ctx, B, hidden, n_vis, n_keep, out_idx, out_hidden, st);
+    DART_CUDA(ctx, cudaGetLastError());
+    return copy_debug(ctx, B, n_vis, P, dbg, st);
+}
+
 // The caller's pivots: scores and similarities from one read of the keys, then steps 4-5.
 int launch_onepass(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, const int64_t *pos_in, int vis_offset,
                    int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos, const dart_opts &o,
@@ -508,6 +571,11 @@ int launch_reduce(dart_ctx *ctx, int B, const void *hidden, const void *keys, co
 {
     const bool fused = o.path == DART_PATH_FUSED || (o.path == DART_PATH_AUTO && fused_applies(ctx, P));
     if (fused && !fused_applies(ctx, P)) return DART_ERR_UNSUPPORTED;
+    if (o.path == DART_PATH_RESIDENT) {
+        if (!resident_applies(ctx, n_vis, P) || o.pivots_in || (o.cosine_on_hidden && keys && keys != hidden))
+            return DART_ERR_UNSUPPORTED;
+        return launch_resident(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o, dbg, st);
+    }
     if (o.text_pivots && !fused) return DART_ERR_UNSUPPORTED; // only the tensor-core kernel takes a text row's norm from the row
     if (o.cosine_on_hidden && keys && keys != hidden)
         return launch_two_pass(ctx, B, hidden, keys, hidden, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o,
@@ -654,6 +722,7 @@ int dart_destroy(dart_ctx *ctx)
     cudaFree(ctx->piv_rows);
     cudaFree(ctx->status);
     cudaFree(ctx->counters);
+    cudaFree(ctx->res_cand);
     for (int k = 0; k < 2; ++k) {
         cudaFree(ctx->st_hidden[k]);
         cudaFree(ctx->st_keys[k]);
@@ -690,7 +759,8 @@ int dart_reduce_ex(dart_ctx *ctx, const void *hidden, const void *keys, const in
     if (opts) o = *opts;
     if (o.norm_kind == 0) o.norm_kind = 1;
     if (o.norm_kind != 1 && o.norm_kind != 2) return DART_ERR_UNSUPPORTED;
-    if (o.path != DART_PATH_AUTO && o.path != DART_PATH_STAGED && o.path != DART_PATH_FUSED && o.path != DART_PATH_TWO_PASS)
+    if (o.path != DART_PATH_AUTO && o.path != DART_PATH_STAGED && o.path != DART_PATH_FUSED && o.path != DART_PATH_TWO_PASS &&
+        o.path != DART_PATH_RESIDENT)
         return DART_ERR_UNSUPPORTED;
     if (o.rule != DART_RULE_QUOTAS && o.rule != DART_RULE_GLOBAL) return DART_ERR_UNSUPPORTED;
     if (o.cosine_on_hidden && o.norm_kind != 1) return DART_ERR_UNSUPPORTED; // the hidden rows' sums of squares take the slot
