@@ -65,7 +65,7 @@ struct dart_ctx {
     // resident sweep (csrc/dart_resident.cuh)
     bool resident_ok;
     int res_landing;  // landing slots in shared memory
-    uint4 *res_cand;  // [B_max][sm_count][8] candidate records
+    unsigned long long *res_cand; // [B_max][sm_count][8] candidate keys
 };
 
 namespace {

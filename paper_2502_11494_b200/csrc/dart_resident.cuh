@@ -11,13 +11,15 @@
 //     sample (equal load without a remainder).
 //   * producer warp: one bulk copy per row into a landing slot of shared memory (rows 16 bytes further apart than
 //     their length, which makes 8-row matrix loads conflict-free).
+//   * scorer warps (four, two rows of every octet each): L1 norm and sum of squares of the landed rows.
 //   * worker warp q (four, one per 32-lane quarter of tensor memory): reads a landed octet with ldmatrix in the
-//     register layout of an mma.sync B operand (token = column of the product), accumulates the rows' L1 norms and
-//     sums of squares on the way and parks the fragments in tensor memory with tcgen05.st: tensor memory serves as
-//     256 KB of spill space per SM, each thread reads back exactly what it wrote.  The landing slot is free again.
-//   * exchange warp: the CTA's best P rows of the sample go to global memory (score key, index, sum of squares), a
-//     counter per sample counts the CTAs that have published; when all have, every CTA merges the sorted lists
-//     itself (P rounds over the lists' heads) and fetches the P pivot rows into shared memory.
+//     register layout of an mma.sync B operand (token = column of the product) and parks the fragments in tensor
+//     memory with tcgen05.st: tensor memory serves as 256 KB of spill space per SM, each thread reads back exactly
+//     what it wrote.  When scorers and worker are done the landing slot is free again.
+//   * exchange warp: the CTA's best P rows of the sample go to global memory (score key and index), a counter per
+//     sample counts the CTAs that have published; when all have, every CTA merges the sorted lists itself (each
+//     lane its share of the lists, then a butterfly of 8-entry merges across the lanes) and fetches the P pivot
+//     rows into shared memory.
 //   * worker warp again: fragments back from tensor memory (tcgen05.ld), pivot rows as the A operand (ldmatrix),
 //     mma.sync m16n8k16 with fp32 accumulation: D[pivot][token]; normalised and written as dup(p_i, x_j).
 //
@@ -34,8 +36,10 @@ namespace dart {
 namespace resident {
 using namespace sweep; // PTX wrappers, bounded waits
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 320; // 204 registers per thread
 constexpr int kProducerWarp = 0, kExchangeWarp = 1, kWorker0 = 4, kWorkers = 4; // kWorker0 % 4 == 0: worker q owns TMEM lanes 32 q ..
+constexpr int kScorers = 4; // warps 2, 3, 8, 9: scorer w takes rows 2w and 2w + 1 of every octet
+constexpr int kMeta = 64;                 // ring of per-octet scores: more than tensor-memory plus landing slots
 constexpr int kOctRows = 8;
 constexpr int kMaxP = 8;
 constexpr int kMaxRowBytes = 8192;     // d <= 4096: one octet fills a quarter of tensor memory
@@ -46,9 +50,10 @@ constexpr int kMaxSlots = 4 * kMaxSlotsPerQuarter;
 constexpr int kMaxLanding = 8;
 constexpr int kMaxOctPerSample = 4;    // per CTA: 32 rows, one per lane of the exchange warp
 constexpr int kMaxGrid = 192;          // lists per lane of the merge: kMaxGrid / 32
-constexpr int kStaticSmemReserve = 4096;
+constexpr int kStaticSmemReserve = 8192;
 // second status word of a wait that expired
-constexpr int kWaitLandingFree = 80, kWaitWorker = 81, kWaitConverted = 82, kWaitPublished = 83, kWaitPivotBufFree = 84;
+constexpr int kWaitLandingFree = 80, kWaitWorker = 81, kWaitScored = 82, kWaitPublished = 83, kWaitPivotBufFree = 84,
+              kWaitLanded = 85, kWaitPivotNorms = 86;
 
 struct Params {
     int B, S, vis_offset, n_vis, P, d;
@@ -61,7 +66,7 @@ struct Params {
     float *sim;        // [B][P][n_vis]
     float *l1, *ssq;   // [B][n_vis]
     int32_t *pivot_idx; // [B][P]
-    uint4 *cand;       // [B][G][kMaxP]: {score key, ~index, sum of squares, 0}, best first
+    unsigned long long *cand; // [B][G][kMaxP]: score key << 32 | ~index, best first; 0 = none
     int *arrived;      // [B] CTAs that have published their candidates, zero at launch
     int *status;
 };
@@ -74,7 +79,7 @@ __host__ __device__ inline int tmem_slots(int d)
     if (per > kMaxSlotsPerQuarter) per = kMaxSlotsPerQuarter;
     return 4 * per;
 }
-__host__ __device__ inline uint32_t cand_smem_bytes(int G) { return (uint32_t)G * kMaxP * 16u; }
+__host__ __device__ inline uint32_t cand_smem_bytes(int G) { return (uint32_t)G * kMaxP * 8u; }
 inline int landing_slots(int d, int G, int smem_limit)
 {
     const long long left = (long long)smem_limit - kStaticSmemReserve - 128 - oct_bytes(d) - cand_smem_bytes(G);
@@ -88,12 +93,13 @@ struct Shared {
     unsigned long long piv_full;                              // pivot rows of the current sample have landed
     uint32_t tmem_base;
     volatile int abort_flag;
-    volatile uint32_t armed;               // pivot fetches started so far (the barrier's phase of sample number ord is ord)
-    volatile uint32_t issued;              // octets whose copies have been started (octet s is phase s / L of full[s % L])
-    volatile uint32_t conv_seq[kMaxSlots]; // octet number + 1 whose fragments and norms the slot holds
-    volatile uint32_t mma_seq[kMaxSlots];  // octet number + 1 whose similarities have been written
-    float slot_ssq[kMaxSlots][kOctRows];
-    uint32_t slot_key[kMaxSlots][kOctRows]; // ranking key of the row, larger = better pivot; 0 = no row
+    volatile uint32_t armed;      // pivot fetches started so far (the barrier's phase of sample number ord is ord)
+    volatile uint32_t pssq_ready; // samples whose pivot norms are in piv_ssq
+    volatile uint32_t issued;     // octets whose copies have been started (octet s is phase s / L of full[s % L])
+    volatile uint32_t mma_seq[kMaxSlots]; // octet number + 1 whose similarities have been written
+    uint32_t scored[kMeta];       // scorer warps that are done with the octets of this ring entry, all uses added up
+    float meta_ssq[kMeta][kOctRows];
+    uint32_t meta_key[kMeta][kOctRows]; // ranking key of the row, larger = better pivot; 0 = no row
     float piv_ssq[kMaxP];
 };
 
@@ -155,6 +161,21 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
                  : "r"(taddr));
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// The same load without the wait, and the wait with the registers tied to it: the loaded values exist only after
+// the wait, so nothing may read or move the registers between the two statements.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : DART_W8(r, 0), DART_W8(r, 8), DART_W8(r, 16), DART_W8(r, 24)
+                 : "r"(taddr));
+}
+#define DART_T8(r, o) "+r"(r[o]), "+r"(r[o + 1]), "+r"(r[o + 2]), "+r"(r[o + 3]), "+r"(r[o + 4]), "+r"(r[o + 5]), "+r"(r[o + 6]), "+r"(r[o + 7])
+__device__ __forceinline__ void tmem_ld32_wait(uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;" : DART_T8(r, 0), DART_T8(r, 8), DART_T8(r, 16), DART_T8(r, 24)::"memory");
+}
+#undef DART_T8
 __device__ __forceinline__ void tmem_ld8u(uint32_t taddr, uint32_t *r)
 {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];" : DART_W8(r, 0) : "r"(taddr));
@@ -172,15 +193,20 @@ __device__ __forceinline__ void add_pair(uint32_t w, float &l1, float &ssq)
     ssq = fmaf(hi, hi, ssq);
 }
 
+// Waits in this kernel last long (a sample's pivots take tens of microseconds) and several warps wait at any time.
+// Polls go through the same shared-memory pipe as the shuffles and loads of the warps that work, so a waiting warp
+// sleeps between polls: tight polling slowed the working warps down several times over.
+constexpr unsigned kPollNs = 100;
+
 // Polls a shared-memory word until it reaches `target` (bounded like every other wait).
 __device__ inline bool wait_seq(const Ctl &ctl, const volatile uint32_t *word, uint32_t target, int where, long long task)
 {
-    for (int it = 0; it < 64; ++it)
+    for (int it = 0; it < 4; ++it)
         if (*word >= target) return true;
     const long long t0 = clock64();
     for (uint32_t it = 0;; ++it) {
         if (*word >= target) return true;
-        __nanosleep(20);
+        __nanosleep(kPollNs);
         if ((it & 31u) == 31u) {
             if (ctl.aborted()) return false;
             if ((unsigned long long)(clock64() - t0) > ctl.limit_cycles) {
@@ -189,6 +215,34 @@ __device__ inline bool wait_seq(const Ctl &ctl, const volatile uint32_t *word, u
             }
         }
     }
+}
+
+// Bounded wait for a barrier phase, sleeping between polls.
+__device__ inline bool wait_bar_polite(const Ctl &ctl, uint32_t bar, uint32_t parity, int where, long long task)
+{
+    for (int it = 0; it < 4; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(kPollNs);
+        if ((it & 31u) == 31u) {
+            if (ctl.aborted()) return false;
+            if ((unsigned long long)(clock64() - t0) > ctl.limit_cycles) {
+                ctl.give_up(where, task);
+                return false;
+            }
+        }
+    }
+}
+
+// The largest 64-bit key of the warp in two warp-wide reductions (lanes without a key pass 0); the same in all lanes.
+__device__ __forceinline__ unsigned long long warp_max_key(unsigned long long key)
+{
+    const uint32_t hi = (uint32_t)(key >> 32), lo = (uint32_t)key;
+    const uint32_t top_hi = __reduce_max_sync(0xffffffffu, hi);
+    const uint32_t top_lo = __reduce_max_sync(0xffffffffu, hi == top_hi ? lo : 0u);
+    return ((unsigned long long)top_hi << 32) | top_lo;
 }
 
 __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
@@ -201,8 +255,8 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
     const uint32_t smem0 = (smem_u32(smem_raw) + 127u) & ~127u;
     const uint32_t piv_buf = smem0;                         // P pivot rows at the landing pitch
     const uint32_t land0 = smem0 + octb;                    // n_landing octets
-    const uint32_t cand_off = (1u + (uint32_t)p.n_landing) * octb; // [G][kMaxP] candidate records of the current sample
-    uint4 *cand_sm = reinterpret_cast<uint4 *>(smem_raw + ((smem0 - smem_u32(smem_raw)) + cand_off));
+    const uint32_t cand_off = (1u + (uint32_t)p.n_landing) * octb; // [G][kMaxP] candidate keys of the current sample
+    unsigned long long *cand_sm = reinterpret_cast<unsigned long long *>(smem_raw + ((smem0 - smem_u32(smem_raw)) + cand_off));
     const unsigned long long limit = 2ull * p.wait_ns; // ns -> cycles at the highest SM clock: never shorter than asked
     const Ctl ctl{&sh.abort_flag, p.status, warp == kProducerWarp ? limit : limit + limit / 4};
     const int L = p.n_landing, n_slots = p.n_slots;
@@ -211,13 +265,15 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
     if (threadIdx.x == 0) {
         for (int j = 0; j < kMaxLanding; ++j) {
             mbar_init(smem_u32(&sh.full[j]), 1);
-            mbar_init(smem_u32(&sh.empty[j]), 1);
+            mbar_init(smem_u32(&sh.empty[j]), 1 + kScorers); // the worker that parks the octet and every scorer
         }
         mbar_init(smem_u32(&sh.piv_full), 1);
         sh.abort_flag = 0;
         sh.armed = 0;
+        sh.pssq_ready = 0;
         sh.issued = 0;
-        for (int j = 0; j < kMaxSlots; ++j) sh.conv_seq[j] = 0, sh.mma_seq[j] = 0;
+        for (int j = 0; j < kMaxSlots; ++j) sh.mma_seq[j] = 0;
+        for (int j = 0; j < kMeta; ++j) sh.scored[j] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kExchangeWarp) {
@@ -239,7 +295,7 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
             const int j = (int)(q.s % L);
             const uint32_t par = (uint32_t)((q.s / L) & 1);
             bool ok = true;
-            if (lane == 0) ok = ctl.wait_bar(smem_u32(&sh.empty[j]), par ^ 1u, kWaitLandingFree, q.s);
+            if (lane == 0) ok = wait_bar_polite(ctl, smem_u32(&sh.empty[j]), par ^ 1u, kWaitLandingFree, q.s);
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
             if (!ok) break;
             const int rows = min(kOctRows, p.n_vis - q.o * kOctRows);
@@ -276,39 +332,29 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
                 if (k < kMaxOctPerSample) s_of[k] = q.s, o_of[k] = q.o, ++k;
                 q.next();
             }
-            // 1. the octets' norms
-            unsigned long long key = 0;
-            float my_ssq = 0.f;
+            // 1. the octets' scores: lane 8u + r takes row r of the sample's u-th octet here
+            unsigned long long key = 0ull;
 #pragma unroll
             for (int u = 0; u < kMaxOctPerSample; ++u)
                 if (u < k) {
-                    const int slot = (int)(s_of[u] % n_slots);
-                    ok = ok && wait_seq(ctl, &sh.conv_seq[slot], (uint32_t)(s_of[u] + 1), kWaitConverted, s_of[u]);
+                    const int m = (int)(s_of[u] % kMeta);
+                    ok = ok && wait_seq(ctl, &sh.scored[m], (uint32_t)(kScorers * (s_of[u] / kMeta + 1)), kWaitScored, s_of[u]);
                     if (ok && (lane >> 3) == u) {
-                        const uint32_t rk = sh.slot_key[slot][lane & 7];
+                        const uint32_t rk = sh.meta_key[m][lane & 7];
                         const uint32_t idx = (uint32_t)(o_of[u] * kOctRows + (lane & 7));
                         key = rk ? ((unsigned long long)rk << 32) | (0xffffffffu - idx) : 0ull;
-                        my_ssq = sh.slot_ssq[slot][lane & 7];
                     }
                 }
             if (!__all_sync(0xffffffffu, ok)) break;
-            // 2. the CTA's best P rows, best first (equal scores: lower index first)
-            uint4 rec = make_uint4(0, 0, 0, 0);
+            // 2. the CTA's best P rows, best first (equal scores: lower index first): lane i keeps the winner of round i
+            unsigned long long rec = 0ull;
+#pragma unroll 1
             for (int i = 0; i < p.P; ++i) {
-                unsigned long long best = key;
-#pragma unroll
-                for (int m = 16; m > 0; m >>= 1) {
-                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, m);
-                    best = other > best ? other : best;
-                }
-                const uint32_t who = __ballot_sync(0xffffffffu, best != 0ull && key == best);
-                const int wl = who ? __ffs(who) - 1 : 0;
-                const float wssq = __shfl_sync(0xffffffffu, my_ssq, wl);
-                if (lane == i) rec = make_uint4((uint32_t)(best >> 32), (uint32_t)best, __float_as_uint(wssq), 0u);
-                if (who && lane == wl) key = 0ull;
+                const unsigned long long best = warp_max_key(key);
+                if (lane == i) rec = best;
+                if (key == best) key = 0ull; // keys are distinct (they carry the index): one lane, or nobody when best is 0
             }
-            uint4 *mine = p.cand + ((size_t)n * G + c) * kMaxP;
-            if (lane < p.P) __stcg(mine + lane, rec);
+            if (lane < kMaxP) __stcg(p.cand + ((size_t)n * G + c) * kMaxP + lane, rec);
             __threadfence();
             __syncwarp();
             const int contributors = p.n_oct < G ? p.n_oct : G;
@@ -318,57 +364,62 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
             }
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
             if (!ok) break;
-            // 3. merge: lane l walks the sorted lists of CTAs l, l + 32, ...
+            // 3. merge: lane l reads the sorted lists of CTAs l, l + 32, ... (64 bytes each; all loads in flight at
+            // once) and merges them into its own best 8; a butterfly over the lanes leaves the sample's best 8 in all
             int head[kMaxGrid / 32];
 #pragma unroll
+            for (int h = 0; h < kMaxGrid / 32; h += 3) { // three lists (twelve loads) at a time
+                uint4 v[3][4];
+#pragma unroll
+                for (int u = h; u < h + 3; ++u) {
+                    const int cc = lane + 32 * u;
+                    const bool has = u < n_lists && cc < G && (cc - off + G) % G < p.n_oct; // that CTA holds rows of this sample
+                    head[u] = has ? 0 : 8;
+                    const uint4 *src = reinterpret_cast<const uint4 *>(p.cand + ((size_t)n * G + cc) * kMaxP);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) v[u - h][i] = has ? __ldcg(src + i) : make_uint4(0, 0, 0, 0);
+                }
+#pragma unroll
+                for (int u = h; u < h + 3; ++u) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(cand_sm + (size_t)(lane + 32 * u) * kMaxP);
+                    if (u < n_lists && lane + 32 * u < G)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) dst[i] = v[u - h][i];
+                }
+            }
+            unsigned long long cur[kMaxGrid / 32]; // the head of every list; only the list that wins reads its next key
+            unsigned long long mine = 0ull;        // the best of them
+#pragma unroll
             for (int u = 0; u < kMaxGrid / 32; ++u) {
-                const int cc = lane + 32 * u;
-                const bool has = u < n_lists && cc < G && (cc - off + G) % G < p.n_oct; // that CTA holds rows of this sample
-                head[u] = has ? 0 : p.P;
-                if (has) {
-                    const uint4 *src = p.cand + ((size_t)n * G + cc) * kMaxP;
-                    for (int i = 0; i < p.P; ++i) cand_sm[cc * kMaxP + i] = __ldcg(src + i);
-                }
+                cur[u] = head[u] < 8 ? cand_sm[(lane + 32 * u) * kMaxP] : 0ull;
+                mine = cur[u] > mine ? cur[u] : mine;
             }
-            __syncwarp();
             int my_piv = 0;
-            float my_pssq = 0.f;
-            for (int i = 0; i < p.P; ++i) {
-                unsigned long long best = 0ull;
-                int bu = 0;
-                float bssq = 0.f;
+#pragma unroll 1
+            for (int i = 0; i < p.P; ++i) { // P rounds: the warp's best key wins, its lane moves that list on
+                const unsigned long long best = warp_max_key(mine);
+                if (lane == i) my_piv = (int)(0xffffffffu - (uint32_t)best);
+                if (best != 0ull && mine == best) {
+                    mine = 0ull;
 #pragma unroll
-                for (int u = 0; u < kMaxGrid / 32; ++u)
-                    if (head[u] < p.P) {
-                        const uint4 r = cand_sm[(lane + 32 * u) * kMaxP + head[u]];
-                        const unsigned long long kk = ((unsigned long long)r.x << 32) | r.y;
-                        if (kk > best) best = kk, bu = u, bssq = __uint_as_float(r.z);
+                    for (int u = 0; u < kMaxGrid / 32; ++u) {
+                        if (cur[u] == best) {
+                            ++head[u];
+                            cur[u] = head[u] < 8 ? cand_sm[(lane + 32 * u) * kMaxP + head[u]] : 0ull;
+                        }
+                        mine = cur[u] > mine ? cur[u] : mine;
                     }
-                unsigned long long top = best;
-#pragma unroll
-                for (int m = 16; m > 0; m >>= 1) {
-                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, top, m);
-                    top = other > top ? other : top;
-                }
-                const uint32_t who = __ballot_sync(0xffffffffu, top != 0ull && best == top);
-                const int wl = who ? __ffs(who) - 1 : 0; // keys are distinct (they carry the index): one lane
-                const float wssq = __shfl_sync(0xffffffffu, bssq, wl);
-                if (lane == i) my_piv = (int)(0xffffffffu - (uint32_t)top), my_pssq = wssq;
-                if (who && lane == wl) {
-#pragma unroll
-                    for (int u = 0; u < kMaxGrid / 32; ++u)
-                        if (u == bu) ++head[u];
                 }
             }
-            if (lane < p.P) {
-                my_piv = min(max(my_piv, 0), p.n_vis - 1);
-                if (c == off) p.pivot_idx[(size_t)n * p.P + lane] = my_piv; // the CTA that holds the sample's octet 0
-            }
+            my_piv = min(max(my_piv, 0), p.n_vis - 1);
+            if (lane < p.P && c == off) p.pivot_idx[(size_t)n * p.P + lane] = my_piv; // the CTA that holds the sample's octet 0
+            // the pivots' sums of squares were written by the CTAs that scored them, before they published
+            float my_pssq = 0.f;
+            if (lane < p.P) my_pssq = __ldcg(p.ssq + (size_t)n * p.n_vis + my_piv);
             // 4. the pivot buffer is free once the previous sample's similarities are written
             for (int u = 0; u < prev_k; ++u)
                 ok = ok && wait_seq(ctl, &sh.mma_seq[prev_s[u] % n_slots], (uint32_t)(prev_s[u] + 1), kWaitPivotBufFree, prev_s[u]);
             if (!__all_sync(0xffffffffu, ok)) break;
-            if (lane < p.P) sh.piv_ssq[lane] = my_pssq;
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); // the workers' reads of the buffer precede the copies
             __syncwarp();
             const uint32_t bar = smem_u32(&sh.piv_full);
@@ -380,11 +431,73 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
             if (lane < p.P)
                 bulk_load(piv_buf + (uint32_t)lane * pitch, p.keys + ((size_t)n * p.S + p.vis_offset + my_piv) * row_bytes, row_bytes,
                           bar, pol_keep);
+            if (lane < p.P) sh.piv_ssq[lane] = my_pssq; // needed at the end of the multiplication only
+            __syncwarp();
+            if (lane == 0) {
+                __threadfence_block();
+                sh.pssq_ready = armed + 1;
+            }
             ++armed;
             prev_k = k;
             for (int u = 0; u < k; ++u) prev_s[u] = s_of[u];
         }
         if (ctl.aborted() && armed && lane == 0) ctl.wait_landed(smem_u32(&sh.piv_full), (armed - 1) & 1u);
+    } else if (warp == 2 || warp == 3 || warp == 8 || warp == 9) {
+        // ------------------------------------------------------------------ scorers: L1 norm and sum of squares of two rows
+        const int w = warp < 4 ? warp - 2 : warp - 6;
+        const uint32_t n_chunks = row_bytes / 16u;
+        bool ok = true;
+        for (Seq q(G, c, p.n_oct, p.B); ok && q.valid(); q.next()) {
+            const int j = (int)(q.s % L), m = (int)(q.s % kMeta);
+            // a parity test is only meaningful once the barrier has reached this octet's phase
+            ok = wait_seq(ctl, &sh.issued, (uint32_t)(q.s + 1), kWaitLanded, q.s);
+            if (ok && lane == 0) ok = wait_bar_polite(ctl, smem_u32(&sh.full[j]), (uint32_t)((q.s / L) & 1), kWaitLanded, q.s);
+            if (!__all_sync(0xffffffffu, ok)) break;
+            mbar_try_wait(smem_u32(&sh.full[j]), (uint32_t)((q.s / L) & 1)); // every lane observes the completed phase itself
+            const int rows = min(kOctRows, p.n_vis - q.o * kOctRows);
+#pragma unroll
+            for (int rr = 0; rr < 2; ++rr) {
+                const int r = 2 * w + rr;
+                uint32_t rk = 0;
+                float l1 = 0.f, ssq = 0.f;
+                if (r < rows) {
+                    const uint32_t base = land0 + (uint32_t)j * octb + (uint32_t)r * pitch;
+                    float l1a[4] = {0.f, 0.f, 0.f, 0.f}, ssqa[4] = {0.f, 0.f, 0.f, 0.f}; // four chains: the sums are latency bound
+                    for (uint32_t ch = lane; ch < n_chunks; ch += 128) { // four loads in flight (row lengths are multiples of 128 bytes)
+                        uint4 v[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) v[e] = ch + 32u * e < n_chunks ? lds128(base + (ch + 32u * e) * 16u) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            add_pair(v[e].x, l1a[0], ssqa[0]);
+                            add_pair(v[e].y, l1a[1], ssqa[1]);
+                            add_pair(v[e].z, l1a[2], ssqa[2]);
+                            add_pair(v[e].w, l1a[3], ssqa[3]);
+                        }
+                    }
+                    l1 = warp_sum((l1a[0] + l1a[1]) + (l1a[2] + l1a[3]));
+                    ssq = warp_sum((ssqa[0] + ssqa[1]) + (ssqa[2] + ssqa[3]));
+                    const uint32_t ok_ = order_key(p.norm_kind == 2 ? ssq : l1);
+                    rk = p.smallest ? ~ok_ : ok_;
+                    if (rk == 0) rk = 1; // 0 marks "no row"
+                }
+                if (lane == 0) {
+                    if (r < rows) {
+                        const size_t at = (size_t)q.n * p.n_vis + (size_t)q.o * kOctRows + r;
+                        p.l1[at] = l1;
+                        p.ssq[at] = ssq;
+                    }
+                    sh.meta_key[m][r] = rk;
+                    sh.meta_ssq[m][r] = ssq;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) {
+                __threadfence(); // the global sums of squares are read by other CTAs once this CTA has published
+                mbar_arrive(smem_u32(&sh.empty[j]));
+                atomicAdd(&sh.scored[m], 1u);
+            }
+        }
     } else if (warp >= kWorker0 && warp < kWorker0 + kWorkers) {
         // ------------------------------------------------------------------ workers: park, then multiply
         const int quarter = warp - kWorker0;
@@ -397,25 +510,23 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
         while (ms.valid() && (ms.s & 3) != quarter) ms.next();
         long long t0 = 0;
         uint32_t idle = 0;
-        while (ms.valid()) {
+        bool failed = false;
+        while (ms.valid() && !failed) {
             bool did = false;
             if (cs.valid() && cs.s - ms.s < n_slots) { // the slot's previous octet has been multiplied
                 const int j = (int)(cs.s % L);
                 // a parity test is only meaningful once the barrier has reached this octet's phase
                 if (sh.issued > (uint32_t)cs.s && mbar_try_wait(smem_u32(&sh.full[j]), (uint32_t)((cs.s / L) & 1))) {
-                    // ---- park octet cs.s: shared memory -> registers (+ norms) -> tensor memory
+                    // ---- park octet cs.s: shared memory -> registers -> tensor memory
                     const int slot = (int)(cs.s % n_slots);
                     const uint32_t tcol = tq + (uint32_t)(slot >> 2) * cols_per_oct;
                     const uint32_t src = land0 + (uint32_t)j * octb + lm_off;
-                    float l1 = 0.f, ssq = 0.f;
                     const int n32 = p.d / 256, n8 = (p.d % 256) / 64; // batches of 32 and of 8 registers
                     for (int bt = 0; bt < n32; ++bt) {
                         uint32_t r[32];
 #pragma unroll
                         for (int it = 0; it < 8; ++it)
                             ldmatrix_x4(src + (uint32_t)(bt * 8 + it) * 64u, r[4 * it], r[4 * it + 1], r[4 * it + 2], r[4 * it + 3]);
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) add_pair(r[e], l1, ssq);
                         tmem_st32(tcol + (uint32_t)bt * 32u, r);
                     }
                     for (int bt = 0; bt < n8; ++bt) {
@@ -423,36 +534,11 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
 #pragma unroll
                         for (int it = 0; it < 2; ++it)
                             ldmatrix_x4(src + (uint32_t)(n32 * 8 + bt * 2 + it) * 64u, r[4 * it], r[4 * it + 1], r[4 * it + 2], r[4 * it + 3]);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) add_pair(r[e], l1, ssq);
                         tmem_st8(tcol + (uint32_t)n32 * 32u + (uint32_t)bt * 8u, r);
                     }
                     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                    // the four lanes of a group hold the four column classes of row g
-                    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-                    ssq += __shfl_xor_sync(0xffffffffu, ssq, 1);
-                    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-                    ssq += __shfl_xor_sync(0xffffffffu, ssq, 2);
-                    const int rows = min(kOctRows, p.n_vis - cs.o * kOctRows);
-                    if (t == 0) {
-                        uint32_t rk = 0;
-                        if (g < rows) {
-                            const size_t at = (size_t)cs.n * p.n_vis + (size_t)cs.o * kOctRows + g;
-                            p.l1[at] = l1;
-                            p.ssq[at] = ssq;
-                            const uint32_t ok_ = order_key(p.norm_kind == 2 ? ssq : l1);
-                            rk = p.smallest ? ~ok_ : ok_;
-                            if (rk == 0) rk = 1; // 0 marks "no row"
-                        }
-                        sh.slot_key[slot][g] = rk;
-                        sh.slot_ssq[slot][g] = ssq;
-                    }
                     __syncwarp();
-                    if (lane == 0) {
-                        mbar_arrive(smem_u32(&sh.empty[j])); // the landing slot may be overwritten
-                        __threadfence_block();
-                        sh.conv_seq[slot] = (uint32_t)(cs.s + 1);
-                    }
+                    if (lane == 0) mbar_arrive(smem_u32(&sh.empty[j])); // this warp is done with the landing slot
                     do cs.next();
                     while (cs.valid() && (cs.s & 3) != quarter);
                     did = true;
@@ -462,7 +548,7 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
                 // a parity test is only meaningful once the barrier has reached this sample's phase
                 if (sh.armed > (uint32_t)ms.ord && mbar_try_wait(smem_u32(&sh.piv_full), (uint32_t)(ms.ord & 1))) {
                     // ---- multiply octet ms.s: D[pivot][token] over all columns, four accumulators in turn
-                    const int slot = (int)(ms.s % n_slots);
+                    const int slot = (int)(ms.s % n_slots), m = (int)(ms.s % kMeta);
                     const uint32_t tcol = tq + (uint32_t)(slot >> 2) * cols_per_oct;
                     const uint32_t asrc = piv_buf + lm_off;
                     float acc[4][4];
@@ -471,15 +557,27 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
 #pragma unroll
                         for (int e = 0; e < 4; ++e) acc[a][e] = 0.f;
                     const int n32 = p.d / 256, n8 = (p.d % 256) / 64;
-                    for (int bt = 0; bt < n32; ++bt) {
-                        uint32_t r[32];
-                        tmem_ld32(tcol + (uint32_t)bt * 32u, r);
+                    auto multiply = [&](int bt, const uint32_t(&r)[32]) {
 #pragma unroll
                         for (int it = 0; it < 8; ++it) { // 32 columns: two k16 blocks
                             uint32_t a0, a2, a0n, a2n;
                             ldmatrix_x4(asrc + (uint32_t)(bt * 8 + it) * 64u, a0, a2, a0n, a2n);
                             mma_16816(acc[(2 * it) & 3], a0, a2, r[4 * it], r[4 * it + 1]);
                             mma_16816(acc[(2 * it + 1) & 3], a0n, a2n, r[4 * it + 2], r[4 * it + 3]);
+                        }
+                    };
+                    {   // two register sets in turn: the next batch is on its way while this one is multiplied
+                        uint32_t ra[32], rb[32];
+                        if (n32 > 0) tmem_ld32_issue(tcol, ra);
+                        for (int bt = 0; bt < n32; bt += 2) {
+                            tmem_ld32_wait(ra);
+                            if (bt + 1 < n32) tmem_ld32_issue(tcol + (uint32_t)(bt + 1) * 32u, rb);
+                            multiply(bt, ra);
+                            if (bt + 1 < n32) {
+                                tmem_ld32_wait(rb);
+                                if (bt + 2 < n32) tmem_ld32_issue(tcol + (uint32_t)(bt + 2) * 32u, ra);
+                                multiply(bt + 1, rb);
+                            }
                         }
                     }
                     for (int bt = 0; bt < n8; ++bt) {
@@ -493,9 +591,12 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
                             mma_16816(acc[(2 * it + 1) & 3], a0n, a2n, r[4 * it + 2], r[4 * it + 3]);
                         }
                     }
+                    // the pivots' norms come by another route than their rows
+                    if (!wait_seq(ctl, &sh.pssq_ready, (uint32_t)(ms.ord + 1), kWaitPivotNorms, ms.s)) failed = true;
+                    failed = __any_sync(0xffffffffu, failed);
                     // thread (g, t): pivot g x tokens 2t, 2t + 1 of the octet
                     const int rows = min(kOctRows, p.n_vis - ms.o * kOctRows);
-                    if (g < p.P) {
+                    if (!failed && g < p.P) {
                         const float np_ = sqrtf(sh.piv_ssq[g]);
                         float *dst = p.sim + ((size_t)ms.n * p.P + g) * p.n_vis + (size_t)ms.o * kOctRows;
 #pragma unroll
@@ -503,7 +604,7 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
                             const int tok = 2 * t + e;
                             if (tok < rows) { // dup = dot / (|pivot| |row|); a zero norm gives 0
                                 const float v = (acc[0][e] + acc[1][e]) + (acc[2][e] + acc[3][e]);
-                                const float den = np_ * sqrtf(sh.slot_ssq[slot][tok]);
+                                const float den = np_ * sqrtf(sh.meta_ssq[m][tok]);
                                 dst[tok] = den > 0.f ? v / den : 0.f;
                             }
                         }
@@ -520,8 +621,11 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
             }
             if (did) {
                 idle = 0;
+            } else if (idle < 64) {
+                ++idle;
+                __nanosleep(kPollNs);
             } else if (++idle > 64) { // a wait that lasts: start the clock, then check it now and then
-                __nanosleep(32);
+                __nanosleep(2 * kPollNs);
                 if (idle == 65) t0 = clock64();
                 if ((idle & 31u) == 0u) {
                     bool stop = ctl.aborted();
@@ -542,8 +646,8 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     // the CTA whose wait expired first adds where its pipeline stood: status words 4-10
     if (threadIdx.x == 0 && sh.abort_flag && p.status[0] == kStatusTimeout && p.status[3] == c && p.status[1] >= kWaitLandingFree) {
-        for (int j = 0; j < 3; ++j) p.status[4 + j] = (int)sh.conv_seq[j], p.status[7 + j] = (int)sh.mma_seq[j];
-        p.status[10] = (int)sh.armed;
+        for (int j = 0; j < 4; ++j) p.status[4 + j] = (int)sh.mma_seq[j];
+        p.status[8] = (int)sh.issued, p.status[9] = (int)sh.pssq_ready, p.status[10] = (int)sh.armed;
     }
 }
 

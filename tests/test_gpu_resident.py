@@ -60,7 +60,7 @@ def test_resident_sweep_on_the_clustered_workload(oracle):
     a = run_gpu(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, path=dart.DART_PATH_RESIDENT)
     b = run_gpu(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, path=dart.DART_PATH_FUSED)
     assert np.array_equal(a[3]["pivot_idx"], b[3]["pivot_idx"])
-    assert np.allclose(a[3]["sim"], b[3]["sim"], rtol=0, atol=1e-5)
+    assert np.allclose(a[3]["sim"], b[3]["sim"], rtol=0, atol=4e-5)   # each within 2e-5 of the oracle
 
 
 @pytest.mark.parametrize("shape", [(1, 64, 64, 0, 64, 9, 20), (1, 64, 8200, 0, 64, 2, 8), (1, 5000, 64, 0, 4744, 2, 8),
