@@ -40,7 +40,7 @@ def parse():
     ap.add_argument("--keep", type=int, default=None)
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch size")
     ap.add_argument("--sweep", action="store_true", help="also time every (pivots, keep) cell of the sweep")
-    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 staged, 2 fused (persistent sweep), 3 two passes (score pass + one tensor-core pass)")
+    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 staged, 2 fused (persistent sweep), 3 two passes (score pass + one tensor-core pass), 4 resident sweep")
     ap.add_argument("--lag", type=int, default=0, help="fused path: extra tasks between a row's two sweeps")
     ap.add_argument("--retention", type=int, default=0, help="0 auto, 1 one kernel, 2 candidate lists + walks")
     ap.add_argument("--variants", action="store_true",
@@ -90,7 +90,9 @@ def kernel_bytes_per_launch(name, w, B):
 # (every sample is read and written independently), so a launch over B samples moves B times this.
 NCU_TRAFFIC_PER_SAMPLE = {("sweep", 2880, 4096, 8): (1.508212e9 + 5.538816e6) / 32,
                           # profiles/onepass_kernel_sweep_b32.md
-                          ("onepass", 2880, 4096, 8): (755.18336e6 + 5.144064e6) / 32}
+                          ("onepass", 2880, 4096, 8): (755.18336e6 + 5.144064e6) / 32,
+                          # profiles/resident_kernel_sweep_b32.md
+                          ("resident", 2880, 4096, 8): (755.081728e6 + 5.729792e6) / 32}
 
 
 def measured_peak():
