@@ -345,7 +345,7 @@ def main():
         roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": achieved / peak,
                     "traffic": (NCU_TRAFFIC_PER_SAMPLE[(dom, w.n_vis, w.d, w.n_pivot)] * B
-                                if (dom, w.n_vis, w.d, w.n_pivot) in NCU_TRAFFIC_PER_SAMPLE and args.path == 0 else None),
+                                if (dom, w.n_vis, w.d, w.n_pivot) in NCU_TRAFFIC_PER_SAMPLE and args.lag == 0 else None),
                     "peak_source": peak_src + " copy bandwidth",
                     "avg_launch_ms": avg_ms,
                     "shares": {k: v[0] / max(sum(x[0] for x in prof.values()), 1e-9) for k, v in prof.items()}}
