@@ -285,6 +285,75 @@ static int retention_quotas(const double *dup, const int32_t *pivot_idx, int n_v
 }
 
 /*
+ * Retention with INDEPENDENT pivots (Eq. 9-10 read literally: R = P u U_i R_i, every R_i built from all
+ * non-pivot tokens whatever the other pivots took).  Pivot i takes its q_i non-pivot tokens of lowest dup
+ * (quotas as in dart_oracle_retention; equal values: lower index first); a token that is lowest for two
+ * pivots is retained once, so |R| <= n_keep and the packed length depends on the data.
+ *   owner  [n_vis] -1 dropped, i = the first pivot in rank order that took the token, P + i = pivot of rank i
+ *   eps    [P]     the largest dup pivot i took, NaN if its quota is 0
+ *   gap    scalar  min over pivots of (best dup left behind by that pivot - eps_i), +inf if none
+ *   n_kept         |R|
+ */
+int dart_oracle_retention_union(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep,
+                                uint8_t *keep, int32_t *owner, double *eps, double *gap_out, int32_t *n_kept)
+{
+    if (P < 1 || P > n_keep || n_keep > n_vis) return ORACLE_ERR_SHAPE;
+    keyed_t *cand = (keyed_t *)malloc((size_t)n_vis * sizeof *cand);
+    uint8_t *is_pivot = (uint8_t *)calloc((size_t)n_vis, 1);
+    if (!cand || !is_pivot) {
+        free(cand);
+        free(is_pivot);
+        return ORACLE_ERR_NOMEM;
+    }
+    memset(keep, 0, (size_t)n_vis);
+    if (owner)
+        for (int j = 0; j < n_vis; ++j) owner[j] = OWNER_DROPPED;
+    for (int i = 0; i < P; ++i) {
+        const int p = pivot_idx[i];
+        if (p < 0 || p >= n_vis || is_pivot[p]) {
+            free(cand);
+            free(is_pivot);
+            return ORACLE_ERR_SHAPE; /* pivots must be distinct vision tokens */
+        }
+        is_pivot[p] = 1;
+        keep[p] = 1;
+        if (owner) owner[p] = P + i;
+    }
+    const int q = (n_keep - P) / P, r = (n_keep - P) % P;
+    double gap = INFINITY;
+    for (int i = 0; i < P; ++i) {
+        const int qi = q + (i < r ? 1 : 0);
+        if (eps) eps[i] = NAN;
+        if (qi == 0) continue;
+        int m = 0;
+        for (int j = 0; j < n_vis; ++j)
+            if (!is_pivot[j]) { /* every non-pivot token, also those another pivot has taken */
+                cand[m].v = dup[(size_t)i * (size_t)n_vis + j];
+                cand[m].idx = j;
+                ++m;
+            }
+        qsort(cand, (size_t)m, sizeof *cand, cmp_asc); /* m = n_vis - P >= n_keep - P >= qi */
+        for (int t = 0; t < qi; ++t) {
+            const int j = cand[t].idx;
+            if (owner && !keep[j]) owner[j] = i;
+            keep[j] = 1;
+        }
+        if (eps) eps[i] = cand[qi - 1].v;
+        if (m > qi) {
+            const double g = cand[qi].v - cand[qi - 1].v;
+            if (g < gap) gap = g;
+        }
+    }
+    int32_t cnt = 0;
+    for (int j = 0; j < n_vis; ++j) cnt += keep[j];
+    if (n_kept) *n_kept = cnt;
+    if (gap_out) *gap_out = gap;
+    free(cand);
+    free(is_pivot);
+    return ORACLE_OK;
+}
+
+/*
  * Retention with ONE threshold for all pivots (a second reading of Def. 2 / Eq. 8-9): a token is an
  * eps-duplicate of the pivot set if its dup to SOME pivot exceeds eps, so a token's duplication is its
  * highest dup over the pivots, u_j = max_i dup(p_i, x_j); the n_keep - P non-pivot tokens of lowest u_j are
@@ -405,7 +474,10 @@ int dart_oracle_compact(const uint8_t *keep, const uint16_t *hidden, const int64
  * pivots_in: NULL, or [B, P] distinct vision-relative indices that replace the pivot step (their
  * order is the order of the pivots' turns); the retention step rejects repeated or out-of-range ones.
  * rule: 0 = one threshold per pivot from equal quotas (dart_oracle_retention), 1 = one threshold for all
- * (dart_oracle_retention_global).
+ * (dart_oracle_retention_global), 2 = independent pivots (dart_oracle_retention_union): the packed length of a
+ * sample then depends on its data, the outputs are packed WITHOUT padding (sample b's rows start at row
+ * cu_seqlens_out[b] of out_hidden / out_idx / out_pos, whose capacity stays B * S_out rows) and
+ * cu_seqlens_out [B + 1] is required.
  * cosine_on_hidden: the paper ranks pivots by the K-norm but defines dup on "tokens" (Def. 2) without saying
  * which tensor represents them.  0: the key rows (one tensor for both); 1: the pivots are still chosen by the
  * key rows' scores, Eq. 7 is evaluated on the hidden rows.  Then l1_out holds the key rows' L1 scores and
@@ -420,12 +492,13 @@ int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const in
                           uint16_t *out_hidden, int32_t *out_idx, int64_t *out_pos,
                           double *l1_out, double *l2_out, int32_t *pivot_out, double *dup_out,
                           uint8_t *keep_out, int32_t *owner_out, double *eps_out,
-                          double *pivot_gap_out, double *retain_gap_out)
+                          double *pivot_gap_out, double *retain_gap_out, int32_t *cu_seqlens_out)
 {
     if (B < 0 || S < 1 || d < 1 || vis_offset < 0 || n_vis < 1 || vis_offset + n_vis > S) return ORACLE_ERR_SHAPE;
     if (n_pivot < 1 || n_pivot > n_keep || n_keep > n_vis) return ORACLE_ERR_SHAPE;
     if (norm_kind != 1 && norm_kind != 2) return ORACLE_ERR_SHAPE;
-    if (rule != 0 && rule != 1) return ORACLE_ERR_SHAPE;
+    if (rule != 0 && rule != 1 && rule != 2) return ORACLE_ERR_SHAPE;
+    if (rule == 2 && !cu_seqlens_out) return ORACLE_ERR_SHAPE;
     if (text_pivots && (!pivots_in || rule != 0)) return ORACLE_ERR_SHAPE; /* text pivots are the caller's, quota rule only */
     const int P = n_pivot, S_out = S - n_vis + n_keep;
     double *l1 = (double *)malloc((size_t)n_vis * sizeof(double));
@@ -436,6 +509,8 @@ int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const in
     uint8_t *keep = (uint8_t *)malloc((size_t)n_vis);
     int rc = ORACLE_OK;
     if (!l1 || !l2 || !hl1 || !dup || !piv || !keep) rc = ORACLE_ERR_NOMEM;
+    size_t cu = 0; /* rows packed so far (rule 2) */
+    if (cu_seqlens_out) cu_seqlens_out[0] = 0;
     for (int b = 0; b < B && rc == ORACLE_OK; ++b) {
         const uint16_t *h = hidden + (size_t)b * (size_t)S * (size_t)d;
         const uint16_t *k = keys ? keys + (size_t)b * (size_t)S * (size_t)d : h;
@@ -461,18 +536,24 @@ int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const in
         else
             rc = dart_oracle_similarity((cosine_on_hidden && keys) ? h : k, S, d, vis_offset, n_vis, piv, P, l2, dup);
         if (rc) break;
-        rc = (text_pivots ? dart_oracle_retention_any : rule == 1 ? dart_oracle_retention_global : dart_oracle_retention)(
-            dup, piv, n_vis, P, n_keep, keep, owner_out ? owner_out + (size_t)b * n_vis : NULL,
-            eps_out ? eps_out + (size_t)b * P : NULL, &rgap);
+        if (rule == 2)
+            rc = dart_oracle_retention_union(dup, piv, n_vis, P, n_keep, keep, owner_out ? owner_out + (size_t)b * n_vis : NULL,
+                                             eps_out ? eps_out + (size_t)b * P : NULL, &rgap, NULL);
+        else
+            rc = (text_pivots ? dart_oracle_retention_any : rule == 1 ? dart_oracle_retention_global : dart_oracle_retention)(
+                dup, piv, n_vis, P, n_keep, keep, owner_out ? owner_out + (size_t)b * n_vis : NULL,
+                eps_out ? eps_out + (size_t)b * P : NULL, &rgap);
         if (rc) break;
-        rc = dart_oracle_compact(keep, h, pos, S, d, vis_offset, n_vis,
-                                 out_hidden ? out_hidden + (size_t)b * (size_t)S_out * (size_t)d : NULL,
-                                 out_idx + (size_t)b * S_out, out_pos + (size_t)b * S_out, &so);
+        const size_t row0 = rule == 2 ? cu : (size_t)b * (size_t)S_out;
+        rc = dart_oracle_compact(keep, h, pos, S, d, vis_offset, n_vis, out_hidden ? out_hidden + row0 * (size_t)d : NULL,
+                                 out_idx + row0, out_pos + row0, &so);
         if (rc) break;
-        if (so != S_out) {
+        if (rule == 2 ? so > S_out : so != S_out) {
             rc = ORACLE_ERR_SHAPE;
             break;
         }
+        cu += (size_t)so;
+        if (cu_seqlens_out) cu_seqlens_out[b + 1] = (int32_t)cu;
         if (l1_out) memcpy(l1_out + (size_t)b * n_vis, l1, (size_t)n_vis * sizeof(double));
         if (l2_out) memcpy(l2_out + (size_t)b * n_vis, l2, (size_t)n_vis * sizeof(double));
         if (pivot_out) memcpy(pivot_out + (size_t)b * P, piv, (size_t)P * sizeof(int32_t));
@@ -501,5 +582,5 @@ int dart_oracle_reduce(const uint16_t *hidden, const uint16_t *keys, const int64
 {
     return dart_oracle_reduce_ex(hidden, keys, pos_in, NULL, B, S, d, vis_offset, n_vis, n_pivot, n_keep, norm_kind,
                                  largest, 0, 0, 0, out_hidden, out_idx, out_pos, l1_out, l2_out, pivot_out, dup_out, keep_out,
-                                 owner_out, eps_out, pivot_gap_out, retain_gap_out);
+                                 owner_out, eps_out, pivot_gap_out, retain_gap_out, NULL);
 }

@@ -40,7 +40,7 @@ def _load():
         _lib = ctypes.CDLL(build())
         for name in ("dart_oracle_scores", "dart_oracle_pivots", "dart_oracle_similarity",
                      "dart_oracle_retention", "dart_oracle_retention_global", "dart_oracle_retention_any",
-                     "dart_oracle_similarity_any", "dart_oracle_compact",
+                     "dart_oracle_retention_union", "dart_oracle_similarity_any", "dart_oracle_compact",
                      "dart_oracle_gather_rows", "dart_oracle_reduce", "dart_oracle_reduce_ex"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
@@ -149,6 +149,22 @@ def retention_any(dup, pivot_idx, n_keep: int):
     return keep, owner, eps, gap.value
 
 
+def retention_union(dup, pivot_idx, n_keep: int):
+    """Independent pivots: (keep, owner, eps [P], gap, n_kept); a token two pivots take counts once."""
+    dd = np.ascontiguousarray(dup, np.float64)
+    P, n_vis = dd.shape
+    piv = np.ascontiguousarray(pivot_idx, np.int32)
+    keep = np.empty(n_vis, np.uint8)
+    owner = np.empty(n_vis, np.int32)
+    eps = np.empty(P, np.float64)
+    gap = ctypes.c_double(0.0)
+    cnt = ctypes.c_int32(0)
+    _check(_load().dart_oracle_retention_union(_p(dd, ctypes.c_double), _p(piv, ctypes.c_int32), n_vis, P, n_keep,
+                                               _p(keep, ctypes.c_uint8), _p(owner, ctypes.c_int32),
+                                               _p(eps, ctypes.c_double), ctypes.byref(gap), ctypes.byref(cnt)), "retention_union")
+    return keep, owner, eps, gap.value, cnt.value
+
+
 def retention_global(dup, pivot_idx, n_keep: int):
     """dup [P, n_vis] -> (keep, owner, eps [P], gap) with one threshold on max_i dup for all pivots."""
     dd = np.ascontiguousarray(dup, np.float64)
@@ -208,6 +224,7 @@ class OracleResult:
     eps: np.ndarray         # [B, P] fp64
     pivot_gap: np.ndarray   # [B] relative score gap along the pivot ranking
     retain_gap: np.ndarray  # [B] absolute dup gap at the retention boundaries
+    cu_seqlens: np.ndarray | None = None  # [B + 1] int32, rule 2 only: sample b's rows are cu[b] .. cu[b + 1] of the flat outputs
 
     @property
     def margin(self) -> np.ndarray:
@@ -221,6 +238,7 @@ def reduce(hidden, keys, vis_offset: int, n_vis: int, n_pivot: int, n_keep: int,
            text_pivots: bool = False) -> OracleResult:
     """The whole step over a batch.  hidden/keys: [B, S, d] bf16 bits (keys None -> hidden is scored).
     pivots_in: None, or [B, n_pivot] distinct vision-relative indices that replace the pivot step.
+    rule: 0 quotas with masking, 1 one threshold for all pivots, 2 independent pivots (flat outputs + .cu_seqlens).
     rule: 0 = per-pivot thresholds from equal quotas, 1 = one threshold for all pivots.
     cosine_on_hidden: pivots by the key rows' scores, Eq. 7 on the hidden rows (then .l2 holds the hidden rows' norms).
     text_pivots: entries of pivots_in outside [0, n_vis) name text tokens (indices relative to the vision block)."""
@@ -243,6 +261,13 @@ def reduce(hidden, keys, vis_offset: int, n_vis: int, n_pivot: int, n_keep: int,
     eps = np.empty((B, n_pivot), np.float64)
     pg = np.empty(B, np.float64)
     rg = np.empty(B, np.float64)
+    cu = None
+    if rule == 2:  # the packed length depends on the data: what is not written stays -1 / 0
+        cu = np.zeros(B + 1, np.int32)
+        oi.fill(-1)
+        op.fill(-1)
+        if oh is not None:
+            oh.fill(0)
     piv_in = None if pivots_in is None else np.ascontiguousarray(pivots_in, np.int32)
     if piv_in is not None and piv_in.shape != (B, n_pivot):
         raise ValueError("pivots_in must be [B, n_pivot]")
@@ -252,5 +277,8 @@ def reduce(hidden, keys, vis_offset: int, n_vis: int, n_pivot: int, n_keep: int,
         _p(oh, ctypes.c_uint16), _p(oi, ctypes.c_int32), _p(op, ctypes.c_int64),
         _p(l1, ctypes.c_double), _p(l2, ctypes.c_double), _p(piv, ctypes.c_int32), _p(dup, ctypes.c_double),
         _p(keep, ctypes.c_uint8), _p(owner, ctypes.c_int32), _p(eps, ctypes.c_double),
-        _p(pg, ctypes.c_double), _p(rg, ctypes.c_double)), "reduce")
-    return OracleResult(oh, oi, op, l1, l2, piv, dup, keep, owner, eps, pg, rg)
+        _p(pg, ctypes.c_double), _p(rg, ctypes.c_double), _p(cu, ctypes.c_int32)), "reduce")
+    if rule == 2:  # flat outputs [B * S_out(, d)], rows beyond cu[B] are -1 / 0
+        oh = None if oh is None else oh.reshape(B * S_out, d)
+        oi, op = oi.reshape(-1), op.reshape(-1)
+    return OracleResult(oh, oi, op, l1, l2, piv, dup, keep, owner, eps, pg, rg, cu)

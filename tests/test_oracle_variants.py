@@ -237,3 +237,72 @@ def test_text_pivots_through_the_whole_step(oracle):
         assert r.out_idx.shape[1] == S - nv + Kp
     with pytest.raises(RuntimeError):
         oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=piv)                 # text pivots must be asked for
+
+
+# ----------------------------------------------------------------------------- independent pivots (the literal union of Eq. 10)
+
+def test_union_retention_against_brute_force_and_its_invariants(oracle):
+    rng = np.random.default_rng(31)
+    for trial in range(20):
+        nv = int(rng.integers(6, 40))
+        P = int(rng.integers(1, 5))
+        Kp = int(rng.integers(P, nv + 1))
+        dup = rng.uniform(-1, 1, (P, nv))
+        piv = rng.permutation(nv)[:P].astype(np.int32)
+        keep, owner, eps, gap, cnt = oracle.retention_union(dup, piv, Kp)
+        q, r = divmod(Kp - P, P)
+        expect = set(piv.tolist())
+        others = [j for j in range(nv) if j not in set(piv.tolist())]
+        first = {}
+        for i in range(P):
+            qi = q + (1 if i < r else 0)
+            mine = sorted(others, key=lambda j: (dup[i, j], j))[:qi]      # whatever the other pivots took
+            for j in mine:
+                first.setdefault(j, i)
+            expect |= set(mine)
+            if qi:
+                assert eps[i] == max(dup[i, j] for j in mine)
+                assert all(dup[i, j] >= eps[i] for j in others if j not in mine)
+            else:
+                assert np.isnan(eps[i])
+        assert set(np.nonzero(keep)[0].tolist()) == expect and cnt == len(expect)
+        assert P <= cnt <= Kp                                              # Eq. 10's union can fall short of the budget
+        assert all(owner[p] == P + i for i, p in enumerate(piv))
+        assert all(owner[j] == i for j, i in first.items())
+        assert (owner[~keep.astype(bool)] == -1).all()
+
+
+def test_union_coincides_with_the_quota_rule_when_the_picks_are_disjoint(oracle):
+    """One pivot: nothing to mask.  Pivots with disjoint neighbourhoods: masking never bites."""
+    rng = np.random.default_rng(32)
+    dup = rng.uniform(-1, 1, (1, 30))
+    a, b = oracle.retention_union(dup, [4], 11), oracle.retention(dup, [4], 11)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1]) and a[4] == 11
+    dup = np.ones((2, 20))
+    dup[0, 2:6] = [-.9, -.8, -.7, -.6]        # pivot 0 (token 0) is far from tokens 2..5
+    dup[1, 10:14] = [-.9, -.8, -.7, -.6]      # pivot 1 (token 1) from tokens 10..13
+    a, b = oracle.retention_union(dup, [0, 1], 10), oracle.retention(dup, [0, 1], 10)
+    assert np.array_equal(a[0], b[0]) and a[4] == 10
+    dup[1] = dup[0]                            # the same neighbourhood: the union keeps it once
+    keep, owner, eps, gap, cnt = oracle.retention_union(dup, [0, 1], 10)
+    assert cnt == 2 + 4 and (owner[2:6] == 0).all()
+
+
+def test_union_through_the_whole_step_is_packed_without_padding(oracle):
+    rng = np.random.default_rng(33)
+    B, S, d, vo, nv, P, Kp = 3, 50, 16, 4, 40, 3, 12
+    hb, _ = rand_tokens(rng, B * S, d)
+    kb, _ = rand_tokens(rng, B * S, d)
+    hb, kb = hb.reshape(B, S, d), kb.reshape(B, S, d)
+    r = oracle.reduce(hb, kb, vo, nv, P, Kp, rule=2)
+    cu = r.cu_seqlens
+    assert cu[0] == 0 and np.all(np.diff(cu) >= S - nv + P) and np.all(np.diff(cu) <= S - nv + Kp)
+    for b in range(B):
+        _, l2 = oracle.scores(kb[b], vo, nv)
+        dup = oracle.similarity(kb[b], vo, nv, r.pivot_idx[b], l2)
+        keep, owner, eps, _, cnt = oracle.retention_union(dup, r.pivot_idx[b], Kp)
+        oh, oi, op = oracle.compact(keep, hb[b], vo, nv)
+        assert cu[b + 1] - cu[b] == S - nv + cnt
+        assert np.array_equal(r.out_idx[cu[b]:cu[b + 1]], oi) and np.array_equal(r.out_hidden[cu[b]:cu[b + 1]], oh)
+        assert np.array_equal(r.out_pos[cu[b]:cu[b + 1]], op) and np.array_equal(r.keep[b], keep)
+    assert (r.out_idx[cu[B]:] == -1).all()
