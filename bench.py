@@ -375,6 +375,14 @@ def main():
         ms_g, _, prof_g = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_g, False)
         variants["one_threshold"] = {"ms_per_step": ms_g / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_g * 1e-3),
                                      "retain_ms": prof_g["retain"][0] / max(prof_g["retain"][1], 1)}
+        # (a2) independent pivots (Eq. 10's union): variable-length packed outputs + cu_seqlens
+        cu = torch.zeros(B + 1, dtype=torch.int32, device=dev)
+        o_u = dart.dart_opts(path=args.path, sweep_lag=args.lag, retention=args.retention, rule=dart.DART_RULE_UNION,
+                             cu_seqlens=cu.data_ptr())
+        ms_u, _, prof_u = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_u, False)
+        variants["independent_pivots"] = {"ms_per_step": ms_u / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_u * 1e-3),
+                                          "retain_ms": prof_u["retain"][0] / max(prof_u["retain"][1], 1) * 3,  # three launches
+                                          "mean_kept_vision_tokens": float(cu[-1].item()) / B - (w.S - w.n_vis)}
         # (b) pivots named by the caller (here: random distinct tokens): steps 3-5 only wait for the norms
         piv = torch.stack([torch.randperm(w.n_vis, device=dev)[:w.n_pivot] for _ in range(B)]).to(torch.int32).contiguous()
         o_p = dart.dart_opts(path=args.path, sweep_lag=args.lag, retention=args.retention, pivots_in=piv.data_ptr())

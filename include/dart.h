@@ -79,6 +79,15 @@ enum {
                               are kept, ties to the lower index.  dbg->eps holds the threshold n_pivot times, dbg->owner the
                               pivot a kept token is most similar to (the first of equals). */
 
+#define DART_RULE_UNION 2  /* independent pivots (Eq. 9-10 read literally: R = P u U_i R_i): pivot i keeps its q_i non-pivot
+                              tokens of lowest dup whatever the other pivots keep; a token two pivots keep counts once, so
+                              a sample keeps between n_pivot and n_keep vision tokens.  The outputs are then packed WITHOUT
+                              padding, as variable-length attention kernels take them: out_hidden, out_idx and out_pos
+                              are flat arrays with room for B * S_out rows, sample b's rows are
+                              cu_seqlens[b] .. cu_seqlens[b + 1] - 1, and rows from cu_seqlens[B] on are not written.
+                              Needs dart_opts.cu_seqlens.  dbg->owner names the first pivot in rank order that kept a
+                              token. */
+
 typedef struct dart_ctx dart_ctx; /* opaque: workspace, device status word, profiling events */
 
 /* Maxima a context is sized for.  d is fixed per context (a multiple of 8). */
@@ -122,6 +131,8 @@ typedef struct {
                               pivots' turns in step 4.  This covers the paper's other ways to choose pivots (Sec. 5.2:
                               random, attention score, value norm): the caller ranks, the library does steps 3-5.
                               Repeated or out-of-range indices end the call with DART_ERR_CHECK in dart_status. */
+    int32_t *cu_seqlens;   /* DART_RULE_UNION only: [B + 1] int32, device, written by the call: cu_seqlens[0] = 0,
+                              cu_seqlens[b + 1] = cu_seqlens[b] + packed length of sample b. */
 } dart_opts;
 
 /* Optional per-step outputs of dart_reduce_ex; every member is a device pointer or NULL. */

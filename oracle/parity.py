@@ -233,3 +233,68 @@ def check_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, n_vis,
             if not same:
                 rep.notes.append("sample %d differs below margin %.2e (valid under tolerance)" % (b, margin[b]))
     return rep
+
+
+def check_union_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, n_vis, n_pivot, n_keep,
+                      out_hidden, out_idx, out_pos, cu_seqlens, dbg, pos_in=None, largest=True, norm_kind=1,
+                      require_exact_above=MARGIN) -> ParityReport:
+    """Retention with independent pivots: flat outputs, sample b's rows are cu_seqlens[b] .. cu_seqlens[b + 1] - 1.
+    Above the margin everything equals the oracle; below it every pivot's picks are replayed against the oracle's
+    fp64 similarities with the candidate's own thresholds (dbg["eps"])."""
+    B, S = hidden_bits.shape[0], hidden_bits.shape[1]
+    rep = ParityReport()
+    margin = ora.margin
+    cu = np.asarray(cu_seqlens, np.int64)
+    assert cu[0] == 0 and len(cu) == B + 1
+    for b in range(B):
+        rep.samples += 1
+        rep.min_margin = min(rep.min_margin, float(margin[b]))
+        lo, hi = int(cu[b]), int(cu[b + 1])
+        kept = hi - lo - (S - n_vis)
+        assert n_pivot <= kept <= n_keep, "sample %d keeps %d vision tokens" % (b, kept)
+        pin = None if pos_in is None else pos_in[b]
+        check_packed_outputs(None if out_hidden is None else out_hidden[lo:hi], out_idx[lo:hi], out_pos[lo:hi],
+                             hidden_bits[b], pin, vis_offset, n_vis, kept)
+        olo, ohi = int(ora.cu_seqlens[b]), int(ora.cu_seqlens[b + 1])
+        same = hi - lo == ohi - olo and np.array_equal(out_idx[lo:hi], ora.out_idx[olo:ohi])
+        rep.exact += int(same)
+        check_scores(dbg["l1"][b], dbg["ssq"][b], ora.l1[b], ora.l2[b], rep)
+        kept_gpu = np.zeros(n_vis, bool)
+        kept_gpu[out_idx[lo:hi][vis_offset:vis_offset + kept] - vis_offset] = True
+        assert np.array_equal(dbg["keep"][b].astype(bool), kept_gpu), "keep flags and out_idx disagree"
+        assert np.array_equal(dbg["owner"][b] >= 0, kept_gpu), "owner and out_idx disagree"
+        piv = dbg["pivot_idx"][b]
+        same_piv = np.array_equal(piv, ora.pivot_idx[b])
+        if ora.pivot_gap[b] > require_exact_above:
+            assert same_piv, "sample %d: pivots differ although the score gap is %g" % (b, ora.pivot_gap[b])
+        if same_piv and ora.dup is not None:
+            check_sim(dbg["sim"][b], ora.dup[b], rep)
+        if margin[b] > require_exact_above:
+            rep.above_margin += 1
+            assert same, "sample %d: kept indices differ although the margin is %g" % (b, margin[b])
+            assert np.array_equal(dbg["owner"][b], ora.owner[b])
+            continue
+        # valid under tolerance: every pivot's own threshold separates what it took from what it left
+        assert len(set(piv.tolist())) == n_pivot
+        score = ora.l1[b] if norm_kind == 1 else ora.l2[b]
+        sgn = 1.0 if largest else -1.0
+        others = np.setdiff1d(np.arange(n_vis), piv)
+        if len(others):
+            assert (sgn * score[piv]).min() >= (sgn * score[others]).max() * (1 - MARGIN * np.sign((sgn * score[others]).max()))
+        dup = _o.similarity(keys_bits[b], vis_offset, n_vis, piv, ora.l2[b])
+        e = dbg["eps"][b].astype(np.float64)
+        allowed = np.zeros(n_vis, bool)
+        allowed[piv] = True
+        for i, qi in enumerate(quotas(n_pivot, n_keep)):
+            if qi == 0:
+                assert np.isnan(e[i])
+                continue
+            below = dup[i, others] < e[i] - MARGIN
+            upto = dup[i, others] <= e[i] + MARGIN
+            assert below.sum() <= qi <= upto.sum(), "pivot %d: its threshold does not cut off %d tokens" % (i, qi)
+            assert kept_gpu[others[below]].all(), "pivot %d left behind a token well below its threshold" % i
+            allowed[others[upto]] = True
+        assert not (kept_gpu & ~allowed).any(), "a kept token lies above every pivot's threshold"
+        if not same:
+            rep.notes.append("sample %d differs below margin %.2e (valid under tolerance)" % (b, margin[b]))
+    return rep

@@ -38,6 +38,7 @@ struct dart_ctx {
     float *l1, *ssq, *sim, *eps;
     int32_t *pivot_idx, *owner;
     void *piv_rows;  // [B_max][P_max rounded to 16][d] bf16: compact copy of the pivot rows (NULL: not available)
+    int32_t *len;    // [B_max] packed length of every sample (retention with independent pivots)
     int32_t *cand;   // [B_max][P_max][cand_stride] sorted candidate lists of the two-phase retention (NULL: not available)
     int cand_stride;
     uint8_t *keep;
@@ -199,6 +200,21 @@ void launch_retention(dart_ctx *ctx, int B, const int64_t *pos_in, int vis_offse
             ctx->status);
         return;
     }
+    if (o.rule == DART_RULE_UNION) { // independent pivots: selections, scan of the packed lengths, index lists at their offsets
+        {
+            Prof p(ctx, st, SLOT_RETAIN);
+            retain_union_kernel<<<B, kSelectThreads, retain_union_smem_bytes(n_vis), st>>>(
+                ctx->sim, ctx->pivot_idx, S, n_vis, P, n_keep, ctx->keep, ctx->owner, ctx->eps, ctx->len, ctx->status);
+        }
+        {
+            Prof p(ctx, st, SLOT_RETAIN);
+            cu_seqlens_kernel<<<1, 256, 0, st>>>(ctx->len, B, o.cu_seqlens, ctx->status);
+        }
+        Prof p(ctx, st, SLOT_RETAIN);
+        pack_varlen_kernel<<<B, kWalkThreads, retain_union_smem_bytes(n_vis), st>>>(ctx->keep, o.cu_seqlens, pos_in, S, vis_offset, n_vis,
+                                                                                    out_idx, out_pos, ctx->status);
+        return;
+    }
     const int m_pad = next_pow2(m > 1 ? m : 1);
     const bool can_lists = ctx->cand && m <= ctx->cand_stride && m <= kCandMax &&
                            candidates_smem_bytes(n_vis, m_pad) <= (size_t)ctx->max_smem_optin - 2048 &&
@@ -227,6 +243,23 @@ void launch_retention(dart_ctx *ctx, int B, const int64_t *pos_in, int vis_offse
                                                                           S, vis_offset, n_vis, P, n_keep, out_idx, out_pos,
                                                                           ctx->keep, ctx->owner, ctx->eps, ctx->status);
     }
+}
+
+// Step 5b.  With independent pivots the rows are packed at the samples' offsets (cu_seqlens) instead of B equal blocks.
+void launch_gather(dart_ctx *ctx, int B, const void *hidden, int n_vis, int n_keep, const int32_t *out_idx, void *out_hidden,
+                   const dart_opts &o, cudaStream_t st)
+{
+    using namespace dart;
+    const int S = ctx->S, d8 = ctx->desc.d / 8, S_out = S - n_vis + n_keep;
+    Prof pr(ctx, st, SLOT_GATHER);
+    const long long orows = (long long)B * S_out;
+    const unsigned grid = (unsigned)((orows + kGatherWarps - 1) / kGatherWarps);
+    if (o.rule == DART_RULE_UNION)
+        gather_varlen_kernel<<<grid, kGatherWarps * 32, 0, st>>>((const uint4 *)hidden, out_idx, o.cu_seqlens, B, S, d8, orows,
+                                                                ctx->status, (uint4 *)out_hidden);
+    else
+        gather_kernel<<<grid, kGatherWarps * 32, 0, st>>>((const uint4 *)hidden, out_idx, S, S_out, d8, orows, ctx->status,
+                                                         (uint4 *)out_hidden);
 }
 
 // Step 2 with the caller's pivots: checked and copied into the workspace.
@@ -268,13 +301,7 @@ int launch_staged(dart_ctx *ctx, int B, const void *hidden, const void *keys_in,
         ctx->launches += (P - 1) / kSimPivotChunk;
     }
     launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
-    {
-        Prof p(ctx, st, SLOT_GATHER);
-        long long orows = (long long)B * S_out;
-        unsigned grid = (unsigned)((orows + kGatherWarps - 1) / kGatherWarps);
-        gather_kernel<<<grid, kGatherWarps * 32, 0, st>>>((const uint4 *)hidden, out_idx, S, S_out, d8, orows,
-                                                         ctx->status, (uint4 *)out_hidden);
-    }
+    launch_gather(ctx, B, hidden, n_vis, n_keep, out_idx, out_hidden, o, st);
     DART_CUDA(ctx, cudaGetLastError());
     return copy_debug(ctx, B, n_vis, P, dbg, st);
 }
@@ -399,13 +426,7 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
                                                    smem_bytes(p.N, p.row_bytes, p.n1, p.n2), st));
     }
     launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
-    {
-        Prof pr(ctx, st, SLOT_GATHER);
-        long long orows = (long long)B * S_out;
-        unsigned grid = (unsigned)((orows + kGatherWarps - 1) / kGatherWarps);
-        gather_kernel<<<grid, kGatherWarps * 32, 0, st>>>((const uint4 *)hidden, out_idx, S, S_out, d8, orows,
-                                                         ctx->status, (uint4 *)out_hidden);
-    }
+    launch_gather(ctx, B, hidden, n_vis, n_keep, out_idx, out_hidden, o, st);
     DART_CUDA(ctx, cudaGetLastError());
     return copy_debug(ctx, B, n_vis, P, dbg, st);
 }
@@ -450,17 +471,6 @@ int launch_onepass_kernel(dart_ctx *ctx, int B, const void *src, bool scores_els
     return DART_OK;
 }
 
-void launch_gather(dart_ctx *ctx, int B, const void *hidden, int n_vis, int n_keep, const int32_t *out_idx, void *out_hidden,
-                   cudaStream_t st)
-{
-    using namespace dart;
-    const int S = ctx->S, d8 = ctx->desc.d / 8, S_out = S - n_vis + n_keep;
-    Prof pr(ctx, st, SLOT_GATHER);
-    const long long orows = (long long)B * S_out;
-    const unsigned grid = (unsigned)((orows + kGatherWarps - 1) / kGatherWarps);
-    gather_kernel<<<grid, kGatherWarps * 32, 0, st>>>((const uint4 *)hidden, out_idx, S, S_out, d8, orows, ctx->status,
-                                                     (uint4 *)out_hidden);
-}
 
 // The resident sweep applies when a sample's rows fit the chip: at most 8 pivots and, per CTA, no more octets of one
 // sample than the exchange warp has lane groups and tensor memory has slots.
@@ -497,7 +507,7 @@ int launch_resident(dart_ctx *ctx, int B, const void *hidden, const void *keys_i
                                                    args, R::smem_bytes(ctx->desc.d, ctx->sm_count, p.n_landing), st));
     }
     launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
-    launch_gather(ctx, B, hidden, n_vis, n_keep, out_idx, out_hidden, st);
+    launch_gather(ctx, B, hidden, n_vis, n_keep, out_idx, out_hidden, o, st);
     DART_CUDA(ctx, cudaGetLastError());
     return copy_debug(ctx, B, n_vis, P, dbg, st);
 }
@@ -511,7 +521,7 @@ int launch_onepass(dart_ctx *ctx, int B, const void *hidden, const void *keys_in
     int rc = launch_onepass_kernel(ctx, B, keys_in ? keys_in : hidden, false, vis_offset, n_vis, P, o, st);
     if (rc != DART_OK) return rc;
     launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
-    launch_gather(ctx, B, hidden, n_vis, n_keep, out_idx, out_hidden, st);
+    launch_gather(ctx, B, hidden, n_vis, n_keep, out_idx, out_hidden, o, st);
     DART_CUDA(ctx, cudaGetLastError());
     return copy_debug(ctx, B, n_vis, P, dbg, st);
 }
@@ -560,7 +570,7 @@ int launch_two_pass(dart_ctx *ctx, int B, const void *hidden, const void *keys, 
         ctx->launches += (P - 1) / kSimPivotChunk;
     }
     launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
-    launch_gather(ctx, B, hidden, n_vis, n_keep, out_idx, out_hidden, st);
+    launch_gather(ctx, B, hidden, n_vis, n_keep, out_idx, out_hidden, o, st);
     DART_CUDA(ctx, cudaGetLastError());
     return copy_debug(ctx, B, n_vis, P, dbg, st);
 }
@@ -634,6 +644,7 @@ int dart_create(dart_ctx **out, const dart_desc *desc)
     if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->pivot_idx, np);
     if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->owner, nv);
     if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->keep, nv);
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->len, (size_t)desc->B_max);
     if (rc == DART_OK) {
         // candidate lists of the two-phase retention: at most kCandMax entries per pivot; contexts whose maxima
         // would need more than 1 GiB go without (they use the one-kernel retention)
@@ -718,6 +729,7 @@ int dart_destroy(dart_ctx *ctx)
     cudaFree(ctx->pivot_idx);
     cudaFree(ctx->owner);
     cudaFree(ctx->keep);
+    cudaFree(ctx->len);
     cudaFree(ctx->cand);
     cudaFree(ctx->piv_rows);
     cudaFree(ctx->status);
@@ -762,7 +774,12 @@ int dart_reduce_ex(dart_ctx *ctx, const void *hidden, const void *keys, const in
     if (o.path != DART_PATH_AUTO && o.path != DART_PATH_STAGED && o.path != DART_PATH_FUSED && o.path != DART_PATH_TWO_PASS &&
         o.path != DART_PATH_RESIDENT)
         return DART_ERR_UNSUPPORTED;
-    if (o.rule != DART_RULE_QUOTAS && o.rule != DART_RULE_GLOBAL) return DART_ERR_UNSUPPORTED;
+    if (o.rule != DART_RULE_QUOTAS && o.rule != DART_RULE_GLOBAL && o.rule != DART_RULE_UNION) return DART_ERR_UNSUPPORTED;
+    if (o.rule == DART_RULE_UNION) {
+        if (!o.cu_seqlens) return DART_ERR_NULL;
+        if ((uintptr_t)o.cu_seqlens & 3u) return DART_ERR_ALIGN;
+        if (dart::retain_union_smem_bytes(n_vis) > (size_t)ctx->max_smem_optin - 2048) return DART_ERR_UNSUPPORTED;
+    }
     if (o.cosine_on_hidden && o.norm_kind != 1) return DART_ERR_UNSUPPORTED; // the hidden rows' sums of squares take the slot
     if ((uintptr_t)o.pivots_in & 3u) return DART_ERR_ALIGN;
     if (o.text_pivots && (!o.pivots_in || o.rule != DART_RULE_QUOTAS)) return DART_ERR_UNSUPPORTED;

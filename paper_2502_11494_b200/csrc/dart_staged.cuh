@@ -614,10 +614,143 @@ retain_global_kernel(const float *__restrict__ sim, const int32_t *__restrict__ 
 }
 
 // ------------------------------------------------------------------------------------------------
+// Steps 4 and 5a with INDEPENDENT pivots (Eq. 9-10 read literally: R = P u U_i R_i): pivot i takes its q_i
+// non-pivot tokens of lowest dup whatever the other pivots took; a token two pivots take is kept once, so a
+// sample keeps between P and n_keep vision tokens and the packed length depends on the data.  Three launches:
+// the selections (one CTA per sample; writes the keep flags and the sample's packed length), an exclusive
+// scan of the lengths (cu_seqlens, the layout variable-length attention kernels take), and the packed index
+// lists written at the samples' offsets.
+// ------------------------------------------------------------------------------------------------
+constexpr int kGatherWarps = 8; // warps per CTA of the gather kernels, one output row each
+inline size_t retain_union_smem_bytes(int n_vis) { return ((size_t)n_vis + 15) / 16 * 16; }
+
+__global__ void __launch_bounds__(kSelectThreads)
+retain_union_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx, int S, int n_vis, int P, int n_keep,
+                    uint8_t *__restrict__ keep_out, int32_t *__restrict__ owner_out, float *__restrict__ eps_out,
+                    int32_t *__restrict__ len_out, const int *__restrict__ status)
+{
+    extern __shared__ __align__(16) uint8_t flags[]; // [n_vis] 0 free, 1 kept, 2 pivot
+    __shared__ SelectSmem sel;
+    if (*status != 0) return; // an earlier kernel of this call failed: its outputs are undefined
+    const int b = blockIdx.x;
+    int32_t *owner = owner_out ? owner_out + (size_t)b * n_vis : nullptr;
+    for (int j = threadIdx.x; j < n_vis; j += blockDim.x) {
+        flags[j] = 0;
+        if (owner) owner[j] = -1;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < P; i += blockDim.x) {
+        const int pv = pivot_idx[(size_t)b * P + i];
+        flags[pv] = 2;
+        if (owner) owner[pv] = P + i;
+    }
+    __syncthreads();
+    const int q = (n_keep - P) / P, r = (n_keep - P) % P;
+    for (int i = 0; i < P; ++i) {
+        const int qi = q + (i < r ? 1 : 0);
+        if (qi == 0) {
+            if (eps_out && threadIdx.x == 0) eps_out[(size_t)b * P + i] = __int_as_float(0x7fc00000);
+            continue;
+        }
+        const float *row = sim + ((size_t)b * P + i) * n_vis;
+        auto keyfn = [&](int j, uint32_t &key) { // every non-pivot token is a candidate of every pivot
+            if (flags[j] == 2) return false;
+            key = order_key(row[j]);
+            return true;
+        };
+        uint32_t T, need_eq, cnt_eq;
+        block_select_threshold(CtaGroup(), keyfn, n_vis, (uint32_t)qi, sel, T, need_eq, cnt_eq);
+        block_select_apply(CtaGroup(), keyfn, n_vis, T, need_eq, cnt_eq, sel, [&](int j, uint32_t) {
+            if (flags[j] == 0) { // the first pivot in rank order that takes a token owns it
+                flags[j] = 1;
+                if (owner) owner[j] = i;
+            }
+        });
+        if (eps_out && threadIdx.x == 0) eps_out[(size_t)b * P + i] = order_key_inv(T);
+        __syncthreads();
+    }
+    int mine = 0;
+    for (int j = threadIdx.x; j < n_vis; j += blockDim.x) {
+        const uint8_t f = flags[j] != 0;
+        mine += f;
+        keep_out[(size_t)b * n_vis + j] = f;
+    }
+    __shared__ int total;
+    if (threadIdx.x == 0) total = 0;
+    __syncthreads();
+    if (mine) atomicAdd(&total, mine);
+    __syncthreads();
+    if (threadIdx.x == 0) len_out[b] = S - n_vis + total;
+}
+
+// cu[0] = 0, cu[b + 1] = cu[b] + len[b]: one CTA, chunks of blockDim.x lengths with a running carry
+__global__ void __launch_bounds__(256) cu_seqlens_kernel(const int32_t *__restrict__ len, int B, int32_t *__restrict__ cu,
+                                                         const int *__restrict__ status)
+{
+    __shared__ int32_t buf[256];
+    __shared__ int32_t carry;
+    if (*status != 0) return;
+    if (threadIdx.x == 0) carry = 0, cu[0] = 0;
+    __syncthreads();
+    for (int b0 = 0; b0 < B; b0 += blockDim.x) {
+        const int b = b0 + threadIdx.x;
+        buf[threadIdx.x] = b < B ? len[b] : 0;
+        __syncthreads();
+        for (int o = 1; o < (int)blockDim.x; o <<= 1) { // inclusive scan
+            const int32_t v = threadIdx.x >= (unsigned)o ? buf[threadIdx.x - o] : 0;
+            __syncthreads();
+            buf[threadIdx.x] += v;
+            __syncthreads();
+        }
+        if (b < B) cu[b + 1] = carry + buf[threadIdx.x];
+        __syncthreads();
+        if (threadIdx.x == blockDim.x - 1) carry += buf[threadIdx.x];
+        __syncthreads();
+    }
+}
+
+// The packed index list and position ids of every sample at its offset cu[b].
+__global__ void __launch_bounds__(kWalkThreads)
+pack_varlen_kernel(const uint8_t *__restrict__ keep_in, const int32_t *__restrict__ cu, const int64_t *__restrict__ pos_in, int S,
+                   int vis_offset, int n_vis, int32_t *__restrict__ out_idx, int64_t *__restrict__ out_pos,
+                   const int *__restrict__ status)
+{
+    extern __shared__ __align__(16) uint8_t keep[]; // [n_vis]
+    __shared__ uint32_t warp_tot[kWalkThreads / 32];
+    if (*status != 0) return;
+    const int b = blockIdx.x;
+    for (int j = threadIdx.x; j < n_vis; j += blockDim.x) keep[j] = keep_in[(size_t)b * n_vis + j];
+    __syncthreads();
+    const int start = cu[b], kept = cu[b + 1] - start - (S - n_vis);
+    pack_indices(keep, S, vis_offset, n_vis, kept, pos_in ? pos_in + (size_t)b * S : nullptr, out_idx + start, out_pos + start,
+                 warp_tot);
+}
+
+// Step 5b for packed rows of variable length: output row t belongs to the sample b with cu[b] <= t < cu[b + 1].
+// One warp per output row (as gather_kernel); rows at and beyond cu[B] do not exist.
+__global__ void __launch_bounds__(kGatherWarps * 32)
+gather_varlen_kernel(const uint4 *__restrict__ hidden, const int32_t *__restrict__ out_idx, const int32_t *__restrict__ cu, int B,
+                     int S, int d8, long long rows_cap, const int *__restrict__ status, uint4 *__restrict__ out_hidden)
+{
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * kGatherWarps + (threadIdx.x >> 5);
+    if (row >= rows_cap || *status != 0 || row >= cu[B]) return;
+    int lo = 0, hi = B; // the largest b with cu[b] <= row
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if ((long long)cu[mid] <= row) lo = mid;
+        else hi = mid;
+    }
+    const int s = out_idx[row];
+    const uint4 *src = hidden + ((size_t)lo * S + s) * (size_t)d8;
+    uint4 *dst = out_hidden + (size_t)row * (size_t)d8;
+    for (int c = lane; c < d8; c += 32) st_stream(dst + c, ld_stream(src + c));
+}
+
+// ------------------------------------------------------------------------------------------------
 // Step 5b: gather the kept hidden rows into the packed sequence.  One warp per output row,
 // 128-bit loads and streaming stores, 8 loads in flight per lane.
 // ------------------------------------------------------------------------------------------------
-constexpr int kGatherWarps = 8;
 
 __global__ void __launch_bounds__(kGatherWarps * 32)
 gather_kernel(const uint4 *__restrict__ hidden, const int32_t *__restrict__ out_idx, int S, int S_out, int d8,

@@ -20,7 +20,7 @@ DART_ERR_CUDA, DART_ERR_NOMEM, DART_ERR_TIMEOUT, DART_ERR_CHECK, DART_ERR_UNSUPP
 DART_FLAG_HOST_STAGING = 1
 DART_PATH_AUTO, DART_PATH_STAGED, DART_PATH_FUSED, DART_PATH_TWO_PASS, DART_PATH_RESIDENT = 0, 1, 2, 3, 4
 DART_RETAIN_AUTO, DART_RETAIN_SERIAL, DART_RETAIN_LISTS = 0, 1, 2
-DART_RULE_QUOTAS, DART_RULE_GLOBAL = 0, 1
+DART_RULE_QUOTAS, DART_RULE_GLOBAL, DART_RULE_UNION = 0, 1, 2
 
 EXPORTS = (
     "dart_create", "dart_destroy", "dart_set_shape", "dart_reduce", "dart_reduce_ex", "dart_reduce_host",
@@ -41,7 +41,8 @@ class dart_opts(ctypes.Structure):
     _fields_ = [("norm_kind", ctypes.c_int32), ("pivot_smallest", ctypes.c_int32), ("path", ctypes.c_int32),
                 ("wait_limit", ctypes.c_int32), ("sweep_lag", ctypes.c_int32),
                 ("test_withhold_pivots", ctypes.c_int32), ("retention", ctypes.c_int32), ("rule", ctypes.c_int32),
-                ("cosine_on_hidden", ctypes.c_int32), ("text_pivots", ctypes.c_int32), ("pivots_in", ctypes.c_void_p)]
+                ("cosine_on_hidden", ctypes.c_int32), ("text_pivots", ctypes.c_int32), ("pivots_in", ctypes.c_void_p),
+                ("cu_seqlens", ctypes.c_void_p)]
 
 
 class dart_debug(ctypes.Structure):

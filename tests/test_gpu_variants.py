@@ -347,3 +347,79 @@ def test_text_pivots_random_shapes(oracle, seed):
     ora = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=piv, text_pivots=True)
     rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, dbg=dbg, pivots_given=True, text_pivots=True)
     assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5, (B, S, d, vo, nv, P, Kp)
+
+
+# ----------------------------------------------------------------------------- independent pivots, variable-length outputs
+
+def run_union(keys, hidden, vo, nv, P, Kp, path):
+    B, S, d = hidden.shape
+    if path in (dart.DART_PATH_FUSED, dart.DART_PATH_TWO_PASS) and (d % 64 or P > 256):
+        pytest.skip("the tensor-core paths need d % 64 == 0 and at most 256 pivots")
+    S_out = S - nv + Kp
+    out = (torch.zeros((B * S_out, d), dtype=torch.bfloat16, device="cuda"),
+           torch.full((B * S_out,), -1, dtype=torch.int32, device="cuda"),
+           torch.full((B * S_out,), -1, dtype=torch.int64, device="cuda"))
+    cu = torch.full((B + 1,), -7, dtype=torch.int32, device="cuda")
+    ctx = dart.Dart(B, S, d, P, Kp)
+    try:
+        res = ctx.reduce(hidden, keys, vo, nv, P, Kp, out=out, debug=True,
+                         opts=dart.dart_opts(path=path, rule=dart.DART_RULE_UNION, cu_seqlens=cu.data_ptr()))
+        torch.cuda.synchronize()
+        assert ctx.status() == dart.DART_OK, dart.dart_status_detail(ctx.handle)
+    finally:
+        ctx.close()
+    return _np(res[0]), _np(res[1]), _np(res[2]), {k: _np(v) for k, v in res[3].items()}, _np(cu)
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
+@pytest.mark.parametrize("shape", SHAPES + [(2, 64, 64, 0, 64, 5, 5), (2, 64, 64, 0, 64, 3, 64), (300, 40, 64, 3, 30, 2, 9)],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_independent_pivots_give_variable_lengths(oracle, shape, path):
+    B, S, d, vo, nv, P, Kp = shape
+    k, h = gaussian(B, S, d, seed=600 + sum(shape))
+    oh, oi, op, dbg, cu = run_union(k, h, vo, nv, P, Kp, path)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, rule=2)
+    rep = parity.check_union_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, cu, dbg)
+    assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5
+    assert (oi[cu[-1]:] == -1).all() and (op[cu[-1]:] == -1).all() and not oh[cu[-1]:].any()   # nothing beyond the packed rows
+
+
+def test_independent_pivots_on_clustered_tokens_keep_fewer_than_the_budget(oracle):
+    """Duplicates make several pivots pick the same far-away tokens: the union falls short of n_keep."""
+    w = W.LLAVA15_B64.with_(B=6)
+    k, h = W.make_batch(w, device="cuda")
+    oh, oi, op, dbg, cu = run_union(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, dart.DART_PATH_AUTO)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, rule=2)
+    rep = parity.check_union_batch(ora, kb, hb, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, oh, oi, op, cu, dbg)
+    assert rep.exact >= rep.above_margin and rep.exact >= 5, rep.notes
+    kept = np.diff(cu) - (w.S - w.n_vis)
+    assert (kept <= w.n_keep).all() and (kept < w.n_keep).any()
+
+
+def test_independent_pivots_need_cu_seqlens():
+    k, h = gaussian(1, 64, 64, seed=68)
+    ctx = dart.Dart(1, 64, 64, 2, 8)
+    with pytest.raises(dart.DartError) as e:
+        ctx.reduce(h, k, 0, 64, 2, 8, opts=dart.dart_opts(rule=dart.DART_RULE_UNION))
+    assert e.value.code == dart.DART_ERR_NULL
+    ctx.close()
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_independent_pivots_random_shapes(oracle, seed):
+    rng = np.random.default_rng(3000 + seed)
+    d = int(rng.choice([8, 24, 64, 128, 320, 1024]))
+    nv = int(rng.integers(1, 600))
+    vo, after = int(rng.integers(0, 40)), int(rng.integers(0, 40))
+    P = int(rng.integers(1, min(nv, 24) + 1))
+    Kp = int(rng.integers(P, nv + 1))
+    B = int(rng.integers(1, 6))
+    path = int(rng.choice(PATHS)) if d % 64 == 0 else dart.DART_PATH_STAGED
+    k, h = gaussian(B, vo + nv + after, d, seed=800 + seed)
+    oh, oi, op, dbg, cu = run_union(k, h, vo, nv, P, Kp, path)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, rule=2)
+    rep = parity.check_union_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, cu, dbg)
+    assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5, (B, vo, nv, after, d, P, Kp, path)
