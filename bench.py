@@ -53,7 +53,7 @@ def parse():
 def pick_workload(args):
     from paper_2502_11494_b200 import workloads as W
 
-    w = {c.name: c for c in W.CONFIGS}[args.workload]
+    w = {c.name: c for c in W.CONFIGS + W.EXTRA}[args.workload]
     kw = {}
     if args.pivots:
         kw["n_pivot"] = args.pivots

@@ -74,6 +74,16 @@ VIDEO_B4 = Workload("video_b4", 4, 4, 40, 4608, 60, 3584, 32, 512, "video", n_fr
 SWEEP_B256 = Workload("sweep_b256", 5, 256, 40, 2880, 60, 4096, 8, 320, "crops", n_crops=5, shared_frac=0.3)
 
 CONFIGS = (LLAVA15_B1, LLAVA15_B64, LLAVA_NEXT_B8, VIDEO_B4, SWEEP_B256)
+
+# Two more shapes the paper applies the step to (appendix): a vision-language-action model that keeps 56 of its 256
+# image tokens per control step (batch of 16 environments, an instruction of a few tokens after the image), and
+# audio tokens of a long utterance reduced by 20 / 30 / 50 % with 8 pivots (1500 tokens of width 3072 stand for two
+# minutes of speech; consecutive frames drift like the video generator's).  Not benchmark configurations: parity
+# cases and `bench.py --workload` choices.
+VLA_B16 = Workload("vla_b16", 6, 16, 1, 256, 20, 4096, 8, 56, "cluster", centres_lo=24, centres_hi=64)
+AUDIO_B8 = Workload("audio_b8", 7, 8, 10, 1500, 30, 3072, 8, 750, "video", n_frames=100, drift=0.05)
+AUDIO_KEEP = (1200, 1050, 750)  # 20 %, 30 %, 50 % of the audio tokens removed
+EXTRA = (VLA_B16, AUDIO_B8)
 SWEEP_PIVOTS = (8, 32, 128)
 SWEEP_KEEP = (64, 320, 640)
 

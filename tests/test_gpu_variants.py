@@ -423,3 +423,29 @@ def test_independent_pivots_random_shapes(oracle, seed):
     ora = oracle.reduce(hb, kb, vo, nv, P, Kp, rule=2)
     rep = parity.check_union_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, cu, dbg)
     assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5, (B, vo, nv, after, d, P, Kp, path)
+
+
+# ----------------------------------------------------------------------------- the paper's other shapes (appendix)
+
+@pytest.mark.parametrize("path", [dart.DART_PATH_AUTO] + PATHS, ids=lambda p: PATH_IDS.get(p, "auto"))
+def test_vision_language_action_shape(oracle, path):
+    """256 image tokens -> 56, 8 pivots, per control step of a batch of environments."""
+    w = W.VLA_B16.with_(B=4)
+    k, h = W.make_batch(w, device="cuda")
+    oh, oi, op, dbg, _ = run(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, path)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep)
+    rep = parity.check_batch(ora, kb, hb, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, oh, oi, op, dbg=dbg)
+    assert rep.exact >= rep.above_margin and rep.exact >= 3 and rep.max_abs_sim < 2e-5, rep.notes
+
+
+@pytest.mark.parametrize("keep", W.AUDIO_KEEP)
+def test_audio_token_shape(oracle, keep):
+    """1500 audio tokens of width 3072 reduced by 20, 30 and 50 %."""
+    w = W.AUDIO_B8.with_(B=2, n_keep=keep)
+    k, h = W.make_batch(w, device="cuda")
+    oh, oi, op, dbg, _ = run(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, dart.DART_PATH_AUTO)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep)
+    rep = parity.check_batch(ora, kb, hb, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, oh, oi, op, dbg=dbg)
+    assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5, rep.notes
