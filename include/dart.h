@@ -62,9 +62,9 @@ enum {
 #define DART_PATH_RESIDENT 4 /* steps 1-3 from ONE read of the keys: every sample is spread over all SMs and stays in their
                               shared and tensor memory until its pivots are known.  Needs n_pivot <= 8, d % 64 == 0,
                               d <= 4096, n_vis <= 32 rows per SM (and the pivots chosen by score, one tensor for
-                              steps 1-3), else UNSUPPORTED.  Measured at half the speed of FUSED on the large batched
-                              workloads (the wait for a sample's pivots is longer than the chip can cover): AUTO never
-                              takes it. */
+                              steps 1-3), else UNSUPPORTED.  The fastest path for a few samples (AUTO takes it up to
+                              four); at half the speed of FUSED on the large batched workloads, where the wait for a
+                              sample's pivots is longer than the samples that fit the chip can cover. */
 
 /* dart_opts.retention */
 #define DART_RETAIN_AUTO 0   /* two phases when the batch alone cannot fill the GPU, else one kernel */
