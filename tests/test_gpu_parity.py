@@ -331,3 +331,31 @@ def test_profile_slots_cover_every_launch():
     assert rc == dart.DART_OK and sum(n for _, n in prof.values()) >= 1
     assert all(ms >= 0 for ms, _ in prof.values())
     ctx.close()
+
+
+@pytest.mark.parametrize("B", [1, 6])
+def test_the_call_can_be_captured_in_a_cuda_graph(B):
+    """All work goes to the caller's stream and nothing synchronises the host: a captured call replays with the
+    same outputs (one sample takes the resident sweep, six the persistent one; both launch cooperatively)."""
+    w = W.LLAVA15_B64.with_(B=B)
+    k, h = W.make_batch(w, device="cuda")
+    ctx = dart.Dart(w.B, w.S, w.d, w.n_pivot, w.n_keep)
+    try:
+        ref = ctx.reduce(h, k, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep)
+        torch.cuda.synchronize()
+        out = tuple(torch.zeros_like(t) for t in ref)
+        s, g = torch.cuda.Stream(), torch.cuda.CUDAGraph()
+        with torch.cuda.stream(s):
+            ctx.reduce(h, k, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, out=out, stream=s)
+            s.synchronize()
+            g.capture_begin()
+            ctx.reduce(h, k, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, out=out, stream=s)
+            g.capture_end()
+        for t in out:
+            t.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert ctx.status() == dart.DART_OK
+        assert all(torch.equal(a, b) for a, b in zip(out, ref))
+    finally:
+        ctx.close()
