@@ -526,13 +526,20 @@ retain_walk_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pi
                     remaining -= __popc(took);
                     __syncwarp(); // the flags are visible to the next chunk and the next pivot
                 }
-                if (eps_out && lane == 0 && last >= 0) eps_out[(size_t)b * P + i] = sim[((size_t)b * P + i) * n_vis + last];
+                // eps_i = dup of the last token taken; its index is parked in the output word and turned into the value
+                // after the walk by another thread: a load from global memory here would stall every pivot's turn
+                if (eps_out && lane == 0) eps_out[(size_t)b * P + i] = __int_as_float(last);
                 off += M;
             }
         }
         __syncthreads();
         i0 = i1;
     }
+    if (eps_out)
+        for (int i = threadIdx.x; i < n_active; i += blockDim.x) {
+            const int last = __float_as_int(eps_out[(size_t)b * P + i]);
+            eps_out[(size_t)b * P + i] = last >= 0 ? sim[((size_t)b * P + i) * n_vis + last] : __int_as_float(0x7fc00000);
+        }
     pack_indices(keep, S, vis_offset, n_vis, n_keep, pos_in ? pos_in + (size_t)b * S : nullptr, out_idx + (size_t)b * S_out,
                  out_pos + (size_t)b * S_out, warp_tot);
     if (keep_out)
