@@ -275,7 +275,7 @@ int launch_staged(dart_ctx *ctx, int B, const void *hidden, const void *keys_in,
                   const dart_opts &o, const dart_debug *dbg, cudaStream_t st)
 {
     using namespace dart;
-    const int S = ctx->S, d8 = ctx->desc.d / 8, S_out = S - n_vis + n_keep;
+    const int S = ctx->S, d8 = ctx->desc.d / 8;
     const uint4 *keys = (const uint4 *)(keys_in ? keys_in : hidden);
     const long long rows = (long long)B * n_vis;
     {
@@ -390,7 +390,7 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
 {
     using namespace dart;
     using namespace dart::sweep;
-    const int S = ctx->S, d8 = ctx->desc.d / 8, S_out = S - n_vis + n_keep;
+    const int S = ctx->S, d8 = ctx->desc.d / 8;
     const void *keys = keys_in ? keys_in : hidden;
     Params p = {};
     p.B = B, p.S = S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.N = (P + 15) / 16 * 16, p.d8 = d8;
