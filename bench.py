@@ -85,13 +85,11 @@ def kernel_bytes_per_launch(name, w, B):
     }[name]
 
 
-# DRAM traffic of one launch per sample (dram__bytes_read.sum + dram__bytes_write.sum), from the ncu capture of the
-# sweep workload at batch 32 summarised in profiles/sweep_kernel_sweep_b32.md; traffic is proportional to the batch
-# (every sample is read and written independently), so a launch over B samples moves B times this.
+# DRAM traffic of one launch per sample (dram__bytes_read.sum + dram__bytes_write.sum), from ncu captures of each kernel
+# on the sweep workload at batch 32; traffic is proportional to the batch (every sample is read and written
+# independently), so a launch over B samples moves B times this.
 NCU_TRAFFIC_PER_SAMPLE = {("sweep", 2880, 4096, 8): (1.508212e9 + 5.538816e6) / 32,
-                          # profiles/onepass_kernel_sweep_b32.md
                           ("onepass", 2880, 4096, 8): (755.18336e6 + 5.144064e6) / 32,
-                          # profiles/resident_kernel_sweep_b32.md
                           ("resident", 2880, 4096, 8): (755.081728e6 + 5.729792e6) / 32}
 
 

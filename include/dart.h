@@ -202,7 +202,9 @@ int dart_reduce_ex(dart_ctx *ctx, const void *hidden, const void *keys, const in
  * after everything has completed.  All pointers are host memory (pinned memory makes the copies
  * asynchronous); keys may be NULL.  Needs a context created with DART_FLAG_HOST_STAGING
  * (else UNSUPPORTED).  The shape of the call is the one set by dart_set_shape; B may exceed the
- * chunk size but not B_max.
+ * chunk size but not B_max.  Since the call waits for its own work it also reads (and clears) the
+ * device status word: a bounded wait that gave up or a failed self-check is returned as
+ * DART_ERR_TIMEOUT / DART_ERR_CHECK and the host outputs are then not valid.
  */
 int dart_reduce_host(dart_ctx *ctx, const void *hidden, const void *keys, int vis_offset, int n_vis,
                      int n_pivot, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos);
@@ -275,11 +277,16 @@ int dart_profile_read(dart_ctx *ctx, float *ms, int32_t *launches, const char **
  *   device     CUDA device ordinal the pointers belong to;  stream: a cudaStream_t on that device
  * Limits: B * n_vis <= DART_STATIC_MAX_ROWS and n_pivot <= 1024, else DART_ERR_BAD_SHAPE; d % 8 == 0;
  * 1 <= n_pivot <= n_vis; vis_offset + n_vis <= S.
- * The first call on a device looks up the array's device address (no allocation); make that call
- * before any stream capture begins.  Every call on a device uses the same array and leaves its
+ * The first call on a device looks up the array's device address; make that call before any stream
+ * capture begins.  The look-up itself allocates nothing, but the CUDA runtime loads a library's
+ * image into device memory lazily (the default since CUDA 12.2): the kernels and the 2 MiB array
+ * are placed on the device by that first call, or when the library is loaded if
+ * CUDA_MODULE_LOADING=EAGER is set.  A host that gives all free memory to its own pool must
+ * therefore make one call (any valid small call will do) BEFORE it sizes the pool; a first call
+ * that finds no memory left returns DART_ERR_NOMEM.  Every call on a device uses the same array and leaves its
  * scores there: nothing in it has to start at zero (each call overwrites the rows it reads), but
  * two calls whose kernels overlap on the GPU, from different streams or threads, race on it.
- * Calls cudaMalloc, cudaFree or an allocating routine never.  Errors: NULL, BAD_SHAPE, ALIGN, CUDA.
+ * Calls cudaMalloc, cudaFree or an allocating routine never.  Errors: NULL, BAD_SHAPE, ALIGN, NOMEM, CUDA.
  */
 #define DART_STATIC_MAX_ROWS 262144
 int dart_pivots_static(const void *keys, int B, int S, int d, int vis_offset, int n_vis, int n_pivot,

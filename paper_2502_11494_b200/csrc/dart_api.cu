@@ -617,6 +617,18 @@ int launch_reduce(dart_ctx *ctx, int B, const void *hidden, const void *keys, co
                                  o, dbg, st);
 }
 
+// Reads the device status word, keeps its detail and clears it.  The caller has synchronised the work that may write it.
+int read_status(dart_ctx *ctx)
+{
+    int word[12] = {0};
+    DART_CUDA(ctx, cudaMemcpy(word, ctx->status, sizeof word, cudaMemcpyDeviceToHost));
+    if (word[0] != 0) {
+        for (int k = 0; k < 11; ++k) ctx->status_detail[k] = word[k + 1];
+        DART_CUDA(ctx, cudaMemset(ctx->status, 0, sizeof word));
+    }
+    return word[0];
+}
+
 } // namespace
 
 extern "C" {
@@ -676,8 +688,12 @@ int dart_create(dart_ctx **out, const dart_desc *desc)
                                       desc->S_max + 16 + dart::kRetainCacheBytes) != cudaSuccess)
             rc = DART_ERR_CUDA;
     }
-    if (rc == DART_OK && cudaFuncSetAttribute(dart::retain_global_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              ctx->max_smem_optin - 2048) != cudaSuccess)
+    if (rc == DART_OK && (cudaFuncSetAttribute(dart::retain_global_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               ctx->max_smem_optin - 2048) != cudaSuccess ||
+                          cudaFuncSetAttribute(dart::retain_union_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               ctx->max_smem_optin - 2048) != cudaSuccess ||
+                          cudaFuncSetAttribute(dart::pack_varlen_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               ctx->max_smem_optin - 2048) != cudaSuccess))
         rc = DART_ERR_CUDA;
     if (rc == DART_OK && ctx->cand) {
         // the two-phase kernels may use up to the device's shared memory; shapes that need more fall back at launch
@@ -854,7 +870,9 @@ int dart_reduce_host(dart_ctx *ctx, const void *hidden, const void *keys, int vi
     DART_CUDA(ctx, e1);
     DART_CUDA(ctx, e2);
     DART_CUDA(ctx, e3);
-    return DART_OK;
+    // everything has completed: a bounded wait that gave up or a failed self-check made the later kernels skip
+    // their writes, so the host buffers must not be handed back with a success code
+    return read_status(ctx);
 }
 
 int dart_status(dart_ctx *ctx)
@@ -862,14 +880,8 @@ int dart_status(dart_ctx *ctx)
     if (!ctx) return DART_ERR_NULL;
     DeviceGuard g(ctx->desc.device);
     if (!g.ok) return DART_ERR_CUDA;
-    int word[12] = {0};
     DART_CUDA(ctx, cudaDeviceSynchronize());
-    DART_CUDA(ctx, cudaMemcpy(word, ctx->status, sizeof word, cudaMemcpyDeviceToHost));
-    if (word[0] != 0) {
-        for (int k = 0; k < 11; ++k) ctx->status_detail[k] = word[k + 1];
-        DART_CUDA(ctx, cudaMemset(ctx->status, 0, sizeof word));
-    }
-    return word[0];
+    return read_status(ctx);
 }
 
 int dart_status_detail(const dart_ctx *ctx, int32_t detail[11])
@@ -945,8 +957,14 @@ int dart_pivots_static(const void *keys, int B, int S, int d, int vis_offset, in
     {
         std::lock_guard<std::mutex> lock(g_static_mutex);
         if (!g_static_ptr[device]) { // set-up, once per device, with that device current
+            // With lazy module loading this is where the library's image (kernels and this array) is placed in
+            // device memory: a device whose memory is already handed out answers cudaErrorMemoryAllocation.
             float *ptr = nullptr;
-            if (cudaGetSymbolAddress((void **)&ptr, g_static_scores) != cudaSuccess || !ptr) return DART_ERR_CUDA;
+            const cudaError_t e = cudaGetSymbolAddress((void **)&ptr, g_static_scores);
+            if (e != cudaSuccess || !ptr) {
+                cudaGetLastError(); // not sticky: leave no error behind for the caller's next CUDA call
+                return e == cudaErrorMemoryAllocation ? DART_ERR_NOMEM : DART_ERR_CUDA;
+            }
             g_static_ptr[device] = ptr;
         }
         scratch = g_static_ptr[device];
@@ -959,7 +977,8 @@ int dart_pivots_static(const void *keys, int B, int S, int d, int vis_offset, in
         (const uint4 *)keys, S, d / 8, vis_offset, n_vis, rows, l1, ssq);
     const int P_pad = next_pow2(n_pivot);
     pivot_kernel<<<B, kSelectThreads, (size_t)P_pad * 8, st>>>(l1, n_vis, n_pivot, P_pad, 0, pivot_idx);
-    return cudaGetLastError() == cudaSuccess ? DART_OK : DART_ERR_CUDA;
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? DART_OK : e == cudaErrorMemoryAllocation ? DART_ERR_NOMEM : DART_ERR_CUDA;
 }
 
 int dart_gather_rows(const void *src, const int32_t *idx, int B, int S, int S_out, int row_bytes, void *out, int device,

@@ -398,6 +398,18 @@ def test_independent_pivots_on_clustered_tokens_keep_fewer_than_the_budget(oracl
     assert (kept <= w.n_keep).all() and (kept < w.n_keep).any()
 
 
+@pytest.mark.parametrize("path", [dart.DART_PATH_STAGED, dart.DART_PATH_TWO_PASS], ids=PATH_IDS.get)
+def test_independent_pivots_on_a_sample_beyond_48k_tokens(oracle, path):
+    """The keep flags of a sample live in dynamic shared memory: past 48 KB the kernels need the opt-in limit."""
+    B, S, d, vo, nv, P, Kp = 1, 50300, 64, 20, 50250, 3, 400
+    k, h = gaussian(B, S, d, seed=77)
+    oh, oi, op, dbg, cu = run_union(k, h, vo, nv, P, Kp, path)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, rule=2)
+    rep = parity.check_union_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, cu, dbg)
+    assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5
+
+
 def test_independent_pivots_need_cu_seqlens():
     k, h = gaussian(1, 64, 64, seed=68)
     ctx = dart.Dart(1, 64, 64, 2, 8)
