@@ -40,7 +40,9 @@ def parse():
     ap.add_argument("--keep", type=int, default=None)
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch size")
     ap.add_argument("--sweep", action="store_true", help="also time every (pivots, keep) cell of the sweep")
-    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 staged, 2 fused (persistent sweep), 3 two passes (score pass + one tensor-core pass), 4 resident sweep")
+    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 staged, 2 fused (persistent sweep), 3 two passes (score pass + one tensor-core pass), 4 resident sweep, 5 split (resident for a share of the tiles, second read for the rest)")
+    ap.add_argument("--tune", type=int, default=0, help="path 6: 16 * n1 + n2 ring depths")
+    ap.add_argument("--split", type=int, default=0, help="path 5: k keeps tiles with index %% k == 0 on the chip, -k all others")
     ap.add_argument("--lag", type=int, default=0, help="fused path: extra tasks between a row's two sweeps")
     ap.add_argument("--retention", type=int, default=0, help="0 auto, 1 one kernel, 2 candidate lists + walks")
     ap.add_argument("--variants", action="store_true",
@@ -79,6 +81,7 @@ def kernel_bytes_per_launch(name, w, B):
         "sweep": keys,                       # fused scores + pivots + similarities: the keys count once
         "onepass": keys,                     # the caller's pivots: scores + similarities from one pass
         "resident": keys,                    # scores + pivots + similarities, rows held on the chip: one read
+        "pair": keys,                        # paired sweeps: the second read of a row is meant to come from the L2
         "gather": 2 * (2 * w.d * w.S_out) * B,
         "pivot": 4 * w.n_vis * B,
         "retain": 4 * w.n_pivot * w.n_vis * B + 12 * w.S_out * B,
@@ -317,7 +320,7 @@ def main():
     ctx = dart.Dart(B, w.S, w.d, max(w.n_pivot, max(W.SWEEP_PIVOTS) if args.sweep else 0),
                     max(w.n_keep, max(W.SWEEP_KEEP) if args.sweep else 0), device=local, flags=flags)
     dart.dart_set_shape(ctx.handle, B, w.S)
-    opts = dart.dart_opts(0, 0, args.path, 0, args.lag, 0, args.retention)
+    opts = dart.dart_opts(0, 0, args.path, 0, args.lag, 0, args.retention, resident_split=args.split, tune=args.tune)
 
     def alloc_outs(wl):
         return (torch.empty((B, wl.S_out, wl.d), dtype=torch.bfloat16, device=dev),

@@ -66,6 +66,15 @@ enum {
                               four); at half the speed of FUSED on the large batched workloads, where the wait for a
                               sample's pivots is longer than the samples that fit the chip can cover. */
 
+#define DART_PATH_SPLIT 5    /* RESIDENT for a share of every sample's 128-row tiles, one tensor-core pass (as in TWO_PASS)
+                              for the others once the pivots are known: the rows that stay on the chip are read once, the
+                              others twice.  dart_opts.resident_split sets the share.  Same limits as RESIDENT. */
+
+#define DART_PATH_PAIRED 6   /* persistent kernel in which the same SM reads a block of 16 key rows twice, a few microseconds
+                              apart (scores first; similarities as soon as every SM has merged the SMs' short candidate
+                              lists into the sample's pivots), so that the second read comes from the L2.  Needs
+                              n_pivot <= 16, d % 64 == 0, pivots chosen by score, else UNSUPPORTED. */
+
 /* dart_opts.retention */
 #define DART_RETAIN_AUTO 0   /* two phases when the batch alone cannot fill the GPU, else one kernel */
 #define DART_RETAIN_SERIAL 1 /* one kernel, one CTA per sample: the pivots' selections one after the other */
@@ -133,6 +142,9 @@ typedef struct {
                               Repeated or out-of-range indices end the call with DART_ERR_CHECK in dart_status. */
     int32_t *cu_seqlens;   /* DART_RULE_UNION only: [B + 1] int32, device, written by the call: cu_seqlens[0] = 0,
                               cu_seqlens[b + 1] = cu_seqlens[b] + packed length of sample b. */
+    int32_t resident_split; /* DART_PATH_SPLIT: 0 = default (every second tile stays on the chip); k >= 2: the tiles with
+                              index % k == 0 stay (a share of 1/k); -k: all other tiles stay (a share of 1 - 1/k) */
+    int32_t tune;          /* 0 = defaults.  DART_PATH_PAIRED: 256 * n1 + 16 * n2 + n3 = depths of the three shared-memory rings (tuning) */
 } dart_opts;
 
 /* Optional per-step outputs of dart_reduce_ex; every member is a device pointer or NULL. */

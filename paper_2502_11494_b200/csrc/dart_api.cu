@@ -11,11 +11,12 @@
 #include "dart_sweep.cuh"
 #include "dart_onepass.cuh"
 #include "dart_resident.cuh"
+#include "dart_pair.cuh"
 
 namespace {
 
-enum Slot { SLOT_SCORE = 0, SLOT_PIVOT, SLOT_SIM, SLOT_RETAIN, SLOT_GATHER, SLOT_SWEEP, SLOT_ONEPASS, SLOT_RESIDENT, SLOT_COUNT };
-const char *const kSlotNames[SLOT_COUNT] = {"score", "pivot", "sim", "retain", "gather", "sweep", "onepass", "resident"};
+enum Slot { SLOT_SCORE = 0, SLOT_PIVOT, SLOT_SIM, SLOT_RETAIN, SLOT_GATHER, SLOT_SWEEP, SLOT_ONEPASS, SLOT_RESIDENT, SLOT_PAIR, SLOT_COUNT };
+const char *const kSlotNames[SLOT_COUNT] = {"score", "pivot", "sim", "retain", "gather", "sweep", "onepass", "resident", "pair"};
 
 typedef CUresult (*TensorMapEncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                       const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -67,6 +68,10 @@ struct dart_ctx {
     bool resident_ok;
     int res_landing;  // landing slots in shared memory
     unsigned long long *res_cand; // [B_max][sm_count][8] candidate keys
+    // paired sweeps (csrc/dart_pair.cuh)
+    bool pair_ok;
+    unsigned long long *pair_cand; // [B_max][sm_count][16] candidate keys
+    int32_t *pair_res;             // [B_max][32] resolved pivots and their norms
 };
 
 namespace {
@@ -334,13 +339,14 @@ int fused_setup(dart_ctx *ctx)
     int per_sm = 0;
     int n1 = 0, n2 = 0;
     ring_depths(16, (uint32_t)D.d * 2, ctx->max_smem_optin, n1, n2);
-    if (n1 < 2) return DART_OK;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sweep_kernel, kThreads,
-                                                      smem_bytes(16, (uint32_t)D.d * 2, n1, n2)) !=
-            cudaSuccess ||
-        per_sm < 1)
-        return DART_ERR_CUDA;
-    ctx->fused_ok = true;
+    if (n1 >= 2) { // else the rows are too wide for the persistent sweep's rings: the other tensor-core kernels may still fit
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sweep_kernel, kThreads,
+                                                          smem_bytes(16, (uint32_t)D.d * 2, n1, n2)) !=
+                cudaSuccess ||
+            per_sm < 1)
+            return DART_ERR_CUDA;
+        ctx->fused_ok = true;
+    }
     // the resident sweep: rows of at most 8 KB, two landing slots or more, one CTA per SM
     ctx->resident_ok = false;
     if (D.d * 2 <= dart::resident::kMaxRowBytes && ctx->sm_count <= dart::resident::kMaxGrid) {
@@ -357,6 +363,24 @@ int fused_setup(dart_ctx *ctx)
             if (rc != DART_OK) return rc;
             ctx->res_landing = L;
             ctx->resident_ok = true;
+        }
+    }
+    // paired sweeps: rows of at most 16 KB, two ring-1 stages or more, one CTA per SM
+    ctx->pair_ok = false;
+    if (ctx->sm_count <= dart::pair::kMaxGrid) {
+        namespace Q = dart::pair;
+        int n1 = 0, n2 = 0, n3 = 0, per = 0;
+        Q::ring_depths(1, (uint32_t)D.d * 2, ctx->sm_count, ctx->max_smem_optin, n1, n2, n3, 0, 2, 2); // the least it takes; checked per call
+        if (n1 >= 2 &&
+            cudaFuncSetAttribute(Q::pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 ctx->max_smem_optin - Q::kStaticSmemReserve) == cudaSuccess &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, Q::pair_kernel, Q::kThreads,
+                                                          Q::smem_bytes(1, (uint32_t)D.d * 2, ctx->sm_count, n1, n2, n3)) == cudaSuccess &&
+            per >= 1) {
+            rc = ws_alloc(ctx, &ctx->pair_cand, (size_t)D.B_max * ctx->sm_count * Q::kMaxP);
+            if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->pair_res, (size_t)D.B_max * 2 * Q::kMaxP);
+            if (rc != DART_OK) return rc;
+            ctx->pair_ok = true;
         }
     }
     // the one-pass kernel for the caller's pivots uses the same tensor maps
@@ -434,7 +458,7 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
 // One pass over `src` (csrc/dart_onepass.cuh) with the pivots already in the workspace: sums of squares of src's rows
 // (and their L1 scores unless `scores_elsewhere`: then the scores came from another tensor) and the similarities.
 int launch_onepass_kernel(dart_ctx *ctx, int B, const void *src, bool scores_elsewhere, int vis_offset, int n_vis, int P,
-                          const dart_opts &o, cudaStream_t st)
+                          const dart_opts &o, cudaStream_t st, dart::TileSplit split = dart::TileSplit{1, 0})
 {
     using namespace dart;
     using sweep::kSubRows;
@@ -443,6 +467,8 @@ int launch_onepass_kernel(dart_ctx *ctx, int B, const void *src, bool scores_els
     onepass::Params p = {};
     p.B = B, p.S = S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.N = (P + 15) / 16 * 16;
     p.n_atoms = ctx->n_atoms, p.n_rt = (n_vis + kTileRows - 1) / kTileRows;
+    p.split = split, p.n_sel = split.k <= 1 ? p.n_rt : split.n_streamed(p.n_rt);
+    if (p.n_sel == 0) return DART_OK; // every tile stayed on the chip
     p.aps = onepass::atoms_per_stage(p.N, ctx->max_smem_optin);
     p.n_st = onepass::ring_depth(p.N, p.aps, ctx->max_smem_optin);
     if (p.n_st < 2) return DART_ERR_UNSUPPORTED;
@@ -465,7 +491,7 @@ int launch_onepass_kernel(dart_ctx *ctx, int B, const void *src, bool scores_els
             (const uint4 *)src, ctx->pivot_idx, S, ctx->desc.d / 8, vis_offset, n_vis, P, p.N, prow, (uint4 *)ctx->piv_rows);
     }
     Prof pr(ctx, st, SLOT_ONEPASS);
-    const long long tasks = (long long)B * p.n_rt;
+    const long long tasks = (long long)B * p.n_sel;
     const unsigned grid = (unsigned)(tasks < ctx->sm_count ? tasks : ctx->sm_count); // no CTA waits for another
     onepass::onepass_kernel<<<grid, onepass::kThreads, onepass::smem_bytes(p.N, p.aps, p.n_st), st>>>(tm_tile, tm_keys, tm_row, tm_piv, p);
     return DART_OK;
@@ -486,10 +512,11 @@ bool resident_applies(const dart_ctx *ctx, int n_vis, int P)
 // Steps 1-3 from one read of the keys (csrc/dart_resident.cuh), then steps 4-5.
 int launch_resident(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, const int64_t *pos_in, int vis_offset,
                     int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos, const dart_opts &o,
-                    const dart_debug *dbg, cudaStream_t st)
+                    const dart_debug *dbg, cudaStream_t st, dart::TileSplit split = dart::TileSplit{1, 0})
 {
     namespace R = dart::resident;
     R::Params p = {};
+    p.split = split;
     p.B = B, p.S = ctx->S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.d = ctx->desc.d;
     p.n_oct = (n_vis + R::kOctRows - 1) / R::kOctRows;
     p.n_slots = R::tmem_slots(ctx->desc.d), p.n_landing = ctx->res_landing;
@@ -505,6 +532,53 @@ int launch_resident(dart_ctx *ctx, int B, const void *hidden, const void *keys_i
         // every CTA waits for all others (the candidates of a sample come from all of them): co-residency is required
         DART_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)R::resident_kernel, dim3((unsigned)ctx->sm_count), dim3(R::kThreads),
                                                    args, R::smem_bytes(ctx->desc.d, ctx->sm_count, p.n_landing), st));
+    }
+    if (split.k > 1) { // the tiles that did not stay on the chip: their norms and similarities from a second read
+        int rc = launch_onepass_kernel(ctx, B, p.keys, true, vis_offset, n_vis, P, o, st, split);
+        if (rc != DART_OK) return rc;
+    }
+    launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
+    launch_gather(ctx, B, hidden, n_vis, n_keep, out_idx, out_hidden, o, st);
+    DART_CUDA(ctx, cudaGetLastError());
+    return copy_debug(ctx, B, n_vis, P, dbg, st);
+}
+
+bool pair_applies(const dart_ctx *ctx, int P) { return ctx->pair_ok && P <= dart::pair::kMaxP; }
+
+// Steps 1-3 by the paired sweeps (csrc/dart_pair.cuh), then steps 4-5.
+int launch_pair(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, const int64_t *pos_in, int vis_offset, int n_vis,
+                int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos, const dart_opts &o, const dart_debug *dbg,
+                cudaStream_t st)
+{
+    namespace Q = dart::pair;
+    const void *keys = keys_in ? keys_in : hidden;
+    Q::Params p = {};
+    p.B = B, p.S = ctx->S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.d = ctx->desc.d;
+    p.n_atoms = ctx->n_atoms, p.T1 = (n_vis + Q::kBlockRows - 1) / Q::kBlockRows;
+    p.row_bytes = (uint32_t)ctx->desc.d * 2, p.stage1_bytes = Q::stage1_bytes(p.row_bytes);
+    p.stage2_bytes = Q::stage2_bytes(P), p.stage3_bytes = Q::stage3_bytes(P);
+    Q::ring_depths(P, p.row_bytes, ctx->sm_count, ctx->max_smem_optin, p.n1, p.n2, p.n3, (o.tune >> 8) & 15, (o.tune >> 4) & 15, o.tune & 15);
+    if (p.n1 < 2) Q::ring_depths(P, p.row_bytes, ctx->sm_count, ctx->max_smem_optin, p.n1, p.n2, p.n3, 0, 2, 2); // wide rows: the shallowest rings
+    if (p.n1 < 2) return DART_ERR_UNSUPPORTED;
+    if ((long long)B * p.T1 >= (1ll << 30)) return DART_ERR_UNSUPPORTED;
+    p.lead = o.sweep_lag; // tuning: how far the first sweep may run ahead of the second, in samples
+    p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest, p.withhold = o.test_withhold_pivots;
+    p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
+    p.keys = (const char *)keys;
+    p.sim = ctx->sim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
+    p.cand = ctx->pair_cand, p.arrived = ctx->counters, p.res_ready = ctx->counters + B, p.res = ctx->pair_res, p.status = ctx->status;
+    CUtensorMap tm_blk;
+    int rc = encode_2d(ctx, &tm_blk, keys, (uint64_t)ctx->desc.d, (uint64_t)B * ctx->S, Q::kBlockRows);
+    if (rc != DART_OK) return rc;
+    DART_CUDA(ctx, cudaMemsetAsync(ctx->counters, 0, (size_t)B * 2 * sizeof(int), st));
+    {
+        Prof pr(ctx, st, SLOT_PAIR);
+        const long long blocks = (long long)B * p.T1;
+        const unsigned grid = (unsigned)(blocks < ctx->sm_count ? blocks : ctx->sm_count);
+        void *args[2] = {&tm_blk, &p};
+        // every CTA waits for the lists of all others: co-residency is required
+        DART_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)Q::pair_kernel, dim3(grid), dim3(Q::kThreads), args,
+                                                   Q::smem_bytes(P, p.row_bytes, (int)grid, p.n1, p.n2, p.n3), st));
     }
     launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
     launch_gather(ctx, B, hidden, n_vis, n_keep, out_idx, out_hidden, o, st);
@@ -581,10 +655,21 @@ int launch_reduce(dart_ctx *ctx, int B, const void *hidden, const void *keys, co
 {
     const bool fused = o.path == DART_PATH_FUSED || (o.path == DART_PATH_AUTO && fused_applies(ctx, P));
     if (fused && !fused_applies(ctx, P)) return DART_ERR_UNSUPPORTED;
-    if (o.path == DART_PATH_RESIDENT) {
+    if (o.path == DART_PATH_RESIDENT || o.path == DART_PATH_SPLIT) {
         if (!resident_applies(ctx, n_vis, P) || o.pivots_in || (o.cosine_on_hidden && keys && keys != hidden))
             return DART_ERR_UNSUPPORTED;
-        return launch_resident(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o, dbg, st);
+        dart::TileSplit split{1, 0};
+        if (o.path == DART_PATH_SPLIT) {
+            const int k = o.resident_split == 0 ? 2 : (o.resident_split < 0 ? -o.resident_split : o.resident_split);
+            if (k < 2 || k > 64) return DART_ERR_UNSUPPORTED;
+            split = dart::TileSplit{k, o.resident_split < 0 ? 1 : 0};
+        }
+        return launch_resident(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o, dbg, st,
+                               split);
+    }
+    if (o.path == DART_PATH_PAIRED) {
+        if (!pair_applies(ctx, P) || o.pivots_in || (o.cosine_on_hidden && keys && keys != hidden)) return DART_ERR_UNSUPPORTED;
+        return launch_pair(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o, dbg, st);
     }
     if (o.text_pivots && !fused) return DART_ERR_UNSUPPORTED; // only the tensor-core kernel takes a text row's norm from the row
     if (o.cosine_on_hidden && keys && keys != hidden)
@@ -756,6 +841,8 @@ int dart_destroy(dart_ctx *ctx)
     cudaFree(ctx->status);
     cudaFree(ctx->counters);
     cudaFree(ctx->res_cand);
+    cudaFree(ctx->pair_cand);
+    cudaFree(ctx->pair_res);
     for (int k = 0; k < 2; ++k) {
         cudaFree(ctx->st_hidden[k]);
         cudaFree(ctx->st_keys[k]);
@@ -793,7 +880,7 @@ int dart_reduce_ex(dart_ctx *ctx, const void *hidden, const void *keys, const in
     if (o.norm_kind == 0) o.norm_kind = 1;
     if (o.norm_kind != 1 && o.norm_kind != 2) return DART_ERR_UNSUPPORTED;
     if (o.path != DART_PATH_AUTO && o.path != DART_PATH_STAGED && o.path != DART_PATH_FUSED && o.path != DART_PATH_TWO_PASS &&
-        o.path != DART_PATH_RESIDENT)
+        o.path != DART_PATH_RESIDENT && o.path != DART_PATH_SPLIT && o.path != DART_PATH_PAIRED)
         return DART_ERR_UNSUPPORTED;
     if (o.rule != DART_RULE_QUOTAS && o.rule != DART_RULE_GLOBAL && o.rule != DART_RULE_UNION) return DART_ERR_UNSUPPORTED;
     if (o.rule == DART_RULE_UNION) {

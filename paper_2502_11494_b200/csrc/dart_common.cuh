@@ -49,6 +49,24 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
+// ---- which row tiles stay on the chip ------------------------------------------------------------
+// The split path shares a sample's 128-row tiles between two kernels: the resident sweep keeps some of them in
+// tensor memory until the sample's pivots are known, the rest is streamed a second time by the one-pass kernel.
+// k <= 1: every tile stays on the chip.  inv == 0: tiles with rt % k == 0 stay (a fraction 1/k); inv == 1: tiles
+// with rt % k != 0 stay (a fraction 1 - 1/k).
+struct TileSplit {
+    int k, inv;
+    __host__ __device__ __forceinline__ bool on_chip(int rt) const { return k <= 1 || ((rt % k == 0) != (inv != 0)); }
+    // tiles among n_rt that are streamed, and the i-th of them
+    __host__ __device__ __forceinline__ int n_streamed(int n_rt) const
+    {
+        if (k <= 1) return 0;
+        const int zero = (n_rt + k - 1) / k; // tiles with rt % k == 0
+        return inv ? zero : n_rt - zero;
+    }
+    __host__ __device__ __forceinline__ int streamed(int i) const { return inv ? i * k : i + i / (k - 1) + 1; }
+};
+
 // ---- thread groups ---------------------------------------------------------------------------------
 // The selection helpers below run either on a whole CTA or on a group of warps inside one
 // (a named barrier), so that a few warps of a persistent kernel can select while others stream.

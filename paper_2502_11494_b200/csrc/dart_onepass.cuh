@@ -45,6 +45,8 @@ struct Params {
     int n_atoms, n_rt;                 // 64-column atoms per row; row tiles per sample
     int n_st, aps;                     // ring depth; atoms per stage (<= kMaxAtomsPerStage)
     int compact;                       // pivot tiles come from the compact copy [B][N][d] (tm_piv), not by gather4
+    int n_sel;                         // row tiles per sample this launch takes: n_rt, or the streamed tiles of `split`
+    TileSplit split;                   // k <= 1: all tiles
     unsigned long long wait_ns;
     float *sim;                        // [B][P][n_vis] dup(p_i, x_j)
     float *l1, *ssq;                   // [B][n_vis]; l1 may be NULL (the scores come from another tensor)
@@ -142,7 +144,13 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = sh.tmem_base;
-    const uint32_t total = (uint32_t)p.B * (uint32_t)p.n_rt; // tasks: (sample, row tile), sample-major
+    const uint32_t total = (uint32_t)p.B * (uint32_t)p.n_sel; // tasks: (sample, row tile), sample-major
+    // task g -> (sample, row tile); with a split only the tiles that did not stay on the chip are taken
+    auto task = [&](uint32_t g, int &b, int &rt) {
+        b = (int)(g / (uint32_t)p.n_sel);
+        const int i = (int)(g - (uint32_t)b * (uint32_t)p.n_sel);
+        rt = p.split.k <= 1 ? i : p.split.streamed(i);
+    };
     const int na = p.n_atoms;
 
     if (warp == 0) {
@@ -156,7 +164,8 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
         int cur_b = -1;
         int my_piv[kMaxN / 128][4]; // lane l loads pivot ranks 4l..4l+3, 4(l+32).., as rows of the key tensor
         for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
-            const int b = (int)(g / (uint32_t)p.n_rt), rt = (int)(g - (uint32_t)b * (uint32_t)p.n_rt);
+            int b, rt;
+            task(g, b, rt);
             if (b != cur_b) {
 #pragma unroll
                 for (int k = 0; k < kMaxN / 128; ++k)
@@ -251,7 +260,8 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
         uint32_t n = 0;
         bool dead = false; // warp-uniform
         for (uint32_t g = blockIdx.x; !dead && g < total; g += gridDim.x) {
-            const int b = (int)(g / (uint32_t)p.n_rt), rt = (int)(g - (uint32_t)b * (uint32_t)p.n_rt);
+            int b, rt;
+            task(g, b, rt);
             const int rows = min(kTileRows, p.n_vis - rt * kTileRows);
             float a0 = 0.f, a1 = 0.f, q0 = 0.f, q1 = 0.f; // own tile row
             for (int a = 0; a < na; a += p.aps) {
@@ -324,7 +334,8 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
         const int row = quarter * 32 + lane; // tile row owned by this thread
         uint32_t n = 0;
         for (uint32_t g = blockIdx.x; g < total; g += gridDim.x) {
-            const int b = (int)(g / (uint32_t)p.n_rt), rt = (int)(g - (uint32_t)b * (uint32_t)p.n_rt);
+            int b, rt;
+            task(g, b, rt);
             const int rows = min(kTileRows, p.n_vis - rt * kTileRows);
             const int j = rt * kTileRows + row;
             const uint32_t acc = n & 1u;

@@ -43,6 +43,7 @@ constexpr int kProducerWarp = 0, kExchangeWarp = 1, kWorker0 = 4, kWorkers = 4; 
 constexpr int kScorers = 4; // warps 2, 3, 8, 9: scorer w takes rows 2w and 2w + 1 of every octet
 constexpr int kMeta = 64;                 // ring of per-octet scores: more than tensor-memory plus landing slots
 constexpr int kOctRows = 8;
+constexpr int kOctPerTile = kTileRows / kOctRows; // octets per 128-row tile (the unit of Params::split)
 constexpr int kMaxP = 8;
 constexpr int kMaxRowBytes = 8192;     // d <= 4096: one octet fills a quarter of tensor memory
 constexpr int kRowPad = 16;            // bytes between rows in shared memory beyond their length
@@ -63,6 +64,7 @@ struct Params {
     int n_slots;    // tensor-memory slots (a multiple of 4)
     int n_landing;  // landing slots in shared memory
     int norm_kind, smallest;
+    TileSplit split;   // which 128-row tiles stay on the chip; the octets of the others are scored here and nothing else
     unsigned long long wait_ns;
     const char *keys;  // [B][S][d] bf16
     float *sim;        // [B][P][n_vis]
@@ -517,6 +519,16 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
             bool did = false;
             if (cs.valid() && cs.s - ms.s < n_slots) { // the slot's previous octet has been multiplied
                 const int j = (int)(cs.s % L);
+                if (!p.split.on_chip(cs.o / kOctPerTile)) {
+                    // an octet of a streamed tile: nothing to park.  The landing slot still counts this warp among those
+                    // that release it, and its barrier is in this octet's phase once the copies have been started.
+                    if (sh.issued > (uint32_t)cs.s) {
+                        if (lane == 0) mbar_arrive(smem_u32(&sh.empty[j]));
+                        do cs.next();
+                        while (cs.valid() && (cs.s & 3) != quarter);
+                        did = true;
+                    }
+                } else
                 // a parity test is only meaningful once the barrier has reached this octet's phase
                 if (sh.issued > (uint32_t)cs.s && mbar_try_wait(smem_u32(&sh.full[j]), (uint32_t)((cs.s / L) & 1))) {
                     // ---- park octet cs.s: shared memory -> registers -> tensor memory
@@ -547,6 +559,12 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
                 }
             }
             if (!did && ms.s < cs.s + (cs.valid() ? 0 : (1ll << 40))) { // parked and waiting for its sample's pivots
+                if (!p.split.on_chip(ms.o / kOctPerTile)) { // never parked: nothing of it waits for the pivot buffer
+                    if (lane == 0) sh.mma_seq[ms.s % n_slots] = (uint32_t)(ms.s + 1);
+                    do ms.next();
+                    while (ms.valid() && (ms.s & 3) != quarter);
+                    did = true;
+                } else
                 // a parity test is only meaningful once the barrier has reached this sample's phase
                 if (sh.armed > (uint32_t)ms.ord && mbar_try_wait(smem_u32(&sh.piv_full), (uint32_t)(ms.ord & 1))) {
                     // ---- multiply octet ms.s: D[pivot][token] over all columns, four accumulators in turn

@@ -18,7 +18,7 @@ DART_OK = 0
 DART_ERR_NULL, DART_ERR_BAD_SHAPE, DART_ERR_ALIGN, DART_ERR_ALIAS = -1, -2, -3, -4
 DART_ERR_CUDA, DART_ERR_NOMEM, DART_ERR_TIMEOUT, DART_ERR_CHECK, DART_ERR_UNSUPPORTED = -5, -6, -7, -8, -9
 DART_FLAG_HOST_STAGING = 1
-DART_PATH_AUTO, DART_PATH_STAGED, DART_PATH_FUSED, DART_PATH_TWO_PASS, DART_PATH_RESIDENT = 0, 1, 2, 3, 4
+DART_PATH_AUTO, DART_PATH_STAGED, DART_PATH_FUSED, DART_PATH_TWO_PASS, DART_PATH_RESIDENT, DART_PATH_SPLIT, DART_PATH_PAIRED = 0, 1, 2, 3, 4, 5, 6
 DART_RETAIN_AUTO, DART_RETAIN_SERIAL, DART_RETAIN_LISTS = 0, 1, 2
 DART_RULE_QUOTAS, DART_RULE_GLOBAL, DART_RULE_UNION = 0, 1, 2
 
@@ -42,7 +42,7 @@ class dart_opts(ctypes.Structure):
                 ("wait_limit", ctypes.c_int32), ("sweep_lag", ctypes.c_int32),
                 ("test_withhold_pivots", ctypes.c_int32), ("retention", ctypes.c_int32), ("rule", ctypes.c_int32),
                 ("cosine_on_hidden", ctypes.c_int32), ("text_pivots", ctypes.c_int32), ("pivots_in", ctypes.c_void_p),
-                ("cu_seqlens", ctypes.c_void_p)]
+                ("cu_seqlens", ctypes.c_void_p), ("resident_split", ctypes.c_int32), ("tune", ctypes.c_int32)]
 
 
 class dart_debug(ctypes.Structure):

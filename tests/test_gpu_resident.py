@@ -34,6 +34,37 @@ def test_resident_sweep_matches_the_oracle(oracle, shape):
     assert rep.max_rel_l1 < 5e-5 and rep.max_rel_l2 < 5e-5 and rep.max_abs_sim < 2e-5
 
 
+def run_split(k, h, vo, nv, P, Kp, split):
+    B, S, d = h.shape
+    ctx = dart.Dart(B, S, d, P, Kp)
+    try:
+        res = ctx.reduce(h, k, vo, nv, P, Kp, debug=True, opts=dart.dart_opts(path=dart.DART_PATH_SPLIT, resident_split=split))
+        torch.cuda.synchronize()
+        assert ctx.status() == dart.DART_OK, dart.dart_status_detail(ctx.handle)
+    finally:
+        ctx.close()
+    return res
+
+
+@pytest.mark.parametrize("split", [0, 2, 3, -3, -4, 40], ids=lambda s: "split%d" % s)
+@pytest.mark.parametrize("shape", [SHAPES[3], SHAPES[5], SHAPES[6], SHAPES[8]], ids=lambda s: "x".join(map(str, s)))
+def test_split_between_chip_and_second_read_matches_the_oracle(oracle, shape, split):
+    """Some 128-row tiles wait on the chip for the pivots, the others are read a second time by the one-pass
+    kernel: whatever the share, every row gets its similarities from exactly one of the two."""
+    from oracle import parity
+    from test_gpu_parity import _np
+
+    B, S, d, vo, nv, P, Kp = shape
+    k, h = gaussian(B, S, d, seed=900 + sum(shape))
+    res = run_split(k, h, vo, nv, P, Kp, split)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp)
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, _np(res[0]), _np(res[1]), _np(res[2]),
+                             dbg={n: _np(v) for n, v in res[3].items()})
+    assert rep.exact >= rep.above_margin
+    assert rep.max_rel_l1 < 5e-5 and rep.max_rel_l2 < 5e-5 and rep.max_abs_sim < 2e-5
+
+
 @pytest.mark.parametrize("norm_kind,smallest", [(1, 1), (2, 0), (2, 1)])
 def test_resident_sweep_ranking_variants(oracle, norm_kind, smallest):
     k, h = gaussian(3, 500, 256, seed=77)
