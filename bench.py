@@ -152,20 +152,6 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def time_oracle(w, keys_bits, hidden_bits, budget_s):
-    """Time the oracle, single-threaded and as it stands, on as many leading samples as fit the budget."""
-    import oracle
-
-    t0 = time.perf_counter()
-    oracle.reduce(hidden_bits[:1], keys_bits[:1], w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, want_dup=False)
-    t1 = time.perf_counter() - t0
-    n = int(max(1, min(keys_bits.shape[0], budget_s / max(t1, 1e-6))))
-    t0 = time.perf_counter()
-    oracle.reduce(hidden_bits[:n], keys_bits[:n], w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, want_dup=False)
-    dt = time.perf_counter() - t0
-    return n, dt
-
-
 def run_reference(args):
     """The reference arm: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
@@ -241,8 +227,10 @@ def workload_config(w, B):
                    if needs_flush(w, B) else "inputs larger than L2 (no flush needed)")}
 
 
-def time_steps(ctx, dart, torch, w, keys, hidden, outs, steps, warmup, opts, dist_on):
-    """Warm up, then time exactly `steps` reductions with CUDA events on the launching stream."""
+def time_steps(ctx, dart, torch, w, keys, hidden, outs, steps, warmup, opts, dist_on, profile_steps=None):
+    """Warm up, then time exactly `steps` reductions with CUDA events on the launching stream (no per-kernel events in
+    that loop).  A second, profiled pass of `profile_steps` steps brackets every kernel launch with events: per-kernel
+    durations and shares come from there.  Returns (total ms, per-step ms list, launches, profile dict)."""
     import torch.distributed as dist
 
     st = torch.cuda.current_stream()
@@ -255,43 +243,100 @@ def time_steps(ctx, dart, torch, w, keys, hidden, outs, steps, warmup, opts, dis
         if rc != 0:
             raise dart.DartError(rc, "dart_reduce_ex")
 
+    flush = needs_flush(w, keys.shape[0])
+    junk = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=keys.device) if flush else None
+
+    def run(n):
+        """n steps; small inputs: a buffer larger than L2 is written before every step and the steps are timed one by one"""
+        if flush:
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+            for e0, e1 in evs:
+                junk.fill_(1)
+                e0.record(st)
+                step()
+                e1.record(st)
+            torch.cuda.synchronize()
+            per = [e0.elapsed_time(e1) for e0, e1 in evs]
+            return sum(per), per
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+        evs[0].record(st)
+        for i in range(n):
+            step()
+            evs[i + 1].record(st)
+        torch.cuda.synchronize()
+        return evs[0].elapsed_time(evs[n]), [evs[i].elapsed_time(evs[i + 1]) for i in range(n)]
+
     for _ in range(warmup):
         step()
     torch.cuda.synchronize()
+    dart.dart_profile_enable(ctx.handle, False)
     dart.dart_profile_read(ctx.handle)
-    dart.dart_profile_enable(ctx.handle, True)
     n0 = dart.dart_launch_count(ctx.handle)
     if dist_on:
         dist.barrier()
     torch.cuda.synchronize()
-    if needs_flush(w, keys.shape[0]):
-        # small inputs: write a buffer larger than L2 before every step and time the steps one by one
-        junk = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=keys.device)
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-        for e0, e1 in evs:
-            junk.fill_(1)
-            e0.record(st)
-            step()
-            e1.record(st)
-        torch.cuda.synchronize()
-        ms = sum(e0.elapsed_time(e1) for e0, e1 in evs)
-        del junk
-    else:
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(st)
-        for _ in range(steps):
-            step()
-        e1.record(st)
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1)
+    ms, per = run(steps)
     if dist_on:
         dist.barrier()
     launches = dart.dart_launch_count(ctx.handle) - n0
+    # profiled pass (same call, every launch bracketed by events on the same stream)
+    dart.dart_profile_enable(ctx.handle, True)
+    run(profile_steps if profile_steps else max(3, min(steps, 20)))
     dart.dart_profile_enable(ctx.handle, False)
     _, prof = dart.dart_profile_read(ctx.handle)
     if ctx.status() != 0:
         raise RuntimeError("device status word reports an error")
-    return ms, launches, prof
+    return ms, per, launches, prof
+
+
+def oracle_leg(w, keys, hidden, ref_idx, budget_s):
+    """The CPU baseline: the oracle as it stands, single-threaded on one core (the stated baseline) and the same
+    single-threaded code over samples on all host cores (context).  The samples it computes are also compared with the
+    timed run's kept indices: exact-match rate and a histogram of the oracle's selection margins."""
+    import math
+    from concurrent.futures import ThreadPoolExecutor
+
+    import numpy as np
+
+    import oracle
+    from paper_2502_11494_b200 import workloads as W
+
+    oracle.build()
+    B = keys.shape[0]
+    cores = os.cpu_count() or 1
+    kb, hb = W.bits(keys[:1]), W.bits(hidden[:1])
+    t0 = time.perf_counter()
+    oracle.reduce(hb, kb, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, want_dup=False, want_hidden=False)
+    t1 = time.perf_counter() - t0
+    n1 = int(max(1, min(B, (budget_s / 2) / max(t1, 1e-6))))
+    nall = int(max(1, min(B, 256, cores * (budget_s / 2) / max(t1, 1e-6))))
+    nb = max(n1, nall)
+    kb, hb = W.bits(keys[:nb]), W.bits(hidden[:nb])   # only the samples the two timed passes touch go to the host
+    t0 = time.perf_counter()
+    oracle.reduce(hb[:n1], kb[:n1], w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, want_dup=False, want_hidden=False)
+    dt1 = time.perf_counter() - t0
+
+    def one(i):
+        return oracle.reduce(hb[i:i + 1], kb[i:i + 1], w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, want_dup=False, want_hidden=False)
+
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=cores) as pool:
+        res = list(pool.map(one, range(nall)))
+    dta = time.perf_counter() - t0
+    ref = ref_idx[:nall].cpu().numpy()
+    exact = sum(int(np.array_equal(ref[i], res[i].out_idx[0])) for i in range(nall))
+    margins = np.array([float(r.margin[0]) for r in res])
+    edges = [0.0, 1e-6, 1e-5, 1e-4, 1e-3, 1e-2, math.inf]
+    hist = {("<%g" % edges[k + 1]) if k + 1 < len(edges) - 1 else ">=%g" % edges[k]: int(((margins >= edges[k]) & (margins < edges[k + 1])).sum())
+            for k in range(len(edges) - 1)}
+    return {
+        "value": n1 * w.n_vis / dt1, "unit": UNIT, "cores": 1, "kind": "oracle",
+        "sample": "first %d of %d samples of %s, one pass, %.1f s" % (n1, B, w.name, dt1),
+        "all_cores": {"value": nall * w.n_vis / dta, "unit": UNIT, "cores": cores,
+                      "sample": "first %d samples, one single-threaded oracle call per sample on %d host threads, %.1f s" % (nall, cores, dta)},
+        "parity_on_sample": {"samples": nall, "identical_to_timed_run": exact, "exact_match_rate": exact / nall,
+                             "above_margin_1e-3": int((margins > 1e-3).sum()), "margin_histogram": hist},
+    }
 
 
 def main():
@@ -330,7 +375,7 @@ def main():
     outs = alloc_outs(w)
     sampler = ClockSampler(local)
     sampler.start()
-    ms, launches, prof = time_steps(ctx, dart, torch, w, keys, hidden, outs, args.steps, args.warmup, opts, dist_on)
+    ms, per_step, launches, prof = time_steps(ctx, dart, torch, w, keys, hidden, outs, args.steps, args.warmup, opts, dist_on)
     clocks = sampler.stop()
     ref_idx = outs[1].clone()  # the timed run's kept indices (the variants below write into the same buffers)
     ms = max_over_ranks(ms, dev, dist_on)
@@ -349,7 +394,7 @@ def main():
                     "traffic": (NCU_TRAFFIC_PER_SAMPLE[(dom, w.n_vis, w.d, w.n_pivot)] * B
                                 if (dom, w.n_vis, w.d, w.n_pivot) in NCU_TRAFFIC_PER_SAMPLE and args.lag == 0 else None),
                     "peak_source": peak_src + " copy bandwidth",
-                    "avg_launch_ms": avg_ms,
+                    "avg_launch_ms": avg_ms, "timing": "CUDA events around every launch of a separate profiled pass on the launching stream",
                     "shares": {k: v[0] / max(sum(x[0] for x in prof.values()), 1e-9) for k, v in prof.items()}}
     path_gbs = path_bytes_per_sample(w) * B / (ms_per_step * 1e-3) / 1e9
     path_roof = {"algorithmic_bytes_per_step": path_bytes_per_sample(w) * B, "achieved": path_gbs, "unit": "GB/s",
@@ -361,7 +406,7 @@ def main():
         for (p, k) in W.sweep_cells():
             wc = w.with_(n_pivot=p, n_keep=k)
             o2 = alloc_outs(wc)
-            ms2, _, _ = time_steps(ctx, dart, torch, wc, keys, hidden, o2, max(3, args.steps // 4), 2, opts, False)
+            ms2, _, _, _ = time_steps(ctx, dart, torch, wc, keys, hidden, o2, max(3, args.steps // 4), 2, opts, False, profile_steps=1)
             n2 = max(3, args.steps // 4)
             sweep.append({"n_pivot": p, "n_keep": k, "ms_per_step": ms2 / n2,
                           "tokens_per_s": B * wc.n_vis * n2 / (ms2 * 1e-3),
@@ -374,21 +419,21 @@ def main():
         n_v = max(3, args.steps // 4)
         # (a) retention with one threshold for all pivots
         o_g = dart.dart_opts(path=args.path, sweep_lag=args.lag, retention=args.retention, rule=dart.DART_RULE_GLOBAL)
-        ms_g, _, prof_g = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_g, False)
+        ms_g, _, _, prof_g = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_g, False, profile_steps=3)
         variants["one_threshold"] = {"ms_per_step": ms_g / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_g * 1e-3),
                                      "retain_ms": prof_g["retain"][0] / max(prof_g["retain"][1], 1)}
         # (a2) independent pivots (Eq. 10's union): variable-length packed outputs + cu_seqlens
         cu = torch.zeros(B + 1, dtype=torch.int32, device=dev)
         o_u = dart.dart_opts(path=args.path, sweep_lag=args.lag, retention=args.retention, rule=dart.DART_RULE_UNION,
                              cu_seqlens=cu.data_ptr())
-        ms_u, _, prof_u = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_u, False)
+        ms_u, _, _, prof_u = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_u, False, profile_steps=3)
         variants["independent_pivots"] = {"ms_per_step": ms_u / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_u * 1e-3),
                                           "retain_ms": prof_u["retain"][0] / max(prof_u["retain"][1], 1) * 3,  # three launches
                                           "mean_kept_vision_tokens": float(cu[-1].item()) / B - (w.S - w.n_vis)}
         # (b) pivots named by the caller (here: random distinct tokens): steps 3-5 only wait for the norms
         piv = torch.stack([torch.randperm(w.n_vis, device=dev)[:w.n_pivot] for _ in range(B)]).to(torch.int32).contiguous()
         o_p = dart.dart_opts(path=args.path, sweep_lag=args.lag, retention=args.retention, pivots_in=piv.data_ptr())
-        ms_p, _, prof_p = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_p, False)
+        ms_p, _, _, prof_p = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_p, False, profile_steps=3)
         variants["pivots_given"] = {"ms_per_step": ms_p / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_p * 1e-3),
                                     "path_frac_of_measured_copy": path_bytes_per_sample(w) * B / (ms_p / n_v * 1e-3) / 1e9 / peak}
         if prof_p.get("onepass", (0, 0))[1]:
@@ -401,13 +446,13 @@ def main():
         # (b1) the caller's pivots drawn from the whole sample, text tokens included (indices relative to the vision block)
         piv_t = (torch.stack([torch.randperm(w.S, device=dev)[:w.n_pivot] for _ in range(B)]) - w.vis_offset).to(torch.int32).contiguous()
         o_t = dart.dart_opts(path=args.path, sweep_lag=args.lag, retention=args.retention, text_pivots=1, pivots_in=piv_t.data_ptr())
-        ms_t, _, _ = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_t, False)
+        ms_t, _, _, _ = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_t, False, profile_steps=1)
         variants["text_pivots"] = {"ms_per_step": ms_t / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_t * 1e-3),
                                    "path_frac_of_measured_copy": path_bytes_per_sample(w) * B / (ms_t / n_v * 1e-3) / 1e9 / peak}
         del piv_t
         # (b2) pivots ranked by the key rows, Eq. 7 on the hidden rows: keys once (scores), hidden once (one pass)
         o_h = dart.dart_opts(path=args.path, sweep_lag=args.lag, retention=args.retention, cosine_on_hidden=1)
-        ms_h, _, prof_h = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_h, False)
+        ms_h, _, _, prof_h = time_steps(ctx, dart, torch, w, keys, hidden, outs, n_v, 2, o_h, False, profile_steps=3)
         bytes_h = (path_bytes_per_sample(w) + 2 * w.d * w.n_vis) * B   # one more read of n_vis x d than the main method
         variants["cosine_on_hidden"] = {"ms_per_step": ms_h / n_v, "tokens_per_s": B * w.n_vis * n_v / (ms_h * 1e-3),
                                         "algorithmic_bytes_per_step": bytes_h,
@@ -473,19 +518,14 @@ def main():
 
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:
-        import oracle
-
-        oracle.build()
-        nb = min(B, 128)
-        kb, hb = W.bits(keys[:nb]), W.bits(hidden[:nb])
-        n, dt = time_oracle(w, kb, hb, budget_s=15.0)
-        cpu = {"value": n * w.n_vis / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": "first %d of %d samples of %s, one pass, %.1f s" % (n, B, w.name, dt)}
+        cpu = oracle_leg(w, keys, hidden, ref_idx, budget_s=20.0)
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "ms_per_step_median": sorted(per_step)[len(per_step) // 2], "ms_per_step_best": min(per_step),
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
             "config": workload_config(w, B), "roofline": roofline, "path_roofline": path_roof,
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,

@@ -117,8 +117,11 @@ typedef struct {
     int32_t path;          /* DART_PATH_* */
     int32_t wait_limit;    /* 0: default (2 s); > 0: time limit in microseconds of every bounded device-side wait */
     int32_t sweep_lag;     /* 0: default; > 0: fused path, extra tasks between a row's two sweeps (tuning) */
-    int32_t test_withhold_pivots; /* testing only: nonzero makes the fused kernel never publish a sample's pivots, so that
-                                     its bounded waits expire and the call ends with DART_ERR_TIMEOUT in dart_status */
+    int32_t test_withhold_pivots; /* testing only: nonzero withholds one hand-over inside the kernel that waits (the persistent
+                                     sweep never publishes a sample's pivots; the resident sweep's CTAs never count themselves in;
+                                     the one-pass kernel's first pivot-norm warp never hands its norms over; the paired sweeps:
+                                     1 = the lists are never counted in, 2 = the pivots' norms never reach the epilogue), so that
+                                     the bounded waits expire and the call ends with DART_ERR_TIMEOUT in dart_status */
     int32_t retention;     /* DART_RETAIN_*: how step 4 is scheduled (same result either way) */
     int32_t rule;          /* DART_RULE_*: which tokens step 4 retains */
     int32_t cosine_on_hidden; /* 0: Eq. 7 on the key rows that are scored (one tensor for steps 1-3).  1: the pivots are still
@@ -144,7 +147,9 @@ typedef struct {
                               cu_seqlens[b + 1] = cu_seqlens[b] + packed length of sample b. */
     int32_t resident_split; /* DART_PATH_SPLIT: 0 = default (every second tile stays on the chip); k >= 2: the tiles with
                               index % k == 0 stay (a share of 1/k); -k: all other tiles stay (a share of 1 - 1/k) */
-    int32_t tune;          /* 0 = defaults.  DART_PATH_PAIRED: 256 * n1 + 16 * n2 + n3 = depths of the three shared-memory rings (tuning) */
+    int32_t tune;          /* 0 = defaults.  DART_PATH_PAIRED: 256 * n1 + 16 * n2 + n3 = depths of the three shared-memory rings.
+                              DART_PATH_FUSED: >= 2 cuts the second pass of a row tile into eight column chunks (one task each)
+                              and keeps the first pass within `tune` steps of the second (both tuning options) */
 } dart_opts;
 
 /* Optional per-step outputs of dart_reduce_ex; every member is a device pointer or NULL. */
@@ -245,8 +250,10 @@ int dart_status(dart_ctx *ctx);
  * Where the last non-zero status came from (as read by the last dart_status call that returned an error):
  * detail[0] = which bounded wait of the fused kernel expired (1 pivots not published, 2 ring stage not freed,
  * 3 drain, 4 accumulator not freed, 5/6 tile not loaded (MMA / row sums), 7 accumulator not filled, 8/9 mailbox,
- * 10 sweep-1 tasks not all counted, 11/12 selection queue; 64-70 the one-pass kernel's waits (stage not freed, tile not
- * loaded (MMA / norms), accumulator not freed / not filled, norms not taken / not ready); 100 = a failed check of
+ * 10 sweep-1 tasks not all counted, 11/12 selection queue, 13 first pass held back; 40-55 the paired sweeps' waits (44 a
+ * sample's lists not all counted in, 50 its pivots not published, 51 their norms not handed over, ...); 64-70 the one-pass
+ * kernel's waits (stage not freed, tile not loaded (MMA / norms), accumulator not freed / not filled, norms not taken /
+ * not ready); 80-86 the resident sweep's waits (83 = a sample's candidates not all published); 100 = a failed check of
  * opts->pivots_in),
  * detail[1] = index of the step in the kernel's schedule (or the sample), detail[2] = CTA; for wait 1 also
  * detail[3] = sample.  For bug reports.

@@ -15,6 +15,9 @@
 
 namespace {
 
+constexpr int kSweepChunks = 8;     // column chunks per row tile of the persistent sweep's second pass
+constexpr int kSweepChunkMaxP = 16; // ... for up to this many pivots
+
 enum Slot { SLOT_SCORE = 0, SLOT_PIVOT, SLOT_SIM, SLOT_RETAIN, SLOT_GATHER, SLOT_SWEEP, SLOT_ONEPASS, SLOT_RESIDENT, SLOT_PAIR, SLOT_COUNT };
 const char *const kSlotNames[SLOT_COUNT] = {"score", "pivot", "sim", "retain", "gather", "sweep", "onepass", "resident", "pair"};
 
@@ -63,6 +66,7 @@ struct dart_ctx {
     int sm_count, n_atoms;
     int *counters;
     size_t counters_bytes;
+    float *sim_share;     // [kSweepChunks][B_max][min(P_max, 16)][S_max]: the column chunks' shares of the similarities (NULL: none)
     TensorMapEncodeFn encode;
     // resident sweep (csrc/dart_resident.cuh)
     bool resident_ok;
@@ -293,8 +297,9 @@ int launch_staged(dart_ctx *ctx, int B, const void *hidden, const void *keys_in,
     } else {
         Prof p(ctx, st, SLOT_PIVOT);
         int P_pad = next_pow2(P);
-        pivot_kernel<<<B, kSelectThreads, (size_t)P_pad * 8, st>>>(o.norm_kind == 2 ? ctx->ssq : ctx->l1, n_vis, P,
-                                                                  P_pad, o.pivot_smallest, ctx->pivot_idx);
+        const bool cached = n_vis <= kPivotCacheMax;
+        pivot_kernel<<<B, kSelectThreads, pivot_smem_bytes(n_vis, P_pad, cached), st>>>(o.norm_kind == 2 ? ctx->ssq : ctx->l1, n_vis, P,
+                                                                                       P_pad, o.pivot_smallest, cached, ctx->pivot_idx);
     }
     {
         Prof p(ctx, st, SLOT_SIM);
@@ -333,6 +338,11 @@ int fused_setup(dart_ctx *ctx)
     ctx->counters_bytes = (size_t)D.B_max * 2 * sizeof(int);
     if (rc == DART_OK) rc = ws_alloc(ctx, (uint8_t **)&ctx->counters, ctx->counters_bytes);
     if (rc != DART_OK) return rc;
+    {   // shares of the similarities for up to 16 pivots; contexts that would need more than 1 GiB go without
+        const size_t n = (size_t)kSweepChunks * D.B_max * (D.P_max < kSweepChunkMaxP ? D.P_max : kSweepChunkMaxP) * D.S_max;
+        if (n * sizeof(float) <= ((size_t)1 << 30)) rc = ws_alloc(ctx, &ctx->sim_share, n);
+        if (rc != DART_OK) return rc;
+    }
     if (cudaFuncSetAttribute(sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - kStaticSmemReserve) !=
         cudaSuccess)
         return DART_ERR_CUDA;
@@ -419,7 +429,15 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     Params p = {};
     p.B = B, p.S = S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.N = (P + 15) / 16 * 16, p.d8 = d8;
     p.n_atoms = ctx->n_atoms, p.n_rt = (n_vis + kTileRows - 1) / kTileRows;
-    p.T1 = (n_vis + kS1Rows - 1) / kS1Rows, p.T2 = p.n_rt, p.Tm = p.T1 > p.T2 ? p.T1 : p.T2;
+    // Option (dart_opts.tune >= 2): the second pass over a row tile is cut into chunks of columns, one task each (the size of
+    // a first-pass task), so that a sample's second pass is spread over all SMs like its first; every chunk writes its share of
+    // the similarities and sim_sum_kernel adds them up; the first pass then runs at most `tune` steps ahead of the second.
+    // Measured on the 256-sample workload: no gain (1.81-1.89 ms against 1.86 ms): the pivots of a sample take three to
+    // four rounds of steps to appear, and holding the first pass back that closely stalls it as much as the L2 then saves.
+    p.n_kc = (ctx->sim_share && P <= kSweepChunkMaxP && o.tune >= 2) ? (p.n_atoms < kSweepChunks ? p.n_atoms : kSweepChunks) : 1;
+    p.apc = (p.n_atoms + p.n_kc - 1) / p.n_kc;
+    p.n_kc = (p.n_atoms + p.apc - 1) / p.apc;
+    p.T1 = (n_vis + kS1Rows - 1) / kS1Rows, p.T2 = p.n_rt * p.n_kc, p.Tm = p.T1 > p.T2 ? p.T1 : p.T2;
     p.row_bytes = (uint32_t)ctx->desc.d * 2, p.stage1_bytes = stage1_bytes(p.row_bytes);
     ring_depths(p.N, p.row_bytes, ctx->max_smem_optin, p.n1, p.n2);
     if (p.n1 < 2) return DART_ERR_UNSUPPORTED;
@@ -430,9 +448,11 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     if (n_all + p.lag >= (1ll << 30)) return DART_ERR_UNSUPPORTED;
     p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest;
     p.withhold_pivots = o.test_withhold_pivots;
+    p.keep_l2 = p.n_kc > 1;
+    p.ahead = o.tune >= 2 ? (uint32_t)o.tune : 0u;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
     p.keys = (const char *)keys;
-    p.sim = ctx->sim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
+    p.sim = p.n_kc > 1 ? ctx->sim_share : ctx->sim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
     p.s1_done = ctx->counters, p.piv_ready = ctx->counters + B;
     p.status = ctx->status;
     // the same tensor with a 128-row box (full tiles), a 32-row box (short last tiles) and a one-row box (pivot rows)
@@ -448,6 +468,17 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
         void *args[4] = {&tm_tile, &tm_keys, &tm_row, &p};
         DART_CUDA(ctx, cudaLaunchCooperativeKernel((const void *)sweep_kernel, dim3((unsigned)grid), dim3(kThreads), args,
                                                    smem_bytes(p.N, p.row_bytes, p.n1, p.n2), st));
+    }
+    if (p.n_kc > 1) {
+        Prof pr(ctx, st, SLOT_SIM);
+        const long long n = (long long)B * P * n_vis; // the shares of every chunk lie n floats apart
+        const bool vec = n % 4 == 0;
+        const long long items = vec ? n / 4 : n, want = (items + kSimSumThreads - 1) / kSimSumThreads;
+        const unsigned grid = (unsigned)(want < 8ll * ctx->sm_count ? want : 8ll * ctx->sm_count);
+        if (vec)
+            sim_sum_kernel<float4><<<grid, kSimSumThreads, 0, st>>>((const float4 *)ctx->sim_share, items, p.n_kc, (float4 *)ctx->sim);
+        else
+            sim_sum_kernel<float><<<grid, kSimSumThreads, 0, st>>>(ctx->sim_share, items, p.n_kc, ctx->sim);
     }
     launch_retention(ctx, B, pos_in, vis_offset, n_vis, P, n_keep, out_idx, out_pos, o, st);
     launch_gather(ctx, B, hidden, n_vis, n_keep, out_idx, out_hidden, o, st);
@@ -473,6 +504,7 @@ int launch_onepass_kernel(dart_ctx *ctx, int B, const void *src, bool scores_els
     p.n_st = onepass::ring_depth(p.N, p.aps, ctx->max_smem_optin);
     if (p.n_st < 2) return DART_ERR_UNSUPPORTED;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
+    p.withhold = o.test_withhold_pivots;
     p.sim = ctx->sim, p.l1 = scores_elsewhere ? nullptr : ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
     p.status = ctx->status;
     p.compact = ctx->piv_rows != nullptr && P > onepass::kGatherMaxP;
@@ -520,7 +552,7 @@ int launch_resident(dart_ctx *ctx, int B, const void *hidden, const void *keys_i
     p.B = B, p.S = ctx->S, p.vis_offset = vis_offset, p.n_vis = n_vis, p.P = P, p.d = ctx->desc.d;
     p.n_oct = (n_vis + R::kOctRows - 1) / R::kOctRows;
     p.n_slots = R::tmem_slots(ctx->desc.d), p.n_landing = ctx->res_landing;
-    p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest;
+    p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest, p.withhold = o.test_withhold_pivots;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
     p.keys = (const char *)(keys_in ? keys_in : hidden);
     p.sim = ctx->sim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
@@ -623,8 +655,9 @@ int launch_two_pass(dart_ctx *ctx, int B, const void *hidden, const void *keys, 
     } else {
         Prof p(ctx, st, SLOT_PIVOT);
         const int P_pad = next_pow2(P);
-        pivot_kernel<<<B, kSelectThreads, (size_t)P_pad * 8, st>>>(o.norm_kind == 2 ? ctx->ssq : ctx->l1, n_vis, P, P_pad,
-                                                                  o.pivot_smallest, ctx->pivot_idx);
+        const bool cached = n_vis <= kPivotCacheMax;
+        pivot_kernel<<<B, kSelectThreads, pivot_smem_bytes(n_vis, P_pad, cached), st>>>(o.norm_kind == 2 ? ctx->ssq : ctx->l1, n_vis, P, P_pad,
+                                                                                       o.pivot_smallest, cached, ctx->pivot_idx);
     }
     if (tensor_cores) {
         int rc = launch_onepass_kernel(ctx, B, sim_src, true, vis_offset, n_vis, P, o, st);
@@ -780,6 +813,9 @@ int dart_create(dart_ctx **out, const dart_desc *desc)
                           cudaFuncSetAttribute(dart::pack_varlen_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                ctx->max_smem_optin - 2048) != cudaSuccess))
         rc = DART_ERR_CUDA;
+    if (rc == DART_OK && cudaFuncSetAttribute(dart::pivot_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)dart::pivot_smem_bytes(dart::kPivotCacheMax, 1024, true)) != cudaSuccess)
+        rc = DART_ERR_CUDA;
     if (rc == DART_OK && ctx->cand) {
         // the two-phase kernels may use up to the device's shared memory; shapes that need more fall back at launch
         if (cudaFuncSetAttribute(dart::candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -840,6 +876,7 @@ int dart_destroy(dart_ctx *ctx)
     cudaFree(ctx->piv_rows);
     cudaFree(ctx->status);
     cudaFree(ctx->counters);
+    cudaFree(ctx->sim_share);
     cudaFree(ctx->res_cand);
     cudaFree(ctx->pair_cand);
     cudaFree(ctx->pair_res);
@@ -1063,7 +1100,7 @@ int dart_pivots_static(const void *keys, int B, int S, int d, int vis_offset, in
     score_kernel<<<(unsigned)((rows + kScoreWarps - 1) / kScoreWarps), kScoreWarps * 32, 0, st>>>(
         (const uint4 *)keys, S, d / 8, vis_offset, n_vis, rows, l1, ssq);
     const int P_pad = next_pow2(n_pivot);
-    pivot_kernel<<<B, kSelectThreads, (size_t)P_pad * 8, st>>>(l1, n_vis, n_pivot, P_pad, 0, pivot_idx);
+    pivot_kernel<<<B, kSelectThreads, pivot_smem_bytes(n_vis, P_pad, false), st>>>(l1, n_vis, n_pivot, P_pad, 0, 0, pivot_idx);
     const cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? DART_OK : e == cudaErrorMemoryAllocation ? DART_ERR_NOMEM : DART_ERR_CUDA;
 }

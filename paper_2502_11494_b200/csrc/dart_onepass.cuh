@@ -47,6 +47,7 @@ struct Params {
     int compact;                       // pivot tiles come from the compact copy [B][N][d] (tm_piv), not by gather4
     int n_sel;                         // row tiles per sample this launch takes: n_rt, or the streamed tiles of `split`
     TileSplit split;                   // k <= 1: all tiles
+    int withhold;                      // test hook: the first pivot-norm warp never hands its norms over, so that the bounded waits expire
     unsigned long long wait_ns;
     float *sim;                        // [B][P][n_vis] dup(p_i, x_j)
     float *l1, *ssq;                   // [B][n_vis]; l1 may be NULL (the scores come from another tensor)
@@ -115,7 +116,8 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
     };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned long long limit = 2ull * p.wait_ns; // ns -> cycles at the highest SM clock: never shorter than asked
-    const Ctl ctl{&sh.abort_flag, p.status, warp == 0 ? limit : limit + limit / 4};
+    // the epilogue waits for everything else, so its waits are nearest to whatever is missing: shortest limit; then the producer
+    const Ctl ctl{&sh.abort_flag, p.status, warp >= kEpi0 ? limit : warp == 0 ? limit + limit / 8 : limit + limit / 4};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -325,7 +327,7 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
             for (int k = 0; k < kMaxN / kPivThreads; ++k)
                 if (u + kPivThreads * k < p.P) sh.piv_ssq[acc][u + kPivThreads * k] = pq[k][0] + pq[k][1];
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sh.norm_full[acc]));
+            if (lane == 0 && !(p.withhold && warp == kPivWarp0)) mbar_arrive(smem_u32(&sh.norm_full[acc]));
             ++n;
         }
     } else if (warp >= kEpi0 && warp < kEpi0 + kEpiWarps) {

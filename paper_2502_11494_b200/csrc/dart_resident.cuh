@@ -65,6 +65,7 @@ struct Params {
     int n_landing;  // landing slots in shared memory
     int norm_kind, smallest;
     TileSplit split;   // which 128-row tiles stay on the chip; the octets of the others are scored here and nothing else
+    int withhold;      // test hook: no CTA ever counts itself in after publishing its candidates, so that the bounded waits expire
     unsigned long long wait_ns;
     const char *keys;  // [B][S][d] bf16
     float *sim;        // [B][P][n_vis]
@@ -262,7 +263,8 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
     const uint32_t cand_off = (1u + (uint32_t)p.n_landing) * octb; // [G][kMaxP] candidate keys of the current sample
     unsigned long long *cand_sm = reinterpret_cast<unsigned long long *>(smem_raw + ((smem0 - smem_u32(smem_raw)) + cand_off));
     const unsigned long long limit = 2ull * p.wait_ns; // ns -> cycles at the highest SM clock: never shorter than asked
-    const Ctl ctl{&sh.abort_flag, p.status, warp == kProducerWarp ? limit : limit + limit / 4};
+    // the exchange warp is the one that waits for other CTAs: shortest limit, so that its wait reports first; then the producer
+    const Ctl ctl{&sh.abort_flag, p.status, warp == kExchangeWarp ? limit : warp == kProducerWarp ? limit + limit / 8 : limit + limit / 4};
     const int L = p.n_landing, n_slots = p.n_slots;
     const uint32_t cols_per_oct = (uint32_t)p.d / 8u;
 
@@ -363,7 +365,7 @@ __global__ void __launch_bounds__(kThreads, 1) resident_kernel(const Params p)
             __syncwarp();
             const int contributors = p.n_oct < G ? p.n_oct : G;
             if (lane == 0) {
-                atomicAdd(p.arrived + n, 1);
+                if (!p.withhold) atomicAdd(p.arrived + n, 1);
                 ok = ctl.wait_flag(p.arrived + n, kWaitPublished, n, contributors);
             }
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;

@@ -58,48 +58,60 @@ score_kernel(const uint4 *__restrict__ keys, int S, int d8, int vis_offset, int 
 // ------------------------------------------------------------------------------------------------
 constexpr int kSelectThreads = 512;
 
+// n distinct 64-bit entries of `list` in ascending order without a single barrier between compare-exchange stages: every
+// thread counts the entries smaller than its own (shared-memory broadcasts) and hands (rank, entry) to `put`.  Cheaper than
+// a bitonic sort (log^2 n barriers) while n^2 / threads stays small.
+constexpr int kRankSortMax = 1024;
+template <typename Put>
+__device__ __forceinline__ void rank_sort(const unsigned long long *list, int n, Put put)
+{
+    for (int t = threadIdx.x; t < n; t += blockDim.x) {
+        const unsigned long long x = list[t];
+        int r = 0;
+        for (int u = 0; u < n; ++u) r += list[u] < x ? 1 : 0;
+        put(r, x);
+    }
+}
+
+inline size_t pivot_smem_bytes(int n_vis, int P_pad, bool cached) { return (size_t)P_pad * 8 + (cached ? (size_t)n_vis * 4 : 0); }
+constexpr int kPivotCacheMax = 32768; // scores of a sample that are kept in shared memory as keys (128 KB)
+
 __global__ void __launch_bounds__(kSelectThreads)
-pivot_kernel(const float *__restrict__ score, int n_vis, int P, int P_pad, int smallest,
+pivot_kernel(const float *__restrict__ score, int n_vis, int P, int P_pad, int smallest, int cached,
              int32_t *__restrict__ pivot_idx)
 {
-    extern __shared__ unsigned long long piv_list[]; // [P_pad]
+    extern __shared__ unsigned long long piv_list[]; // [P_pad], then (cached) the sample's keys [n_vis]
+    uint32_t *keys = reinterpret_cast<uint32_t *>(piv_list + P_pad);
     __shared__ SelectSmem sel;
     __shared__ uint32_t n_picked;
     const int b = blockIdx.x;
     const float *s = score + (size_t)b * n_vis;
-    // smaller key = better pivot
+    // smaller key = better pivot.  The select reads every key five times: from shared memory when the sample fits.
+    if (cached)
+        for (int j = threadIdx.x; j < n_vis; j += blockDim.x) {
+            const uint32_t k = order_key(s[j]);
+            keys[j] = smallest ? k : ~k;
+        }
     auto keyfn = [&](int j, uint32_t &key) {
-        uint32_t k = order_key(s[j]);
-        key = smallest ? k : ~k;
+        if (cached) {
+            key = keys[j];
+        } else {
+            uint32_t k = order_key(s[j]);
+            key = smallest ? k : ~k;
+        }
         return true;
     };
     for (int i = threadIdx.x; i < P_pad; i += blockDim.x) piv_list[i] = ~0ull;
     if (threadIdx.x == 0) n_picked = 0;
+    __syncthreads();
     uint32_t T, need_eq, cnt_eq;
     block_select_threshold(CtaGroup(), keyfn, n_vis, (uint32_t)P, sel, T, need_eq, cnt_eq);
     block_select_apply(CtaGroup(), keyfn, n_vis, T, need_eq, cnt_eq, sel, [&](int j, uint32_t key) {
         uint32_t slot = atomicAdd(&n_picked, 1u);
         piv_list[slot] = ((unsigned long long)key << 32) | (uint32_t)j;
     });
-    // ascending bitonic sort of (key, index): rank 0 = best score, ties to the lower index
-    for (int k = 2; k <= P_pad; k <<= 1) {
-        for (int jj = k >> 1; jj > 0; jj >>= 1) {
-            for (int i = threadIdx.x; i < P_pad; i += blockDim.x) {
-                int l = i ^ jj;
-                if (l > i) {
-                    unsigned long long x = piv_list[i], y = piv_list[l];
-                    bool up = ((i & k) == 0);
-                    if ((x > y) == up) {
-                        piv_list[i] = y;
-                        piv_list[l] = x;
-                    }
-                }
-            }
-            __syncthreads();
-        }
-    }
-    for (int i = threadIdx.x; i < P; i += blockDim.x)
-        pivot_idx[(size_t)b * P + i] = (int32_t)(piv_list[i] & 0xffffffffu);
+    // ascending order of (key, index): rank 0 = best score, ties to the lower index
+    rank_sort(piv_list, P, [&](int r, unsigned long long x) { pivot_idx[(size_t)b * P + r] = (int32_t)(x & 0xffffffffu); });
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -441,13 +453,18 @@ candidates_kernel(const float *__restrict__ sim, const int32_t *__restrict__ piv
         key = keys[j];
         return true;
     };
+    int32_t *out = cand + ((size_t)b * P + i) * cand_stride;
     uint32_t T, need_eq, cnt_eq;
     block_select_threshold(CtaGroup(), keyfn, n_vis, (uint32_t)M, sel, T, need_eq, cnt_eq);
     block_select_apply(CtaGroup(), keyfn, n_vis, T, need_eq, cnt_eq, sel, [&](int j, uint32_t key) {
         const uint32_t slot = atomicAdd(&n_picked, 1u);
         if (slot < (uint32_t)mp) list[slot] = ((unsigned long long)key << 32) | (uint32_t)j;
     });
-    // ascending bitonic sort of (key, index): lowest dup first, equal dups by index
+    if (M <= kRankSortMax) { // lowest dup first, equal dups by index
+        rank_sort(list, M, [&](int r, unsigned long long x) { out[r] = (int32_t)(x & 0xffffffffu); });
+        return;
+    }
+    // ascending bitonic sort of (key, index)
     for (int k = 2; k <= mp; k <<= 1) {
         for (int jj = k >> 1; jj > 0; jj >>= 1) {
             for (int t = threadIdx.x; t < mp; t += blockDim.x) {
@@ -464,7 +481,6 @@ candidates_kernel(const float *__restrict__ sim, const int32_t *__restrict__ piv
             __syncthreads();
         }
     }
-    int32_t *out = cand + ((size_t)b * P + i) * cand_stride;
     for (int t = threadIdx.x; t < M; t += blockDim.x) out[t] = (int32_t)(list[t] & 0xffffffffu);
 }
 
@@ -782,6 +798,26 @@ gather_kernel(const uint4 *__restrict__ hidden, const int32_t *__restrict__ out_
             int c = c0 + u * 32 + lane;
             if (c < d8) st_stream(dst + c, v[u]);
         }
+    }
+}
+
+// Adds up the column chunks' shares of the similarities (the persistent sweep cuts every row tile into chunks of columns
+// so that all SMs re-read a sample at the same time): sim[i] = share[0][i] + share[1][i] + ... in this fixed order.
+constexpr int kSimSumThreads = 256;
+template <typename V>
+__global__ void __launch_bounds__(kSimSumThreads) sim_sum_kernel(const V *__restrict__ share, long long n, int n_kc, V *__restrict__ sim)
+{
+    for (long long i = (long long)blockIdx.x * kSimSumThreads + threadIdx.x; i < n; i += (long long)gridDim.x * kSimSumThreads) {
+        V a = __ldcs(share + i);
+        for (int k = 1; k < n_kc; ++k) {
+            const V b = __ldcs(share + (size_t)k * n + i);
+            if constexpr (sizeof(V) == 16) {
+                a.x += b.x, a.y += b.y, a.z += b.z, a.w += b.w;
+            } else {
+                a += b;
+            }
+        }
+        sim[i] = a;
     }
 }
 

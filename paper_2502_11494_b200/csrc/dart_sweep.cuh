@@ -59,7 +59,7 @@ constexpr int kStaticSmemReserve = 28672;
 constexpr int kStatusTimeout = -7;
 // which wait expired (second status word)
 enum { kWaitPivots = 1, kWaitEmptyStage, kWaitDrain, kWaitAccumFree, kWaitStageMma, kWaitStageRows, kWaitAccumFull,
-       kWaitMailSlot, kWaitMail, kWaitTasks, kWaitDutySlot, kWaitDuty };
+       kWaitMailSlot, kWaitMail, kWaitTasks, kWaitDutySlot, kWaitDuty, kWaitAhead };
 
 using Workers = WarpGroup<kWorkerWarp0, kWorkerWarps, 1>;
 using Selectors = WarpGroup<kSelWarp0, kSelWarps, 2>;
@@ -67,16 +67,19 @@ using Selectors = WarpGroup<kSelWarp0, kSelWarps, 2>;
 struct Params {
     int B, S, vis_offset, n_vis, P, N; // N = P rounded up to a multiple of 16 (MMA N)
     int d8;                            // row width in 16-byte units
-    int n_atoms, n_rt;                 // sweep 2: 64-column atoms per row; row tiles (tasks) per sample
+    int n_atoms, n_rt;                 // sweep 2: 64-column atoms per row; row tiles per sample
+    int n_kc, apc;                     // sweep 2: column chunks per row tile (tasks per tile) and atoms per chunk
     int T1, T2, Tm;                    // tasks per sample: sweep 1, sweep 2; slots per sample = max of both
     int n1, n2;                        // depth of ring 1 and ring 2 (<= kMaxStages each)
     uint32_t row_bytes, stage1_bytes;  // d * 2; shared-memory bytes of a ring-1 stage (4 rows, 1 KB granules)
     uint32_t lag;                      // steps between the two sweeps (Tm <= lag <= B * Tm)
     int norm_kind, smallest;
     int withhold_pivots;               // test hook: never publish pivots, so that the bounded waits expire
+    int keep_l2;                       // first-pass reads ask the L2 to keep the row (the second pass follows within microseconds)
+    uint32_t ahead;                    // 0: no limit; else the first pass runs at most this many steps ahead of the CTA's second pass
     unsigned long long wait_ns;        // time limit of every wait
     const char *keys;                  // [B][S][d] bf16
-    float *sim;                        // [B][P][n_vis] dup(p_i, x_j)
+    float *sim;                        // [B][P][n_vis] dup(p_i, x_j); with n_kc > 1: [n_kc][B][P][n_vis], every chunk's share of it
     float *l1, *ssq;                   // [B][n_vis]
     int32_t *pivot_idx;                // [B][P]
     int *s1_done;                      // [B] sweep-1 tasks counted per sample
@@ -87,7 +90,7 @@ struct Params {
 struct Task {
     int b;
     int u;      // sweep 1: task index within the sample (rows 16 u ...)
-    int rt;     // sweep 2: row tile
+    int rt, kc; // sweep 2: row tile and column chunk
 };
 
 // Schedule.  Every sample owns Tm consecutive slots in each sweep (a slot beyond the sweep's own task count is
@@ -105,9 +108,9 @@ __device__ __forceinline__ bool decode(const Params &p, uint32_t q, int kind, Ta
     t.u = (int)u;
     if (kind == 0) return u < (uint32_t)p.T1;
     // a sample's T2 sweep-2 tasks are spread evenly over its Tm slots (every stride-th slot carries one)
-    const uint32_t stride = Tm / (uint32_t)p.T2;
-    t.rt = (int)(u / stride);
-    return u % stride == 0 && t.rt < p.T2;
+    const uint32_t stride = Tm / (uint32_t)p.T2, idx = u / stride;
+    t.rt = (int)(idx / (uint32_t)p.n_kc), t.kc = (int)(idx - (uint32_t)t.rt * (uint32_t)p.n_kc); // a tile's chunks side by side
+    return u % stride == 0 && idx < (uint32_t)p.T2;
 }
 
 
@@ -320,6 +323,7 @@ struct Shared {
     uint32_t tmem_base, n_picked;
     float pivot_norm[kEpiWarps][kMaxN]; // per epilogue warp: Euclidean norms of the current sample's pivots
     int abort_flag;
+    volatile uint32_t s2_step;          // the step whose second-pass task the MMA issuer looks at next
 };
 static_assert(sizeof(Shared) + 64 <= kStaticSmemReserve, "static shared memory exceeds its reserve");
 
@@ -493,6 +497,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             mbar_init(smem_u32(&sh.duty_empty[m]), 1);
         }
         sh.abort_flag = 0;
+        sh.s2_step = blockIdx.x;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     uint32_t tmem_cols = 32;
@@ -512,16 +517,31 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
     if (warp == 0) {
         // ------------------------------------------------------------------ sweep-1 producer
         if (lane == 0) {
+            // With the second pass cut into column chunks a row is read again a few microseconds later: the L2 is asked to keep
+            // it.  With whole-tile tasks the second read comes ~100 MB of newer rows later, and nothing is kept.
             unsigned long long pol_keep;
-            // the second read of a row follows once the sample's pivots exist, 13-20 us later: by then ~100 MB of newer rows
-            // have passed and the L2 (which keeps a row for about 57 MB of traffic) no longer has it, so nothing is kept
-            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_keep));
+            if (p.keep_l2)
+                asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+            else
+                asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_keep));
             Ring ring(p.n1);
             long long issued = 0;
             bool ok = true;
             for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
                 Task t;
                 if (!decode(p, g, 0, t)) continue;
+                if (p.ahead) { // not too far ahead of the second pass: what it reads again should still be in the L2
+                    const long long t0 = clock64();
+                    for (uint32_t it = 0; g > p.ahead && sh.s2_step < g - p.ahead; ++it) {
+                        __nanosleep(64);
+                        if ((it & 31u) == 31u && (ctl.aborted() || (unsigned long long)(clock64() - t0) > ctl.limit_cycles)) {
+                            if (!ctl.aborted()) ctl.give_up(kWaitAhead, g);
+                            ok = false;
+                            break;
+                        }
+                    }
+                    if (!ok) break;
+                }
                 const int row0 = t.u * kS1Rows, rows = min(kS1Rows, p.n_vis - row0);
                 const char *src = p.keys + ((size_t)t.b * p.S + p.vis_offset + row0) * (size_t)p.row_bytes;
                 for (int r = 0; r < rows; r += kS1StageRows) {
@@ -572,11 +592,11 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                     }
                 cur_b = t.b;
             }
-            const int na = p.n_atoms;
+            const int a_lo = t.kc * p.apc, na = min(p.n_atoms, a_lo + p.apc);
             const int rows = min(kTileRows, p.n_vis - t.rt * kTileRows);
             const int n_sub = (rows + kSubRows - 1) / kSubRows;
             const int y0 = t.b * p.S + p.vis_offset + t.rt * kTileRows;
-            for (int a = 0; a < na; ++a) {
+            for (int a = a_lo; a < na; ++a) {
                 const uint32_t full = smem_u32(&sh.full2[ring.stage]);
                 if (lane == 0) {
                     ok = ctl.wait_bar(smem_u32(&sh.empty2[ring.stage]), ring.phase ^ 1u, kWaitEmptyStage, g);
@@ -616,14 +636,15 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             bool ok = true;
             for (uint32_t g = blockIdx.x; ok && g < total; g += gridDim.x) {
                 Task t;
+                sh.s2_step = g;
                 if (!decode(p, g, 1, t)) continue;
-                const int na = p.n_atoms;
+                const int a_lo = t.kc * p.apc, na = min(p.n_atoms, a_lo + p.apc);
                 const uint32_t acc = s2n & 1u;
                 ok = ctl.wait_bar(smem_u32(&sh.tmem_empty[acc]), ((s2n >> 1) & 1u) ^ 1u, kWaitAccumFree, g);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem_base + acc * (uint32_t)p.N;
-                for (int a = 0; a < na; ++a) {
+                for (int a = a_lo; a < na; ++a) {
                     ok = ctl.wait_bar(smem_u32(&sh.full2[ring.stage]), ring.phase, kWaitStageMma, g);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -631,7 +652,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
 #pragma unroll
                     for (int k = 0; k < kAtomCols / 16; ++k) // 16 columns = 32 bytes per MMA: advance the start address
                         umma_bf16(d_tmem, da + (unsigned long long)(2 * k), db + (unsigned long long)(2 * k), idesc,
-                                  (a | k) != 0);
+                                  ((a - a_lo) | k) != 0);
                     umma_commit(smem_u32(&sh.empty2[ring.stage])); // frees the stage once the MMAs have read it
                     ring.advance();
                 }
@@ -639,6 +660,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
                 umma_commit(smem_u32(&sh.tmem_full[acc]));
                 ++s2n;
             }
+            sh.s2_step = 0xfffffff0u; // nothing holds the first pass back any more
             if (!ok || ctl.aborted()) { // TMEM is freed at the end: first let the MMAs issued so far finish
                 umma_commit(smem_u32(&sh.mma_drain));
                 ctl.wait_landed(smem_u32(&sh.mma_drain), 0);
@@ -672,7 +694,8 @@ sweep_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant_
             }
             const float nj = row < rows ? sqrtf(__ldcg(p.ssq + (size_t)t.b * p.n_vis + j)) : 0.f;
             const uint32_t taddr = tmem_base + acc * (uint32_t)p.N + ((uint32_t)(quarter * 32) << 16);
-            float *dst = p.sim + (size_t)t.b * p.P * p.n_vis + j;
+            // a chunk's share of dup: its part of the dot product over the same two norms; the shares are added up afterwards
+            float *dst = p.sim + ((size_t)t.kc * p.B + t.b) * p.P * p.n_vis + j;
             for (int c0 = 0; c0 < p.P; c0 += 8) {
                 float v[8];
                 tmem_ld8(taddr + (uint32_t)c0, v); // warp-collective: rows outside the tile still take part

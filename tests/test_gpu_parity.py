@@ -298,6 +298,27 @@ def test_fused_path_with_short_and_long_lags(oracle, lag):
     assert all(np.array_equal(a[3][n], b[3][n], equal_nan=(n == "eps")) for n in a[3])
 
 
+@pytest.mark.parametrize("ahead", [2, 200, 2000])
+def test_fused_path_with_the_second_pass_cut_into_column_chunks(oracle, ahead):
+    """Option of the persistent sweep: every row tile's second pass as eight tasks of 512 columns whose shares of the
+    similarities are added up afterwards, the first pass held within `ahead` steps of the second."""
+    w = W.LLAVA_NEXT_B8.with_(B=3)
+    k, h = W.make_batch(w, device="cuda")
+    ctx = dart.Dart(w.B, w.S, w.d, w.n_pivot, w.n_keep)
+    try:
+        res = ctx.reduce(h, k, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, debug=True,
+                         opts=dart.dart_opts(path=dart.DART_PATH_FUSED, tune=ahead))
+        torch.cuda.synchronize()
+        assert ctx.status() == dart.DART_OK, dart.dart_status_detail(ctx.handle)
+    finally:
+        ctx.close()
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep)
+    rep = parity.check_batch(ora, kb, hb, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, _np(res[0]), _np(res[1]), _np(res[2]),
+                             dbg={n: _np(v) for n, v in res[3].items()})
+    assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5
+
+
 def test_expired_wait_is_reported_not_hung():
     """Bounded waits: with the pivots withheld (a flag that nothing sets) the fused kernel must give up within
     its time limit, say where, exit normally, and leave the context usable for the next call."""

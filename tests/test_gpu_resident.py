@@ -105,3 +105,29 @@ def test_resident_sweep_says_what_it_does_not_take(shape):
         ctx.reduce(h, k, vo, nv, P, Kp, opts=dart.dart_opts(path=dart.DART_PATH_RESIDENT))
     assert e.value.code == dart.DART_ERR_UNSUPPORTED
     ctx.close()
+
+
+@pytest.mark.parametrize("path,where,opts", [
+    (dart.DART_PATH_RESIDENT, 83, {}),                       # no CTA counts itself in: the exchange warps wait for the others
+    (dart.DART_PATH_TWO_PASS, 70, {}),                       # one-pass kernel: a norm warp never hands its norms to the epilogue
+], ids=["resident sweep", "one-pass kernel"])
+def test_expired_waits_of_the_other_kernels_are_reported_not_hung(path, where, opts):
+    """Bounded waits of the resident sweep (what AUTO runs for up to four samples) and of the one-pass kernel: with one
+    hand-over withheld - a counter that nothing advances, a barrier that one warp never arrives at - the kernel must
+    give up within its time limit, say where, free its tensor memory, exit normally and leave the context usable."""
+    w = W.LLAVA15_B64.with_(B=3)
+    k, h = W.make_batch(w, device="cuda")
+    ctx = dart.Dart(w.B, w.S, w.d, w.n_pivot, w.n_keep)
+    ctx.reduce(h, k, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep,
+               opts=dart.dart_opts(path=path, wait_limit=20000, test_withhold_pivots=1))      # 20 ms limit
+    torch.cuda.synchronize()
+    assert ctx.status() == dart.DART_ERR_TIMEOUT
+    rc, detail = dart.dart_status_detail(ctx.handle)
+    assert rc == dart.DART_OK and detail[0] == where, detail
+    assert ctx.status() == dart.DART_OK                                   # reading cleared it
+    good = ctx.reduce(h, k, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, opts=dart.dart_opts(path=path))   # same context
+    torch.cuda.synchronize()
+    assert ctx.status() == dart.DART_OK
+    ref = run_gpu(k, h, w.vis_offset, w.n_vis, w.n_pivot, w.n_keep, path=dart.DART_PATH_STAGED, debug=False)
+    assert np.array_equal(good[1].cpu().numpy(), ref[1]) and np.array_equal(W.bits(good[0]), ref[0])
+    ctx.close()
