@@ -294,8 +294,25 @@ static int retention_quotas(const double *dup, const int32_t *pivot_idx, int n_v
  *   gap    scalar  min over pivots of (best dup left behind by that pivot - eps_i), +inf if none
  *   n_kept         |R|
  */
+static int retention_union(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep, int text_pivots,
+                           uint8_t *keep, int32_t *owner, double *eps, double *gap_out, int32_t *n_kept);
+
 int dart_oracle_retention_union(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep,
                                 uint8_t *keep, int32_t *owner, double *eps, double *gap_out, int32_t *n_kept)
+{
+    return retention_union(dup, pivot_idx, n_vis, P, n_keep, 0, keep, owner, eps, gap_out, n_kept);
+}
+
+/* The same with pivots that may be text tokens (index outside [0, n_vis), see dart_oracle_retention_any): a text pivot
+ * takes its picks like any pivot but is no vision token, so the quotas split n_keep - Pv, Pv = the pivots inside the block. */
+int dart_oracle_retention_union_any(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep,
+                                    uint8_t *keep, int32_t *owner, double *eps, double *gap_out, int32_t *n_kept)
+{
+    return retention_union(dup, pivot_idx, n_vis, P, n_keep, 1, keep, owner, eps, gap_out, n_kept);
+}
+
+static int retention_union(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep, int text_pivots,
+                           uint8_t *keep, int32_t *owner, double *eps, double *gap_out, int32_t *n_kept)
 {
     if (P < 1 || P > n_keep || n_keep > n_vis) return ORACLE_ERR_SHAPE;
     keyed_t *cand = (keyed_t *)malloc((size_t)n_vis * sizeof *cand);
@@ -308,8 +325,18 @@ int dart_oracle_retention_union(const double *dup, const int32_t *pivot_idx, int
     memset(keep, 0, (size_t)n_vis);
     if (owner)
         for (int j = 0; j < n_vis; ++j) owner[j] = OWNER_DROPPED;
+    int Pv = 0;
     for (int i = 0; i < P; ++i) {
         const int p = pivot_idx[i];
+        if (text_pivots && (p < 0 || p >= n_vis)) { /* a text token: only distinctness is checked */
+            for (int k = 0; k < i; ++k)
+                if (pivot_idx[k] == p) {
+                    free(cand);
+                    free(is_pivot);
+                    return ORACLE_ERR_SHAPE;
+                }
+            continue;
+        }
         if (p < 0 || p >= n_vis || is_pivot[p]) {
             free(cand);
             free(is_pivot);
@@ -318,8 +345,9 @@ int dart_oracle_retention_union(const double *dup, const int32_t *pivot_idx, int
         is_pivot[p] = 1;
         keep[p] = 1;
         if (owner) owner[p] = P + i;
+        ++Pv;
     }
-    const int q = (n_keep - P) / P, r = (n_keep - P) % P;
+    const int q = (n_keep - Pv) / P, r = (n_keep - Pv) % P;
     double gap = INFINITY;
     for (int i = 0; i < P; ++i) {
         const int qi = q + (i < r ? 1 : 0);
@@ -332,7 +360,7 @@ int dart_oracle_retention_union(const double *dup, const int32_t *pivot_idx, int
                 cand[m].idx = j;
                 ++m;
             }
-        qsort(cand, (size_t)m, sizeof *cand, cmp_asc); /* m = n_vis - P >= n_keep - P >= qi */
+        qsort(cand, (size_t)m, sizeof *cand, cmp_asc); /* m = n_vis - Pv >= n_keep - Pv >= qi */
         for (int t = 0; t < qi; ++t) {
             const int j = cand[t].idx;
             if (owner && !keep[j]) owner[j] = i;
@@ -362,8 +390,25 @@ int dart_oracle_retention_union(const double *dup, const int32_t *pivot_idx, int
  *   eps    [P]     the one threshold, repeated; NaN when n_keep = P
  *   gap    scalar  (u of the best token NOT taken) - eps, +inf if none is left behind
  */
+static int retention_global(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep, int text_pivots,
+                            uint8_t *keep, int32_t *owner, double *eps, double *gap_out);
+
 int dart_oracle_retention_global(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep,
                                  uint8_t *keep, int32_t *owner, double *eps, double *gap_out)
+{
+    return retention_global(dup, pivot_idx, n_vis, P, n_keep, 0, keep, owner, eps, gap_out);
+}
+
+/* The same with pivots that may be text tokens (index outside [0, n_vis)): they count among the pivots a token is compared
+ * with, but not among the vision tokens kept, so n_keep - Pv non-pivot tokens are retained, Pv = the pivots inside the block. */
+int dart_oracle_retention_global_any(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep,
+                                     uint8_t *keep, int32_t *owner, double *eps, double *gap_out)
+{
+    return retention_global(dup, pivot_idx, n_vis, P, n_keep, 1, keep, owner, eps, gap_out);
+}
+
+static int retention_global(const double *dup, const int32_t *pivot_idx, int n_vis, int P, int n_keep, int text_pivots,
+                            uint8_t *keep, int32_t *owner, double *eps, double *gap_out)
 {
     if (P < 1 || P > n_keep || n_keep > n_vis) return ORACLE_ERR_SHAPE;
     keyed_t *cand = (keyed_t *)malloc((size_t)n_vis * sizeof *cand);
@@ -376,8 +421,18 @@ int dart_oracle_retention_global(const double *dup, const int32_t *pivot_idx, in
     memset(keep, 0, (size_t)n_vis);
     if (owner)
         for (int j = 0; j < n_vis; ++j) owner[j] = OWNER_DROPPED;
+    int Pv = 0;
     for (int i = 0; i < P; ++i) {
         int p = pivot_idx[i];
+        if (text_pivots && (p < 0 || p >= n_vis)) { /* a text token: only distinctness is checked */
+            for (int k = 0; k < i; ++k)
+                if (pivot_idx[k] == p) {
+                    free(cand);
+                    free(nearest);
+                    return ORACLE_ERR_SHAPE;
+                }
+            continue;
+        }
         if (p < 0 || p >= n_vis || keep[p]) {
             free(cand);
             free(nearest);
@@ -385,6 +440,7 @@ int dart_oracle_retention_global(const double *dup, const int32_t *pivot_idx, in
         }
         keep[p] = 1;
         if (owner) owner[p] = P + i;
+        ++Pv;
     }
     int m = 0;
     for (int j = 0; j < n_vis; ++j) {
@@ -401,7 +457,7 @@ int dart_oracle_retention_global(const double *dup, const int32_t *pivot_idx, in
         nearest[j] = arg;
         ++m;
     }
-    const int take = n_keep - P;
+    const int take = n_keep - Pv;
     qsort(cand, (size_t)m, sizeof *cand, cmp_asc);
     for (int t = 0; t < take; ++t) {
         keep[cand[t].idx] = 1;
@@ -412,6 +468,79 @@ int dart_oracle_retention_global(const double *dup, const int32_t *pivot_idx, in
     if (gap_out) *gap_out = (take > 0 && m > take) ? cand[take].v - cand[take - 1].v : INFINITY;
     free(cand);
     free(nearest);
+    return ORACLE_OK;
+}
+
+/*
+ * Pivots from both modalities (Sec. 5.4 finds that pivots from either modality alone do worse; the pivot-selection
+ * table's caption uses "4 visual and 4 text tokens"): the Pv vision tokens and the Pt text tokens of largest (or
+ * smallest) score, each group ranked like dart_oracle_pivots (equal scores: lower sequence position first).
+ *   score_all [S] the score of EVERY token of the sample (K-norm of its key row)
+ *   pivot_idx [Pv + Pt] relative to the vision block (a text token before it is negative, one after it >= n_vis):
+ *             the vision pivots in rank order, then the text pivots in rank order (reading: the paper does not say in
+ *             which order pivots of different modality take their turns)
+ * Needs Pv <= n_vis and Pt <= S - n_vis.
+ */
+int dart_oracle_pivots_mixed(const double *score_all, int S, int vis_offset, int n_vis, int Pv, int Pt, int largest,
+                             int32_t *pivot_idx)
+{
+    if (S < 1 || vis_offset < 0 || n_vis < 0 || vis_offset + n_vis > S || Pv < 0 || Pt < 0 || Pv > n_vis || Pt > S - n_vis)
+        return ORACLE_ERR_SHAPE;
+    keyed_t *t = (keyed_t *)malloc((size_t)S * sizeof *t);
+    if (!t) return ORACLE_ERR_NOMEM;
+    int m = 0;
+    for (int j = 0; j < n_vis; ++j) {
+        t[m].v = score_all[vis_offset + j];
+        t[m].idx = j;
+        ++m;
+    }
+    qsort(t, (size_t)m, sizeof *t, largest ? cmp_desc : cmp_asc);
+    for (int i = 0; i < Pv; ++i) pivot_idx[i] = t[i].idx;
+    m = 0;
+    for (int s = 0; s < S; ++s) {
+        if (s >= vis_offset && s < vis_offset + n_vis) continue;
+        t[m].v = score_all[s];
+        t[m].idx = s - vis_offset; /* ascending with the sequence position, so ties go to the earlier token */
+        ++m;
+    }
+    qsort(t, (size_t)m, sizeof *t, largest ? cmp_desc : cmp_asc);
+    for (int i = 0; i < Pt; ++i) pivot_idx[Pv + i] = t[i].idx;
+    free(t);
+    return ORACLE_OK;
+}
+
+/*
+ * The output of SplitMix64 (Steele, Lea, Flood: "Fast splittable pseudorandom number generators", OOPSLA 2014) for the
+ * state `state` AFTER its increment by the golden gamma: the generator's next() is mix(state += gamma).
+ */
+static uint64_t splitmix64_mix(uint64_t z)
+{
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+/* The k-th output (k = 0, 1, ...) of a SplitMix64 generator seeded with `seed`: a counter-based form of the same sequence. */
+uint64_t dart_oracle_splitmix64(uint64_t seed, uint64_t k) { return splitmix64_mix(seed + (k + 1) * 0x9E3779B97F4A7C15ull); }
+
+/*
+ * Random pivots (Sec. 5.2 also draws the pivots at random, five seeds): P distinct vision tokens of sample b, uniformly at
+ * random without replacement.  Every token gets a 32-bit ticket, the upper half of output number (b * 2^32 + j) of a
+ * SplitMix64 generator seeded with `seed`; the P tokens with the smallest tickets are the pivots, smallest first, equal
+ * tickets to the lower index.  (Any P-subset is equally likely because the tickets are exchangeable.)
+ */
+int dart_oracle_pivots_random(uint64_t seed, int b, int n_vis, int P, int32_t *pivot_idx)
+{
+    if (n_vis < 1 || P < 1 || P > n_vis || b < 0) return ORACLE_ERR_SHAPE;
+    keyed_t *t = (keyed_t *)malloc((size_t)n_vis * sizeof *t);
+    if (!t) return ORACLE_ERR_NOMEM;
+    for (int j = 0; j < n_vis; ++j) {
+        t[j].v = (double)(uint32_t)(dart_oracle_splitmix64(seed, ((uint64_t)b << 32) | (uint32_t)j) >> 32);
+        t[j].idx = j;
+    }
+    qsort(t, (size_t)n_vis, sizeof *t, cmp_asc);
+    for (int i = 0; i < P; ++i) pivot_idx[i] = t[i].idx;
+    free(t);
     return ORACLE_OK;
 }
 
@@ -483,12 +612,16 @@ int dart_oracle_compact(const uint8_t *keep, const uint16_t *hidden, const int64
  * key rows' scores, Eq. 7 is evaluated on the hidden rows.  Then l1_out holds the key rows' L1 scores and
  * l2_out the HIDDEN rows' Euclidean norms (Eq. 7's denominators).  Ignored when keys is NULL.
  * text_pivots: entries of pivots_in outside [0, n_vis) name text tokens (index relative to the vision block);
- * see dart_oracle_similarity_any and dart_oracle_retention_any.  Needs pivots_in and rule 0.
+ * see dart_oracle_similarity_any and the dart_oracle_retention*_any functions.  Needs pivots_in or pivot_source 1.
+ * pivot_source (without pivots_in): 0 = the n_pivot vision tokens of best score; 1 = n_pivot - n_text_pivots vision
+ * tokens and n_text_pivots text tokens of best score (dart_oracle_pivots_mixed; implies text_pivots); 2 = random
+ * vision tokens (dart_oracle_pivots_random with `seed` and the sample's number b).
  */
 int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const int64_t *pos_in,
                           const int32_t *pivots_in,
                           int B, int S, int d, int vis_offset, int n_vis, int n_pivot, int n_keep,
                           int norm_kind, int largest, int rule, int cosine_on_hidden, int text_pivots,
+                          int pivot_source, int n_text_pivots, uint64_t seed,
                           uint16_t *out_hidden, int32_t *out_idx, int64_t *out_pos,
                           double *l1_out, double *l2_out, int32_t *pivot_out, double *dup_out,
                           uint8_t *keep_out, int32_t *owner_out, double *eps_out,
@@ -499,8 +632,15 @@ int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const in
     if (norm_kind != 1 && norm_kind != 2) return ORACLE_ERR_SHAPE;
     if (rule != 0 && rule != 1 && rule != 2) return ORACLE_ERR_SHAPE;
     if (rule == 2 && !cu_seqlens_out) return ORACLE_ERR_SHAPE;
-    if (text_pivots && (!pivots_in || rule != 0)) return ORACLE_ERR_SHAPE; /* text pivots are the caller's, quota rule only */
+    if (pivot_source < 0 || pivot_source > 2 || (pivot_source && pivots_in)) return ORACLE_ERR_SHAPE;
+    if (pivot_source == 1) {
+        if (n_text_pivots < 0 || n_text_pivots > n_pivot || n_text_pivots > S - n_vis || n_pivot - n_text_pivots > n_vis) return ORACLE_ERR_SHAPE;
+        text_pivots = 1;
+    }
+    if (text_pivots && !pivots_in && pivot_source != 1) return ORACLE_ERR_SHAPE; /* text pivots come from the caller or from source 1 */
     const int P = n_pivot, S_out = S - n_vis + n_keep;
+    double *all1 = (double *)malloc((size_t)S * sizeof(double));
+    double *all2 = (double *)malloc((size_t)S * sizeof(double));
     double *l1 = (double *)malloc((size_t)n_vis * sizeof(double));
     double *l2 = (double *)malloc((size_t)n_vis * sizeof(double));
     double *hl1 = (double *)malloc((size_t)n_vis * sizeof(double));
@@ -508,7 +648,7 @@ int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const in
     int32_t *piv = (int32_t *)malloc((size_t)P * sizeof(int32_t));
     uint8_t *keep = (uint8_t *)malloc((size_t)n_vis);
     int rc = ORACLE_OK;
-    if (!l1 || !l2 || !hl1 || !dup || !piv || !keep) rc = ORACLE_ERR_NOMEM;
+    if (!l1 || !l2 || !hl1 || !dup || !piv || !keep || !all1 || !all2) rc = ORACLE_ERR_NOMEM;
     size_t cu = 0; /* rows packed so far (rule 2) */
     if (cu_seqlens_out) cu_seqlens_out[0] = 0;
     for (int b = 0; b < B && rc == ORACLE_OK; ++b) {
@@ -522,6 +662,16 @@ int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const in
         if (pivots_in) { /* the caller names the pivots and their order (Sec. 5.2 compares several ways to choose them) */
             memcpy(piv, pivots_in + (size_t)b * P, (size_t)P * sizeof(int32_t));
             pgap = INFINITY; /* nothing is ranked, so no ranking can be close */
+        } else if (pivot_source == 1) { /* both modalities: the scores of all S tokens */
+            rc = dart_oracle_scores(k, S, d, 0, S, all1, all2);
+            if (rc) break;
+            rc = dart_oracle_pivots_mixed(norm_kind == 1 ? all1 : all2, S, vis_offset, n_vis, P - n_text_pivots, n_text_pivots, largest, piv);
+            if (rc) break;
+            pgap = 0.0; /* the gaps of the two rankings are not tracked: compare under tolerance */
+        } else if (pivot_source == 2) {
+            rc = dart_oracle_pivots_random(seed, b, n_vis, P, piv);
+            if (rc) break;
+            pgap = INFINITY; /* integer tickets: nothing can be close */
         } else {
             rc = dart_oracle_pivots(norm_kind == 1 ? l1 : l2, n_vis, P, largest, piv, &pgap);
             if (rc) break;
@@ -537,10 +687,15 @@ int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const in
             rc = dart_oracle_similarity((cosine_on_hidden && keys) ? h : k, S, d, vis_offset, n_vis, piv, P, l2, dup);
         if (rc) break;
         if (rule == 2)
-            rc = dart_oracle_retention_union(dup, piv, n_vis, P, n_keep, keep, owner_out ? owner_out + (size_t)b * n_vis : NULL,
-                                             eps_out ? eps_out + (size_t)b * P : NULL, &rgap, NULL);
+            rc = (text_pivots ? dart_oracle_retention_union_any : dart_oracle_retention_union)(
+                dup, piv, n_vis, P, n_keep, keep, owner_out ? owner_out + (size_t)b * n_vis : NULL,
+                eps_out ? eps_out + (size_t)b * P : NULL, &rgap, NULL);
+        else if (rule == 1)
+            rc = (text_pivots ? dart_oracle_retention_global_any : dart_oracle_retention_global)(
+                dup, piv, n_vis, P, n_keep, keep, owner_out ? owner_out + (size_t)b * n_vis : NULL,
+                eps_out ? eps_out + (size_t)b * P : NULL, &rgap);
         else
-            rc = (text_pivots ? dart_oracle_retention_any : rule == 1 ? dart_oracle_retention_global : dart_oracle_retention)(
+            rc = (text_pivots ? dart_oracle_retention_any : dart_oracle_retention)(
                 dup, piv, n_vis, P, n_keep, keep, owner_out ? owner_out + (size_t)b * n_vis : NULL,
                 eps_out ? eps_out + (size_t)b * P : NULL, &rgap);
         if (rc) break;
@@ -568,6 +723,8 @@ int dart_oracle_reduce_ex(const uint16_t *hidden, const uint16_t *keys, const in
     free(dup);
     free(piv);
     free(keep);
+    free(all1);
+    free(all2);
     return rc;
 }
 
@@ -581,6 +738,6 @@ int dart_oracle_reduce(const uint16_t *hidden, const uint16_t *keys, const int64
                        double *pivot_gap_out, double *retain_gap_out)
 {
     return dart_oracle_reduce_ex(hidden, keys, pos_in, NULL, B, S, d, vis_offset, n_vis, n_pivot, n_keep, norm_kind,
-                                 largest, 0, 0, 0, out_hidden, out_idx, out_pos, l1_out, l2_out, pivot_out, dup_out, keep_out,
+                                 largest, 0, 0, 0, 0, 0, 0, out_hidden, out_idx, out_pos, l1_out, l2_out, pivot_out, dup_out, keep_out,
                                  owner_out, eps_out, pivot_gap_out, retain_gap_out, NULL);
 }

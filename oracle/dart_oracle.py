@@ -41,8 +41,11 @@ def _load():
         for name in ("dart_oracle_scores", "dart_oracle_pivots", "dart_oracle_similarity",
                      "dart_oracle_retention", "dart_oracle_retention_global", "dart_oracle_retention_any",
                      "dart_oracle_retention_union", "dart_oracle_similarity_any", "dart_oracle_compact",
-                     "dart_oracle_gather_rows", "dart_oracle_reduce", "dart_oracle_reduce_ex"):
+                     "dart_oracle_gather_rows", "dart_oracle_reduce", "dart_oracle_reduce_ex", "dart_oracle_retention_union_any",
+                     "dart_oracle_retention_global_any", "dart_oracle_pivots_mixed", "dart_oracle_pivots_random"):
             getattr(_lib, name).restype = ctypes.c_int
+        _lib.dart_oracle_splitmix64.restype = ctypes.c_uint64
+        _lib.dart_oracle_splitmix64.argtypes = [ctypes.c_uint64, ctypes.c_uint64]
     return _lib
 
 
@@ -149,7 +152,28 @@ def retention_any(dup, pivot_idx, n_keep: int):
     return keep, owner, eps, gap.value
 
 
-def retention_union(dup, pivot_idx, n_keep: int):
+def splitmix64(seed: int, k: int) -> int:
+    """Output number k (0-based) of a SplitMix64 generator seeded with ``seed``."""
+    return int(_load().dart_oracle_splitmix64(ctypes.c_uint64(seed & (2**64 - 1)), ctypes.c_uint64(k & (2**64 - 1))))
+
+
+def pivots_mixed(score_all, vis_offset: int, n_vis: int, Pv: int, Pt: int, largest: bool = True):
+    """score_all [S] -> [Pv + Pt] pivots relative to the vision block: Pv vision tokens, then Pt text tokens, each by rank."""
+    s = np.ascontiguousarray(score_all, np.float64)
+    piv = np.empty(Pv + Pt, np.int32)
+    _check(_load().dart_oracle_pivots_mixed(_p(s, ctypes.c_double), s.shape[0], vis_offset, n_vis, Pv, Pt, int(bool(largest)),
+                                            _p(piv, ctypes.c_int32)), "pivots_mixed")
+    return piv
+
+
+def pivots_random(seed: int, b: int, n_vis: int, P: int):
+    """P distinct random vision tokens of sample b: the smallest 32-bit SplitMix64 tickets, smallest first."""
+    piv = np.empty(P, np.int32)
+    _check(_load().dart_oracle_pivots_random(ctypes.c_uint64(seed & (2**64 - 1)), b, n_vis, P, _p(piv, ctypes.c_int32)), "pivots_random")
+    return piv
+
+
+def retention_union(dup, pivot_idx, n_keep: int, text_pivots: bool = False):
     """Independent pivots: (keep, owner, eps [P], gap, n_kept); a token two pivots take counts once."""
     dd = np.ascontiguousarray(dup, np.float64)
     P, n_vis = dd.shape
@@ -159,13 +183,14 @@ def retention_union(dup, pivot_idx, n_keep: int):
     eps = np.empty(P, np.float64)
     gap = ctypes.c_double(0.0)
     cnt = ctypes.c_int32(0)
-    _check(_load().dart_oracle_retention_union(_p(dd, ctypes.c_double), _p(piv, ctypes.c_int32), n_vis, P, n_keep,
+    fn = _load().dart_oracle_retention_union_any if text_pivots else _load().dart_oracle_retention_union
+    _check(fn(_p(dd, ctypes.c_double), _p(piv, ctypes.c_int32), n_vis, P, n_keep,
                                                _p(keep, ctypes.c_uint8), _p(owner, ctypes.c_int32),
                                                _p(eps, ctypes.c_double), ctypes.byref(gap), ctypes.byref(cnt)), "retention_union")
     return keep, owner, eps, gap.value, cnt.value
 
 
-def retention_global(dup, pivot_idx, n_keep: int):
+def retention_global(dup, pivot_idx, n_keep: int, text_pivots: bool = False):
     """dup [P, n_vis] -> (keep, owner, eps [P], gap) with one threshold on max_i dup for all pivots."""
     dd = np.ascontiguousarray(dup, np.float64)
     P, n_vis = dd.shape
@@ -174,7 +199,8 @@ def retention_global(dup, pivot_idx, n_keep: int):
     owner = np.empty(n_vis, np.int32)
     eps = np.empty(P, np.float64)
     gap = ctypes.c_double(0.0)
-    _check(_load().dart_oracle_retention_global(_p(dd, ctypes.c_double), _p(piv, ctypes.c_int32), n_vis, P, n_keep,
+    fn = _load().dart_oracle_retention_global_any if text_pivots else _load().dart_oracle_retention_global
+    _check(fn(_p(dd, ctypes.c_double), _p(piv, ctypes.c_int32), n_vis, P, n_keep,
                                                 _p(keep, ctypes.c_uint8), _p(owner, ctypes.c_int32),
                                                 _p(eps, ctypes.c_double), ctypes.byref(gap)), "retention_global")
     return keep, owner, eps, gap.value
@@ -235,13 +261,15 @@ class OracleResult:
 def reduce(hidden, keys, vis_offset: int, n_vis: int, n_pivot: int, n_keep: int,
            pos_in=None, norm_kind: int = 1, largest: bool = True, want_dup: bool = True,
            want_hidden: bool = True, pivots_in=None, rule: int = 0, cosine_on_hidden: bool = False,
-           text_pivots: bool = False) -> OracleResult:
+           text_pivots: bool = False, pivot_source: int = 0, n_text_pivots: int = 0, seed: int = 0) -> OracleResult:
     """The whole step over a batch.  hidden/keys: [B, S, d] bf16 bits (keys None -> hidden is scored).
     pivots_in: None, or [B, n_pivot] distinct vision-relative indices that replace the pivot step.
     rule: 0 quotas with masking, 1 one threshold for all pivots, 2 independent pivots (flat outputs + .cu_seqlens).
     rule: 0 = per-pivot thresholds from equal quotas, 1 = one threshold for all pivots.
     cosine_on_hidden: pivots by the key rows' scores, Eq. 7 on the hidden rows (then .l2 holds the hidden rows' norms).
-    text_pivots: entries of pivots_in outside [0, n_vis) name text tokens (indices relative to the vision block)."""
+    text_pivots: entries of pivots_in outside [0, n_vis) name text tokens (indices relative to the vision block).
+    pivot_source (without pivots_in): 0 = vision tokens by score, 1 = n_pivot - n_text_pivots vision and n_text_pivots text
+    tokens by score, 2 = random vision tokens from ``seed``."""
     h = _u16(hidden)
     B, S, d = h.shape
     k = None if keys is None else _u16(keys)
@@ -274,6 +302,7 @@ def reduce(hidden, keys, vis_offset: int, n_vis: int, n_pivot: int, n_keep: int,
     _check(_load().dart_oracle_reduce_ex(
         _p(h, ctypes.c_uint16), _p(k, ctypes.c_uint16), _p(pos, ctypes.c_int64), _p(piv_in, ctypes.c_int32),
         B, S, d, vis_offset, n_vis, n_pivot, n_keep, norm_kind, int(bool(largest)), int(rule), int(bool(cosine_on_hidden)), int(bool(text_pivots)),
+        int(pivot_source), int(n_text_pivots), ctypes.c_uint64(seed & (2**64 - 1)),
         _p(oh, ctypes.c_uint16), _p(oi, ctypes.c_int32), _p(op, ctypes.c_int64),
         _p(l1, ctypes.c_double), _p(l2, ctypes.c_double), _p(piv, ctypes.c_int32), _p(dup, ctypes.c_double),
         _p(keep, ctypes.c_uint8), _p(owner, ctypes.c_int32), _p(eps, ctypes.c_double),

@@ -306,3 +306,128 @@ def test_union_through_the_whole_step_is_packed_without_padding(oracle):
         assert np.array_equal(r.out_idx[cu[b]:cu[b + 1]], oi) and np.array_equal(r.out_hidden[cu[b]:cu[b + 1]], oh)
         assert np.array_equal(r.out_pos[cu[b]:cu[b + 1]], op) and np.array_equal(r.keep[b], keep)
     assert (r.out_idx[cu[B]:] == -1).all()
+
+
+# ----------------------------------------------------------------------------- text pivots under the other two retention rules
+
+def test_text_pivots_under_one_threshold_and_independent_pivots(oracle):
+    """Text pivots count among the pivots a token is compared with but not among the vision tokens kept: replayed by
+    brute force with hand-written budgets; with vision pivots only the functions coincide with the plain ones."""
+    rng = np.random.default_rng(41)
+    nv, P = 40, 5
+    dup = rng.uniform(-1, 1, (P, nv))
+    piv = np.array([7, -3, 22, nv + 4, -1], np.int32)            # two vision pivots, three text pivots
+    n_keep = 16                                                  # 2 vision pivots + 14 more vision tokens
+    # one threshold: the 14 non-pivot tokens of lowest max_i dup
+    keep, owner, eps, gap = oracle.retention_global(dup, piv, n_keep, text_pivots=True)
+    u = dup.max(axis=0)
+    cands = [j for j in range(nv) if j not in (7, 22)]
+    best = sorted(cands, key=lambda j: (u[j], j))[:14]
+    assert int(keep.sum()) == n_keep and keep[7] == 1 and keep[22] == 1
+    assert sorted(best) == sorted(j for j in cands if keep[j])
+    assert np.all(eps == max(u[j] for j in best)) and owner[7] == P + 0 and owner[22] == P + 2
+    assert all(owner[j] == int(np.argmax(dup[:, j])) for j in best)
+    rest = sorted(cands, key=lambda j: (u[j], j))[14:]
+    assert math.isclose(gap, u[rest[0]] - max(u[j] for j in best))
+    # independent pivots: 14 over 5 pivots: quotas 3, 3, 3, 3, 2, every pivot from all non-pivot tokens
+    keep, owner, eps, gap, cnt = oracle.retention_union(dup, piv, n_keep, text_pivots=True)
+    kept = {7, 22}
+    for i, qi in enumerate([3, 3, 3, 3, 2]):
+        mine = sorted(cands, key=lambda j: (dup[i, j], j))[:qi]
+        assert eps[i] == max(dup[i, j] for j in mine)
+        for j in mine:
+            if j not in kept:
+                assert owner[j] == i                               # the first pivot in rank order that took it
+            kept.add(j)
+    assert set(np.nonzero(keep)[0].tolist()) == kept and cnt == len(kept) and 2 + 3 <= cnt <= n_keep
+    # vision pivots only: the plain functions
+    vis = np.array([7, 22, 30], np.int32)
+    d3 = dup[:3]
+    for a, b in [(oracle.retention_global(d3, vis, 12, text_pivots=True), oracle.retention_global(d3, vis, 12)),
+                 (oracle.retention_union(d3, vis, 12, text_pivots=True), oracle.retention_union(d3, vis, 12))]:
+        assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1]) and np.array_equal(a[2], b[2], equal_nan=True)
+    with pytest.raises(RuntimeError):
+        oracle.retention_global(dup, piv, n_keep)                # text pivots must be asked for
+    with pytest.raises(RuntimeError):
+        oracle.retention_union(dup, np.array([7, -3, 22, -3, -1], np.int32), n_keep, text_pivots=True)   # repeated
+
+
+# ----------------------------------------------------------------------------- pivots from both modalities, random pivots
+
+def test_pivots_from_both_modalities_against_numpy(oracle):
+    """Pv vision and Pt text tokens of best score, each group in rank order: numpy's stable argsort on the same
+    scores is the independent routine; planted equal scores go to the earlier token."""
+    rng = np.random.default_rng(42)
+    S, vo, nv = 60, 9, 40
+    s = rng.uniform(1, 2, S)
+    s[vo + 5] = s[vo + 31] = 3.0            # a tie among the vision tokens
+    s[2] = s[S - 1] = 2.5                   # a tie among the text tokens (before and after the block)
+    for largest in (True, False):
+        key = -s if largest else s
+        vis = np.argsort(key[vo:vo + nv], kind="stable")
+        text_pos = np.array([t for t in range(S) if not vo <= t < vo + nv])
+        txt = text_pos[np.argsort(key[text_pos], kind="stable")] - vo
+        for Pv, Pt in [(4, 4), (0, 3), (5, 0), (nv, S - nv)]:
+            got = oracle.pivots_mixed(s, vo, nv, Pv, Pt, largest)
+            assert got[:Pv].tolist() == vis[:Pv].tolist() and got[Pv:].tolist() == txt[:Pt].tolist()
+    got = oracle.pivots_mixed(s, vo, nv, 2, 2, True)
+    assert got.tolist() == [5, 31, 2 - vo, S - 1 - vo]           # the ties, lower position first; text tokens outside [0, nv)
+    with pytest.raises(RuntimeError):
+        oracle.pivots_mixed(s, vo, nv, 2, S - nv + 1)            # more text pivots than text tokens
+
+
+def test_splitmix64_reference_outputs(oracle):
+    """The generator behind the random pivots against the outputs that the reference implementation of SplitMix64
+    (Steele, Lea and Flood, OOPSLA 2014) is commonly tabulated with for the seed 1234567."""
+    expect = [6457827717110365317, 3203168211198807973, 9817491932198370423, 4593380528125082431, 16408922859458223821]
+    assert [oracle.splitmix64(1234567, k) for k in range(5)] == expect
+    assert oracle.splitmix64(0, 0) == 0xE220A8397B1DCDAF         # the first output for seed 0 (the xoshiro seeding example)
+
+
+def test_random_pivots_are_a_uniform_draw_without_replacement(oracle):
+    nv, P = 50, 6
+    a = oracle.pivots_random(99, 3, nv, P)
+    assert len(set(a.tolist())) == P and a.min() >= 0 and a.max() < nv
+    assert np.array_equal(a, oracle.pivots_random(99, 3, nv, P))                     # a function of (seed, sample) only
+    assert not np.array_equal(a, oracle.pivots_random(99, 4, nv, P)) and not np.array_equal(a, oracle.pivots_random(100, 3, nv, P))
+    # re-derived from the pinned generator: tickets = upper halves of outputs b * 2^32 + j, smallest first, ties by index
+    tickets = np.array([oracle.splitmix64(99, (3 << 32) | j) >> 32 for j in range(nv)], np.uint64)
+    assert a.tolist() == np.argsort(tickets, kind="stable")[:P].tolist()
+    assert sorted(oracle.pivots_random(5, 0, nv, nv).tolist()) == list(range(nv))     # P = n_vis: a permutation
+    # every token is drawn about equally often: 4000 draws of 6 of 50 -> 480 expected per token, sigma ~ 21
+    hits = np.zeros(nv, np.int64)
+    for seed in range(4000):
+        hits[oracle.pivots_random(seed, 0, nv, P)] += 1
+    assert hits.sum() == 4000 * P and abs(hits - 480).max() < 6 * 21
+
+
+def test_pivot_sources_through_the_whole_step(oracle):
+    """The batch entry point with pivots from both modalities / random pivots = the step functions composed by hand."""
+    rng = np.random.default_rng(43)
+    B, S, d, vo, nv, P, Kp = 3, 70, 32, 8, 50, 6, 18
+    hb, _ = rand_tokens(rng, B * S, d)
+    kb, _ = rand_tokens(rng, B * S, d)
+    hb, kb = hb.reshape(B, S, d), kb.reshape(B, S, d)
+    for rule in (0, 1, 2):
+        r = oracle.reduce(hb, kb, vo, nv, P, Kp, pivot_source=1, n_text_pivots=2, rule=rule)
+        cu = r.cu_seqlens
+        for b in range(B):
+            l1_all, _ = oracle.scores(kb[b], 0, S)
+            piv = oracle.pivots_mixed(l1_all, vo, nv, P - 2, 2)
+            assert np.array_equal(r.pivot_idx[b], piv) and (piv[:4] >= 0).all() and ((piv[4:] < 0) | (piv[4:] >= nv)).all()
+            dup = oracle.similarity_any(kb[b], vo, nv, piv)
+            keep = (oracle.retention_any(dup, piv, Kp) if rule == 0 else oracle.retention_global(dup, piv, Kp, True) if rule == 1
+                    else oracle.retention_union(dup, piv, Kp, True))[0]
+            assert np.array_equal(r.keep[b], keep)
+            oh, oi, op = oracle.compact(keep, hb[b], vo, nv)
+            got = r.out_idx[b] if rule != 2 else r.out_idx[cu[b]:cu[b + 1]]
+            assert np.array_equal(got, oi)
+    r = oracle.reduce(hb, kb, vo, nv, P, Kp, pivot_source=2, seed=2024)
+    for b in range(B):
+        piv = oracle.pivots_random(2024, b, nv, P)
+        assert np.array_equal(r.pivot_idx[b], piv)
+        _, l2 = oracle.scores(kb[b], vo, nv)
+        keep = oracle.retention(oracle.similarity(kb[b], vo, nv, piv, l2), piv, Kp)[0]
+        assert np.array_equal(r.keep[b], keep)
+    with pytest.raises(RuntimeError):
+        oracle.reduce(hb, kb, vo, nv, P, Kp, pivot_source=1, n_text_pivots=S - nv + 1)
