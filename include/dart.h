@@ -75,6 +75,19 @@ enum {
                               lists into the sample's pivots), so that the second read comes from the L2.  Needs
                               n_pivot <= 16, d % 64 == 0, pivots chosen by score, else UNSUPPORTED. */
 
+/* dart_opts.pivot_source: where step 2 takes the pivots from when the caller does not name them (pivots_in == NULL) */
+#define DART_PIVOTS_BY_SCORE 0 /* the n_pivot vision tokens of best score (dart_reduce) */
+#define DART_PIVOTS_MIXED 1    /* both modalities (Sec. 5.4; the pivot-selection table uses 4 visual and 4 text tokens):
+                                  the n_pivot - n_text_pivots vision tokens and the n_text_pivots text tokens of best score
+                                  (same score and direction as BY_SCORE, equal scores to the earlier token); the vision
+                                  pivots take their turns first, in rank order, then the text pivots in rank order.  Text
+                                  pivots behave as described at text_pivots.  Needs n_text_pivots <= the text tokens of a
+                                  sample and n_pivot - n_text_pivots <= n_vis, else BAD_SHAPE. */
+#define DART_PIVOTS_RANDOM 2   /* n_pivot distinct vision tokens drawn uniformly at random (Sec. 5.2): token j of sample b
+                                  gets the upper 32 bits of output number (sample_base + b) * 2^32 + j of a SplitMix64
+                                  generator seeded with `seed`; the smallest n_pivot tickets win, smallest first, equal
+                                  tickets to the lower index.  The same seed gives the same pivots on every run. */
+
 /* dart_opts.retention */
 #define DART_RETAIN_AUTO 0   /* two phases when the batch alone cannot fill the GPU, else one kernel */
 #define DART_RETAIN_SERIAL 1 /* one kernel, one CTA per sample: the pivots' selections one after the other */
@@ -135,9 +148,9 @@ typedef struct {
                               before it has a negative index and one after it an index >= n_vis; the range is
                               [-vis_offset, S - vis_offset), entries distinct.  A text pivot takes its turn in step 4 like
                               any other but is no vision token: with Pv the pivots inside the vision block, step 4 uses
-                              q = (n_keep - Pv) / P and r = (n_keep - Pv) % P, and n_keep vision tokens are kept as
-                              always.  dbg->owner marks only the vision pivots.  Needs pivots_in, DART_RULE_QUOTAS and a
-                              shape the FUSED path takes (else UNSUPPORTED). */
+                              q = (n_keep - Pv) / P and r = (n_keep - Pv) % P (DART_RULE_GLOBAL: n_keep - Pv tokens beside
+                              the pivots), and n_keep vision tokens are kept as always (DART_RULE_UNION: at most).
+                              dbg->owner marks only the vision pivots.  Needs pivots_in (else UNSUPPORTED). */
     const int32_t *pivots_in; /* NULL: pivots by score (steps 1-2).  Else [B, n_pivot] int32, device: the caller's pivots
                               as vision-relative indices, distinct and in [0, n_vis); their order is the order of the
                               pivots' turns in step 4.  This covers the paper's other ways to choose pivots (Sec. 5.2:
@@ -147,6 +160,12 @@ typedef struct {
                               cu_seqlens[b + 1] = cu_seqlens[b] + packed length of sample b. */
     int32_t resident_split; /* DART_PATH_SPLIT: 0 = default (every second tile stays on the chip); k >= 2: the tiles with
                               index % k == 0 stay (a share of 1/k); -k: all other tiles stay (a share of 1 - 1/k) */
+    int32_t pivot_source;  /* DART_PIVOTS_*: BY_SCORE (0) unless pivots_in is NULL and another source is wanted.  The other
+                              sources run on the paths that take the caller's pivots (AUTO, STAGED, FUSED, TWO_PASS). */
+    int32_t n_text_pivots; /* DART_PIVOTS_MIXED: how many of the n_pivot pivots are text tokens */
+    uint64_t seed;         /* DART_PIVOTS_RANDOM */
+    int32_t sample_base;   /* DART_PIVOTS_RANDOM: number of the call's first sample in the ticket stream (>= 0), so that a batch
+                              split over several calls or GPUs draws what the whole batch would */
     int32_t tune;          /* 0 = defaults.  DART_PATH_PAIRED: 256 * n1 + 16 * n2 + n3 = depths of the three shared-memory rings.
                               DART_PATH_FUSED: >= 2 cuts the second pass of a row tile into eight column chunks (one task each)
                               and keeps the first pass within `tune` steps of the second (both tuning options) */

@@ -103,9 +103,12 @@ def check_valid_under_tolerance(keys_bits, vis_offset, n_vis, n_keep, pivot_idx,
     pivots_given the caller chose the pivots and nothing about their ranking is checked; rule 1 is the
     variant with one threshold for all pivots; text_pivots (with pivots_given, rule 0): pivots outside [0, n_vis) are
     text tokens."""
-    if text_pivots:
-        assert pivots_given and rule == 0
+    if text_pivots and rule == 0:
+        assert pivots_given
         return _replay_text_pivots(keys_bits, vis_offset, n_vis, n_keep, pivot_idx, owner, tol)
+    if text_pivots:
+        assert pivots_given and rule == 1
+        return _replay_text_pivots_one_threshold(keys_bits, vis_offset, n_vis, n_keep, pivot_idx, owner, tol)
     P = len(pivot_idx)
     assert len(set(pivot_idx.tolist())) == P, "pivots must be distinct"
     s = ora_score
@@ -152,6 +155,32 @@ def check_valid_under_tolerance(keys_bits, vis_offset, n_vis, n_keep, pivot_idx,
         kept[mine] = True
     assert int(kept.sum()) == n_keep
     assert np.array_equal(np.nonzero(owner >= 0)[0], np.nonzero(kept)[0]), "owner and kept set disagree"
+    return kept
+
+
+def _replay_text_pivots_one_threshold(keys_bits, vis_offset, n_vis, n_keep, pivot_idx, owner, tol):
+    """One threshold for all pivots, some of which are text tokens: n_keep - Pv tokens beside the vision pivots."""
+    P = len(pivot_idx)
+    assert len(set(pivot_idx.tolist())) == P, "pivots must be distinct"
+    dup = _o.similarity_any(keys_bits, vis_offset, n_vis, pivot_idx)
+    kept = np.zeros(n_vis, bool)
+    for i, p in enumerate(pivot_idx.tolist()):
+        if 0 <= p < n_vis:
+            kept[p] = True
+            assert int(owner[p]) == P + i, "vision pivots carry their rank in owner"
+    Pv = int(kept.sum())
+    assert int((owner >= P).sum()) == Pv, "only vision pivots are marked as pivots"
+    u = dup.max(axis=0)
+    mine = np.nonzero((owner >= 0) & (owner < P))[0]
+    assert len(mine) == n_keep - Pv, "retained %d tokens beside the pivots, budget %d" % (len(mine), n_keep - Pv)
+    if len(mine):
+        assert np.all(dup[owner[mine], mine] >= u[mine] - tol), "owner is not (nearly) the most similar pivot"
+        left = ~kept
+        left[mine] = False
+        if left.any():
+            assert u[left].min() >= u[mine].max() - tol, "a token %g below the threshold was left behind" % (u[mine].max() - u[left].min())
+    kept[mine] = True
+    assert int(kept.sum()) == n_keep
     return kept
 
 
@@ -220,8 +249,9 @@ def check_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, n_vis,
             check_sim(dbg["sim"][b], ora.dup[b], rep)
         if margin[b] > require_exact_above:
             assert np.array_equal(dbg["owner"][b], ora.owner[b])
-            qs = (quotas_any(dbg["pivot_idx"][b], n_vis, n_keep) if text_pivots else
-                  quotas(n_pivot, n_keep) if rule == 0 else [n_keep - n_pivot] * n_pivot)
+            Pv_b = int(sum(0 <= int(x) < n_vis for x in dbg["pivot_idx"][b]))
+            qs = ([n_keep - Pv_b] * n_pivot if rule == 1 else
+                  quotas_any(dbg["pivot_idx"][b], n_vis, n_keep) if text_pivots else quotas(n_pivot, n_keep))
             has = np.array([q > 0 for q in qs])
             e = dbg["eps"][b].astype(np.float64)
             assert np.all(np.isnan(e[~has])) and np.all(np.abs(e[has] - ora.eps[b][has]) <= REL_TOL * np.abs(ora.eps[b][has]) + SIM_ABS_FLOOR)
@@ -237,7 +267,7 @@ def check_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, n_vis,
 
 def check_union_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, n_vis, n_pivot, n_keep,
                       out_hidden, out_idx, out_pos, cu_seqlens, dbg, pos_in=None, largest=True, norm_kind=1,
-                      require_exact_above=MARGIN) -> ParityReport:
+                      require_exact_above=MARGIN, text_pivots=False) -> ParityReport:
     """Retention with independent pivots: flat outputs, sample b's rows are cu_seqlens[b] .. cu_seqlens[b + 1] - 1.
     Above the margin everything equals the oracle; below it every pivot's picks are replayed against the oracle's
     fp64 similarities with the candidate's own thresholds (dbg["eps"])."""
@@ -251,7 +281,8 @@ def check_union_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, 
         rep.min_margin = min(rep.min_margin, float(margin[b]))
         lo, hi = int(cu[b]), int(cu[b + 1])
         kept = hi - lo - (S - n_vis)
-        assert n_pivot <= kept <= n_keep, "sample %d keeps %d vision tokens" % (b, kept)
+        Pv_b = int(sum(0 <= int(x) < n_vis for x in dbg["pivot_idx"][b]))
+        assert Pv_b <= kept <= n_keep, "sample %d keeps %d vision tokens" % (b, kept)
         pin = None if pos_in is None else pos_in[b]
         check_packed_outputs(None if out_hidden is None else out_hidden[lo:hi], out_idx[lo:hi], out_pos[lo:hi],
                              hidden_bits[b], pin, vis_offset, n_vis, kept)
@@ -279,13 +310,14 @@ def check_union_batch(ora: _o.OracleResult, keys_bits, hidden_bits, vis_offset, 
         score = ora.l1[b] if norm_kind == 1 else ora.l2[b]
         sgn = 1.0 if largest else -1.0
         others = np.setdiff1d(np.arange(n_vis), piv)
-        if len(others):
+        if len(others) and not text_pivots:   # (text pivots are the caller's: nothing about their ranking to check)
             assert (sgn * score[piv]).min() >= (sgn * score[others]).max() * (1 - MARGIN * np.sign((sgn * score[others]).max()))
-        dup = _o.similarity(keys_bits[b], vis_offset, n_vis, piv, ora.l2[b])
+        dup = (_o.similarity_any(keys_bits[b], vis_offset, n_vis, piv) if text_pivots else
+               _o.similarity(keys_bits[b], vis_offset, n_vis, piv, ora.l2[b]))
         e = dbg["eps"][b].astype(np.float64)
         allowed = np.zeros(n_vis, bool)
-        allowed[piv] = True
-        for i, qi in enumerate(quotas(n_pivot, n_keep)):
+        allowed[piv[(piv >= 0) & (piv < n_vis)]] = True
+        for i, qi in enumerate(quotas_any(piv, n_vis, n_keep) if text_pivots else quotas(n_pivot, n_keep)):
             if qi == 0:
                 assert np.isnan(e[i])
                 continue

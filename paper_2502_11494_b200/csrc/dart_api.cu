@@ -76,6 +76,9 @@ struct dart_ctx {
     bool pair_ok;
     unsigned long long *pair_cand; // [B_max][sm_count][16] candidate keys
     int32_t *pair_res;             // [B_max][32] resolved pivots and their norms
+    // pivots chosen inside the library from other sources than the vision tokens' scores (dart_opts.pivot_source)
+    int32_t *pivot_src;            // [B_max][P_max]
+    float *text_score;             // [2][B_max][S_max]: L1 scores, then sums of squares, of the text rows (before | after the block)
 };
 
 namespace {
@@ -684,8 +687,58 @@ int launch_two_pass(dart_ctx *ctx, int B, const void *hidden, const void *keys, 
 
 int launch_reduce(dart_ctx *ctx, int B, const void *hidden, const void *keys, const int64_t *pos_in, int vis_offset,
                   int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos, const dart_opts &o,
+                  const dart_debug *dbg, cudaStream_t st);
+
+// Step 2 from another source than the vision tokens' scores (dart_opts.pivot_source): the pivots are written to the
+// workspace by a kernel of their own and the call goes on as if the caller had named them.
+int launch_with_pivot_source(dart_ctx *ctx, int B, const void *hidden, const void *keys, const int64_t *pos_in, int vis_offset,
+                             int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos,
+                             const dart_opts &o, const dart_debug *dbg, cudaStream_t st)
+{
+    using namespace dart;
+    const int S = ctx->S, d8 = ctx->desc.d / 8, P_pad = next_pow2(P);
+    const uint4 *k = (const uint4 *)(keys ? keys : hidden);
+    dart_opts o2 = o;
+    o2.pivot_source = 0, o2.pivots_in = ctx->pivot_src;
+    if (o.pivot_source == DART_PIVOTS_RANDOM) {
+        Prof p(ctx, st, SLOT_PIVOT);
+        pivot_random_kernel<<<B, kSelectThreads, (size_t)P_pad * 8, st>>>(o.seed, o.sample_base, n_vis, P, P_pad, ctx->pivot_src);
+    } else { // both modalities: the scores of the vision rows and of the text rows before and after them
+        const int Pt = o.n_text_pivots, n_after = S - vis_offset - n_vis;
+        const size_t half = (size_t)ctx->desc.B_max * ctx->desc.S_max;
+        float *tb = ctx->text_score, *ta = ctx->text_score + (size_t)B * vis_offset; // L1 scores; the sums of squares lie `half` further
+        {
+            Prof p(ctx, st, SLOT_SCORE);
+            const long long rows = (long long)B * n_vis;
+            score_kernel<<<(unsigned)((rows + kScoreWarps - 1) / kScoreWarps), kScoreWarps * 32, 0, st>>>(k, S, d8, vis_offset, n_vis, rows,
+                                                                                                        ctx->l1, ctx->ssq);
+            ++ctx->launches;
+            if (vis_offset > 0) {
+                const long long r = (long long)B * vis_offset;
+                score_kernel<<<(unsigned)((r + kScoreWarps - 1) / kScoreWarps), kScoreWarps * 32, 0, st>>>(k, S, d8, 0, vis_offset, r, tb, tb + half);
+            }
+            if (n_after > 0) {
+                const long long r = (long long)B * n_after;
+                score_kernel<<<(unsigned)((r + kScoreWarps - 1) / kScoreWarps), kScoreWarps * 32, 0, st>>>(k, S, d8, vis_offset + n_vis, n_after, r,
+                                                                                                      ta, ta + half);
+            }
+        }
+        Prof p(ctx, st, SLOT_PIVOT);
+        const size_t shift = o.norm_kind == 2 ? half : 0; // which of the two scores ranks the pivots
+        pivot_mixed_kernel<<<B, kSelectThreads, (size_t)P_pad * 8, st>>>((o.norm_kind == 2 ? ctx->ssq : ctx->l1), tb + shift, ta + shift, S,
+                                                                        vis_offset, n_vis, P - Pt, Pt, P_pad, o.pivot_smallest, ctx->pivot_src);
+        o2.text_pivots = 1;
+    }
+    DART_CUDA(ctx, cudaGetLastError());
+    return launch_reduce(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o2, dbg, st);
+}
+
+int launch_reduce(dart_ctx *ctx, int B, const void *hidden, const void *keys, const int64_t *pos_in, int vis_offset,
+                  int n_vis, int P, int n_keep, void *out_hidden, int32_t *out_idx, int64_t *out_pos, const dart_opts &o,
                   const dart_debug *dbg, cudaStream_t st)
 {
+    if (o.pivot_source != DART_PIVOTS_BY_SCORE)
+        return launch_with_pivot_source(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o, dbg, st);
     const bool fused = o.path == DART_PATH_FUSED || (o.path == DART_PATH_AUTO && fused_applies(ctx, P));
     if (fused && !fused_applies(ctx, P)) return DART_ERR_UNSUPPORTED;
     if (o.path == DART_PATH_RESIDENT || o.path == DART_PATH_SPLIT) {
@@ -704,7 +757,6 @@ int launch_reduce(dart_ctx *ctx, int B, const void *hidden, const void *keys, co
         if (!pair_applies(ctx, P) || o.pivots_in || (o.cosine_on_hidden && keys && keys != hidden)) return DART_ERR_UNSUPPORTED;
         return launch_pair(ctx, B, hidden, keys, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o, dbg, st);
     }
-    if (o.text_pivots && !fused) return DART_ERR_UNSUPPORTED; // only the tensor-core kernel takes a text row's norm from the row
     if (o.cosine_on_hidden && keys && keys != hidden)
         return launch_two_pass(ctx, B, hidden, keys, hidden, pos_in, vis_offset, n_vis, P, n_keep, out_hidden, out_idx, out_pos, o,
                                dbg, fused, st);
@@ -780,6 +832,8 @@ int dart_create(dart_ctx **out, const dart_desc *desc)
     if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->owner, nv);
     if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->keep, nv);
     if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->len, (size_t)desc->B_max);
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->pivot_src, np);
+    if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->text_score, 2 * nv);
     if (rc == DART_OK) {
         // candidate lists of the two-phase retention: at most kCandMax entries per pivot; contexts whose maxima
         // would need more than 1 GiB go without (they use the one-kernel retention)
@@ -872,6 +926,8 @@ int dart_destroy(dart_ctx *ctx)
     cudaFree(ctx->owner);
     cudaFree(ctx->keep);
     cudaFree(ctx->len);
+    cudaFree(ctx->pivot_src);
+    cudaFree(ctx->text_score);
     cudaFree(ctx->cand);
     cudaFree(ctx->piv_rows);
     cudaFree(ctx->status);
@@ -927,7 +983,18 @@ int dart_reduce_ex(dart_ctx *ctx, const void *hidden, const void *keys, const in
     }
     if (o.cosine_on_hidden && o.norm_kind != 1) return DART_ERR_UNSUPPORTED; // the hidden rows' sums of squares take the slot
     if ((uintptr_t)o.pivots_in & 3u) return DART_ERR_ALIGN;
-    if (o.text_pivots && (!o.pivots_in || o.rule != DART_RULE_QUOTAS)) return DART_ERR_UNSUPPORTED;
+    if (o.pivot_source != DART_PIVOTS_BY_SCORE && o.pivot_source != DART_PIVOTS_MIXED && o.pivot_source != DART_PIVOTS_RANDOM)
+        return DART_ERR_UNSUPPORTED;
+    if (o.pivot_source != DART_PIVOTS_BY_SCORE) {
+        // the pivots then reach steps 3-5 like the caller's: only the paths that take those
+        if (o.pivots_in) return DART_ERR_UNSUPPORTED;
+        if (o.path == DART_PATH_RESIDENT || o.path == DART_PATH_SPLIT || o.path == DART_PATH_PAIRED) return DART_ERR_UNSUPPORTED;
+        if (o.pivot_source == DART_PIVOTS_MIXED &&
+            (o.n_text_pivots < 0 || o.n_text_pivots > n_pivot || o.n_text_pivots > ctx->S - n_vis || n_pivot - o.n_text_pivots > n_vis))
+            return DART_ERR_BAD_SHAPE;
+        if (o.sample_base < 0) return DART_ERR_BAD_SHAPE;
+    }
+    if (o.text_pivots && !o.pivots_in) return DART_ERR_UNSUPPORTED;
     if (o.rule == DART_RULE_GLOBAL &&
         dart::retain_global_smem_bytes(n_vis) > (size_t)ctx->max_smem_optin - 2048)
         return DART_ERR_UNSUPPORTED; // the sample's duplication values must fit shared memory

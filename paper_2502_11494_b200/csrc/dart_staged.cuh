@@ -76,6 +76,25 @@ __device__ __forceinline__ void rank_sort(const unsigned long long *list, int n,
 inline size_t pivot_smem_bytes(int n_vis, int P_pad, bool cached) { return (size_t)P_pad * 8 + (cached ? (size_t)n_vis * 4 : 0); }
 constexpr int kPivotCacheMax = 32768; // scores of a sample that are kept in shared memory as keys (128 KB)
 
+// The k elements of smallest key among n (KeyFn(j, key&) as in block_select_threshold), handed to put(rank, j) in
+// ascending (key, index) order.  All threads of the CTA; list: k_pad entries of shared memory.
+template <typename KeyFn, typename Put>
+__device__ __forceinline__ void cta_smallest_k(KeyFn keyfn, int n, int k, int k_pad, unsigned long long *list, SelectSmem &sel,
+                                               uint32_t *n_picked, Put put)
+{
+    for (int i = threadIdx.x; i < k_pad; i += blockDim.x) list[i] = ~0ull;
+    if (threadIdx.x == 0) *n_picked = 0;
+    __syncthreads();
+    uint32_t T, need_eq, cnt_eq;
+    block_select_threshold(CtaGroup(), keyfn, n, (uint32_t)k, sel, T, need_eq, cnt_eq);
+    block_select_apply(CtaGroup(), keyfn, n, T, need_eq, cnt_eq, sel, [&](int j, uint32_t key) {
+        uint32_t slot = atomicAdd(n_picked, 1u);
+        list[slot] = ((unsigned long long)key << 32) | (uint32_t)j;
+    });
+    rank_sort(list, k, [&](int r, unsigned long long x) { put(r, (int)(x & 0xffffffffu)); });
+    __syncthreads();
+}
+
 __global__ void __launch_bounds__(kSelectThreads)
 pivot_kernel(const float *__restrict__ score, int n_vis, int P, int P_pad, int smallest, int cached,
              int32_t *__restrict__ pivot_idx)
@@ -101,17 +120,68 @@ pivot_kernel(const float *__restrict__ score, int n_vis, int P, int P_pad, int s
         }
         return true;
     };
-    for (int i = threadIdx.x; i < P_pad; i += blockDim.x) piv_list[i] = ~0ull;
-    if (threadIdx.x == 0) n_picked = 0;
-    __syncthreads();
-    uint32_t T, need_eq, cnt_eq;
-    block_select_threshold(CtaGroup(), keyfn, n_vis, (uint32_t)P, sel, T, need_eq, cnt_eq);
-    block_select_apply(CtaGroup(), keyfn, n_vis, T, need_eq, cnt_eq, sel, [&](int j, uint32_t key) {
-        uint32_t slot = atomicAdd(&n_picked, 1u);
-        piv_list[slot] = ((unsigned long long)key << 32) | (uint32_t)j;
-    });
     // ascending order of (key, index): rank 0 = best score, ties to the lower index
-    rank_sort(piv_list, P, [&](int r, unsigned long long x) { pivot_idx[(size_t)b * P + r] = (int32_t)(x & 0xffffffffu); });
+    cta_smallest_k(keyfn, n_vis, P, P_pad, piv_list, sel, &n_picked, [&](int r, int j) { pivot_idx[(size_t)b * P + r] = j; });
+}
+
+// Pivots from both modalities (Sec. 5.4; the pivot-selection table fixes "4 visual and 4 text tokens"): the Pv vision
+// tokens and the Pt text tokens of best score, the vision pivots in rank order first, then the text pivots in rank order,
+// as indices relative to the vision block (a text token before it is negative, one after it >= n_vis).
+//   score_vis [B][n_vis]; score_before [B][vis_offset]; score_after [B][S - vis_offset - n_vis]
+__global__ void __launch_bounds__(kSelectThreads)
+pivot_mixed_kernel(const float *__restrict__ score_vis, const float *__restrict__ score_before, const float *__restrict__ score_after,
+                   int S, int vis_offset, int n_vis, int Pv, int Pt, int P_pad, int smallest, int32_t *__restrict__ pivot_idx)
+{
+    extern __shared__ unsigned long long piv_list[]; // [P_pad]
+    __shared__ SelectSmem sel;
+    __shared__ uint32_t n_picked;
+    const int b = blockIdx.x, P = Pv + Pt, n_after = S - vis_offset - n_vis, n_text = vis_offset + n_after;
+    const float *sv = score_vis + (size_t)b * n_vis;
+    auto vis_key = [&](int j, uint32_t &key) {
+        const uint32_t k = order_key(sv[j]);
+        key = smallest ? k : ~k;
+        return true;
+    };
+    if (Pv > 0)
+        cta_smallest_k(vis_key, n_vis, Pv, P_pad, piv_list, sel, &n_picked, [&](int r, int j) { pivot_idx[(size_t)b * P + r] = j; });
+    // text token t: position t before the block, or vis_offset + n_vis + (t - vis_offset) after it
+    auto text_key = [&](int t, uint32_t &key) {
+        const float v = t < vis_offset ? score_before[(size_t)b * vis_offset + t] : score_after[(size_t)b * n_after + (t - vis_offset)];
+        const uint32_t k = order_key(v);
+        key = smallest ? k : ~k;
+        return true;
+    };
+    if (Pt > 0)
+        cta_smallest_k(text_key, n_text, Pt, P_pad, piv_list, sel, &n_picked, [&](int r, int t) {
+            pivot_idx[(size_t)b * P + Pv + r] = t < vis_offset ? t - vis_offset : n_vis + (t - vis_offset);
+        });
+}
+
+// Output number k of a SplitMix64 generator seeded with `seed` (Steele, Lea, Flood, OOPSLA 2014): mix(seed + (k + 1) gamma)
+__device__ __forceinline__ unsigned long long splitmix64_at(unsigned long long seed, unsigned long long k)
+{
+    unsigned long long z = seed + (k + 1ull) * 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+// Random pivots (Sec. 5.2 also draws them at random): every vision token of sample b0 + blockIdx.x gets a 32-bit ticket,
+// the upper half of output number (sample * 2^32 + token) of the generator; the P smallest tickets win, smallest first,
+// equal tickets to the lower index: a uniform draw without replacement.
+__global__ void __launch_bounds__(kSelectThreads)
+pivot_random_kernel(unsigned long long seed, int b0, int n_vis, int P, int P_pad, int32_t *__restrict__ pivot_idx)
+{
+    extern __shared__ unsigned long long piv_list[]; // [P_pad]
+    __shared__ SelectSmem sel;
+    __shared__ uint32_t n_picked;
+    const int b = blockIdx.x;
+    const unsigned long long hi = (unsigned long long)(uint32_t)(b0 + b) << 32;
+    auto keyfn = [&](int j, uint32_t &key) {
+        key = (uint32_t)(splitmix64_at(seed, hi | (uint32_t)j) >> 32);
+        return true;
+    };
+    cta_smallest_k(keyfn, n_vis, P, P_pad, piv_list, sel, &n_picked, [&](int r, int j) { pivot_idx[(size_t)b * P + r] = j; });
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -130,13 +200,38 @@ sim_alu_kernel(const uint4 *__restrict__ keys, int S, int d8, int vis_offset, in
                const int32_t *__restrict__ pivot_idx, const float *__restrict__ ssq, float *__restrict__ sim)
 {
     extern __shared__ uint4 piv_rows[]; // [kSimPivotChunk][d8]
+    __shared__ float piv_norm[kSimPivotChunk];
     const int b = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint4 *base = keys + ((size_t)b * S + vis_offset) * (size_t)d8;
     const int np = min(kSimPivotChunk, P - p0);
+    // a pivot outside [0, n_vis) is a text token of the same sample (checked and clamped to the sample by step 2)
     for (int i = threadIdx.x; i < kSimPivotChunk * d8; i += blockDim.x) {
         int p = i / d8, c = i - p * d8;
-        piv_rows[i] = (p < np) ? __ldg(base + (size_t)pivot_idx[(size_t)b * P + p0 + p] * d8 + c)
+        piv_rows[i] = (p < np) ? __ldg(base + (long long)pivot_idx[(size_t)b * P + p0 + p] * d8 + c)
                                : make_uint4(0, 0, 0, 0);
+    }
+    __syncthreads();
+    // Euclidean norms of the pivots: a vision token's comes from step 1; a text token was not scored, so warp p sums the
+    // squares of the staged row p (lanes over 16-byte chunks, fixed order)
+    for (int p = warp; p < np; p += kSimWarps) {
+        const int pv = pivot_idx[(size_t)b * P + p0 + p];
+        float q = 0.f;
+        if (pv < 0 || pv >= n_vis) {
+            for (int c = lane; c < d8; c += 32) {
+                const uint4 w = piv_rows[p * d8 + c];
+                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float lo = bf16_lo(ww[e]), hi = bf16_hi(ww[e]);
+                    q = fmaf(lo, lo, q);
+                    q = fmaf(hi, hi, q);
+                }
+            }
+            q = warp_sum(q);
+        } else {
+            q = ssq[(size_t)b * n_vis + pv];
+        }
+        if (lane == 0) piv_norm[p] = sqrtf(q);
     }
     __syncthreads();
     const int tile0 = blockIdx.x * kSimRowsPerCta;
@@ -180,8 +275,7 @@ sim_alu_kernel(const uint4 *__restrict__ keys, int S, int d8, int vis_offset, in
 #pragma unroll
                 for (int p = 0; p < kSimPivotChunk; ++p) {
                     if (p >= np) break;
-                    float np_ = sqrtf(ssq[(size_t)b * n_vis + pivot_idx[(size_t)b * P + p0 + p]]);
-                    float den = np_ * nj;
+                    float den = piv_norm[p] * nj;
                     sim[((size_t)b * P + p0 + p) * n_vis + row] = den > 0.f ? acc[r][p] / den : 0.f;
                 }
             }
@@ -594,13 +688,9 @@ retain_global_kernel(const float *__restrict__ sim, const int32_t *__restrict__ 
         if (owner) owner[j] = -1;
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < P; i += blockDim.x) {
-        const int pv = pivot_idx[(size_t)b * P + i];
-        keep[pv] = 1;
-        if (owner) owner[pv] = P + i;
-    }
-    __syncthreads();
-    const int take = n_keep - P;
+    // pivots outside the vision block are text tokens: compared with, but neither marked nor counted
+    const int Pv = mark_pivots(pivot_idx + (size_t)b * P, P, n_vis, keep, owner, &sel.cnt);
+    const int take = n_keep - Pv;
     float eps = __int_as_float(0x7fc00000);
     if (take > 0) {
         auto keyfn = [&](int j, uint32_t &key) {
@@ -662,13 +752,21 @@ retain_union_kernel(const float *__restrict__ sim, const int32_t *__restrict__ p
         if (owner) owner[j] = -1;
     }
     __syncthreads();
+    // pivots outside the vision block are text tokens: they pick like any pivot, but are neither marked nor counted
+    __shared__ int n_vis_pivots;
+    if (threadIdx.x == 0) n_vis_pivots = 0;
+    __syncthreads();
     for (int i = threadIdx.x; i < P; i += blockDim.x) {
         const int pv = pivot_idx[(size_t)b * P + i];
-        flags[pv] = 2;
-        if (owner) owner[pv] = P + i;
+        if (pv >= 0 && pv < n_vis) {
+            flags[pv] = 2;
+            if (owner) owner[pv] = P + i;
+            atomicAdd(&n_vis_pivots, 1);
+        }
     }
     __syncthreads();
-    const int q = (n_keep - P) / P, r = (n_keep - P) % P;
+    const int Pv = n_vis_pivots;
+    const int q = (n_keep - Pv) / P, r = (n_keep - Pv) % P;
     for (int i = 0; i < P; ++i) {
         const int qi = q + (i < r ? 1 : 0);
         if (qi == 0) {

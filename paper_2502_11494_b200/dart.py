@@ -21,6 +21,7 @@ DART_FLAG_HOST_STAGING = 1
 DART_PATH_AUTO, DART_PATH_STAGED, DART_PATH_FUSED, DART_PATH_TWO_PASS, DART_PATH_RESIDENT, DART_PATH_SPLIT, DART_PATH_PAIRED = 0, 1, 2, 3, 4, 5, 6
 DART_RETAIN_AUTO, DART_RETAIN_SERIAL, DART_RETAIN_LISTS = 0, 1, 2
 DART_RULE_QUOTAS, DART_RULE_GLOBAL, DART_RULE_UNION = 0, 1, 2
+DART_PIVOTS_BY_SCORE, DART_PIVOTS_MIXED, DART_PIVOTS_RANDOM = 0, 1, 2
 
 EXPORTS = (
     "dart_create", "dart_destroy", "dart_set_shape", "dart_reduce", "dart_reduce_ex", "dart_reduce_host",
@@ -42,7 +43,9 @@ class dart_opts(ctypes.Structure):
                 ("wait_limit", ctypes.c_int32), ("sweep_lag", ctypes.c_int32),
                 ("test_withhold_pivots", ctypes.c_int32), ("retention", ctypes.c_int32), ("rule", ctypes.c_int32),
                 ("cosine_on_hidden", ctypes.c_int32), ("text_pivots", ctypes.c_int32), ("pivots_in", ctypes.c_void_p),
-                ("cu_seqlens", ctypes.c_void_p), ("resident_split", ctypes.c_int32), ("tune", ctypes.c_int32)]
+                ("cu_seqlens", ctypes.c_void_p), ("resident_split", ctypes.c_int32), ("pivot_source", ctypes.c_int32),
+                ("n_text_pivots", ctypes.c_int32), ("seed", ctypes.c_uint64), ("sample_base", ctypes.c_int32),
+                ("tune", ctypes.c_int32)]
 
 
 class dart_debug(ctypes.Structure):

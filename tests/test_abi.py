@@ -44,8 +44,8 @@ def test_struct_layouts_match_the_header():
     from paper_2502_11494_b200 import dart
 
     assert ctypes.sizeof(dart.dart_desc) == 28
-    assert ctypes.sizeof(dart.dart_opts) == 64 and dart.dart_opts.pivots_in.offset == 40 and dart.dart_opts.cu_seqlens.offset == 48
-    assert dart.dart_opts.resident_split.offset == 56
+    assert ctypes.sizeof(dart.dart_opts) == 88 and dart.dart_opts.pivots_in.offset == 40 and dart.dart_opts.cu_seqlens.offset == 48
+    assert dart.dart_opts.resident_split.offset == 56 and dart.dart_opts.seed.offset == 72 and dart.dart_opts.tune.offset == 84
     assert ctypes.sizeof(dart.dart_debug) == 7 * ctypes.sizeof(ctypes.c_void_p)
 
 

@@ -249,7 +249,7 @@ TEXT_SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("path", [dart.DART_PATH_AUTO, dart.DART_PATH_FUSED], ids=PATH_IDS.get)
+@pytest.mark.parametrize("path", [dart.DART_PATH_AUTO, dart.DART_PATH_FUSED, dart.DART_PATH_STAGED], ids=lambda p: PATH_IDS.get(p, "auto"))
 @pytest.mark.parametrize("retention", [dart.DART_RETAIN_SERIAL, dart.DART_RETAIN_LISTS], ids=["serial", "lists"])
 @pytest.mark.parametrize("shape", TEXT_SHAPES, ids=lambda s: "x".join(map(str, s)))
 def test_pivots_from_the_text_tokens(oracle, shape, retention, path):
@@ -307,16 +307,133 @@ def test_bad_text_pivots_are_reported_not_used(fault):
     assert detail[1][0] == 100 and detail[1][1] == 1 and detail[1][2] in (0, 3)
 
 
-def test_text_pivots_need_given_pivots_quotas_and_the_tensor_core_path():
+def test_text_pivots_need_given_pivots():
     k, h = gaussian(1, 64, 64, seed=67)
+    ctx = dart.Dart(1, 64, 64, 2, 8)
+    with pytest.raises(dart.DartError) as e:
+        ctx.reduce(h, k, 4, 50, 2, 8, opts=dart.dart_opts(text_pivots=1))
+    assert e.value.code == dart.DART_ERR_UNSUPPORTED
+    ctx.close()
+
+
+@pytest.mark.parametrize("path", [dart.DART_PATH_STAGED, dart.DART_PATH_FUSED], ids=PATH_IDS.get)
+@pytest.mark.parametrize("shape", TEXT_SHAPES[:3] + [(3, 333, 264, 17, 301, 7, 60)], ids=lambda s: "x".join(map(str, s)))
+def test_text_pivots_under_one_threshold(oracle, shape, path):
+    B, S, d, vo, nv, P, Kp = shape
+    k, h = gaussian(B, S, d, seed=440 + sum(shape))
+    piv = text_pivots(B, vo, nv, S, P, seed=1 + sum(shape))
+    oh, oi, op, dbg, _ = run(k, h, vo, nv, P, Kp, path, pivots=torch.from_numpy(piv).cuda(), rule=dart.DART_RULE_GLOBAL, text=True)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=piv, text_pivots=True, rule=1)
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, dbg=dbg, pivots_given=True, text_pivots=True, rule=1)
+    assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5
+
+
+@pytest.mark.parametrize("path", [dart.DART_PATH_STAGED, dart.DART_PATH_FUSED], ids=PATH_IDS.get)
+@pytest.mark.parametrize("shape", TEXT_SHAPES[:3] + [(3, 333, 264, 17, 301, 7, 60)], ids=lambda s: "x".join(map(str, s)))
+def test_text_pivots_with_independent_pivots(oracle, shape, path):
+    B, S, d, vo, nv, P, Kp = shape
+    k, h = gaussian(B, S, d, seed=470 + sum(shape))
+    piv = text_pivots(B, vo, nv, S, P, seed=2 + sum(shape))
+    oh, oi, op, dbg, cu = run_union(k, h, vo, nv, P, Kp, path, pivots=torch.from_numpy(piv).cuda(), text=True)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=piv, text_pivots=True, rule=2)
+    rep = parity.check_union_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, cu, dbg, text_pivots=True)
+    assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5
+
+
+# ----------------------------------------------------------------------------- pivots chosen inside the library from other sources
+
+SOURCE_SHAPES = [
+    (2, 120, 64, 9, 100, 4, 30),
+    (3, 333, 264, 17, 301, 7, 60),       # d not a multiple of 64: plain kernels only
+    (2, 700, 4096, 40, 576, 8, 64),      # the LLaVA-1.5 shape: 4 visual and 4 text pivots
+    (1, 3000, 512, 60, 2880, 16, 320),
+    (1, 400, 3584, 0, 333, 40, 100),     # text after the vision block only
+]
+
+
+def run_source(keys, hidden, vo, nv, P, Kp, path, source, n_text=0, seed=0, base=0, rule=dart.DART_RULE_QUOTAS, norm_kind=0, smallest=0):
+    B, S, d = hidden.shape
+    if path in (dart.DART_PATH_FUSED, dart.DART_PATH_TWO_PASS) and d % 64:
+        pytest.skip("the tensor-core paths need d % 64 == 0")
+    ctx = dart.Dart(B, S, d, P, Kp)
+    try:
+        res = ctx.reduce(hidden, keys, vo, nv, P, Kp, debug=True,
+                         opts=dart.dart_opts(path=path, rule=rule, pivot_source=source, n_text_pivots=n_text, seed=seed, sample_base=base,
+                                             norm_kind=norm_kind, pivot_smallest=smallest))
+        torch.cuda.synchronize()
+        assert ctx.status() == dart.DART_OK, dart.dart_status_detail(ctx.handle)
+    finally:
+        ctx.close()
+    return _np(res[0]), _np(res[1]), _np(res[2]), {n: _np(v) for n, v in res[3].items()}
+
+
+@pytest.mark.parametrize("path", [dart.DART_PATH_AUTO, dart.DART_PATH_STAGED, dart.DART_PATH_FUSED], ids=lambda p: PATH_IDS.get(p, "auto"))
+@pytest.mark.parametrize("shape", SOURCE_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_pivots_from_both_modalities(oracle, shape, path):
+    """Half of the pivots are the text tokens of largest K-norm, half the vision tokens (the ablation's 4 + 4)."""
+    B, S, d, vo, nv, P, Kp = shape
+    k, h = gaussian(B, S, d, seed=520 + sum(shape))
+    Pt = min(P // 2, S - nv)
+    oh, oi, op, dbg = run_source(k, h, vo, nv, P, Kp, path, dart.DART_PIVOTS_MIXED, n_text=Pt)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, pivot_source=1, n_text_pivots=Pt)
+    assert np.array_equal(dbg["pivot_idx"], ora.pivot_idx)       # Gaussian scores: no near-ties at these seeds
+    assert ((ora.pivot_idx[:, P - Pt:] < 0) | (ora.pivot_idx[:, P - Pt:] >= nv)).all()
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, dbg=dbg, pivots_given=True, text_pivots=True)
+    assert rep.samples == B and rep.max_abs_sim < 2e-5
+
+
+@pytest.mark.parametrize("norm_kind,smallest,rule", [(2, 0, dart.DART_RULE_QUOTAS), (1, 1, dart.DART_RULE_GLOBAL)])
+def test_pivots_from_both_modalities_variants(oracle, norm_kind, smallest, rule):
+    B, S, d, vo, nv, P, Kp = 2, 300, 128, 30, 220, 6, 40
+    k, h = gaussian(B, S, d, seed=530)
+    oh, oi, op, dbg = run_source(k, h, vo, nv, P, Kp, dart.DART_PATH_AUTO, dart.DART_PIVOTS_MIXED, n_text=2, rule=rule,
+                                 norm_kind=norm_kind, smallest=smallest)
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, pivot_source=1, n_text_pivots=2, rule=rule, norm_kind=norm_kind, largest=not smallest)
+    assert np.array_equal(dbg["pivot_idx"], ora.pivot_idx)
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, dbg=dbg, pivots_given=True, text_pivots=True, rule=rule,
+                             norm_kind=norm_kind, largest=not smallest)
+    assert rep.samples == B
+
+
+@pytest.mark.parametrize("path", [dart.DART_PATH_AUTO, dart.DART_PATH_STAGED, dart.DART_PATH_FUSED], ids=lambda p: PATH_IDS.get(p, "auto"))
+@pytest.mark.parametrize("shape", SOURCE_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_random_pivots_from_a_seed(oracle, shape, path):
+    """The tickets are integers: the pivots equal the oracle's bit for bit, on every path and every run."""
+    B, S, d, vo, nv, P, Kp = shape
+    k, h = gaussian(B, S, d, seed=560 + sum(shape))
+    oh, oi, op, dbg = run_source(k, h, vo, nv, P, Kp, path, dart.DART_PIVOTS_RANDOM, seed=20240229 + sum(shape))
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp, pivot_source=2, seed=20240229 + sum(shape))
+    assert np.array_equal(dbg["pivot_idx"], ora.pivot_idx)
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, oh, oi, op, dbg=dbg, pivots_given=True)
+    assert rep.exact >= rep.above_margin and rep.max_abs_sim < 2e-5
+
+
+def test_random_pivots_of_a_split_batch_are_those_of_the_whole_batch(oracle):
+    B, S, d, vo, nv, P, Kp = 5, 200, 64, 10, 170, 5, 30
+    k, h = gaussian(B, S, d, seed=590)
+    whole = run_source(k, h, vo, nv, P, Kp, dart.DART_PATH_AUTO, dart.DART_PIVOTS_RANDOM, seed=7)[3]["pivot_idx"]
+    tail = run_source(k[3:].contiguous(), h[3:].contiguous(), vo, nv, P, Kp, dart.DART_PATH_AUTO, dart.DART_PIVOTS_RANDOM, seed=7, base=3)[3]["pivot_idx"]
+    assert np.array_equal(whole[3:], tail)
+    assert np.array_equal(whole, np.stack([oracle.pivots_random(7, b, nv, P) for b in range(B)]))
+
+
+def test_pivot_sources_say_what_they_do_not_take():
+    k, h = gaussian(1, 64, 64, seed=591)
     piv = torch.zeros(1, 2, dtype=torch.int32, device="cuda")
     ctx = dart.Dart(1, 64, 64, 2, 8)
-    for o in (dart.dart_opts(text_pivots=1),
-              dart.dart_opts(text_pivots=1, pivots_in=piv.data_ptr(), rule=dart.DART_RULE_GLOBAL),
-              dart.dart_opts(text_pivots=1, pivots_in=piv.data_ptr(), path=dart.DART_PATH_STAGED)):
+    for o, code in [(dart.dart_opts(pivot_source=3), dart.DART_ERR_UNSUPPORTED),
+                    (dart.dart_opts(pivot_source=1, pivots_in=piv.data_ptr()), dart.DART_ERR_UNSUPPORTED),
+                    (dart.dart_opts(pivot_source=2, path=dart.DART_PATH_RESIDENT), dart.DART_ERR_UNSUPPORTED),
+                    (dart.dart_opts(pivot_source=1, n_text_pivots=3), dart.DART_ERR_BAD_SHAPE),          # more than n_pivot
+                    (dart.dart_opts(pivot_source=2, sample_base=-1), dart.DART_ERR_BAD_SHAPE)]:
         with pytest.raises(dart.DartError) as e:
             ctx.reduce(h, k, 4, 50, 2, 8, opts=o)
-        assert e.value.code == dart.DART_ERR_UNSUPPORTED
+        assert e.value.code == code
     ctx.close()
 
 
@@ -351,7 +468,7 @@ def test_text_pivots_random_shapes(oracle, seed):
 
 # ----------------------------------------------------------------------------- independent pivots, variable-length outputs
 
-def run_union(keys, hidden, vo, nv, P, Kp, path):
+def run_union(keys, hidden, vo, nv, P, Kp, path, pivots=None, text=False):
     B, S, d = hidden.shape
     if path in (dart.DART_PATH_FUSED, dart.DART_PATH_TWO_PASS) and (d % 64 or P > 256):
         pytest.skip("the tensor-core paths need d % 64 == 0 and at most 256 pivots")
@@ -363,7 +480,8 @@ def run_union(keys, hidden, vo, nv, P, Kp, path):
     ctx = dart.Dart(B, S, d, P, Kp)
     try:
         res = ctx.reduce(hidden, keys, vo, nv, P, Kp, out=out, debug=True,
-                         opts=dart.dart_opts(path=path, rule=dart.DART_RULE_UNION, cu_seqlens=cu.data_ptr()))
+                         opts=dart.dart_opts(path=path, rule=dart.DART_RULE_UNION, cu_seqlens=cu.data_ptr(), text_pivots=int(text),
+                                             pivots_in=None if pivots is None else pivots.data_ptr()))
         torch.cuda.synchronize()
         assert ctx.status() == dart.DART_OK, dart.dart_status_detail(ctx.handle)
     finally:
