@@ -91,9 +91,9 @@ def kernel_bytes_per_launch(name, w, B):
 # DRAM traffic of one launch per sample (dram__bytes_read.sum + dram__bytes_write.sum), from ncu captures of each kernel
 # on the sweep workload at batch 32; traffic is proportional to the batch (every sample is read and written
 # independently), so a launch over B samples moves B times this.
-NCU_TRAFFIC_PER_SAMPLE = {("sweep", 2880, 4096, 8): (1.508212e9 + 5.538816e6) / 32,
-                          ("onepass", 2880, 4096, 8): (755.18336e6 + 5.144064e6) / 32,
-                          ("resident", 2880, 4096, 8): (755.081728e6 + 5.729792e6) / 32}
+NCU_TRAFFIC_PER_SAMPLE = {("sweep", 2880, 4096, 8): (1.508338e9 + 8.540928e6) / 32,
+                          ("onepass", 2880, 4096, 8): (755.072256e6 + 5.508864e6) / 32,
+                          ("resident", 2880, 4096, 8): (755.073536e6 + 6.136064e6) / 32}
 
 
 def measured_peak():
@@ -392,7 +392,7 @@ def main():
         roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": achieved / peak,
                     "traffic": (NCU_TRAFFIC_PER_SAMPLE[(dom, w.n_vis, w.d, w.n_pivot)] * B
-                                if (dom, w.n_vis, w.d, w.n_pivot) in NCU_TRAFFIC_PER_SAMPLE and args.lag == 0 else None),
+                                if (dom, w.n_vis, w.d, w.n_pivot) in NCU_TRAFFIC_PER_SAMPLE and args.lag == 0 and args.tune == 0 else None),
                     "peak_source": peak_src + " copy bandwidth",
                     "avg_launch_ms": avg_ms, "timing": "CUDA events around every launch of a separate profiled pass on the launching stream",
                     "shares": {k: v[0] / max(sum(x[0] for x in prof.values()), 1e-9) for k, v in prof.items()}}
