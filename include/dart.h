@@ -89,10 +89,16 @@ enum {
                                   tickets to the lower index.  The same seed gives the same pivots on every run. */
 
 /* dart_opts.retention */
-#define DART_RETAIN_AUTO 0   /* two phases when the batch alone cannot fill the GPU, else one kernel */
+#define DART_RETAIN_AUTO 0   /* candidate bands when their workspace exists (always, unless the context's maxima would need
+                                more than 1 GiB of it); else two phases with sorted lists when the batch alone cannot fill
+                                the GPU, else one kernel */
 #define DART_RETAIN_SERIAL 1 /* one kernel, one CTA per sample: the pivots' selections one after the other */
 #define DART_RETAIN_LISTS 2  /* two phases: sorted candidate lists for all (sample, pivot) pairs at once, then the pivots'
                                 turns as walks over the lists; needs n_keep - n_pivot <= 4096, else the one-kernel form runs */
+#define DART_RETAIN_BANDS 3  /* two phases: per (sample, pivot) pair one warp stores, unsorted, the lowest band of the
+                                pivot's dups that holds at least the tokens the pivot could need; then the pivots' turns,
+                                each taking its quota's smallest free entries of its band.  Needs n_keep - n_pivot <= 6144,
+                                else as without it. */
 
 /* dart_opts.rule */
 #define DART_RULE_QUOTAS 0 /* one threshold per pivot: pivot i keeps its q_i not-yet-kept tokens of lowest dup (dart_reduce) */

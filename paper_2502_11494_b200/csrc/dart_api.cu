@@ -45,6 +45,9 @@ struct dart_ctx {
     int32_t *len;    // [B_max] packed length of every sample (retention with independent pivots)
     int32_t *cand;   // [B_max][P_max][cand_stride] sorted candidate lists of the two-phase retention (NULL: not available)
     int cand_stride;
+    unsigned long long *band; // [B_max][P_max][band_stride] unsorted candidate bands of the band retention (NULL: not available)
+    int32_t *band_n;          // [B_max][P_max] their lengths
+    int band_stride;
     uint8_t *keep;
     int *status; // device status word, followed by three words of detail
     int32_t status_detail[11];
@@ -231,6 +234,23 @@ void launch_retention(dart_ctx *ctx, int B, const int64_t *pos_in, int vis_offse
     const bool can_lists = ctx->cand && m <= ctx->cand_stride && m <= kCandMax &&
                            candidates_smem_bytes(n_vis, m_pad) <= (size_t)ctx->max_smem_optin - 2048 &&
                            walk_smem_bytes(n_vis) <= (size_t)ctx->max_smem_optin - 2048;
+    // bands: a list must hold the m tokens of the exact route and fit one staging round of phase 2
+    const int band_cap = ctx->band_stride < kPickStageEntries ? ctx->band_stride : kPickStageEntries;
+    const bool can_bands = ctx->band && m > 0 && m <= band_cap && n_vis <= kBandMaxTokens && band_smem_bytes(n_vis, band_cap) <= (size_t)ctx->max_smem_optin - 2048 &&
+                           pick_smem_bytes(n_vis, P) <= (size_t)ctx->max_smem_optin - 2048;
+    const bool bands = can_bands && (mode == DART_RETAIN_BANDS || mode == DART_RETAIN_AUTO);
+    if (bands) {
+        {
+            Prof p(ctx, st, SLOT_RETAIN);
+            band_kernel<<<dim3((unsigned)P, (unsigned)B), 32, band_smem_bytes(n_vis, band_cap), st>>>(
+                ctx->sim, ctx->pivot_idx, n_vis, P, n_keep, band_cap, ctx->band, ctx->band_n, ctx->status);
+        }
+        Prof p(ctx, st, SLOT_RETAIN);
+        retain_pick_kernel<<<B, kPickThreads, pick_smem_bytes(n_vis, P), st>>>(
+            ctx->pivot_idx, ctx->band, ctx->band_n, band_cap, pos_in, S, vis_offset, n_vis, P, n_keep, out_idx, out_pos, ctx->keep,
+            ctx->owner, ctx->eps, ctx->status);
+        return;
+    }
     // Both forms do the same selections; the lists spread them over B * P CTAs instead of B, which pays while B
     // CTAs cannot fill the SMs (measured: batch 4-64 up to 4x faster, batch 256 at 8 pivots 20 % slower).
     const bool two_phase = can_lists && (mode == DART_RETAIN_LISTS || (mode == DART_RETAIN_AUTO && B <= ctx->sm_count));
@@ -841,6 +861,15 @@ int dart_create(dart_ctx **out, const dart_desc *desc)
         const size_t entries = np * (size_t)ctx->cand_stride;
         if (entries * sizeof(int32_t) <= ((size_t)1 << 30)) rc = ws_alloc(ctx, &ctx->cand, entries);
     }
+    if (rc == DART_OK) {
+        // candidate bands of the band retention; contexts whose maxima would need more than 1 GiB go without
+        ctx->band_stride = dart::band_stride(desc->Kp_max);
+        const size_t entries = np * (size_t)ctx->band_stride;
+        if (entries * sizeof(unsigned long long) <= ((size_t)1 << 30)) {
+            rc = ws_alloc(ctx, &ctx->band, entries);
+            if (rc == DART_OK) rc = ws_alloc(ctx, &ctx->band_n, np);
+        }
+    }
     if (rc == DART_OK && desc->P_max > dart::onepass::kGatherMaxP) {
         // compact pivot rows for the one-pass kernel at many pivots; contexts that would need more than 2 GiB go without
         const size_t bytes = (size_t)desc->B_max * ((desc->P_max + 15) / 16 * 16) * desc->d * 2;
@@ -875,6 +904,13 @@ int dart_create(dart_ctx **out, const dart_desc *desc)
         if (cudaFuncSetAttribute(dart::candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  ctx->max_smem_optin - 2048) != cudaSuccess ||
             cudaFuncSetAttribute(dart::retain_walk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 ctx->max_smem_optin - 2048) != cudaSuccess)
+            rc = DART_ERR_CUDA;
+    }
+    if (rc == DART_OK && ctx->band) {
+        if (cudaFuncSetAttribute(dart::band_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 ctx->max_smem_optin - 2048) != cudaSuccess ||
+            cudaFuncSetAttribute(dart::retain_pick_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  ctx->max_smem_optin - 2048) != cudaSuccess)
             rc = DART_ERR_CUDA;
     }
@@ -998,7 +1034,8 @@ int dart_reduce_ex(dart_ctx *ctx, const void *hidden, const void *keys, const in
     if (o.rule == DART_RULE_GLOBAL &&
         dart::retain_global_smem_bytes(n_vis) > (size_t)ctx->max_smem_optin - 2048)
         return DART_ERR_UNSUPPORTED; // the sample's duplication values must fit shared memory
-    if (o.retention != DART_RETAIN_AUTO && o.retention != DART_RETAIN_SERIAL && o.retention != DART_RETAIN_LISTS)
+    if (o.retention != DART_RETAIN_AUTO && o.retention != DART_RETAIN_SERIAL && o.retention != DART_RETAIN_LISTS &&
+        o.retention != DART_RETAIN_BANDS)
         return DART_ERR_UNSUPPORTED;
     if ((uintptr_t)pos_in & 7u) return DART_ERR_ALIGN;
     DeviceGuard g(ctx->desc.device);

@@ -657,6 +657,409 @@ retain_walk_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pi
 }
 
 // ------------------------------------------------------------------------------------------------
+// Steps 4 and 5a in two phases with candidate BANDS: one warp and one read of the row per (sample, pivot).
+//
+// Pivot i's picks are among the Q_i smallest (dup, index) pairs of its row (see above), hence among ANY set of its
+// row's tokens that contains those Q_i.  Phase 1 (band_kernel) therefore does no exact selection and no sort: it lays
+// a histogram of kBandBins equal bins over the row's range [min, max], finds the first bin at which the running count
+// reaches Q_i and stores every token up to and including that bin, grouped by bin (a counting sort: the histogram's
+// prefix sums are the bins' offsets), each entry tagged with its bin.  The band is a few entries longer than Q_i
+// (about one bin's population).  When it would not fit the list (a range stretched by an outlier) the last bin alone is
+// cut into kBandBins bins again, up to kBandLevels levels; rows that still do not fit (many equal values) or that hold
+// a value that is not finite take the exact route: the Q_i-th smallest key by bitwise search, then every key below it
+// and the lowest-index keys equal to it, Q_i entries under one tag.
+// Phase 2 (retain_pick_kernel), one CTA per sample, takes the pivots' turns in rank order.  A warp walks pivot i's
+// band from its lowest bin, moving the entries that are still free to the front, until it has passed the bin that holds
+// the q_i-th free entry; the free entries of the bins before that one are all taken, and the rest of the quota is
+// taken from that one bin, smallest (dup, index) first.  eps_i is the last dup taken.  The result equals
+// retain_kernel's exactly.
+//
+// An entry is 64 bits: the order-preserving key of the dup (32), the tag (8), the token's index (24).  Entries with the
+// same key share their tag, so comparing entries compares (dup, index).
+// Dynamic shared memory, phase 1: n_vis * 4 rounded to 16 + 4 per entry of a list.  Phase 2: n_vis rounded to 16 (keep flags) + P * 4 rounded to
+// 16 (band lengths) + 2 * kPickStageEntries * 8 (two buffers of staged bands).
+// ------------------------------------------------------------------------------------------------
+constexpr int kBandBins = 256;
+constexpr int kBandLevels = 3;
+constexpr int kBandMaxTokens = 1 << 24; // an entry has 24 bits for the token's index
+constexpr int kPickThreads = 256;
+constexpr int kPickStageEntries = 6144; // 48 KB of staged entries per buffer of phase 2
+constexpr int kPickAhead = 4;           // chunks of 32 entries read ahead in phase 2
+inline int band_stride(int m) { return (m + m / 4 + 64 + 1) & ~1; } // entries per list for up to m tokens beside the pivots
+inline size_t band_smem_bytes(int n_vis, int stride) { return ((size_t)n_vis * 4 + 15) / 16 * 16 + (size_t)stride * 4; }
+inline size_t pick_smem_bytes(int n_vis, int P)
+{
+    return ((size_t)n_vis + 15) / 16 * 16 + ((size_t)P * 4 + 15) / 16 * 16 + (size_t)2 * kPickStageEntries * 8;
+}
+__device__ __forceinline__ unsigned long long band_entry(uint32_t key, uint32_t tag, uint32_t j)
+{
+    return ((unsigned long long)key << 32) | (tag << 24) | j;
+}
+__device__ __forceinline__ uint32_t entry_tag(unsigned long long e) { return ((uint32_t)e >> 24) & 255u; }
+__device__ __forceinline__ uint32_t entry_index(unsigned long long e) { return (uint32_t)e & 0xffffffu; }
+
+// Asynchronous copies global -> shared memory that pass no register: many in flight per thread.
+template <int kBytes>
+__device__ __forceinline__ void copy_async(void *dst_smem, const void *src)
+{
+    static_assert(kBytes == 8 || kBytes == 16, "cp.async.ca takes 4, 8 or 16 bytes");
+    asm volatile("cp.async.ca.shared.global [%0], [%1], %2;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_smem)), "l"(src), "n"(kBytes)
+                 : "memory");
+}
+__device__ __forceinline__ void copy_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int kPending>
+__device__ __forceinline__ void copy_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory"); }
+
+// k-th smallest (k >= 1) of the keys a warp holds, given each lane's count of its keys below a value.
+template <typename CountFn>
+__device__ __forceinline__ uint32_t warp_kth_key(CountFn count_below, uint32_t k)
+{
+    uint32_t v = 0; // the largest value with fewer than k keys below it
+    for (int bit = 31; bit >= 0; --bit) {
+        const uint32_t t = v | (1u << bit);
+        if (__reduce_add_sync(0xffffffffu, count_below(t)) < k) v = t;
+    }
+    return v;
+}
+
+__global__ void __launch_bounds__(32)
+band_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx, int n_vis, int P, int n_keep, int stride,
+            unsigned long long *__restrict__ band, int32_t *__restrict__ band_n, const int *__restrict__ status)
+{
+    extern __shared__ __align__(16) uint8_t band_smem[];
+    uint32_t *vs = reinterpret_cast<uint32_t *>(band_smem); // [n_vis rounded up to 4] the row's dups as bit patterns
+    __shared__ uint32_t hist[kBandBins];                    // the bins' counts, then their offsets in the list
+    __shared__ uint32_t n_low;                              // entries below the interval of a finer level handed out so far
+    __shared__ uint32_t n_queued;                           // the band's tokens found so far
+    if (*status != 0) return; // an earlier kernel of this call failed: its outputs are undefined
+    const int i = blockIdx.x, b = blockIdx.y, lane = threadIdx.x;
+    const uint32_t lt = (1u << lane) - 1u;
+    constexpr uint32_t kNotAToken = 0xffffffffu; // a pivot, or the filler behind the row: a NaN no arithmetic produces
+    const float *row = sim + ((size_t)b * P + i) * n_vis;
+    const int n4 = (n_vis + 3) / 4; // groups of four values
+    const bool aligned = (n_vis & 3) == 0; // rows start on 16-byte boundaries
+    if (aligned) { // the whole row is on its way before anything else is looked at
+        for (int j = lane; j < n4; j += 32) copy_async<16>(vs + 4 * j, row + 4 * j);
+        copy_async_commit();
+    } else {
+#pragma unroll 8
+        for (int j = lane; j < n4 * 4; j += 32) vs[j] = __float_as_uint(__ldcs(row + (j < n_vis ? j : 0))); // (filler: a value of the row)
+    }
+    const int32_t *piv = pivot_idx + (size_t)b * P;
+    uint32_t mine = 0;
+    for (int t = lane; t < P; t += 32) mine += (piv[t] >= 0 && piv[t] < n_vis) ? 1u : 0u;
+    const int Pv = (int)__reduce_add_sync(0xffffffffu, mine);
+    const int q = (n_keep - Pv) / P, r = (n_keep - Pv) % P;
+    copy_async_wait<0>();
+    __syncwarp();
+    if (q + (i < r ? 1 : 0) == 0) { // this pivot keeps nothing
+        if (lane == 0) band_n[(size_t)b * P + i] = 0;
+        return;
+    }
+    const uint32_t C = (uint32_t)quota_prefix(i, q, r);
+    // the row's smallest and largest value (pivots included: they only stretch the upper end; a NaN is passed over)
+    const uint4 *vs4 = reinterpret_cast<const uint4 *>(vs);
+    uint32_t *queue = vs + (size_t)n4 * 4; // [stride] the band's tokens, in no order
+    float f_lo = __int_as_float(0x7f800000), f_hi = __int_as_float(0xff800000), f_sum = 0.0f;
+#pragma unroll 2
+    for (int j = lane; j < n4; j += 32) {
+        const uint4 v = vs4[j];
+        f_lo = fminf(fminf(f_lo, __uint_as_float(v.x)), fminf(fminf(__uint_as_float(v.y), __uint_as_float(v.z)), __uint_as_float(v.w)));
+        f_hi = fmaxf(fmaxf(f_hi, __uint_as_float(v.x)), fmaxf(fmaxf(__uint_as_float(v.y), __uint_as_float(v.z)), __uint_as_float(v.w)));
+        f_sum += (__uint_as_float(v.x) + __uint_as_float(v.y)) + (__uint_as_float(v.z) + __uint_as_float(v.w));
+    }
+    f_lo = order_key_inv(__reduce_min_sync(0xffffffffu, order_key(f_lo)));
+    f_hi = order_key_inv(__reduce_max_sync(0xffffffffu, order_key(f_hi)));
+    f_sum = warp_sum(f_sum);
+    for (int t = lane; t < P; t += 32)
+        if (piv[t] >= 0 && piv[t] < n_vis) vs[piv[t]] = kNotAToken;
+    if (lane < n4 * 4 - n_vis) vs[n_vis + lane] = kNotAToken;
+    if (lane == 0) n_queued = 0;
+    __syncwarp();
+    // The band: every value below lo, and the values of [lo, hi] whose bin is at most last_bin.  A level lays its bins
+    // over the smallest and largest value of the interval it looks at; while the band is too long for the list the
+    // next level looks at the last bin alone.  (kNotAToken compares false with everything: it is in no interval.)
+    // The first level's bins span [min, 2 * mean - min] only (whatever lies above goes into the last bin): a band is the
+    // row's low end, and a few large dups - the pivot's own cluster - would otherwise take most of the bins.
+    float lo = f_lo, hi = f_hi;
+    const float spread = 2.0f * (f_sum / (float)(n4 * 4) - f_lo);
+    float scale = (float)kBandBins / (spread > 0.0f && spread < f_hi - f_lo ? spread : f_hi - f_lo);
+    // equal values, an infinite one, a NaN, or places that overflow
+    bool exact = !(f_hi > f_lo) || !(f_hi - f_lo < 3.0e38f) || !((f_hi - f_lo) * scale < 3.0e38f);
+    uint32_t before = 0, last_bin = 0, n_band = 0, my_off = 0;
+    int level = 0;
+    auto bin_of = [&](float f) { return min((int)((f - lo) * scale), kBandBins - 1); }; // for lo <= f <= hi: not negative, monotone
+    uint32_t c[kBandBins / 32];
+    while (!exact) {
+        for (int t = lane; t < kBandBins; t += 32) hist[t] = 0;
+        __syncwarp();
+#pragma unroll 2
+        for (int j = lane; j < n4; j += 32) {
+            const uint4 v = vs4[j];
+            const float f[4] = {__uint_as_float(v.x), __uint_as_float(v.y), __uint_as_float(v.z), __uint_as_float(v.w)};
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+                if (f[t] >= lo && f[t] <= hi) atomicAdd(&hist[bin_of(f[t])], 1u);
+        }
+        __syncwarp();
+        // lane l owns bins [8l, 8l + 8): the first bin at which the running count reaches the rest of C, and the counts there
+        const uint32_t want = C - before; // >= 1, and the interval holds at least that many values
+        uint32_t sum = 0;
+#pragma unroll
+        for (int t = 0; t < kBandBins / 32; ++t) {
+            c[t] = hist[lane * (kBandBins / 32) + t];
+            sum += c[t];
+        }
+        uint32_t incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        my_off = before + incl - sum; // where this lane's first bin starts in the list
+        if (level == 0 && __shfl_sync(0xffffffffu, incl, 31) != (uint32_t)(n_vis - Pv)) { // a NaN among the values
+            exact = true;
+            break;
+        }
+        uint32_t my_bin = 0, my_upto = 0, my_cnt = 0;
+        const bool here = incl - sum < want && want <= incl; // exactly one lane
+        if (here) {
+            uint32_t run = incl - sum;
+#pragma unroll
+            for (int t = 0; t < kBandBins / 32; ++t) {
+                if (run < want && want <= run + c[t]) {
+                    my_bin = lane * (kBandBins / 32) + t;
+                    my_upto = run + c[t];
+                    my_cnt = c[t];
+                }
+                run += c[t];
+            }
+        }
+        const int src = __ffs(__ballot_sync(0xffffffffu, here)) - 1;
+        last_bin = __shfl_sync(0xffffffffu, my_bin, src);
+        n_band = before + __shfl_sync(0xffffffffu, my_upto, src);
+        const uint32_t in_last = __shfl_sync(0xffffffffu, my_cnt, src);
+        if (n_band <= (uint32_t)stride) break;
+        // look at the last bin alone: its smallest and largest value
+        float n_lo = __int_as_float(0x7f800000), n_hi = __int_as_float(0xff800000);
+        for (int j = lane; j < n4 * 4; j += 32) {
+            const float f = __uint_as_float(vs[j]);
+            if (f >= lo && f <= hi && bin_of(f) == (int)last_bin) {
+                n_lo = fminf(n_lo, f);
+                n_hi = fmaxf(n_hi, f);
+            }
+        }
+        n_lo = order_key_inv(__reduce_min_sync(0xffffffffu, order_key(n_lo)));
+        n_hi = order_key_inv(__reduce_max_sync(0xffffffffu, order_key(n_hi)));
+        before = n_band - in_last;
+        lo = n_lo;
+        hi = n_hi;
+        scale = (float)kBandBins / (n_hi - n_lo);
+        exact = ++level == kBandLevels || !(n_hi > n_lo) || !(scale < 3.0e38f);
+    }
+    unsigned long long *out = band + ((size_t)b * P + i) * stride;
+    if (!exact) {
+        // the bins' offsets
+        __syncwarp();
+#pragma unroll
+        for (int t = 0; t < kBandBins / 32; ++t) {
+            hist[lane * (kBandBins / 32) + t] = my_off;
+            my_off += c[t];
+        }
+        if (lane == 0) n_low = 0;
+        // the band's tokens: few of the row's, so they are queued first and then handled with all lanes busy
+        const float edge = last_bin == kBandBins - 1 ? 3.0e38f : (float)(last_bin + 1); // bin <= last_bin <=> place < edge
+#pragma unroll 2
+        for (int j = lane; j < n4; j += 32) {
+            const uint4 v = vs4[j];
+            const float f[4] = {__uint_as_float(v.x), __uint_as_float(v.y), __uint_as_float(v.z), __uint_as_float(v.w)};
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+                if ((f[t] - lo) * scale < edge && f[t] <= hi) queue[atomicAdd(&n_queued, 1u)] = (uint32_t)(4 * j + t);
+        }
+        __syncwarp();
+        // every entry asks its bin for the next slot
+        for (uint32_t e = lane; e < n_band; e += 32) {
+            const uint32_t j = queue[e];
+            const float f = __uint_as_float(vs[j]);
+            uint32_t slot, tag = 0; // tags grow with the bins; at finer levels tag 0 is what lies below the interval
+            if (f < lo) {
+                slot = atomicAdd(&n_low, 1u);
+            } else {
+                const int bin = bin_of(f);
+                slot = atomicAdd(&hist[bin], 1u);
+                tag = level == 0 ? (uint32_t)bin : (uint32_t)(bin >> 1) + 1u;
+            }
+            out[slot] = band_entry(order_key(f), tag, j);
+        }
+        if (lane == 0) band_n[(size_t)b * P + i] = (int32_t)n_band;
+        return;
+    }
+    // the exact route: C entries (C <= stride by the host's choice of stride), equal keys in index order, one tag
+    auto key_of = [&](int j) { return vs[j] == kNotAToken ? 0xffffffffu : min(order_key(__uint_as_float(vs[j])), 0xfffffffeu); };
+    const uint32_t T = warp_kth_key(
+        [&](uint32_t t) {
+            uint32_t n = 0;
+            for (int j = lane; j < n_vis; j += 32) n += key_of(j) < t ? 1u : 0u;
+            return n;
+        },
+        C);
+    uint32_t below = 0;
+    for (int j = lane; j < n_vis; j += 32) below += key_of(j) < T ? 1u : 0u;
+    const uint32_t need_eq = C - __reduce_add_sync(0xffffffffu, below);
+    uint32_t eq_seen = 0, n_out = 0;
+    for (int j0 = 0; j0 < n_vis; j0 += 32) {
+        const int j = j0 + lane;
+        const uint32_t key = j < n_vis ? key_of(j) : 0xffffffffu;
+        const bool eq = j < n_vis && key == T;
+        const uint32_t beq = __ballot_sync(0xffffffffu, eq);
+        const bool in = j < n_vis && (key < T || (eq && eq_seen + __popc(beq & lt) < need_eq));
+        const uint32_t bal = __ballot_sync(0xffffffffu, in);
+        if (in) out[n_out + __popc(bal & lt)] = band_entry(key, 0u, (uint32_t)j);
+        n_out += __popc(bal);
+        eq_seen += __popc(beq);
+    }
+    if (lane == 0) band_n[(size_t)b * P + i] = (int32_t)n_out;
+}
+
+__global__ void __launch_bounds__(kPickThreads)
+retain_pick_kernel(const int32_t *__restrict__ pivot_idx, const unsigned long long *__restrict__ band,
+                   const int32_t *__restrict__ band_n, int stride, const int64_t *__restrict__ pos_in, int S, int vis_offset,
+                   int n_vis, int P, int n_keep, int32_t *__restrict__ out_idx, int64_t *__restrict__ out_pos,
+                   uint8_t *__restrict__ keep_out, int32_t *__restrict__ owner_out, float *__restrict__ eps_out,
+                   const int *__restrict__ status)
+{
+    extern __shared__ __align__(16) uint8_t keep[]; // [n_vis] flags, the bands' lengths, two buffers of staged bands
+    int32_t *len = reinterpret_cast<int32_t *>(keep + ((size_t)n_vis + 15) / 16 * 16);                                  // [P]
+    unsigned long long *stage = reinterpret_cast<unsigned long long *>(reinterpret_cast<uint8_t *>(len) + ((size_t)P * 4 + 15) / 16 * 16); // [2][kPickStageEntries]
+    __shared__ uint32_t warp_tot[kPickThreads / 32];
+    if (*status != 0) return;
+    const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t lt = (1u << lane) - 1u;
+    const int S_out = S - n_vis + n_keep;
+    int32_t *owner = owner_out ? owner_out + (size_t)b * n_vis : nullptr;
+    for (int j = threadIdx.x; j < n_vis; j += blockDim.x) {
+        keep[j] = 0;
+        if (owner) owner[j] = -1;
+    }
+    for (int i = threadIdx.x; i < P; i += blockDim.x) len[i] = band_n[(size_t)b * P + i];
+    __syncthreads();
+    const int Pv = mark_pivots(pivot_idx + (size_t)b * P, P, n_vis, keep, owner, &warp_tot[0]);
+    const int q = (n_keep - Pv) / P, r = (n_keep - Pv) % P;
+    const int n_active = q > 0 ? P : r; // pivots with a quota (all later ones keep nothing)
+    if (eps_out)
+        for (int i = n_active + threadIdx.x; i < P; i += blockDim.x) eps_out[(size_t)b * P + i] = __int_as_float(0x7fc00000);
+    // Rounds: the bands of as many pivots as fit one buffer; while warp 0 takes the turns of one round's pivots in
+    // rank order, the next round's bands arrive in the other buffer.
+    auto round_end = [&](int i0) { // the pivots [i0, i1) of the round that starts at i0 (every thread computes the same)
+        int i1 = i0, total = 0;
+        while (i1 < n_active && (i1 == i0 || total + len[i1] <= kPickStageEntries)) total += len[i1++];
+        return i1;
+    };
+    auto fetch = [&](int i0, int i1, unsigned long long *buf) {
+        for (int i = i0, off = 0; i < i1; off += len[i], ++i) {
+            const unsigned long long *src = band + ((size_t)b * P + i) * stride;
+            for (int t = threadIdx.x; t < len[i]; t += blockDim.x) copy_async<8>(buf + off + t, src + t);
+        }
+        copy_async_commit();
+    };
+    int i0 = 0, i1 = round_end(0);
+    fetch(i0, i1, stage);
+    for (int round = 0; i0 < n_active; ++round) {
+        unsigned long long *buf = stage + (size_t)(round & 1) * kPickStageEntries;
+        const int i2 = round_end(i1);
+        fetch(i1, i2, stage + (size_t)((round + 1) & 1) * kPickStageEntries); // (an empty group after the last round)
+        copy_async_wait<1>();                                                 // this round's bands have arrived
+        __syncthreads();
+        if (warp == 0) {
+            for (int i = i0, off = 0; i < i1; off += len[i], ++i) {
+                unsigned long long *L = buf + off;
+                const int n = len[i], qi = q + (i < r ? 1 : 0);
+                // the free entries to the front (an entry moves towards the front only), bin after bin, until the bin
+                // that holds the qi-th free entry (its tag: tq) has been passed
+                int F = 0, tq = -1;
+                bool passed = false;
+                for (int t0 = 0; t0 < n && !passed; t0 += 32 * kPickAhead) {
+                    // kPickAhead chunks of 32 entries and their flags are read before the first is looked at (entries move
+                    // to places before t0 only, and no flag changes here)
+                    unsigned long long ent[kPickAhead];
+                    bool fr[kPickAhead];
+#pragma unroll
+                    for (int u = 0; u < kPickAhead; ++u) ent[u] = t0 + 32 * u + lane < n ? L[t0 + 32 * u + lane] : ~0ull;
+#pragma unroll
+                    for (int u = 0; u < kPickAhead; ++u) fr[u] = ent[u] != ~0ull && !keep[entry_index(ent[u])];
+#pragma unroll
+                    for (int u = 0; u < kPickAhead; ++u) {
+                        if (passed || t0 + 32 * u >= n) break;
+                        const bool valid = ent[u] != ~0ull;
+                        const int tag = (int)entry_tag(ent[u]);
+                        bool free = fr[u] && (tq < 0 || tag <= tq);
+                        uint32_t bal = __ballot_sync(0xffffffffu, free);
+                        if (tq < 0 && F + __popc(bal) >= qi) { // the qi-th free entry is in this chunk
+                            const uint32_t it = __ballot_sync(0xffffffffu, free && F + (int)__popc(bal & lt) == qi - 1);
+                            tq = __shfl_sync(0xffffffffu, tag, __ffs(it) - 1);
+                            free = free && tag <= tq;
+                            bal = __ballot_sync(0xffffffffu, free);
+                        }
+                        if (free) L[F + __popc(bal & lt)] = ent[u];
+                        F += __popc(bal);
+                        passed = tq >= 0 && __any_sync(0xffffffffu, valid && tag > tq);
+                    }
+                    __syncwarp();
+                }
+                // the free entries of the bins before tq are all taken (they stand first: the band is grouped by bin)
+                int sure = 0;
+                for (int e0 = 0; e0 < F; e0 += 32) {
+                    const bool mine = e0 + lane < F && (tq < 0 || (int)entry_tag(L[e0 + lane]) < tq);
+                    if (mine) {
+                        const uint32_t j = entry_index(L[e0 + lane]);
+                        keep[j] = 1;
+                        if (owner) owner[j] = i;
+                    }
+                    const uint32_t bal = __ballot_sync(0xffffffffu, mine);
+                    sure += __popc(bal);
+                    if (bal != 0xffffffffu) break;
+                }
+                // the rest of the quota from bin tq, L[sure .. F): the smallest remaining entry again and again
+                unsigned long long from = 0, best = 0;
+                for (int k = sure; k < qi && k < F; ++k) {
+                    unsigned long long m = ~0ull;
+                    for (int e = sure + lane; e < F; e += 32) {
+                        const unsigned long long v = L[e];
+                        if (v >= from && v < m) m = v;
+                    }
+                    const uint32_t hi = __reduce_min_sync(0xffffffffu, (uint32_t)(m >> 32));
+                    const uint32_t lo = __reduce_min_sync(0xffffffffu, (uint32_t)(m >> 32) == hi ? (uint32_t)m : 0xffffffffu);
+                    best = ((unsigned long long)hi << 32) | lo;
+                    from = best + 1;
+                    if (lane == 0) {
+                        keep[entry_index(best)] = 1;
+                        if (owner) owner[entry_index(best)] = i;
+                    }
+                }
+                if (F <= qi && F > 0) { // (fewer free entries than the quota cannot happen; the largest taken, for eps)
+                    unsigned long long m = 0;
+                    for (int e = lane; e < F; e += 32) m = L[e] > m ? L[e] : m;
+                    const uint32_t hi = __reduce_max_sync(0xffffffffu, (uint32_t)(m >> 32));
+                    best = (unsigned long long)hi << 32;
+                }
+                __syncwarp(); // the flags are visible to the next pivot's turn
+                if (eps_out && lane == 0)
+                    eps_out[(size_t)b * P + i] = F > 0 ? order_key_inv((uint32_t)(best >> 32)) : __int_as_float(0x7fc00000);
+            }
+        }
+        __syncthreads(); // the buffer may be filled again
+        i0 = i1;
+        i1 = i2;
+    }
+    copy_async_wait<0>();
+    pack_indices(keep, S, vis_offset, n_vis, n_keep, pos_in ? pos_in + (size_t)b * S : nullptr, out_idx + (size_t)b * S_out,
+                 out_pos + (size_t)b * S_out, warp_tot);
+    if (keep_out)
+        for (int j = threadIdx.x; j < n_vis; j += blockDim.x) keep_out[(size_t)b * n_vis + j] = keep[j];
+}
+
+// ------------------------------------------------------------------------------------------------
 // Steps 4 and 5a with ONE threshold for all pivots (Def. 2 / Eq. 8-9 read with a common eps): a token's
 // duplication is its highest dup to any pivot, u_j = max_i dup[i][j]; the n_keep - P non-pivot tokens of
 // lowest u_j are kept (radix select on order-preserving keys, ties to the lower index), eps = the largest

@@ -111,6 +111,80 @@ def test_both_forms_of_the_retention_agree(oracle, shape):
     assert rep.exact >= rep.above_margin
 
 
+def _band_inputs(kind, B, S, d, vo, nv, P, seed):
+    """Key rows that drive the band retention through each of its routes."""
+    k, h = gaussian(B, S, d, seed=seed)
+    g = torch.Generator(device="cuda").manual_seed(seed + 1)
+    v = torch.randn(d, generator=g, device="cuda")
+    vis = slice(vo, vo + nv)
+    if kind == "same pivots":
+        # the P rows of largest norm are copies of one direction: every pivot ranks the tokens alike, so each band is
+        # all but used up by the pivots before it
+        idx = vo + torch.randperm(nv, generator=g, device="cuda")[:P]
+        k[:, idx] = (3.0 * v + 0.01 * torch.randn(B, P, d, generator=g, device="cuda")).to(k.dtype)
+    elif kind == "equal tokens":
+        # all vision rows but the pivots are one and the same row: every dup of a row ties, no band fits its list and the
+        # index decides
+        k[:, vis] = k[:, vo:vo + 1].clone()
+        idx = vo + torch.randperm(nv, generator=g, device="cuda")[:P]
+        k[:, idx] = (2.0 * k[:, idx].float() + torch.randn(B, P, d, generator=g, device="cuda")).to(k.dtype)
+    elif kind == "stretched range":
+        # one token opposite to the pivots' direction and the rest packed within a sliver of the range: the first
+        # level of bins holds nearly all tokens in one bin
+        k[:, vis] = (v + 0.02 * torch.randn(B, nv, d, generator=g, device="cuda")).to(k.dtype)
+        k[:, vo + nv // 3] = (-v).to(k.dtype)
+        idx = vo + torch.randperm(nv, generator=g, device="cuda")[:P]
+        k[:, idx] = (3.0 * v + 0.3 * torch.randn(B, P, d, generator=g, device="cuda")).to(k.dtype)
+    elif kind == "lanes of large keys":
+        # tokens whose index mod 32 is 12 or more lie along the pivots' direction, the others are unrelated to it
+        j = torch.arange(nv, device="cuda")
+        along = vo + j[(j % 32) >= 12]
+        k[:, along] = (v + 0.05 * torch.randn(B, along.numel(), d, generator=g, device="cuda")).to(k.dtype)
+        idx = vo + (torch.randperm(nv // 32, generator=g, device="cuda")[:P] * 32 + 20)
+        k[:, idx] = (3.0 * v + 0.3 * torch.randn(B, P, d, generator=g, device="cuda")).to(k.dtype)
+    else:
+        assert kind == "gaussian"
+    return k, h
+
+
+BAND_CASES = [
+    # (kind, (B, S, d, vis_offset, n_vis, P, Kp))
+    ("gaussian", (3, 700, 64, 10, 640, 128, 640)),        # quotas of four
+    ("gaussian", (2, 1000, 64, 0, 900, 20, 600)),         # quotas of 29
+    ("gaussian", (2, 130, 64, 7, 101, 3, 40)),            # fewer tokens than bins; rows not a multiple of 16 bytes
+    ("gaussian", (2, 7000, 64, 0, 7000, 2, 6146)),        # the longest bands: 6144 tokens beside the pivots
+    ("gaussian", (2, 7000, 64, 0, 7000, 2, 6200)),        # more than that: the sorted lists or the one-kernel form run
+    ("gaussian", (2, 2000, 64, 0, 2000, 60, 1900)),       # bands of several rounds of staging
+    ("gaussian", (2, 3000, 128, 40, 2880, 32, 320)),      # a sweep cell's shape
+    ("gaussian", (2, 700, 64, 10, 640, 128, 130)),        # most pivots keep nothing beside themselves
+    ("same pivots", (2, 1100, 64, 20, 1000, 48, 300)),
+    ("same pivots", (2, 700, 64, 10, 640, 128, 640)),
+    ("equal tokens", (2, 700, 64, 10, 640, 16, 200)),
+    ("equal tokens", (1, 2100, 64, 10, 2000, 4, 1500)),
+    ("stretched range", (2, 1400, 64, 30, 1280, 16, 120)),
+    ("stretched range", (2, 3000, 64, 0, 2880, 8, 320)),
+    ("lanes of large keys", (2, 1400, 64, 30, 1280, 16, 120)),
+    ("lanes of large keys", (1, 1400, 64, 30, 1280, 8, 264)),
+]
+
+
+@pytest.mark.parametrize("kind,shape", BAND_CASES, ids=lambda v: v if isinstance(v, str) else "x".join(map(str, v)))
+def test_candidate_bands_make_the_same_selections(oracle, kind, shape):
+    """Unsorted candidate bands (the lowest histogram band of each pivot's dups that holds the tokens it could need)
+    against the one-kernel form, bitwise, and against the oracle: plain rows, pivots that rank the tokens alike, rows of
+    equal values (the exact route), rows whose range an outlier stretches (the finer levels of bins)."""
+    B, S, d, vo, nv, P, Kp = shape
+    k, h = _band_inputs(kind, B, S, d, vo, nv, P, seed=11 + sum(shape))
+    a = run_gpu(k, h, vo, nv, P, Kp, path=dart.DART_PATH_STAGED, retention=dart.DART_RETAIN_SERIAL)
+    b = run_gpu(k, h, vo, nv, P, Kp, path=dart.DART_PATH_STAGED, retention=dart.DART_RETAIN_BANDS)
+    assert all(np.array_equal(x, y) for x, y in zip(a[:3], b[:3]))
+    assert all(np.array_equal(a[3][n], b[3][n], equal_nan=(n == "eps")) for n in a[3])
+    kb, hb = W.bits(k), W.bits(h)
+    ora = oracle.reduce(hb, kb, vo, nv, P, Kp)
+    rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, b[0], b[1], b[2], dbg=b[3])
+    assert rep.exact >= rep.above_margin
+
+
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
 def test_keys_null_scores_the_hidden_states(oracle, path):
     _, h = gaussian(2, 120, 256, seed=7)
