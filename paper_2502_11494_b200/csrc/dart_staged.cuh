@@ -980,68 +980,123 @@ retain_pick_kernel(const int32_t *__restrict__ pivot_idx, const unsigned long lo
                 int F = 0, tq = -1;
                 bool passed = false;
                 for (int t0 = 0; t0 < n && !passed; t0 += 32 * kPickAhead) {
-                    // kPickAhead chunks of 32 entries and their flags are read before the first is looked at (entries move
-                    // to places before t0 only, and no flag changes here)
+                    // kPickAhead chunks of 32 entries and their flags are read, and the votes on them taken, before the
+                    // first is looked at (entries move to places before t0 only, and no flag changes here)
                     unsigned long long ent[kPickAhead];
                     bool fr[kPickAhead];
+                    uint32_t fb[kPickAhead];
 #pragma unroll
                     for (int u = 0; u < kPickAhead; ++u) ent[u] = t0 + 32 * u + lane < n ? L[t0 + 32 * u + lane] : ~0ull;
 #pragma unroll
                     for (int u = 0; u < kPickAhead; ++u) fr[u] = ent[u] != ~0ull && !keep[entry_index(ent[u])];
 #pragma unroll
-                    for (int u = 0; u < kPickAhead; ++u) {
-                        if (passed || t0 + 32 * u >= n) break;
-                        const bool valid = ent[u] != ~0ull;
-                        const int tag = (int)entry_tag(ent[u]);
-                        bool free = fr[u] && (tq < 0 || tag <= tq);
-                        uint32_t bal = __ballot_sync(0xffffffffu, free);
-                        if (tq < 0 && F + __popc(bal) >= qi) { // the qi-th free entry is in this chunk
-                            const uint32_t it = __ballot_sync(0xffffffffu, free && F + (int)__popc(bal & lt) == qi - 1);
-                            tq = __shfl_sync(0xffffffffu, tag, __ffs(it) - 1);
-                            free = free && tag <= tq;
-                            bal = __ballot_sync(0xffffffffu, free);
+                    for (int u = 0; u < kPickAhead; ++u) fb[u] = __ballot_sync(0xffffffffu, fr[u]);
+                    int u0 = 0; // the first chunk of the group that is filtered by tag
+                    if (tq < 0) {
+                        int hit = -1, run = F; // the chunk that holds the qi-th free entry, the free entries before that chunk
+#pragma unroll
+                        for (int u = 0; u < kPickAhead; ++u) {
+                            const int c = __popc(fb[u]);
+                            if (hit < 0 && run + c >= qi) hit = u;
+                            if (hit < 0) run += c;
                         }
-                        if (free) L[F + __popc(bal & lt)] = ent[u];
-                        F += __popc(bal);
-                        passed = tq >= 0 && __any_sync(0xffffffffu, valid && tag > tq);
+#pragma unroll
+                        for (int u = 0; u < kPickAhead; ++u)
+                            if (hit < 0 || u < hit) {
+                                if (fr[u]) L[F + __popc(fb[u] & lt)] = ent[u];
+                                F += __popc(fb[u]);
+                            }
+                        u0 = kPickAhead;
+#pragma unroll
+                        for (int u = 0; u < kPickAhead; ++u)
+                            if (u == hit) {
+                                const uint32_t it = __ballot_sync(0xffffffffu, fr[u] && F + (int)__popc(fb[u] & lt) == qi - 1);
+                                tq = __shfl_sync(0xffffffffu, (int)entry_tag(ent[u]), __ffs(it) - 1);
+                                u0 = u;
+                            }
+                    }
+                    if (tq >= 0) { // from chunk u0 on: entries up to tag tq only; the first chunk that reaches beyond it is the last
+                        uint32_t tb[kPickAhead], gb[kPickAhead];
+#pragma unroll
+                        for (int u = 0; u < kPickAhead; ++u) {
+                            const int tag = (int)entry_tag(ent[u]);
+                            tb[u] = __ballot_sync(0xffffffffu, fr[u] && tag <= tq);
+                            gb[u] = __ballot_sync(0xffffffffu, ent[u] != ~0ull && tag > tq);
+                        }
+#pragma unroll
+                        for (int u = 0; u < kPickAhead; ++u)
+                            if (u >= u0 && !passed) {
+                                if (fr[u] && (int)entry_tag(ent[u]) <= tq) L[F + __popc(tb[u] & lt)] = ent[u];
+                                F += __popc(tb[u]);
+                                passed = gb[u] != 0u;
+                            }
                     }
                     __syncwarp();
                 }
-                // the free entries of the bins before tq are all taken (they stand first: the band is grouped by bin)
-                int sure = 0;
-                for (int e0 = 0; e0 < F; e0 += 32) {
-                    const bool mine = e0 + lane < F && (tq < 0 || (int)entry_tag(L[e0 + lane]) < tq);
-                    if (mine) {
-                        const uint32_t j = entry_index(L[e0 + lane]);
-                        keep[j] = 1;
-                        if (owner) owner[j] = i;
+                unsigned long long best = 0;
+                if (F <= 32) {
+                    // (the usual case) one entry per lane: those of the bins before tq are all taken, and the rest of the
+                    // quota from bin tq, the smallest remaining entry again and again
+                    const bool mine = lane < F;
+                    const unsigned long long v = mine ? L[lane] : ~0ull;
+                    const bool early = mine && (tq < 0 || (int)entry_tag(v) < tq);
+                    const int sure = __popc(__ballot_sync(0xffffffffu, early));
+                    const int need = (qi < F ? qi : F) - sure;
+                    bool take = early;
+                    if (need >= F - sure) {
+                        take = mine;
+                    } else {
+                        unsigned long long m = mine && !early ? v : ~0ull;
+                        for (int k = 0; k < need; ++k) {
+                            const uint32_t hi = __reduce_min_sync(0xffffffffu, (uint32_t)(m >> 32));
+                            const uint32_t lo = __reduce_min_sync(0xffffffffu, (uint32_t)(m >> 32) == hi ? (uint32_t)m : 0xffffffffu);
+                            if (m == (((unsigned long long)hi << 32) | lo)) {
+                                take = true;
+                                m = ~0ull;
+                            }
+                        }
                     }
-                    const uint32_t bal = __ballot_sync(0xffffffffu, mine);
-                    sure += __popc(bal);
-                    if (bal != 0xffffffffu) break;
-                }
-                // the rest of the quota from bin tq, L[sure .. F): the smallest remaining entry again and again
-                unsigned long long from = 0, best = 0;
-                for (int k = sure; k < qi && k < F; ++k) {
-                    unsigned long long m = ~0ull;
-                    for (int e = sure + lane; e < F; e += 32) {
-                        const unsigned long long v = L[e];
-                        if (v >= from && v < m) m = v;
+                    if (take) {
+                        keep[entry_index(v)] = 1;
+                        if (owner) owner[entry_index(v)] = i;
                     }
-                    const uint32_t hi = __reduce_min_sync(0xffffffffu, (uint32_t)(m >> 32));
-                    const uint32_t lo = __reduce_min_sync(0xffffffffu, (uint32_t)(m >> 32) == hi ? (uint32_t)m : 0xffffffffu);
-                    best = ((unsigned long long)hi << 32) | lo;
-                    from = best + 1;
-                    if (lane == 0) {
-                        keep[entry_index(best)] = 1;
-                        if (owner) owner[entry_index(best)] = i;
+                    best = (unsigned long long)__reduce_max_sync(0xffffffffu, take ? (uint32_t)(v >> 32) : 0u) << 32; // eps: the largest taken
+                } else {
+                    // the free entries of the bins before tq are all taken (they stand first: the band is grouped by bin)
+                    int sure = 0;
+                    for (int e0 = 0; e0 < F; e0 += 32) {
+                        const bool mine = e0 + lane < F && (tq < 0 || (int)entry_tag(L[e0 + lane]) < tq);
+                        if (mine) {
+                            const uint32_t j = entry_index(L[e0 + lane]);
+                            keep[j] = 1;
+                            if (owner) owner[j] = i;
+                        }
+                        const uint32_t bal = __ballot_sync(0xffffffffu, mine);
+                        sure += __popc(bal);
+                        if (bal != 0xffffffffu) break;
                     }
-                }
-                if (F <= qi && F > 0) { // (fewer free entries than the quota cannot happen; the largest taken, for eps)
-                    unsigned long long m = 0;
-                    for (int e = lane; e < F; e += 32) m = L[e] > m ? L[e] : m;
-                    const uint32_t hi = __reduce_max_sync(0xffffffffu, (uint32_t)(m >> 32));
-                    best = (unsigned long long)hi << 32;
+                    // the rest of the quota from bin tq, L[sure .. F): the smallest remaining entry again and again
+                    unsigned long long from = 0;
+                    for (int k = sure; k < qi && k < F; ++k) {
+                        unsigned long long m = ~0ull;
+                        for (int e = sure + lane; e < F; e += 32) {
+                            const unsigned long long v = L[e];
+                            if (v >= from && v < m) m = v;
+                        }
+                        const uint32_t hi = __reduce_min_sync(0xffffffffu, (uint32_t)(m >> 32));
+                        const uint32_t lo = __reduce_min_sync(0xffffffffu, (uint32_t)(m >> 32) == hi ? (uint32_t)m : 0xffffffffu);
+                        best = ((unsigned long long)hi << 32) | lo;
+                        from = best + 1;
+                        if (lane == 0) {
+                            keep[entry_index(best)] = 1;
+                            if (owner) owner[entry_index(best)] = i;
+                        }
+                    }
+                    if (F <= qi) { // (fewer free entries than the quota cannot happen; the largest taken, for eps)
+                        unsigned long long m = 0;
+                        for (int e = lane; e < F; e += 32) m = L[e] > m ? L[e] : m;
+                        best = (unsigned long long)__reduce_max_sync(0xffffffffu, (uint32_t)(m >> 32)) << 32;
+                    }
                 }
                 __syncwarp(); // the flags are visible to the next pivot's turn
                 if (eps_out && lane == 0)
