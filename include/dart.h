@@ -89,9 +89,8 @@ enum {
                                   tickets to the lower index.  The same seed gives the same pivots on every run. */
 
 /* dart_opts.retention */
-#define DART_RETAIN_AUTO 0   /* candidate bands when their workspace exists (always, unless the context's maxima would need
-                                more than 1 GiB of it); else two phases with sorted lists when the batch alone cannot fill
-                                the GPU, else one kernel */
+#define DART_RETAIN_AUTO 0   /* more samples than SMs: candidate bands; else sorted lists; where the chosen form's
+                                workspace or shared memory does not fit: the other one, else one kernel */
 #define DART_RETAIN_SERIAL 1 /* one kernel, one CTA per sample: the pivots' selections one after the other */
 #define DART_RETAIN_LISTS 2  /* two phases: sorted candidate lists for all (sample, pivot) pairs at once, then the pivots'
                                 turns as walks over the lists; needs n_keep - n_pivot <= 4096, else the one-kernel form runs */

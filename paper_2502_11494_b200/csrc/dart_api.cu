@@ -231,14 +231,19 @@ void launch_retention(dart_ctx *ctx, int B, const int64_t *pos_in, int vis_offse
         return;
     }
     const int m_pad = next_pow2(m > 1 ? m : 1);
-    const bool can_lists = ctx->cand && m <= ctx->cand_stride && m <= kCandMax &&
-                           candidates_smem_bytes(n_vis, m_pad) <= (size_t)ctx->max_smem_optin - 2048 &&
-                           walk_smem_bytes(n_vis) <= (size_t)ctx->max_smem_optin - 2048;
     // bands: a list must hold the m tokens of the exact route and fit one staging round of phase 2
     const int band_cap = ctx->band_stride < kPickStageEntries ? ctx->band_stride : kPickStageEntries;
     const bool can_bands = ctx->band && m > 0 && m <= band_cap && n_vis <= kBandMaxTokens && band_smem_bytes(n_vis, band_cap) <= (size_t)ctx->max_smem_optin - 2048 &&
                            pick_smem_bytes(n_vis, P) <= (size_t)ctx->max_smem_optin - 2048;
-    const bool bands = can_bands && (mode == DART_RETAIN_BANDS || mode == DART_RETAIN_AUTO);
+    // Which form: all do the same selections.  One kernel per sample takes B CTAs through P selections each; sorted
+    // lists spread the selections over B * P CTAs, which pays while B CTAs cannot fill the SMs (measured: batch 4-64 up
+    // to 4x faster than one kernel); bands need one warp per selection and no sort, which pays once the batch fills the
+    // GPU (measured at batch 256: 8 pivots 93 -> 56 us, 32 pivots 0.36 -> 0.16 ms, 128 pivots 1.38 -> 0.49 ms), while for
+    // a few samples their turns, one warp per sample, take longer than the sorted lists' walks.
+    const bool can_lists = ctx->cand && m <= ctx->cand_stride && m <= kCandMax &&
+                               candidates_smem_bytes(n_vis, m_pad) <= (size_t)ctx->max_smem_optin - 2048 &&
+                               walk_smem_bytes(n_vis) <= (size_t)ctx->max_smem_optin - 2048;
+    const bool bands = can_bands && (mode == DART_RETAIN_BANDS || (mode == DART_RETAIN_AUTO && (B > ctx->sm_count || !can_lists)));
     if (bands) {
         {
             Prof p(ctx, st, SLOT_RETAIN);
@@ -251,8 +256,6 @@ void launch_retention(dart_ctx *ctx, int B, const int64_t *pos_in, int vis_offse
             ctx->owner, ctx->eps, ctx->status);
         return;
     }
-    // Both forms do the same selections; the lists spread them over B * P CTAs instead of B, which pays while B
-    // CTAs cannot fill the SMs (measured: batch 4-64 up to 4x faster, batch 256 at 8 pivots 20 % slower).
     const bool two_phase = can_lists && (mode == DART_RETAIN_LISTS || (mode == DART_RETAIN_AUTO && B <= ctx->sm_count));
     if (!two_phase) {
         Prof p(ctx, st, SLOT_RETAIN);
