@@ -250,7 +250,7 @@ TEXT_SHAPES = [
 
 
 @pytest.mark.parametrize("path", [dart.DART_PATH_AUTO, dart.DART_PATH_FUSED, dart.DART_PATH_STAGED], ids=lambda p: PATH_IDS.get(p, "auto"))
-@pytest.mark.parametrize("retention", [dart.DART_RETAIN_SERIAL, dart.DART_RETAIN_LISTS], ids=["serial", "lists"])
+@pytest.mark.parametrize("retention", [dart.DART_RETAIN_SERIAL, dart.DART_RETAIN_LISTS, dart.DART_RETAIN_BANDS], ids=["serial", "lists", "bands"])
 @pytest.mark.parametrize("shape", TEXT_SHAPES, ids=lambda s: "x".join(map(str, s)))
 def test_pivots_from_the_text_tokens(oracle, shape, retention, path):
     B, S, d, vo, nv, P, Kp = shape
@@ -453,7 +453,7 @@ def test_text_pivots_random_shapes(oracle, seed):
     try:
         piv_t = torch.from_numpy(piv).cuda()
         res = ctx.reduce(h, k, vo, nv, P, Kp, debug=True,
-                         opts=dart.dart_opts(retention=int(rng.integers(0, 3)), text_pivots=1, pivots_in=piv_t.data_ptr()))
+                         opts=dart.dart_opts(retention=int(rng.integers(0, 4)), text_pivots=1, pivots_in=piv_t.data_ptr()))
         torch.cuda.synchronize()
         assert ctx.status() == dart.DART_OK, dart.dart_status_detail(ctx.handle)
     finally:
