@@ -44,7 +44,7 @@ def parse():
     ap.add_argument("--tune", type=int, default=0, help="path 6: 16 * n1 + n2 ring depths")
     ap.add_argument("--split", type=int, default=0, help="path 5: k keeps tiles with index %% k == 0 on the chip, -k all others")
     ap.add_argument("--lag", type=int, default=0, help="fused path: extra tasks between a row's two sweeps")
-    ap.add_argument("--retention", type=int, default=0, help="0 auto, 1 one kernel, 2 candidate lists + walks")
+    ap.add_argument("--retention", type=int, default=0, help="0 auto, 1 one kernel, 2 sorted lists + walks, 3 bands + turns, 4 bands and turns in one launch")
     ap.add_argument("--variants", action="store_true",
                     help="also time the variants: one threshold for all pivots, pivots given by the caller, KV-row gather")
     ap.add_argument("--no-e2e", action="store_true")

@@ -89,8 +89,9 @@ enum {
                                   tickets to the lower index.  The same seed gives the same pivots on every run. */
 
 /* dart_opts.retention */
-#define DART_RETAIN_AUTO 0   /* more samples than SMs: candidate bands; else sorted lists; where the chosen form's
-                                workspace or shared memory does not fit: the other one, else one kernel */
+#define DART_RETAIN_AUTO 0   /* more samples than SMs: candidate bands; else the bands in one launch for up to 8 pivots
+                                and sorted lists for more; where the chosen form's workspace or shared memory does not
+                                fit: another one, else one kernel */
 #define DART_RETAIN_SERIAL 1 /* one kernel, one CTA per sample: the pivots' selections one after the other */
 #define DART_RETAIN_LISTS 2  /* two phases: sorted candidate lists for all (sample, pivot) pairs at once, then the pivots'
                                 turns as walks over the lists; needs n_keep - n_pivot <= 4096, else the one-kernel form runs */
@@ -98,6 +99,10 @@ enum {
                                 pivot's dups that holds at least the tokens the pivot could need; then the pivots' turns,
                                 each taking its quota's smallest free entries of its band.  Needs n_keep - n_pivot <= 6144,
                                 else as without it. */
+
+#define DART_RETAIN_FUSED 4  /* the bands' two phases in one launch, one CTA per sample (a few warps build the sample's
+                                bands, then the CTA takes the turns): for batches that cannot fill the GPU.  Same limits as
+                                DART_RETAIN_BANDS, else as without it. */
 
 /* dart_opts.rule */
 #define DART_RULE_QUOTAS 0 /* one threshold per pivot: pivot i keeps its q_i not-yet-kept tokens of lowest dup (dart_reduce) */

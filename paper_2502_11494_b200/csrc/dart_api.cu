@@ -243,6 +243,20 @@ void launch_retention(dart_ctx *ctx, int B, const int64_t *pos_in, int vis_offse
     const bool can_lists = ctx->cand && m <= ctx->cand_stride && m <= kCandMax &&
                                candidates_smem_bytes(n_vis, m_pad) <= (size_t)ctx->max_smem_optin - 2048 &&
                                walk_smem_bytes(n_vis) <= (size_t)ctx->max_smem_optin - 2048;
+    // ... and both phases of the bands in one launch for batches that cannot fill the GPU: as many band-building warps as
+    // shared memory takes beside the flags
+    int band_warps = P < kPickThreads / 32 ? P : kPickThreads / 32;
+    while (band_warps > 1 && retain_fused_smem_bytes(n_vis, P, band_cap, band_warps) > (size_t)ctx->max_smem_optin - 2048) --band_warps;
+    const bool can_fused = can_bands && retain_fused_smem_bytes(n_vis, P, band_cap, band_warps) <= (size_t)ctx->max_smem_optin - 2048;
+    // (measured, us: one sample of 576 tokens 23 -> 20, 64 samples 29 -> 23 against the sorted lists; with more pivots than
+    // band-building warps the lists stay ahead: 16 pivots, 8 samples of 2880 tokens 45 vs 55; 32 pivots, 4 samples 66 vs 123)
+    if (can_fused && (mode == DART_RETAIN_FUSED || (mode == DART_RETAIN_AUTO && B <= ctx->sm_count && P <= band_warps))) {
+        Prof p(ctx, st, SLOT_RETAIN);
+        retain_fused_kernel<<<B, kPickThreads, retain_fused_smem_bytes(n_vis, P, band_cap, band_warps), st>>>(
+            ctx->sim, ctx->pivot_idx, ctx->band, ctx->band_n, band_cap, pos_in, S, vis_offset, n_vis, P, n_keep, out_idx, out_pos,
+            ctx->keep, ctx->owner, ctx->eps, ctx->status, band_warps);
+        return;
+    }
     const bool bands = can_bands && (mode == DART_RETAIN_BANDS || (mode == DART_RETAIN_AUTO && (B > ctx->sm_count || !can_lists)));
     if (bands) {
         {
@@ -914,6 +928,8 @@ int dart_create(dart_ctx **out, const dart_desc *desc)
         if (cudaFuncSetAttribute(dart::band_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  ctx->max_smem_optin - 2048) != cudaSuccess ||
             cudaFuncSetAttribute(dart::retain_pick_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 ctx->max_smem_optin - 2048) != cudaSuccess ||
+            cudaFuncSetAttribute(dart::retain_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  ctx->max_smem_optin - 2048) != cudaSuccess)
             rc = DART_ERR_CUDA;
     }
@@ -1038,7 +1054,7 @@ int dart_reduce_ex(dart_ctx *ctx, const void *hidden, const void *keys, const in
         dart::retain_global_smem_bytes(n_vis) > (size_t)ctx->max_smem_optin - 2048)
         return DART_ERR_UNSUPPORTED; // the sample's duplication values must fit shared memory
     if (o.retention != DART_RETAIN_AUTO && o.retention != DART_RETAIN_SERIAL && o.retention != DART_RETAIN_LISTS &&
-        o.retention != DART_RETAIN_BANDS)
+        o.retention != DART_RETAIN_BANDS && o.retention != DART_RETAIN_FUSED)
         return DART_ERR_UNSUPPORTED;
     if ((uintptr_t)pos_in & 7u) return DART_ERR_ALIGN;
     DeviceGuard g(ctx->desc.device);

@@ -686,7 +686,7 @@ constexpr int kPickThreads = 256;
 constexpr int kPickStageEntries = 6144; // 48 KB of staged entries per buffer of phase 2
 constexpr int kPickAhead = 4;           // chunks of 32 entries read ahead in phase 2
 inline int band_stride(int m) { return (m + m / 4 + 64 + 1) & ~1; } // entries per list for up to m tokens beside the pivots
-inline size_t band_smem_bytes(int n_vis, int stride) { return ((size_t)n_vis * 4 + 15) / 16 * 16 + (size_t)stride * 4; }
+__host__ __device__ inline size_t band_smem_bytes(int n_vis, int stride) { return ((size_t)n_vis * 4 + 15) / 16 * 16 + (size_t)stride * 4; }
 inline size_t pick_smem_bytes(int n_vis, int P)
 {
     return ((size_t)n_vis + 15) / 16 * 16 + ((size_t)P * 4 + 15) / 16 * 16 + (size_t)2 * kPickStageEntries * 8;
@@ -722,20 +722,21 @@ __device__ __forceinline__ uint32_t warp_kth_key(CountFn count_below, uint32_t k
     return v;
 }
 
-__global__ void __launch_bounds__(32)
-band_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx, int n_vis, int P, int n_keep, int stride,
-            unsigned long long *__restrict__ band, int32_t *__restrict__ band_n, const int *__restrict__ status)
+// Phase 1 for one row, by one warp: the band of pivot i of a sample (row = its dups, piv = the sample's pivots) into
+// out[0 .. *out_n).  vs: the warp's shared memory, n_vis rounded up to 4 words for the row + `stride` words for the queue.
+struct BandScratch {
+    uint32_t hist[kBandBins]; // the bins' counts, then their offsets in the list
+    uint32_t n_low;           // entries below the interval of a finer level handed out so far
+    uint32_t n_queued;        // the band's tokens found so far
+    uint32_t pad[2];
+};
+__device__ void band_of_row(const float *__restrict__ row, const int32_t *__restrict__ piv, int i, int n_vis, int P, int n_keep,
+                            int stride, uint32_t *vs, BandScratch &sc, unsigned long long *__restrict__ out,
+                            int32_t *__restrict__ out_n)
 {
-    extern __shared__ __align__(16) uint8_t band_smem[];
-    uint32_t *vs = reinterpret_cast<uint32_t *>(band_smem); // [n_vis rounded up to 4] the row's dups as bit patterns
-    __shared__ uint32_t hist[kBandBins];                    // the bins' counts, then their offsets in the list
-    __shared__ uint32_t n_low;                              // entries below the interval of a finer level handed out so far
-    __shared__ uint32_t n_queued;                           // the band's tokens found so far
-    if (*status != 0) return; // an earlier kernel of this call failed: its outputs are undefined
-    const int i = blockIdx.x, b = blockIdx.y, lane = threadIdx.x;
+    const int lane = threadIdx.x & 31;
     const uint32_t lt = (1u << lane) - 1u;
     constexpr uint32_t kNotAToken = 0xffffffffu; // a pivot, or the filler behind the row: a NaN no arithmetic produces
-    const float *row = sim + ((size_t)b * P + i) * n_vis;
     const int n4 = (n_vis + 3) / 4; // groups of four values
     const bool aligned = (n_vis & 3) == 0; // rows start on 16-byte boundaries
     if (aligned) { // the whole row is on its way before anything else is looked at
@@ -745,7 +746,6 @@ band_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx
 #pragma unroll 8
         for (int j = lane; j < n4 * 4; j += 32) vs[j] = __float_as_uint(__ldcs(row + (j < n_vis ? j : 0))); // (filler: a value of the row)
     }
-    const int32_t *piv = pivot_idx + (size_t)b * P;
     uint32_t mine = 0;
     for (int t = lane; t < P; t += 32) mine += (piv[t] >= 0 && piv[t] < n_vis) ? 1u : 0u;
     const int Pv = (int)__reduce_add_sync(0xffffffffu, mine);
@@ -753,7 +753,7 @@ band_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx
     copy_async_wait<0>();
     __syncwarp();
     if (q + (i < r ? 1 : 0) == 0) { // this pivot keeps nothing
-        if (lane == 0) band_n[(size_t)b * P + i] = 0;
+        if (lane == 0) *out_n = 0;
         return;
     }
     const uint32_t C = (uint32_t)quota_prefix(i, q, r);
@@ -774,7 +774,7 @@ band_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx
     for (int t = lane; t < P; t += 32)
         if (piv[t] >= 0 && piv[t] < n_vis) vs[piv[t]] = kNotAToken;
     if (lane < n4 * 4 - n_vis) vs[n_vis + lane] = kNotAToken;
-    if (lane == 0) n_queued = 0;
+    if (lane == 0) sc.n_queued = 0;
     __syncwarp();
     // The band: every value below lo, and the values of [lo, hi] whose bin is at most last_bin.  A level lays its bins
     // over the smallest and largest value of the interval it looks at; while the band is too long for the list the
@@ -791,7 +791,7 @@ band_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx
     auto bin_of = [&](float f) { return min((int)((f - lo) * scale), kBandBins - 1); }; // for lo <= f <= hi: not negative, monotone
     uint32_t c[kBandBins / 32];
     while (!exact) {
-        for (int t = lane; t < kBandBins; t += 32) hist[t] = 0;
+        for (int t = lane; t < kBandBins; t += 32) sc.hist[t] = 0;
         __syncwarp();
 #pragma unroll 2
         for (int j = lane; j < n4; j += 32) {
@@ -799,7 +799,7 @@ band_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx
             const float f[4] = {__uint_as_float(v.x), __uint_as_float(v.y), __uint_as_float(v.z), __uint_as_float(v.w)};
 #pragma unroll
             for (int t = 0; t < 4; ++t)
-                if (f[t] >= lo && f[t] <= hi) atomicAdd(&hist[bin_of(f[t])], 1u);
+                if (f[t] >= lo && f[t] <= hi) atomicAdd(&sc.hist[bin_of(f[t])], 1u);
         }
         __syncwarp();
         // lane l owns bins [8l, 8l + 8): the first bin at which the running count reaches the rest of C, and the counts there
@@ -807,7 +807,7 @@ band_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx
         uint32_t sum = 0;
 #pragma unroll
         for (int t = 0; t < kBandBins / 32; ++t) {
-            c[t] = hist[lane * (kBandBins / 32) + t];
+            c[t] = sc.hist[lane * (kBandBins / 32) + t];
             sum += c[t];
         }
         uint32_t incl = sum;
@@ -857,16 +857,15 @@ band_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx
         scale = (float)kBandBins / (n_hi - n_lo);
         exact = ++level == kBandLevels || !(n_hi > n_lo) || !(scale < 3.0e38f);
     }
-    unsigned long long *out = band + ((size_t)b * P + i) * stride;
     if (!exact) {
         // the bins' offsets
         __syncwarp();
 #pragma unroll
         for (int t = 0; t < kBandBins / 32; ++t) {
-            hist[lane * (kBandBins / 32) + t] = my_off;
+            sc.hist[lane * (kBandBins / 32) + t] = my_off;
             my_off += c[t];
         }
-        if (lane == 0) n_low = 0;
+        if (lane == 0) sc.n_low = 0;
         // the band's tokens: few of the row's, so they are queued first and then handled with all lanes busy
         const float edge = last_bin == kBandBins - 1 ? 3.0e38f : (float)(last_bin + 1); // bin <= last_bin <=> place < edge
 #pragma unroll 2
@@ -875,7 +874,7 @@ band_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx
             const float f[4] = {__uint_as_float(v.x), __uint_as_float(v.y), __uint_as_float(v.z), __uint_as_float(v.w)};
 #pragma unroll
             for (int t = 0; t < 4; ++t)
-                if ((f[t] - lo) * scale < edge && f[t] <= hi) queue[atomicAdd(&n_queued, 1u)] = (uint32_t)(4 * j + t);
+                if ((f[t] - lo) * scale < edge && f[t] <= hi) queue[atomicAdd(&sc.n_queued, 1u)] = (uint32_t)(4 * j + t);
         }
         __syncwarp();
         // every entry asks its bin for the next slot
@@ -884,15 +883,15 @@ band_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx
             const float f = __uint_as_float(vs[j]);
             uint32_t slot, tag = 0; // tags grow with the bins; at finer levels tag 0 is what lies below the interval
             if (f < lo) {
-                slot = atomicAdd(&n_low, 1u);
+                slot = atomicAdd(&sc.n_low, 1u);
             } else {
                 const int bin = bin_of(f);
-                slot = atomicAdd(&hist[bin], 1u);
+                slot = atomicAdd(&sc.hist[bin], 1u);
                 tag = level == 0 ? (uint32_t)bin : (uint32_t)(bin >> 1) + 1u;
             }
             out[slot] = band_entry(order_key(f), tag, j);
         }
-        if (lane == 0) band_n[(size_t)b * P + i] = (int32_t)n_band;
+        if (lane == 0) *out_n = (int32_t)n_band;
         return;
     }
     // the exact route: C entries (C <= stride by the host's choice of stride), equal keys in index order, one tag
@@ -919,22 +918,30 @@ band_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx
         n_out += __popc(bal);
         eq_seen += __popc(beq);
     }
-    if (lane == 0) band_n[(size_t)b * P + i] = (int32_t)n_out;
+    if (lane == 0) *out_n = (int32_t)n_out;
 }
 
-__global__ void __launch_bounds__(kPickThreads)
-retain_pick_kernel(const int32_t *__restrict__ pivot_idx, const unsigned long long *__restrict__ band,
-                   const int32_t *__restrict__ band_n, int stride, const int64_t *__restrict__ pos_in, int S, int vis_offset,
-                   int n_vis, int P, int n_keep, int32_t *__restrict__ out_idx, int64_t *__restrict__ out_pos,
-                   uint8_t *__restrict__ keep_out, int32_t *__restrict__ owner_out, float *__restrict__ eps_out,
-                   const int *__restrict__ status)
+__global__ void __launch_bounds__(32)
+band_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx, int n_vis, int P, int n_keep, int stride,
+            unsigned long long *__restrict__ band, int32_t *__restrict__ band_n, const int *__restrict__ status)
 {
-    extern __shared__ __align__(16) uint8_t keep[]; // [n_vis] flags, the bands' lengths, two buffers of staged bands
-    int32_t *len = reinterpret_cast<int32_t *>(keep + ((size_t)n_vis + 15) / 16 * 16);                                  // [P]
-    unsigned long long *stage = reinterpret_cast<unsigned long long *>(reinterpret_cast<uint8_t *>(len) + ((size_t)P * 4 + 15) / 16 * 16); // [2][kPickStageEntries]
-    __shared__ uint32_t warp_tot[kPickThreads / 32];
-    if (*status != 0) return;
-    const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    extern __shared__ __align__(16) uint8_t band_smem[];
+    __shared__ BandScratch sc;
+    if (*status != 0) return; // an earlier kernel of this call failed: its outputs are undefined
+    const int i = blockIdx.x, b = blockIdx.y;
+    band_of_row(sim + ((size_t)b * P + i) * n_vis, pivot_idx + (size_t)b * P, i, n_vis, P, n_keep, stride,
+                reinterpret_cast<uint32_t *>(band_smem), sc, band + ((size_t)b * P + i) * stride, band_n + (size_t)b * P + i);
+}
+
+// Phase 2 for one sample, by a CTA of kPickThreads threads.  keep: [n_vis] flags; len: [P]; stage: two buffers of
+// kPickStageEntries entries; warp_tot: one word per warp.
+__device__ void pick_sample(const int b, const int32_t *__restrict__ pivot_idx, const unsigned long long *__restrict__ band,
+                            const int32_t *__restrict__ band_n, int stride, const int64_t *__restrict__ pos_in, int S, int vis_offset,
+                            int n_vis, int P, int n_keep, int32_t *__restrict__ out_idx, int64_t *__restrict__ out_pos,
+                            uint8_t *__restrict__ keep_out, int32_t *__restrict__ owner_out, float *__restrict__ eps_out,
+                            uint8_t *keep, int32_t *len, unsigned long long *stage, uint32_t *warp_tot)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t lt = (1u << lane) - 1u;
     const int S_out = S - n_vis + n_keep;
     int32_t *owner = owner_out ? owner_out + (size_t)b * n_vis : nullptr;
@@ -1112,6 +1119,60 @@ retain_pick_kernel(const int32_t *__restrict__ pivot_idx, const unsigned long lo
                  out_pos + (size_t)b * S_out, warp_tot);
     if (keep_out)
         for (int j = threadIdx.x; j < n_vis; j += blockDim.x) keep_out[(size_t)b * n_vis + j] = keep[j];
+}
+
+__global__ void __launch_bounds__(kPickThreads)
+retain_pick_kernel(const int32_t *__restrict__ pivot_idx, const unsigned long long *__restrict__ band,
+                   const int32_t *__restrict__ band_n, int stride, const int64_t *__restrict__ pos_in, int S, int vis_offset,
+                   int n_vis, int P, int n_keep, int32_t *__restrict__ out_idx, int64_t *__restrict__ out_pos,
+                   uint8_t *__restrict__ keep_out, int32_t *__restrict__ owner_out, float *__restrict__ eps_out,
+                   const int *__restrict__ status)
+{
+    extern __shared__ __align__(16) uint8_t keep[]; // [n_vis] flags, the bands' lengths, two buffers of staged bands
+    int32_t *len = reinterpret_cast<int32_t *>(keep + ((size_t)n_vis + 15) / 16 * 16);                                  // [P]
+    unsigned long long *stage = reinterpret_cast<unsigned long long *>(reinterpret_cast<uint8_t *>(len) + ((size_t)P * 4 + 15) / 16 * 16); // [2][kPickStageEntries]
+    __shared__ uint32_t warp_tot[kPickThreads / 32];
+    if (*status != 0) return;
+    pick_sample(blockIdx.x, pivot_idx, band, band_n, stride, pos_in, S, vis_offset, n_vis, P, n_keep, out_idx, out_pos, keep_out,
+                owner_out, eps_out, keep, len, stage, warp_tot);
+}
+
+// Both phases in one launch, one CTA per sample, for batches that cannot fill the GPU anyway: band_warps warps build the
+// sample's bands, a pivot each at a time (through the same workspace in global memory: the CTA reads back what it wrote),
+// then the CTA takes the turns.  Dynamic shared memory: the flags and lengths of phase 2, then whichever is larger of
+// phase 2's two staging buffers and phase 1's band_warps x (row + queue + scratch).
+__host__ __device__ inline size_t fused_warp_bytes(int n_vis, int stride) { return band_smem_bytes(n_vis, stride) + sizeof(BandScratch); }
+inline size_t retain_fused_smem_bytes(int n_vis, int P, int stride, int band_warps)
+{
+    const size_t phase1 = (size_t)band_warps * ((fused_warp_bytes(n_vis, stride) + 15) / 16 * 16);
+    const size_t phase2 = (size_t)2 * kPickStageEntries * 8;
+    return ((size_t)n_vis + 15) / 16 * 16 + ((size_t)P * 4 + 15) / 16 * 16 + (phase1 > phase2 ? phase1 : phase2);
+}
+__global__ void __launch_bounds__(kPickThreads)
+retain_fused_kernel(const float *__restrict__ sim, const int32_t *__restrict__ pivot_idx, unsigned long long *__restrict__ band,
+                    int32_t *__restrict__ band_n, int stride, const int64_t *__restrict__ pos_in, int S, int vis_offset, int n_vis,
+                    int P, int n_keep, int32_t *__restrict__ out_idx, int64_t *__restrict__ out_pos, uint8_t *__restrict__ keep_out,
+                    int32_t *__restrict__ owner_out, float *__restrict__ eps_out, const int *__restrict__ status, int band_warps)
+{
+    extern __shared__ __align__(16) uint8_t keep[];
+    int32_t *len = reinterpret_cast<int32_t *>(keep + ((size_t)n_vis + 15) / 16 * 16);
+    uint8_t *work = reinterpret_cast<uint8_t *>(len) + ((size_t)P * 4 + 15) / 16 * 16;
+    __shared__ uint32_t warp_tot[kPickThreads / 32];
+    if (*status != 0) return;
+    const int b = blockIdx.x, warp = threadIdx.x >> 5;
+    if (warp < band_warps) {
+        const size_t per_warp = (fused_warp_bytes(n_vis, stride) + 15) / 16 * 16;
+        uint32_t *vs = reinterpret_cast<uint32_t *>(work + (size_t)warp * per_warp);
+        BandScratch &sc = *reinterpret_cast<BandScratch *>(work + (size_t)warp * per_warp + band_smem_bytes(n_vis, stride));
+        for (int i = warp; i < P; i += band_warps) {
+            band_of_row(sim + ((size_t)b * P + i) * n_vis, pivot_idx + (size_t)b * P, i, n_vis, P, n_keep, stride, vs, sc,
+                        band + ((size_t)b * P + i) * stride, band_n + (size_t)b * P + i);
+            __syncwarp(); // the row's buffer is free for the next one
+        }
+    }
+    __syncthreads(); // the bands are written; the work area changes hands
+    pick_sample(b, pivot_idx, band, band_n, stride, pos_in, S, vis_offset, n_vis, P, n_keep, out_idx, out_pos, keep_out, owner_out,
+                eps_out, keep, len, reinterpret_cast<unsigned long long *>(work), warp_tot);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -19,7 +19,7 @@ DART_ERR_NULL, DART_ERR_BAD_SHAPE, DART_ERR_ALIGN, DART_ERR_ALIAS = -1, -2, -3, 
 DART_ERR_CUDA, DART_ERR_NOMEM, DART_ERR_TIMEOUT, DART_ERR_CHECK, DART_ERR_UNSUPPORTED = -5, -6, -7, -8, -9
 DART_FLAG_HOST_STAGING = 1
 DART_PATH_AUTO, DART_PATH_STAGED, DART_PATH_FUSED, DART_PATH_TWO_PASS, DART_PATH_RESIDENT, DART_PATH_SPLIT, DART_PATH_PAIRED = 0, 1, 2, 3, 4, 5, 6
-DART_RETAIN_AUTO, DART_RETAIN_SERIAL, DART_RETAIN_LISTS, DART_RETAIN_BANDS = 0, 1, 2, 3
+DART_RETAIN_AUTO, DART_RETAIN_SERIAL, DART_RETAIN_LISTS, DART_RETAIN_BANDS, DART_RETAIN_FUSED = 0, 1, 2, 3, 4
 DART_RULE_QUOTAS, DART_RULE_GLOBAL, DART_RULE_UNION = 0, 1, 2
 DART_PIVOTS_BY_SCORE, DART_PIVOTS_MIXED, DART_PIVOTS_RANDOM = 0, 1, 2
 

@@ -24,7 +24,7 @@ def random_case(seed):
     return dict(B=B, S=before + n_vis + after, d=d, vo=before, nv=n_vis, P=P, Kp=Kp,
                 path=int(rng.choice([dart.DART_PATH_STAGED, dart.DART_PATH_FUSED, dart.DART_PATH_TWO_PASS])),
                 norm_kind=int(rng.choice([1, 2])), smallest=int(rng.integers(0, 2)),
-                retention=int(rng.integers(0, 4)), rule=int(rng.integers(0, 2)),
+                retention=int(rng.integers(0, 5)), rule=int(rng.integers(0, 2)),
                 given=bool(rng.integers(0, 2)), on_hidden=bool(rng.integers(0, 2)), keys_null=bool(rng.integers(0, 4) == 0))
 
 

@@ -177,8 +177,10 @@ def test_candidate_bands_make_the_same_selections(oracle, kind, shape):
     k, h = _band_inputs(kind, B, S, d, vo, nv, P, seed=11 + sum(shape))
     a = run_gpu(k, h, vo, nv, P, Kp, path=dart.DART_PATH_STAGED, retention=dart.DART_RETAIN_SERIAL)
     b = run_gpu(k, h, vo, nv, P, Kp, path=dart.DART_PATH_STAGED, retention=dart.DART_RETAIN_BANDS)
-    assert all(np.array_equal(x, y) for x, y in zip(a[:3], b[:3]))
-    assert all(np.array_equal(a[3][n], b[3][n], equal_nan=(n == "eps")) for n in a[3])
+    c = run_gpu(k, h, vo, nv, P, Kp, path=dart.DART_PATH_STAGED, retention=dart.DART_RETAIN_FUSED)   # both phases in one launch
+    for o in (b, c):
+        assert all(np.array_equal(x, y) for x, y in zip(a[:3], o[:3]))
+        assert all(np.array_equal(a[3][n], o[3][n], equal_nan=(n == "eps")) for n in a[3])
     kb, hb = W.bits(k), W.bits(h)
     ora = oracle.reduce(hb, kb, vo, nv, P, Kp)
     rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, b[0], b[1], b[2], dbg=b[3])

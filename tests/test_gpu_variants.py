@@ -453,7 +453,7 @@ def test_text_pivots_random_shapes(oracle, seed):
     try:
         piv_t = torch.from_numpy(piv).cuda()
         res = ctx.reduce(h, k, vo, nv, P, Kp, debug=True,
-                         opts=dart.dart_opts(retention=int(rng.integers(0, 4)), text_pivots=1, pivots_in=piv_t.data_ptr()))
+                         opts=dart.dart_opts(retention=int(rng.integers(0, 5)), text_pivots=1, pivots_in=piv_t.data_ptr()))
         torch.cuda.synchronize()
         assert ctx.status() == dart.DART_OK, dart.dart_status_detail(ctx.handle)
     finally:
