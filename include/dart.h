@@ -178,7 +178,9 @@ typedef struct {
                               split over several calls or GPUs draws what the whole batch would */
     int32_t tune;          /* 0 = defaults.  DART_PATH_PAIRED: 256 * n1 + 16 * n2 + n3 = depths of the three shared-memory rings.
                               DART_PATH_FUSED: >= 2 cuts the second pass of a row tile into eight column chunks (one task each)
-                              and keeps the first pass within `tune` steps of the second (both tuning options) */
+                              and keeps the first pass within `tune` steps of the second (low 12 bits).  One-pass kernel:
+                              bit 0x1000 = one row tile per task, bit 0x2000 = two where they fit (default: two when every
+                              CTA gets at least two tasks).  All of them tuning options: same results. */
 } dart_opts;
 
 /* Optional per-step outputs of dart_reduce_ex; every member is a device pointer or NULL. */

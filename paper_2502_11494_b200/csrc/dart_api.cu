@@ -474,7 +474,7 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     // the similarities and sim_sum_kernel adds them up; the first pass then runs at most `tune` steps ahead of the second.
     // Measured on the 256-sample workload: no gain (1.81-1.89 ms against 1.86 ms): the pivots of a sample take three to
     // four rounds of steps to appear, and holding the first pass back that closely stalls it as much as the L2 then saves.
-    p.n_kc = (ctx->sim_share && P <= kSweepChunkMaxP && o.tune >= 2) ? (p.n_atoms < kSweepChunks ? p.n_atoms : kSweepChunks) : 1;
+    p.n_kc = (ctx->sim_share && P <= kSweepChunkMaxP && (o.tune & 0xfff) >= 2) ? (p.n_atoms < kSweepChunks ? p.n_atoms : kSweepChunks) : 1;
     p.apc = (p.n_atoms + p.n_kc - 1) / p.n_kc;
     p.n_kc = (p.n_atoms + p.apc - 1) / p.apc;
     p.T1 = (n_vis + kS1Rows - 1) / kS1Rows, p.T2 = p.n_rt * p.n_kc, p.Tm = p.T1 > p.T2 ? p.T1 : p.T2;
@@ -489,7 +489,7 @@ int launch_fused(dart_ctx *ctx, int B, const void *hidden, const void *keys_in, 
     p.norm_kind = o.norm_kind, p.smallest = o.pivot_smallest;
     p.withhold_pivots = o.test_withhold_pivots;
     p.keep_l2 = p.n_kc > 1;
-    p.ahead = o.tune >= 2 ? (uint32_t)o.tune : 0u;
+    p.ahead = (o.tune & 0xfff) >= 2 ? (uint32_t)(o.tune & 0xfff) : 0u;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
     p.keys = (const char *)keys;
     p.sim = p.n_kc > 1 ? ctx->sim_share : ctx->sim, p.l1 = ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
@@ -540,14 +540,24 @@ int launch_onepass_kernel(dart_ctx *ctx, int B, const void *src, bool scores_els
     p.n_atoms = ctx->n_atoms, p.n_rt = (n_vis + kTileRows - 1) / kTileRows;
     p.split = split, p.n_sel = split.k <= 1 ? p.n_rt : split.n_streamed(p.n_rt);
     if (p.n_sel == 0) return DART_OK; // every tile stayed on the chip
-    p.aps = onepass::atoms_per_stage(p.N, ctx->max_smem_optin);
-    p.n_st = onepass::ring_depth(p.N, p.aps, ctx->max_smem_optin);
+    p.compact = ctx->piv_rows != nullptr && P > onepass::kGatherMaxP;
+    // Two row tiles per task share every pivot tile that is fetched (two accumulators per buffer: 4 N <= 512 columns of
+    // tensor memory), if that still leaves a ring of three stages and every CTA at least two tasks.  With many pivots a
+    // pivot tile is as large as a token tile and the SM's share of the L2 bandwidth bounds the kernel; with few, a task of
+    // 256 rows halves what is paid per task (measured at batch 256 x 2880 tokens: 8 pivots 1.25 -> 1.01 ms, 16: 1.14 ->
+    // 1.00, 32: 1.31 -> 1.04, 64: 1.37 -> 1.22, 128: 1.75 -> 1.61).  (tune bits 0x1000 / 0x2000 force one / two tiles.)
+    p.tg = 1;
+    const bool two_fit = split.k <= 1 && 4 * p.N <= 512 &&
+                         onepass::ring_depth(p.N, onepass::atoms_per_stage(p.N, ctx->max_smem_optin, 2), ctx->max_smem_optin, 2) >= 3;
+    if (two_fit && (long long)B * ((p.n_rt + 1) / 2) >= 2ll * ctx->sm_count && !(o.tune & 0x1000)) p.tg = 2;
+    if (two_fit && (o.tune & 0x2000)) p.tg = 2;
+    p.aps = onepass::atoms_per_stage(p.N, ctx->max_smem_optin, p.tg);
+    p.n_st = onepass::ring_depth(p.N, p.aps, ctx->max_smem_optin, p.tg);
     if (p.n_st < 2) return DART_ERR_UNSUPPORTED;
     p.wait_ns = o.wait_limit > 0 ? (unsigned long long)o.wait_limit * 1000ull : 2000000000ull;
     p.withhold = o.test_withhold_pivots;
     p.sim = ctx->sim, p.l1 = scores_elsewhere ? nullptr : ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
     p.status = ctx->status;
-    p.compact = ctx->piv_rows != nullptr && P > onepass::kGatherMaxP;
     CUtensorMap tm_tile, tm_keys, tm_row, tm_piv;
     int rc = encode_2d(ctx, &tm_tile, src, (uint64_t)ctx->desc.d, (uint64_t)B * S, kTileRows);
     if (rc == DART_OK) rc = encode_2d(ctx, &tm_keys, src, (uint64_t)ctx->desc.d, (uint64_t)B * S, kSubRows);
@@ -563,9 +573,9 @@ int launch_onepass_kernel(dart_ctx *ctx, int B, const void *src, bool scores_els
             (const uint4 *)src, ctx->pivot_idx, S, ctx->desc.d / 8, vis_offset, n_vis, P, p.N, prow, (uint4 *)ctx->piv_rows);
     }
     Prof pr(ctx, st, SLOT_ONEPASS);
-    const long long tasks = (long long)B * p.n_sel;
+    const long long tasks = (long long)B * ((p.n_sel + p.tg - 1) / p.tg);
     const unsigned grid = (unsigned)(tasks < ctx->sm_count ? tasks : ctx->sm_count); // no CTA waits for another
-    onepass::onepass_kernel<<<grid, onepass::kThreads, onepass::smem_bytes(p.N, p.aps, p.n_st), st>>>(tm_tile, tm_keys, tm_row, tm_piv, p);
+    onepass::onepass_kernel<<<grid, onepass::kThreads, onepass::smem_bytes(p.N, p.aps, p.n_st, p.tg), st>>>(tm_tile, tm_keys, tm_row, tm_piv, p);
     return DART_OK;
 }
 

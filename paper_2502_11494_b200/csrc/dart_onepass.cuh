@@ -44,6 +44,7 @@ struct Params {
     int B, S, vis_offset, n_vis, P, N; // N = P rounded up to a multiple of 16 (MMA N)
     int n_atoms, n_rt;                 // 64-column atoms per row; row tiles per sample
     int n_st, aps;                     // ring depth; atoms per stage (<= kMaxAtomsPerStage)
+    int tg;                            // row tiles per task (1 or 2): two tiles share every pivot tile that is fetched
     int compact;                       // pivot tiles come from the compact copy [B][N][d] (tm_piv), not by gather4
     int n_sel;                         // row tiles per sample this launch takes: n_rt, or the streamed tiles of `split`
     TileSplit split;                   // k <= 1: all tiles
@@ -61,25 +62,25 @@ struct Shared {
     unsigned long long mma_drain;
     uint32_t tmem_base;
     int abort_flag;
-    float row_ssq[2][kTileRows]; // per accumulator buffer: sum of squares of the tile's rows
+    float row_ssq[2][2][kTileRows]; // per accumulator buffer and tile of the task: sum of squares of the tile's rows
     float piv_ssq[2][kMaxN];     // ... and of the sample's pivot rows
 };
 static_assert(sizeof(Shared) + 64 <= kStaticSmemReserve, "static shared memory exceeds its reserve");
 
-__host__ __device__ inline uint32_t stage_bytes(int N, int aps) { return (uint32_t)aps * (kAtomBytes + b_stage_bytes(N)); }
-__host__ inline int ring_depth(int N, int aps, size_t smem_limit)
+__host__ __device__ inline uint32_t stage_bytes(int N, int aps, int tg = 1) { return (uint32_t)aps * ((uint32_t)tg * kAtomBytes + b_stage_bytes(N)); }
+__host__ inline int ring_depth(int N, int aps, size_t smem_limit, int tg = 1)
 {
-    const size_t n = (smem_limit - 1024 - kStaticSmemReserve) / stage_bytes(N, aps);
+    const size_t n = (smem_limit - 1024 - kStaticSmemReserve) / stage_bytes(N, aps, tg);
     return (int)(n > (size_t)kStages ? (size_t)kStages : n);
 }
 // As many atoms per stage as still leave three stages (with many pivots the pivot tiles crowd them out)
-__host__ inline int atoms_per_stage(int N, size_t smem_limit)
+__host__ inline int atoms_per_stage(int N, size_t smem_limit, int tg = 1)
 {
     int aps = kMaxAtomsPerStage;
-    while (aps > 1 && ring_depth(N, aps, smem_limit) < 3) aps >>= 1;
+    while (aps > 1 && ring_depth(N, aps, smem_limit, tg) < 3) aps >>= 1;
     return aps;
 }
-__host__ inline size_t smem_bytes(int N, int aps, int n_st) { return 1024 + (size_t)n_st * stage_bytes(N, aps); }
+__host__ inline size_t smem_bytes(int N, int aps, int n_st, int tg = 1) { return 1024 + (size_t)n_st * stage_bytes(N, aps, tg); }
 
 // |x| and x^2 of one 128-byte row of a 128B-swizzled tile, added to the four running sums in column order:
 // logical 16-byte chunk c of row r sits at chunk position c ^ (r & 7)
@@ -109,10 +110,12 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
     __shared__ Shared sh;
     const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bstage = b_stage_bytes(p.N);
-    // stage s: p.aps token tiles, then as many pivot tiles
-    auto a_addr = [&](int s, int h) { return smem0 + (uint32_t)s * stage_bytes(p.N, p.aps) + (uint32_t)h * kAtomBytes; };
+    // stage s: p.aps x p.tg token tiles (atom-major), then p.aps pivot tiles
+    auto a_addr = [&](int s, int h, int w = 0) {
+        return smem0 + (uint32_t)s * stage_bytes(p.N, p.aps, p.tg) + (uint32_t)(h * p.tg + w) * kAtomBytes;
+    };
     auto b_addr = [&](int s, int h) {
-        return smem0 + (uint32_t)s * stage_bytes(p.N, p.aps) + (uint32_t)p.aps * kAtomBytes + (uint32_t)h * bstage;
+        return smem0 + (uint32_t)s * stage_bytes(p.N, p.aps, p.tg) + (uint32_t)(p.aps * p.tg) * kAtomBytes + (uint32_t)h * bstage;
     };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned long long limit = 2ull * p.wait_ns; // ns -> cycles at the highest SM clock: never shorter than asked
@@ -135,7 +138,7 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     uint32_t tmem_cols = 32;
-    while (tmem_cols < 2u * p.N) tmem_cols <<= 1;
+    while (tmem_cols < 2u * (uint32_t)p.tg * p.N) tmem_cols <<= 1;
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)),
                      "r"(tmem_cols)
@@ -146,13 +149,15 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = sh.tmem_base;
-    const uint32_t total = (uint32_t)p.B * (uint32_t)p.n_sel; // tasks: (sample, row tile), sample-major
-    // task g -> (sample, row tile); with a split only the tiles that did not stay on the chip are taken
+    const uint32_t per_sample = (uint32_t)(p.n_sel + p.tg - 1) / (uint32_t)p.tg;
+    const uint32_t total = (uint32_t)p.B * per_sample; // tasks: (sample, first row tile), sample-major
+    // task g -> (sample, row tile); with a split only the tiles that did not stay on the chip are taken (one tile per task then)
     auto task = [&](uint32_t g, int &b, int &rt) {
-        b = (int)(g / (uint32_t)p.n_sel);
-        const int i = (int)(g - (uint32_t)b * (uint32_t)p.n_sel);
+        b = (int)(g / per_sample);
+        const int i = (int)(g - (uint32_t)b * per_sample) * p.tg;
         rt = p.split.k <= 1 ? i : p.split.streamed(i);
     };
+    auto tile_rows = [&](int rt, int w) { return max(0, min(kTileRows, p.n_vis - (rt + w) * kTileRows)); }; // 0: no such tile
     const int na = p.n_atoms;
 
     if (warp == 0) {
@@ -178,27 +183,32 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
                     }
                 cur_b = b;
             }
-            const int rows = min(kTileRows, p.n_vis - rt * kTileRows);
-            const int n_sub = (rows + kSubRows - 1) / kSubRows;
             const int y0 = b * p.S + p.vis_offset + rt * kTileRows;
+            uint32_t tile_tx = 0; // bytes of one atom of the task's tiles
+            for (int w = 0; w < p.tg; ++w) {
+                const int rows = tile_rows(rt, w);
+                tile_tx += rows == kTileRows ? (uint32_t)kAtomBytes : (uint32_t)((rows + kSubRows - 1) / kSubRows) * kSubBytes;
+            }
             for (int a = 0; a < na; a += p.aps) {
                 const int nh = min(p.aps, na - a); // atoms in this stage
                 const uint32_t full = smem_u32(&sh.full[ring.stage]);
                 if (lane == 0) {
                     ok = ctl.wait_bar(smem_u32(&sh.empty[ring.stage]), ring.phase ^ 1u, kWaitStageFree, g);
                     if (ok)
-                        mbar_arrive_expect_tx(full, (uint32_t)nh * ((rows == kTileRows ? (uint32_t)kAtomBytes : (uint32_t)n_sub * kSubBytes) +
-                                                                    (p.compact ? (uint32_t)p.N * 128u : (uint32_t)((p.P + 3) / 4) * 512u)));
+                        mbar_arrive_expect_tx(full, (uint32_t)nh * (tile_tx + (p.compact ? (uint32_t)p.N * 128u : (uint32_t)((p.P + 3) / 4) * 512u)));
                 }
                 ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
                 if (!ok) break;
                 for (int h = 0; h < nh; ++h) {
                     const int x = (a + h) * kAtomCols;
-                    const uint32_t dst = a_addr(ring.stage, h);
-                    if (rows == kTileRows) {
-                        if (lane == h) tma_load_2d(dst, &tm_tile, x, y0, full, pol_drop); // one lane per atom: issued side by side
-                    } else if (lane < n_sub) {
-                        tma_load_2d(dst + (uint32_t)lane * kSubBytes, &tm_keys, x, y0 + lane * kSubRows, full, pol_drop);
+                    for (int w = 0; w < p.tg; ++w) {
+                        const int rows = tile_rows(rt, w), n_sub = (rows + kSubRows - 1) / kSubRows;
+                        const uint32_t dst = a_addr(ring.stage, h, w);
+                        if (rows == kTileRows) {
+                            if (lane == h + kMaxAtomsPerStage * 2 * w) tma_load_2d(dst, &tm_tile, x, y0 + w * kTileRows, full, pol_drop); // one lane per tile: issued side by side
+                        } else if (lane < n_sub) {
+                            tma_load_2d(dst + (uint32_t)lane * kSubBytes, &tm_keys, x, y0 + w * kTileRows + lane * kSubRows, full, pol_drop);
+                        }
                     }
                     if (p.compact) { // rows b N .. b N + N - 1 of the compact copy: the sample's pivots in rank order, zero padded
                         if (lane == kMaxAtomsPerStage + h) tma_load_2d(b_addr(ring.stage, h), &tm_piv, x, b * p.N, full, pol_keep);
@@ -231,17 +241,23 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
                 ok = ctl.wait_bar(smem_u32(&sh.tmem_empty[acc]), ((n >> 1) & 1u) ^ 1u, kWaitAccumFree1, g);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t d_tmem = tmem_base + acc * (uint32_t)p.N;
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)(p.tg * p.N);
+                int rt_b, rt_t;
+                task(g, rt_b, rt_t);
+                const int nt = p.tg > 1 && tile_rows(rt_t, 1) > 0 ? 2 : 1; // tiles of this task
                 for (int a = 0; a < na; a += p.aps) {
                     ok = ctl.wait_bar(smem_u32(&sh.full[ring.stage]), ring.phase, kWaitStageMma, g);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     for (int h = 0; h < min(p.aps, na - a); ++h) {
-                        const unsigned long long da = umma_desc(a_addr(ring.stage, h)), db = umma_desc(b_addr(ring.stage, h));
+                        const unsigned long long db = umma_desc(b_addr(ring.stage, h));
+                        for (int w = 0; w < nt; ++w) { // the task's tiles share the pivot tile
+                            const unsigned long long da = umma_desc(a_addr(ring.stage, h, w));
 #pragma unroll
-                        for (int k = 0; k < kAtomCols / 16; ++k) // 16 columns = 32 bytes per MMA: advance the start address
-                            umma_bf16(d_tmem, da + (unsigned long long)(2 * k), db + (unsigned long long)(2 * k), idesc,
-                                      (a | h | k) != 0);
+                            for (int k = 0; k < kAtomCols / 16; ++k) // 16 columns = 32 bytes per MMA: advance the start address
+                                umma_bf16(d_tmem + (uint32_t)(w * p.N), da + (unsigned long long)(2 * k), db + (unsigned long long)(2 * k),
+                                          idesc, (a | h | k) != 0);
+                        }
                     }
                     umma_commit(smem_u32(&sh.empty[ring.stage])); // the tensor cores' share of releasing the stage
                     ring.advance();
@@ -264,14 +280,17 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
         for (uint32_t g = blockIdx.x; !dead && g < total; g += gridDim.x) {
             int b, rt;
             task(g, b, rt);
-            const int rows = min(kTileRows, p.n_vis - rt * kTileRows);
-            float a0 = 0.f, a1 = 0.f, q0 = 0.f, q1 = 0.f; // own tile row
+            const int rows = tile_rows(rt, 0), rows2 = p.tg > 1 ? tile_rows(rt, 1) : 0;
+            float a0 = 0.f, a1 = 0.f, q0 = 0.f, q1 = 0.f; // own row of the task's first tile
+            float c0 = 0.f, c1 = 0.f, r0 = 0.f, r1 = 0.f; // ... and of its second tile
             for (int a = 0; a < na; a += p.aps) {
                 dead = !ctl.wait_bar(smem_u32(&sh.full[ring.stage]), ring.phase, kWaitStageNorm, g);
                 dead = __any_sync(0xffffffffu, dead);
                 if (dead) break;
-                for (int h = 0; h < min(p.aps, na - a); ++h) // atoms in column order: the sums do not depend on the staging
+                for (int h = 0; h < min(p.aps, na - a); ++h) { // atoms in column order: the sums do not depend on the staging
                     if (t < rows) add_row(a_addr(ring.stage, h), t, a0, a1, q0, q1);
+                    if (t < rows2) add_row(a_addr(ring.stage, h, 1), t, c0, c1, r0, r1);
+                }
                 __syncwarp(); // the warp's reads of the stage are done
                 if (lane == 0) mbar_arrive(smem_u32(&sh.empty[ring.stage]));
                 ring.advance();
@@ -282,12 +301,18 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
             dead = !ctl.wait_bar(smem_u32(&sh.norm_empty[acc]), ((n >> 1) & 1u) ^ 1u, kWaitNormFree, g);
             dead = __any_sync(0xffffffffu, dead);
             if (dead) break;
-            const float q = q0 + q1;
-            sh.row_ssq[acc][t] = t < rows ? q : 0.f;
+            const float q = q0 + q1, r = r0 + r1;
+            sh.row_ssq[acc][0][t] = t < rows ? q : 0.f;
+            sh.row_ssq[acc][1][t] = t < rows2 ? r : 0.f;
             if (t < rows) {
                 const size_t o = (size_t)b * p.n_vis + rt * kTileRows + t;
                 if (p.l1) p.l1[o] = a0 + a1;
                 p.ssq[o] = q;
+            }
+            if (t < rows2) {
+                const size_t o = (size_t)b * p.n_vis + (rt + 1) * kTileRows + t;
+                if (p.l1) p.l1[o] = c0 + c1;
+                p.ssq[o] = r;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh.norm_full[acc])); // release: the warp's norms are ordered before it
@@ -338,26 +363,29 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
         for (uint32_t g = blockIdx.x; g < total; g += gridDim.x) {
             int b, rt;
             task(g, b, rt);
-            const int rows = min(kTileRows, p.n_vis - rt * kTileRows);
-            const int j = rt * kTileRows + row;
             const uint32_t acc = n & 1u;
             bool ok = ctl.wait_bar(smem_u32(&sh.norm_full[acc]), (n >> 1) & 1u, kWaitNormFull, g);
             if (ok) ok = ctl.wait_bar(smem_u32(&sh.tmem_full[acc]), (n >> 1) & 1u, kWaitAccumFull1, g);
             if (!__all_sync(0xffffffffu, ok)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const float nj = sqrtf(sh.row_ssq[acc][row]);
-            const uint32_t taddr = tmem_base + acc * (uint32_t)p.N + ((uint32_t)(quarter * 32) << 16);
-            float *dst = p.sim + (size_t)b * p.P * p.n_vis + j;
-            for (int c0 = 0; c0 < p.P; c0 += 8) {
-                float v[8];
-                tmem_ld8(taddr + (uint32_t)c0, v); // warp-collective: rows outside the tile still take part
-                if (row < rows) {
+            for (int w = 0; w < p.tg; ++w) { // the task's tiles, one accumulator each
+                const int rows = tile_rows(rt, w);
+                if (rows == 0) break;
+                const int j = (rt + w) * kTileRows + row;
+                const float nj = sqrtf(sh.row_ssq[acc][w][row]);
+                const uint32_t taddr = tmem_base + acc * (uint32_t)(p.tg * p.N) + (uint32_t)(w * p.N) + ((uint32_t)(quarter * 32) << 16);
+                float *dst = p.sim + (size_t)b * p.P * p.n_vis + j;
+                for (int c0 = 0; c0 < p.P; c0 += 8) {
+                    float v[8];
+                    tmem_ld8(taddr + (uint32_t)c0, v); // warp-collective: rows outside the tile still take part
+                    if (row < rows) {
 #pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        if (c0 + e < p.P) { // dup = dot / (|pivot| |row|); a zero norm gives 0; a warp writes 128 contiguous bytes
-                            const float den = sqrtf(sh.piv_ssq[acc][c0 + e]) * nj;
-                            dst[(size_t)(c0 + e) * p.n_vis] = den > 0.f ? v[e] / den : 0.f;
-                        }
+                        for (int e = 0; e < 8; ++e)
+                            if (c0 + e < p.P) { // dup = dot / (|pivot| |row|); a zero norm gives 0; a warp writes 128 contiguous bytes
+                                const float den = sqrtf(sh.piv_ssq[acc][c0 + e]) * nj;
+                                dst[(size_t)(c0 + e) * p.n_vis] = den > 0.f ? v[e] / den : 0.f;
+                            }
+                    }
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");

@@ -187,6 +187,44 @@ def test_candidate_bands_make_the_same_selections(oracle, kind, shape):
     assert rep.exact >= rep.above_margin
 
 
+# (B, S, d, vis_offset, n_vis, P, Kp): one, two and three row tiles, ragged and whole last tiles, few and many pivots
+TWO_TILE_SHAPES = [
+    (2, 140, 64, 5, 100, 3, 30),        # less than one tile
+    (3, 300, 128, 10, 256, 8, 64),      # exactly two tiles: one task
+    (2, 330, 64, 0, 300, 9, 50),        # two whole tiles and a ragged third: the last task has one tile
+    (2, 700, 256, 40, 640, 16, 100),    # five whole tiles: the last task has one tile
+    (1, 1500, 64, 7, 1410, 128, 600),   # pivot tiles as large as the row tiles, a ragged last tile that is a task's second
+    (2, 3000, 4096, 40, 2880, 8, 320),  # the benchmark's shape
+]
+
+
+@pytest.mark.parametrize("tiles", [1, 2], ids=["one tile per task", "two tiles per task"])
+@pytest.mark.parametrize("shape", TWO_TILE_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_one_pass_kernel_with_one_and_two_row_tiles_per_task(oracle, shape, tiles):
+    """The one-pass kernel takes one 128-row tile per task or two that share every pivot tile (two accumulators):
+    both against the oracle, with pivots by score (score pass first) and with the caller's pivots."""
+    B, S, d, vo, nv, P, Kp = shape
+    k, h = gaussian(B, S, d, seed=21 + sum(shape))
+    kb, hb = W.bits(k), W.bits(h)
+    tune = 0x1000 if tiles == 1 else 0x2000
+    g = torch.Generator(device="cuda").manual_seed(5)
+    piv = torch.stack([torch.randperm(nv, generator=g, device="cuda")[:P] for _ in range(B)]).to(torch.int32).contiguous()
+    for given in (False, True):
+        ctx = dart.Dart(B, S, d, P, Kp)
+        try:
+            opts = dart.dart_opts(path=dart.DART_PATH_TWO_PASS, tune=tune, pivots_in=piv.data_ptr() if given else 0)
+            res = ctx.reduce(h, k, vo, nv, P, Kp, opts=opts, debug=True)
+            torch.cuda.synchronize()
+            assert ctx.status() == dart.DART_OK, dart.dart_status_detail(ctx.handle)
+        finally:
+            ctx.close()
+        dbg = {n: _np(v) for n, v in res[3].items()}
+        ora = oracle.reduce(hb, kb, vo, nv, P, Kp, pivots_in=piv.cpu().numpy() if given else None)
+        rep = parity.check_batch(ora, kb, hb, vo, nv, P, Kp, _np(res[0]), _np(res[1]), _np(res[2]), dbg=dbg, pivots_given=given)
+        assert rep.exact >= rep.above_margin
+        assert rep.max_rel_l2 < 5e-5 and rep.max_abs_sim < 2e-5
+
+
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS.get)
 def test_keys_null_scores_the_hidden_states(oracle, path):
     _, h = gaussian(2, 120, 256, seed=7)
