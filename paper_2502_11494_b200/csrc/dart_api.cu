@@ -898,7 +898,7 @@ int dart_create(dart_ctx **out, const dart_desc *desc)
         }
     }
     if (rc == DART_OK && desc->P_max > dart::onepass::kGatherMaxP) {
-        // compact pivot rows for the one-pass kernel at many pivots; contexts that would need more than 2 GiB go without
+        // compact pivot rows for the one-pass kernel; contexts that would need more than 2 GiB go without (gather4 then)
         const size_t bytes = (size_t)desc->B_max * ((desc->P_max + 15) / 16 * 16) * desc->d * 2;
         if (bytes <= ((size_t)2 << 30)) rc = ws_alloc(ctx, (uint8_t **)&ctx->piv_rows, bytes);
     }

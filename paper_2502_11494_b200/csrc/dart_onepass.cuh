@@ -10,9 +10,9 @@
 // dealt out round-robin to a persistent grid of one CTA per SM.
 //
 // Per CTA (384 threads):
-//   warp 0     producer: per 64-column atom one 128-row TMA tile (128-byte swizzle) and the pivot rows - by
-//              tile::gather4 straight from the key tensor (4 rows per op: fine for a few pivots), or as ONE box from
-//              a compact copy of the sample's pivot rows (many pivots: gather4 ops would bound the kernel) -
+//   warp 0     producer: per 64-column atom one or two 128-row TMA tiles (128-byte swizzle) and the pivot rows - as
+//              ONE box from a compact copy of the sample's pivot rows, or, where the context has no room for that
+//              copy, by tile::gather4 straight from the key tensor (4 rows per op, ~13 ops per us: slower) -
 //              up to four atoms per stage of a ring
 //   warp 1     one thread issues tcgen05.mma; tcgen05.commit releases the stage on the tensor cores' behalf
 //   warps 4-7  norms: thread t owns tile row t and sums its 128 bytes of every atom, in column order whatever
@@ -36,7 +36,9 @@ constexpr int kEpi0 = 8;          // kEpi0 % 4 == 0: warp w reads TMEM lanes 32 
 constexpr int kStages = 10;       // at most
 constexpr int kMaxAtomsPerStage = 4; // a stage holds up to four 64-column atoms: the producer's issue latency (wait, expect,
                                      // issue: ~0.3 us) is paid per stage; measured at 8 pivots: 1 atom 1.40 ms, 2 1.14, 4 1.02
-constexpr int kGatherMaxP = 8;    // up to this many pivots the pivot rows come by gather4 (two ops per atom)
+constexpr int kGatherMaxP = 0;    // up to this many pivots the pivot rows come by gather4 even when the compact copy exists: none
+                                  // (gather4 ops issue at ~13 per us and SM: at 8 pivots 128 of them per row tile cost more than
+                                  // the copy; measured per launch, 256 x 2880 tokens, 8 pivots: 1.01 -> 0.95 ms)
 constexpr int kStaticSmemReserve = 8192;
 enum { kWaitStageFree = 64, kWaitStageMma, kWaitStageNorm, kWaitAccumFree1, kWaitAccumFull1, kWaitNormFree, kWaitNormFull };
 
