@@ -92,7 +92,7 @@ def kernel_bytes_per_launch(name, w, B):
 # on the sweep workload at batch 32; traffic is proportional to the batch (every sample is read and written
 # independently), so a launch over B samples moves B times this.
 NCU_TRAFFIC_PER_SAMPLE = {("sweep", 2880, 4096, 8): (1.508338e9 + 8.540928e6) / 32,
-                          ("onepass", 2880, 4096, 8): (755.095552e6 + 5.012736e6) / 32,
+                          ("onepass", 2880, 4096, 8): (759.286272e6 + 5.440000e6) / 32,
                           ("resident", 2880, 4096, 8): (755.073536e6 + 6.136064e6) / 32}
 
 
