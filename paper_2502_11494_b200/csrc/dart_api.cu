@@ -542,14 +542,20 @@ int launch_onepass_kernel(dart_ctx *ctx, int B, const void *src, bool scores_els
     if (p.n_sel == 0) return DART_OK; // every tile stayed on the chip
     p.compact = ctx->piv_rows != nullptr && P > onepass::kGatherMaxP;
     // Two row tiles per task share every pivot tile that is fetched (two accumulators per buffer: 4 N <= 512 columns of
-    // tensor memory), if that still leaves a ring of three stages and every CTA at least two tasks.  With many pivots a
+    // tensor memory), if that still leaves a ring of three stages and shortens the longest queue of tasks.  With many pivots a
     // pivot tile is as large as a token tile and the SM's share of the L2 bandwidth bounds the kernel; with few, a task of
     // 256 rows halves what is paid per task (measured at batch 256 x 2880 tokens: 8 pivots 1.25 -> 1.01 ms, 16: 1.14 ->
     // 1.00, 32: 1.31 -> 1.04, 64: 1.37 -> 1.22, 128: 1.75 -> 1.61).  (tune bits 0x1000 / 0x2000 force one / two tiles.)
     p.tg = 1;
     const bool two_fit = split.k <= 1 && 4 * p.N <= 512 &&
                          onepass::ring_depth(p.N, onepass::atoms_per_stage(p.N, ctx->max_smem_optin, 2), ctx->max_smem_optin, 2) >= 3;
-    if (two_fit && (long long)B * ((p.n_rt + 1) / 2) >= 2ll * ctx->sm_count && !(o.tune & 0x1000)) p.tg = 2;
+    // the longest queue of any CTA, in tiles plus 0.4 of a tile per task (the fit above): 8 x 23 tiles on 148 SMs are
+    // 2 x 1.4 as single tiles and 1 x 2.4 as pairs (measured 65 and 53 us), 16 x 23 are 3 x 1.4 and 2 x 2.4 (94 and 102 us)
+    auto queue_cost = [&](int tg) {
+        const long long tasks = (long long)B * ((p.n_rt + tg - 1) / tg);
+        return (double)((tasks + ctx->sm_count - 1) / ctx->sm_count) * (tg + 0.4);
+    };
+    if (two_fit && queue_cost(2) < queue_cost(1) && !(o.tune & 0x1000)) p.tg = 2;
     if (two_fit && (o.tune & 0x2000)) p.tg = 2;
     p.aps = onepass::atoms_per_stage(p.N, ctx->max_smem_optin, p.tg);
     p.n_st = onepass::ring_depth(p.N, p.aps, ctx->max_smem_optin, p.tg);
@@ -816,10 +822,15 @@ int launch_reduce(dart_ctx *ctx, int B, const void *hidden, const void *keys, co
     // than the sweep's shared-memory score buffer holds: it then selects from global memory and stalls (measured at
     // 4608 tokens, batch 4: 253 us against 111 us).  (2) 32 pivots or more: the sweep fetches pivot tiles four rows per
     // TMA op, the one-pass kernel as one box from a compact copy (batch 256: 32 pivots 2.83 -> 2.71 ms, 128 pivots
-    // 6.15 -> 4.65 ms; at 16 pivots the sweep is still ahead, 2.33 against 2.40 ms).
+    // 6.15 -> 4.65 ms; below that the two are within 1 % of each other at batch 256).  (3) Between half a 128-row tile
+    // and two tiles per SM: the persistent sweep has nothing to overlap a sample's pivot dependency with (measured, us per
+    // step: 8 samples of 2880 tokens 178 -> 165, 12 samples 218 -> 201, 16 samples of 576 tokens 115 -> 104; with fewer
+    // tiles still, the two extra launches cost more: 8 samples of 576 tokens 84 -> 95).
+    const long long row_tiles = (long long)B * ((n_vis + dart::sweep::kTileRows - 1) / dart::sweep::kTileRows);
     const bool two_pass = o.path == DART_PATH_TWO_PASS ||
                           (o.path == DART_PATH_AUTO && fused_applies(ctx, P) && !o.pivots_in &&
-                           (n_vis > dart::sweep::kSelMax || (P >= 32 && ctx->piv_rows)));
+                           (n_vis > dart::sweep::kSelMax || (P >= 32 && ctx->piv_rows) ||
+                            (2 * row_tiles >= ctx->sm_count && row_tiles < 2ll * ctx->sm_count)));
     if (two_pass) {
         if (!fused_applies(ctx, P)) return DART_ERR_UNSUPPORTED;
         const void *k = keys ? keys : hidden;
