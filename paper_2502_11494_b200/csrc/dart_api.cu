@@ -564,8 +564,9 @@ int launch_onepass_kernel(dart_ctx *ctx, int B, const void *src, bool scores_els
     p.withhold = o.test_withhold_pivots;
     p.sim = ctx->sim, p.l1 = scores_elsewhere ? nullptr : ctx->l1, p.ssq = ctx->ssq, p.pivot_idx = ctx->pivot_idx;
     p.status = ctx->status;
-    CUtensorMap tm_tile, tm_keys, tm_row, tm_piv;
+    CUtensorMap tm_tile, tm_keys, tm_row, tm_piv, tm_pair;
     int rc = encode_2d(ctx, &tm_tile, src, (uint64_t)ctx->desc.d, (uint64_t)B * S, kTileRows);
+    if (rc == DART_OK) rc = encode_2d(ctx, &tm_pair, src, (uint64_t)ctx->desc.d, (uint64_t)B * S, 2 * kTileRows);
     if (rc == DART_OK) rc = encode_2d(ctx, &tm_keys, src, (uint64_t)ctx->desc.d, (uint64_t)B * S, kSubRows);
     if (rc == DART_OK) rc = encode_2d(ctx, &tm_row, src, (uint64_t)ctx->desc.d, (uint64_t)B * S, 1);
     if (rc == DART_OK)
@@ -581,7 +582,7 @@ int launch_onepass_kernel(dart_ctx *ctx, int B, const void *src, bool scores_els
     Prof pr(ctx, st, SLOT_ONEPASS);
     const long long tasks = (long long)B * ((p.n_sel + p.tg - 1) / p.tg);
     const unsigned grid = (unsigned)(tasks < ctx->sm_count ? tasks : ctx->sm_count); // no CTA waits for another
-    onepass::onepass_kernel<<<grid, onepass::kThreads, onepass::smem_bytes(p.N, p.aps, p.n_st, p.tg), st>>>(tm_tile, tm_keys, tm_row, tm_piv, p);
+    onepass::onepass_kernel<<<grid, onepass::kThreads, onepass::smem_bytes(p.N, p.aps, p.n_st, p.tg), st>>>(tm_tile, tm_keys, tm_row, tm_piv, tm_pair, p);
     return DART_OK;
 }
 

@@ -106,7 +106,8 @@ __device__ __forceinline__ void add_row(uint32_t tile, int r, float &a0, float &
 
 __global__ void __launch_bounds__(kThreads, 1)
 onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constant__ CUtensorMap tm_keys,
-               const __grid_constant__ CUtensorMap tm_row, const __grid_constant__ CUtensorMap tm_piv, const Params p)
+               const __grid_constant__ CUtensorMap tm_row, const __grid_constant__ CUtensorMap tm_piv,
+               const __grid_constant__ CUtensorMap tm_pair, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ Shared sh;
@@ -186,6 +187,7 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
                 cur_b = b;
             }
             const int y0 = b * p.S + p.vis_offset + rt * kTileRows;
+            const bool pair_box = p.tg == 2 && tile_rows(rt, 0) == kTileRows && tile_rows(rt, 1) == kTileRows;
             uint32_t tile_tx = 0; // bytes of one atom of the task's tiles
             for (int w = 0; w < p.tg; ++w) {
                 const int rows = tile_rows(rt, w);
@@ -203,6 +205,9 @@ onepass_kernel(const __grid_constant__ CUtensorMap tm_tile, const __grid_constan
                 if (!ok) break;
                 for (int h = 0; h < nh; ++h) {
                     const int x = (a + h) * kAtomCols;
+                    if (pair_box) { // two whole tiles, one below the other in the tensor and in the stage: one box of 256 rows
+                        if (lane == h) tma_load_2d(a_addr(ring.stage, h, 0), &tm_pair, x, y0, full, pol_drop);
+                    } else
                     for (int w = 0; w < p.tg; ++w) {
                         const int rows = tile_rows(rt, w), n_sub = (rows + kSubRows - 1) / kSubRows;
                         const uint32_t dst = a_addr(ring.stage, h, w);
