@@ -49,6 +49,23 @@ def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(dart.dart_debug) == 7 * ctypes.sizeof(ctypes.c_void_p)
 
 
+def test_binding_constants_equal_the_header_defines():
+    """Every numeric DART_* #define of the header that the binding names has the same value there."""
+    from paper_2502_11494_b200 import dart
+
+    text = open(os.path.join(ROOT, "include", "dart.h")).read()
+    defines = {m.group(1): int(m.group(2), 0) for m in re.finditer(r"^#define\s+(DART_[A-Z_0-9]+)\s+\(?(-?(?:0x[0-9a-fA-F]+|\d+))\)?", text, flags=re.M)}
+    assert len(defines) >= 20
+    checked = 0
+    for name, value in defines.items():
+        if hasattr(dart, name):
+            assert getattr(dart, name) == value, name
+            checked += 1
+    for name in ("DART_RETAIN_BANDS", "DART_RETAIN_FUSED", "DART_PATH_PAIRED", "DART_PATH_SPLIT", "DART_PIVOTS_RANDOM", "DART_RULE_UNION"):
+        assert name in defines and hasattr(dart, name), name
+    assert checked >= 18
+
+
 def test_null_arguments_are_rejected_without_a_device(built):
     from paper_2502_11494_b200 import dart
 
